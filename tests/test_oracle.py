@@ -1,0 +1,379 @@
+"""Pins for the CPU oracle: each function is tied to something other than
+itself -- closed forms, the paper's identities (Eq. 1, Eq. 2, Eq. 3), textbook
+theorems (Eckart-Young) and brute force on tiny inputs."""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+
+from oracle import ffsplit_oracle as orc
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+ACTS = [orc.ACT_GELU_ERF, orc.ACT_GELU_TANH, orc.ACT_SWIGLU]
+
+
+def _tiny(rng, s=5, d=4, m=7, act=orc.ACT_GELU_ERF, bias=True):
+    X = rng.normal(size=(s, d))
+    W1 = rng.normal(size=(d, m)) * 0.7
+    W1u = rng.normal(size=(d, m)) * 0.7 if act == orc.ACT_SWIGLU else None
+    W2 = rng.normal(size=(m, d + 1))          # non-square output on purpose
+    b1 = rng.normal(size=m) if (bias and act != orc.ACT_SWIGLU) else None
+    b2 = rng.normal(size=d + 1) if bias else None
+    return X, W1, W1u, b1, W2, b2
+
+
+# ---------------------------------------------------------------- activations
+def test_activation_golden_values():
+    fn = {"gelu_erf": orc.gelu_erf, "silu": orc.silu}
+    n = 0
+    for line in open(os.path.join(GOLDEN, "activation_values.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        name, x, v = line.split()
+        assert abs(float(fn[name](np.array([float(x)]))[0]) - float(v)) < 1e-14
+        n += 1
+    assert n == 7
+
+
+def test_gelu_erf_is_x_times_normal_cdf():
+    for x in np.linspace(-6, 6, 49):
+        phi = 0.5 * math.erfc(-x / math.sqrt(2.0))
+        assert abs(orc.gelu_erf(np.array([x]))[0] - x * phi) < 1e-14
+
+
+def test_activation_symmetries():
+    x = np.linspace(-5, 5, 101)
+    # x*Phi(x) - (-x)*Phi(-x) = x
+    assert np.allclose(orc.gelu_erf(x) - orc.gelu_erf(-x), x, atol=1e-14)
+    assert np.allclose(orc.gelu_tanh(x) - orc.gelu_tanh(-x), x, atol=1e-14)
+    # SiLU(x) + SiLU(-x) = x tanh(x/2)
+    assert np.allclose(orc.silu(x) + orc.silu(-x), x * np.tanh(x / 2), atol=1e-14)
+    # tanh form tracks the erf form to < 1e-3 everywhere, and is not identical
+    gap = np.max(np.abs(orc.gelu_tanh(x) - orc.gelu_erf(x)))
+    assert 1e-5 < gap < 1e-3
+    # value of the tanh form at 1 written out term by term
+    inner = math.sqrt(2 / math.pi) * (1 + 0.044715)
+    assert abs(orc.gelu_tanh(np.array([1.0]))[0] - 0.5 * (1 + math.tanh(inner))) < 1e-15
+
+
+# ---------------------------------------------------------------- dense FFN
+def test_dense_ffn_hand_worked_example():
+    # one token x = (1, 0): z = first row of W1 = (0, 1, -1); GELU = (0, Phi(1), -Phi(-1))
+    X = np.array([[1.0, 0.0]])
+    W1 = np.array([[0.0, 1.0, -1.0], [5.0, 6.0, 7.0]])
+    W2 = np.array([[9.0, 9.0], [1.0, 2.0], [3.0, 4.0]])
+    p1, pm1 = 0.8413447460685429, 0.15865525393145707
+    want = np.array([[p1 * 1 - pm1 * 3, p1 * 2 - pm1 * 4]])
+    got = orc.dense_ffn(X, W1, None, W2, None, orc.ACT_GELU_ERF)
+    assert np.allclose(got, want, atol=1e-14)
+    # bias shifts: b1 = (1, 0, 0) makes z_0 = 1; b2 adds (10, 20)
+    got = orc.dense_ffn(X, W1, np.array([1.0, 0, 0]), W2, np.array([10.0, 20.0]), orc.ACT_GELU_ERF)
+    assert np.allclose(got, want + p1 * 9 + np.array([[10.0, 20.0]]), atol=1e-13)
+
+
+@pytest.mark.parametrize("act", ACTS)
+def test_dense_ffn_equals_rank_one_sum(rng, act):
+    """Eq. 1: FFN(X) = sum_j sigma(X U_{:,j}) V_{j,:}, written with scalar loops."""
+    X, W1, W1u, b1, W2, b2 = _tiny(rng, act=act)
+    s, d = X.shape
+    m, dout = W2.shape
+    Y = np.zeros((s, dout))
+    for j in range(m):
+        col = np.zeros(s)
+        for t in range(s):
+            z = sum(X[t, i] * W1[i, j] for i in range(d))
+            if act == orc.ACT_SWIGLU:
+                u = sum(X[t, i] * W1u[i, j] for i in range(d))
+                col[t] = z / (1 + math.exp(-z)) * u
+            else:
+                z += b1[j]
+                if act == orc.ACT_GELU_ERF:
+                    col[t] = z * 0.5 * math.erfc(-z / math.sqrt(2))
+                else:
+                    col[t] = 0.5 * z * (1 + math.tanh(math.sqrt(2 / math.pi) * (z + 0.044715 * z ** 3)))
+        Y += np.outer(col, W2[j, :])
+    Y += b2[None, :]
+    assert np.allclose(orc.dense_ffn(X, W1, b1, W2, b2, act, W1u), Y, rtol=1e-12, atol=1e-12)
+
+
+# ---------------------------------------------------------------- score
+@pytest.mark.parametrize("act", ACTS)
+def test_score_is_the_removal_residual(rng, act):
+    """Eq. 3: ||FFN(X) - FFN_{without j}(X)||_F^2 = ||sigma(X U_j)||^2 ||V_j||^2."""
+    X, W1, W1u, b1, W2, b2 = _tiny(rng, s=9, act=act)
+    e, w, sc = orc.neuron_scores(X, W1, b1, W2, act, orc.SCORE_EQ3, W1u)
+    full = orc.dense_ffn(X, W1, b1, W2, b2, act, W1u)
+    for j in range(W1.shape[1]):
+        W1r = np.delete(W1, j, axis=1)
+        W1ur = None if W1u is None else np.delete(W1u, j, axis=1)
+        b1r = None if b1 is None else np.delete(b1, j)
+        W2r = np.delete(W2, j, axis=0)
+        less = orc.dense_ffn(X, W1r, b1r, W2r, b2, act, W1ur)
+        resid = np.sum((full - less) ** 2)
+        assert abs(resid - sc[j]) <= 1e-10 * max(resid, 1e-30)
+    assert np.allclose(e * w, sc)
+
+
+def test_score_modes_by_explicit_contributions(rng):
+    X, W1, W1u, b1, W2, b2 = _tiny(rng, s=6)
+    H = orc.neuron_activations(X, W1, b1, orc.ACT_GELU_ERF)
+    _, _, s_act = orc.neuron_scores(X, W1, b1, W2, orc.ACT_GELU_ERF, orc.SCORE_ACT_ONLY)
+    _, _, s_sum = orc.neuron_scores(X, W1, b1, W2, orc.ACT_GELU_ERF, orc.SCORE_SUM_NORM)
+    for j in range(W1.shape[1]):
+        contrib = np.outer(H[:, j], W2[j, :])                  # s x d_out
+        assert abs(s_act[j] - np.linalg.norm(H[:, j]) ** 2) < 1e-12
+        assert abs(s_sum[j] - sum(np.linalg.norm(contrib[t]) for t in range(X.shape[0]))) < 1e-12
+    # ranking by Eq. 3 is unchanged by a square root; the unsquared sum may differ
+    _, _, s3 = orc.neuron_scores(X, W1, b1, W2, orc.ACT_GELU_ERF, orc.SCORE_EQ3)
+    assert np.array_equal(orc.select_heavy(s3, 3)[0], orc.select_heavy(np.sqrt(s3), 3)[0])
+
+
+def test_score_is_additive_over_token_batches(rng):
+    X, W1, W1u, b1, W2, b2 = _tiny(rng, s=10)
+    e, w, _ = orc.neuron_scores(X, W1, b1, W2, orc.ACT_GELU_ERF)
+    e1, _, _ = orc.neuron_scores(X[:4], W1, b1, W2, orc.ACT_GELU_ERF)
+    e2, _, _ = orc.neuron_scores(X[4:], W1, b1, W2, orc.ACT_GELU_ERF)
+    assert np.allclose(e, e1 + e2, rtol=1e-13)
+
+
+# ---------------------------------------------------------------- select
+def _select_by_python_sort(s, k):
+    order = sorted(range(len(s)), key=lambda j: (-float(s[j]), j))
+    heavy = sorted(order[:k])
+    light = sorted(order[k:])
+    return heavy, light
+
+
+def test_select_exhaustive_tie_patterns():
+    for m in range(1, 8):
+        for pattern in itertools.product((0.0, 1.0, 2.5), repeat=m) if m <= 5 else \
+                itertools.product((0.0, 1.0), repeat=m):
+            s = np.array(pattern, dtype=np.float32)
+            for k in range(m + 1):
+                h, l = orc.select_heavy(s, k)
+                hw, lw = _select_by_python_sort(s, k)
+                assert list(h) == hw and list(l) == lw
+                h2, l2 = orc.select_heavy_argmax_rounds(s, k)
+                assert list(h2) == hw and list(l2) == lw
+
+
+def test_select_random_against_argmax_rounds(rng):
+    for m, k in [(1, 1), (17, 5), (64, 64), (100, 0), (257, 31)]:
+        s = (rng.random(m) ** 3).astype(np.float32)
+        s[rng.integers(0, m, size=m // 3)] = s[0]            # many equal keys
+        h, l = orc.select_heavy(s, k)
+        h2, l2 = orc.select_heavy_argmax_rounds(s, k)
+        assert np.array_equal(h, h2) and np.array_equal(l, l2)
+        assert h.dtype == np.int32 and len(h) == k and len(l) == m - k
+        assert sorted(set(h.tolist()) | set(l.tolist())) == list(range(m))
+        if k:
+            assert s[h].min() >= (s[l].max() if len(l) else -1)
+
+
+def test_select_edge_cases_and_invariances(rng):
+    s = rng.random(50).astype(np.float32)
+    assert np.array_equal(orc.select_heavy(s, 50)[0], np.arange(50))
+    assert len(orc.select_heavy(s, 0)[0]) == 0
+    assert np.array_equal(orc.select_heavy(s, 7)[0], orc.select_heavy(s.astype(np.float64) ** 2, 7)[0])
+    # all keys equal: the k lowest indices win
+    assert np.array_equal(orc.select_heavy(np.ones(9, np.float32), 4)[0], np.arange(4))
+    with pytest.raises(ValueError):
+        orc.select_heavy(np.array([1.0, np.nan]), 1)
+    with pytest.raises(ValueError):
+        orc.select_heavy(s, 51)
+
+
+def test_planted_heavy_hitters_are_recovered():
+    from ffsplit_synth import custom_config, make_layer
+    from conftest import f64
+    for act in ("gelu_erf", "swiglu"):
+        cfg = custom_config(64, 256, 13, 16, act=act, dtype="f32")
+        L = make_layer(cfg, 0)
+        X = L.tokens(128)
+        _, _, s = orc.neuron_scores(f64(X), f64(L.W1), f64(L.b1), f64(L.W2), act, orc.SCORE_EQ3, f64(L.W1u))
+        heavy, _ = orc.select_heavy(s, 13)
+        assert np.array_equal(heavy, L.planted.numpy())
+        # and the gap to the best light neuron is wide (x100 from the V rows)
+        light_best = np.max(np.delete(s, heavy))
+        assert s[heavy].min() > 10 * light_best
+
+
+# ---------------------------------------------------------------- factors
+def test_light_factors_eckart_young(rng):
+    W = rng.normal(size=(12, 30))
+    sig2 = np.sort(np.linalg.eigvalsh(W @ W.T))[::-1]         # squared singular values, another routine
+    for r in (0, 1, 5, 12):
+        A, B = orc.light_factors(W, r)
+        assert A.shape == (12, r) and B.shape == (r, 30)
+        resid = np.sum((W - A @ B) ** 2)
+        assert abs(resid - np.sum(sig2[r:])) < 1e-9
+    A, B = orc.light_factors(W, 12)
+    assert np.allclose(A @ B, W, atol=1e-12)
+    # balanced split: both factors carry sqrt(sigma)
+    A, B = orc.light_factors(W, 4)
+    assert np.allclose(np.linalg.norm(A, axis=0), np.linalg.norm(B, axis=1), rtol=1e-10)
+
+
+def test_light_factors_known_spectrum(rng):
+    Q1, _ = np.linalg.qr(rng.normal(size=(10, 10)))
+    Q2, _ = np.linalg.qr(rng.normal(size=(25, 10)))
+    s = np.array([9.0, 7, 5, 3, 2, 1, .5, .25, .1, .05])
+    W = (Q1 * s) @ Q2.T
+    A, B = orc.light_factors(W, 3)
+    assert np.allclose(A @ B, (Q1[:, :3] * s[:3]) @ Q2[:, :3].T, atol=1e-12)
+
+
+# ---------------------------------------------------------------- split FFN
+def _full_rank_factors(sw, act):
+    f = {}
+    f["A1"], f["B1"] = orc.light_factors(sw["U2"], min(sw["U2"].shape))
+    f["A2"], f["B2"] = orc.light_factors(sw["V2"], min(sw["V2"].shape))
+    if act == orc.ACT_SWIGLU:
+        f["A1u"], f["B1u"] = orc.light_factors(sw["U2u"], min(sw["U2u"].shape))
+    return f
+
+
+@pytest.mark.parametrize("act", ACTS)
+def test_split_reproduces_dense(rng, act):
+    """Eq. 2 holds for any index set; k = d_ff, k = 0 and full-rank light factors
+    all give back the dense FFN."""
+    X, W1, W1u, b1, W2, b2 = _tiny(rng, s=6, d=5, m=11, act=act)
+    dense = orc.dense_ffn(X, W1, b1, W2, b2, act, W1u)
+    m = W1.shape[1]
+    for heavy in ([], [3], [0, 4, 10], [10, 2, 7, 1], list(range(m))):
+        y = orc.split_ffn(X, W1, b1, W2, b2, heavy, None, act, W1u)
+        assert np.allclose(y, dense, rtol=1e-12, atol=1e-12)
+        if len(heavy) < m:
+            sw = orc.split_weights(W1, b1, W2, heavy, W1u)
+            y = orc.split_ffn(X, W1, b1, W2, b2, heavy, _full_rank_factors(sw, act), act, W1u)
+            assert np.allclose(y, dense, rtol=1e-10, atol=1e-10)
+    # ascending full set is the same summation order as the dense FFN
+    y = orc.split_ffn(X, W1, b1, W2, b2, np.arange(m), None, act, W1u)
+    assert np.array_equal(y, dense)
+
+
+@pytest.mark.parametrize("act", ACTS)
+def test_split_truncated_rank_is_exact_on_low_rank_light_slices(rng, act):
+    """If the light slices have rank <= r, the rank-r factors lose nothing."""
+    s, d, m, r = 7, 8, 20, 3
+    heavy = [1, 5, 6, 19]
+    light = [j for j in range(m) if j not in heavy]
+    X = rng.normal(size=(s, d))
+
+    def low_rank_except_heavy(shape_rows, along_cols):
+        W = rng.normal(size=shape_rows)
+        L = rng.normal(size=(d, r)) @ rng.normal(size=(r, len(light)))
+        if along_cols:
+            W[:, light] = L
+        else:
+            W[light, :] = L.T
+        return W
+
+    W1 = low_rank_except_heavy((d, m), True)
+    W1u = low_rank_except_heavy((d, m), True) if act == orc.ACT_SWIGLU else None
+    W2 = low_rank_except_heavy((m, d), False)
+    b1 = rng.normal(size=m) if act != orc.ACT_SWIGLU else None
+    b2 = rng.normal(size=d)
+    sw = orc.split_weights(W1, b1, W2, heavy, W1u)
+    f = {}
+    f["A1"], f["B1"] = orc.light_factors(sw["U2"], r)
+    f["A2"], f["B2"] = orc.light_factors(sw["V2"], r)
+    if act == orc.ACT_SWIGLU:
+        f["A1u"], f["B1u"] = orc.light_factors(sw["U2u"], r)
+    y = orc.split_ffn(X, W1, b1, W2, b2, heavy, f, act, W1u)
+    assert np.allclose(y, orc.dense_ffn(X, W1, b1, W2, b2, act, W1u), rtol=1e-9, atol=1e-9)
+    # rank 0 drops the light part: what is left is the FFN over the heavy neurons only
+    f0 = {key: (v[:, :0] if key.startswith("A") else v[:0, :]) for key, v in f.items()}
+    y0 = orc.split_ffn(X, W1, b1, W2, b2, heavy, f0, act, W1u)
+    only = orc.dense_ffn(X, W1[:, heavy], None if b1 is None else b1[heavy], W2[heavy, :], b2, act,
+                         None if W1u is None else W1u[:, heavy])
+    assert np.allclose(y0, only, rtol=1e-12, atol=1e-12)
+
+
+def test_split_truncation_changes_the_output_and_uses_the_given_factors(rng):
+    X, W1, W1u, b1, W2, b2 = _tiny(rng, s=6, d=6, m=14)
+    heavy = [0, 3, 9]
+    sw = orc.split_weights(W1, b1, W2, heavy)
+    f = {}
+    f["A1"], f["B1"] = orc.light_factors(sw["U2"], 2)
+    f["A2"], f["B2"] = orc.light_factors(sw["V2"], 2)
+    y = orc.split_ffn(X, W1, b1, W2, b2, heavy, f, orc.ACT_GELU_ERF)
+    # same thing spelled out with the reconstructed light matrices
+    U2h, V2h = f["A1"] @ f["B1"], f["A2"] @ f["B2"]
+    W1c, W2c = W1.copy(), W2.copy()
+    W1c[:, sw["light"]] = U2h
+    W2c[sw["light"], :] = V2h
+    assert np.allclose(y, orc.dense_ffn(X, W1c, b1, W2c, b2, orc.ACT_GELU_ERF), rtol=1e-11, atol=1e-11)
+    assert not np.allclose(y, orc.dense_ffn(X, W1, b1, W2, b2, orc.ACT_GELU_ERF), atol=1e-3)
+
+
+@pytest.mark.parametrize("act", ACTS)
+def test_split_permutation_and_padding_invariance(rng, act):
+    X, W1, W1u, b1, W2, b2 = _tiny(rng, s=4, d=5, m=9, act=act)
+    heavy = np.array([2, 7, 8])
+    sw = orc.split_weights(W1, b1, W2, heavy, W1u)
+    f = {}
+    f["A1"], f["B1"] = orc.light_factors(sw["U2"], 2)
+    f["A2"], f["B2"] = orc.light_factors(sw["V2"], 2)
+    if act == orc.ACT_SWIGLU:
+        f["A1u"], f["B1u"] = orc.light_factors(sw["U2u"], 2)
+    y = orc.split_ffn(X, W1, b1, W2, b2, heavy, f, act, W1u)
+    # relabel neurons: move every neuron j to position perm_inv[j]; keep the light
+    # order inside the factors by permuting only heavy labels among themselves and
+    # shifting the whole layer by appended zero neurons (padding)
+    m = W1.shape[1]
+    pad = 3
+    W1p = np.concatenate([W1, np.zeros((W1.shape[0], pad))], axis=1)
+    W2p = np.concatenate([W2, np.zeros((pad, W2.shape[1]))], axis=0)
+    W1up = None if W1u is None else np.concatenate([W1u, np.zeros((W1u.shape[0], pad))], axis=1)
+    b1p = None if b1 is None else np.concatenate([b1, np.zeros(pad)])
+    heavy_p = np.concatenate([heavy, np.arange(m, m + pad)])      # zero neurons join the heavy set
+    yp = orc.split_ffn(X, W1p, b1p, W2p, b2, heavy_p, f, act, W1up)
+    assert np.allclose(yp, y, rtol=1e-13, atol=1e-13)
+    # permutation of the whole neuron axis, exact light part (Eq. 1 is a sum over neurons)
+    perm = rng.permutation(m)
+    inv = np.argsort(perm)
+    y_exact = orc.split_ffn(X, W1, b1, W2, b2, heavy, None, act, W1u)
+    yq = orc.split_ffn(X, W1[:, perm], None if b1 is None else b1[perm], W2[perm, :], b2, inv[heavy], None, act,
+                       None if W1u is None else W1u[:, perm])
+    assert np.allclose(yq, y_exact, rtol=1e-12, atol=1e-12)
+
+
+def test_split_weights_are_plain_gathers(rng):
+    X, W1, W1u, b1, W2, b2 = _tiny(rng, m=9)
+    sw = orc.split_weights(W1, b1, W2, [7, 2])
+    assert np.array_equal(sw["U1"][:, 0], W1[:, 7]) and np.array_equal(sw["V1"][1], W2[2])
+    assert list(sw["light"]) == [0, 1, 3, 4, 5, 6, 8]
+    assert np.array_equal(sw["U2"][:, 2], W1[:, 3]) and np.array_equal(sw["V2"][6], W2[8])
+    assert np.array_equal(sw["b1_light"], b1[sw["light"]])
+
+
+# ---------------------------------------------------------------- model size
+def test_param_reduction_matches_the_paper():
+    rows = [l.split() for l in open(os.path.join(GOLDEN, "param_reduction.txt")) if l[0] != "#" and l.strip()]
+    heavy_pc, rank_pc, printed = (float(v) for v in rows[0])
+    d, m, layers = 768, 3072, 12                    # BERT-base
+    k = round(heavy_pc / 100 * m)
+    r = round(rank_pc / 100 * min(d, m - k))
+    ffn = orc.ffn_weight_params(d, m)
+    split = orc.split_weight_params(d, m, k, r)
+    assert ffn == 2 * d * m and split == 2 * (d * k + r * (d + m - k))
+    attn = 4 * d * d
+    # weights only, and with biases + LayerNorm + pooler counted: the printed figure lies between
+    red_w = (ffn - split) / (ffn + attn)
+    other = layers * (4 * d + m + d + 4 * d) + d * d + d
+    red_all = layers * (ffn - split) / (layers * (ffn + attn) + other)
+    assert red_all * 100 <= printed + 0.15 and printed - 0.15 <= red_w * 100
+    assert abs(red_w * 100 - printed) < 0.5
+    # k = d_ff with no light part is the dense FFN
+    assert orc.split_weight_params(d, m, m, 0) == ffn
+    assert orc.split_weight_params(64, 256, 16, 8, n_in=2) == 3 * (64 * 16 + 8 * (64 + 240))
+
+
+def test_error_metrics():
+    a = np.array([[3.0, 4.0]])
+    assert orc.rel_frobenius(a, a) == 0
+    assert abs(orc.rel_frobenius(a + np.array([[0.3, 0.4]]), a) - 0.1) < 1e-15
+    assert abs(orc.normalised_max_abs(a + np.array([[0.0, -0.2]]), a) - 0.05) < 1e-15
