@@ -1,0 +1,200 @@
+/*
+ * ffsplit.h -- C ABI of the split feed-forward network library (FFSplit, arXiv 2401.04044).
+ *
+ * The library follows the paper's statement of the problem, per FFN layer:
+ *   weights U = W1 [d, m], V = W2 [m, d]  (Section 2: FFN(X) = sigma(X U) V)
+ *   -> calibration scores per neuron                      (Eq. 3, Section 4.2)
+ *   -> heavy-hitter index set h2 = top-k neurons          (Sections 4.1, 5.1.1)
+ *   -> split weights U1 = U[:, h2], V1 = V[h2, :] kept dense, the remaining
+ *      U2, V2 replaced by rank-r factors                  (Figure 3 caption, Section 5.1.1)
+ *   -> forward FFN(X) = FFN_1(X) + FFN_2(X)               (Eq. 2)
+ *
+ * Conventions for every entry point
+ *   - All tensors are row-major and dense.  "dev" pointers are CUDA device
+ *     memory owned by the caller; the library never allocates, frees or keeps
+ *     a tensor pointer past the call (the workspace is kept until replaced;
+ *     a packed blob's address is remembered as a cache key only).
+ *   - Storage dtype (ffsplit_dtype) applies to X, Y, weights, biases and
+ *     factors alike: FFSPLIT_BF16 computes with bf16 tensor-core products and
+ *     fp32 accumulation; FFSPLIT_F32 computes in plain fp32 (no TF32).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls
+ *     enqueue work and return; argument errors are returned synchronously and
+ *     launch nothing.  Conditions only the device can see (non-finite score,
+ *     unsorted index list, a wait that ran out) are recorded in a status word
+ *     inside the workspace and returned by ffsplit_poll().
+ *   - Device pointers must be 16-byte aligned (FFSPLIT_ERR_ALIGN otherwise).
+ *     For FFSPLIT_BF16, d must be a multiple of 8 (rows of X start 16-byte aligned).
+ *   - Same inputs give bitwise the same outputs on every call.
+ *   - Functions return FFSPLIT_OK (0) or an error code; ffsplit_last_error()
+ *     gives the text for the last failing call on that context.
+ *   - A context is bound to one device and is not thread-safe.
+ */
+#ifndef FFSPLIT_H_
+#define FFSPLIT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  FFSPLIT_OK = 0,
+  FFSPLIT_ERR_INVALID_ARG = 1,
+  FFSPLIT_ERR_SHAPE = 2,
+  FFSPLIT_ERR_ALIGN = 3,
+  FFSPLIT_ERR_DTYPE = 4,
+  FFSPLIT_ERR_BUFFER_TOO_SMALL = 5,
+  FFSPLIT_ERR_NONFINITE = 6,
+  FFSPLIT_ERR_BAD_BLOB = 7,
+  FFSPLIT_ERR_ARCH = 8,
+  FFSPLIT_ERR_CUDA = 9,
+  FFSPLIT_ERR_TIMEOUT = 10,
+  FFSPLIT_ERR_BAD_INDEX = 11
+} ffsplit_status;
+
+typedef enum { FFSPLIT_F32 = 0, FFSPLIT_BF16 = 1 } ffsplit_dtype;
+
+/* sigma of Section 2.  GELU_ERF is x*Phi(x); GELU_TANH the tanh form; SWIGLU is
+ * SiLU(X W1) * (X W1u) with no bias (named in Section 2 as the other dominant family). */
+typedef enum { FFSPLIT_GELU_ERF = 0, FFSPLIT_GELU_TANH = 1, FFSPLIT_SWIGLU = 2 } ffsplit_act;
+
+/* Which reading of the importance score is accumulated (see ffsplit_score). */
+typedef enum { FFSPLIT_SCORE_EQ3 = 0, FFSPLIT_SCORE_ACT_ONLY = 1, FFSPLIT_SCORE_SUM_NORM = 2 } ffsplit_score_mode;
+
+typedef struct {
+  int32_t d;       /* hidden width (columns of X)                */
+  int32_t m;       /* d_ff, number of FFN neurons                */
+  int32_t act;     /* ffsplit_act                                */
+  int32_t dtype;   /* ffsplit_dtype of every tensor of the layer */
+} ffsplit_shape;
+
+/* One dense FFN layer.  All dev pointers in the storage dtype. */
+typedef struct {
+  const void* W1;   /* dev [d, m]   U (GELU) or the gate projection (SwiGLU) */
+  const void* W1u;  /* dev [d, m]   SwiGLU up projection, else NULL           */
+  const void* b1;   /* dev [m]      first-layer bias, NULL = zeros (must be NULL for SwiGLU) */
+  const void* W2;   /* dev [m, d]   V                                          */
+  const void* b2;   /* dev [d]      output bias, NULL = zeros                  */
+} ffsplit_weights;
+
+/* Rank-r factors of the light slices, light neurons in ascending index order
+ * (Section 5.1.1: SVD on U2 and V2 only).  U2 ~ A1 B1, V2 ~ A2 B2. */
+typedef struct {
+  const void* A1;   /* dev [d, r]        */
+  const void* B1;   /* dev [r, m-k]      */
+  const void* A1u;  /* dev [d, r]        SwiGLU up slice, else NULL */
+  const void* B1u;  /* dev [r, m-k]      SwiGLU up slice, else NULL */
+  const void* A2;   /* dev [m-k, r]      */
+  const void* B2;   /* dev [r, d]        */
+  int32_t r;
+} ffsplit_factors;
+
+typedef struct ffsplit_ctx ffsplit_ctx;
+
+/* Create / destroy a context on CUDA device `device` (host memory only; no
+ * device allocation).  Fails with FFSPLIT_ERR_ARCH unless the device is
+ * compute capability 10.x, FFSPLIT_ERR_CUDA if the runtime reports an error. */
+ffsplit_status ffsplit_create(ffsplit_ctx** out, int device);
+ffsplit_status ffsplit_destroy(ffsplit_ctx* ctx);
+
+/* Bytes of caller-provided scratch needed for ffsplit_forward() with up to
+ * T_fwd tokens and ffsplit_score() with up to T_cal tokens per call on a layer
+ * of this shape split with (k, r).  Pass 0 for a phase that is not used.
+ * Always >= 256 (the status block). */
+ffsplit_status ffsplit_workspace_size(const ffsplit_shape* shape, int64_t T_fwd, int64_t T_cal,
+                                      int32_t k, int32_t r, size_t* bytes);
+
+/* Give the context its scratch memory (dev, 256-byte aligned).  The first 256
+ * bytes hold the device status block and are cleared here, synchronously.
+ * The workspace must outlive every call that uses the context, and calls that
+ * share a workspace must not overlap on the GPU. */
+ffsplit_status ffsplit_set_workspace(ffsplit_ctx* ctx, void* dev_ptr, size_t bytes);
+
+/* Heavy-hitter scoring over one batch of calibration tokens (Eq. 3; Section
+ * 4.2, "go over a small training set").
+ *   X       dev [T, d] calibration tokens, T >= 1
+ *   energy  dev float[m], caller-owned accumulator: e_j = sum_t H[t,j]^2 with
+ *           H = sigma(X W1 + b1) (sum_t |H[t,j]| for SCORE_SUM_NORM).
+ *           accumulate = 0 overwrites it, 1 adds this batch to it.
+ *   scores  dev float[m] or NULL.  When given: s_j = e_j * w_j (EQ3),
+ *           e_j (ACT_ONLY) or e_j * sqrt(w_j) (SUM_NORM), w_j = sum_c W2[j,c]^2,
+ *           formed from the accumulated energy after this batch.
+ * The T x m activation matrix is never written to memory.  Uses the workspace. */
+ffsplit_status ffsplit_score(ffsplit_ctx* ctx, const ffsplit_shape* shape, const ffsplit_weights* weights,
+                             const void* X, int64_t T, int32_t mode, int32_t accumulate,
+                             float* energy, float* scores, void* stream);
+
+/* Deterministic top-k (Section 4.1: the neurons with the highest output norm
+ * are the heavy hitters).  Equal scores go to the lower index.
+ *   scores     dev float[m], finite (a NaN/Inf sets FFSPLIT_ERR_NONFINITE in the status block)
+ *   heavy_idx  dev int32[k], ascending           (may be NULL when k == 0)
+ *   light_idx  dev int32[m-k], ascending, or NULL if not wanted
+ * 0 <= k <= m. */
+ffsplit_status ffsplit_select(ffsplit_ctx* ctx, const float* scores, int32_t m, int32_t k,
+                              int32_t* heavy_idx, int32_t* light_idx, void* stream);
+
+/* Size of the packed layer: `padded_bytes` is what ffsplit_pack() writes (tile
+ * padding and header included), `logical_bytes` counts the split model's
+ * weights and biases only: sizeof(dtype) * ((n_in+1) * (d k + r (d + m - k)) + m + d). */
+ffsplit_status ffsplit_pack_size(const ffsplit_shape* shape, int32_t k, int32_t r,
+                                 size_t* padded_bytes, size_t* logical_bytes);
+
+/* Build the split layer (Figure 3 caption: U1 = U[:, h2], V1 = V[h2, :], kept
+ * unchanged; the light slices are given as factors).
+ *   heavy_idx  dev int32[k], strictly ascending, each in [0, m)  (else
+ *              FFSPLIT_ERR_BAD_INDEX in the status block)
+ *   factors    NULL (or r == 0) drops the light part: required when k == m;
+ *              with k < m it yields FFN_1 alone
+ *   blob       dev, 256-byte aligned, blob_bytes >= padded_bytes; position
+ *              independent (may be copied or saved and reloaded as bytes)
+ * The heavy slices in the blob are bit-exact copies of the inputs. */
+ffsplit_status ffsplit_pack(ffsplit_ctx* ctx, const ffsplit_shape* shape, const ffsplit_weights* weights,
+                            const int32_t* heavy_idx, int32_t k, const ffsplit_factors* factors,
+                            void* blob, size_t blob_bytes, void* stream);
+
+/* Register a blob that reached device memory by other means than ffsplit_pack()
+ * on this context (a copy, a reload).  Reads and validates its header
+ * (synchronous 256-byte copy).  FFSPLIT_ERR_BAD_BLOB if it is not a blob. */
+ffsplit_status ffsplit_blob_open(ffsplit_ctx* ctx, const void* blob, size_t blob_bytes);
+
+/* Where one matrix of the blob lives, for inspection and tests.
+ * which: 0 heavy U1^T [k_pad, d] (1: SwiGLU up), 2 A1^T [r_pad, d] (3: up),
+ *        4 B1^T [mL_pad, r_pad] (5: up), 6 A2^T [r_pad, mL_pad],
+ *        7 [V1 ; B2]^T [d, k_pad + r_pad], 8 b1[h2] f32, 9 b1[light] f32, 10 b2 f32.
+ * Returns byte offset, rows, cols and leading dimension (elements). */
+ffsplit_status ffsplit_blob_section(ffsplit_ctx* ctx, const void* blob, int32_t which,
+                                    size_t* offset, int64_t* rows, int64_t* cols, int64_t* ld);
+
+/* Split forward (Eq. 2): Y = sigma(X U1 + b1[h2]) V1 + sigma((X A1) B1 + b1[light]) (A2 B2) + b2.
+ *   X dev [T, d], Y dev [T, d], T >= 1, both in the blob's dtype.  Uses the workspace.
+ * A blob packed with k == m is the dense FFN through the same kernels. */
+ffsplit_status ffsplit_forward(ffsplit_ctx* ctx, const void* blob, const void* X, int64_t T,
+                               void* Y, void* stream);
+
+/* Same computation with HOST buffers: X_host [T, d] is copied to the device,
+ * the forward runs, Y is copied back to Y_host [T, d]; all three on `stream`
+ * (pinned host memory makes the copies asynchronous).  The workspace must have
+ * been sized for T_fwd >= T. */
+ffsplit_status ffsplit_forward_host(ffsplit_ctx* ctx, const void* blob, const void* X_host, int64_t T,
+                                    void* Y_host, void* stream);
+
+/* Synchronise `stream`, then return and clear the device status word
+ * (FFSPLIT_OK if no kernel recorded a condition). */
+ffsplit_status ffsplit_poll(ffsplit_ctx* ctx, void* stream);
+
+/* Number of kernels this context has launched so far. */
+int64_t ffsplit_launch_count(const ffsplit_ctx* ctx);
+
+/* Text for the last error returned on this context ("" if none).  Valid until
+ * the next call on the context.  ctx may be NULL (returns a static string). */
+const char* ffsplit_last_error(const ffsplit_ctx* ctx);
+
+/* Library version, major*10000 + minor*100 + patch. */
+int32_t ffsplit_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FFSPLIT_H_ */
