@@ -1,0 +1,164 @@
+// Internal declarations shared by the translation units of libffsplit.
+// Nothing here is part of the public ABI (see include/ffsplit.h).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <unordered_map>
+#include <vector>
+
+#include "ffsplit.h"
+
+namespace ffs {
+
+// ----------------------------------------------------------------------------
+// Device status block: the first 256 bytes of the workspace.
+// word 0: first ffsplit_status recorded by a kernel (0 = none)
+// word 1: detail (an index, a CTA id ...), word 2: kernel id
+// ----------------------------------------------------------------------------
+constexpr size_t kStatusBytes = 256;
+
+enum KernelId : int {
+  KID_SELECT = 1, KID_PACK = 2, KID_GEMM_TC = 3, KID_GEMM_SIMT = 4, KID_SCORE = 5, KID_DECODE = 6, KID_FUSED = 7
+};
+
+__device__ __forceinline__ void record_status(int* status, int code, int detail, int kid) {
+  if (atomicCAS(status, 0, code) == 0) {
+    status[1] = detail;
+    status[2] = kid;
+  }
+}
+
+// ----------------------------------------------------------------------------
+// Epilogue description shared by the tensor-core and the SIMT GEMM.
+// The GEMM computes acc[row, n] = sum_k A[row, k] * B[n, k]  (both operands
+// K-major).  Per output column n:
+//   v = acc + (n < n_bias ? bias[n] : 0)
+//   if (n < n_act) v = act(v)            (gated: v = silu(acc0) * acc1)
+//   n <  n_split : C0[row * ld0 + n]            = v
+//   n >= n_split : C1[row * ld1 + (n - n_split)] = v
+// Score mode (col_partial != nullptr): nothing is stored; instead one partial
+// per row group g and column: col_partial[g * N + n] = sum over the group's valid
+// rows of act(v)^2 (or |act(v)|).  Row groups are 32 rows (tensor-core kernel)
+// or 64 rows (SIMT kernel).
+// ----------------------------------------------------------------------------
+struct Epilogue {
+  void* C0;
+  void* C1;
+  long long ld0;
+  long long ld1;
+  const float* bias;
+  float* col_partial;
+  int n_split;
+  int n_act;
+  int n_bias;
+  int act;        // ffsplit_act
+  int score_abs;  // 1: accumulate |v| instead of v^2
+};
+
+struct GemmArgs {
+  const void* A0;   // [M, K], leading dimension lda0
+  const void* B0;   // [N, K], leading dimension ldb0
+  const void* A1;   // gated GEMM: second operand pair (acc1), else nullptr
+  const void* B1;
+  long long lda0, ldb0, lda1, ldb1;
+  long long M;
+  int N;
+  int K;
+  Epilogue epi;
+};
+
+// ----------------------------------------------------------------------------
+// Packed-layer header: the first 256 bytes of a blob.
+// ----------------------------------------------------------------------------
+constexpr uint32_t kBlobMagic = 0x46465350u;  // "FFSP"
+constexpr uint32_t kBlobVersion = 1;
+constexpr int kNumSections = 11;
+
+struct BlobHeader {
+  uint32_t magic, version;
+  int32_t d, m, act, dtype;
+  int32_t k, r, n_in;
+  int32_t k_pad, r_pad, ml_pad, ml;     // ml = m - k
+  int32_t reserved0;
+  uint64_t total_bytes, logical_bytes;
+  uint64_t off[kNumSections];           // byte offsets from the blob start
+  uint8_t pad[256 - 4 * 14 - 8 * 2 - 8 * kNumSections];
+};
+static_assert(sizeof(BlobHeader) == 256, "blob header is 256 bytes");
+
+enum Section : int {
+  SEC_U1T = 0, SEC_U1UT = 1, SEC_A1T = 2, SEC_A1UT = 3, SEC_B1T = 4, SEC_B1UT = 5,
+  SEC_A2T = 6, SEC_V1B2T = 7, SEC_B1H = 8, SEC_B1L = 9, SEC_B2 = 10
+};
+
+// ----------------------------------------------------------------------------
+// Host context
+// ----------------------------------------------------------------------------
+struct TmapKey {
+  const void* ptr; long long rows, cols, ld; int box_rows; int box_cols;
+  bool operator==(const TmapKey& o) const {
+    return ptr == o.ptr && rows == o.rows && cols == o.cols && ld == o.ld && box_rows == o.box_rows &&
+           box_cols == o.box_cols;
+  }
+};
+struct TmapKeyHash {
+  size_t operator()(const TmapKey& k) const {
+    size_t h = reinterpret_cast<size_t>(k.ptr);
+    auto mix = [&h](size_t v) { h ^= v + 0x9e3779b97f4a7c15ull + (h << 6) + (h >> 2); };
+    mix((size_t)k.rows); mix((size_t)k.cols); mix((size_t)k.ld); mix((size_t)k.box_rows); mix((size_t)k.box_cols);
+    return h;
+  }
+};
+
+}  // namespace ffs
+
+struct ffsplit_ctx {
+  int device = 0;
+  int num_sms = 0;
+  int cc_major = 0, cc_minor = 0;
+  char* ws = nullptr;
+  size_t ws_bytes = 0;
+  long long launches = 0;
+  std::string err;
+  std::unordered_map<const void*, ffs::BlobHeader> blobs;
+  std::unordered_map<ffs::TmapKey, CUtensorMap, ffs::TmapKeyHash> tmaps;
+  void* encode_fn = nullptr;  // cuTensorMapEncodeTiled
+  bool attr_tc_set = false;
+  bool attr_fused_set = false;
+  int* status() const { return reinterpret_cast<int*>(ws); }
+};
+
+namespace ffs {
+
+ffsplit_status fail(ffsplit_ctx* ctx, ffsplit_status code, const std::string& msg);
+ffsplit_status check_cuda(ffsplit_ctx* ctx, cudaError_t e, const char* what);
+
+inline int round_up(int v, int q) { return (v + q - 1) / q * q; }
+inline long long round_up_ll(long long v, long long q) { return (v + q - 1) / q * q; }
+inline size_t elem_size(int dtype) { return dtype == FFSPLIT_BF16 ? 2 : 4; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// launchers (each returns a CUDA error state through check_cuda)
+ffsplit_status launch_gemm(ffsplit_ctx* ctx, int dtype, const GemmArgs& g, cudaStream_t st);
+ffsplit_status launch_select(ffsplit_ctx* ctx, const float* scores, int m, int k, int* heavy, int* light,
+                             cudaStream_t st);
+ffsplit_status launch_row_energy(ffsplit_ctx* ctx, int dtype, const void* W2, int m, int d, float* w, cudaStream_t st);
+ffsplit_status launch_transpose(ffsplit_ctx* ctx, int dtype, const void* in, long long ldi, int rows, int cols,
+                                void* out, long long ldo, int rows_pad_out, int cols_pad_out, const int* row_idx,
+                                int idx_limit, cudaStream_t st);
+ffsplit_status launch_gather_cols_t(ffsplit_ctx* ctx, int dtype, const void* in, long long ldi, int rows,
+                                    const int* col_idx, int ncols, int idx_limit, void* out, long long ldo,
+                                    int rows_out_pad, cudaStream_t st);
+ffsplit_status launch_pack_bias(ffsplit_ctx* ctx, int dtype, const void* b1, const void* b2, const int* heavy, int m,
+                                int k, int d, float* b1h, int k_pad, float* b1l, int ml_pad, float* b2o,
+                                cudaStream_t st);
+ffsplit_status launch_score_finalize(ffsplit_ctx* ctx, const float* partial, int groups, int m, const float* w,
+                                     float* energy, float* scores, int mode, int accumulate, cudaStream_t st);
+ffsplit_status launch_to_f32(ffsplit_ctx* ctx, int dtype, const void* in, int n, float* out, cudaStream_t st);
+
+}  // namespace ffs
