@@ -1,0 +1,389 @@
+// bf16 tensor-core GEMM building block for sm_100a.
+//
+//   acc[row, n] = sum_k A[row, k] * B[n, k]      A: [M, K], B: [N, K], both K-major bf16
+//
+// One persistent CTA per SM walks output tiles of 128 x block_n.  Warp roles:
+//   warp 0  (one lane)  TMA producer: global -> 128B-swizzled shared tiles, 4-stage ring
+//   warp 1  (one lane)  tcgen05.mma issuer; accumulators live in tensor memory (TMEM),
+//                       two buffers so the epilogue of tile i overlaps the MMAs of tile i+1
+//   warps 2-5           epilogue: tcgen05.ld -> bias / activation / gating -> global
+// The gated form (SwiGLU) runs two operand pairs into two accumulators of the same
+// tile and combines them as silu(acc0) * acc1.
+// The score form does not store the tile; it reduces act(acc)^2 over the tile's rows
+// with warp shuffles and writes one partial per 32-row group and column (Eq. 3's
+// ||sigma(X U_j)||^2 accumulated over tokens).
+//
+// Every mbarrier wait is bounded; on expiry the CTA records FFSPLIT_ERR_TIMEOUT in
+// the status block, drains what it has in flight, frees its TMEM and returns.
+#include "epilogue.cuh"
+#include "internal.h"
+#include "ptx.cuh"
+
+namespace ffs {
+namespace tc {
+
+constexpr int BLOCK_M = 128;
+constexpr int BLOCK_K = 64;
+constexpr int MAX_BLOCK_N = 256;
+constexpr int STAGES = 4;
+constexpr int A_STAGE_BYTES = BLOCK_M * BLOCK_K * 2;
+constexpr int B_STAGE_BYTES = MAX_BLOCK_N * BLOCK_K * 2;
+constexpr int TMEM_COLS = 512;
+constexpr int ACC_STRIDE = 256;   // TMEM columns per accumulator buffer
+constexpr int GATE_OFFSET = 128;  // second accumulator of a gated tile
+constexpr int NUM_THREADS = 192;
+constexpr int BAR_BYTES = 256;
+constexpr int SMEM_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + BAR_BYTES + 1024;
+
+struct Params {
+  long long M;
+  int N, K;
+  int block_n;
+  int tiles_m, tiles_n;
+  int dual;
+  Epilogue epi;
+  int* status;
+};
+
+// Bias, activation and store of 16 consecutive columns of one row.  n_act, n_bias
+// and n_split are multiples of 16 (or >= N), so the branches are uniform per chunk.
+__device__ __forceinline__ void epilogue_chunk_store(const Params& p, long long row, int n0, float* v) {
+  const Epilogue& e = p.epi;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    const int n = n0 + i;
+    float x = v[i];
+    if (n < e.n_bias) x += __ldg(e.bias + n);
+    if (!p.dual && n < e.n_act) x = act_gelu(x, e.act);
+    v[i] = x;
+  }
+  if (row >= p.M) return;
+  const bool first = n0 < e.n_split;
+  __nv_bfloat16* base = first ? reinterpret_cast<__nv_bfloat16*>(e.C0) + row * e.ld0 + n0
+                              : reinterpret_cast<__nv_bfloat16*>(e.C1) + row * e.ld1 + (n0 - e.n_split);
+  const int limit = first ? (e.n_split < p.N ? e.n_split : p.N) : p.N;
+  if (n0 + 16 <= limit && (reinterpret_cast<uintptr_t>(base) & 15u) == 0) {
+    uint4 a, b;
+    a.x = pack_bf16x2(v[0], v[1]);   a.y = pack_bf16x2(v[2], v[3]);
+    a.z = pack_bf16x2(v[4], v[5]);   a.w = pack_bf16x2(v[6], v[7]);
+    b.x = pack_bf16x2(v[8], v[9]);   b.y = pack_bf16x2(v[10], v[11]);
+    b.z = pack_bf16x2(v[12], v[13]); b.w = pack_bf16x2(v[14], v[15]);
+    reinterpret_cast<uint4*>(base)[0] = a;
+    reinterpret_cast<uint4*>(base)[1] = b;
+  } else {
+#pragma unroll
+    for (int i = 0; i < 16; ++i)
+      if (n0 + i < limit) base[i] = __float2bfloat16_rn(v[i]);
+  }
+}
+
+// Sum v[i] over the 32 lanes of the warp for each of 16 columns with a fixed
+// exchange tree (16 shuffles).  Afterwards lane l holds the total of column l >> 1.
+__device__ __forceinline__ float warp_column_sums16(const float* v, int lane) {
+  float w[8], x[4], y[2], z;
+  const bool b4 = lane & 16, b3 = lane & 8, b2 = lane & 4, b1 = lane & 2;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const float send = b4 ? v[i] : v[i + 8];
+    const float keep = b4 ? v[i + 8] : v[i];
+    w[i] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float send = b3 ? w[i] : w[i + 4];
+    const float keep = b3 ? w[i + 4] : w[i];
+    x[i] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+  }
+#pragma unroll
+  for (int i = 0; i < 2; ++i) {
+    const float send = b2 ? x[i] : x[i + 2];
+    const float keep = b2 ? x[i + 2] : x[i];
+    y[i] = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+  }
+  {
+    const float send = b1 ? y[0] : y[1];
+    const float keep = b1 ? y[1] : y[0];
+    z = keep + __shfl_xor_sync(0xffffffffu, send, 2);
+  }
+  z += __shfl_xor_sync(0xffffffffu, z, 1);
+  return z;
+}
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmB0,
+               const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1, const Params p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* smem_a = smem;
+  uint8_t* smem_b = smem + STAGES * A_STAGE_BYTES;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES));
+  uint64_t* full = bars;                  // [STAGES] TMA -> MMA
+  uint64_t* empty = bars + STAGES;        // [STAGES] MMA -> TMA
+  uint64_t* tfull = bars + 2 * STAGES;    // [2] MMA -> epilogue
+  uint64_t* tempty = tfull + 2;           // [2] epilogue -> MMA
+  uint64_t* drain = tempty + 2;           // [1] used only when giving up
+  uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(drain + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      ptx::mbar_init(&full[s], 1);
+      ptx::mbar_init(&empty[s], 1);
+    }
+    for (int a = 0; a < 2; ++a) {
+      ptx::mbar_init(&tfull[a], 1);
+      ptx::mbar_init(&tempty[a], 4);
+    }
+    ptx::mbar_init(drain, 1);
+    *abort_flag = 0;
+    ptx::mbar_fence_init();
+    ptx::prefetch_tmap(&tmA0);
+    ptx::prefetch_tmap(&tmB0);
+    if (p.dual) {
+      ptx::prefetch_tmap(&tmA1);
+      ptx::prefetch_tmap(&tmB1);
+    }
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(tmem_holder, TMEM_COLS);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_holder;
+
+  const int nkb = (p.K + BLOCK_K - 1) / BLOCK_K;
+  const int total_kb = p.dual ? 2 * nkb : nkb;
+  const int num_tiles = p.tiles_m * p.tiles_n;
+  const uint32_t stage_tx = A_STAGE_BYTES + p.block_n * BLOCK_K * 2;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      // ------------------------------------------------------------ TMA producer
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        const int m_blk = tile / p.tiles_n, n_blk = tile % p.tiles_n;
+        for (int kb = 0; kb < total_kb; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          if (!ptx::mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; break; }
+          ptx::mbar_expect_tx(&full[s], stage_tx);
+          const bool second = p.dual && kb >= nkb;
+          const int kk = (second ? kb - nkb : kb) * BLOCK_K;
+          ptx::tma_load_2d(second ? &tmA1 : &tmA0, smem_a + s * A_STAGE_BYTES, &full[s], kk, m_blk * BLOCK_M);
+          ptx::tma_load_2d(second ? &tmB1 : &tmB0, smem_b + s * B_STAGE_BYTES, &full[s], kk, n_blk * p.block_n);
+        }
+      }
+      if (!ok) {
+        // give the copies already issued a bounded chance to land before the CTA exits
+        const uint32_t first = it > STAGES ? it - STAGES : 0;
+        for (uint32_t j = first; j < it; ++j) {
+          const long long t0 = clock64();
+          while (!ptx::mbar_try_wait(&full[j % STAGES], (j / STAGES) & 1) &&
+                 clock64() - t0 < ptx::kWaitLimitCycles / 8) {}
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    if (lane == 0) {
+      // ------------------------------------------------------------ MMA issuer
+      const uint32_t idesc = ptx::umma_idesc_bf16(BLOCK_M, p.block_n);
+      uint32_t it = 0, tl = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tl) {
+        const uint32_t acc = tl & 1, aph = (tl >> 1) & 1;
+        if (!ptx::mbar_wait(&tempty[acc], aph ^ 1, abort_flag)) { ok = false; break; }
+        ptx::tc_fence_after();
+        for (int kb = 0; kb < total_kb; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          if (!ptx::mbar_wait(&full[s], ph, abort_flag)) { ok = false; break; }
+          ptx::tc_fence_after();
+          const bool second = p.dual && kb >= nkb;
+          const int kbl = second ? kb - nkb : kb;
+          const uint32_t d_tmem = tmem_base + acc * ACC_STRIDE + (second ? GATE_OFFSET : 0);
+          const uint64_t a_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_a + s * A_STAGE_BYTES));
+          const uint64_t b_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_b + s * B_STAGE_BYTES));
+#pragma unroll
+          for (int k = 0; k < BLOCK_K / 16; ++k) {
+            // 16 elements (32 bytes) further along K inside the swizzled row: +2 in the address field
+            ptx::umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kbl | k) != 0 ? 1u : 0u);
+          }
+          ptx::umma_commit(&empty[s]);
+        }
+        if (ok) ptx::umma_commit(&tfull[acc]);
+      }
+      if (!ok) {
+        // wait (bounded) until the MMAs issued so far have retired before TMEM is freed
+        ptx::umma_commit(drain);
+        const long long t0 = clock64();
+        while (!ptx::mbar_try_wait(drain, 0) && clock64() - t0 < ptx::kWaitLimitCycles / 8) {}
+      }
+    }
+    __syncwarp();
+  } else {
+    // -------------------------------------------------------------- epilogue warps
+    const int q = warp & 3;  // TMEM lane quarter this warp may read
+    uint32_t tl = 0;
+    for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++tl) {
+      const int m_blk = tile / p.tiles_n, n_blk = tile % p.tiles_n;
+      const uint32_t acc = tl & 1, aph = (tl >> 1) & 1;
+      if (!ptx::mbar_wait(&tfull[acc], aph, abort_flag)) break;
+      ptx::tc_fence_after();
+      const long long row = static_cast<long long>(m_blk) * BLOCK_M + q * 32 + lane;
+      const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * ACC_STRIDE;
+      for (int c = 0; c < p.block_n; c += 16) {
+        const int n0 = n_blk * p.block_n + c;
+        if (n0 >= p.N) break;
+        float v[16];
+        ptx::tmem_ld16(t_row + c, v);
+        if (p.dual) {
+          float u[16];
+          ptx::tmem_ld16(t_row + GATE_OFFSET + c, u);
+          ptx::tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 16; ++i) v[i] = silu_f(v[i]) * u[i];
+        } else {
+          ptx::tmem_ld_wait();
+        }
+        if (p.epi.col_partial == nullptr) {
+          epilogue_chunk_store(p, row, n0, v);
+        } else {
+          const Epilogue& e = p.epi;
+#pragma unroll
+          for (int i = 0; i < 16; ++i) {
+            const int n = n0 + i;
+            float x = v[i];
+            if (n < e.n_bias) x += __ldg(e.bias + n);
+            if (!p.dual) x = act_gelu(x, e.act);
+            x = e.score_abs ? fabsf(x) : x * x;
+            v[i] = (row < p.M) ? x : 0.0f;
+          }
+          const float tot = warp_column_sums16(v, lane);
+          const int n = n0 + (lane >> 1);
+          if ((lane & 1) == 0 && n < p.N)
+            e.col_partial[(static_cast<long long>(m_blk) * 4 + q) * p.N + n] = tot;
+        }
+      }
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&tempty[acc]);
+    }
+  }
+
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) record_status(p.status, FFSPLIT_ERR_TIMEOUT, blockIdx.x, KID_GEMM_TC);
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, TMEM_COLS);
+  }
+}
+
+}  // namespace tc
+
+// ---------------------------------------------------------------------------------
+// Host side: tensor maps and launch
+// ---------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// 2-D bf16 tensor map over a row-major [rows, cols] matrix with pitch ld, box
+// [box_rows, 64 columns], 128-byte swizzle, zero fill outside the matrix.
+ffsplit_status get_tmap_bf16(ffsplit_ctx* ctx, const void* ptr, long long rows, long long cols, long long ld,
+                             int box_rows, CUtensorMap* out) {
+  TmapKey key{ptr, rows, cols, ld, box_rows, tc::BLOCK_K};
+  auto it = ctx->tmaps.find(key);
+  if (it != ctx->tmaps.end()) {
+    *out = it->second;
+    return FFSPLIT_OK;
+  }
+  if (!ctx->encode_fn) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess || qres != cudaDriverEntryPointSuccess || !fn)
+      return fail(ctx, FFSPLIT_ERR_CUDA, "cuTensorMapEncodeTiled is not available from the driver");
+    ctx->encode_fn = fn;
+  }
+  if (!aligned16(ptr) || (ld * 2) % 16 != 0)
+    return fail(ctx, FFSPLIT_ERR_ALIGN, "tensor-core operand needs a 16-byte aligned base and row pitch");
+  cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+  cuuint64_t strides[1] = {static_cast<cuuint64_t>(ld) * 2};
+  cuuint32_t box[2] = {static_cast<cuuint32_t>(tc::BLOCK_K), static_cast<cuuint32_t>(box_rows)};
+  cuuint32_t estr[2] = {1, 1};
+  CUtensorMap tm;
+  CUresult r = reinterpret_cast<EncodeTiledFn>(ctx->encode_fn)(
+      &tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS)
+    return fail(ctx, FFSPLIT_ERR_CUDA, "cuTensorMapEncodeTiled failed (" + std::to_string((int)r) + ")");
+  if (ctx->tmaps.size() > 8192) ctx->tmaps.clear();
+  ctx->tmaps.emplace(key, tm);
+  *out = tm;
+  return FFSPLIT_OK;
+}
+
+// Pick the tile width: fewest waves weighted by tile cost, wider tiles on ties.
+static int choose_block_n(int N, long long tiles_m, int num_sms, bool dual) {
+  const int max_bn = dual ? 128 : 256;
+  int best = 32;
+  double best_cost = 1e300;
+  for (int bn = max_bn; bn >= 32; bn -= 16) {
+    const long long tiles = tiles_m * ((N + bn - 1) / bn);
+    const long long waves = (tiles + num_sms - 1) / num_sms;
+    const double cost = static_cast<double>(waves) * (bn + 40);
+    if (cost < best_cost - 1e-9) {
+      best_cost = cost;
+      best = bn;
+    }
+  }
+  return best;
+}
+
+ffsplit_status launch_gemm_tc(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_t st) {
+  const bool dual = g.A1 != nullptr;
+  if (g.M <= 0 || g.N <= 0 || g.K <= 0) return FFSPLIT_OK;
+  tc::Params p;
+  p.M = g.M;
+  p.N = g.N;
+  p.K = g.K;
+  p.dual = dual ? 1 : 0;
+  p.tiles_m = static_cast<int>((g.M + tc::BLOCK_M - 1) / tc::BLOCK_M);
+  p.block_n = choose_block_n(g.N, p.tiles_m, ctx->num_sms, dual);
+  p.tiles_n = (g.N + p.block_n - 1) / p.block_n;
+  p.epi = g.epi;
+  p.status = ctx->status();
+  CUtensorMap tA0, tB0, tA1, tB1;
+  ffsplit_status s;
+  if ((s = get_tmap_bf16(ctx, g.A0, g.M, g.K, g.lda0, tc::BLOCK_M, &tA0)) != FFSPLIT_OK) return s;
+  if ((s = get_tmap_bf16(ctx, g.B0, g.N, g.K, g.ldb0, p.block_n, &tB0)) != FFSPLIT_OK) return s;
+  if (dual) {
+    if ((s = get_tmap_bf16(ctx, g.A1, g.M, g.K, g.lda1, tc::BLOCK_M, &tA1)) != FFSPLIT_OK) return s;
+    if ((s = get_tmap_bf16(ctx, g.B1, g.N, g.K, g.ldb1, p.block_n, &tB1)) != FFSPLIT_OK) return s;
+  } else {
+    tA1 = tA0;
+    tB1 = tB0;
+  }
+  if (!ctx->attr_tc_set) {
+    cudaError_t e = cudaFuncSetAttribute(tc::gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         tc::SMEM_BYTES);
+    if (e != cudaSuccess) return check_cuda(ctx, e, "cudaFuncSetAttribute(gemm_tc_kernel)");
+    ctx->attr_tc_set = true;
+  }
+  const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n;
+  const int grid = static_cast<int>(tiles < ctx->num_sms ? tiles : ctx->num_sms);
+  tc::gemm_tc_kernel<<<grid, tc::NUM_THREADS, tc::SMEM_BYTES, st>>>(tA0, tB0, tA1, tB1, p);
+  ctx->launches++;
+  return check_cuda(ctx, cudaGetLastError(), "gemm_tc_kernel launch");
+}
+
+}  // namespace ffs
