@@ -7,7 +7,7 @@
 
 #include "ffsplit.h"
 
-namespace ffs {
+namespace ffsp {
 
 __device__ __forceinline__ float gelu_erf_f(float z) { return 0.5f * z * (1.0f + erff(z * 0.70710678118654752f)); }
 __device__ __forceinline__ float gelu_tanh_f(float z) {
@@ -35,4 +35,4 @@ template <typename T> __device__ __forceinline__ T from_float(float v);
 template <> __device__ __forceinline__ float from_float<float>(float v) { return v; }
 template <> __device__ __forceinline__ __nv_bfloat16 from_float<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
 
-}  // namespace ffs
+}  // namespace ffsp

@@ -19,7 +19,7 @@
 #include "internal.h"
 #include "ptx.cuh"
 
-namespace ffs {
+namespace ffsp {
 namespace tc {
 
 constexpr int BLOCK_M = 128;
@@ -386,4 +386,4 @@ ffsplit_status launch_gemm_tc(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_t 
   return check_cuda(ctx, cudaGetLastError(), "gemm_tc_kernel launch");
 }
 
-}  // namespace ffs
+}  // namespace ffsp

@@ -13,7 +13,7 @@
 
 #include "ffsplit.h"
 
-namespace ffs {
+namespace ffsp {
 
 // ----------------------------------------------------------------------------
 // Device status block: the first 256 bytes of the workspace.
@@ -115,7 +115,7 @@ struct TmapKeyHash {
   }
 };
 
-}  // namespace ffs
+}  // namespace ffsp
 
 struct ffsplit_ctx {
   int device = 0;
@@ -125,15 +125,15 @@ struct ffsplit_ctx {
   size_t ws_bytes = 0;
   long long launches = 0;
   std::string err;
-  std::unordered_map<const void*, ffs::BlobHeader> blobs;
-  std::unordered_map<ffs::TmapKey, CUtensorMap, ffs::TmapKeyHash> tmaps;
+  std::unordered_map<const void*, ffsp::BlobHeader> blobs;
+  std::unordered_map<ffsp::TmapKey, CUtensorMap, ffsp::TmapKeyHash> tmaps;
   void* encode_fn = nullptr;  // cuTensorMapEncodeTiled
   bool attr_tc_set = false;
   bool attr_fused_set = false;
   int* status() const { return reinterpret_cast<int*>(ws); }
 };
 
-namespace ffs {
+namespace ffsp {
 
 ffsplit_status fail(ffsplit_ctx* ctx, ffsplit_status code, const std::string& msg);
 ffsplit_status check_cuda(ffsplit_ctx* ctx, cudaError_t e, const char* what);
@@ -161,4 +161,4 @@ ffsplit_status launch_score_finalize(ffsplit_ctx* ctx, const float* partial, int
                                      float* energy, float* scores, int mode, int accumulate, cudaStream_t st);
 ffsplit_status launch_to_f32(ffsplit_ctx* ctx, int dtype, const void* in, int n, float* out, cudaStream_t st);
 
-}  // namespace ffs
+}  // namespace ffsp

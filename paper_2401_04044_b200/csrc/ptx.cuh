@@ -5,7 +5,7 @@
 #include <cuda.h>
 #include <stdint.h>
 
-namespace ffs {
+namespace ffsp {
 namespace ptx {
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -141,4 +141,4 @@ __device__ __forceinline__ uint32_t umma_idesc_bf16(int M, int N) {
 }
 
 }  // namespace ptx
-}  // namespace ffs
+}  // namespace ffsp
