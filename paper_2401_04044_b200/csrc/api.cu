@@ -1,0 +1,536 @@
+// C ABI of libffsplit: argument validation, memory layouts (workspace, packed
+// blob) and the sequencing of kernels for score / select / pack / forward.
+#include <cstring>
+
+#include "internal.h"
+
+using namespace ffsp;
+
+namespace ffsp {
+
+ffsplit_status fail(ffsplit_ctx* ctx, ffsplit_status code, const std::string& msg) {
+  if (ctx) ctx->err = msg;
+  return code;
+}
+
+ffsplit_status check_cuda(ffsplit_ctx* ctx, cudaError_t e, const char* what) {
+  if (e == cudaSuccess) return FFSPLIT_OK;
+  if (ctx) ctx->err = std::string(what) + ": " + cudaGetErrorString(e);
+  return FFSPLIT_ERR_CUDA;
+}
+
+ffsplit_status launch_decode_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* blob, const void* X,
+                                     long long T, void* Y, char* ws_after_status, cudaStream_t st);
+bool decode_path_applies(const ffsplit_ctx* ctx, const BlobHeader& h, long long T);
+size_t decode_workspace_bytes(const BlobHeader& h, long long T);
+
+namespace {
+
+constexpr size_t kAlign = 256;
+inline size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
+
+struct SplitDims {
+  int k, r, ml, k_pad, r_pad, ml_pad, kp_rp, n_in;
+};
+
+SplitDims make_dims(const ffsplit_shape& s, int k, int r) {
+  SplitDims o;
+  o.k = k;
+  o.r = r;
+  o.ml = s.m - k;
+  o.n_in = s.act == FFSPLIT_SWIGLU ? 2 : 1;
+  o.k_pad = round_up(k, 16);
+  o.r_pad = round_up(r, 16);
+  o.ml_pad = r > 0 ? round_up(o.ml, 16) : 0;
+  if (o.k_pad + o.r_pad == 0) o.k_pad = 16;  // keeps the last GEMM non-empty: Y = b2
+  o.kp_rp = o.k_pad + o.r_pad;
+  return o;
+}
+
+ffsplit_status check_shape(ffsplit_ctx* ctx, const ffsplit_shape* s) {
+  if (!s) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "shape is NULL");
+  if (s->d < 1 || s->m < 1) return fail(ctx, FFSPLIT_ERR_SHAPE, "d and m must be >= 1");
+  if (s->act < 0 || s->act > 2) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "unknown activation");
+  if (s->dtype != FFSPLIT_F32 && s->dtype != FFSPLIT_BF16) return fail(ctx, FFSPLIT_ERR_DTYPE, "unknown dtype");
+  if (s->dtype == FFSPLIT_BF16 && s->d % 8 != 0)
+    return fail(ctx, FFSPLIT_ERR_SHAPE, "bf16 layers need d to be a multiple of 8");
+  return FFSPLIT_OK;
+}
+
+ffsplit_status check_split(ffsplit_ctx* ctx, const ffsplit_shape* s, int k, int r) {
+  if (k < 0 || k > s->m) return fail(ctx, FFSPLIT_ERR_SHAPE, "k must be in [0, m]");
+  const int ml = s->m - k;
+  const int rmax = s->d < ml ? s->d : ml;
+  if (r < 0 || r > rmax) return fail(ctx, FFSPLIT_ERR_SHAPE, "r must be in [0, min(d, m - k)]");
+  return FFSPLIT_OK;
+}
+
+void layout_blob(const ffsplit_shape& s, const SplitDims& D, BlobHeader* h) {
+  std::memset(h, 0, sizeof(*h));
+  const size_t es = elem_size(s.dtype);
+  h->magic = kBlobMagic;
+  h->version = kBlobVersion;
+  h->d = s.d; h->m = s.m; h->act = s.act; h->dtype = s.dtype;
+  h->k = D.k; h->r = D.r; h->n_in = D.n_in;
+  h->k_pad = D.k_pad; h->r_pad = D.r_pad; h->ml_pad = D.ml_pad; h->ml = D.ml;
+  size_t off = sizeof(BlobHeader);
+  // U1^T, A1^T (and the SwiGLU up factor) are adjacent with the same pitch d, so
+  // that [U1 | A1]^T and [A1 | A1u]^T can each be read as one matrix.
+  h->off[SEC_U1T] = off;  off += (size_t)D.k_pad * s.d * es;
+  h->off[SEC_A1T] = off;  off += (size_t)D.r_pad * s.d * es;
+  if (D.n_in == 2) { h->off[SEC_A1UT] = off; off += (size_t)D.r_pad * s.d * es; }
+  off = align_up(off);
+  if (D.n_in == 2) { h->off[SEC_U1UT] = off; off = align_up(off + (size_t)D.k_pad * s.d * es); }
+  h->off[SEC_B1T] = off;  off = align_up(off + (size_t)D.ml_pad * D.r_pad * es);
+  if (D.n_in == 2) { h->off[SEC_B1UT] = off; off = align_up(off + (size_t)D.ml_pad * D.r_pad * es); }
+  h->off[SEC_A2T] = off;  off = align_up(off + (size_t)D.r_pad * D.ml_pad * es);
+  h->off[SEC_V1B2T] = off; off = align_up(off + (size_t)s.d * D.kp_rp * es);
+  h->off[SEC_B1H] = off;  off = align_up(off + (size_t)D.k_pad * 4);
+  h->off[SEC_B1L] = off;  off = align_up(off + (size_t)D.ml_pad * 4);
+  h->off[SEC_B2] = off;   off = align_up(off + (size_t)s.d * 4);
+  h->total_bytes = off;
+  const size_t params = (size_t)(D.n_in + 1) * ((size_t)s.d * D.k + (size_t)D.r * (s.d + D.ml));
+  h->logical_bytes = es * (params + s.m + s.d);
+}
+
+SplitDims dims_of(const BlobHeader& h) {
+  SplitDims D;
+  D.k = h.k; D.r = h.r; D.ml = h.ml; D.k_pad = h.k_pad; D.r_pad = h.r_pad; D.ml_pad = h.ml_pad;
+  D.kp_rp = h.k_pad + h.r_pad; D.n_in = h.n_in;
+  return D;
+}
+
+bool header_valid(const BlobHeader& h, size_t blob_bytes) {
+  if (h.magic != kBlobMagic || h.version != kBlobVersion) return false;
+  ffsplit_shape s{h.d, h.m, h.act, h.dtype};
+  if (s.d < 1 || s.m < 1 || s.act < 0 || s.act > 2 || (s.dtype != 0 && s.dtype != 1)) return false;
+  if (h.k < 0 || h.k > h.m || h.r < 0) return false;
+  BlobHeader ref;
+  layout_blob(s, make_dims(s, h.k, h.r), &ref);
+  if (std::memcmp(&ref, &h, sizeof(BlobHeader)) != 0) return false;
+  return blob_bytes == 0 || blob_bytes >= h.total_bytes;
+}
+
+struct FwdLayout { size_t ap, q, hl, xs, ys, end; };
+FwdLayout fwd_layout(const SplitDims& D, int d, size_t es, long long T) {
+  FwdLayout L;
+  size_t off = 0;
+  L.ap = off; off = align_up(off + (size_t)T * D.kp_rp * es);
+  L.q = off;  off = align_up(off + (size_t)T * D.n_in * D.r_pad * es);
+  L.hl = off; off = align_up(off + (size_t)T * D.ml_pad * es);
+  L.xs = off; off = align_up(off + (size_t)T * d * es);
+  L.ys = off; off = align_up(off + (size_t)T * d * es);
+  L.end = off;
+  return L;
+}
+
+struct ScoreLayout { size_t w1t, w1ut, b1f, w, partial, end; int groups; };
+ScoreLayout score_layout(const ffsplit_shape& s, long long T) {
+  ScoreLayout L;
+  const size_t es = elem_size(s.dtype);
+  size_t off = 0;
+  L.w1t = off;  off = align_up(off + (size_t)s.m * s.d * es);
+  L.w1ut = off; if (s.act == FFSPLIT_SWIGLU) off = align_up(off + (size_t)s.m * s.d * es);
+  L.b1f = off;  off = align_up(off + (size_t)s.m * 4);
+  L.w = off;    off = align_up(off + (size_t)s.m * 4);
+  L.groups = s.dtype == FFSPLIT_BF16 ? 4 * (int)((T + 127) / 128) : (int)((T + 63) / 64);
+  L.partial = off; off = align_up(off + (size_t)L.groups * s.m * 4);
+  L.end = off;
+  return L;
+}
+
+ffsplit_status check_ctx(ffsplit_ctx* ctx, bool need_ws) {
+  if (!ctx) return FFSPLIT_ERR_INVALID_ARG;
+  ctx->err.clear();
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return check_cuda(ctx, e, "cudaGetDevice");
+  if (dev != ctx->device) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "the context's device is not the current device");
+  if (need_ws && (!ctx->ws || ctx->ws_bytes < kStatusBytes))
+    return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL, "no workspace set (ffsplit_set_workspace)");
+  return FFSPLIT_OK;
+}
+
+const BlobHeader* find_blob(ffsplit_ctx* ctx, const void* blob, ffsplit_status* st) {
+  auto it = ctx->blobs.find(blob);
+  if (it != ctx->blobs.end()) return &it->second;
+  *st = ffsplit_blob_open(ctx, blob, 0);
+  if (*st != FFSPLIT_OK) return nullptr;
+  return &ctx->blobs.find(blob)->second;
+}
+
+// The three-stage split forward (Eq. 2) as a sequence of GEMMs with fused epilogues.
+ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* blob, const void* X, long long T,
+                           void* Y, cudaStream_t st) {
+  const SplitDims D = dims_of(h);
+  const size_t es = elem_size(h.dtype);
+  const int d = h.d;
+  char* base = ctx->ws + kStatusBytes;
+  const FwdLayout L = fwd_layout(D, d, es, T);
+  if (kStatusBytes + L.xs > ctx->ws_bytes)
+    return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL, "workspace too small for this forward (ffsplit_workspace_size)");
+  if (decode_path_applies(ctx, h, T)) return launch_decode_forward(ctx, h, blob, X, T, Y, base, st);
+  char* AP = base + L.ap;
+  char* Q = base + L.q;
+  char* HL = base + L.hl;
+  const float* b1h = reinterpret_cast<const float*>(blob + h.off[SEC_B1H]);
+  const float* b1l = reinterpret_cast<const float*>(blob + h.off[SEC_B1L]);
+  const float* b2 = reinterpret_cast<const float*>(blob + h.off[SEC_B2]);
+  const bool gated = h.act == FFSPLIT_SWIGLU;
+  const bool light = D.r_pad > 0 && D.ml > 0;
+  ffsplit_status s;
+  GemmArgs g;
+
+  // ---- stage 1: [A_H | Q] = X [U1 | A1], activation on the heavy columns only
+  if (!gated) {
+    std::memset(&g, 0, sizeof(g));
+    g.A0 = X; g.lda0 = d;
+    g.B0 = blob + h.off[SEC_U1T]; g.ldb0 = d;
+    g.M = T; g.N = D.kp_rp; g.K = d;
+    g.epi.C0 = AP; g.epi.ld0 = D.kp_rp;
+    g.epi.C1 = Q; g.epi.ld1 = D.r_pad;
+    g.epi.n_split = D.k_pad; g.epi.n_act = D.k_pad; g.epi.n_bias = D.k_pad;
+    g.epi.bias = b1h; g.epi.act = h.act;
+    if ((s = launch_gemm(ctx, h.dtype, g, st)) != FFSPLIT_OK) return s;
+  } else {
+    std::memset(&g, 0, sizeof(g));
+    g.A0 = X; g.lda0 = d; g.B0 = blob + h.off[SEC_U1T]; g.ldb0 = d;
+    g.A1 = X; g.lda1 = d; g.B1 = blob + h.off[SEC_U1UT]; g.ldb1 = d;
+    g.M = T; g.N = D.k_pad; g.K = d;
+    g.epi.C0 = AP; g.epi.ld0 = D.kp_rp;
+    g.epi.n_split = D.k_pad; g.epi.n_act = D.k_pad; g.epi.act = h.act;
+    if ((s = launch_gemm(ctx, h.dtype, g, st)) != FFSPLIT_OK) return s;
+    if (light) {
+      std::memset(&g, 0, sizeof(g));
+      g.A0 = X; g.lda0 = d; g.B0 = blob + h.off[SEC_A1T]; g.ldb0 = d;  // [A1 | A1u]^T
+      g.M = T; g.N = 2 * D.r_pad; g.K = d;
+      g.epi.C0 = Q; g.epi.ld0 = 2 * D.r_pad; g.epi.n_split = g.N; g.epi.act = h.act;
+      if ((s = launch_gemm(ctx, h.dtype, g, st)) != FFSPLIT_OK) return s;
+    }
+  }
+  // ---- stage 2: P = sigma(Q B1 + b1[light]) A2, written next to A_H
+  if (light) {
+    std::memset(&g, 0, sizeof(g));
+    g.A0 = Q; g.lda0 = (long long)D.n_in * D.r_pad;
+    g.B0 = blob + h.off[SEC_B1T]; g.ldb0 = D.r_pad;
+    if (gated) {
+      g.A1 = Q + (size_t)D.r_pad * es; g.lda1 = g.lda0;
+      g.B1 = blob + h.off[SEC_B1UT]; g.ldb1 = D.r_pad;
+    }
+    g.M = T; g.N = D.ml_pad; g.K = D.r_pad;
+    g.epi.C0 = HL; g.epi.ld0 = D.ml_pad;
+    g.epi.n_split = g.N; g.epi.n_act = g.N; g.epi.n_bias = gated ? 0 : g.N;
+    g.epi.bias = b1l; g.epi.act = h.act;
+    if ((s = launch_gemm(ctx, h.dtype, g, st)) != FFSPLIT_OK) return s;
+
+    std::memset(&g, 0, sizeof(g));
+    g.A0 = HL; g.lda0 = D.ml_pad;
+    g.B0 = blob + h.off[SEC_A2T]; g.ldb0 = D.ml_pad;
+    g.M = T; g.N = D.r_pad; g.K = D.ml_pad;
+    g.epi.C0 = AP + (size_t)D.k_pad * es; g.epi.ld0 = D.kp_rp;
+    g.epi.n_split = g.N; g.epi.act = h.act;
+    if ((s = launch_gemm(ctx, h.dtype, g, st)) != FFSPLIT_OK) return s;
+  }
+  // ---- stage 3: Y = [A_H | P] [V1 ; B2] + b2 (heavy and light parts in one accumulator)
+  std::memset(&g, 0, sizeof(g));
+  g.A0 = AP; g.lda0 = D.kp_rp;
+  g.B0 = blob + h.off[SEC_V1B2T]; g.ldb0 = D.kp_rp;
+  g.M = T; g.N = d; g.K = light ? D.kp_rp : D.k_pad;
+  g.epi.C0 = Y; g.epi.ld0 = d;
+  g.epi.n_split = d; g.epi.n_bias = d; g.epi.bias = b2; g.epi.act = h.act;
+  return launch_gemm(ctx, h.dtype, g, st);
+}
+
+}  // namespace
+}  // namespace ffsp
+
+// =====================================================================================
+extern "C" {
+
+int32_t ffsplit_version(void) { return 100; }
+
+const char* ffsplit_last_error(const ffsplit_ctx* ctx) {
+  return ctx ? ctx->err.c_str() : "no context";
+}
+
+int64_t ffsplit_launch_count(const ffsplit_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+ffsplit_status ffsplit_create(ffsplit_ctx** out, int device) {
+  if (!out) return FFSPLIT_ERR_INVALID_ARG;
+  *out = nullptr;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) {
+    cudaGetLastError();
+    return FFSPLIT_ERR_CUDA;
+  }
+  int major = 0, minor = 0, sms = 0;
+  if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess ||
+      cudaDeviceGetAttribute(&minor, cudaDevAttrComputeCapabilityMinor, device) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess)
+    return FFSPLIT_ERR_CUDA;
+  if (major != 10) return FFSPLIT_ERR_ARCH;
+  ffsplit_ctx* c = new ffsplit_ctx();
+  c->device = device;
+  c->cc_major = major;
+  c->cc_minor = minor;
+  c->num_sms = sms;
+  *out = c;
+  return FFSPLIT_OK;
+}
+
+ffsplit_status ffsplit_destroy(ffsplit_ctx* ctx) {
+  delete ctx;
+  return FFSPLIT_OK;
+}
+
+ffsplit_status ffsplit_workspace_size(const ffsplit_shape* shape, int64_t T_fwd, int64_t T_cal, int32_t k, int32_t r,
+                                      size_t* bytes) {
+  if (!bytes) return FFSPLIT_ERR_INVALID_ARG;
+  ffsplit_status s = check_shape(nullptr, shape);
+  if (s != FFSPLIT_OK) return s;
+  if ((s = check_split(nullptr, shape, k, r)) != FFSPLIT_OK) return s;
+  if (T_fwd < 0 || T_cal < 0) return FFSPLIT_ERR_INVALID_ARG;
+  const SplitDims D = make_dims(*shape, k, r);
+  size_t need = 0;
+  if (T_fwd > 0) {
+    need = fwd_layout(D, shape->d, elem_size(shape->dtype), T_fwd).end;
+    BlobHeader h;
+    layout_blob(*shape, D, &h);
+    const size_t dec = decode_workspace_bytes(h, T_fwd);
+    if (dec > need) need = dec;
+  }
+  if (T_cal > 0) {
+    const size_t sc = score_layout(*shape, T_cal).end;
+    if (sc > need) need = sc;
+  }
+  *bytes = kStatusBytes + need;
+  return FFSPLIT_OK;
+}
+
+ffsplit_status ffsplit_set_workspace(ffsplit_ctx* ctx, void* dev_ptr, size_t bytes) {
+  ffsplit_status s = check_ctx(ctx, false);
+  if (s != FFSPLIT_OK) return s;
+  if (!dev_ptr || bytes < kStatusBytes) return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL, "workspace needs >= 256 bytes");
+  if (reinterpret_cast<uintptr_t>(dev_ptr) % kAlign != 0)
+    return fail(ctx, FFSPLIT_ERR_ALIGN, "workspace must be 256-byte aligned");
+  cudaError_t e = cudaMemset(dev_ptr, 0, kStatusBytes);
+  if (e != cudaSuccess) return check_cuda(ctx, e, "cudaMemset(status block)");
+  ctx->ws = static_cast<char*>(dev_ptr);
+  ctx->ws_bytes = bytes;
+  ctx->tmaps.clear();
+  return FFSPLIT_OK;
+}
+
+ffsplit_status ffsplit_poll(ffsplit_ctx* ctx, void* stream) {
+  ffsplit_status s = check_ctx(ctx, true);
+  if (s != FFSPLIT_OK) return s;
+  cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return check_cuda(ctx, e, "cudaStreamSynchronize");
+  int words[4] = {0, 0, 0, 0};
+  e = cudaMemcpy(words, ctx->ws, sizeof(words), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return check_cuda(ctx, e, "cudaMemcpy(status block)");
+  if (words[0] == 0) return FFSPLIT_OK;
+  e = cudaMemset(ctx->ws, 0, kStatusBytes);
+  if (e != cudaSuccess) return check_cuda(ctx, e, "cudaMemset(status block)");
+  ctx->err = "device status " + std::to_string(words[0]) + " (detail " + std::to_string(words[1]) + ", kernel " +
+             std::to_string(words[2]) + ")";
+  return static_cast<ffsplit_status>(words[0]);
+}
+
+ffsplit_status ffsplit_score(ffsplit_ctx* ctx, const ffsplit_shape* shape, const ffsplit_weights* wt, const void* X,
+                             int64_t T, int32_t mode, int32_t accumulate, float* energy, float* scores, void* stream) {
+  ffsplit_status s = check_ctx(ctx, true);
+  if (s != FFSPLIT_OK) return s;
+  if ((s = check_shape(ctx, shape)) != FFSPLIT_OK) return s;
+  if (!wt || !wt->W1 || !wt->W2 || !X || !energy) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "NULL tensor");
+  if (T < 1) return fail(ctx, FFSPLIT_ERR_SHAPE, "T must be >= 1");
+  if (mode < 0 || mode > 2) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "unknown score mode");
+  const bool gated = shape->act == FFSPLIT_SWIGLU;
+  if (gated && (!wt->W1u || wt->b1)) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "SwiGLU needs W1u and no b1");
+  if (!aligned16(wt->W1) || !aligned16(wt->W2) || !aligned16(X) || (gated && !aligned16(wt->W1u)))
+    return fail(ctx, FFSPLIT_ERR_ALIGN, "tensors must be 16-byte aligned");
+  const ScoreLayout L = score_layout(*shape, T);
+  if (kStatusBytes + L.end > ctx->ws_bytes)
+    return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL, "workspace too small for this score call");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char* base = ctx->ws + kStatusBytes;
+  const int d = shape->d, m = shape->m, dt = shape->dtype;
+  // U^T (K-major for the contraction over d)
+  if ((s = launch_transpose(ctx, dt, wt->W1, m, d, m, base + L.w1t, d, d, m, nullptr, d, st)) != FFSPLIT_OK) return s;
+  if (gated && (s = launch_transpose(ctx, dt, wt->W1u, m, d, m, base + L.w1ut, d, d, m, nullptr, d, st)) != FFSPLIT_OK)
+    return s;
+  float* b1f = reinterpret_cast<float*>(base + L.b1f);
+  float* w = reinterpret_cast<float*>(base + L.w);
+  float* partial = reinterpret_cast<float*>(base + L.partial);
+  if (!gated && (s = launch_to_f32(ctx, dt, wt->b1, m, b1f, st)) != FFSPLIT_OK) return s;
+  if (scores && mode != FFSPLIT_SCORE_ACT_ONLY &&
+      (s = launch_row_energy(ctx, dt, wt->W2, m, d, w, st)) != FFSPLIT_OK)
+    return s;
+  GemmArgs g;
+  std::memset(&g, 0, sizeof(g));
+  g.A0 = X; g.lda0 = d; g.B0 = base + L.w1t; g.ldb0 = d;
+  if (gated) { g.A1 = X; g.lda1 = d; g.B1 = base + L.w1ut; g.ldb1 = d; }
+  g.M = T; g.N = m; g.K = d;
+  g.epi.col_partial = partial;
+  g.epi.n_bias = gated ? 0 : m; g.epi.bias = b1f; g.epi.n_act = m; g.epi.n_split = m;
+  g.epi.act = shape->act; g.epi.score_abs = mode == FFSPLIT_SCORE_SUM_NORM;
+  if ((s = launch_gemm(ctx, dt, g, st)) != FFSPLIT_OK) return s;
+  return launch_score_finalize(ctx, partial, L.groups, m, w, energy, scores, mode, accumulate, st);
+}
+
+ffsplit_status ffsplit_select(ffsplit_ctx* ctx, const float* scores, int32_t m, int32_t k, int32_t* heavy_idx,
+                              int32_t* light_idx, void* stream) {
+  ffsplit_status s = check_ctx(ctx, true);
+  if (s != FFSPLIT_OK) return s;
+  if (!scores) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "scores is NULL");
+  if (m < 1 || k < 0 || k > m) return fail(ctx, FFSPLIT_ERR_SHAPE, "need m >= 1 and 0 <= k <= m");
+  if (k > 0 && !heavy_idx) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "heavy_idx is NULL");
+  return launch_select(ctx, scores, m, k, heavy_idx, light_idx, static_cast<cudaStream_t>(stream));
+}
+
+ffsplit_status ffsplit_pack_size(const ffsplit_shape* shape, int32_t k, int32_t r, size_t* padded_bytes,
+                                 size_t* logical_bytes) {
+  ffsplit_status s = check_shape(nullptr, shape);
+  if (s != FFSPLIT_OK) return s;
+  if ((s = check_split(nullptr, shape, k, r)) != FFSPLIT_OK) return s;
+  BlobHeader h;
+  layout_blob(*shape, make_dims(*shape, k, r), &h);
+  if (padded_bytes) *padded_bytes = h.total_bytes;
+  if (logical_bytes) *logical_bytes = h.logical_bytes;
+  return FFSPLIT_OK;
+}
+
+ffsplit_status ffsplit_pack(ffsplit_ctx* ctx, const ffsplit_shape* shape, const ffsplit_weights* wt,
+                            const int32_t* heavy_idx, int32_t k, const ffsplit_factors* f, void* blob,
+                            size_t blob_bytes, void* stream) {
+  ffsplit_status s = check_ctx(ctx, true);
+  if (s != FFSPLIT_OK) return s;
+  if ((s = check_shape(ctx, shape)) != FFSPLIT_OK) return s;
+  const int r = f ? f->r : 0;
+  if ((s = check_split(ctx, shape, k, r)) != FFSPLIT_OK) return s;
+  if (!wt || !wt->W1 || !wt->W2 || !blob) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "NULL tensor");
+  if (k > 0 && !heavy_idx) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "heavy_idx is NULL");
+  const bool gated = shape->act == FFSPLIT_SWIGLU;
+  if (gated && (!wt->W1u || wt->b1)) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "SwiGLU needs W1u and no b1");
+  if (r > 0 && (!f->A1 || !f->B1 || !f->A2 || !f->B2 || (gated && (!f->A1u || !f->B1u))))
+    return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "NULL factor");
+  if (!aligned16(wt->W1) || !aligned16(wt->W2) || (gated && !aligned16(wt->W1u)))
+    return fail(ctx, FFSPLIT_ERR_ALIGN, "tensors must be 16-byte aligned");
+  if (reinterpret_cast<uintptr_t>(blob) % kAlign != 0) return fail(ctx, FFSPLIT_ERR_ALIGN, "blob must be 256-byte aligned");
+  const SplitDims D = make_dims(*shape, k, r);
+  BlobHeader h;
+  layout_blob(*shape, D, &h);
+  if (blob_bytes < h.total_bytes) return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL, "blob buffer too small (ffsplit_pack_size)");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char* b = static_cast<char*>(blob);
+  const int d = shape->d, m = shape->m, dt = shape->dtype;
+  const size_t es = elem_size(dt);
+  // heavy slices: U1^T = (U[:, h2])^T, V1 = V[h2, :] -- plain copies of the inputs
+  if ((s = launch_gather_cols_t(ctx, dt, wt->W1, m, d, heavy_idx, k, m, b + h.off[SEC_U1T], d, D.k_pad, st)) != FFSPLIT_OK)
+    return s;
+  if (gated &&
+      (s = launch_gather_cols_t(ctx, dt, wt->W1u, m, d, heavy_idx, k, m, b + h.off[SEC_U1UT], d, D.k_pad, st)) != FFSPLIT_OK)
+    return s;
+  if ((s = launch_transpose(ctx, dt, wt->W2, d, k, d, b + h.off[SEC_V1B2T], D.kp_rp, D.k_pad, d, heavy_idx, m, st)) !=
+      FFSPLIT_OK)
+    return s;
+  if (D.r_pad > 0) {
+    const int ml = D.ml;
+    if ((s = launch_transpose(ctx, dt, f->A1, r, d, r, b + h.off[SEC_A1T], d, d, D.r_pad, nullptr, d, st)) != FFSPLIT_OK) return s;
+    if ((s = launch_transpose(ctx, dt, f->B1, ml, r, ml, b + h.off[SEC_B1T], D.r_pad, D.r_pad, D.ml_pad, nullptr, r, st)) != FFSPLIT_OK) return s;
+    if (gated) {
+      if ((s = launch_transpose(ctx, dt, f->A1u, r, d, r, b + h.off[SEC_A1UT], d, d, D.r_pad, nullptr, d, st)) != FFSPLIT_OK) return s;
+      if ((s = launch_transpose(ctx, dt, f->B1u, ml, r, ml, b + h.off[SEC_B1UT], D.r_pad, D.r_pad, D.ml_pad, nullptr, r, st)) != FFSPLIT_OK) return s;
+    }
+    if ((s = launch_transpose(ctx, dt, f->A2, r, ml, r, b + h.off[SEC_A2T], D.ml_pad, D.ml_pad, D.r_pad, nullptr, ml, st)) != FFSPLIT_OK) return s;
+    if ((s = launch_transpose(ctx, dt, f->B2, d, r, d, b + h.off[SEC_V1B2T] + (size_t)D.k_pad * es, D.kp_rp, D.r_pad, d,
+                              nullptr, r, st)) != FFSPLIT_OK)
+      return s;
+  }
+  if ((s = launch_pack_bias(ctx, dt, wt->b1, wt->b2, heavy_idx, m, k, d, reinterpret_cast<float*>(b + h.off[SEC_B1H]),
+                            D.k_pad, reinterpret_cast<float*>(b + h.off[SEC_B1L]), D.ml_pad,
+                            reinterpret_cast<float*>(b + h.off[SEC_B2]), st)) != FFSPLIT_OK)
+    return s;
+  cudaError_t e = cudaMemcpyAsync(blob, &h, sizeof(h), cudaMemcpyHostToDevice, st);
+  if (e != cudaSuccess) return check_cuda(ctx, e, "cudaMemcpyAsync(blob header)");
+  ctx->blobs[blob] = h;
+  return FFSPLIT_OK;
+}
+
+ffsplit_status ffsplit_blob_open(ffsplit_ctx* ctx, const void* blob, size_t blob_bytes) {
+  ffsplit_status s = check_ctx(ctx, false);
+  if (s != FFSPLIT_OK) return s;
+  if (!blob) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "blob is NULL");
+  if (reinterpret_cast<uintptr_t>(blob) % kAlign != 0) return fail(ctx, FFSPLIT_ERR_ALIGN, "blob must be 256-byte aligned");
+  BlobHeader h;
+  cudaError_t e = cudaMemcpy(&h, blob, sizeof(h), cudaMemcpyDeviceToHost);
+  if (e != cudaSuccess) return check_cuda(ctx, e, "cudaMemcpy(blob header)");
+  if (!header_valid(h, blob_bytes)) return fail(ctx, FFSPLIT_ERR_BAD_BLOB, "not a packed layer (bad header)");
+  ctx->blobs[blob] = h;
+  return FFSPLIT_OK;
+}
+
+ffsplit_status ffsplit_blob_section(ffsplit_ctx* ctx, const void* blob, int32_t which, size_t* offset, int64_t* rows,
+                                    int64_t* cols, int64_t* ld) {
+  ffsplit_status s = check_ctx(ctx, false);
+  if (s != FFSPLIT_OK) return s;
+  if (which < 0 || which >= kNumSections) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "unknown section");
+  const BlobHeader* h = find_blob(ctx, blob, &s);
+  if (!h) return s;
+  const SplitDims D = dims_of(*h);
+  int64_t R = 0, C = 0, LD = 0;
+  switch (which) {
+    case SEC_U1T: R = D.k_pad; C = h->d; LD = h->d; break;
+    case SEC_U1UT: R = D.n_in == 2 ? D.k_pad : 0; C = h->d; LD = h->d; break;
+    case SEC_A1T: R = D.r_pad; C = h->d; LD = h->d; break;
+    case SEC_A1UT: R = D.n_in == 2 ? D.r_pad : 0; C = h->d; LD = h->d; break;
+    case SEC_B1T: R = D.ml_pad; C = D.r_pad; LD = D.r_pad; break;
+    case SEC_B1UT: R = D.n_in == 2 ? D.ml_pad : 0; C = D.r_pad; LD = D.r_pad; break;
+    case SEC_A2T: R = D.r_pad; C = D.ml_pad; LD = D.ml_pad; break;
+    case SEC_V1B2T: R = h->d; C = D.kp_rp; LD = D.kp_rp; break;
+    case SEC_B1H: R = 1; C = D.k_pad; LD = D.k_pad; break;
+    case SEC_B1L: R = 1; C = D.ml_pad; LD = D.ml_pad; break;
+    case SEC_B2: R = 1; C = h->d; LD = h->d; break;
+  }
+  if (offset) *offset = h->off[which];
+  if (rows) *rows = R;
+  if (cols) *cols = C;
+  if (ld) *ld = LD;
+  return FFSPLIT_OK;
+}
+
+ffsplit_status ffsplit_forward(ffsplit_ctx* ctx, const void* blob, const void* X, int64_t T, void* Y, void* stream) {
+  ffsplit_status s = check_ctx(ctx, true);
+  if (s != FFSPLIT_OK) return s;
+  if (!blob || !X || !Y) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "NULL tensor");
+  if (T < 1) return fail(ctx, FFSPLIT_ERR_SHAPE, "T must be >= 1");
+  if (!aligned16(X) || !aligned16(Y)) return fail(ctx, FFSPLIT_ERR_ALIGN, "X and Y must be 16-byte aligned");
+  const BlobHeader* h = find_blob(ctx, blob, &s);
+  if (!h) return s;
+  return run_forward(ctx, *h, static_cast<const char*>(blob), X, T, Y, static_cast<cudaStream_t>(stream));
+}
+
+ffsplit_status ffsplit_forward_host(ffsplit_ctx* ctx, const void* blob, const void* X_host, int64_t T, void* Y_host,
+                                    void* stream) {
+  ffsplit_status s = check_ctx(ctx, true);
+  if (s != FFSPLIT_OK) return s;
+  if (!blob || !X_host || !Y_host) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "NULL tensor");
+  if (T < 1) return fail(ctx, FFSPLIT_ERR_SHAPE, "T must be >= 1");
+  const BlobHeader* h = find_blob(ctx, blob, &s);
+  if (!h) return s;
+  const SplitDims D = dims_of(*h);
+  const size_t es = elem_size(h->dtype);
+  const FwdLayout L = fwd_layout(D, h->d, es, T);
+  if (kStatusBytes + L.end > ctx->ws_bytes)
+    return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL, "workspace too small for this forward (ffsplit_workspace_size)");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char* base = ctx->ws + kStatusBytes;
+  const size_t bytes = (size_t)T * h->d * es;
+  cudaError_t e = cudaMemcpyAsync(base + L.xs, X_host, bytes, cudaMemcpyHostToDevice, st);
+  if (e != cudaSuccess) return check_cuda(ctx, e, "cudaMemcpyAsync(X)");
+  if ((s = run_forward(ctx, *h, static_cast<const char*>(blob), base + L.xs, T, base + L.ys, st)) != FFSPLIT_OK) return s;
+  e = cudaMemcpyAsync(Y_host, base + L.ys, bytes, cudaMemcpyDeviceToHost, st);
+  return check_cuda(ctx, e, "cudaMemcpyAsync(Y)");
+}
+
+}  // extern "C"
