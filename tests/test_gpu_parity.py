@@ -1,0 +1,320 @@
+"""CUDA path vs the CPU oracle, element by element, on the same seeded inputs.
+Every call goes through the C ABI (ctypes).  Index outputs must be bit-exact;
+float outputs within 1e-2 relative Frobenius / 2e-2 normalised max-abs for bf16
+and 1e-5 for fp32."""
+import numpy as np
+import pytest
+import torch
+
+from conftest import f64
+from ffsplit_synth import CONFIGS, custom_config, make_layer, random_scores
+from helpers import SCORE_RTOL, GpuLayer, assert_close, oracle_factors, oracle_split
+from oracle import ffsplit_oracle as orc
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    from paper_2401_04044_b200 import Context, build
+    build.build()
+    c = Context(0)
+    c.ensure_workspace(1 << 20)
+    yield c
+    c.close()
+
+
+# ------------------------------------------------------------------ select
+@pytest.mark.parametrize("m,k,ties", [(1, 1, 0), (1, 0, 0), (7, 3, 2), (1000, 50, 0), (1024, 1024, 0), (3072, 154, 0),
+                                      (4096, 205, 5), (20480, 2048, 0), (20480, 1024, 3), (50000, 777, 40),
+                                      (1025, 0, 0), (33, 32, 1)])
+def test_select_matches_oracle_bit_exactly(ctx, m, k, ties):
+    s = random_scores(m, seed=m + k, ties=ties)
+    heavy_ref, light_ref = orc.select_heavy(s.numpy(), k)
+    sd = s.cuda()
+    heavy = torch.full((max(k, 1),), -7, dtype=torch.int32, device="cuda")
+    light = torch.full((max(m - k, 1),), -7, dtype=torch.int32, device="cuda")
+    ctx.select(sd, k, heavy, light)
+    ctx.poll()
+    assert np.array_equal(heavy[:k].cpu().numpy(), heavy_ref)
+    assert np.array_equal(light[:m - k].cpu().numpy(), light_ref)
+    # light output is optional
+    ctx.select(sd, k, heavy, None)
+    ctx.poll()
+    assert np.array_equal(heavy[:k].cpu().numpy(), heavy_ref)
+
+
+def test_select_signed_zero_and_negative_keys(ctx):
+    s = torch.tensor([0.0, -0.0, 1.0, -1.0, 0.0, 2.0, -0.0], dtype=torch.float32)
+    for k in range(8):
+        ref = orc.select_heavy(np.where(s.numpy() == 0, 0.0, s.numpy()), k)[0]
+        heavy = torch.zeros(max(k, 1), dtype=torch.int32, device="cuda")
+        ctx.select(s.cuda(), k, heavy, None)
+        ctx.poll()
+        assert np.array_equal(heavy[:k].cpu().numpy(), ref)
+
+
+def test_select_reports_non_finite_scores(ctx):
+    from paper_2401_04044_b200 import FFSplitError
+    s = torch.rand(100)
+    s[17] = float("nan")
+    heavy = torch.zeros(5, dtype=torch.int32, device="cuda")
+    ctx.select(s.cuda(), 5, heavy, None)
+    with pytest.raises(FFSplitError) as e:
+        ctx.poll()
+    assert e.value.code == 6
+    ctx.poll()   # the status word was cleared
+
+
+# ------------------------------------------------------------------ score
+SCORE_CASES = [
+    ("f32", "gelu_erf", 64, 200, 100),
+    ("f32", "swiglu", 40, 130, 70),
+    ("f32", "gelu_tanh", 33, 65, 64),
+    ("bf16", "gelu_erf", 72, 300, 200),
+    ("bf16", "swiglu", 128, 520, 300),
+    ("bf16", "gelu_tanh", 64, 256, 129),
+]
+
+
+@pytest.mark.parametrize("dt,act,d,m,T", SCORE_CASES)
+@pytest.mark.parametrize("mode", [0, 1, 2])
+def test_score_matches_oracle(ctx, dt, act, d, m, T, mode):
+    cfg = custom_config(d, m, max(1, m // 20), 16, act=act, dtype=dt)
+    L = make_layer(cfg, 0)
+    G = GpuLayer(ctx, L)
+    G.reserve(0, T, 0, 0)
+    X = L.tokens(T)
+    energy, scores = G.score(X, mode=mode)
+    e_ref, w_ref, s_ref = orc.neuron_scores(f64(X), f64(L.W1), f64(L.b1), f64(L.W2), act,
+                                            [orc.SCORE_EQ3, orc.SCORE_ACT_ONLY, orc.SCORE_SUM_NORM][mode], f64(L.W1u))
+    rt = SCORE_RTOL[dt]
+    assert np.allclose(f64(energy), e_ref, rtol=rt, atol=rt * e_ref.max() * 1e-3)
+    assert np.allclose(f64(scores), s_ref, rtol=rt, atol=rt * s_ref.max() * 1e-3)
+    # accumulation over calibration batches gives the same totals; identical calls are bitwise equal
+    energy2, scores2 = G.score(X, mode=mode, batches=3)
+    assert np.allclose(f64(scores2), s_ref, rtol=rt, atol=rt * s_ref.max() * 1e-3)
+    energy3, scores3 = G.score(X, mode=mode)
+    assert torch.equal(scores, scores3) and torch.equal(energy, energy3)
+
+
+@pytest.mark.parametrize("dt,act", [("f32", "gelu_erf"), ("bf16", "gelu_erf"), ("bf16", "swiglu")])
+def test_planted_heavy_hitters_recovered_end_to_end(ctx, dt, act):
+    cfg = custom_config(128, 640, 32, 16, act=act, dtype=dt)
+    L = make_layer(cfg, 1)
+    G = GpuLayer(ctx, L)
+    G.reserve(0, 384, 0, 0)
+    X = L.tokens(384)
+    _, scores = G.score(X)
+    heavy, light = G.select(scores, cfg.k)
+    _, _, s_ref = orc.neuron_scores(f64(X), f64(L.W1), f64(L.b1), f64(L.W2), act, orc.SCORE_EQ3, f64(L.W1u))
+    heavy_ref, light_ref = orc.select_heavy(s_ref, cfg.k)
+    assert np.array_equal(heavy.cpu().numpy(), heavy_ref) and np.array_equal(light.cpu().numpy(), light_ref)
+    assert np.array_equal(heavy_ref, L.planted.numpy())
+
+
+# ------------------------------------------------------------------ pack
+@pytest.mark.parametrize("dt,act", [("f32", "gelu_erf"), ("bf16", "gelu_erf"), ("bf16", "swiglu"), ("f32", "swiglu")])
+def test_pack_heavy_slices_are_bit_exact_gathers(ctx, dt, act):
+    from paper_2401_04044_b200 import read_section
+    cfg = custom_config(72, 300, 37, 24, act=act, dtype=dt)
+    L = make_layer(cfg, 2)
+    G = GpuLayer(ctx, L)
+    G.reserve(8, 0, cfg.k, cfg.r)
+    heavy = torch.sort(torch.randperm(cfg.m, generator=torch.Generator().manual_seed(5))[:cfg.k]).values
+    fac = oracle_factors(L, heavy.numpy(), cfg.r)
+    blob, logical = G.pack(heavy, fac)
+    tdt = cfg.torch_dtype
+    sw = orc.split_weights(f64(L.W1), f64(L.b1), f64(L.W2), heavy.numpy(), f64(L.W1u))
+    k, r, ml = cfg.k, cfg.r, cfg.m - cfg.k
+    U1T = read_section(ctx, blob, 0, tdt)
+    assert np.array_equal(f64(U1T[:k]), sw["U1"].T) and not U1T[k:].any()
+    V1B2T = read_section(ctx, blob, 7, tdt)
+    kp = U1T.shape[0]
+    assert np.array_equal(f64(V1B2T[:, :k]), sw["V1"].T) and not V1B2T[:, k:kp].any()
+    assert np.array_equal(f64(V1B2T[:, kp:kp + r]), f64(fac["B2"]).T) and not V1B2T[:, kp + r:].any()
+    A1T = read_section(ctx, blob, 2, tdt)
+    assert np.array_equal(f64(A1T[:r]), f64(fac["A1"]).T) and not A1T[r:].any()
+    B1T = read_section(ctx, blob, 4, tdt)
+    assert np.array_equal(f64(B1T[:ml, :r]), f64(fac["B1"]).T) and not B1T[ml:].any() and not B1T[:, r:].any()
+    A2T = read_section(ctx, blob, 6, tdt)
+    assert np.array_equal(f64(A2T[:r, :ml]), f64(fac["A2"]).T) and not A2T[r:].any() and not A2T[:, ml:].any()
+    if act == "swiglu":
+        assert np.array_equal(f64(read_section(ctx, blob, 1, tdt)[:k]), sw["U1u"].T)
+        assert np.array_equal(f64(read_section(ctx, blob, 3, tdt)[:r]), f64(fac["A1u"]).T)
+        assert np.array_equal(f64(read_section(ctx, blob, 5, tdt)[:ml, :r]), f64(fac["B1u"]).T)
+    else:
+        assert np.array_equal(f64(read_section(ctx, blob, 8, torch.float32)[0, :k]), sw["b1_heavy"])
+        assert np.array_equal(f64(read_section(ctx, blob, 9, torch.float32)[0, :ml]), sw["b1_light"])
+        assert np.array_equal(f64(read_section(ctx, blob, 10, torch.float32)[0]), f64(L.b2))
+    n_in = 2 if act == "swiglu" else 1
+    es = 4 if dt == "f32" else 2
+    assert logical == es * (orc.split_weight_params(cfg.d, cfg.m, k, r, n_in) + cfg.m + cfg.d)
+    # a copied blob is accepted after registration and gives the same output
+    X = L.tokens(8)
+    Y = G.forward(blob, X)
+    blob2 = blob.clone()
+    ctx.blob_open(blob2)
+    assert torch.equal(G.forward(blob2, X), Y)
+
+
+def test_pack_rejects_unsorted_indices_and_garbage_blobs(ctx):
+    from paper_2401_04044_b200 import FFSplitError
+    cfg = custom_config(64, 128, 4, 0, dtype="f32")
+    L = make_layer(cfg, 0)
+    G = GpuLayer(ctx, L)
+    G.reserve(8, 0, 4, 0)
+    with pytest.raises(FFSplitError) as e:
+        G.pack(torch.tensor([5, 3, 9, 200], dtype=torch.int32), None)
+    assert e.value.code == 11
+    junk = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    with pytest.raises(FFSplitError) as e:
+        ctx.blob_open(junk)
+    assert e.value.code == 7
+
+
+# ------------------------------------------------------------------ forward
+FWD_CASES = [
+    # dtype, act, d, m, k, r, T
+    ("f32", "gelu_erf", 64, 256, 16, 16, 50),
+    ("f32", "gelu_erf", 60, 250, 13, 7, 129),        # nothing a multiple of anything
+    ("f32", "swiglu", 48, 200, 10, 12, 70),
+    ("f32", "gelu_tanh", 64, 256, 16, 16, 64),
+    ("bf16", "gelu_erf", 64, 256, 16, 16, 128),
+    ("bf16", "gelu_erf", 72, 300, 37, 24, 200),      # ragged K tail, ragged tiles
+    ("bf16", "gelu_erf", 256, 1024, 100, 64, 700),   # several tiles in every stage
+    ("bf16", "gelu_tanh", 128, 512, 26, 32, 130),
+    ("bf16", "swiglu", 72, 300, 37, 24, 200),
+    ("bf16", "swiglu", 256, 1000, 50, 64, 513),
+    ("bf16", "gelu_erf", 128, 512, 26, 32, 1),       # single token
+    ("bf16", "gelu_erf", 128, 512, 26, 32, 16),
+    ("bf16", "swiglu", 128, 512, 26, 32, 4),
+]
+
+
+@pytest.mark.parametrize("dt,act,d,m,k,r,T", FWD_CASES)
+def test_split_forward_matches_oracle(ctx, dt, act, d, m, k, r, T):
+    cfg = custom_config(d, m, k, r, act=act, dtype=dt)
+    L = make_layer(cfg, 3)
+    G = GpuLayer(ctx, L)
+    G.reserve(T, 0, k, r)
+    heavy = L.planted
+    fac = oracle_factors(L, heavy.numpy(), r)
+    blob, _ = G.pack(heavy, fac)
+    X = L.tokens(T)
+    Y = G.forward(blob, X)
+    Yref = oracle_split(L, heavy.numpy(), fac, X)
+    assert_close(Y, Yref, dt, "split forward")
+    assert torch.equal(G.forward(blob, X), Y), "forward is not bitwise reproducible"
+
+
+@pytest.mark.parametrize("dt,act", [("f32", "gelu_erf"), ("bf16", "gelu_erf"), ("bf16", "swiglu"), ("f32", "swiglu")])
+def test_degenerate_splits(ctx, dt, act):
+    """k = m is the dense FFN; k = 0 is plain low-rank; r = 0 keeps FFN_1 only;
+    full-rank light factors give back the dense FFN."""
+    cfg = custom_config(64, 192, 20, 16, act=act, dtype=dt)
+    L = make_layer(cfg, 4)
+    G = GpuLayer(ctx, L)
+    T = 150
+    for kk, rr in [(cfg.m, 0), (0, 16), (20, 0), (20, 64)]:
+        G.reserve(T, 0, kk, rr)
+    X = L.tokens(T)
+    dense_ref = orc.dense_ffn(f64(X), f64(L.W1), f64(L.b1), f64(L.W2), f64(L.b2), act, f64(L.W1u))
+    # k = m
+    blob, _ = G.pack(torch.arange(cfg.m), None)
+    Yd = G.forward(blob, X)
+    assert_close(Yd, dense_ref, dt, "k = m")
+    # k = 0, rank r
+    none = torch.arange(0)
+    fac = oracle_factors(L, none.numpy(), 16)
+    blob, _ = G.pack(none, fac)
+    assert_close(G.forward(blob, X), oracle_split(L, none.numpy(), fac, X), dt, "k = 0")
+    # r = 0 with k < m
+    blob, _ = G.pack(L.planted, None)
+    fac0 = {n: (v[:, :0] if n.startswith("A") else v[:0, :]) for n, v in fac.items()}
+    assert_close(G.forward(blob, X), oracle_split(L, L.planted.numpy(), fac0, X), dt, "r = 0")
+    # full-rank light factors reproduce the dense FFN (up to the factors' own rounding)
+    fac = oracle_factors(L, L.planted.numpy(), 64)
+    blob, _ = G.pack(L.planted, fac)
+    Yf = G.forward(blob, X)
+    assert_close(Yf, oracle_split(L, L.planted.numpy(), fac, X), dt, "full rank vs oracle split")
+    loose = 3e-2 if dt == "bf16" else 1e-4
+    assert orc.rel_frobenius(f64(Yf), dense_ref) < loose
+
+
+def test_output_invariant_under_neuron_permutation(ctx):
+    cfg = custom_config(64, 256, 16, 0, dtype="f32")
+    L = make_layer(cfg, 5)
+    G = GpuLayer(ctx, L)
+    G.reserve(64, 0, 256, 0)
+    X = L.tokens(64)
+    blob, _ = G.pack(torch.arange(cfg.m), None)
+    Y = G.forward(blob, X)
+    perm = torch.randperm(cfg.m, generator=torch.Generator().manual_seed(1))
+    L2 = make_layer(cfg, 5)
+    L2.W1, L2.b1, L2.W2 = L.W1[:, perm].contiguous(), L.b1[perm].contiguous(), L.W2[perm, :].contiguous()
+    G2 = GpuLayer(ctx, L2)
+    blob2, _ = G2.pack(torch.arange(cfg.m), None)
+    Y2 = G2.forward(blob2, X)
+    assert orc.rel_frobenius(f64(Y2), f64(Y)) < 1e-5
+
+
+def test_forward_from_host_buffers(ctx):
+    cfg = custom_config(128, 512, 26, 32, dtype="bf16")
+    L = make_layer(cfg, 6)
+    G = GpuLayer(ctx, L)
+    G.reserve(300, 0, cfg.k, cfg.r)
+    fac = oracle_factors(L, L.planted.numpy(), cfg.r)
+    blob, _ = G.pack(L.planted, fac)
+    X = L.tokens(300)
+    Y = G.forward(blob, X)
+    Xh = X.pin_memory()
+    Yh = torch.empty_like(Xh).pin_memory()
+    ctx.forward_host(blob, Xh, Yh)
+    ctx.poll()
+    assert torch.equal(Yh, Y.cpu())
+
+
+# ------------------------------------------------------------------ the paper-shaped configs
+def test_config1_fp32_end_to_end(ctx):
+    cfg = CONFIGS[1]
+    L = make_layer(cfg, 0)
+    G = GpuLayer(ctx, L)
+    G.reserve(128, cfg.t_cal, cfg.k, cfg.r)
+    Xc = L.tokens(cfg.t_cal)
+    _, scores = G.score(Xc)
+    heavy, light = G.select(scores, cfg.k)
+    _, _, s_ref = orc.neuron_scores(f64(Xc), f64(L.W1), f64(L.b1), f64(L.W2), cfg.act)
+    heavy_ref, light_ref = orc.select_heavy(s_ref, cfg.k)
+    assert np.array_equal(heavy.cpu().numpy(), heavy_ref) and np.array_equal(light.cpu().numpy(), light_ref)
+    assert np.array_equal(heavy_ref, L.planted.numpy())
+    assert np.allclose(f64(scores), s_ref, rtol=1e-4)
+    fac = oracle_factors(L, heavy_ref, cfg.r)
+    blob, _ = G.pack(heavy, fac)
+    X = L.tokens(128)
+    assert_close(G.forward(blob, X), oracle_split(L, heavy_ref, fac, X), "f32", "config 1")
+
+
+@pytest.mark.parametrize("cid,layer,T", [(2, 0, 4096), (2, 11, 4096), (3, 0, 64), (3, 5, 200)])
+def test_bf16_configs_one_layer_end_to_end(ctx, cid, layer, T):
+    cfg = CONFIGS[cid]
+    L = make_layer(cfg, layer)
+    G = GpuLayer(ctx, L)
+    G.reserve(T, cfg.t_cal, cfg.k, cfg.r)
+    G.reserve(T, 0, cfg.m, 0)
+    Xc = L.tokens(cfg.t_cal)
+    _, scores = G.score(Xc, batches=2)
+    heavy, light = G.select(scores, cfg.k)
+    _, _, s_ref = orc.neuron_scores(f64(Xc), f64(L.W1), f64(L.b1), f64(L.W2), cfg.act)
+    heavy_ref, light_ref = orc.select_heavy(s_ref, cfg.k)
+    assert np.array_equal(heavy.cpu().numpy(), heavy_ref) and np.array_equal(light.cpu().numpy(), light_ref)
+    assert np.array_equal(heavy_ref, L.planted.numpy())
+    assert np.allclose(f64(scores), s_ref, rtol=2e-3)
+    fac = oracle_factors(L, heavy_ref, cfg.r)
+    blob, _ = G.pack(heavy, fac)
+    X = L.tokens(T)
+    assert_close(G.forward(blob, X), oracle_split(L, heavy_ref, fac, X), "bf16", f"config {cid}")
+    # dense comparator through the same kernels
+    blobd, _ = G.pack(torch.arange(cfg.m), None)
+    dense_ref = orc.dense_ffn(f64(X), f64(L.W1), f64(L.b1), f64(L.W2), f64(L.b2), cfg.act)
+    assert_close(G.forward(blobd, X), dense_ref, "bf16", f"config {cid} dense")
