@@ -52,7 +52,7 @@ class GpuLayer:
         Xd = to_dev(X)
         chunks = torch.chunk(Xd, batches, dim=0)
         for i, xc in enumerate(chunks):
-            xc = xc.contiguous()
+            xc = xc.clone()      # own allocation: chunk views of an odd-width X are not 16-byte aligned
             self.ctx.score(self.shape, self.W1, self.b1, self.W2, xc, energy,
                            scores if i == len(chunks) - 1 else None, mode=mode, accumulate=i > 0, W1u=self.W1u)
         self.ctx.poll()
