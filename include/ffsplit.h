@@ -184,6 +184,18 @@ ffsplit_status ffsplit_forward_host(ffsplit_ctx* ctx, const void* blob, const vo
  * (FFSPLIT_OK if no kernel recorded a condition). */
 ffsplit_status ffsplit_poll(ffsplit_ctx* ctx, void* stream);
 
+/* Per-launch device timing of the library's main kernels, for roofline reports.
+ * Between ffsplit_profile_begin() and ffsplit_profile_end() every launch of a
+ * kernel class is bracketed by CUDA events on its stream.  profile_end
+ * synchronises `stream` and returns, for `kernel_class` (0 tensor-core GEMM,
+ * 1 fp32 GEMM, 2 few-token streaming forward): the number of launches, the sum
+ * of their durations in milliseconds and the sum of their algorithmic work
+ * (FLOPs for the GEMMs, bytes for the streaming kernel; unpadded sizes).
+ * Profiling adds event overhead between kernels: never time a step with it on. */
+ffsplit_status ffsplit_profile_begin(ffsplit_ctx* ctx);
+ffsplit_status ffsplit_profile_end(ffsplit_ctx* ctx, void* stream, int32_t kernel_class, int32_t* launches,
+                                   double* total_ms, double* total_work);
+
 /* Number of kernels this context has launched so far. */
 int64_t ffsplit_launch_count(const ffsplit_ctx* ctx);
 

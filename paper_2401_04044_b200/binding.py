@@ -32,7 +32,7 @@ EXPORTS = [
     "ffsplit_create", "ffsplit_destroy", "ffsplit_workspace_size", "ffsplit_set_workspace", "ffsplit_score",
     "ffsplit_select", "ffsplit_pack_size", "ffsplit_pack", "ffsplit_blob_open", "ffsplit_blob_section",
     "ffsplit_forward", "ffsplit_forward_host", "ffsplit_poll", "ffsplit_launch_count", "ffsplit_last_error",
-    "ffsplit_version",
+    "ffsplit_version", "ffsplit_profile_begin", "ffsplit_profile_end",
 ]
 
 
@@ -83,6 +83,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.ffsplit_forward.argtypes = [vp, vp, vp, i64, vp, vp]
     lib.ffsplit_forward_host.argtypes = [vp, vp, vp, i64, vp, vp]
     lib.ffsplit_poll.argtypes = [vp, vp]
+    lib.ffsplit_profile_begin.argtypes = [vp]
+    lib.ffsplit_profile_end.argtypes = [vp, vp, i32, P(i32), P(C.c_double), P(C.c_double)]
     lib.ffsplit_launch_count.argtypes = [vp]
     lib.ffsplit_launch_count.restype = i64
     lib.ffsplit_last_error.argtypes = [vp]
@@ -209,6 +211,16 @@ class Context:
 
     def poll(self, stream=None):
         self._check(self.lib.ffsplit_poll(self.h, _stream_ptr(stream)), "ffsplit_poll")
+
+    def profile_begin(self):
+        self._check(self.lib.ffsplit_profile_begin(self.h), "ffsplit_profile_begin")
+
+    def profile_end(self, kernel_class: int = 0, stream=None):
+        """-> (launches, total milliseconds, total algorithmic work) of one kernel class."""
+        n, ms, work = C.c_int32(), C.c_double(), C.c_double()
+        self._check(self.lib.ffsplit_profile_end(self.h, _stream_ptr(stream), kernel_class, C.byref(n), C.byref(ms),
+                                                 C.byref(work)), "ffsplit_profile_end")
+        return n.value, ms.value, work.value
 
     def launch_count(self) -> int:
         return int(self.lib.ffsplit_launch_count(self.h))

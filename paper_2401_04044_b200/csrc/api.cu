@@ -19,6 +19,22 @@ ffsplit_status check_cuda(ffsplit_ctx* ctx, cudaError_t e, const char* what) {
   return FFSPLIT_ERR_CUDA;
 }
 
+int prof_open(ffsplit_ctx* ctx, int cls, double work, cudaStream_t st) {
+  if (!ctx->profiling) return -1;
+  ffsplit_ctx::ProfRec r;
+  r.cls = cls;
+  r.work = work;
+  if (cudaEventCreate(&r.a) != cudaSuccess) return -1;
+  if (cudaEventCreate(&r.b) != cudaSuccess) { cudaEventDestroy(r.a); return -1; }
+  cudaEventRecord(r.a, st);
+  ctx->prof.push_back(r);
+  return static_cast<int>(ctx->prof.size()) - 1;
+}
+
+void prof_close(ffsplit_ctx* ctx, int handle, cudaStream_t st) {
+  if (handle >= 0) cudaEventRecord(ctx->prof[handle].b, st);
+}
+
 ffsplit_status launch_decode_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* blob, const void* X,
                                      long long T, void* Y, char* ws_after_status, cudaStream_t st);
 bool decode_path_applies(const ffsplit_ctx* ctx, const BlobHeader& h, long long T);
@@ -187,6 +203,7 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
     g.A0 = X; g.lda0 = d;
     g.B0 = blob + h.off[SEC_U1T]; g.ldb0 = d;
     g.M = T; g.N = D.kp_rp; g.K = d;
+    g.algo_flops = 2.0 * T * d * (D.k + D.r);
     g.epi.C0 = AP; g.epi.ld0 = D.kp_rp;
     g.epi.C1 = Q; g.epi.ld1 = D.r_pad;
     g.epi.n_split = D.k_pad; g.epi.n_act = D.k_pad; g.epi.n_bias = D.k_pad;
@@ -197,6 +214,7 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
     g.A0 = X; g.lda0 = d; g.B0 = blob + h.off[SEC_U1T]; g.ldb0 = d;
     g.A1 = X; g.lda1 = d; g.B1 = blob + h.off[SEC_U1UT]; g.ldb1 = d;
     g.M = T; g.N = D.k_pad; g.K = d;
+    g.algo_flops = 4.0 * T * d * D.k;
     g.epi.C0 = AP; g.epi.ld0 = D.kp_rp;
     g.epi.n_split = D.k_pad; g.epi.n_act = D.k_pad; g.epi.act = h.act;
     if ((s = launch_gemm(ctx, h.dtype, g, st)) != FFSPLIT_OK) return s;
@@ -204,6 +222,7 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
       std::memset(&g, 0, sizeof(g));
       g.A0 = X; g.lda0 = d; g.B0 = blob + h.off[SEC_A1T]; g.ldb0 = d;  // [A1 | A1u]^T
       g.M = T; g.N = 2 * D.r_pad; g.K = d;
+      g.algo_flops = 4.0 * T * d * D.r;
       g.epi.C0 = Q; g.epi.ld0 = 2 * D.r_pad; g.epi.n_split = g.N; g.epi.act = h.act;
       if ((s = launch_gemm(ctx, h.dtype, g, st)) != FFSPLIT_OK) return s;
     }
@@ -218,6 +237,7 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
       g.B1 = blob + h.off[SEC_B1UT]; g.ldb1 = D.r_pad;
     }
     g.M = T; g.N = D.ml_pad; g.K = D.r_pad;
+    g.algo_flops = 2.0 * D.n_in * T * D.r * D.ml;
     g.epi.C0 = HL; g.epi.ld0 = D.ml_pad;
     g.epi.n_split = g.N; g.epi.n_act = g.N; g.epi.n_bias = gated ? 0 : g.N;
     g.epi.bias = b1l; g.epi.act = h.act;
@@ -227,6 +247,7 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
     g.A0 = HL; g.lda0 = D.ml_pad;
     g.B0 = blob + h.off[SEC_A2T]; g.ldb0 = D.ml_pad;
     g.M = T; g.N = D.r_pad; g.K = D.ml_pad;
+    g.algo_flops = 2.0 * T * D.r * D.ml;
     g.epi.C0 = AP + (size_t)D.k_pad * es; g.epi.ld0 = D.kp_rp;
     g.epi.n_split = g.N; g.epi.act = h.act;
     if ((s = launch_gemm(ctx, h.dtype, g, st)) != FFSPLIT_OK) return s;
@@ -236,6 +257,7 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
   g.A0 = AP; g.lda0 = D.kp_rp;
   g.B0 = blob + h.off[SEC_V1B2T]; g.ldb0 = D.kp_rp;
   g.M = T; g.N = d; g.K = light ? D.kp_rp : D.k_pad;
+  g.algo_flops = 2.0 * T * d * (D.k + (light ? D.r : 0));
   g.epi.C0 = Y; g.epi.ld0 = d;
   g.epi.n_split = d; g.epi.n_bias = d; g.epi.bias = b2; g.epi.act = h.act;
   return launch_gemm(ctx, h.dtype, g, st);
@@ -251,6 +273,38 @@ int32_t ffsplit_version(void) { return 100; }
 
 const char* ffsplit_last_error(const ffsplit_ctx* ctx) {
   return ctx ? ctx->err.c_str() : "no context";
+}
+
+ffsplit_status ffsplit_profile_begin(ffsplit_ctx* ctx) {
+  ffsplit_status s = check_ctx(ctx, false);
+  if (s != FFSPLIT_OK) return s;
+  for (auto& r : ctx->prof) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
+  ctx->prof.clear();
+  ctx->profiling = true;
+  return FFSPLIT_OK;
+}
+
+ffsplit_status ffsplit_profile_end(ffsplit_ctx* ctx, void* stream, int32_t kernel_class, int32_t* launches,
+                                   double* total_ms, double* total_work) {
+  ffsplit_status s = check_ctx(ctx, false);
+  if (s != FFSPLIT_OK) return s;
+  ctx->profiling = false;
+  cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
+  if (e != cudaSuccess) return check_cuda(ctx, e, "cudaStreamSynchronize");
+  int n = 0;
+  double ms = 0.0, work = 0.0;
+  for (auto& r : ctx->prof) {
+    if (r.cls != kernel_class) continue;
+    float t = 0.f;
+    if (cudaEventSynchronize(r.b) == cudaSuccess && cudaEventElapsedTime(&t, r.a, r.b) == cudaSuccess) {
+      ++n; ms += t; work += r.work;
+    }
+  }
+  cudaGetLastError();
+  if (launches) *launches = n;
+  if (total_ms) *total_ms = ms;
+  if (total_work) *total_work = work;
+  return FFSPLIT_OK;
 }
 
 int64_t ffsplit_launch_count(const ffsplit_ctx* ctx) { return ctx ? ctx->launches : 0; }
@@ -279,6 +333,7 @@ ffsplit_status ffsplit_create(ffsplit_ctx** out, int device) {
 }
 
 ffsplit_status ffsplit_destroy(ffsplit_ctx* ctx) {
+  if (ctx) for (auto& r : ctx->prof) { cudaEventDestroy(r.a); cudaEventDestroy(r.b); }
   delete ctx;
   return FFSPLIT_OK;
 }
@@ -371,6 +426,7 @@ ffsplit_status ffsplit_score(ffsplit_ctx* ctx, const ffsplit_shape* shape, const
   g.A0 = X; g.lda0 = d; g.B0 = base + L.w1t; g.ldb0 = d;
   if (gated) { g.A1 = X; g.lda1 = d; g.B1 = base + L.w1ut; g.ldb1 = d; }
   g.M = T; g.N = m; g.K = d;
+  g.algo_flops = 2.0 * (gated ? 2 : 1) * T * (double)d * m;
   g.epi.col_partial = partial;
   g.epi.n_bias = gated ? 0 : m; g.epi.bias = b1f; g.epi.n_act = m; g.epi.n_split = m;
   g.epi.act = shape->act; g.epi.score_abs = mode == FFSPLIT_SCORE_SUM_NORM;

@@ -143,8 +143,10 @@ ffsplit_status launch_gemm_simt(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_
   const long long tiles_m = (g.M + simt::TM - 1) / simt::TM;
   if (tiles_m > 65535) return fail(ctx, FFSPLIT_ERR_SHAPE, "fp32 path: more than 65535*64 rows in one call");
   dim3 grid((g.N + simt::TN - 1) / simt::TN, static_cast<unsigned>(tiles_m));
+  const int ph = prof_open(ctx, PROF_GEMM_SIMT, g.algo_flops, st);
   if (g.A1) simt::gemm_simt_kernel<true><<<grid, 256, 0, st>>>(p);
   else simt::gemm_simt_kernel<false><<<grid, 256, 0, st>>>(p);
+  prof_close(ctx, ph, st);
   ctx->launches++;
   return check_cuda(ctx, cudaGetLastError(), "gemm_simt_kernel launch");
 }

@@ -381,7 +381,9 @@ ffsplit_status launch_gemm_tc(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_t 
   }
   const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n;
   const int grid = static_cast<int>(tiles < ctx->num_sms ? tiles : ctx->num_sms);
+  const int ph = prof_open(ctx, PROF_GEMM_TC, g.algo_flops, st);
   tc::gemm_tc_kernel<<<grid, tc::NUM_THREADS, tc::SMEM_BYTES, st>>>(tA0, tB0, tA1, tB1, p);
+  prof_close(ctx, ph, st);
   ctx->launches++;
   return check_cuda(ctx, cudaGetLastError(), "gemm_tc_kernel launch");
 }

@@ -69,6 +69,7 @@ struct GemmArgs {
   long long M;
   int N;
   int K;
+  double algo_flops;  // unpadded FLOPs of this product, for profiling reports
   Epilogue epi;
 };
 
@@ -128,6 +129,9 @@ struct ffsplit_ctx {
   std::unordered_map<const void*, ffsp::BlobHeader> blobs;
   std::unordered_map<ffsp::TmapKey, CUtensorMap, ffsp::TmapKeyHash> tmaps;
   void* encode_fn = nullptr;  // cuTensorMapEncodeTiled
+  struct ProfRec { int cls; cudaEvent_t a, b; double work; };
+  bool profiling = false;
+  std::vector<ProfRec> prof;
   bool attr_tc_set = false;
   bool attr_fused_set = false;
   int* status() const { return reinterpret_cast<int*>(ws); }
@@ -142,6 +146,11 @@ inline int round_up(int v, int q) { return (v + q - 1) / q * q; }
 inline long long round_up_ll(long long v, long long q) { return (v + q - 1) / q * q; }
 inline size_t elem_size(int dtype) { return dtype == FFSPLIT_BF16 ? 2 : 4; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Profiling brackets: no-ops unless ffsplit_profile_begin() is active.
+enum ProfClass : int { PROF_GEMM_TC = 0, PROF_GEMM_SIMT = 1, PROF_DECODE = 2 };
+int prof_open(ffsplit_ctx* ctx, int cls, double work, cudaStream_t st);
+void prof_close(ffsplit_ctx* ctx, int handle, cudaStream_t st);
 
 // launchers (each returns a CUDA error state through check_cuda)
 ffsplit_status launch_gemm(ffsplit_ctx* ctx, int dtype, const GemmArgs& g, cudaStream_t st);
