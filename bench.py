@@ -216,11 +216,23 @@ def run_ours(args):
     cfg = CONFIGS[CFG_ID]
     T = cfg.t_fwd[0]
     ctx = Context(local_rank)
-    wl = StackWorkload(cfg, ctx, cfg.layers, T, device)
+    n_layers = args.layers or cfg.layers
+    wl = StackWorkload(cfg, ctx, n_layers, T, device)
     flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=device)
 
     def flush():
         flush_buf.add_(1)
+
+    if args.only:
+        # one phase alone, few launches: the form used under a profiler
+        wl.calibrate()
+        fn = {"step": wl.step, "forward": wl.forward, "dense": lambda: wl.forward(dense=True),
+              "calibrate": wl.calibrate}[args.only]
+        ms = time_region(fn, args.steps, args.warmup, flush, barrier)
+        ctx.poll()
+        if rank == 0:
+            print(json.dumps({"only": args.only, "layers": n_layers, "tokens": T, "ms_per_call": ms}))
+        return
 
     sampler = ClockSampler(local_rank) if rank == 0 else None
     n0 = ctx.launch_count()
@@ -431,8 +443,12 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--only", default=None, choices=["step", "forward", "dense", "calibrate"],
+                    help="run one phase alone and print its times (for profiler captures)")
+    ap.add_argument("--layers", type=int, default=0, help="with --only: number of layers of the stack to build")
     args = ap.parse_args()
-    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "ours" and not args.only:
+        args.warmup = max(args.warmup, 3)
     if args.impl == "reference":
         run_reference(args)
     else:
