@@ -17,6 +17,35 @@ __device__ __forceinline__ float gelu_tanh_f(float z) {
 __device__ __forceinline__ float silu_f(float z) { return z / (1.0f + __expf(-z)); }
 __device__ __forceinline__ float silu_precise_f(float z) { return z / (1.0f + expf(-z)); }
 
+// Fast GELU for bf16 outputs: x * Phi(x) ~ 0.5 x (1 + tanh(x (c0 + c1 x^2 + c2 x^4))) with one
+// MUFU tanh.  For the erf definition (c0, c1, c2) are a minimax fit of atanh(erf(x / sqrt 2)) / x
+// (max abs error of the fit 2.6e-5 with an exact tanh); for the tanh definition they are the
+// definition's own constants.  x^2 is clamped at 36: beyond |x| = 6, Phi is 0 or 1 to 1e-9 and
+// the clamp keeps the fitted polynomial positive.  tanh.approx.f32 adds up to 2^-11 relative.
+struct GeluCoef { float c0, c1, c2; };
+__device__ __forceinline__ GeluCoef gelu_coef(int act) {
+  GeluCoef c;
+  if (act == FFSPLIT_GELU_TANH) { c.c0 = 0.79788456080286536f; c.c1 = 0.035677408136300125f; c.c2 = 0.0f; }
+  else { c.c0 = 7.97507884e-01f; c.c1 = 3.70056460e-02f; c.c2 = -3.51516789e-04f; }
+  return c;
+}
+__device__ __forceinline__ float tanh_approx(float u) {
+  float t;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(u));
+  return t;
+}
+__device__ __forceinline__ float gelu_fast(float x, const GeluCoef& c) {
+  const float x2 = fminf(x * x, 36.0f);
+  const float u = x * fmaf(fmaf(c.c2, x2, c.c1), x2, c.c0);
+  const float hx = 0.5f * x;
+  return fmaf(hx, tanh_approx(u), hx);
+}
+// SiLU with one MUFU: x * sigmoid(x) = 0.5 x (1 + tanh(x / 2)).
+__device__ __forceinline__ float silu_fast(float x) {
+  const float hx = 0.5f * x;
+  return fmaf(hx, tanh_approx(hx), hx);
+}
+
 // GELU variants by runtime switch (uniform across the grid).
 __device__ __forceinline__ float act_gelu(float z, int act) {
   return act == FFSPLIT_GELU_TANH ? gelu_tanh_f(z) : gelu_erf_f(z);

@@ -6,7 +6,8 @@
 //   warp 0  (one lane)  TMA producer: global -> 128B-swizzled shared tiles, 4-stage ring
 //   warp 1  (one lane)  tcgen05.mma issuer; accumulators live in tensor memory (TMEM),
 //                       two buffers so the epilogue of tile i overlaps the MMAs of tile i+1
-//   warps 2-5           epilogue: tcgen05.ld -> bias / activation / gating -> global
+//   warps 2-9           epilogue: tcgen05.ld -> bias / activation / gating -> global; two warps
+//                       per TMEM lane quarter, taking alternate 16-column chunks
 // The gated form (SwiGLU) runs two operand pairs into two accumulators of the same
 // tile and combines them as silu(acc0) * acc1.
 // The score form does not store the tile; it reduces act(acc)^2 over the tile's rows
@@ -31,7 +32,8 @@ constexpr int B_STAGE_BYTES = MAX_BLOCK_N * BLOCK_K * 2;
 constexpr int TMEM_COLS = 512;
 constexpr int ACC_STRIDE = 256;   // TMEM columns per accumulator buffer
 constexpr int GATE_OFFSET = 128;  // second accumulator of a gated tile
-constexpr int NUM_THREADS = 192;
+constexpr int NUM_THREADS = 320;
+constexpr int EPI_WARPS = 8;
 constexpr int BAR_BYTES = 256;
 constexpr int SMEM_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + BAR_BYTES + 1024;
 
@@ -47,15 +49,28 @@ struct Params {
 
 // Bias, activation and store of 16 consecutive columns of one row.  n_act, n_bias
 // and n_split are multiples of 16 (or >= N), so the branches are uniform per chunk.
-__device__ __forceinline__ void epilogue_chunk_store(const Params& p, long long row, int n0, float* v) {
-  const Epilogue& e = p.epi;
+__device__ __forceinline__ void add_bias16(const Epilogue& e, int n0, float* v) {
+  if (n0 + 16 <= e.n_bias) {
+    const float4* b = reinterpret_cast<const float4*>(e.bias + n0);
 #pragma unroll
-  for (int i = 0; i < 16; ++i) {
-    const int n = n0 + i;
-    float x = v[i];
-    if (n < e.n_bias) x += __ldg(e.bias + n);
-    if (!p.dual && n < e.n_act) x = act_gelu(x, e.act);
-    v[i] = x;
+    for (int i = 0; i < 4; ++i) {
+      const float4 t = __ldg(b + i);
+      v[4 * i] += t.x; v[4 * i + 1] += t.y; v[4 * i + 2] += t.z; v[4 * i + 3] += t.w;
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 16; ++i)
+      if (n0 + i < e.n_bias) v[i] += __ldg(e.bias + n0 + i);
+  }
+}
+
+__device__ __forceinline__ void epilogue_chunk_store(const Params& p, const GeluCoef& gc, long long row, int n0,
+                                                     float* v) {
+  const Epilogue& e = p.epi;
+  if (n0 < e.n_bias) add_bias16(e, n0, v);
+  if (!p.dual && n0 < e.n_act) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i] = gelu_fast(v[i], gc);
   }
   if (row >= p.M) return;
   const bool first = n0 < e.n_split;
@@ -135,7 +150,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     }
     for (int a = 0; a < 2; ++a) {
       ptx::mbar_init(&tfull[a], 1);
-      ptx::mbar_init(&tempty[a], 4);
+      ptx::mbar_init(&tempty[a], EPI_WARPS);
     }
     ptx::mbar_init(drain, 1);
     *abort_flag = 0;
@@ -229,7 +244,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     __syncwarp();
   } else {
     // -------------------------------------------------------------- epilogue warps
-    const int q = warp & 3;  // TMEM lane quarter this warp may read
+    const int q = warp & 3;             // TMEM lane quarter this warp may read
+    const int half = (warp - 2) >> 2;   // which alternate 16-column chunks this warp takes
+    const GeluCoef gc = gelu_coef(p.epi.act);
     uint32_t tl = 0;
     for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++tl) {
       const int m_blk = tile / p.tiles_n, n_blk = tile % p.tiles_n;
@@ -238,7 +255,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       ptx::tc_fence_after();
       const long long row = static_cast<long long>(m_blk) * BLOCK_M + q * 32 + lane;
       const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * ACC_STRIDE;
-      for (int c = 0; c < p.block_n; c += 16) {
+      for (int c = half * 16; c < p.block_n; c += 32) {
         const int n0 = n_blk * p.block_n + c;
         if (n0 >= p.N) break;
         float v[16];
@@ -248,20 +265,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           ptx::tmem_ld16(t_row + GATE_OFFSET + c, u);
           ptx::tmem_ld_wait();
 #pragma unroll
-          for (int i = 0; i < 16; ++i) v[i] = silu_f(v[i]) * u[i];
+          for (int i = 0; i < 16; ++i)
+            v[i] = (p.epi.col_partial ? silu_precise_f(v[i]) : silu_fast(v[i])) * u[i];
         } else {
           ptx::tmem_ld_wait();
         }
         if (p.epi.col_partial == nullptr) {
-          epilogue_chunk_store(p, row, n0, v);
+          epilogue_chunk_store(p, gc, row, n0, v);
         } else {
           const Epilogue& e = p.epi;
+          if (n0 < e.n_bias) add_bias16(e, n0, v);
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
-            const int n = n0 + i;
             float x = v[i];
-            if (n < e.n_bias) x += __ldg(e.bias + n);
-            if (!p.dual) x = act_gelu(x, e.act);
+            if (!p.dual) x = act_gelu(x, e.act);   // scores decide indices: full-precision activation
             x = e.score_abs ? fabsf(x) : x * x;
             v[i] = (row < p.M) ? x : 0.0f;
           }
