@@ -102,12 +102,13 @@ ffsplit_status ffsplit_destroy(ffsplit_ctx* ctx);
 /* Bytes of caller-provided scratch needed for ffsplit_forward() with up to
  * T_fwd tokens and ffsplit_score() with up to T_cal tokens per call on a layer
  * of this shape split with (k, r).  Pass 0 for a phase that is not used.
- * Always >= 256 (the status block). */
+ * Always >= 65536 (the control block: device status word and kernel tickets). */
 ffsplit_status ffsplit_workspace_size(const ffsplit_shape* shape, int64_t T_fwd, int64_t T_cal,
                                       int32_t k, int32_t r, size_t* bytes);
 
-/* Give the context its scratch memory (dev, 256-byte aligned).  The first 256
- * bytes hold the device status block and are cleared here, synchronously.
+/* Give the context its scratch memory (dev, 256-byte aligned, >= 65536 bytes).  The
+ * first 65536 bytes hold the device status word and kernel tickets and are cleared
+ * here, synchronously.
  * The workspace must outlive every call that uses the context, and calls that
  * share a workspace must not overlap on the GPU. */
 ffsplit_status ffsplit_set_workspace(ffsplit_ctx* ctx, void* dev_ptr, size_t bytes);

@@ -1,5 +1,6 @@
 // C ABI of libffsplit: argument validation, memory layouts (workspace, packed
 // blob) and the sequencing of kernels for score / select / pack / forward.
+#include <cstdlib>
 #include <cstring>
 
 #include "internal.h"
@@ -128,12 +129,20 @@ bool header_valid(const BlobHeader& h, size_t blob_bytes) {
 }
 
 struct FwdLayout { size_t ap, q, hl, xs, ys, end; };
-FwdLayout fwd_layout(const SplitDims& D, int d, size_t es, long long T) {
+// The T x mL buffer of the unfused light chain doubles as the fp32 partial buffer of
+// the fused kernel (only one of the two paths runs in a call).
+FwdLayout fwd_layout(const SplitDims& D, int d, int dtype, int act, long long T) {
   FwdLayout L;
+  const size_t es = elem_size(dtype);
   size_t off = 0;
   L.ap = off; off = align_up(off + (size_t)T * D.kp_rp * es);
   L.q = off;  off = align_up(off + (size_t)T * D.n_in * D.r_pad * es);
-  L.hl = off; off = align_up(off + (size_t)T * D.ml_pad * es);
+  size_t hl = (size_t)T * D.ml_pad * es;
+  if (fused_light_applies(dtype, act, D.r_pad, D.ml_pad)) {
+    const size_t fs = fused_light_scratch_bytes(T, D.r_pad);
+    if (fs > hl) hl = fs;
+  }
+  L.hl = off; off = align_up(off + hl);
   L.xs = off; off = align_up(off + (size_t)T * d * es);
   L.ys = off; off = align_up(off + (size_t)T * d * es);
   L.end = off;
@@ -162,7 +171,7 @@ ffsplit_status check_ctx(ffsplit_ctx* ctx, bool need_ws) {
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return check_cuda(ctx, e, "cudaGetDevice");
   if (dev != ctx->device) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "the context's device is not the current device");
-  if (need_ws && (!ctx->ws || ctx->ws_bytes < kStatusBytes))
+  if (need_ws && (!ctx->ws || ctx->ws_bytes < kCtrlBytes))
     return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL, "no workspace set (ffsplit_set_workspace)");
   return FFSPLIT_OK;
 }
@@ -181,9 +190,9 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
   const SplitDims D = dims_of(h);
   const size_t es = elem_size(h.dtype);
   const int d = h.d;
-  char* base = ctx->ws + kStatusBytes;
-  const FwdLayout L = fwd_layout(D, d, es, T);
-  if (kStatusBytes + L.xs > ctx->ws_bytes)
+  char* base = ctx->ws + kCtrlBytes;
+  const FwdLayout L = fwd_layout(D, d, h.dtype, h.act, T);
+  if (kCtrlBytes + L.xs > ctx->ws_bytes)
     return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL, "workspace too small for this forward (ffsplit_workspace_size)");
   if (decode_path_applies(ctx, h, T)) return launch_decode_forward(ctx, h, blob, X, T, Y, base, st);
   char* AP = base + L.ap;
@@ -228,7 +237,17 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
     }
   }
   // ---- stage 2: P = sigma(Q B1 + b1[light]) A2, written next to A_H
-  if (light) {
+  if (ctx->use_fused < 0) {
+    const char* env = std::getenv("FFSPLIT_NO_FUSED");
+    ctx->use_fused = (env && env[0] == '1') ? 0 : 1;
+  }
+  const long long tiles_m = (T + 127) / 128;
+  if (light && ctx->use_fused && fused_light_applies(h.dtype, h.act, D.r_pad, D.ml_pad) && tiles_m <= kMaxTicketTiles) {
+    if ((s = launch_fused_light(ctx, Q, D.r_pad, T, blob + h.off[SEC_B1T], blob + h.off[SEC_A2T], b1l, D.r_pad,
+                                D.ml_pad, h.act, AP + (size_t)D.k_pad * es, D.kp_rp, HL, ctx->tickets(),
+                                4.0 * T * D.r * D.ml, st)) != FFSPLIT_OK)
+      return s;
+  } else if (light) {
     std::memset(&g, 0, sizeof(g));
     g.A0 = Q; g.lda0 = (long long)D.n_in * D.r_pad;
     g.B0 = blob + h.off[SEC_B1T]; g.ldb0 = D.r_pad;
@@ -348,7 +367,7 @@ ffsplit_status ffsplit_workspace_size(const ffsplit_shape* shape, int64_t T_fwd,
   const SplitDims D = make_dims(*shape, k, r);
   size_t need = 0;
   if (T_fwd > 0) {
-    need = fwd_layout(D, shape->d, elem_size(shape->dtype), T_fwd).end;
+    need = fwd_layout(D, shape->d, shape->dtype, shape->act, T_fwd).end;
     BlobHeader h;
     layout_blob(*shape, D, &h);
     const size_t dec = decode_workspace_bytes(h, T_fwd);
@@ -358,18 +377,18 @@ ffsplit_status ffsplit_workspace_size(const ffsplit_shape* shape, int64_t T_fwd,
     const size_t sc = score_layout(*shape, T_cal).end;
     if (sc > need) need = sc;
   }
-  *bytes = kStatusBytes + need;
+  *bytes = kCtrlBytes + need;
   return FFSPLIT_OK;
 }
 
 ffsplit_status ffsplit_set_workspace(ffsplit_ctx* ctx, void* dev_ptr, size_t bytes) {
   ffsplit_status s = check_ctx(ctx, false);
   if (s != FFSPLIT_OK) return s;
-  if (!dev_ptr || bytes < kStatusBytes) return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL, "workspace needs >= 256 bytes");
+  if (!dev_ptr || bytes < kCtrlBytes) return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL, "workspace needs >= 65536 bytes");
   if (reinterpret_cast<uintptr_t>(dev_ptr) % kAlign != 0)
     return fail(ctx, FFSPLIT_ERR_ALIGN, "workspace must be 256-byte aligned");
-  cudaError_t e = cudaMemset(dev_ptr, 0, kStatusBytes);
-  if (e != cudaSuccess) return check_cuda(ctx, e, "cudaMemset(status block)");
+  cudaError_t e = cudaMemset(dev_ptr, 0, kCtrlBytes);
+  if (e != cudaSuccess) return check_cuda(ctx, e, "cudaMemset(control block)");
   ctx->ws = static_cast<char*>(dev_ptr);
   ctx->ws_bytes = bytes;
   ctx->tmaps.clear();
@@ -385,8 +404,8 @@ ffsplit_status ffsplit_poll(ffsplit_ctx* ctx, void* stream) {
   e = cudaMemcpy(words, ctx->ws, sizeof(words), cudaMemcpyDeviceToHost);
   if (e != cudaSuccess) return check_cuda(ctx, e, "cudaMemcpy(status block)");
   if (words[0] == 0) return FFSPLIT_OK;
-  e = cudaMemset(ctx->ws, 0, kStatusBytes);
-  if (e != cudaSuccess) return check_cuda(ctx, e, "cudaMemset(status block)");
+  e = cudaMemset(ctx->ws, 0, kCtrlBytes);
+  if (e != cudaSuccess) return check_cuda(ctx, e, "cudaMemset(control block)");
   ctx->err = "device status " + std::to_string(words[0]) + " (detail " + std::to_string(words[1]) + ", kernel " +
              std::to_string(words[2]) + ")";
   return static_cast<ffsplit_status>(words[0]);
@@ -405,10 +424,10 @@ ffsplit_status ffsplit_score(ffsplit_ctx* ctx, const ffsplit_shape* shape, const
   if (!aligned16(wt->W1) || !aligned16(wt->W2) || !aligned16(X) || (gated && !aligned16(wt->W1u)))
     return fail(ctx, FFSPLIT_ERR_ALIGN, "tensors must be 16-byte aligned");
   const ScoreLayout L = score_layout(*shape, T);
-  if (kStatusBytes + L.end > ctx->ws_bytes)
+  if (kCtrlBytes + L.end > ctx->ws_bytes)
     return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL, "workspace too small for this score call");
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  char* base = ctx->ws + kStatusBytes;
+  char* base = ctx->ws + kCtrlBytes;
   const int d = shape->d, m = shape->m, dt = shape->dtype;
   // U^T (K-major for the contraction over d)
   if ((s = launch_transpose(ctx, dt, wt->W1, m, d, m, base + L.w1t, d, d, m, nullptr, d, st)) != FFSPLIT_OK) return s;
@@ -576,11 +595,11 @@ ffsplit_status ffsplit_forward_host(ffsplit_ctx* ctx, const void* blob, const vo
   if (!h) return s;
   const SplitDims D = dims_of(*h);
   const size_t es = elem_size(h->dtype);
-  const FwdLayout L = fwd_layout(D, h->d, es, T);
-  if (kStatusBytes + L.end > ctx->ws_bytes)
+  const FwdLayout L = fwd_layout(D, h->d, h->dtype, h->act, T);
+  if (kCtrlBytes + L.end > ctx->ws_bytes)
     return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL, "workspace too small for this forward (ffsplit_workspace_size)");
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  char* base = ctx->ws + kStatusBytes;
+  char* base = ctx->ws + kCtrlBytes;
   const size_t bytes = (size_t)T * h->d * es;
   cudaError_t e = cudaMemcpyAsync(base + L.xs, X_host, bytes, cudaMemcpyHostToDevice, st);
   if (e != cudaSuccess) return check_cuda(ctx, e, "cudaMemcpyAsync(X)");

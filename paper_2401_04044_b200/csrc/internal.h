@@ -21,6 +21,11 @@ namespace ffsp {
 // word 1: detail (an index, a CTA id ...), word 2: kernel id
 // ----------------------------------------------------------------------------
 constexpr size_t kStatusBytes = 256;
+// Control block at the start of the workspace: the status block, then the ticket
+// counters of the fused light-chain kernel (zero between launches).  Cleared when
+// the workspace is installed and whenever ffsplit_poll() reports a device condition.
+constexpr size_t kCtrlBytes = 65536;
+constexpr long long kMaxTicketTiles = (kCtrlBytes - kStatusBytes) / 4;
 
 enum KernelId : int {
   KID_SELECT = 1, KID_PACK = 2, KID_GEMM_TC = 3, KID_GEMM_SIMT = 4, KID_SCORE = 5, KID_DECODE = 6, KID_FUSED = 7
@@ -135,6 +140,8 @@ struct ffsplit_ctx {
   bool attr_tc_set = false;
   bool attr_fused_set = false;
   int* status() const { return reinterpret_cast<int*>(ws); }
+  int* tickets() const { return reinterpret_cast<int*>(ws + ffsp::kStatusBytes); }
+  int use_fused = -1;  // -1: not decided yet (environment FFSPLIT_NO_FUSED=1 turns the fused kernel off)
 };
 
 namespace ffsp {
@@ -168,6 +175,12 @@ ffsplit_status launch_pack_bias(ffsplit_ctx* ctx, int dtype, const void* b1, con
                                 cudaStream_t st);
 ffsplit_status launch_score_finalize(ffsplit_ctx* ctx, const float* partial, int groups, int m, const float* w,
                                      float* energy, float* scores, int mode, int accumulate, cudaStream_t st);
+bool fused_light_applies(int dtype, int act, int r_pad, int ml_pad);
+size_t fused_light_scratch_bytes(long long T, int r_pad);
+ffsplit_status launch_fused_light(ffsplit_ctx* ctx, const void* Q, long long ldq, long long T, const void* B1T,
+                                  const void* A2T, const float* b1l, int r_pad, int ml_pad, int act, void* P,
+                                  long long ldp, char* scratch, int* tickets, double algo_flops,
+                                  cudaStream_t st);
 ffsplit_status launch_to_f32(ffsplit_ctx* ctx, int dtype, const void* in, int n, float* out, cudaStream_t st);
 
 }  // namespace ffsp

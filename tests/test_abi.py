@@ -55,8 +55,8 @@ def test_host_side_argument_errors(lib):
     assert lib.ffsplit_pack_size(C.byref(ok), 257, 0, C.byref(n), None) == 2      # k > m
     assert lib.ffsplit_pack_size(C.byref(ok), 250, 7, C.byref(n), None) == 2      # r > m - k
     assert lib.ffsplit_pack_size(C.byref(ok), 8, 65, C.byref(n), None) == 2       # r > d
-    assert lib.ffsplit_workspace_size(C.byref(ok), 128, 256, 8, 16, C.byref(n)) == 0 and n.value >= 256
-    assert lib.ffsplit_workspace_size(C.byref(ok), 0, 0, 8, 16, C.byref(n)) == 0 and n.value == 256
+    assert lib.ffsplit_workspace_size(C.byref(ok), 128, 256, 8, 16, C.byref(n)) == 0 and n.value >= 65536
+    assert lib.ffsplit_workspace_size(C.byref(ok), 0, 0, 8, 16, C.byref(n)) == 0 and n.value == 65536
     assert lib.ffsplit_workspace_size(C.byref(b.Shape(64, 256, 7, b.BF16)), 1, 1, 8, 16, C.byref(n)) == 1
     assert lib.ffsplit_workspace_size(C.byref(b.Shape(64, 256, 0, 5)), 1, 1, 8, 16, C.byref(n)) == 4
     assert lib.ffsplit_last_error(None) == b"no context"

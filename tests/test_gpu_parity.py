@@ -208,6 +208,46 @@ def test_split_forward_matches_oracle(ctx, dt, act, d, m, k, r, T):
     assert torch.equal(G.forward(blob, X), Y), "forward is not bitwise reproducible"
 
 
+# fused light chain (bf16 GELU, r_pad <= 256): ring depths, ragged ranks, one token tile spread over many CTAs
+FUSED_CASES = [
+    (256, 1024, 40, 256, 300),     # r = 256: two-slot rings
+    (128, 2000, 30, 80, 128),      # r_pad = 80: second k-block mostly zero fill; 16 CTAs on one token tile
+    (128, 700, 10, 16, 1000),      # smallest rank
+    (512, 4096, 205, 256, 1500),   # many chunks per CTA
+    (64, 130, 2, 48, 77),          # 3 chunks only: fewer chunks than the split cap
+]
+
+
+@pytest.mark.parametrize("d,m,k,r,T", FUSED_CASES)
+@pytest.mark.parametrize("act", ["gelu_erf", "gelu_tanh"])
+def test_fused_light_chain_matches_oracle_and_unfused_path(ctx, act, d, m, k, r, T, monkeypatch):
+    from paper_2401_04044_b200 import Context
+    cfg = custom_config(d, m, k, r, act=act, dtype="bf16")
+    L = make_layer(cfg, 7)
+    G = GpuLayer(ctx, L)
+    G.reserve(T, 0, k, r)
+    fac = oracle_factors(L, L.planted.numpy(), r)
+    blob, _ = G.pack(L.planted, fac)
+    X = L.tokens(T)
+    Y = G.forward(blob, X)
+    Yref = oracle_split(L, L.planted.numpy(), fac, X)
+    assert_close(Y, Yref, "bf16", "fused light chain")
+    assert torch.equal(G.forward(blob, X), Y), "fused forward is not bitwise reproducible"
+    # the same blob through the unfused GEMM chain (second context, fused kernel switched off)
+    monkeypatch.setenv("FFSPLIT_NO_FUSED", "1")
+    ctx2 = Context(0)
+    try:
+        ctx2.ensure_workspace(ctx2.workspace_size(G.shape, T, 0, k, r))
+        Xd = X.cuda()
+        Y2 = torch.empty_like(Xd)
+        ctx2.forward(blob, Xd, Y2)
+        ctx2.poll()
+    finally:
+        ctx2.close()
+    assert_close(Y2, Yref, "bf16", "unfused light chain")
+    assert orc.rel_frobenius(f64(Y2), f64(Y)) < 1e-2
+
+
 @pytest.mark.parametrize("dt,act", [("f32", "gelu_erf"), ("bf16", "gelu_erf"), ("bf16", "swiglu"), ("f32", "swiglu")])
 def test_degenerate_splits(ctx, dt, act):
     """k = m is the dense FFN; k = 0 is plain low-rank; r = 0 keeps FFN_1 only;
