@@ -232,7 +232,17 @@ fused_light_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
     const GeluCoef gc = gelu_coef(p.act);
     bool ok = true;
+    {
+      // bring this CTA's slice of b1[light] towards the SM before the first chunk needs it
+      const int te = threadIdx.x - 64;
+      const char* b0 = reinterpret_cast<const char*>(p.b1l + static_cast<long long>(c_begin) * CHUNK);
+      const long long bytes = (static_cast<long long>(min(c_end * CHUNK, p.ml_pad)) - static_cast<long long>(c_begin) * CHUNK) * 4;
+      for (long long off = static_cast<long long>(te) * 128; off < bytes; off += 256 * 128)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(b0 + off));
+    }
     for (int i = 0; i < my_chunks; ++i) {
+      if (warp == 2 && lane < 2 && i + 1 < my_chunks && (c_begin + i + 1) * CHUNK + lane * 32 < p.ml_pad)
+        asm volatile("prefetch.global.L1 [%0];" ::"l"(p.b1l + static_cast<long long>(c_begin + i + 1) * CHUNK + lane * 32));
       const int sb = i & 1;
       const uint32_t ph = (i >> 1) & 1;
       if (!ptx::mbar_wait(&sfull[sb], ph, abort_flag)) { ok = false; break; }
@@ -275,12 +285,13 @@ fused_light_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&hfull[sb]);
     }
-    // ---- the tile's accumulator
+    // ---- the tile's accumulator: TMEM -> shared memory (fp32, padded rows) -> coalesced global
     if (ok && my_chunks > 0) ok = ptx::mbar_wait(pfull, 0, abort_flag);
     if (ok) {
       ptx::tc_fence_after();
-      const long long row = static_cast<long long>(m_blk) * BLOCK_M + row_in_tile;
-      const long long rows_total = static_cast<long long>(gridDim.y) * BLOCK_M;
+      // every MMA and every TMA load of this CTA has completed: the operand buffers are free
+      float* stage = reinterpret_cast<float*>(smem);
+      const int pitch = p.r_pad + 4;   // keeps the row-per-thread float4 writes free of bank conflicts
       for (int c = half * 16; c < p.r_pad; c += 32) {
         float v[16];
         if (my_chunks > 0) {
@@ -290,29 +301,33 @@ fused_light_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 #pragma unroll
           for (int j = 0; j < 16; ++j) v[j] = 0.f;
         }
-        if (p.splits == 1) {
-          if (row < p.T) {
-            uint4 a, b;
-            a.x = pack_bf16x2(v[0], v[1]);   a.y = pack_bf16x2(v[2], v[3]);
-            a.z = pack_bf16x2(v[4], v[5]);   a.w = pack_bf16x2(v[6], v[7]);
-            b.x = pack_bf16x2(v[8], v[9]);   b.y = pack_bf16x2(v[10], v[11]);
-            b.z = pack_bf16x2(v[12], v[13]); b.w = pack_bf16x2(v[14], v[15]);
-            uint4* dst = reinterpret_cast<uint4*>(p.P + row * p.ldp + c);
-            dst[0] = a;
-            dst[1] = b;
-          }
-        } else {
-          float4* dst = reinterpret_cast<float4*>(p.partial + (static_cast<long long>(split) * rows_total + row) * p.r_pad + c);
+        float4* dst = reinterpret_cast<float4*>(stage + row_in_tile * pitch + c);
 #pragma unroll
-          for (int j = 0; j < 4; ++j) dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-        }
+        for (int j = 0; j < 4; ++j) dst[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
       }
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(redbar);
+      ok = ptx::mbar_wait(redbar, 0, abort_flag);
+    }
+    if (ok) {
+      const int te = threadIdx.x - 64;            // 0..255 among the epilogue threads
+      const int q4 = p.r_pad >> 2;                 // float4 per row
+      const int n4 = BLOCK_M * q4;
+      const long long row0 = static_cast<long long>(m_blk) * BLOCK_M;
+      const long long rows_total = static_cast<long long>(gridDim.y) * BLOCK_M;
+      const int pitch = p.r_pad + 4;
+      const float* stage = reinterpret_cast<const float*>(smem);
       if (p.splits > 1) {
+        float4* mine = reinterpret_cast<float4*>(p.partial + (static_cast<long long>(split) * rows_total + row0) * p.r_pad);
+        for (int e = te; e < n4; e += 256) {
+          const int r = e / q4, c4 = e - r * q4;
+          mine[e] = *reinterpret_cast<const float4*>(stage + r * pitch + 4 * c4);
+        }
         // publish the partial, take a ticket; the last CTA of this token tile reduces
         __threadfence();
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(redbar);
-        ok = ptx::mbar_wait(redbar, 0, abort_flag);
+        ok = ptx::mbar_wait(redbar, 1, abort_flag);
         if (ok) {
           if (warp == 2 && lane == 0) {
             const int t = atomicAdd(p.tickets + m_blk, 1);
@@ -321,36 +336,29 @@ fused_light_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           }
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(redbar);
-          ok = ptx::mbar_wait(redbar, 1, abort_flag);
+          ok = ptx::mbar_wait(redbar, 0, abort_flag);
         }
-        if (ok && *last_flag) {
-          __threadfence();
-          for (int c = half * 16; c < p.r_pad; c += 32) {
-            float acc[16];
-#pragma unroll
-            for (int j = 0; j < 16; ++j) acc[j] = 0.f;
-            for (int s = 0; s < p.splits; ++s) {   // fixed order
-              const float4* src = reinterpret_cast<const float4*>(
-                  p.partial + (static_cast<long long>(s) * rows_total + row) * p.r_pad + c);
-#pragma unroll
-              for (int j = 0; j < 4; ++j) {
-                const float4 t = __ldcg(src + j);
-                acc[4 * j] += t.x; acc[4 * j + 1] += t.y; acc[4 * j + 2] += t.z; acc[4 * j + 3] += t.w;
-              }
-            }
-            if (row < p.T) {
-              uint4 a, b;
-              a.x = pack_bf16x2(acc[0], acc[1]);   a.y = pack_bf16x2(acc[2], acc[3]);
-              a.z = pack_bf16x2(acc[4], acc[5]);   a.w = pack_bf16x2(acc[6], acc[7]);
-              b.x = pack_bf16x2(acc[8], acc[9]);   b.y = pack_bf16x2(acc[10], acc[11]);
-              b.z = pack_bf16x2(acc[12], acc[13]); b.w = pack_bf16x2(acc[14], acc[15]);
-              uint4* dst = reinterpret_cast<uint4*>(p.P + row * p.ldp + c);
-              dst[0] = a;
-              dst[1] = b;
-            }
+      }
+      if (ok && (p.splits == 1 || *last_flag)) {
+        if (p.splits > 1) __threadfence();
+        for (int e = te; e < n4; e += 256) {
+          const int r = e / q4, c4 = e - r * q4;
+          const float4 own = *reinterpret_cast<const float4*>(stage + r * pitch + 4 * c4);
+          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int s = 0; s < p.splits; ++s) {     // fixed order: the sum does not depend on which CTA is last
+            float4 t = own;
+            if (s != split)
+              t = __ldcg(reinterpret_cast<const float4*>(p.partial + (static_cast<long long>(s) * rows_total + row0) * p.r_pad) + e);
+            acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
           }
-          if (warp == 2 && lane == 0) p.tickets[m_blk] = 0;   // ready for the next launch
+          if (row0 + r < p.T) {
+            uint2 o;
+            o.x = pack_bf16x2(acc.x, acc.y);
+            o.y = pack_bf16x2(acc.z, acc.w);
+            *reinterpret_cast<uint2*>(p.P + (row0 + r) * p.ldp + 4 * c4) = o;
+          }
         }
+        if (p.splits > 1 && warp == 2 && lane == 0) p.tickets[m_blk] = 0;   // ready for the next launch
       }
     }
   }

@@ -3,7 +3,7 @@
 //   acc[row, n] = sum_k A[row, k] * B[n, k]      A: [M, K], B: [N, K], both K-major bf16
 //
 // One persistent CTA per SM walks output tiles of 128 x block_n.  Warp roles:
-//   warp 0  (one lane)  TMA producer: global -> 128B-swizzled shared tiles, 4-stage ring
+//   warp 0  (one lane)  TMA producer: global -> 128B-swizzled shared tiles, ring of up to 8 stages
 //   warp 1  (one lane)  tcgen05.mma issuer; accumulators live in tensor memory (TMEM),
 //                       two buffers so the epilogue of tile i overlaps the MMAs of tile i+1
 //   warps 2-9           epilogue: tcgen05.ld -> bias / activation / gating -> global; two warps
@@ -25,22 +25,21 @@ namespace tc {
 
 constexpr int BLOCK_M = 128;
 constexpr int BLOCK_K = 64;
-constexpr int MAX_BLOCK_N = 256;
-constexpr int STAGES = 4;
+constexpr int MAX_STAGES = 8;
 constexpr int A_STAGE_BYTES = BLOCK_M * BLOCK_K * 2;
-constexpr int B_STAGE_BYTES = MAX_BLOCK_N * BLOCK_K * 2;
 constexpr int TMEM_COLS = 512;
 constexpr int ACC_STRIDE = 256;   // TMEM columns per accumulator buffer
 constexpr int GATE_OFFSET = 128;  // second accumulator of a gated tile
 constexpr int NUM_THREADS = 320;
 constexpr int EPI_WARPS = 8;
 constexpr int BAR_BYTES = 256;
-constexpr int SMEM_BYTES = STAGES * (A_STAGE_BYTES + B_STAGE_BYTES) + BAR_BYTES + 1024;
+constexpr int MAX_SMEM = 232448;
 
 struct Params {
   long long M;
   int N, K;
   int block_n;
+  int stages;        // depth of the shared-memory ring (as many as fit, at most 8)
   int tiles_m, tiles_n;
   int dual;
   Epilogue epi;
@@ -129,12 +128,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
                const __grid_constant__ CUtensorMap tmA1, const __grid_constant__ CUtensorMap tmB1, const Params p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  const int STAGES = p.stages;
+  const int B_STAGE_BYTES = p.block_n * BLOCK_K * 2;
   uint8_t* smem_a = smem;
   uint8_t* smem_b = smem + STAGES * A_STAGE_BYTES;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES));
-  uint64_t* full = bars;                  // [STAGES] TMA -> MMA
-  uint64_t* empty = bars + STAGES;        // [STAGES] MMA -> TMA
-  uint64_t* tfull = bars + 2 * STAGES;    // [2] MMA -> epilogue
+  uint64_t* full = bars;                      // [MAX_STAGES] TMA -> MMA
+  uint64_t* empty = bars + MAX_STAGES;        // [MAX_STAGES] MMA -> TMA
+  uint64_t* tfull = bars + 2 * MAX_STAGES;    // [2] MMA -> epilogue
   uint64_t* tempty = tfull + 2;           // [2] epilogue -> MMA
   uint64_t* drain = tempty + 2;           // [1] used only when giving up
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(drain + 1);
@@ -174,7 +175,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   const int nkb = (p.K + BLOCK_K - 1) / BLOCK_K;
   const int total_kb = p.dual ? 2 * nkb : nkb;
   const int num_tiles = p.tiles_m * p.tiles_n;
-  const uint32_t stage_tx = A_STAGE_BYTES + p.block_n * BLOCK_K * 2;
+  const uint32_t stage_tx = A_STAGE_BYTES + B_STAGE_BYTES;
 
   if (warp == 0) {
     if (lane == 0) {
@@ -392,14 +393,18 @@ ffsplit_status launch_gemm_tc(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_t 
   }
   if (!ctx->attr_tc_set) {
     cudaError_t e = cudaFuncSetAttribute(tc::gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         tc::SMEM_BYTES);
+                                         tc::MAX_SMEM);
     if (e != cudaSuccess) return check_cuda(ctx, e, "cudaFuncSetAttribute(gemm_tc_kernel)");
     ctx->attr_tc_set = true;
   }
+  const int stage_bytes = tc::A_STAGE_BYTES + p.block_n * tc::BLOCK_K * 2;
+  p.stages = (tc::MAX_SMEM - tc::BAR_BYTES - 1024) / stage_bytes;
+  if (p.stages > tc::MAX_STAGES) p.stages = tc::MAX_STAGES;
+  const int smem_bytes = p.stages * stage_bytes + tc::BAR_BYTES + 1024;
   const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n;
   const int grid = static_cast<int>(tiles < ctx->num_sms ? tiles : ctx->num_sms);
   const int ph = prof_open(ctx, PROF_GEMM_TC, g.algo_flops, st);
-  tc::gemm_tc_kernel<<<grid, tc::NUM_THREADS, tc::SMEM_BYTES, st>>>(tA0, tB0, tA1, tB1, p);
+  tc::gemm_tc_kernel<<<grid, tc::NUM_THREADS, smem_bytes, st>>>(tA0, tB0, tA1, tB1, p);
   prof_close(ctx, ph, st);
   ctx->launches++;
   return check_cuda(ctx, cudaGetLastError(), "gemm_tc_kernel launch");
