@@ -341,21 +341,55 @@ fused_light_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       }
       if (ok && (p.splits == 1 || *last_flag)) {
         if (p.splits > 1) __threadfence();
-        for (int e = te; e < n4; e += 256) {
-          const int r = e / q4, c4 = e - r * q4;
-          const float4 own = *reinterpret_cast<const float4*>(stage + r * pitch + 4 * c4);
-          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-          for (int s = 0; s < p.splits; ++s) {     // fixed order: the sum does not depend on which CTA is last
-            float4 t = own;
-            if (s != split)
-              t = __ldcg(reinterpret_cast<const float4*>(p.partial + (static_cast<long long>(s) * rows_total + row0) * p.r_pad) + e);
-            acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
+        // Batches of 4 x 4 independent loads per thread: the sum over splits is taken in split order
+        // (so it does not depend on which CTA is last) but the loads do not wait for one another.
+        constexpr int EG = 4;
+        for (int e0 = te; e0 < n4; e0 += 256 * EG) {
+          float4 acc[EG];
+#pragma unroll
+          for (int j = 0; j < EG; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+          for (int s0 = 0; s0 < p.splits; s0 += 4) {
+            float4 buf[4][EG];
+#pragma unroll
+            for (int ss = 0; ss < 4; ++ss) {
+              const int sp = s0 + ss;
+#pragma unroll
+              for (int j = 0; j < EG; ++j) {
+                const int e = e0 + j * 256;
+                buf[ss][j] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (sp < p.splits && e < n4) {
+                  if (sp == split) {
+                    const int r = e / q4, c4 = e - r * q4;
+                    buf[ss][j] = *reinterpret_cast<const float4*>(stage + r * pitch + 4 * c4);
+                  } else {
+                    buf[ss][j] = __ldcg(reinterpret_cast<const float4*>(
+                                            p.partial + (static_cast<long long>(sp) * rows_total + row0) * p.r_pad) + e);
+                  }
+                }
+              }
+            }
+#pragma unroll
+            for (int ss = 0; ss < 4; ++ss) {
+              if (s0 + ss < p.splits) {
+#pragma unroll
+                for (int j = 0; j < EG; ++j) {
+                  acc[j].x += buf[ss][j].x; acc[j].y += buf[ss][j].y; acc[j].z += buf[ss][j].z; acc[j].w += buf[ss][j].w;
+                }
+              }
+            }
           }
-          if (row0 + r < p.T) {
-            uint2 o;
-            o.x = pack_bf16x2(acc.x, acc.y);
-            o.y = pack_bf16x2(acc.z, acc.w);
-            *reinterpret_cast<uint2*>(p.P + (row0 + r) * p.ldp + 4 * c4) = o;
+#pragma unroll
+          for (int j = 0; j < EG; ++j) {
+            const int e = e0 + j * 256;
+            if (e < n4) {
+              const int r = e / q4, c4 = e - r * q4;
+              if (row0 + r < p.T) {
+                uint2 o;
+                o.x = pack_bf16x2(acc[j].x, acc[j].y);
+                o.y = pack_bf16x2(acc[j].z, acc[j].w);
+                *reinterpret_cast<uint2*>(p.P + (row0 + r) * p.ldp + 4 * c4) = o;
+              }
+            }
           }
         }
         if (p.splits > 1 && warp == 2 && lane == 0) p.tickets[m_blk] = 0;   // ready for the next launch

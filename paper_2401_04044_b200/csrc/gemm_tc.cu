@@ -252,6 +252,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++tl) {
       const int m_blk = tile / p.tiles_n, n_blk = tile % p.tiles_n;
       const uint32_t acc = tl & 1, aph = (tl >> 1) & 1;
+      if (warp == 2 && p.epi.n_bias > 0) {
+        // this tile's slice of the bias vector, on its way to L1 while the MMAs run
+        const int nb = n_blk * p.block_n + lane * 32;
+        if (lane * 32 < p.block_n && nb < p.epi.n_bias) asm volatile("prefetch.global.L1 [%0];" ::"l"(p.epi.bias + nb));
+      }
       if (!ptx::mbar_wait(&tfull[acc], aph, abort_flag)) break;
       ptx::tc_fence_after();
       const long long row = static_cast<long long>(m_blk) * BLOCK_M + q * 32 + lane;
