@@ -1,0 +1,158 @@
+"""Throughput sweep over the synthetic configurations: split vs dense forward per
+FFN layer (prefill and few-token sizes), scoring, and model size.
+
+    python -m paper_2401_04044_b200.sweep --config 5 --tokens 1 32 4096 --out gpurun_out/sweep_cfg5.jsonl
+
+One JSON line per point: tokens/s per layer and per stack, achieved fraction of
+the roofline (the slower of FLOPs at the bf16 tensor peak and bytes at the HBM
+peak), split vs dense speed-up, logical model bytes.  Layers are timed on
+distinct weight copies cycled so that consecutive calls do not find their
+weights in L2.  Light factors for timing runs are random (their values do not
+change the work); parity tests use true SVD factors.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+
+import torch
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from ffsplit_synth import CFG5_HEAVY_PERCENT, CFG5_RANKS, CONFIGS, cfg5_point, make_layer  # noqa: E402
+from paper_2401_04044_b200 import Context, build, make_shape  # noqa: E402
+from paper_2401_04044_b200.factors import light_factors  # noqa: E402
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        j = json.load(open(p))
+        return j["hbm_gbs"], j["bf16_tflops"], "measured"
+    return 6650.0, 1590.0, "fallback"
+
+
+def random_factors(cfg, device, gen):
+    d, ml, r, dt = cfg.d, cfg.m - cfg.k, cfg.r, cfg.torch_dtype
+    mk = lambda *s: (torch.randn(*s, generator=gen, device=device, dtype=torch.float32) * 0.02).to(dt)
+    f = {"A1": mk(d, r), "B1": mk(r, ml), "A2": mk(ml, r), "B2": mk(r, d)}
+    if cfg.act == "swiglu":
+        f["A1u"], f["B1u"] = mk(d, r), mk(r, ml)
+    return f
+
+
+def time_calls(fn, reps, warmup):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    ts = []
+    for _ in range(reps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        b.synchronize()
+        ts.append(a.elapsed_time(b))
+    return ts
+
+
+def run_point(ctx, cfg, tokens, copies, reps, svd, device="cuda"):
+    hbm, tf, src = peaks()
+    shape = make_shape(cfg.d, cfg.m, cfg.act, cfg.torch_dtype)
+    es = 2 if cfg.dtype == "bf16" else 4
+    Tmax = max(tokens)
+    ctx.ensure_workspace(max(ctx.workspace_size(shape, Tmax, 0, cfg.k, cfg.r), ctx.workspace_size(shape, Tmax, 0, cfg.m, 0)))
+    padded, logical = ctx.pack_size(shape, cfg.k, cfg.r)
+    padded_d, logical_d = ctx.pack_size(shape, cfg.m, 0)
+    blobs, blobs_d = [], []
+    gen = torch.Generator(device=device)
+    gen.manual_seed(1234)
+    all_idx = torch.arange(cfg.m, dtype=torch.int32, device=device)
+    for c in range(copies):
+        L = make_layer(cfg, c, device=device)
+        heavy = L.planted.to(torch.int32)
+        if svd:
+            mask = torch.ones(cfg.m, dtype=torch.bool, device=device)
+            mask[heavy.long()] = False
+            fac = light_factors(L.W1, L.W2, torch.nonzero(mask).flatten(), cfg.r, L.W1u)
+        else:
+            fac = random_factors(cfg, device, gen)
+        b = torch.empty(padded, dtype=torch.uint8, device=device)
+        ctx.pack(shape, L.W1, L.b1, L.W2, L.b2, heavy, cfg.k, fac, b, W1u=L.W1u)
+        bd = torch.empty(padded_d, dtype=torch.uint8, device=device)
+        ctx.pack(shape, L.W1, L.b1, L.W2, L.b2, all_idx, cfg.m, None, bd, W1u=L.W1u)
+        ctx.poll()
+        blobs.append(b)
+        blobs_d.append(bd)
+        del L, fac
+    out = []
+    n_in = cfg.n_in
+    for T in tokens:
+        X = (torch.randn(T, cfg.d, generator=gen, device=device, dtype=torch.float32)).to(cfg.torch_dtype)
+        Y = torch.empty_like(X)
+        res = {"config": cfg.name, "d": cfg.d, "m": cfg.m, "k": cfg.k, "r": cfg.r, "act": cfg.act, "dtype": cfg.dtype,
+               "tokens": T, "layers": cfg.layers, "weight_copies_cycled": copies, "peaks": src}
+        for name, bl, params, lbytes in (("split", blobs, (n_in + 1) * (cfg.d * cfg.k + cfg.r * (cfg.d + cfg.m - cfg.k)), logical),
+                                        ("dense", blobs_d, (n_in + 1) * cfg.d * cfg.m, logical_d)):
+            state = {"i": 0}
+
+            def call():
+                ctx.forward(bl[state["i"] % copies], X, Y)
+                state["i"] += 1
+
+            ts = time_calls(call, reps, max(3, copies))
+            ctx.poll()
+            ms = statistics.median(ts)
+            flops = 2.0 * params * T
+            bytes_ = es * (params + cfg.m + cfg.d) + 2 * T * cfg.d * es
+            roof_ms = max(flops / (tf * 1e12), bytes_ / (hbm * 1e9)) * 1e3
+            res[name] = {"ms_per_layer": ms, "ms_best": min(ts), "tokens_per_s_per_layer": T / (ms * 1e-3),
+                         "tokens_per_s_per_stack": T / (ms * 1e-3 * cfg.layers), "roofline_ms": roof_ms,
+                         "roofline_frac": roof_ms / ms, "bound": "tensor" if flops / (tf * 1e12) > bytes_ / (hbm * 1e9) else "hbm",
+                         "tflops": flops / (ms * 1e-3) / 1e12, "gbs": bytes_ / (ms * 1e-3) / 1e9, "model_bytes_per_layer": lbytes}
+        res["split_vs_dense_speedup"] = res["dense"]["ms_per_layer"] / res["split"]["ms_per_layer"]
+        res["size_ratio"] = logical / logical_d
+        out.append(res)
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--config", type=int, required=True)
+    ap.add_argument("--tokens", type=int, nargs="*", default=None)
+    ap.add_argument("--copies", type=int, default=0, help="distinct weight sets cycled (0: enough to exceed 2x L2)")
+    ap.add_argument("--reps", type=int, default=20)
+    ap.add_argument("--svd", action="store_true", help="true SVD factors instead of random ones")
+    ap.add_argument("--sweep5", action="store_true", help="config 5: all heavy fractions x ranks")
+    ap.add_argument("--out", default=None)
+    args = ap.parse_args()
+    build.build()
+    ctx = Context(0)
+    base = CONFIGS[args.config]
+    points = [base]
+    if args.config == 5 and args.sweep5:
+        points = [cfg5_point(h, r) for h in CFG5_HEAVY_PERCENT for r in CFG5_RANKS]
+    tokens = args.tokens or list(base.t_fwd)
+    lines = []
+    for cfg in points:
+        es = 2 if cfg.dtype == "bf16" else 4
+        split_bytes = es * (cfg.n_in + 1) * (cfg.d * cfg.k + cfg.r * (cfg.d + cfg.m - cfg.k))
+        copies = args.copies or max(2, min(24, -(-2 * 126 * (1 << 20) // split_bytes)))
+        for res in run_point(ctx, cfg, tokens, copies, args.reps, args.svd):
+            line = json.dumps(res)
+            print(line, flush=True)
+            lines.append(line)
+        torch.cuda.empty_cache()
+    if args.out:
+        os.makedirs(os.path.dirname(os.path.abspath(args.out)), exist_ok=True)
+        with open(args.out, "w") as f:
+            f.write("\n".join(lines) + "\n")
+
+
+if __name__ == "__main__":
+    main()
