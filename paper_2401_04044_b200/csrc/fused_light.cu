@@ -3,19 +3,25 @@
 //     P = sigma(Q B1 + b1[light]) A2          Q: [T, r], B1: [r, mL], A2: [mL, r]
 //
 // for GELU layers in bf16 with r_pad <= 256.  The T x mL activation matrix never
-// leaves the SM: per 128-token tile and 64-neuron chunk
-//   GEMM-a   S = Q_tile B1[:, chunk]            tcgen05.mma -> TMEM (double buffered)
-//   epilogue H = GELU(S + b1)  -> bf16 -> shared memory in the 128B-swizzled K-major
-//            layout the tensor core reads (double buffered)
-//   GEMM-b   Pacc += H A2[chunk, :]             tcgen05.mma -> TMEM (resident accumulator)
-// Warp roles: warp 0 TMA producer of the Q tile and the B1 ring, warp 1 MMA issuer,
-// warps 2-9 epilogue, warp 10 TMA producer of the A2 ring (the two rings drain at
-// different times: a B1 tile is free once GEMM-a has read it, an A2 tile one chunk later).
-// The mL chunks of one token tile are spread over `splits`
-// CTAs so that the grid covers the SMs; each CTA writes its fp32 partial of P and
-// the last CTA to finish a token tile (atomic ticket) adds the partials in split
-// order -- a fixed order, so the result does not depend on which CTA is last --
-// and stores bf16 P.  Every wait is bounded (see gemm_tc.cu).
+// leaves the SM: per 128-token tile and 128-neuron chunk
+//   GEMM-a   S = Q_tile B1[:, chunk]        tcgen05.mma, operands in shared memory, S in
+//                                           tensor memory (TMEM), two S buffers
+//   epilogue H = GELU(S + b1) -> bf16, written back into the first half of the TMEM
+//            columns it was read from (two bf16 per 32-bit cell)
+//   GEMM-b   Pacc += H A2[chunk, :]         tcgen05.mma with the A operand read from TMEM;
+//                                           Pacc stays in TMEM for the whole tile
+// Chains of dependent small-N MMAs are latency bound on the tensor pipe, hence the
+// 128-wide chunks (N = 128 for GEMM-a, K = 128 for GEMM-b).
+// Warp roles: warp 0 TMA producer of the Q tile, the B1 ring and the bias ring,
+// warp 1 MMA issuer, warps 2-17 epilogue (four warps per TMEM lane quarter, 32
+// columns each), warp 18 TMA producer of the A2 ring.  Both weight rings work at the
+// granularity of one 64-deep k-block so that shared memory holds the Q tile plus
+// about two chunks of each operand.
+// The chunks of one token tile are spread over `splits` CTAs so that the grid covers
+// the SMs; each CTA writes its fp32 partial of P and the last CTA to finish a token
+// tile (atomic ticket) adds the partials in split order -- a fixed order, so the
+// result does not depend on which CTA is last -- and stores bf16 P.
+// Every wait is bounded (see gemm_tc.cu).
 #include "epilogue.cuh"
 #include "internal.h"
 #include "ptx.cuh"
@@ -28,24 +34,30 @@ ffsplit_status get_tmap_bf16(ffsplit_ctx* ctx, const void* ptr, long long rows, 
 namespace fl {
 
 constexpr int BLOCK_M = 128;
-constexpr int CHUNK = 64;          // light neurons per chunk (N of GEMM-a, K of GEMM-b)
+constexpr int CHUNK = 128;         // light neurons per chunk (N of GEMM-a, K of GEMM-b)
 constexpr int KB = 64;             // K elements per shared-memory k-block (one 128-byte swizzle row)
-constexpr int NUM_THREADS = 352;
-constexpr int EPI_WARPS = 8;
-constexpr int MAX_STAGES = 4;
+constexpr int EPI_WARPS = 16;
+constexpr int NUM_THREADS = 32 * (EPI_WARPS + 3);
+constexpr int EPI_THREADS = 32 * EPI_WARPS;
+constexpr int A2_WARP = EPI_WARPS + 2;
+constexpr int MAX_B1_SLOTS = 8;
+constexpr int MAX_A2_SLOTS = 6;
+constexpr int BIAS_SLOTS = 8;
 constexpr int TMEM_COLS = 512;
-constexpr int TMEM_S0 = 256;       // S buffers at columns 256 and 320; P accumulator at 0..255
-constexpr int H_BYTES = BLOCK_M * CHUNK * 2;
+constexpr int TMEM_S0 = 256;       // S buffers at columns 256 and 384; P accumulator at 0..255
 constexpr int QKB_BYTES = BLOCK_M * KB * 2;
 constexpr int B1KB_BYTES = CHUNK * KB * 2;
-constexpr int BAR_BYTES = 512;
+constexpr int BIAS_BYTES = BIAS_SLOTS * CHUNK * 4;
+constexpr int BAR_BYTES = 1024;
 constexpr int MAX_SMEM = 232448;
 
 struct Params {
   long long T;
-  int r_pad, ml_pad, kbq;          // kbq = ceil(r_pad / 64)
-  int n_chunks, splits, stages;     // stages: slots in each of the two rings
-  int b1_slot_bytes, a2_slot_bytes;
+  int r_pad, ml_pad, kbq;           // kbq = ceil(r_pad / 64): k-blocks of Q and of a B1 chunk
+  int n_chunks, splits;
+  int b1_slots, a2_slots;           // ring depths, in k-blocks
+  int a2_slot_bytes;                // r_pad * 128
+  int bias_off;                     // byte offset of the bias ring (after the rings and after the staging area)
   const float* b1l;
   __nv_bfloat16* P; long long ldp;  // output, bf16
   float* partial;                   // [splits][tiles_m * 128][r_pad] fp32 (splits > 1)
@@ -54,28 +66,56 @@ struct Params {
   int* status;
 };
 
+// D[tmem] (+)= A[tmem] * B[smem desc]: A is a 128 x 16 bf16 slab held as 8 TMEM columns.
+__device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
+                                             uint32_t accumulate) {
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "setp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n"
+      "}\n" ::"r"(d_tmem),
+      "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+      "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+      : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+// Untiled bulk copy global -> shared with completion on an mbarrier (16-byte aligned, size % 16 == 0).
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                   ptx::smem_u32(smem_dst)),
+               "l"(gsrc), "r"(bytes), "r"(ptx::smem_u32(bar))
+               : "memory");
+}
+
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 fused_light_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmB1,
                    const __grid_constant__ CUtensorMap tmA2, const Params p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* smem_q = smem;
-  uint8_t* smem_h = smem_q + p.kbq * QKB_BYTES;
-  uint8_t* smem_b1 = smem_h + 2 * H_BYTES;
-  uint8_t* smem_a2 = smem_b1 + p.stages * p.b1_slot_bytes;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem_a2 + p.stages * p.a2_slot_bytes);
-  uint64_t* b1full = bars;                    // [MAX_STAGES] TMA -> MMA (B1 tile of one chunk)
-  uint64_t* b1empty = b1full + MAX_STAGES;    // [MAX_STAGES] GEMM-a done -> TMA
-  uint64_t* a2full = b1empty + MAX_STAGES;    // [MAX_STAGES] TMA -> MMA (A2 tile of one chunk)
-  uint64_t* a2empty = a2full + MAX_STAGES;    // [MAX_STAGES] GEMM-b done -> TMA
-  uint64_t* sfull = a2empty + MAX_STAGES;     // [2] GEMM-a done -> epilogue
-  uint64_t* sempty = sfull + 2;               // [2] epilogue has read S -> MMA
-  uint64_t* hfull = sempty + 2;               // [2] epilogue wrote H -> MMA
-  uint64_t* hempty = hfull + 2;               // [2] GEMM-b has read H -> epilogue
-  uint64_t* qfull = hempty + 2;               // [1]
-  uint64_t* pfull = qfull + 1;                // [1] all GEMM-b done -> epilogue
-  uint64_t* redbar = pfull + 1;               // [1] epilogue warps rendezvous (partials written)
-  uint64_t* drain = redbar + 1;               // [1]
+  uint8_t* smem_b1 = smem_q + p.kbq * QKB_BYTES;
+  uint8_t* smem_a2 = smem_b1 + p.b1_slots * B1KB_BYTES;
+  float* smem_bias = reinterpret_cast<float*>(smem + p.bias_off);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<uint8_t*>(smem_bias) + BIAS_BYTES);
+  uint64_t* b1full = bars;                       // [MAX_B1_SLOTS] TMA -> MMA (one k-block of a B1 chunk)
+  uint64_t* b1empty = b1full + MAX_B1_SLOTS;     // [MAX_B1_SLOTS] MMA -> TMA
+  uint64_t* a2full = b1empty + MAX_B1_SLOTS;     // [MAX_A2_SLOTS] TMA -> MMA (one k-block of an A2 chunk)
+  uint64_t* a2empty = a2full + MAX_A2_SLOTS;     // [MAX_A2_SLOTS] MMA -> TMA
+  uint64_t* biasfull = a2empty + MAX_A2_SLOTS;   // [BIAS_SLOTS] TMA -> epilogue
+  uint64_t* sfull = biasfull + BIAS_SLOTS;       // [2] GEMM-a done -> epilogue
+  uint64_t* hfull = sfull + 2;                   // [2] epilogue wrote H -> MMA
+  uint64_t* qfull = hfull + 2;                   // [1]
+  uint64_t* pfull = qfull + 1;                   // [1] all GEMM-b done -> epilogue
+  uint64_t* redbar = pfull + 1;                  // [1] epilogue warps rendezvous
+  uint64_t* drain = redbar + 1;                  // [1]
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(drain + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
   volatile int* last_flag = abort_flag + 1;
@@ -90,18 +130,10 @@ fused_light_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   const int my_chunks = c_end - c_begin;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < MAX_STAGES; ++s) {
-      ptx::mbar_init(&b1full[s], 1);
-      ptx::mbar_init(&b1empty[s], 1);
-      ptx::mbar_init(&a2full[s], 1);
-      ptx::mbar_init(&a2empty[s], 1);
-    }
-    for (int a = 0; a < 2; ++a) {
-      ptx::mbar_init(&sfull[a], 1);
-      ptx::mbar_init(&sempty[a], EPI_WARPS);
-      ptx::mbar_init(&hfull[a], EPI_WARPS);
-      ptx::mbar_init(&hempty[a], 1);
-    }
+    for (int s = 0; s < MAX_B1_SLOTS; ++s) { ptx::mbar_init(&b1full[s], 1); ptx::mbar_init(&b1empty[s], 1); }
+    for (int s = 0; s < MAX_A2_SLOTS; ++s) { ptx::mbar_init(&a2full[s], 1); ptx::mbar_init(&a2empty[s], 1); }
+    for (int s = 0; s < BIAS_SLOTS; ++s) ptx::mbar_init(&biasfull[s], 1);
+    for (int a = 0; a < 2; ++a) { ptx::mbar_init(&sfull[a], 1); ptx::mbar_init(&hfull[a], EPI_WARPS); }
     ptx::mbar_init(qfull, 1);
     ptx::mbar_init(pfull, 1);
     ptx::mbar_init(redbar, EPI_WARPS);
@@ -124,28 +156,57 @@ fused_light_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 
   if (warp == 0) {
     if (lane == 0) {
-      // ------------------------------------------------------------ TMA producer: Q tile, B1 ring
+      // ------------------------------------------------------------ TMA producer: Q tile, bias ring, B1 ring
       bool ok = true;
       ptx::mbar_expect_tx(qfull, p.kbq * QKB_BYTES);
       for (int kb = 0; kb < p.kbq; ++kb) ptx::tma_load_2d(&tmQ, smem_q + kb * QKB_BYTES, qfull, kb * KB, m_blk * BLOCK_M);
-      int issued = 0;
-      for (int i = 0; i < my_chunks; ++i) {
-        const int slot = i % p.stages;
-        const uint32_t ph = (i / p.stages) & 1;
-        if (!ptx::mbar_wait(&b1empty[slot], ph ^ 1, abort_flag)) { ok = false; break; }
-        uint8_t* st = smem_b1 + slot * p.b1_slot_bytes;
-        ptx::mbar_expect_tx(&b1full[slot], p.b1_slot_bytes);
+      int g = 0;
+      for (int i = 0; i < my_chunks && ok; ++i) {
         const int chunk = c_begin + i;
-        for (int kb = 0; kb < p.kbq; ++kb) ptx::tma_load_2d(&tmB1, st + kb * B1KB_BYTES, &b1full[slot], kb * KB, chunk * CHUNK);
-        issued = i + 1;
+        for (int kb = 0; kb < p.kbq; ++kb, ++g) {
+          const int slot = g % p.b1_slots;
+          if (!ptx::mbar_wait(&b1empty[slot], ((g / p.b1_slots) & 1) ^ 1, abort_flag)) { ok = false; break; }
+          if (kb == 0) {
+            // b1[light] of this chunk; a bias slot is reused 8 chunks later, by when its readers are long done
+            const int n0 = chunk * CHUNK;
+            const int cnt = p.ml_pad - n0 < CHUNK ? p.ml_pad - n0 : CHUNK;
+            ptx::mbar_expect_tx(&biasfull[i % BIAS_SLOTS], cnt * 4);
+            bulk_load(smem_bias + (i % BIAS_SLOTS) * CHUNK, p.b1l + n0, cnt * 4, &biasfull[i % BIAS_SLOTS]);
+          }
+          ptx::mbar_expect_tx(&b1full[slot], B1KB_BYTES);
+          ptx::tma_load_2d(&tmB1, smem_b1 + slot * B1KB_BYTES, &b1full[slot], kb * KB, chunk * CHUNK);
+        }
       }
       if (!ok) {
         const long long t0 = clock64();
         while (!ptx::mbar_try_wait(qfull, 0) && clock64() - t0 < ptx::kWaitLimitCycles / 8) {}
-        const int first = issued > p.stages ? issued - p.stages : 0;
-        for (int j = first; j < issued; ++j) {
+        const int first = g > p.b1_slots ? g - p.b1_slots : 0;
+        for (int j = first; j < g; ++j) {
           const long long t1 = clock64();
-          while (!ptx::mbar_try_wait(&b1full[j % p.stages], (j / p.stages) & 1) &&
+          while (!ptx::mbar_try_wait(&b1full[j % p.b1_slots], (j / p.b1_slots) & 1) &&
+                 clock64() - t1 < ptx::kWaitLimitCycles / 8) {}
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == A2_WARP) {
+    if (lane == 0) {
+      // ------------------------------------------------------------ TMA producer: A2 ring
+      bool ok = true;
+      int g = 0;
+      for (int i = 0; i < my_chunks && ok; ++i) {
+        for (int kb = 0; kb < CHUNK / KB; ++kb, ++g) {
+          const int slot = g % p.a2_slots;
+          if (!ptx::mbar_wait(&a2empty[slot], ((g / p.a2_slots) & 1) ^ 1, abort_flag)) { ok = false; break; }
+          ptx::mbar_expect_tx(&a2full[slot], p.a2_slot_bytes);
+          ptx::tma_load_2d(&tmA2, smem_a2 + slot * p.a2_slot_bytes, &a2full[slot], (c_begin + i) * CHUNK + kb * KB, 0);
+        }
+      }
+      if (!ok) {
+        const int first = g > p.a2_slots ? g - p.a2_slots : 0;
+        for (int j = first; j < g; ++j) {
+          const long long t1 = clock64();
+          while (!ptx::mbar_try_wait(&a2full[j % p.a2_slots], (j / p.a2_slots) & 1) &&
                  clock64() - t1 < ptx::kWaitLimitCycles / 8) {}
         }
       }
@@ -157,40 +218,46 @@ fused_light_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       const uint32_t idesc_a = ptx::umma_idesc_bf16(BLOCK_M, CHUNK);
       const uint32_t idesc_b = ptx::umma_idesc_bf16(BLOCK_M, p.r_pad);
       bool ok = ptx::mbar_wait(qfull, 0, abort_flag);
-      // GEMM-b of chunk j: Pacc += H[j & 1] * A2 tile of chunk j
+      // GEMM-b of chunk j: Pacc += H(j) * A2 tile of chunk j.  H(j) sits in the S buffer j & 1: the
+      // 32 fp32 columns [32 c, 32 c + 32) of S became the 16 packed columns [32 c, 32 c + 16).
       auto gemm_b = [&](int j) -> bool {
-        const int hb = j & 1;
-        if (!ptx::mbar_wait(&hfull[hb], (j >> 1) & 1, abort_flag)) return false;
+        if (!ptx::mbar_wait(&hfull[j & 1], (j >> 1) & 1, abort_flag)) return false;
         ptx::tc_fence_after();
-        const int slot = j % p.stages;
-        if (!ptx::mbar_wait(&a2full[slot], (j / p.stages) & 1, abort_flag)) return false;
-        ptx::tc_fence_after();
-        const uint64_t a_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_h + hb * H_BYTES));
-        const uint64_t b_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_a2 + slot * p.a2_slot_bytes));
+        const uint32_t h_tmem = tmem_base + TMEM_S0 + (j & 1) * CHUNK;
+        for (int kb = 0; kb < CHUNK / KB; ++kb) {
+          const int g = j * (CHUNK / KB) + kb;
+          const int slot = g % p.a2_slots;
+          if (!ptx::mbar_wait(&a2full[slot], (g / p.a2_slots) & 1, abort_flag)) return false;
+          ptx::tc_fence_after();
+          const uint64_t b_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_a2 + slot * p.a2_slot_bytes));
 #pragma unroll
-        for (int k = 0; k < CHUNK / 16; ++k)
-          ptx::umma_bf16(tmem_base, a_desc + 2 * k, b_desc + 2 * k, idesc_b, (j | k) != 0 ? 1u : 0u);
-        ptx::umma_commit(&a2empty[slot]);
-        ptx::umma_commit(&hempty[hb]);
+          for (int k = 0; k < KB / 16; ++k) {
+            const int jj = kb * (KB / 16) + k;   // 16-element slab of this chunk's K range
+            umma_bf16_ts(tmem_base, h_tmem + 32 * (jj >> 1) + 8 * (jj & 1), b_desc + 2 * k, idesc_b,
+                         (j | jj) != 0 ? 1u : 0u);
+          }
+          ptx::umma_commit(&a2empty[slot]);
+        }
         return true;
       };
+      int g = 0;
       for (int i = 0; i < my_chunks && ok; ++i) {
-        const int slot = i % p.stages;
-        if (!ptx::mbar_wait(&b1full[slot], (i / p.stages) & 1, abort_flag)) { ok = false; break; }
-        const int sb = i & 1;
-        if (!ptx::mbar_wait(&sempty[sb], ((i >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
-        ptx::tc_fence_after();
-        const uint32_t d_tmem = tmem_base + TMEM_S0 + sb * CHUNK;
-        for (int kb = 0; kb < p.kbq; ++kb) {
+        // S buffer i & 1 is free: GEMM-b of chunk i - 2 (its last reader) was issued before this point
+        const uint32_t d_tmem = tmem_base + TMEM_S0 + (i & 1) * CHUNK;
+        for (int kb = 0; kb < p.kbq; ++kb, ++g) {
+          const int slot = g % p.b1_slots;
+          if (!ptx::mbar_wait(&b1full[slot], (g / p.b1_slots) & 1, abort_flag)) { ok = false; break; }
+          ptx::tc_fence_after();
           const uint64_t a_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_q + kb * QKB_BYTES));
-          const uint64_t b_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_b1 + slot * p.b1_slot_bytes + kb * B1KB_BYTES));
+          const uint64_t b_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_b1 + slot * B1KB_BYTES));
 #pragma unroll
           for (int k = 0; k < KB / 16; ++k)
             ptx::umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc_a, (kb | k) != 0 ? 1u : 0u);
+          ptx::umma_commit(&b1empty[slot]);
         }
-        ptx::umma_commit(&sfull[sb]);
-        ptx::umma_commit(&b1empty[slot]);
-        if (i > 0) ok = gemm_b(i - 1);   // keeps the tensor core busy while chunk i is in its epilogue
+        if (!ok) break;
+        ptx::umma_commit(&sfull[i & 1]);
+        if (i > 0) ok = gemm_b(i - 1);
       }
       if (ok && my_chunks > 0) ok = gemm_b(my_chunks - 1);
       if (ok) ptx::umma_commit(pfull);
@@ -201,98 +268,58 @@ fused_light_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       }
     }
     __syncwarp();
-  } else if (warp == 10) {
-    if (lane == 0) {
-      // ------------------------------------------------------------ TMA producer: A2 ring
-      bool ok = true;
-      int issued = 0;
-      for (int i = 0; i < my_chunks; ++i) {
-        const int slot = i % p.stages;
-        const uint32_t ph = (i / p.stages) & 1;
-        if (!ptx::mbar_wait(&a2empty[slot], ph ^ 1, abort_flag)) { ok = false; break; }
-        ptx::mbar_expect_tx(&a2full[slot], p.a2_slot_bytes);
-        ptx::tma_load_2d(&tmA2, smem_a2 + slot * p.a2_slot_bytes, &a2full[slot], (c_begin + i) * CHUNK, 0);
-        issued = i + 1;
-      }
-      if (!ok) {
-        const int first = issued > p.stages ? issued - p.stages : 0;
-        for (int j = first; j < issued; ++j) {
-          const long long t1 = clock64();
-          while (!ptx::mbar_try_wait(&a2full[j % p.stages], (j / p.stages) & 1) &&
-                 clock64() - t1 < ptx::kWaitLimitCycles / 8) {}
-        }
-      }
-    }
-    __syncwarp();
   } else {
-    // -------------------------------------------------------------- epilogue warps
-    const int q = warp & 3;
-    const int half = (warp - 2) >> 2;
+    // -------------------------------------------------------------- epilogue warps (2 .. 17)
+    const int q = warp & 3;              // TMEM lane quarter
+    const int cg = (warp - 2) >> 2;      // which 32 of the chunk's 128 columns
     const int row_in_tile = q * 32 + lane;
+    const int te = threadIdx.x - 64;     // 0 .. 511
     const uint32_t t_lane = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
     const GeluCoef gc = gelu_coef(p.act);
     bool ok = true;
-    {
-      // bring this CTA's slice of b1[light] towards the SM before the first chunk needs it
-      const int te = threadIdx.x - 64;
-      const char* b0 = reinterpret_cast<const char*>(p.b1l + static_cast<long long>(c_begin) * CHUNK);
-      const long long bytes = (static_cast<long long>(min(c_end * CHUNK, p.ml_pad)) - static_cast<long long>(c_begin) * CHUNK) * 4;
-      for (long long off = static_cast<long long>(te) * 128; off < bytes; off += 256 * 128)
-        asm volatile("prefetch.global.L2 [%0];" ::"l"(b0 + off));
-    }
     for (int i = 0; i < my_chunks; ++i) {
-      if (warp == 2 && lane < 2 && i + 1 < my_chunks && (c_begin + i + 1) * CHUNK + lane * 32 < p.ml_pad)
-        asm volatile("prefetch.global.L1 [%0];" ::"l"(p.b1l + static_cast<long long>(c_begin + i + 1) * CHUNK + lane * 32));
       const int sb = i & 1;
-      const uint32_t ph = (i >> 1) & 1;
-      if (!ptx::mbar_wait(&sfull[sb], ph, abort_flag)) { ok = false; break; }
+      if (!ptx::mbar_wait(&biasfull[i % BIAS_SLOTS], (i / BIAS_SLOTS) & 1, abort_flag)) { ok = false; break; }
+      if (!ptx::mbar_wait(&sfull[sb], (i >> 1) & 1, abort_flag)) { ok = false; break; }
       ptx::tc_fence_after();
-      float v[32];
-      const int c0 = half * 32;
-      ptx::tmem_ld16(t_lane + TMEM_S0 + sb * CHUNK + c0, v);
-      ptx::tmem_ld16(t_lane + TMEM_S0 + sb * CHUNK + c0 + 16, v + 16);
-      ptx::tmem_ld_wait();
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(&sempty[sb]);
-      const int n0 = (c_begin + i) * CHUNK + c0;
-      if (n0 + 32 <= p.ml_pad) {
-        const float4* b = reinterpret_cast<const float4*>(p.b1l + n0);
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const float4 t = __ldg(b + j);
-          v[4 * j] += t.x; v[4 * j + 1] += t.y; v[4 * j + 2] += t.z; v[4 * j + 3] += t.w;
-        }
-      } else {
-#pragma unroll
-        for (int j = 0; j < 32; ++j)
-          if (n0 + j < p.ml_pad) v[j] += __ldg(p.b1l + n0 + j);
-      }
+      const uint32_t t_s = t_lane + TMEM_S0 + sb * CHUNK + cg * 32;
+      const float* bias = smem_bias + (i % BIAS_SLOTS) * CHUNK + cg * 32;
+      const int n0 = (c_begin + i) * CHUNK + cg * 32;
       uint32_t w[16];
 #pragma unroll
-      for (int j = 0; j < 16; ++j) w[j] = pack_bf16x2(gelu_fast(v[2 * j], gc), gelu_fast(v[2 * j + 1], gc));
-      if (!ptx::mbar_wait(&hempty[sb], ph ^ 1, abort_flag)) { ok = false; break; }
-      // row `row_in_tile` of the [128 x 64] K-major tile: 128 bytes, 16-byte pieces XOR-swizzled by row % 8
-      uint8_t* hrow = smem_h + sb * H_BYTES + row_in_tile * 128;
+      for (int hlf = 0; hlf < 2; ++hlf) {
+        float v[16];
+        ptx::tmem_ld16(t_s + 16 * hlf, v);
+        ptx::tmem_ld_wait();
+        const bool inside = n0 + 16 * hlf + 16 <= p.ml_pad;   // ml_pad is a multiple of 16
+        if (inside) {
 #pragma unroll
-      for (int j = 0; j < 4; ++j) {
-        const int piece = (c0 >> 3) + j;
-        uint4 val;
-        val.x = w[4 * j]; val.y = w[4 * j + 1]; val.z = w[4 * j + 2]; val.w = w[4 * j + 3];
-        *reinterpret_cast<uint4*>(hrow + ((piece ^ (row_in_tile & 7)) << 4)) = val;
+          for (int j = 0; j < 4; ++j) {
+            const float4 b = *reinterpret_cast<const float4*>(bias + 16 * hlf + 4 * j);
+            v[4 * j] += b.x; v[4 * j + 1] += b.y; v[4 * j + 2] += b.z; v[4 * j + 3] += b.w;
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const float lo = inside ? gelu_fast(v[2 * j], gc) : 0.f;
+          const float hi = inside ? gelu_fast(v[2 * j + 1], gc) : 0.f;
+          w[8 * hlf + j] = pack_bf16x2(lo, hi);
+        }
       }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      tmem_st16(t_s, w);   // both 16-column loads of this warp's range have completed
+      tmem_st_wait();
+      ptx::tc_fence_before();
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&hfull[sb]);
     }
     // ---- the tile's accumulator: TMEM -> shared memory (fp32, padded rows) -> coalesced global
     if (ok && my_chunks > 0) ok = ptx::mbar_wait(pfull, 0, abort_flag);
+    const int pitch = p.r_pad + 4;   // keeps the row-per-thread float4 writes free of bank conflicts
+    float* stage = reinterpret_cast<float*>(smem);
     if (ok) {
       ptx::tc_fence_after();
       // every MMA and every TMA load of this CTA has completed: the operand buffers are free
-      float* stage = reinterpret_cast<float*>(smem);
-      const int pitch = p.r_pad + 4;   // keeps the row-per-thread float4 writes free of bank conflicts
-      for (int c = half * 16; c < p.r_pad; c += 32) {
+      for (int c = cg * 16; c < p.r_pad; c += 64) {
         float v[16];
         if (my_chunks > 0) {
           ptx::tmem_ld16(t_lane + c, v);
@@ -310,16 +337,13 @@ fused_light_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       ok = ptx::mbar_wait(redbar, 0, abort_flag);
     }
     if (ok) {
-      const int te = threadIdx.x - 64;            // 0..255 among the epilogue threads
       const int q4 = p.r_pad >> 2;                 // float4 per row
       const int n4 = BLOCK_M * q4;
       const long long row0 = static_cast<long long>(m_blk) * BLOCK_M;
       const long long rows_total = static_cast<long long>(gridDim.y) * BLOCK_M;
-      const int pitch = p.r_pad + 4;
-      const float* stage = reinterpret_cast<const float*>(smem);
       if (p.splits > 1) {
         float4* mine = reinterpret_cast<float4*>(p.partial + (static_cast<long long>(split) * rows_total + row0) * p.r_pad);
-        for (int e = te; e < n4; e += 256) {
+        for (int e = te; e < n4; e += EPI_THREADS) {
           const int r = e / q4, c4 = e - r * q4;
           mine[e] = *reinterpret_cast<const float4*>(stage + r * pitch + 4 * c4);
         }
@@ -341,10 +365,10 @@ fused_light_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       }
       if (ok && (p.splits == 1 || *last_flag)) {
         if (p.splits > 1) __threadfence();
-        // Batches of 4 x 4 independent loads per thread: the sum over splits is taken in split order
+        // Batches of 4 x 3 independent loads per thread: the sum over splits is taken in split order
         // (so it does not depend on which CTA is last) but the loads do not wait for one another.
-        constexpr int EG = 4;
-        for (int e0 = te; e0 < n4; e0 += 256 * EG) {
+        constexpr int EG = 3;
+        for (int e0 = te; e0 < n4; e0 += EPI_THREADS * EG) {
           float4 acc[EG];
 #pragma unroll
           for (int j = 0; j < EG; ++j) acc[j] = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -355,7 +379,7 @@ fused_light_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
               const int sp = s0 + ss;
 #pragma unroll
               for (int j = 0; j < EG; ++j) {
-                const int e = e0 + j * 256;
+                const int e = e0 + j * EPI_THREADS;
                 buf[ss][j] = make_float4(0.f, 0.f, 0.f, 0.f);
                 if (sp < p.splits && e < n4) {
                   if (sp == split) {
@@ -380,7 +404,7 @@ fused_light_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           }
 #pragma unroll
           for (int j = 0; j < EG; ++j) {
-            const int e = e0 + j * 256;
+            const int e = e0 + j * EPI_THREADS;
             if (e < n4) {
               const int r = e / q4, c4 = e - r * q4;
               if (row0 + r < p.T) {
@@ -444,13 +468,21 @@ ffsplit_status launch_fused_light(ffsplit_ctx* ctx, const void* Q, long long ldq
   if (tiles_m > 65535) return fail(ctx, FFSPLIT_ERR_SHAPE, "too many token tiles for one launch");
   p.splits = fused_light_splits(ctx->num_sms, tiles_m, p.n_chunks);
   if (p.splits > 1 && static_cast<long long>(p.splits) * tiles_m > (tiles_m > 256 ? tiles_m : 256)) p.splits = 1;
-  p.b1_slot_bytes = p.kbq * fl::B1KB_BYTES;
   p.a2_slot_bytes = r_pad * fl::KB * 2;
-  const int fixed = p.kbq * fl::QKB_BYTES + 2 * fl::H_BYTES + fl::BAR_BYTES + 1024;
-  int stages = (fl::MAX_SMEM - fixed) / (p.b1_slot_bytes + p.a2_slot_bytes);
-  if (stages > fl::MAX_STAGES) stages = fl::MAX_STAGES;
-  if (stages < 2) return fail(ctx, FFSPLIT_ERR_SHAPE, "fused light chain: shared memory too small for this rank");
-  p.stages = stages;
+  // ring depths: what fits beside the Q tile, balanced in units of chunks (kbq B1 k-blocks, 2 A2 k-blocks)
+  const int fixed = p.kbq * fl::QKB_BYTES + fl::BIAS_BYTES + fl::BAR_BYTES + 1024;
+  int best_b1 = 0, best_a2 = 0;
+  double best = -1.0;
+  for (int nb = 1; nb <= fl::MAX_B1_SLOTS; ++nb)
+    for (int na = 1; na <= fl::MAX_A2_SLOTS; ++na) {
+      if (fixed + nb * fl::B1KB_BYTES + na * p.a2_slot_bytes > fl::MAX_SMEM) continue;
+      const double a = static_cast<double>(nb) / p.kbq, b = static_cast<double>(na) / 2.0;
+      const double score = (a < b ? a : b) + 1e-3 * (a + b);
+      if (score > best) { best = score; best_b1 = nb; best_a2 = na; }
+    }
+  if (best_b1 < 1 || best_a2 < 1) return fail(ctx, FFSPLIT_ERR_SHAPE, "fused light chain: shared memory too small");
+  p.b1_slots = best_b1;
+  p.a2_slots = best_a2;
   p.b1l = b1l;
   p.P = static_cast<__nv_bfloat16*>(P);
   p.ldp = ldp;
@@ -463,7 +495,11 @@ ffsplit_status launch_fused_light(ffsplit_ctx* ctx, const void* Q, long long ldq
   if ((s = get_tmap_bf16(ctx, Q, T, r_pad, ldq, fl::BLOCK_M, &tQ)) != FFSPLIT_OK) return s;
   if ((s = get_tmap_bf16(ctx, B1T, ml_pad, r_pad, r_pad, fl::CHUNK, &tB1)) != FFSPLIT_OK) return s;
   if ((s = get_tmap_bf16(ctx, A2T, r_pad, ml_pad, ml_pad, r_pad, &tA2)) != FFSPLIT_OK) return s;
-  const int smem_bytes = fixed + stages * (p.b1_slot_bytes + p.a2_slot_bytes);
+  const int ring_end = p.kbq * fl::QKB_BYTES + p.b1_slots * fl::B1KB_BYTES + p.a2_slots * p.a2_slot_bytes;
+  const int stage_end = (fl::BLOCK_M * (r_pad + 4) * 4 + 1023) / 1024 * 1024;   // the accumulator's way out reuses the operand buffers
+  p.bias_off = ring_end > stage_end ? ring_end : stage_end;
+  const int smem_bytes = p.bias_off + fl::BIAS_BYTES + fl::BAR_BYTES + 1024;
+  if (smem_bytes > fl::MAX_SMEM) return fail(ctx, FFSPLIT_ERR_SHAPE, "fused light chain: shared memory too small");
   if (!ctx->attr_fused_set) {
     cudaError_t e = cudaFuncSetAttribute(fl::fused_light_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          fl::MAX_SMEM);
