@@ -155,7 +155,7 @@ fused_light_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   const uint32_t tmem_base = *tmem_holder;
 
   if (warp == 0) {
-    if (lane == 0) {
+    if (ptx::elect_one()) {
       // ------------------------------------------------------------ TMA producer: Q tile, bias ring, B1 ring
       bool ok = true;
       ptx::mbar_expect_tx(qfull, p.kbq * QKB_BYTES);
@@ -190,7 +190,7 @@ fused_light_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     }
     __syncwarp();
   } else if (warp == A2_WARP) {
-    if (lane == 0) {
+    if (ptx::elect_one()) {
       // ------------------------------------------------------------ TMA producer: A2 ring
       bool ok = true;
       int g = 0;
@@ -213,7 +213,7 @@ fused_light_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     }
     __syncwarp();
   } else if (warp == 1) {
-    if (lane == 0) {
+    if (ptx::elect_one()) {
       // ------------------------------------------------------------ MMA issuer
       const uint32_t idesc_a = ptx::umma_idesc_bf16(BLOCK_M, CHUNK);
       const uint32_t idesc_b = ptx::umma_idesc_bf16(BLOCK_M, p.r_pad);

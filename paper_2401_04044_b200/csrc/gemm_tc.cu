@@ -178,7 +178,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   const uint32_t stage_tx = A_STAGE_BYTES + B_STAGE_BYTES;
 
   if (warp == 0) {
-    if (lane == 0) {
+    if (ptx::elect_one()) {
       // ------------------------------------------------------------ TMA producer
       uint32_t it = 0;
       bool ok = true;
@@ -207,7 +207,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     }
     __syncwarp();
   } else if (warp == 1) {
-    if (lane == 0) {
+    if (ptx::elect_one()) {
       // ------------------------------------------------------------ MMA issuer
       const uint32_t idesc = ptx::umma_idesc_bf16(BLOCK_M, p.block_n);
       uint32_t it = 0, tl = 0;
