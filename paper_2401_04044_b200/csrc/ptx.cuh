@@ -14,9 +14,10 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
 
 // One lane of a fully converged warp.  The single-thread instructions below (TMA, tcgen05.mma,
 // tcgen05.commit) must be issued under this predicate rather than under `lane == 0`: only then does
-// the compiler know that exactly one lane is active and emit the direct uniform-datapath form.
-// Measured on B200: 220 cycles per tcgen05.mma under `threadIdx.x == 0`, 49-125 (the tensor pipe's
-// own rate for N = 64..256) under elect.sync.
+// the compiler know that exactly one lane is active and emit the direct uniform-datapath form, and
+// only while the guarded region is straight-line code (a data-dependent loop inside it, such as an
+// mbarrier spin, brings the slow form back).  Measured on B200: about 210 cycles per tcgen05.mma in
+// the slow form, 50-125 (the tensor pipe's own rate for N = 64..256) in the fast one.
 __device__ __forceinline__ bool elect_one() {
   uint32_t pred;
   asm volatile(
@@ -75,6 +76,14 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
       }
     }
   }
+}
+
+// The same wait taken by a whole converged warp; every lane returns lane 0's verdict so that the
+// warp stays converged (the loops of the producer and MMA warps are walked by all 32 lanes and only
+// the issuing instructions sit under elect_one(): straight-line code there keeps the fast form).
+__device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort_flag) {
+  const bool ok = mbar_wait(bar, parity, abort_flag);
+  return __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
 }
 
 // ------------------------------------------------------------------ TMA
