@@ -155,138 +155,117 @@ fused_light_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   const uint32_t tmem_base = *tmem_holder;
 
   if (warp == 0) {
-    // -------------------------------------------------------------- TMA producer: Q tile, bias ring, B1 ring
-    // (the whole warp walks the loops and the waits; one elected lane issues the copies)
-    bool ok = true;
     if (ptx::elect_one()) {
+      // ------------------------------------------------------------ TMA producer: Q tile, bias ring, B1 ring
+      bool ok = true;
       ptx::mbar_expect_tx(qfull, p.kbq * QKB_BYTES);
       for (int kb = 0; kb < p.kbq; ++kb) ptx::tma_load_2d(&tmQ, smem_q + kb * QKB_BYTES, qfull, kb * KB, m_blk * BLOCK_M);
-    }
-    __syncwarp();
-    int g = 0;
-    for (int i = 0; i < my_chunks && ok; ++i) {
-      const int chunk = c_begin + i;
-      for (int kb = 0; kb < p.kbq; ++kb, ++g) {
-        const int slot = g % p.b1_slots;
-        if (!ptx::mbar_wait_warp(&b1empty[slot], ((g / p.b1_slots) & 1) ^ 1, abort_flag)) { ok = false; break; }
-        if (kb == 0) {
-          // b1[light] of this chunk; a bias slot is reused 8 chunks later, by when its readers are long done
-          const int n0 = chunk * CHUNK;
-          const int cnt = p.ml_pad - n0 < CHUNK ? p.ml_pad - n0 : CHUNK;
-          if (ptx::elect_one()) {
+      int g = 0;
+      for (int i = 0; i < my_chunks && ok; ++i) {
+        const int chunk = c_begin + i;
+        for (int kb = 0; kb < p.kbq; ++kb, ++g) {
+          const int slot = g % p.b1_slots;
+          if (!ptx::mbar_wait(&b1empty[slot], ((g / p.b1_slots) & 1) ^ 1, abort_flag)) { ok = false; break; }
+          if (kb == 0) {
+            // b1[light] of this chunk; a bias slot is reused 8 chunks later, by when its readers are long done
+            const int n0 = chunk * CHUNK;
+            const int cnt = p.ml_pad - n0 < CHUNK ? p.ml_pad - n0 : CHUNK;
             ptx::mbar_expect_tx(&biasfull[i % BIAS_SLOTS], cnt * 4);
             bulk_load(smem_bias + (i % BIAS_SLOTS) * CHUNK, p.b1l + n0, cnt * 4, &biasfull[i % BIAS_SLOTS]);
           }
-          __syncwarp();
-        }
-        if (ptx::elect_one()) {
           ptx::mbar_expect_tx(&b1full[slot], B1KB_BYTES);
           ptx::tma_load_2d(&tmB1, smem_b1 + slot * B1KB_BYTES, &b1full[slot], kb * KB, chunk * CHUNK);
         }
-        __syncwarp();
       }
-    }
-    if (!ok && lane == 0) {
-      const long long t0 = clock64();
-      while (!ptx::mbar_try_wait(qfull, 0) && clock64() - t0 < ptx::kWaitLimitCycles / 8) {}
-      const int first = g > p.b1_slots ? g - p.b1_slots : 0;
-      for (int j = first; j < g; ++j) {
-        const long long t1 = clock64();
-        while (!ptx::mbar_try_wait(&b1full[j % p.b1_slots], (j / p.b1_slots) & 1) &&
-               clock64() - t1 < ptx::kWaitLimitCycles / 8) {}
+      if (!ok) {
+        const long long t0 = clock64();
+        while (!ptx::mbar_try_wait(qfull, 0) && clock64() - t0 < ptx::kWaitLimitCycles / 8) {}
+        const int first = g > p.b1_slots ? g - p.b1_slots : 0;
+        for (int j = first; j < g; ++j) {
+          const long long t1 = clock64();
+          while (!ptx::mbar_try_wait(&b1full[j % p.b1_slots], (j / p.b1_slots) & 1) &&
+                 clock64() - t1 < ptx::kWaitLimitCycles / 8) {}
+        }
       }
     }
     __syncwarp();
   } else if (warp == A2_WARP) {
-    // -------------------------------------------------------------- TMA producer: A2 ring
-    bool ok = true;
-    int g = 0;
-    for (int i = 0; i < my_chunks && ok; ++i) {
-      for (int kb = 0; kb < CHUNK / KB; ++kb, ++g) {
-        const int slot = g % p.a2_slots;
-        if (!ptx::mbar_wait_warp(&a2empty[slot], ((g / p.a2_slots) & 1) ^ 1, abort_flag)) { ok = false; break; }
-        if (ptx::elect_one()) {
+    if (ptx::elect_one()) {
+      // ------------------------------------------------------------ TMA producer: A2 ring
+      bool ok = true;
+      int g = 0;
+      for (int i = 0; i < my_chunks && ok; ++i) {
+        for (int kb = 0; kb < CHUNK / KB; ++kb, ++g) {
+          const int slot = g % p.a2_slots;
+          if (!ptx::mbar_wait(&a2empty[slot], ((g / p.a2_slots) & 1) ^ 1, abort_flag)) { ok = false; break; }
           ptx::mbar_expect_tx(&a2full[slot], p.a2_slot_bytes);
           ptx::tma_load_2d(&tmA2, smem_a2 + slot * p.a2_slot_bytes, &a2full[slot], (c_begin + i) * CHUNK + kb * KB, 0);
         }
-        __syncwarp();
       }
-    }
-    if (!ok && lane == 0) {
-      const int first = g > p.a2_slots ? g - p.a2_slots : 0;
-      for (int j = first; j < g; ++j) {
-        const long long t1 = clock64();
-        while (!ptx::mbar_try_wait(&a2full[j % p.a2_slots], (j / p.a2_slots) & 1) &&
-               clock64() - t1 < ptx::kWaitLimitCycles / 8) {}
+      if (!ok) {
+        const int first = g > p.a2_slots ? g - p.a2_slots : 0;
+        for (int j = first; j < g; ++j) {
+          const long long t1 = clock64();
+          while (!ptx::mbar_try_wait(&a2full[j % p.a2_slots], (j / p.a2_slots) & 1) &&
+                 clock64() - t1 < ptx::kWaitLimitCycles / 8) {}
+        }
       }
     }
     __syncwarp();
   } else if (warp == 1) {
-    // -------------------------------------------------------------- MMA issuer
-    // (the whole warp walks the loops and the waits; one elected lane issues each k-block's MMAs)
-    const uint32_t idesc_a = ptx::umma_idesc_bf16(BLOCK_M, CHUNK);
-    const uint32_t idesc_b = ptx::umma_idesc_bf16(BLOCK_M, p.r_pad);
-    bool ok = ptx::mbar_wait_warp(qfull, 0, abort_flag);
-    // GEMM-b of chunk j: Pacc += H(j) * A2 tile of chunk j.  H(j) sits in the S buffer j & 1: the
-    // 32 fp32 columns [32 c, 32 c + 32) of S became the 16 packed columns [32 c, 32 c + 16), so the
-    // 16-element slab jj of the chunk's K range starts at column 32 (jj / 2) + 8 (jj % 2).
-    auto gemm_b = [&](int j) -> bool {
-      if (!ptx::mbar_wait_warp(&hfull[j & 1], (j >> 1) & 1, abort_flag)) return false;
-      ptx::tc_fence_after();
-      const uint32_t h_tmem = tmem_base + TMEM_S0 + (j & 1) * CHUNK;
-      for (int kb = 0; kb < CHUNK / KB; ++kb) {
-        const int g = j * (CHUNK / KB) + kb;
-        const int slot = g % p.a2_slots;
-        if (!ptx::mbar_wait_warp(&a2full[slot], (g / p.a2_slots) & 1, abort_flag)) return false;
+    if (ptx::elect_one()) {
+      // ------------------------------------------------------------ MMA issuer
+      const uint32_t idesc_a = ptx::umma_idesc_bf16(BLOCK_M, CHUNK);
+      const uint32_t idesc_b = ptx::umma_idesc_bf16(BLOCK_M, p.r_pad);
+      bool ok = ptx::mbar_wait(qfull, 0, abort_flag);
+      // GEMM-b of chunk j: Pacc += H(j) * A2 tile of chunk j.  H(j) sits in the S buffer j & 1: the
+      // 32 fp32 columns [32 c, 32 c + 32) of S became the 16 packed columns [32 c, 32 c + 16).
+      auto gemm_b = [&](int j) -> bool {
+        if (!ptx::mbar_wait(&hfull[j & 1], (j >> 1) & 1, abort_flag)) return false;
         ptx::tc_fence_after();
-        const uint64_t b_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_a2 + slot * p.a2_slot_bytes));
-        const uint32_t h0 = h_tmem + 64 * kb;   // slabs 4 kb .. 4 kb + 3
-        const uint32_t acc0 = (j | kb) != 0 ? 1u : 0u;
-        if (ptx::elect_one()) {
-          umma_bf16_ts(tmem_base, h0, b_desc, idesc_b, acc0);
-          umma_bf16_ts(tmem_base, h0 + 8, b_desc + 2, idesc_b, 1u);
-          umma_bf16_ts(tmem_base, h0 + 32, b_desc + 4, idesc_b, 1u);
-          umma_bf16_ts(tmem_base, h0 + 40, b_desc + 6, idesc_b, 1u);
+        const uint32_t h_tmem = tmem_base + TMEM_S0 + (j & 1) * CHUNK;
+        for (int kb = 0; kb < CHUNK / KB; ++kb) {
+          const int g = j * (CHUNK / KB) + kb;
+          const int slot = g % p.a2_slots;
+          if (!ptx::mbar_wait(&a2full[slot], (g / p.a2_slots) & 1, abort_flag)) return false;
+          ptx::tc_fence_after();
+          const uint64_t b_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_a2 + slot * p.a2_slot_bytes));
+#pragma unroll
+          for (int k = 0; k < KB / 16; ++k) {
+            const int jj = kb * (KB / 16) + k;   // 16-element slab of this chunk's K range
+            umma_bf16_ts(tmem_base, h_tmem + 32 * (jj >> 1) + 8 * (jj & 1), b_desc + 2 * k, idesc_b,
+                         (j | jj) != 0 ? 1u : 0u);
+          }
           ptx::umma_commit(&a2empty[slot]);
         }
-        __syncwarp();
-      }
-      return true;
-    };
-    int g = 0;
-    for (int i = 0; i < my_chunks && ok; ++i) {
-      // S buffer i & 1 is free: GEMM-b of chunk i - 2 (its last reader) was issued before this point
-      const uint32_t d_tmem = tmem_base + TMEM_S0 + (i & 1) * CHUNK;
-      for (int kb = 0; kb < p.kbq; ++kb, ++g) {
-        const int slot = g % p.b1_slots;
-        if (!ptx::mbar_wait_warp(&b1full[slot], (g / p.b1_slots) & 1, abort_flag)) { ok = false; break; }
-        ptx::tc_fence_after();
-        const uint64_t a_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_q + kb * QKB_BYTES));
-        const uint64_t b_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_b1 + slot * B1KB_BYTES));
-        const uint32_t acc0 = kb != 0 ? 1u : 0u;
-        if (ptx::elect_one()) {
-          ptx::umma_bf16(d_tmem, a_desc, b_desc, idesc_a, acc0);
-          ptx::umma_bf16(d_tmem, a_desc + 2, b_desc + 2, idesc_a, 1u);
-          ptx::umma_bf16(d_tmem, a_desc + 4, b_desc + 4, idesc_a, 1u);
-          ptx::umma_bf16(d_tmem, a_desc + 6, b_desc + 6, idesc_a, 1u);
+        return true;
+      };
+      int g = 0;
+      for (int i = 0; i < my_chunks && ok; ++i) {
+        // S buffer i & 1 is free: GEMM-b of chunk i - 2 (its last reader) was issued before this point
+        const uint32_t d_tmem = tmem_base + TMEM_S0 + (i & 1) * CHUNK;
+        for (int kb = 0; kb < p.kbq; ++kb, ++g) {
+          const int slot = g % p.b1_slots;
+          if (!ptx::mbar_wait(&b1full[slot], (g / p.b1_slots) & 1, abort_flag)) { ok = false; break; }
+          ptx::tc_fence_after();
+          const uint64_t a_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_q + kb * QKB_BYTES));
+          const uint64_t b_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_b1 + slot * B1KB_BYTES));
+#pragma unroll
+          for (int k = 0; k < KB / 16; ++k)
+            ptx::umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc_a, (kb | k) != 0 ? 1u : 0u);
           ptx::umma_commit(&b1empty[slot]);
         }
-        __syncwarp();
+        if (!ok) break;
+        ptx::umma_commit(&sfull[i & 1]);
+        if (i > 0) ok = gemm_b(i - 1);
       }
-      if (!ok) break;
-      if (ptx::elect_one()) ptx::umma_commit(&sfull[i & 1]);
-      __syncwarp();
-      if (i > 0) ok = gemm_b(i - 1);
-    }
-    if (ok && my_chunks > 0) ok = gemm_b(my_chunks - 1);
-    if (ok) {
-      if (ptx::elect_one()) ptx::umma_commit(pfull);
-      __syncwarp();
-    }
-    if (!ok && lane == 0) {
-      ptx::umma_commit(drain);
-      const long long t0 = clock64();
-      while (!ptx::mbar_try_wait(drain, 0) && clock64() - t0 < ptx::kWaitLimitCycles / 8) {}
+      if (ok && my_chunks > 0) ok = gemm_b(my_chunks - 1);
+      if (ok) ptx::umma_commit(pfull);
+      if (!ok) {
+        ptx::umma_commit(drain);
+        const long long t0 = clock64();
+        while (!ptx::mbar_try_wait(drain, 0) && clock64() - t0 < ptx::kWaitLimitCycles / 8) {}
+      }
     }
     __syncwarp();
   } else {

@@ -178,77 +178,69 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   const uint32_t stage_tx = A_STAGE_BYTES + B_STAGE_BYTES;
 
   if (warp == 0) {
-    // -------------------------------------------------------------- TMA producer (whole warp walks, one lane issues)
-    uint32_t it = 0;
-    bool ok = true;
-    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-      const int m_blk = tile / p.tiles_n, n_blk = tile % p.tiles_n;
-      for (int kb = 0; kb < total_kb; ++kb, ++it) {
-        const int s = it % STAGES;
-        const uint32_t ph = (it / STAGES) & 1;
-        if (!ptx::mbar_wait_warp(&empty[s], ph ^ 1, abort_flag)) { ok = false; break; }
-        const bool second = p.dual && kb >= nkb;
-        const int kk = (second ? kb - nkb : kb) * BLOCK_K;
-        const CUtensorMap* ta = second ? &tmA1 : &tmA0;
-        const CUtensorMap* tb = second ? &tmB1 : &tmB0;
-        if (ptx::elect_one()) {
+    if (ptx::elect_one()) {
+      // ------------------------------------------------------------ TMA producer
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        const int m_blk = tile / p.tiles_n, n_blk = tile % p.tiles_n;
+        for (int kb = 0; kb < total_kb; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          if (!ptx::mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; break; }
           ptx::mbar_expect_tx(&full[s], stage_tx);
-          ptx::tma_load_2d(ta, smem_a + s * A_STAGE_BYTES, &full[s], kk, m_blk * BLOCK_M);
-          ptx::tma_load_2d(tb, smem_b + s * B_STAGE_BYTES, &full[s], kk, n_blk * p.block_n);
+          const bool second = p.dual && kb >= nkb;
+          const int kk = (second ? kb - nkb : kb) * BLOCK_K;
+          ptx::tma_load_2d(second ? &tmA1 : &tmA0, smem_a + s * A_STAGE_BYTES, &full[s], kk, m_blk * BLOCK_M);
+          ptx::tma_load_2d(second ? &tmB1 : &tmB0, smem_b + s * B_STAGE_BYTES, &full[s], kk, n_blk * p.block_n);
         }
-        __syncwarp();
       }
-    }
-    if (!ok && lane == 0) {
-      // give the copies already issued a bounded chance to land before the CTA exits
-      const uint32_t first = it > static_cast<uint32_t>(STAGES) ? it - STAGES : 0;
-      for (uint32_t j = first; j < it; ++j) {
-        const long long t0 = clock64();
-        while (!ptx::mbar_try_wait(&full[j % STAGES], (j / STAGES) & 1) &&
-               clock64() - t0 < ptx::kWaitLimitCycles / 8) {}
+      if (!ok) {
+        // give the copies already issued a bounded chance to land before the CTA exits
+        const uint32_t first = it > STAGES ? it - STAGES : 0;
+        for (uint32_t j = first; j < it; ++j) {
+          const long long t0 = clock64();
+          while (!ptx::mbar_try_wait(&full[j % STAGES], (j / STAGES) & 1) &&
+                 clock64() - t0 < ptx::kWaitLimitCycles / 8) {}
+        }
       }
     }
     __syncwarp();
   } else if (warp == 1) {
-    // -------------------------------------------------------------- MMA issuer (whole warp walks, one lane issues)
-    const uint32_t idesc = ptx::umma_idesc_bf16(BLOCK_M, p.block_n);
-    uint32_t it = 0, tl = 0;
-    bool ok = true;
-    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tl) {
-      const uint32_t acc = tl & 1, aph = (tl >> 1) & 1;
-      if (!ptx::mbar_wait_warp(&tempty[acc], aph ^ 1, abort_flag)) { ok = false; break; }
-      ptx::tc_fence_after();
-      for (int kb = 0; kb < total_kb; ++kb, ++it) {
-        const int s = it % STAGES;
-        const uint32_t ph = (it / STAGES) & 1;
-        if (!ptx::mbar_wait_warp(&full[s], ph, abort_flag)) { ok = false; break; }
+    if (ptx::elect_one()) {
+      // ------------------------------------------------------------ MMA issuer
+      const uint32_t idesc = ptx::umma_idesc_bf16(BLOCK_M, p.block_n);
+      uint32_t it = 0, tl = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tl) {
+        const uint32_t acc = tl & 1, aph = (tl >> 1) & 1;
+        if (!ptx::mbar_wait(&tempty[acc], aph ^ 1, abort_flag)) { ok = false; break; }
         ptx::tc_fence_after();
-        const bool second = p.dual && kb >= nkb;
-        const int kbl = second ? kb - nkb : kb;
-        const uint32_t d_tmem = tmem_base + acc * ACC_STRIDE + (second ? GATE_OFFSET : 0);
-        const uint64_t a_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_a + s * A_STAGE_BYTES));
-        const uint64_t b_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_b + s * B_STAGE_BYTES));
-        const uint32_t acc0 = kbl != 0 ? 1u : 0u;
-        if (ptx::elect_one()) {
-          // 16 elements (32 bytes) further along K inside the swizzled row: +2 in the address field
-          ptx::umma_bf16(d_tmem, a_desc, b_desc, idesc, acc0);
-          ptx::umma_bf16(d_tmem, a_desc + 2, b_desc + 2, idesc, 1u);
-          ptx::umma_bf16(d_tmem, a_desc + 4, b_desc + 4, idesc, 1u);
-          ptx::umma_bf16(d_tmem, a_desc + 6, b_desc + 6, idesc, 1u);
+        for (int kb = 0; kb < total_kb; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          if (!ptx::mbar_wait(&full[s], ph, abort_flag)) { ok = false; break; }
+          ptx::tc_fence_after();
+          const bool second = p.dual && kb >= nkb;
+          const int kbl = second ? kb - nkb : kb;
+          const uint32_t d_tmem = tmem_base + acc * ACC_STRIDE + (second ? GATE_OFFSET : 0);
+          const uint64_t a_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_a + s * A_STAGE_BYTES));
+          const uint64_t b_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_b + s * B_STAGE_BYTES));
+#pragma unroll
+          for (int k = 0; k < BLOCK_K / 16; ++k) {
+            // 16 elements (32 bytes) further along K inside the swizzled row: +2 in the address field
+            ptx::umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kbl | k) != 0 ? 1u : 0u);
+          }
           ptx::umma_commit(&empty[s]);
         }
-        __syncwarp();
+        if (ok) ptx::umma_commit(&tfull[acc]);
       }
-      if (ok) {
-        if (ptx::elect_one()) ptx::umma_commit(&tfull[acc]);
-        __syncwarp();
+      if (!ok) {
+        // wait (bounded) until the MMAs issued so far have retired before TMEM is freed
+        ptx::umma_commit(drain);
+        const long long t0 = clock64();
+        while (!ptx::mbar_try_wait(drain, 0) && clock64() - t0 < ptx::kWaitLimitCycles / 8) {}
       }
-    }
-    if (!ok && lane == 0) {
-      // wait (bounded) until the MMAs issued so far have retired before TMEM is freed
-      ptx::umma_commit(drain);
-      const long long t0 = clock64();
-      while (!ptx::mbar_try_wait(drain, 0) && clock64() - t0 < ptx::kWaitLimitCycles / 8) {}
     }
     __syncwarp();
   } else {
