@@ -37,9 +37,10 @@ void prof_close(ffsplit_ctx* ctx, int handle, cudaStream_t st) {
 }
 
 ffsplit_status launch_decode_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* blob, const void* X,
-                                     long long T, void* Y, char* ws_after_status, cudaStream_t st);
+                                     long long T, void* Y, char* AP, char* Q, char* HL, char* scratch,
+                                     cudaStream_t st);
 bool decode_path_applies(const ffsplit_ctx* ctx, const BlobHeader& h, long long T);
-size_t decode_workspace_bytes(const BlobHeader& h, long long T);
+size_t decode_scratch_bytes(int dtype, long long T);
 
 namespace {
 
@@ -128,7 +129,7 @@ bool header_valid(const BlobHeader& h, size_t blob_bytes) {
   return blob_bytes == 0 || blob_bytes >= h.total_bytes;
 }
 
-struct FwdLayout { size_t ap, q, hl, xs, ys, end; };
+struct FwdLayout { size_t ap, q, hl, xs, ys, dscratch, end; };
 // The T x mL buffer of the unfused light chain doubles as the fp32 partial buffer of
 // the fused kernel (only one of the two paths runs in a call).
 FwdLayout fwd_layout(const SplitDims& D, int d, int dtype, int act, long long T) {
@@ -145,6 +146,7 @@ FwdLayout fwd_layout(const SplitDims& D, int d, int dtype, int act, long long T)
   L.hl = off; off = align_up(off + hl);
   L.xs = off; off = align_up(off + (size_t)T * d * es);
   L.ys = off; off = align_up(off + (size_t)T * d * es);
+  L.dscratch = off; off = align_up(off + decode_scratch_bytes(dtype, T));   // few-token path: split-K partials
   L.end = off;
   return L;
 }
@@ -192,12 +194,13 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
   const int d = h.d;
   char* base = ctx->ws + kCtrlBytes;
   const FwdLayout L = fwd_layout(D, d, h.dtype, h.act, T);
-  if (kCtrlBytes + L.xs > ctx->ws_bytes)
+  const bool few = decode_path_applies(ctx, h, T);
+  if (kCtrlBytes + (few ? L.end : L.xs) > ctx->ws_bytes)
     return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL, "workspace too small for this forward (ffsplit_workspace_size)");
-  if (decode_path_applies(ctx, h, T)) return launch_decode_forward(ctx, h, blob, X, T, Y, base, st);
   char* AP = base + L.ap;
   char* Q = base + L.q;
   char* HL = base + L.hl;
+  if (few) return launch_decode_forward(ctx, h, blob, X, T, Y, AP, Q, HL, base + L.dscratch, st);
   const float* b1h = reinterpret_cast<const float*>(blob + h.off[SEC_B1H]);
   const float* b1l = reinterpret_cast<const float*>(blob + h.off[SEC_B1L]);
   const float* b2 = reinterpret_cast<const float*>(blob + h.off[SEC_B2]);
@@ -368,10 +371,6 @@ ffsplit_status ffsplit_workspace_size(const ffsplit_shape* shape, int64_t T_fwd,
   size_t need = 0;
   if (T_fwd > 0) {
     need = fwd_layout(D, shape->d, shape->dtype, shape->act, T_fwd).end;
-    BlobHeader h;
-    layout_blob(*shape, D, &h);
-    const size_t dec = decode_workspace_bytes(h, T_fwd);
-    if (dec > need) need = dec;
   }
   if (T_cal > 0) {
     const size_t sc = score_layout(*shape, T_cal).end;

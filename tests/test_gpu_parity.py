@@ -248,6 +248,35 @@ def test_fused_light_chain_matches_oracle_and_unfused_path(ctx, act, d, m, k, r,
     assert orc.rel_frobenius(f64(Y2), f64(Y)) < 1e-2
 
 
+# few-token (decode) path: every token-tile width, split-K on and off, gated and plain, ragged sizes
+DECODE_CASES = [
+    ("gelu_erf", 1024, 4096, 205, 256),    # GPT-2-medium shape
+    ("gelu_erf", 72, 300, 37, 24),         # nothing a multiple of the tiles
+    ("swiglu", 512, 1400, 70, 128),
+    ("gelu_tanh", 256, 8200, 16, 48),      # many rows: no split across CTAs in the wide product
+]
+
+
+@pytest.mark.parametrize("act,d,m,k,r", DECODE_CASES)
+@pytest.mark.parametrize("T", [1, 3, 8, 9, 16, 17, 32, 33, 64])
+def test_decode_forward_matches_oracle(ctx, act, d, m, k, r, T):
+    cfg = custom_config(d, m, k, r, act=act, dtype="bf16")
+    L = make_layer(cfg, 8)
+    G = GpuLayer(ctx, L)
+    G.reserve(T, 0, k, r)
+    G.reserve(T, 0, m, 0)
+    fac = oracle_factors(L, L.planted.numpy(), r)
+    blob, _ = G.pack(L.planted, fac)
+    X = L.tokens(T)
+    Y = G.forward(blob, X)
+    assert_close(Y, oracle_split(L, L.planted.numpy(), fac, X), "bf16", "decode split forward")
+    assert torch.equal(G.forward(blob, X), Y), "decode forward is not bitwise reproducible"
+    if T in (1, 32):
+        blobd, _ = G.pack(torch.arange(m), None)
+        dense_ref = orc.dense_ffn(f64(X), f64(L.W1), f64(L.b1), f64(L.W2), f64(L.b2), act, f64(L.W1u))
+        assert_close(G.forward(blobd, X), dense_ref, "bf16", "decode dense forward")
+
+
 @pytest.mark.parametrize("dt,act", [("f32", "gelu_erf"), ("bf16", "gelu_erf"), ("bf16", "swiglu"), ("f32", "swiglu")])
 def test_degenerate_splits(ctx, dt, act):
     """k = m is the dense FFN; k = 0 is plain low-rank; r = 0 keeps FFN_1 only;
