@@ -10,14 +10,12 @@
 // pattern, so no shuffle or shared-memory staging of operands is needed.  At these sizes the tensor
 // pipe is idle most of the time; what matters is bytes in flight per SM.
 //
-// Work split: the 8 warps of a CTA form a WR x WK grid: WR groups of 16*RT weight rows, WK disjoint
-// sub-ranges of the CTA's K range (long rows: WK = 8, short rows: WK = 1); the WK accumulators of a
-// row group are added through shared memory in warp order.  The K range is also split across CTAs
-// (`splits`) where that fills the SMs more evenly (the host picks the split that minimises wave
-// quantisation plus the extra partial traffic): each CTA writes an fp32 partial and the last one to
-// arrive (atomic ticket) adds the partials in split order, so results are bitwise reproducible.
-// The epilogue (bias, GELU / SiLU gating, the [A_H | Q] column split) runs once per output
-// element, after the reduction.
+// Work split: a CTA of 8 warps owns 16*RT weight rows and one K range; its warps take disjoint
+// sub-ranges of K and add their accumulators through shared memory in warp order.  When there are
+// few rows the K range is also split across CTAs (`splits`): each CTA writes an fp32 partial and the
+// last one to arrive (atomic ticket) adds the partials in split order, so results are bitwise
+// reproducible.  The epilogue (bias, GELU / SiLU gating, the [A_H | Q] column split) runs once per
+// output element, after the reduction.
 #include <cstring>
 
 #include "epilogue.cuh"
@@ -35,7 +33,6 @@ struct Params {
   const __nv_bfloat16* W0; const __nv_bfloat16* W1; long long ldw;   // [N, K]
   int T, N, K;
   int splits, steps_total;
-  int wk;           // warps along K inside a CTA (1, 2, 4 or 8); WR = 8 / wk row groups
   Epilogue epi;
   float* partial;   // [splits][row groups][16 RT][8 NT] fp32
   int* tickets;     // [row groups], zero before and after the launch
@@ -43,7 +40,7 @@ struct Params {
 
 __device__ __forceinline__ uint4 ldg_stream(const void* p) {
   uint4 v;
-  asm volatile("ld.global.nc.L1::no_allocate.L2::256B.v4.u32 {%0, %1, %2, %3}, [%4];"
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
                : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
   return v;
 }
@@ -61,23 +58,20 @@ template <int RT, int NT, bool DUAL>
 __global__ void __launch_bounds__(THREADS, 1) decode_gemm_kernel(const Params p) {
   extern __shared__ float red[];   // [WARPS][16 RT][8 NT]
   __shared__ int s_last;
-  constexpr int ROWS = 16 * RT;          // weight-row slots per warp
+  constexpr int ROWS = 16 * RT;          // weight-row slots per CTA
   constexpr int TP = 8 * NT;
-  constexpr int OUT_ROWS = DUAL ? ROWS / 2 : ROWS;   // output rows per warp-row group
-  constexpr int ELEMS = ROWS * TP;
+  constexpr int OUT_ROWS = DUAL ? ROWS / 2 : ROWS;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, c = lane & 3;
-  const int WK = p.wk, WR = WARPS / WK;
-  const int wr = warp / WK, wk = warp - wr * WK;
   const int rg = blockIdx.x, split = blockIdx.y;
-  const int row0 = (rg * WR + wr) * OUT_ROWS;
+  const int row0 = rg * OUT_ROWS;
 
   // this warp's range of k steps
   const int cta_lo = static_cast<int>(static_cast<long long>(p.steps_total) * split / p.splits);
   const int cta_hi = static_cast<int>(static_cast<long long>(p.steps_total) * (split + 1) / p.splits);
   const int n_cta = cta_hi - cta_lo;
-  const int s_lo = cta_lo + static_cast<int>(static_cast<long long>(n_cta) * wk / WK);
-  const int s_hi = cta_lo + static_cast<int>(static_cast<long long>(n_cta) * (wk + 1) / WK);
+  const int s_lo = cta_lo + static_cast<int>(static_cast<long long>(n_cta) * warp / WARPS);
+  const int s_hi = cta_lo + static_cast<int>(static_cast<long long>(n_cta) * (warp + 1) / WARPS);
 
   float acc[RT][NT][4];
 #pragma unroll
@@ -150,8 +144,8 @@ __global__ void __launch_bounds__(THREADS, 1) decode_gemm_kernel(const Params p)
     ++s;
   }
 
-  // ---- the WK accumulators of each row group are added in warp order
-  float* mine = red + warp * ELEMS;
+  // ---- add the warps' accumulators in warp order
+  float* mine = red + warp * ROWS * TP;
 #pragma unroll
   for (int i = 0; i < RT; ++i)
 #pragma unroll
@@ -163,17 +157,28 @@ __global__ void __launch_bounds__(THREADS, 1) decode_gemm_kernel(const Params p)
       mine[(16 * i + g + 8) * TP + t + 1] = acc[i][j][3];
     }
   __syncthreads();
-  const int cta_elems = WR * ELEMS;
-  float* mypart = p.partial + (static_cast<long long>(split) * gridDim.x + rg) * (WARPS * ELEMS);
-  for (int idx = threadIdx.x; idx < cta_elems; idx += THREADS) {
-    const int r = idx / ELEMS, rem = idx - r * ELEMS;
+  constexpr int ELEMS = ROWS * TP;
+  constexpr int PER = (ELEMS + THREADS - 1) / THREADS;
+  float tot[PER];
+#pragma unroll
+  for (int e = 0; e < PER; ++e) {
+    const int idx = threadIdx.x + e * THREADS;
     float v = 0.f;
-    for (int w = 0; w < WK; ++w) v += red[(r * WK + w) * ELEMS + rem];
-    if (p.splits > 1) mypart[idx] = v;
-    else red[(r * WK) * ELEMS + rem] = v;   // read and written by this thread only
+    if (idx < ELEMS) {
+#pragma unroll
+      for (int w = 0; w < WARPS; ++w) v += red[w * ROWS * TP + idx];
+    }
+    tot[e] = v;
   }
+  __syncthreads();
   // ---- across CTAs: partials + ticket, the last CTA of the row group adds them in split order
   if (p.splits > 1) {
+    float* mypart = p.partial + (static_cast<long long>(split) * gridDim.x + rg) * ELEMS;
+#pragma unroll
+    for (int e = 0; e < PER; ++e) {
+      const int idx = threadIdx.x + e * THREADS;
+      if (idx < ELEMS) mypart[idx] = tot[e];
+    }
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -184,31 +189,36 @@ __global__ void __launch_bounds__(THREADS, 1) decode_gemm_kernel(const Params p)
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    for (int idx = threadIdx.x; idx < cta_elems; idx += THREADS) {
-      const int r = idx / ELEMS, rem = idx - r * ELEMS;
+#pragma unroll
+    for (int e = 0; e < PER; ++e) {
+      const int idx = threadIdx.x + e * THREADS;
       float v = 0.f;
-      for (int sp = 0; sp < p.splits; ++sp)
-        v += __ldcg(p.partial + (static_cast<long long>(sp) * gridDim.x + rg) * (WARPS * ELEMS) + idx);
-      red[(r * WK) * ELEMS + rem] = v;
+      if (idx < ELEMS) {
+        for (int sp = 0; sp < p.splits; ++sp)
+          v += (sp == split) ? tot[e] : __ldcg(p.partial + (static_cast<long long>(sp) * gridDim.x + rg) * ELEMS + idx);
+      }
+      tot[e] = v;
     }
     if (threadIdx.x == 0) p.tickets[rg] = 0;
   }
+  // ---- totals back to shared memory as [row][t], then the epilogue with n fastest across threads
+#pragma unroll
+  for (int e = 0; e < PER; ++e) {
+    const int idx = threadIdx.x + e * THREADS;
+    if (idx < ELEMS) red[idx] = tot[e];
+  }
   __syncthreads();
-  // ---- epilogue, n fastest across threads
   const Epilogue& ep = p.epi;
   const GeluCoef gc = gelu_coef(ep.act);
-  const int out_cta = WR * OUT_ROWS;
-  for (int idx = threadIdx.x; idx < out_cta * TP; idx += THREADS) {
-    const int t = idx / out_cta, nc = idx - t * out_cta;
-    const int r = nc / OUT_ROWS, nl = nc - r * OUT_ROWS;
-    const int n = rg * out_cta + nc;
+  for (int idx = threadIdx.x; idx < OUT_ROWS * TP; idx += THREADS) {
+    const int t = idx / OUT_ROWS, nl = idx - t * OUT_ROWS;
+    const int n = row0 + nl;
     if (t >= p.T || n >= p.N) continue;
-    const float* src = red + (r * WK) * ELEMS;
     float v;
     if (DUAL) {
-      v = silu_fast(src[nl * TP + t]) * src[(nl + OUT_ROWS) * TP + t];
+      v = silu_fast(red[nl * TP + t]) * red[(nl + OUT_ROWS) * TP + t];
     } else {
-      v = src[nl * TP + t];
+      v = red[nl * TP + t];
       if (n < ep.n_bias) v += __ldg(ep.bias + n);
       if (n < ep.n_act) v = gelu_fast(v, gc);
     }
@@ -217,25 +227,16 @@ __global__ void __launch_bounds__(THREADS, 1) decode_gemm_kernel(const Params p)
   }
 }
 
-// CTAs of this instantiation that fit on one SM (0 on error); sets the shared-memory attribute once.
-template <int RT, int NT, bool DUAL>
-int ctas_per_sm() {
-  static int cached = -1;
-  if (cached < 0) {
-    const int smem = WARPS * 16 * RT * 8 * NT * 4;
-    int n = 0;
-    if (cudaFuncSetAttribute(decode_gemm_kernel<RT, NT, DUAL>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) !=
-            cudaSuccess ||
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, decode_gemm_kernel<RT, NT, DUAL>, THREADS, smem) != cudaSuccess)
-      n = 0;
-    cached = n;
-  }
-  return cached;
-}
-
 template <int RT, int NT, bool DUAL>
 cudaError_t launch_one(const Params& p, int row_groups, cudaStream_t st) {
   const int smem = WARPS * 16 * RT * 8 * NT * 4;
+  static bool attr_done = false;
+  if (!attr_done) {
+    cudaError_t e = cudaFuncSetAttribute(decode_gemm_kernel<RT, NT, DUAL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         smem);
+    if (e != cudaSuccess) return e;
+    attr_done = true;
+  }
   decode_gemm_kernel<RT, NT, DUAL><<<dim3(row_groups, p.splits), THREADS, smem, st>>>(p);
   return cudaGetLastError();
 }
@@ -260,43 +261,18 @@ static ffsplit_status decode_gemm(ffsplit_ctx* ctx, const void* X0, const void* 
   p.tickets = ctx->tickets();
   const int nt = T <= 8 ? 1 : T <= 16 ? 2 : T <= 32 ? 4 : 8;
   const int rt = nt == 8 ? 2 : 4;
-  const int out_rows_w = dual ? 8 * rt : 16 * rt;   // output rows per warp-row group
-  int occ;
-#define FFS_OCC(RT_, NT_) (dual ? dec::ctas_per_sm<RT_, NT_, true>() : dec::ctas_per_sm<RT_, NT_, false>())
-  if (nt == 1) occ = FFS_OCC(4, 1);
-  else if (nt == 2) occ = FFS_OCC(4, 2);
-  else if (nt == 4) occ = FFS_OCC(4, 4);
-  else occ = FFS_OCC(2, 8);
-#undef FFS_OCC
-  if (occ < 1) return fail(ctx, FFSPLIT_ERR_CUDA, "decode kernel cannot be resident (occupancy query failed)");
-  const int slots = occ * ctx->num_sms;
-  // Plan: warps along K inside a CTA (wk), K splits across CTAs.  Cost model: waves of CTAs (quantised)
-  // times the traffic including the fp32 partials; every warp should keep at least 4 k steps.
-  const double w_bytes = 2.0 * N * K;
-  int best_wk = 8, best_splits = 1;
-  double best_cost = 1e300;
-  for (int wk = 8; wk >= 1; wk >>= 1) {
-    const int wr = dec::WARPS / wk;
-    const long long rgs = (N + static_cast<long long>(out_rows_w) * wr - 1) / (static_cast<long long>(out_rows_w) * wr);
-    if (rgs > kMaxTicketTiles) continue;
-    for (int sp = 1; sp <= 16; ++sp) {
-      if (sp > 1 && p.steps_total / (sp * wk) < 4) break;
-      const long long part_rows = rgs * dec::WARPS * 16 * rt;   // row slots of one split's partials
-      if (sp > 1 && sp * part_rows > kDecodeMaxPartialRows) break;
-      const double ctas = static_cast<double>(rgs) * sp;
-      const double waves = ctas / slots;
-      const double quant = (waves <= 1.0) ? 1.0 / (waves < 0.05 ? 0.05 : waves) : static_cast<double>((long long)(waves + 0.999999)) / waves;
-      const double part_bytes = sp > 1 ? 2.0 * sp * rgs * wr * 16.0 * rt * 8 * nt * 4 : 0.0;
-      const double steps_per_warp = static_cast<double>(p.steps_total) / (sp * wk);
-      const double latency_pen = 1.0 + 3.0 / (steps_per_warp + 1.0);   // short warps cannot hide the first load
-      const double cost = quant * (1.0 + part_bytes / w_bytes) * latency_pen + 0.01 * sp;
-      if (cost < best_cost) { best_cost = cost; best_wk = wk; best_splits = sp; }
-    }
-  }
-  p.wk = best_wk;
-  p.splits = best_splits;
-  const int wr = dec::WARPS / p.wk;
-  const int row_groups = static_cast<int>((N + static_cast<long long>(out_rows_w) * wr - 1) / (static_cast<long long>(out_rows_w) * wr));
+  const int out_rows = dual ? 8 * rt : 16 * rt;
+  const int row_groups = (N + out_rows - 1) / out_rows;
+  if (row_groups > kMaxTicketTiles) return fail(ctx, FFSPLIT_ERR_SHAPE, "decode: too many row groups");
+  // enough CTAs to keep every SM streaming, each warp keeping at least two k steps, partials bounded
+  int splits = (2 * ctx->num_sms + row_groups - 1) / row_groups;
+  const int max_by_k = p.steps_total / (2 * dec::WARPS);
+  if (splits > max_by_k) splits = max_by_k;
+  if (splits > 16) splits = 16;
+  const long long rows_slots = static_cast<long long>(row_groups) * 16 * rt;
+  if (splits > 1 && splits * rows_slots > kDecodeMaxPartialRows) splits = static_cast<int>(kDecodeMaxPartialRows / rows_slots);
+  if (splits < 1) splits = 1;
+  p.splits = splits;
   const int ph = prof_open(ctx, PROF_DECODE, algo_bytes, st);
   cudaError_t e;
 #define FFS_DEC(RT_, NT_) (dual ? dec::launch_one<RT_, NT_, true>(p, row_groups, st) : dec::launch_one<RT_, NT_, false>(p, row_groups, st))
