@@ -181,6 +181,30 @@ ffsplit_status ffsplit_forward(ffsplit_ctx* ctx, const void* blob, const void* X
 ffsplit_status ffsplit_forward_host(ffsplit_ctx* ctx, const void* blob, const void* X_host, int64_t T,
                                     void* Y_host, void* stream);
 
+/* The split forward of ffsplit_forward() for callers that cannot allocate device memory.
+ * (The paper has no counterpart to this entry point; it exists for deployment.)
+ *
+ * Who needs it: code that runs the per-token decode step inside a host application that owns
+ * all of the GPU's memory -- an inference server that has handed every free byte to its KV-cache
+ * arena, a plug-in called from inside another runtime's execution step -- where cudaMalloc would
+ * fail, or would stall the device, and where no workspace was set aside for this library.  This
+ * call needs no ffsplit_set_workspace(): its intermediates, K-split partials and counters live in
+ * a 4.06 MiB array built into the library (held by every GPU that loads the library, from load
+ * until the process exits).  It calls no allocator of any kind.
+ *
+ *   blob  dev  a bf16 layer packed by ffsplit_pack() (GELU or SwiGLU)
+ *   X     dev  [T, d], Y dev [T, d], 1 <= T <= 8
+ * Limits, rejected with an error and nothing launched: T > 8 (FFSPLIT_ERR_SHAPE), fp32 layers
+ * (FFSPLIT_ERR_DTYPE), layers whose intermediates T*(k_pad + (n_in+1)*r_pad + mL_pad)*2 bytes
+ * exceed 2 MiB (FFSPLIT_ERR_BUFFER_TOO_SMALL).
+ * The first call on a device looks up the array's device address and sets kernel attributes;
+ * make that first call outside any stream capture.
+ * All calls on a device share the one array and it keeps the previous call's contents: the call
+ * clears the counters it needs at zero itself, but two calls that overlap on the GPU (different
+ * streams, no ordering between them) race on it.  Results equal those of ffsplit_forward(). */
+ffsplit_status ffsplit_forward_noalloc(ffsplit_ctx* ctx, const void* blob, const void* X, int64_t T,
+                                       void* Y, void* stream);
+
 /* Synchronise `stream`, then return and clear the device status word
  * (FFSPLIT_OK if no kernel recorded a condition). */
 ffsplit_status ffsplit_poll(ffsplit_ctx* ctx, void* stream);

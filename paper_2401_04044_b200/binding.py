@@ -32,7 +32,7 @@ EXPORTS = [
     "ffsplit_create", "ffsplit_destroy", "ffsplit_workspace_size", "ffsplit_set_workspace", "ffsplit_score",
     "ffsplit_select", "ffsplit_pack_size", "ffsplit_pack", "ffsplit_blob_open", "ffsplit_blob_section",
     "ffsplit_forward", "ffsplit_forward_host", "ffsplit_poll", "ffsplit_launch_count", "ffsplit_last_error",
-    "ffsplit_version", "ffsplit_profile_begin", "ffsplit_profile_end",
+    "ffsplit_version", "ffsplit_profile_begin", "ffsplit_profile_end", "ffsplit_forward_noalloc",
 ]
 
 
@@ -82,6 +82,7 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.ffsplit_blob_section.argtypes = [vp, vp, i32, P(sz), P(i64), P(i64), P(i64)]
     lib.ffsplit_forward.argtypes = [vp, vp, vp, i64, vp, vp]
     lib.ffsplit_forward_host.argtypes = [vp, vp, vp, i64, vp, vp]
+    lib.ffsplit_forward_noalloc.argtypes = [vp, vp, vp, i64, vp, vp]
     lib.ffsplit_poll.argtypes = [vp, vp]
     lib.ffsplit_profile_begin.argtypes = [vp]
     lib.ffsplit_profile_end.argtypes = [vp, vp, i32, P(i32), P(C.c_double), P(C.c_double)]
@@ -204,6 +205,11 @@ class Context:
     def forward(self, blob, X, Y, stream=None):
         self._check(self.lib.ffsplit_forward(self.h, _ptr(blob), _ptr(X), X.shape[0], _ptr(Y), _stream_ptr(stream)),
                     "ffsplit_forward")
+
+    def forward_noalloc(self, blob, X, Y, stream=None):
+        """ffsplit_forward_noalloc: up to 8 tokens, bf16, scratch built into the library (no workspace needed)."""
+        self._check(self.lib.ffsplit_forward_noalloc(self.h, _ptr(blob), _ptr(X), X.shape[0], _ptr(Y),
+                                                     _stream_ptr(stream)), "ffsplit_forward_noalloc")
 
     def forward_host(self, blob, X_host, Y_host, stream=None):
         self._check(self.lib.ffsplit_forward_host(self.h, _ptr(blob), _ptr(X_host), X_host.shape[0], _ptr(Y_host),

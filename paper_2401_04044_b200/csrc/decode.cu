@@ -248,7 +248,7 @@ constexpr long long kDecodeMaxPartialRows = 65536;
 // One skinny product.  dual: (X0, W0) and (X1, W1) on the same rows, gated.
 static ffsplit_status decode_gemm(ffsplit_ctx* ctx, const void* X0, const void* X1, long long ldx, const void* W0,
                                   const void* W1, long long ldw, int T, int N, int K, const Epilogue& epi,
-                                  float* partial, double algo_bytes, cudaStream_t st) {
+                                  float* partial, double algo_bytes, cudaStream_t st, int* tickets = nullptr) {
   if (N <= 0 || K <= 0) return FFSPLIT_OK;
   const bool dual = W1 != nullptr;
   dec::Params p;
@@ -258,7 +258,7 @@ static ffsplit_status decode_gemm(ffsplit_ctx* ctx, const void* X0, const void* 
   p.steps_total = (K + dec::KSTEP - 1) / dec::KSTEP;
   p.epi = epi;
   p.partial = partial;
-  p.tickets = ctx->tickets();
+  p.tickets = tickets ? tickets : ctx->tickets();
   const int nt = T <= 8 ? 1 : T <= 16 ? 2 : T <= 32 ? 4 : 8;
   const int rt = nt == 8 ? 2 : 4;
   const int out_rows = dual ? 8 * rt : 16 * rt;
@@ -297,9 +297,9 @@ size_t decode_scratch_bytes(int dtype, long long T) {
   return static_cast<size_t>(kDecodeMaxPartialRows) * 64 * 4;
 }
 
-ffsplit_status launch_decode_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* blob, const void* X,
-                                     long long T64, void* Y, char* AP, char* Q, char* HL, char* scratch,
-                                     cudaStream_t st) {
+static ffsplit_status decode_forward_impl(ffsplit_ctx* ctx, const BlobHeader& h, const char* blob, const void* X,
+                                          long long T64, void* Y, char* AP, char* Q, char* HL, char* scratch,
+                                          cudaStream_t st, int* tickets) {
   const int T = static_cast<int>(T64);
   const int d = h.d, k_pad = h.k_pad, r_pad = h.r_pad, ml_pad = h.ml_pad, kp_rp = h.k_pad + h.r_pad;
   const bool gated = h.act == FFSPLIT_SWIGLU;
@@ -318,17 +318,17 @@ ffsplit_status launch_decode_forward(ffsplit_ctx* ctx, const BlobHeader& h, cons
     e.C0 = AP; e.ld0 = kp_rp; e.C1 = Q; e.ld1 = r_pad;
     e.n_split = k_pad; e.n_act = k_pad; e.n_bias = k_pad; e.bias = b1h;
     if ((s = decode_gemm(ctx, X, nullptr, d, blob + h.off[SEC_U1T], nullptr, d, T, kp_rp, d, e, part,
-                         2.0 * d * (h.k + h.r) + 4.0 * h.k + xy / 2, st)) != FFSPLIT_OK) return s;
+                         2.0 * d * (h.k + h.r) + 4.0 * h.k + xy / 2, st, tickets)) != FFSPLIT_OK) return s;
   } else {
     clear();
     e.C0 = AP; e.ld0 = kp_rp; e.n_split = k_pad;
     if ((s = decode_gemm(ctx, X, X, d, blob + h.off[SEC_U1T], blob + h.off[SEC_U1UT], d, T, k_pad, d, e, part,
-                         4.0 * d * h.k + xy / 2, st)) != FFSPLIT_OK) return s;
+                         4.0 * d * h.k + xy / 2, st, tickets)) != FFSPLIT_OK) return s;
     if (light) {
       clear();
       e.C0 = Q; e.ld0 = 2 * r_pad; e.n_split = 2 * r_pad;
       if ((s = decode_gemm(ctx, X, nullptr, d, blob + h.off[SEC_A1T], nullptr, d, T, 2 * r_pad, d, e, part,
-                           4.0 * d * h.r, st)) != FFSPLIT_OK) return s;
+                           4.0 * d * h.r, st, tickets)) != FFSPLIT_OK) return s;
     }
   }
   // ---- stage 2
@@ -339,17 +339,95 @@ ffsplit_status launch_decode_forward(ffsplit_ctx* ctx, const BlobHeader& h, cons
     const long long ldq = static_cast<long long>(h.n_in) * r_pad;
     if ((s = decode_gemm(ctx, Q, gated ? Q + static_cast<size_t>(r_pad) * 2 : nullptr, ldq, blob + h.off[SEC_B1T],
                          gated ? blob + h.off[SEC_B1UT] : nullptr, r_pad, T, ml_pad, r_pad, e, part,
-                         2.0 * h.n_in * h.r * h.ml + (gated ? 0.0 : 4.0 * h.ml), st)) != FFSPLIT_OK) return s;
+                         2.0 * h.n_in * h.r * h.ml + (gated ? 0.0 : 4.0 * h.ml), st, tickets)) != FFSPLIT_OK) return s;
     clear();
     e.C0 = AP + static_cast<size_t>(k_pad) * 2; e.ld0 = kp_rp; e.n_split = r_pad;
     if ((s = decode_gemm(ctx, HL, nullptr, ml_pad, blob + h.off[SEC_A2T], nullptr, ml_pad, T, r_pad, ml_pad, e, part,
-                         2.0 * h.r * h.ml, st)) != FFSPLIT_OK) return s;
+                         2.0 * h.r * h.ml, st, tickets)) != FFSPLIT_OK) return s;
   }
   // ---- stage 3
   clear();
   e.C0 = Y; e.ld0 = d; e.n_split = d; e.n_bias = d; e.bias = b2;
   return decode_gemm(ctx, AP, nullptr, kp_rp, blob + h.off[SEC_V1B2T], nullptr, kp_rp, T, d, light ? kp_rp : k_pad, e,
-                     part, 2.0 * d * (h.k + (light ? h.r : 0)) + 4.0 * d + xy / 2, st);
+                     part, 2.0 * d * (h.k + (light ? h.r : 0)) + 4.0 * d + xy / 2, st, tickets);
+}
+
+// Scratch from the caller's workspace, ticket counters from its control block.
+ffsplit_status launch_decode_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* blob, const void* X,
+                                     long long T, void* Y, char* AP, char* Q, char* HL, char* scratch,
+                                     cudaStream_t st) {
+  return decode_forward_impl(ctx, h, blob, X, T, Y, AP, Q, HL, scratch, st, nullptr);
 }
 
 }  // namespace ffsp
+
+// =====================================================================================
+// Few-token forward that needs no memory from its caller beyond inputs and outputs.
+// =====================================================================================
+namespace {
+
+constexpr int kNoAllocMaxTokens = 8;
+constexpr size_t kNoAllocTicketBytes = ffsp::kCtrlBytes;                 // ticket counters of the K-split reduction
+constexpr size_t kNoAllocPartialBytes = static_cast<size_t>(ffsp::kDecodeMaxPartialRows) * 8 * 4;   // fp32 partials, 8 tokens
+constexpr size_t kNoAllocStageBytes = 2u << 20;                         // A_H | P, Q and the light activations
+constexpr size_t kNoAllocBytes = kNoAllocTicketBytes + kNoAllocPartialBytes + kNoAllocStageBytes;   // 4.06 MiB
+
+// Scratch of ffsplit_forward_noalloc.  Lives in every GPU context that loads the library, from
+// load to exit.  In host code this name is only a handle for cudaGetSymbolAddress -- it is not a
+// device address and must never be handed to a kernel as a pointer.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
+
+constexpr int kMaxDevices = 64;
+char* g_noalloc_ptr[kMaxDevices] = {nullptr};
+
+}  // namespace
+
+extern "C" ffsplit_status ffsplit_forward_noalloc(ffsplit_ctx* ctx, const void* blob, const void* X, int64_t T,
+                                                  void* Y, void* stream) {
+  using namespace ffsp;
+  if (!ctx) return FFSPLIT_ERR_INVALID_ARG;
+  ctx->err.clear();
+  int dev = -1;
+  cudaError_t ce = cudaGetDevice(&dev);
+  if (ce != cudaSuccess) return check_cuda(ctx, ce, "cudaGetDevice");
+  if (dev != ctx->device || dev < 0 || dev >= kMaxDevices)
+    return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "the context's device is not the current device");
+  if (!blob || !X || !Y) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "NULL tensor");
+  if (!aligned16(X) || !aligned16(Y)) return fail(ctx, FFSPLIT_ERR_ALIGN, "X and Y must be 16-byte aligned");
+  if (T < 1 || T > kNoAllocMaxTokens)
+    return fail(ctx, FFSPLIT_ERR_SHAPE, "ffsplit_forward_noalloc handles 1..8 tokens per call");
+  auto it = ctx->blobs.find(blob);
+  if (it == ctx->blobs.end()) {
+    const ffsplit_status s = ffsplit_blob_open(ctx, blob, 0);
+    if (s != FFSPLIT_OK) return s;
+    it = ctx->blobs.find(blob);
+  }
+  const BlobHeader& h = it->second;
+  if (h.dtype != FFSPLIT_BF16) return fail(ctx, FFSPLIT_ERR_DTYPE, "ffsplit_forward_noalloc handles bf16 layers only");
+  // intermediates of one call: [A_H | P], Q, light activations, each 256-byte aligned
+  auto up = [](size_t v) { return (v + 255) / 256 * 256; };
+  const size_t ap_b = up(static_cast<size_t>(T) * (h.k_pad + h.r_pad) * 2);
+  const size_t q_b = up(static_cast<size_t>(T) * h.n_in * h.r_pad * 2);
+  const size_t hl_b = up(static_cast<size_t>(T) * h.ml_pad * 2);
+  if (ap_b + q_b + hl_b > kNoAllocStageBytes)
+    return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL,
+                "layer too wide for the built-in scratch of ffsplit_forward_noalloc (2 MiB of intermediates)");
+  // one-time set-up per device: the device address of the built-in scratch
+  if (!g_noalloc_ptr[dev]) {
+    void* ptr = nullptr;
+    ce = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
+    if (ce != cudaSuccess || !ptr) return check_cuda(ctx, ce != cudaSuccess ? ce : cudaErrorInvalidSymbol, "cudaGetSymbolAddress(scratch)");
+    g_noalloc_ptr[dev] = static_cast<char*>(ptr);
+  }
+  char* base = g_noalloc_ptr[dev];
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // the ticket counters must read zero when the kernels start; the rest is overwritten before it is read
+  ce = cudaMemsetAsync(base, 0, kNoAllocTicketBytes, st);
+  if (ce != cudaSuccess) return check_cuda(ctx, ce, "cudaMemsetAsync(tickets)");
+  char* part = base + kNoAllocTicketBytes;
+  char* AP = part + kNoAllocPartialBytes;
+  char* Q = AP + ap_b;
+  char* HL = Q + q_b;
+  return decode_forward_impl(ctx, h, static_cast<const char*>(blob), X, T, Y, AP, Q, HL, part, st,
+                             reinterpret_cast<int*>(base));
+}
