@@ -183,6 +183,24 @@ def time_region(fn, steps, warmup, flush, dist_barrier):
     return times
 
 
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """The slowest rank's time for a timed region (every rank gets the same number back)."""
+    if world <= 1:
+        return ms
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_tokens_per_s(total_ms: float, tokens_per_rank_step: int, steps: int, world: int, device="cpu") -> float:
+    """Weak scaling: every rank pushes its own batch through its own replica; the job's
+    throughput is all ranks' tokens over the slowest rank's time."""
+    slowest = max_over_ranks(total_ms, world, device)
+    return world * tokens_per_rank_step * steps / (slowest * 1e-3)
+
+
 def flops_per_token(cfg, dense=False):
     n_in = cfg.n_in
     if dense:
@@ -240,11 +258,7 @@ def run_ours(args):
     launches_per_step = (ctx.launch_count() - n0) // (args.steps + args.warmup)
     ctx.poll()
     wl.check_selection_stable()
-    total_ms = sum(step_ms)
-    if world > 1:
-        t = torch.tensor([total_ms], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(sum(step_ms), world, device)
     value = world * T * args.steps / (total_ms * 1e-3)
 
     # ---- phases, each timed the same way (kernel-only, inputs resident)
@@ -287,11 +301,7 @@ def run_ours(args):
         Y_host.copy_(y, non_blocking=True)
 
     e2e_ms = time_region(e2e_step, k_ph, w_ph, flush, barrier)
-    e2e_total = sum(e2e_ms)
-    if world > 1:
-        t = torch.tensor([e2e_total], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_total = float(t.item())
+    e2e_total = max_over_ranks(sum(e2e_ms), world, device)
     es = 2
     h2d = cfg.layers * cfg.t_cal * cfg.d * es + T * cfg.d * es
     d2h = T * cfg.d * es
