@@ -6,8 +6,8 @@
 //   warp 0  (one lane)  TMA producer: global -> 128B-swizzled shared tiles, ring of up to 8 stages
 //   warp 1  (one lane)  tcgen05.mma issuer; accumulators live in tensor memory (TMEM),
 //                       two buffers so the epilogue of tile i overlaps the MMAs of tile i+1
-//   warps 2-9           epilogue: tcgen05.ld -> bias / activation / gating -> global; two warps
-//                       per TMEM lane quarter, taking alternate 16-column chunks
+//   warps 2-17          epilogue: tcgen05.ld -> bias / activation / gating -> global; four warps
+//                       per TMEM lane quarter, taking every fourth 16-column chunk
 // The gated form (SwiGLU) runs two operand pairs into two accumulators of the same
 // tile and combines them as silu(acc0) * acc1.
 // The score form does not store the tile; it reduces act(acc)^2 over the tile's rows
@@ -30,8 +30,8 @@ constexpr int A_STAGE_BYTES = BLOCK_M * BLOCK_K * 2;
 constexpr int TMEM_COLS = 512;
 constexpr int ACC_STRIDE = 256;   // TMEM columns per accumulator buffer
 constexpr int GATE_OFFSET = 128;  // second accumulator of a gated tile
-constexpr int NUM_THREADS = 320;
-constexpr int EPI_WARPS = 8;
+constexpr int EPI_WARPS = 16;
+constexpr int NUM_THREADS = 32 * (EPI_WARPS + 2);
 constexpr int BAR_BYTES = 256;
 constexpr int MAX_SMEM = 232448;
 
@@ -246,7 +246,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   } else {
     // -------------------------------------------------------------- epilogue warps
     const int q = warp & 3;             // TMEM lane quarter this warp may read
-    const int half = (warp - 2) >> 2;   // which alternate 16-column chunks this warp takes
+    const int half = (warp - 2) >> 2;   // which of every EPI_WARPS / 4 consecutive 16-column chunks this warp takes
     const GeluCoef gc = gelu_coef(p.epi.act);
     uint32_t tl = 0;
     for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++tl) {
@@ -261,7 +261,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       ptx::tc_fence_after();
       const long long row = static_cast<long long>(m_blk) * BLOCK_M + q * 32 + lane;
       const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * ACC_STRIDE;
-      for (int c = half * 16; c < p.block_n; c += 32) {
+      for (int c = half * 16; c < p.block_n; c += 4 * EPI_WARPS) {
         const int n0 = n_blk * p.block_n + c;
         if (n0 >= p.N) break;
         float v[16];
