@@ -169,6 +169,8 @@ ScoreLayout score_layout(const ffsplit_shape& s, long long T) {
 ffsplit_status check_ctx(ffsplit_ctx* ctx, bool need_ws) {
   if (!ctx) return FFSPLIT_ERR_INVALID_ARG;
   ctx->err.clear();
+  ctx->prep_active = false;   // a batch left open by a call that failed half-way is dropped
+  ctx->prep.n = 0;
   int dev = -1;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return check_cuda(ctx, e, "cudaGetDevice");
@@ -428,7 +430,8 @@ ffsplit_status ffsplit_score(ffsplit_ctx* ctx, const ffsplit_shape* shape, const
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   char* base = ctx->ws + kCtrlBytes;
   const int d = shape->d, m = shape->m, dt = shape->dtype;
-  // U^T (K-major for the contraction over d)
+  // U^T (K-major for the contraction over d), fp32 bias, ||V_j||^2: one batched launch
+  prep_begin(ctx);
   if ((s = launch_transpose(ctx, dt, wt->W1, m, d, m, base + L.w1t, d, d, m, nullptr, d, st)) != FFSPLIT_OK) return s;
   if (gated && (s = launch_transpose(ctx, dt, wt->W1u, m, d, m, base + L.w1ut, d, d, m, nullptr, d, st)) != FFSPLIT_OK)
     return s;
@@ -439,6 +442,7 @@ ffsplit_status ffsplit_score(ffsplit_ctx* ctx, const ffsplit_shape* shape, const
   if (scores && mode != FFSPLIT_SCORE_ACT_ONLY &&
       (s = launch_row_energy(ctx, dt, wt->W2, m, d, w, st)) != FFSPLIT_OK)
     return s;
+  if ((s = prep_flush(ctx, dt, st)) != FFSPLIT_OK) return s;
   GemmArgs g;
   std::memset(&g, 0, sizeof(g));
   g.A0 = X; g.lda0 = d; g.B0 = base + L.w1t; g.ldb0 = d;
@@ -499,7 +503,9 @@ ffsplit_status ffsplit_pack(ffsplit_ctx* ctx, const ffsplit_shape* shape, const 
   char* b = static_cast<char*>(blob);
   const int d = shape->d, m = shape->m, dt = shape->dtype;
   const size_t es = elem_size(dt);
-  // heavy slices: U1^T = (U[:, h2])^T, V1 = V[h2, :] -- plain copies of the inputs
+  // heavy slices: U1^T = (U[:, h2])^T, V1 = V[h2, :] -- plain copies of the inputs; all of the
+  // gathers, transposes and bias conversions of the layer run as one batched launch
+  prep_begin(ctx);
   if ((s = launch_gather_cols_t(ctx, dt, wt->W1, m, d, heavy_idx, k, m, b + h.off[SEC_U1T], d, D.k_pad, st)) != FFSPLIT_OK)
     return s;
   if (gated &&
@@ -525,9 +531,10 @@ ffsplit_status ffsplit_pack(ffsplit_ctx* ctx, const ffsplit_shape* shape, const 
                             D.k_pad, reinterpret_cast<float*>(b + h.off[SEC_B1L]), D.ml_pad,
                             reinterpret_cast<float*>(b + h.off[SEC_B2]), st)) != FFSPLIT_OK)
     return s;
-  cudaError_t e = cudaMemcpyAsync(blob, &h, sizeof(h), cudaMemcpyHostToDevice, st);
+  if ((s = prep_flush(ctx, dt, st)) != FFSPLIT_OK) return s;
+  ctx->blobs[blob] = h;   // the copy below reads this entry, which outlives the call
+  cudaError_t e = cudaMemcpyAsync(blob, &ctx->blobs[blob], sizeof(h), cudaMemcpyHostToDevice, st);
   if (e != cudaSuccess) return check_cuda(ctx, e, "cudaMemcpyAsync(blob header)");
-  ctx->blobs[blob] = h;
   return FFSPLIT_OK;
 }
 

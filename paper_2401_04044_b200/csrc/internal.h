@@ -103,6 +103,24 @@ enum Section : int {
 };
 
 // ----------------------------------------------------------------------------
+// Batched preparation jobs (see kernels_misc.cu)
+// ----------------------------------------------------------------------------
+constexpr int kMaxPrepJobs = 12;
+struct PrepJob {
+  int kind;
+  int rows, cols, rows_pad, cols_pad, idx_limit;
+  int tiles_x, block_begin;
+  long long ldi, ldo;
+  const void* in; const void* in2;
+  void* out; void* out2; void* out3;
+  const int* idx;
+};
+struct PrepBatch {
+  PrepJob job[kMaxPrepJobs];
+  int n;
+};
+
+// ----------------------------------------------------------------------------
 // Host context
 // ----------------------------------------------------------------------------
 struct TmapKey {
@@ -137,6 +155,9 @@ struct ffsplit_ctx {
   struct ProfRec { int cls; cudaEvent_t a, b; double work; };
   bool profiling = false;
   std::vector<ProfRec> prof;
+  ffsp::PrepBatch prep{};
+  int prep_blocks = 0;
+  bool prep_active = false;
   bool attr_tc_set = false;
   bool attr_fused_set = false;
   int* status() const { return reinterpret_cast<int*>(ws); }
@@ -158,6 +179,10 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 enum ProfClass : int { PROF_GEMM_TC = 0, PROF_GEMM_SIMT = 1, PROF_DECODE = 2 };
 int prof_open(ffsplit_ctx* ctx, int cls, double work, cudaStream_t st);
 void prof_close(ffsplit_ctx* ctx, int handle, cudaStream_t st);
+
+// preparation jobs recorded between these two calls run as one launch
+void prep_begin(ffsplit_ctx* ctx);
+ffsplit_status prep_flush(ffsplit_ctx* ctx, int dtype, cudaStream_t st);
 
 // launchers (each returns a CUDA error state through check_cuda)
 ffsplit_status launch_gemm(ffsplit_ctx* ctx, int dtype, const GemmArgs& g, cudaStream_t st);

@@ -53,18 +53,32 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
         if ((kv & mask) == prefix) atomicAdd(&hist[(kv >> shift) & 255u], 1u);
       }
       __syncthreads();
-      if (tid == 0) {
-        unsigned cum = 0u, remaining = s_remaining;
-        for (int b = 255; b >= 0; --b) {
-          const unsigned c = hist[b];
-          if (cum + c >= remaining) {
-            s_prefix = prefix | (static_cast<unsigned>(b) << shift);
-            s_remaining = remaining - cum;
-            break;
-          }
-          cum += c;
+      if (warp == 0) {
+        // lane l owns bins 8l .. 8l+7; counts of all higher bins by a shuffle suffix scan
+        unsigned mine = 0u;
+#pragma unroll
+        for (int b = 0; b < 8; ++b) mine += hist[8 * lane + b];
+        unsigned incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const unsigned up = __shfl_down_sync(0xffffffffu, incl, o);
+          if (lane + o < 32) incl += up;
         }
-        s_mask = mask | (255u << shift);
+        const unsigned above = incl - mine, remaining = s_remaining;
+        __syncwarp();
+        if (above < remaining && remaining <= above + mine) {   // exactly one lane
+          unsigned cum = above;
+          for (int b = 8 * lane + 7; b >= 8 * lane; --b) {
+            const unsigned c = hist[b];
+            if (cum + c >= remaining) {
+              s_prefix = prefix | (static_cast<unsigned>(b) << shift);
+              s_remaining = remaining - cum;
+              break;
+            }
+            cum += c;
+          }
+        }
+        if (lane == 0) s_mask = mask | (255u << shift);
       }
       __syncthreads();
     }
@@ -130,15 +144,113 @@ ffsplit_status launch_select(ffsplit_ctx* ctx, const float* scores, int m, int k
 }
 
 // ============================================================================
-// w_j = sum_c W2[j, c]^2   (Eq. 3, ||V_{j,:}||^2): one warp per row, 128-bit loads,
-// lane-strided partial sums combined by a fixed shuffle tree.
+// e_j (+)= sum over row groups of the per-group column partials, in a fixed
+// order (8 interleaved slices of the groups, then the 8 slice sums in order);
+// then the score of the chosen reading.
 // ============================================================================
+__global__ void __launch_bounds__(256) score_finalize_kernel(const float* __restrict__ partial, int groups, int m,
+                                                             const float* __restrict__ w, float* __restrict__ energy,
+                                                             float* __restrict__ scores, int mode, int accumulate) {
+  __shared__ float part[8][32];
+  const int cx = threadIdx.x & 31, gy = threadIdx.x >> 5;
+  const int j = blockIdx.x * 32 + cx;
+  float s = 0.f;
+  if (j < m)
+    for (int g = gy; g < groups; g += 8) s += partial[static_cast<long long>(g) * m + j];
+  part[gy][cx] = s;
+  __syncthreads();
+  if (gy != 0 || j >= m) return;
+  float tot = 0.f;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) tot += part[i][cx];
+  const float e = accumulate ? energy[j] + tot : tot;
+  energy[j] = e;
+  if (scores) {
+    float v = e;
+    if (mode == FFSPLIT_SCORE_EQ3) v = e * w[j];
+    else if (mode == FFSPLIT_SCORE_SUM_NORM) v = e * sqrtf(w[j]);
+    scores[j] = v;
+  }
+}
+
+ffsplit_status launch_score_finalize(ffsplit_ctx* ctx, const float* partial, int groups, int m, const float* w,
+                                     float* energy, float* scores, int mode, int accumulate, cudaStream_t st) {
+  score_finalize_kernel<<<(m + 31) / 32, 256, 0, st>>>(partial, groups, m, w, energy, scores, mode, accumulate);
+  ctx->launches++;
+  return check_cuda(ctx, cudaGetLastError(), "score_finalize_kernel launch");
+}
+
+// ============================================================================
+// Small data-movement and reduction jobs of scoring and packing, batched: the
+// jobs recorded between prep_begin() and prep_flush() run as ONE launch whose
+// blocks are dealt out to the jobs (each job is far too small to fill the GPU,
+// and a launch per job costs more than the job).
+//   TRANSPOSE   OUT[c, j] = IN[src(j), c], zero padded   (factors, V1 = V[h2, :], U^T)
+//   GATHER      OUT[j, i] = IN[i, idx[j]], zero padded   (U1^T = (U[:, h2])^T)
+//   TO_F32      out[i] = float(in[i])
+//   ROW_ENERGY  w_j = sum_c W2[j, c]^2                   (Eq. 3, ||V_{j,:}||^2)
+//   PACK_BIAS   b1[h2], b1[light], b2 in fp32 + validation of h2
+// ============================================================================
+enum PrepKind : int { PREP_TRANSPOSE = 0, PREP_GATHER = 1, PREP_TO_F32 = 2, PREP_ROW_ENERGY = 3, PREP_PACK_BIAS = 4 };
+
 template <typename T>
-__global__ void __launch_bounds__(256) row_energy_kernel(const T* __restrict__ W, int m, int d, float* __restrict__ w) {
-  const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+__device__ __forceinline__ void transpose_tile(const PrepJob& q, int bx, int by, T (*tile)[33]) {
+  // OUT[c, j] = IN[src(j), c] for j < rows, c < cols; zero elsewhere in the padded output
+  // [cols_pad, rows_pad].  src(j) = idx ? idx[j] : j; a source row outside [0, idx_limit) reads as zeros.
+  const T* in = static_cast<const T*>(q.in);
+  T* out = static_cast<T*>(q.out);
+  const int j0 = bx * 32, c0 = by * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;  // 32 x 8
+  for (int jj = ty; jj < 32; jj += 8) {
+    const int j = j0 + jj, c = c0 + tx;
+    T v = from_float<T>(0.f);
+    if (j < q.rows && c < q.cols) {
+      const int src = q.idx ? q.idx[j] : j;
+      if (src >= 0 && src < q.idx_limit) v = in[static_cast<long long>(src) * q.ldi + c];
+    }
+    tile[jj][tx] = v;
+  }
+  __syncthreads();
+  for (int cc = ty; cc < 32; cc += 8) {
+    const int c = c0 + cc, j = j0 + tx;
+    if (c < q.cols_pad && j < q.rows_pad) out[static_cast<long long>(c) * q.ldo + j] = tile[tx][cc];
+  }
+}
+
+template <typename T>
+__device__ __forceinline__ void gather_tile(const PrepJob& q, int bx, int by, T (*tile)[33]) {
+  // OUT[j, i] = IN[i, idx[j]] for j < cols (count of gathered columns), i < rows; zero rows up to rows_pad
+  const T* in = static_cast<const T*>(q.in);
+  T* out = static_cast<T*>(q.out);
+  const int j0 = bx * 32, i0 = by * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  const int j = j0 + tx;
+  int src = -1;
+  if (j < q.cols) {
+    src = q.idx[j];
+    if (src < 0 || src >= q.idx_limit) src = -1;
+  }
+  for (int ii = ty; ii < 32; ii += 8) {
+    const int i = i0 + ii;
+    T v = from_float<T>(0.f);
+    if (src >= 0 && i < q.rows) v = in[static_cast<long long>(i) * q.ldi + src];
+    tile[ii][tx] = v;
+  }
+  __syncthreads();
+  for (int jj = ty; jj < 32; jj += 8) {
+    const int jo = j0 + jj, i = i0 + tx;
+    if (jo < q.rows_pad && i < q.rows) out[static_cast<long long>(jo) * q.ldo + i] = tile[tx][jj];
+  }
+}
+
+template <typename T>
+__device__ __forceinline__ void row_energy_rows(const PrepJob& q, int blk) {
+  // one warp per row, 128-bit loads, lane-strided partial sums combined by a fixed shuffle tree
+  const int row = blk * 8 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
-  if (row >= m) return;
-  const T* p = W + static_cast<long long>(row) * d;
+  if (row >= q.rows) return;
+  const int d = q.cols;
+  const T* p = static_cast<const T*>(q.in) + static_cast<long long>(row) * d;
   constexpr int VEC = 16 / sizeof(T);
   float s = 0.f;
   if (d % VEC == 0 && (reinterpret_cast<uintptr_t>(p) & 15u) == 0) {
@@ -159,145 +271,20 @@ __global__ void __launch_bounds__(256) row_energy_kernel(const T* __restrict__ W
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-  if (lane == 0) w[row] = s;
+  if (lane == 0) static_cast<float*>(q.out)[row] = s;
 }
 
-ffsplit_status launch_row_energy(ffsplit_ctx* ctx, int dtype, const void* W2, int m, int d, float* w, cudaStream_t st) {
-  const int grid = (m + 7) / 8;
-  if (dtype == FFSPLIT_BF16)
-    row_energy_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(W2), m, d, w);
-  else
-    row_energy_kernel<float><<<grid, 256, 0, st>>>(static_cast<const float*>(W2), m, d, w);
-  ctx->launches++;
-  return check_cuda(ctx, cudaGetLastError(), "row_energy_kernel launch");
-}
-
-// ============================================================================
-// e_j (+)= sum over row groups of the per-group column partials, in a fixed
-// order; then the score of the chosen reading.
-// ============================================================================
-__global__ void score_finalize_kernel(const float* __restrict__ partial, int groups, int m,
-                                      const float* __restrict__ w, float* __restrict__ energy,
-                                      float* __restrict__ scores, int mode, int accumulate) {
-  const int j = blockIdx.x * blockDim.x + threadIdx.x;
-  if (j >= m) return;
-  float s = 0.f;
-  for (int g = 0; g < groups; ++g) s += partial[static_cast<long long>(g) * m + j];
-  const float e = accumulate ? energy[j] + s : s;
-  energy[j] = e;
-  if (scores) {
-    float v = e;
-    if (mode == FFSPLIT_SCORE_EQ3) v = e * w[j];
-    else if (mode == FFSPLIT_SCORE_SUM_NORM) v = e * sqrtf(w[j]);
-    scores[j] = v;
-  }
-}
-
-ffsplit_status launch_score_finalize(ffsplit_ctx* ctx, const float* partial, int groups, int m, const float* w,
-                                     float* energy, float* scores, int mode, int accumulate, cudaStream_t st) {
-  score_finalize_kernel<<<(m + 255) / 256, 256, 0, st>>>(partial, groups, m, w, energy, scores, mode, accumulate);
-  ctx->launches++;
-  return check_cuda(ctx, cudaGetLastError(), "score_finalize_kernel launch");
-}
-
-// ============================================================================
-// Pack helpers (Figure 3 caption: U1 = U[:, h2], V1 = V[h2, :]).
-// ============================================================================
-// OUT[c, j] = IN[src(j), c] for j < rows, c < cols; zero elsewhere in the padded
-// output [cols_pad, rows_pad].  src(j) = row_idx ? row_idx[j] : j; a source row
-// outside [0, idx_limit) reads as zeros.
 template <typename T>
-__global__ void __launch_bounds__(256) transpose_kernel(const T* __restrict__ in, long long ldi, int rows, int cols,
-                                                        T* __restrict__ out, long long ldo, int rows_pad,
-                                                        int cols_pad, const int* __restrict__ row_idx, int idx_limit) {
-  __shared__ T tile[32][33];
-  const int j0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
-  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;  // 32 x 8
-  for (int jj = ty; jj < 32; jj += 8) {
-    const int j = j0 + jj, c = c0 + tx;
-    T v = from_float<T>(0.f);
-    if (j < rows && c < cols) {
-      const int src = row_idx ? row_idx[j] : j;
-      if (src >= 0 && src < idx_limit) v = in[static_cast<long long>(src) * ldi + c];
-    }
-    tile[jj][tx] = v;
-  }
-  __syncthreads();
-  for (int cc = ty; cc < 32; cc += 8) {
-    const int c = c0 + cc, j = j0 + tx;
-    if (c < cols_pad && j < rows_pad) out[static_cast<long long>(c) * ldo + j] = tile[tx][cc];
-  }
-}
-
-ffsplit_status launch_transpose(ffsplit_ctx* ctx, int dtype, const void* in, long long ldi, int rows, int cols,
-                                void* out, long long ldo, int rows_pad_out, int cols_pad_out, const int* row_idx,
-                                int idx_limit, cudaStream_t st) {
-  if (rows_pad_out <= 0 || cols_pad_out <= 0) return FFSPLIT_OK;
-  dim3 grid((rows_pad_out + 31) / 32, (cols_pad_out + 31) / 32);
-  if (grid.y > 65535) return fail(ctx, FFSPLIT_ERR_SHAPE, "matrix too wide for the transpose kernel");
-  if (dtype == FFSPLIT_BF16)
-    transpose_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(in), ldi, rows, cols,
-                                                          static_cast<__nv_bfloat16*>(out), ldo, rows_pad_out,
-                                                          cols_pad_out, row_idx, idx_limit);
-  else
-    transpose_kernel<float><<<grid, 256, 0, st>>>(static_cast<const float*>(in), ldi, rows, cols,
-                                                  static_cast<float*>(out), ldo, rows_pad_out, cols_pad_out, row_idx,
-                                                  idx_limit);
-  ctx->launches++;
-  return check_cuda(ctx, cudaGetLastError(), "transpose_kernel launch");
-}
-
-// OUT[j, i] = IN[i, col_idx[j]] for j < ncols, i < rows; zero rows for ncols <= j < rows_out_pad.
-template <typename T>
-__global__ void __launch_bounds__(256) gather_cols_kernel(const T* __restrict__ in, long long ldi, int rows,
-                                                          const int* __restrict__ col_idx, int ncols, int idx_limit,
-                                                          T* __restrict__ out, long long ldo, int rows_out_pad) {
-  __shared__ T tile[32][33];
-  const int j0 = blockIdx.x * 32, i0 = blockIdx.y * 32;
-  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-  const int j = j0 + tx;
-  int src = -1;
-  if (j < ncols) {
-    src = col_idx[j];
-    if (src < 0 || src >= idx_limit) src = -1;
-  }
-  for (int ii = ty; ii < 32; ii += 8) {
-    const int i = i0 + ii;
-    T v = from_float<T>(0.f);
-    if (src >= 0 && i < rows) v = in[static_cast<long long>(i) * ldi + src];
-    tile[ii][tx] = v;
-  }
-  __syncthreads();
-  for (int jj = ty; jj < 32; jj += 8) {
-    const int jo = j0 + jj, i = i0 + tx;
-    if (jo < rows_out_pad && i < rows) out[static_cast<long long>(jo) * ldo + i] = tile[tx][jj];
-  }
-}
-
-ffsplit_status launch_gather_cols_t(ffsplit_ctx* ctx, int dtype, const void* in, long long ldi, int rows,
-                                    const int* col_idx, int ncols, int idx_limit, void* out, long long ldo,
-                                    int rows_out_pad, cudaStream_t st) {
-  if (rows_out_pad <= 0 || rows <= 0) return FFSPLIT_OK;
-  dim3 grid((rows_out_pad + 31) / 32, (rows + 31) / 32);
-  if (grid.y > 65535) return fail(ctx, FFSPLIT_ERR_SHAPE, "matrix too tall for the gather kernel");
-  if (dtype == FFSPLIT_BF16)
-    gather_cols_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(in), ldi, rows, col_idx,
-                                                            ncols, idx_limit, static_cast<__nv_bfloat16*>(out), ldo,
-                                                            rows_out_pad);
-  else
-    gather_cols_kernel<float><<<grid, 256, 0, st>>>(static_cast<const float*>(in), ldi, rows, col_idx, ncols,
-                                                    idx_limit, static_cast<float*>(out), ldo, rows_out_pad);
-  ctx->launches++;
-  return check_cuda(ctx, cudaGetLastError(), "gather_cols_kernel launch");
-}
-
-// Biases in fp32: b1[h2] (zero padded), b1[light] (zero padded), b2; also checks
-// that heavy_idx is strictly ascending and in range.
-template <typename T>
-__global__ void pack_bias_kernel(const T* __restrict__ b1, const T* __restrict__ b2, const int* __restrict__ heavy,
-                                 int m, int k, int d, float* __restrict__ b1h, int k_pad, float* __restrict__ b1l,
-                                 int ml_pad, float* __restrict__ b2o, int* status) {
-  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+__device__ __forceinline__ void pack_bias_chunk(const PrepJob& q, int blk, int* status) {
+  // rows = m, cols = k, rows_pad = d, cols_pad = k_pad, idx_limit = ml_pad; in = b1, in2 = b2, idx = h2
+  const T* b1 = static_cast<const T*>(q.in);
+  const T* b2 = static_cast<const T*>(q.in2);
+  const int* heavy = q.idx;
+  float* b1h = static_cast<float*>(q.out);
+  float* b1l = static_cast<float*>(q.out2);
+  float* b2o = static_cast<float*>(q.out3);
+  const int m = q.rows, k = q.cols, d = q.rows_pad, k_pad = q.cols_pad, ml_pad = q.idx_limit;
+  const int j = blk * 256 + threadIdx.x;
   if (j < k) {
     const int h = heavy[j];
     if (h < 0 || h >= m || (j > 0 && heavy[j - 1] >= h)) record_status(status, FFSPLIT_ERR_BAD_INDEX, j, KID_PACK);
@@ -318,6 +305,84 @@ __global__ void pack_bias_kernel(const T* __restrict__ b1, const T* __restrict__
   if (j < d) b2o[j] = b2 ? to_float<T>(b2[j]) : 0.f;
 }
 
+template <typename T>
+__global__ void __launch_bounds__(256) prep_kernel(const PrepBatch batch, int* status) {
+  __shared__ T tile[32][33];
+  int i = 0;
+  while (i + 1 < batch.n && static_cast<int>(blockIdx.x) >= batch.job[i + 1].block_begin) ++i;
+  const PrepJob& q = batch.job[i];
+  const int local = blockIdx.x - q.block_begin;
+  switch (q.kind) {
+    case PREP_TRANSPOSE: transpose_tile<T>(q, local % q.tiles_x, local / q.tiles_x, tile); break;
+    case PREP_GATHER: gather_tile<T>(q, local % q.tiles_x, local / q.tiles_x, tile); break;
+    case PREP_TO_F32: {
+      const int e = local * 256 + threadIdx.x;
+      if (e < q.rows) static_cast<float*>(q.out)[e] = q.in ? to_float<T>(static_cast<const T*>(q.in)[e]) : 0.f;
+      break;
+    }
+    case PREP_ROW_ENERGY: row_energy_rows<T>(q, local); break;
+    default: pack_bias_chunk<T>(q, local, status); break;
+  }
+}
+
+void prep_begin(ffsplit_ctx* ctx) {
+  ctx->prep.n = 0;
+  ctx->prep_blocks = 0;
+  ctx->prep_active = true;
+}
+
+ffsplit_status prep_flush(ffsplit_ctx* ctx, int dtype, cudaStream_t st) {
+  ctx->prep_active = false;
+  if (ctx->prep.n == 0) return FFSPLIT_OK;
+  const int blocks = ctx->prep_blocks;
+  if (dtype == FFSPLIT_BF16) prep_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(ctx->prep, ctx->status());
+  else prep_kernel<float><<<blocks, 256, 0, st>>>(ctx->prep, ctx->status());
+  ctx->prep.n = 0;
+  ctx->launches++;
+  return check_cuda(ctx, cudaGetLastError(), "prep_kernel launch");
+}
+
+// Records a job; outside a prep_begin/prep_flush bracket the job is launched on its own.
+static ffsplit_status add_job(ffsplit_ctx* ctx, int dtype, PrepJob q, long long blocks, cudaStream_t st) {
+  if (blocks <= 0) return FFSPLIT_OK;
+  const bool single = !ctx->prep_active;
+  if (single) prep_begin(ctx);
+  if (ctx->prep.n >= kMaxPrepJobs || ctx->prep_blocks + blocks > 0x7fffffffLL)
+    return fail(ctx, FFSPLIT_ERR_SHAPE, "too many or too large preparation jobs in one batch");
+  q.block_begin = ctx->prep_blocks;
+  ctx->prep.job[ctx->prep.n++] = q;
+  ctx->prep_blocks += static_cast<int>(blocks);
+  return single ? prep_flush(ctx, dtype, st) : FFSPLIT_OK;
+}
+
+ffsplit_status launch_row_energy(ffsplit_ctx* ctx, int dtype, const void* W2, int m, int d, float* w, cudaStream_t st) {
+  PrepJob q{};
+  q.kind = PREP_ROW_ENERGY; q.in = W2; q.rows = m; q.cols = d; q.out = w;
+  return add_job(ctx, dtype, q, (m + 7) / 8, st);
+}
+
+ffsplit_status launch_transpose(ffsplit_ctx* ctx, int dtype, const void* in, long long ldi, int rows, int cols,
+                                void* out, long long ldo, int rows_pad_out, int cols_pad_out, const int* row_idx,
+                                int idx_limit, cudaStream_t st) {
+  if (rows_pad_out <= 0 || cols_pad_out <= 0) return FFSPLIT_OK;
+  PrepJob q{};
+  q.kind = PREP_TRANSPOSE; q.in = in; q.ldi = ldi; q.rows = rows; q.cols = cols; q.out = out; q.ldo = ldo;
+  q.rows_pad = rows_pad_out; q.cols_pad = cols_pad_out; q.idx = row_idx; q.idx_limit = idx_limit;
+  q.tiles_x = (rows_pad_out + 31) / 32;
+  return add_job(ctx, dtype, q, static_cast<long long>(q.tiles_x) * ((cols_pad_out + 31) / 32), st);
+}
+
+ffsplit_status launch_gather_cols_t(ffsplit_ctx* ctx, int dtype, const void* in, long long ldi, int rows,
+                                    const int* col_idx, int ncols, int idx_limit, void* out, long long ldo,
+                                    int rows_out_pad, cudaStream_t st) {
+  if (rows_out_pad <= 0 || rows <= 0) return FFSPLIT_OK;
+  PrepJob q{};
+  q.kind = PREP_GATHER; q.in = in; q.ldi = ldi; q.rows = rows; q.cols = ncols; q.idx = col_idx; q.idx_limit = idx_limit;
+  q.out = out; q.ldo = ldo; q.rows_pad = rows_out_pad;
+  q.tiles_x = (rows_out_pad + 31) / 32;
+  return add_job(ctx, dtype, q, static_cast<long long>(q.tiles_x) * ((rows + 31) / 32), st);
+}
+
 ffsplit_status launch_pack_bias(ffsplit_ctx* ctx, int dtype, const void* b1, const void* b2, const int* heavy, int m,
                                 int k, int d, float* b1h, int k_pad, float* b1l, int ml_pad, float* b2o,
                                 cudaStream_t st) {
@@ -325,33 +390,17 @@ ffsplit_status launch_pack_bias(ffsplit_ctx* ctx, int dtype, const void* b1, con
   if (k_pad > n) n = k_pad;
   if (ml_pad > n) n = ml_pad;
   if (d > n) n = d;
-  const int grid = (n + 255) / 256;
-  if (dtype == FFSPLIT_BF16)
-    pack_bias_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(b1),
-                                                          static_cast<const __nv_bfloat16*>(b2), heavy, m, k, d, b1h,
-                                                          k_pad, b1l, ml_pad, b2o, ctx->status());
-  else
-    pack_bias_kernel<float><<<grid, 256, 0, st>>>(static_cast<const float*>(b1), static_cast<const float*>(b2), heavy,
-                                                  m, k, d, b1h, k_pad, b1l, ml_pad, b2o, ctx->status());
-  ctx->launches++;
-  return check_cuda(ctx, cudaGetLastError(), "pack_bias_kernel launch");
-}
-
-// out[i] = float(in[i]); a NULL input gives zeros.
-template <typename T>
-__global__ void to_f32_kernel(const T* __restrict__ in, int n, float* __restrict__ out) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) out[i] = in ? to_float<T>(in[i]) : 0.f;
+  PrepJob q{};
+  q.kind = PREP_PACK_BIAS; q.in = b1; q.in2 = b2; q.idx = heavy; q.rows = m; q.cols = k; q.rows_pad = d;
+  q.cols_pad = k_pad; q.idx_limit = ml_pad; q.out = b1h; q.out2 = b1l; q.out3 = b2o;
+  return add_job(ctx, dtype, q, (n + 255) / 256, st);
 }
 
 ffsplit_status launch_to_f32(ffsplit_ctx* ctx, int dtype, const void* in, int n, float* out, cudaStream_t st) {
   if (n <= 0) return FFSPLIT_OK;
-  if (dtype == FFSPLIT_BF16)
-    to_f32_kernel<__nv_bfloat16><<<(n + 255) / 256, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(in), n, out);
-  else
-    to_f32_kernel<float><<<(n + 255) / 256, 256, 0, st>>>(static_cast<const float*>(in), n, out);
-  ctx->launches++;
-  return check_cuda(ctx, cudaGetLastError(), "to_f32_kernel launch");
+  PrepJob q{};
+  q.kind = PREP_TO_F32; q.in = in; q.rows = n; q.out = out;
+  return add_job(ctx, dtype, q, (n + 255) / 256, st);
 }
 
 }  // namespace ffsp
