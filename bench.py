@@ -253,9 +253,25 @@ def run_ours(args):
         return
 
     sampler = ClockSampler(local_rank) if rank == 0 else None
+    # The step is launch-bound on the host (about a hundred launches of 5-50 us): capture it once in a
+    # CUDA graph and time replays.  --no-graph times the plain stream launches instead.
+    wl.step()
+    ctx.poll()
     n0 = ctx.launch_count()
-    step_ms = time_region(wl.step, args.steps, args.warmup, flush, barrier)
-    launches_per_step = (ctx.launch_count() - n0) // (args.steps + args.warmup)
+    wl.step()
+    launches_per_step = ctx.launch_count() - n0
+    ctx.poll()
+    step_fn, launch_mode = wl.step, "stream"
+    if not args.no_graph:
+        try:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                wl.step()
+            step_fn, launch_mode = graph.replay, "cuda_graph"
+        except Exception as exc:   # capture refused: fall back to stream launches, and say so
+            launch_mode = f"stream (graph capture failed: {type(exc).__name__})"
+            torch.cuda.synchronize()
+    step_ms = time_region(step_fn, args.steps, args.warmup, flush, barrier)
     ctx.poll()
     wl.check_selection_stable()
     total_ms = max_over_ranks(sum(step_ms), world, device)
@@ -326,6 +342,7 @@ def run_ours(args):
                                    "4096 calibration tokens/layer, prefill 32x128=4096 tokens; step = score+select+pack "
                                    "per layer, then the 12-layer split forward",
                        "l2": "256 MiB buffer rewritten before every timed step (L2 flush)",
+                       "launch": launch_mode,
                        "tokens_per_step": T, "layers": cfg.layers},
             "roofline": roofline,
             "e2e": e2e,
@@ -453,6 +470,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of a CUDA-graph replay")
     ap.add_argument("--only", default=None, choices=["step", "forward", "dense", "calibrate"],
                     help="run one phase alone and print its times (for profiler captures)")
     ap.add_argument("--layers", type=int, default=0, help="with --only: number of layers of the stack to build")
