@@ -133,7 +133,10 @@ __global__ void __launch_bounds__(THREADS, 1) decode_gemm_kernel(const Params p)
   // two steps of weights in flight per warp
   uint4 wa[RT][2], wb[RT][2];
   int s = s_lo;
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next product may start its own prologue
   if (s < s_hi) load_w(wa, s);
+  // everything below reads or writes what the previous kernel of the stream produced or still reads
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   while (s < s_hi) {
     if (s + 1 < s_hi) load_w(wb, s + 1);
     compute(wa, s);
@@ -237,8 +240,17 @@ cudaError_t launch_one(const Params& p, int row_groups, cudaStream_t st) {
     if (e != cudaSuccess) return e;
     attr_done = true;
   }
-  decode_gemm_kernel<RT, NT, DUAL><<<dim3(row_groups, p.splits), THREADS, smem, st>>>(p);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(row_groups, p.splits);
+  cfg.blockDim = dim3(THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, decode_gemm_kernel<RT, NT, DUAL>, p);
 }
 
 }  // namespace dec
