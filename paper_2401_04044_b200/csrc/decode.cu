@@ -276,10 +276,13 @@ static ffsplit_status decode_gemm(ffsplit_ctx* ctx, const void* X0, const void* 
   const int out_rows = dual ? 8 * rt : 16 * rt;
   const int row_groups = (N + out_rows - 1) / out_rows;
   if (row_groups > kMaxTicketTiles) return fail(ctx, FFSPLIT_ERR_SHAPE, "decode: too many row groups");
-  // enough CTAs to keep every SM streaming, each warp keeping at least two k steps, partials bounded
-  int splits = (2 * ctx->num_sms + row_groups - 1) / row_groups;
+  // Several waves of small CTAs (less loss in the last, partly filled wave), each warp keeping at
+  // least two k steps, the fp32 partials (written and read once) at most ~12 % of the weight bytes.
+  int splits = (ctx->decode_ctas_per_sm_target * ctx->num_sms + row_groups - 1) / row_groups;
   const int max_by_k = p.steps_total / (2 * dec::WARPS);
   if (splits > max_by_k) splits = max_by_k;
+  const int max_by_traffic = static_cast<int>(0.03 * K / (8 * nt));
+  if (splits > max_by_traffic) splits = max_by_traffic;
   if (splits > 16) splits = 16;
   const long long rows_slots = static_cast<long long>(row_groups) * 16 * rt;
   if (splits > 1 && splits * rows_slots > kDecodeMaxPartialRows) splits = static_cast<int>(kDecodeMaxPartialRows / rows_slots);

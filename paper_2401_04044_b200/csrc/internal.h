@@ -162,6 +162,7 @@ struct ffsplit_ctx {
   bool attr_fused_set = false;
   int* status() const { return reinterpret_cast<int*>(ws); }
   int* tickets() const { return reinterpret_cast<int*>(ws + ffsp::kStatusBytes); }
+  int decode_ctas_per_sm_target = 6;   // CTAs per SM the few-token kernels aim for when splitting K (FFSPLIT_DECODE_CTAS overrides)
   int use_fused = -1;  // -1: not decided yet (environment FFSPLIT_NO_FUSED=1 turns the fused kernel off)
 };
 
