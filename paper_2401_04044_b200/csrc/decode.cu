@@ -24,24 +24,29 @@
 namespace ffsp {
 namespace dec {
 
-constexpr int WARPS = 8;
-constexpr int THREADS = WARPS * 32;
-constexpr int KSTEP = 32;   // k elements per warp step: one 16-byte load per thread and row
+constexpr int KSTEP = 256;          // k elements per warp step: 512 contiguous bytes of one weight row per load
+constexpr int ROW_PITCH = 576;      // bytes between staged rows: 512 + 64 keeps the fragment reads conflict free
+constexpr int TILE_BYTES = 16 * ROW_PITCH;
+constexpr int STAGES = 2;
 
 struct Params {
   const __nv_bfloat16* X0; const __nv_bfloat16* X1; long long ldx;   // [T, K]; X1 for the gated pair
   const __nv_bfloat16* W0; const __nv_bfloat16* W1; long long ldw;   // [N, K]
   int T, N, K;
   int splits, steps_total;
+  int wk;           // warps along K inside a CTA; WR = warps / wk groups of 16 rows
   Epilogue epi;
-  float* partial;   // [splits][row groups][16 RT][8 NT] fp32
+  float* partial;   // [splits][row groups][WR][16 TILES][8 NT] fp32
   int* tickets;     // [row groups], zero before and after the launch
 };
 
-__device__ __forceinline__ uint4 ldg_stream(const void* p) {
+__device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gsrc, bool valid) {
+  const int bytes = valid ? 16 : 0;   // 0: nothing is read, the 16 bytes are zero filled
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_dst), "l"(gsrc), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
   uint4 v;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0, %1, %2, %3}, [%4];"
-               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
   return v;
 }
 __device__ __forceinline__ void mma_bf16(float* c, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
@@ -52,105 +57,110 @@ __device__ __forceinline__ void mma_bf16(float* c, uint32_t a0, uint32_t a1, uin
                : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// RT row tiles of 16 weight rows per CTA, NT token tiles of 8.  DUAL: the first RT/2 tiles come from
-// (X0, W0), the others from (X1, W1) on the same rows; output row n = silu(acc0[n]) * acc1[n].
-template <int RT, int NT, bool DUAL>
-__global__ void __launch_bounds__(THREADS, 1) decode_gemm_kernel(const Params p) {
-  extern __shared__ float red[];   // [WARPS][16 RT][8 NT]
-  __shared__ int s_last;
-  constexpr int ROWS = 16 * RT;          // weight-row slots per CTA
+// NT token tiles of 8.  DUAL: two tiles of the same 16 rows, (X0, W0) and (X1, W1); output
+// row n = silu(acc0[n]) * acc1[n].  WARPS warps per CTA (8 plain, 4 gated: shared memory).
+template <int NT, bool DUAL>
+__global__ void __launch_bounds__(DUAL ? 128 : 256, 1) decode_gemm_kernel(const Params p) {
+  constexpr int WARPS = DUAL ? 4 : 8;
+  constexpr int THREADS = WARPS * 32;
+  constexpr int TILES = DUAL ? 2 : 1;
   constexpr int TP = 8 * NT;
-  constexpr int OUT_ROWS = DUAL ? ROWS / 2 : ROWS;
+  constexpr int WARP_BYTES = STAGES * TILES * TILE_BYTES;
+  constexpr int ELEMS = 16 * TILES * TP;     // accumulator values of one warp
+  extern __shared__ __align__(16) unsigned char smem[];
+  __shared__ int s_last;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, c = lane & 3;
+  const int WK = p.wk, WR = WARPS / WK;
+  const int wr = warp / WK, wk = warp - wr * WK;
   const int rg = blockIdx.x, split = blockIdx.y;
-  const int row0 = rg * OUT_ROWS;
+  const int row0 = (rg * WR + wr) * 16;
 
   // this warp's range of k steps
   const int cta_lo = static_cast<int>(static_cast<long long>(p.steps_total) * split / p.splits);
   const int cta_hi = static_cast<int>(static_cast<long long>(p.steps_total) * (split + 1) / p.splits);
   const int n_cta = cta_hi - cta_lo;
-  const int s_lo = cta_lo + static_cast<int>(static_cast<long long>(n_cta) * warp / WARPS);
-  const int s_hi = cta_lo + static_cast<int>(static_cast<long long>(n_cta) * (warp + 1) / WARPS);
+  const int s_lo = cta_lo + static_cast<int>(static_cast<long long>(n_cta) * wk / WK);
+  const int s_hi = cta_lo + static_cast<int>(static_cast<long long>(n_cta) * (wk + 1) / WK);
 
-  float acc[RT][NT][4];
+  float acc[TILES][NT][4];
 #pragma unroll
-  for (int i = 0; i < RT; ++i)
+  for (int i = 0; i < TILES; ++i)
 #pragma unroll
     for (int j = 0; j < NT; ++j)
 #pragma unroll
       for (int e = 0; e < 4; ++e) acc[i][j][e] = 0.f;
 
-  // row pointers of this thread: tile i, rows g and g + 8
-  const __nv_bfloat16* wrow[RT][2];
-  bool wok[RT][2];
+  const uint32_t my_smem = static_cast<uint32_t>(__cvta_generic_to_shared(smem)) + warp * WARP_BYTES;
+  // one stage: 16 rows (x TILES) of 512 contiguous bytes each, one row per warp-wide copy
+  auto issue = [&](int step) {
+    const uint32_t dst0 = my_smem + (step & 1) * (TILES * TILE_BYTES) + lane * 16;
+    const int k = step * KSTEP + lane * 8;
+    const bool kin = k < p.K;   // K is a multiple of 8
 #pragma unroll
-  for (int i = 0; i < RT; ++i) {
-    const bool second = DUAL && i >= RT / 2;
-    const int tile = second ? i - RT / 2 : i;
-    const __nv_bfloat16* W = second ? p.W1 : p.W0;
+    for (int i = 0; i < TILES; ++i) {
+      const __nv_bfloat16* W = i ? p.W1 : p.W0;
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      const int n = row0 + tile * 16 + g + 8 * h;
-      wok[i][h] = n < p.N;
-      wrow[i][h] = W + static_cast<long long>(wok[i][h] ? n : 0) * p.ldw + c * 8;
-    }
-  }
-  const uint4 zero4 = make_uint4(0u, 0u, 0u, 0u);
-  auto load_w = [&](uint4 (&w)[RT][2], int step) {
-    const int k = step * KSTEP;
-    const bool kin = k + c * 8 < p.K;   // K is a multiple of 8
-#pragma unroll
-    for (int i = 0; i < RT; ++i)
-#pragma unroll
-      for (int h = 0; h < 2; ++h) w[i][h] = (kin && wok[i][h]) ? ldg_stream(wrow[i][h] + k) : zero4;
-  };
-  auto compute = [&](const uint4 (&w)[RT][2], int step) {
-    const int k = step * KSTEP + c * 8;
-    const bool kin = k < p.K;
-    uint4 xb[DUAL ? 2 : 1][NT];
-#pragma unroll
-    for (int s = 0; s < (DUAL ? 2 : 1); ++s) {
-      const __nv_bfloat16* X = s ? p.X1 : p.X0;
-#pragma unroll
-      for (int j = 0; j < NT; ++j) {
-        const int t = 8 * j + g;
-        xb[s][j] = (kin && t < p.T) ? __ldg(reinterpret_cast<const uint4*>(X + static_cast<long long>(t) * p.ldx + k))
-                                    : zero4;
+      for (int r = 0; r < 16; ++r) {
+        const int n = row0 + r;
+        const bool ok = kin && n < p.N;
+        cp_async16(dst0 + i * TILE_BYTES + r * ROW_PITCH, W + static_cast<long long>(ok ? n : 0) * p.ldw + (ok ? k : 0), ok);
       }
     }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
+  auto compute = [&](int step) {
+    const uint32_t src0 = my_smem + (step & 1) * (TILES * TILE_BYTES) + g * ROW_PITCH + c * 16;
+#pragma unroll(NT >= 4 ? 2 : 8)
+    for (int it = 0; it < 8; ++it) {
+      const int k = step * KSTEP + (it * 4 + c) * 8;
+      const bool kin = k < p.K;
+      uint4 xb[TILES][NT];
 #pragma unroll
-    for (int i = 0; i < RT; ++i) {
-      const int s = (DUAL && i >= RT / 2) ? 1 : 0;
+      for (int i = 0; i < TILES; ++i) {
+        const __nv_bfloat16* X = i ? p.X1 : p.X0;
 #pragma unroll
-      for (int j = 0; j < NT; ++j) {
-        mma_bf16(acc[i][j], w[i][0].x, w[i][1].x, w[i][0].y, w[i][1].y, xb[s][j].x, xb[s][j].y);
-        mma_bf16(acc[i][j], w[i][0].z, w[i][1].z, w[i][0].w, w[i][1].w, xb[s][j].z, xb[s][j].w);
+        for (int j = 0; j < NT; ++j) {
+          const int t = 8 * j + g;
+          xb[i][j] = (kin && t < p.T) ? __ldg(reinterpret_cast<const uint4*>(X + static_cast<long long>(t) * p.ldx + k))
+                                      : make_uint4(0u, 0u, 0u, 0u);
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < TILES; ++i) {
+        // rows g and g + 8 of the tile, the same 16 bytes of k: used as they are for two MMAs (the
+        // order in which a contraction visits k is free as long as both operands agree on it)
+        const uint4 lo = lds128(src0 + i * TILE_BYTES + it * 64);
+        const uint4 hi = lds128(src0 + i * TILE_BYTES + 8 * ROW_PITCH + it * 64);
+#pragma unroll
+        for (int j = 0; j < NT; ++j) {
+          mma_bf16(acc[i][j], lo.x, hi.x, lo.y, hi.y, xb[i][j].x, xb[i][j].y);
+          mma_bf16(acc[i][j], lo.z, hi.z, lo.w, hi.w, xb[i][j].z, xb[i][j].w);
+        }
       }
     }
   };
 
-  // two steps of weights in flight per warp
-  uint4 wa[RT][2], wb[RT][2];
-  int s = s_lo;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next product may start its own prologue
-  if (s < s_hi) load_w(wa, s);
+  if (s_lo < s_hi) issue(s_lo);
+  if (s_lo + 1 < s_hi) issue(s_lo + 1);
   // everything below reads or writes what the previous kernel of the stream produced or still reads
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  while (s < s_hi) {
-    if (s + 1 < s_hi) load_w(wb, s + 1);
-    compute(wa, s);
-    ++s;
-    if (s >= s_hi) break;
-    if (s + 1 < s_hi) load_w(wa, s + 1);
-    compute(wb, s);
-    ++s;
+  for (int s = s_lo; s < s_hi; ++s) {
+    if (s + 1 < s_hi) asm volatile("cp.async.wait_group 1;" ::: "memory");
+    else asm volatile("cp.async.wait_group 0;" ::: "memory");
+    __syncwarp();
+    compute(s);
+    __syncwarp();
+    if (s + 2 < s_hi) issue(s + 2);
   }
 
-  // ---- add the warps' accumulators in warp order
-  float* mine = red + warp * ROWS * TP;
+  // ---- the WK accumulators of each row group are added in warp order (staging buffers are free now)
+  __syncthreads();
+  float* red = reinterpret_cast<float*>(smem);   // [WARPS][16 TILES][TP]
+  float* mine = red + warp * ELEMS;
 #pragma unroll
-  for (int i = 0; i < RT; ++i)
+  for (int i = 0; i < TILES; ++i)
 #pragma unroll
     for (int j = 0; j < NT; ++j) {
       const int t = 8 * j + 2 * c;
@@ -160,28 +170,17 @@ __global__ void __launch_bounds__(THREADS, 1) decode_gemm_kernel(const Params p)
       mine[(16 * i + g + 8) * TP + t + 1] = acc[i][j][3];
     }
   __syncthreads();
-  constexpr int ELEMS = ROWS * TP;
-  constexpr int PER = (ELEMS + THREADS - 1) / THREADS;
-  float tot[PER];
-#pragma unroll
-  for (int e = 0; e < PER; ++e) {
-    const int idx = threadIdx.x + e * THREADS;
+  const int cta_elems = WR * ELEMS;
+  float* mypart = p.partial + (static_cast<long long>(split) * gridDim.x + rg) * (WARPS * ELEMS);
+  for (int idx = threadIdx.x; idx < cta_elems; idx += THREADS) {
+    const int r = idx / ELEMS, rem = idx - r * ELEMS;
     float v = 0.f;
-    if (idx < ELEMS) {
-#pragma unroll
-      for (int w = 0; w < WARPS; ++w) v += red[w * ROWS * TP + idx];
-    }
-    tot[e] = v;
+    for (int w = 0; w < WK; ++w) v += red[(r * WK + w) * ELEMS + rem];
+    if (p.splits > 1) mypart[idx] = v;
+    else red[(r * WK) * ELEMS + rem] = v;   // read and written by this thread only
   }
-  __syncthreads();
   // ---- across CTAs: partials + ticket, the last CTA of the row group adds them in split order
   if (p.splits > 1) {
-    float* mypart = p.partial + (static_cast<long long>(split) * gridDim.x + rg) * ELEMS;
-#pragma unroll
-    for (int e = 0; e < PER; ++e) {
-      const int idx = threadIdx.x + e * THREADS;
-      if (idx < ELEMS) mypart[idx] = tot[e];
-    }
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -192,36 +191,31 @@ __global__ void __launch_bounds__(THREADS, 1) decode_gemm_kernel(const Params p)
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-#pragma unroll
-    for (int e = 0; e < PER; ++e) {
-      const int idx = threadIdx.x + e * THREADS;
+    for (int idx = threadIdx.x; idx < cta_elems; idx += THREADS) {
+      const int r = idx / ELEMS, rem = idx - r * ELEMS;
       float v = 0.f;
-      if (idx < ELEMS) {
-        for (int sp = 0; sp < p.splits; ++sp)
-          v += (sp == split) ? tot[e] : __ldcg(p.partial + (static_cast<long long>(sp) * gridDim.x + rg) * ELEMS + idx);
-      }
-      tot[e] = v;
+      for (int sp = 0; sp < p.splits; ++sp)
+        v += __ldcg(p.partial + (static_cast<long long>(sp) * gridDim.x + rg) * (WARPS * ELEMS) + idx);
+      red[(r * WK) * ELEMS + rem] = v;
     }
     if (threadIdx.x == 0) p.tickets[rg] = 0;
   }
-  // ---- totals back to shared memory as [row][t], then the epilogue with n fastest across threads
-#pragma unroll
-  for (int e = 0; e < PER; ++e) {
-    const int idx = threadIdx.x + e * THREADS;
-    if (idx < ELEMS) red[idx] = tot[e];
-  }
   __syncthreads();
+  // ---- epilogue, n fastest across threads
   const Epilogue& ep = p.epi;
   const GeluCoef gc = gelu_coef(ep.act);
-  for (int idx = threadIdx.x; idx < OUT_ROWS * TP; idx += THREADS) {
-    const int t = idx / OUT_ROWS, nl = idx - t * OUT_ROWS;
-    const int n = row0 + nl;
+  const int out_cta = WR * 16;
+  for (int idx = threadIdx.x; idx < out_cta * TP; idx += THREADS) {
+    const int t = idx / out_cta, nc = idx - t * out_cta;
+    const int r = nc >> 4, nl = nc & 15;
+    const int n = rg * out_cta + nc;
     if (t >= p.T || n >= p.N) continue;
+    const float* src = red + (r * WK) * ELEMS;
     float v;
     if (DUAL) {
-      v = silu_fast(red[nl * TP + t]) * red[(nl + OUT_ROWS) * TP + t];
+      v = silu_fast(src[nl * TP + t]) * src[(nl + 16) * TP + t];
     } else {
-      v = red[nl * TP + t];
+      v = src[nl * TP + t];
       if (n < ep.n_bias) v += __ldg(ep.bias + n);
       if (n < ep.n_act) v = gelu_fast(v, gc);
     }
@@ -230,19 +224,20 @@ __global__ void __launch_bounds__(THREADS, 1) decode_gemm_kernel(const Params p)
   }
 }
 
-template <int RT, int NT, bool DUAL>
+template <int NT, bool DUAL>
 cudaError_t launch_one(const Params& p, int row_groups, cudaStream_t st) {
-  const int smem = WARPS * 16 * RT * 8 * NT * 4;
+  constexpr int WARPS = DUAL ? 4 : 8;
+  constexpr int TILES = DUAL ? 2 : 1;
+  const int smem = WARPS * STAGES * TILES * TILE_BYTES;   // also holds [WARPS][16 TILES][8 NT] floats afterwards
   static bool attr_done = false;
   if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(decode_gemm_kernel<RT, NT, DUAL>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         smem);
+    cudaError_t e = cudaFuncSetAttribute(decode_gemm_kernel<NT, DUAL>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     attr_done = true;
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(row_groups, p.splits);
-  cfg.blockDim = dim3(THREADS);
+  cfg.blockDim = dim3(WARPS * 32);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
@@ -250,17 +245,18 @@ cudaError_t launch_one(const Params& p, int row_groups, cudaStream_t st) {
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, decode_gemm_kernel<RT, NT, DUAL>, p);
+  return cudaLaunchKernelEx(&cfg, decode_gemm_kernel<NT, DUAL>, p);
 }
 
 }  // namespace dec
 
-constexpr long long kDecodeMaxPartialRows = 65536;
+constexpr long long kDecodeScratchBytes = 16ll << 20;   // fp32 partials of one product
 
 // One skinny product.  dual: (X0, W0) and (X1, W1) on the same rows, gated.
 static ffsplit_status decode_gemm(ffsplit_ctx* ctx, const void* X0, const void* X1, long long ldx, const void* W0,
                                   const void* W1, long long ldw, int T, int N, int K, const Epilogue& epi,
-                                  float* partial, double algo_bytes, cudaStream_t st, int* tickets = nullptr) {
+                                  float* partial, double algo_bytes, cudaStream_t st, int* tickets = nullptr,
+                                  long long scratch_bytes = kDecodeScratchBytes) {
   if (N <= 0 || K <= 0) return FFSPLIT_OK;
   const bool dual = W1 != nullptr;
   dec::Params p;
@@ -272,29 +268,38 @@ static ffsplit_status decode_gemm(ffsplit_ctx* ctx, const void* X0, const void* 
   p.partial = partial;
   p.tickets = tickets ? tickets : ctx->tickets();
   const int nt = T <= 8 ? 1 : T <= 16 ? 2 : T <= 32 ? 4 : 8;
-  const int rt = nt == 8 ? 2 : 4;
-  const int out_rows = dual ? 8 * rt : 16 * rt;
-  const int row_groups = (N + out_rows - 1) / out_rows;
-  if (row_groups > kMaxTicketTiles) return fail(ctx, FFSPLIT_ERR_SHAPE, "decode: too many row groups");
-  // Several waves of small CTAs (less loss in the last, partly filled wave), each warp keeping at
-  // least two k steps, the fp32 partials (written and read once) at most ~12 % of the weight bytes.
-  int splits = (ctx->decode_ctas_per_sm_target * ctx->num_sms + row_groups - 1) / row_groups;
-  const int max_by_k = p.steps_total / (2 * dec::WARPS);
-  if (splits > max_by_k) splits = max_by_k;
-  const int max_by_traffic = static_cast<int>(0.03 * K / (8 * nt));
-  if (splits > max_by_traffic) splits = max_by_traffic;
-  if (splits > 16) splits = 16;
-  const long long rows_slots = static_cast<long long>(row_groups) * 16 * rt;
-  if (splits > 1 && splits * rows_slots > kDecodeMaxPartialRows) splits = static_cast<int>(kDecodeMaxPartialRows / rows_slots);
-  if (splits < 1) splits = 1;
-  p.splits = splits;
+  const int warps = dual ? 4 : 8, tiles = dual ? 2 : 1;
+  // Plan: wk warps of a CTA share 16 rows and split the CTA's K range; `splits` CTAs share a row group.
+  // Wanted: at least one CTA per SM, every warp with a few steps (of 256 k) to pipeline, and fp32
+  // partials (written and read once) small beside the weights.
+  int best_wk = 1, best_splits = 1;
+  double best = -1.0;
+  for (int wk = warps; wk >= 1; wk >>= 1) {
+    const int wr = warps / wk;
+    const long long rgs = (N + 16ll * wr - 1) / (16ll * wr);
+    if (rgs > kMaxTicketTiles) continue;
+    for (int sp = 1; sp <= 16; ++sp) {
+      const double steps_per_warp = static_cast<double>(p.steps_total) / (wk * sp);
+      if ((sp > 1 || wk > 1) && steps_per_warp < 1.0) break;
+      const double part_bytes = sp > 1 ? 2.0 * sp * rgs * warps * 16.0 * tiles * 8 * nt * 4 : 0.0;
+      if (sp > 1 && (sp * rgs * warps * 16ll * tiles * 8 * nt * 4 > scratch_bytes || part_bytes > 0.12 * 2.0 * N * K)) break;
+      const double fill = static_cast<double>(rgs) * sp / ctx->num_sms;
+      const double score = (fill < 1.0 ? fill : 1.0) * (steps_per_warp < 3.0 ? steps_per_warp / 3.0 : 1.0) - 0.002 * sp -
+                           0.001 * wk;
+      if (score > best) { best = score; best_wk = wk; best_splits = sp; }
+    }
+  }
+  p.wk = best_wk;
+  p.splits = best_splits;
+  const int wr = warps / p.wk;
+  const int row_groups = static_cast<int>((N + 16ll * wr - 1) / (16ll * wr));
   const int ph = prof_open(ctx, PROF_DECODE, algo_bytes, st);
   cudaError_t e;
-#define FFS_DEC(RT_, NT_) (dual ? dec::launch_one<RT_, NT_, true>(p, row_groups, st) : dec::launch_one<RT_, NT_, false>(p, row_groups, st))
-  if (nt == 1) e = FFS_DEC(4, 1);
-  else if (nt == 2) e = FFS_DEC(4, 2);
-  else if (nt == 4) e = FFS_DEC(4, 4);
-  else e = FFS_DEC(2, 8);
+#define FFS_DEC(NT_) (dual ? dec::launch_one<NT_, true>(p, row_groups, st) : dec::launch_one<NT_, false>(p, row_groups, st))
+  if (nt == 1) e = FFS_DEC(1);
+  else if (nt == 2) e = FFS_DEC(2);
+  else if (nt == 4) e = FFS_DEC(4);
+  else e = FFS_DEC(8);
 #undef FFS_DEC
   prof_close(ctx, ph, st);
   ctx->launches++;
@@ -306,15 +311,15 @@ bool decode_path_applies(const ffsplit_ctx* ctx, const BlobHeader& h, long long 
   return h.dtype == FFSPLIT_BF16 && T >= 1 && T <= 64;
 }
 
-// fp32 partials of one product: at most kDecodeMaxPartialRows row slots of 64 tokens.
+// fp32 partials of one product.
 size_t decode_scratch_bytes(int dtype, long long T) {
   if (dtype != FFSPLIT_BF16 || T > 64 || T < 1) return 0;
-  return static_cast<size_t>(kDecodeMaxPartialRows) * 64 * 4;
+  return static_cast<size_t>(kDecodeScratchBytes);
 }
 
 static ffsplit_status decode_forward_impl(ffsplit_ctx* ctx, const BlobHeader& h, const char* blob, const void* X,
                                           long long T64, void* Y, char* AP, char* Q, char* HL, char* scratch,
-                                          cudaStream_t st, int* tickets) {
+                                          cudaStream_t st, int* tickets, long long scratch_bytes) {
   const int T = static_cast<int>(T64);
   const int d = h.d, k_pad = h.k_pad, r_pad = h.r_pad, ml_pad = h.ml_pad, kp_rp = h.k_pad + h.r_pad;
   const bool gated = h.act == FFSPLIT_SWIGLU;
@@ -333,17 +338,17 @@ static ffsplit_status decode_forward_impl(ffsplit_ctx* ctx, const BlobHeader& h,
     e.C0 = AP; e.ld0 = kp_rp; e.C1 = Q; e.ld1 = r_pad;
     e.n_split = k_pad; e.n_act = k_pad; e.n_bias = k_pad; e.bias = b1h;
     if ((s = decode_gemm(ctx, X, nullptr, d, blob + h.off[SEC_U1T], nullptr, d, T, kp_rp, d, e, part,
-                         2.0 * d * (h.k + h.r) + 4.0 * h.k + xy / 2, st, tickets)) != FFSPLIT_OK) return s;
+                         2.0 * d * (h.k + h.r) + 4.0 * h.k + xy / 2, st, tickets, scratch_bytes)) != FFSPLIT_OK) return s;
   } else {
     clear();
     e.C0 = AP; e.ld0 = kp_rp; e.n_split = k_pad;
     if ((s = decode_gemm(ctx, X, X, d, blob + h.off[SEC_U1T], blob + h.off[SEC_U1UT], d, T, k_pad, d, e, part,
-                         4.0 * d * h.k + xy / 2, st, tickets)) != FFSPLIT_OK) return s;
+                         4.0 * d * h.k + xy / 2, st, tickets, scratch_bytes)) != FFSPLIT_OK) return s;
     if (light) {
       clear();
       e.C0 = Q; e.ld0 = 2 * r_pad; e.n_split = 2 * r_pad;
       if ((s = decode_gemm(ctx, X, nullptr, d, blob + h.off[SEC_A1T], nullptr, d, T, 2 * r_pad, d, e, part,
-                           4.0 * d * h.r, st, tickets)) != FFSPLIT_OK) return s;
+                           4.0 * d * h.r, st, tickets, scratch_bytes)) != FFSPLIT_OK) return s;
     }
   }
   // ---- stage 2
@@ -354,24 +359,24 @@ static ffsplit_status decode_forward_impl(ffsplit_ctx* ctx, const BlobHeader& h,
     const long long ldq = static_cast<long long>(h.n_in) * r_pad;
     if ((s = decode_gemm(ctx, Q, gated ? Q + static_cast<size_t>(r_pad) * 2 : nullptr, ldq, blob + h.off[SEC_B1T],
                          gated ? blob + h.off[SEC_B1UT] : nullptr, r_pad, T, ml_pad, r_pad, e, part,
-                         2.0 * h.n_in * h.r * h.ml + (gated ? 0.0 : 4.0 * h.ml), st, tickets)) != FFSPLIT_OK) return s;
+                         2.0 * h.n_in * h.r * h.ml + (gated ? 0.0 : 4.0 * h.ml), st, tickets, scratch_bytes)) != FFSPLIT_OK) return s;
     clear();
     e.C0 = AP + static_cast<size_t>(k_pad) * 2; e.ld0 = kp_rp; e.n_split = r_pad;
     if ((s = decode_gemm(ctx, HL, nullptr, ml_pad, blob + h.off[SEC_A2T], nullptr, ml_pad, T, r_pad, ml_pad, e, part,
-                         2.0 * h.r * h.ml, st, tickets)) != FFSPLIT_OK) return s;
+                         2.0 * h.r * h.ml, st, tickets, scratch_bytes)) != FFSPLIT_OK) return s;
   }
   // ---- stage 3
   clear();
   e.C0 = Y; e.ld0 = d; e.n_split = d; e.n_bias = d; e.bias = b2;
   return decode_gemm(ctx, AP, nullptr, kp_rp, blob + h.off[SEC_V1B2T], nullptr, kp_rp, T, d, light ? kp_rp : k_pad, e,
-                     part, 2.0 * d * (h.k + (light ? h.r : 0)) + 4.0 * d + xy / 2, st, tickets);
+                     part, 2.0 * d * (h.k + (light ? h.r : 0)) + 4.0 * d + xy / 2, st, tickets, scratch_bytes);
 }
 
 // Scratch from the caller's workspace, ticket counters from its control block.
 ffsplit_status launch_decode_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* blob, const void* X,
                                      long long T, void* Y, char* AP, char* Q, char* HL, char* scratch,
                                      cudaStream_t st) {
-  return decode_forward_impl(ctx, h, blob, X, T, Y, AP, Q, HL, scratch, st, nullptr);
+  return decode_forward_impl(ctx, h, blob, X, T, Y, AP, Q, HL, scratch, st, nullptr, kDecodeScratchBytes);
 }
 
 }  // namespace ffsp
@@ -383,7 +388,7 @@ namespace {
 
 constexpr int kNoAllocMaxTokens = 8;
 constexpr size_t kNoAllocTicketBytes = ffsp::kCtrlBytes;                 // ticket counters of the K-split reduction
-constexpr size_t kNoAllocPartialBytes = static_cast<size_t>(ffsp::kDecodeMaxPartialRows) * 8 * 4;   // fp32 partials, 8 tokens
+constexpr size_t kNoAllocPartialBytes = 2u << 20;                       // fp32 partials of the K-split reduction
 constexpr size_t kNoAllocStageBytes = 2u << 20;                         // A_H | P, Q and the light activations
 constexpr size_t kNoAllocBytes = kNoAllocTicketBytes + kNoAllocPartialBytes + kNoAllocStageBytes;   // 4.06 MiB
 
@@ -444,5 +449,5 @@ extern "C" ffsplit_status ffsplit_forward_noalloc(ffsplit_ctx* ctx, const void* 
   char* Q = AP + ap_b;
   char* HL = Q + q_b;
   return decode_forward_impl(ctx, h, static_cast<const char*>(blob), X, T, Y, AP, Q, HL, part, st,
-                             reinterpret_cast<int*>(base));
+                             reinterpret_cast<int*>(base), static_cast<long long>(kNoAllocPartialBytes));
 }
