@@ -76,12 +76,11 @@ __global__ void __launch_bounds__(DUAL ? 128 : 256, 1) decode_gemm_kernel(const 
   const int rg = blockIdx.x, split = blockIdx.y;
   const int row0 = (rg * WR + wr) * 16;
 
-  // this warp's range of k steps
+  // This CTA's range of k steps; its WK warps take the steps round robin, so that at any time the
+  // warps of a row group read neighbouring 512-byte pieces of the same rows (long runs in DRAM).
   const int cta_lo = static_cast<int>(static_cast<long long>(p.steps_total) * split / p.splits);
   const int cta_hi = static_cast<int>(static_cast<long long>(p.steps_total) * (split + 1) / p.splits);
-  const int n_cta = cta_hi - cta_lo;
-  const int s_lo = cta_lo + static_cast<int>(static_cast<long long>(n_cta) * wk / WK);
-  const int s_hi = cta_lo + static_cast<int>(static_cast<long long>(n_cta) * (wk + 1) / WK);
+  const int my_steps = (cta_hi - cta_lo - wk + WK - 1) / WK;   // steps cta_lo + wk + i * WK
 
   float acc[TILES][NT][4];
 #pragma unroll
@@ -93,8 +92,9 @@ __global__ void __launch_bounds__(DUAL ? 128 : 256, 1) decode_gemm_kernel(const 
 
   const uint32_t my_smem = static_cast<uint32_t>(__cvta_generic_to_shared(smem)) + warp * WARP_BYTES;
   // one stage: 16 rows (x TILES) of 512 contiguous bytes each, one row per warp-wide copy
-  auto issue = [&](int step) {
-    const uint32_t dst0 = my_smem + (step & 1) * (TILES * TILE_BYTES) + lane * 16;
+  auto issue = [&](int i) {
+    const int step = cta_lo + wk + i * WK;
+    const uint32_t dst0 = my_smem + (i & 1) * (TILES * TILE_BYTES) + lane * 16;
     const int k = step * KSTEP + lane * 8;
     const bool kin = k < p.K;   // K is a multiple of 8
 #pragma unroll
@@ -109,8 +109,9 @@ __global__ void __launch_bounds__(DUAL ? 128 : 256, 1) decode_gemm_kernel(const 
     }
     asm volatile("cp.async.commit_group;" ::: "memory");
   };
-  auto compute = [&](int step) {
-    const uint32_t src0 = my_smem + (step & 1) * (TILES * TILE_BYTES) + g * ROW_PITCH + c * 16;
+  auto compute = [&](int i) {
+    const int step = cta_lo + wk + i * WK;
+    const uint32_t src0 = my_smem + (i & 1) * (TILES * TILE_BYTES) + g * ROW_PITCH + c * 16;
 #pragma unroll(NT >= 4 ? 2 : 8)
     for (int it = 0; it < 8; ++it) {
       const int k = step * KSTEP + (it * 4 + c) * 8;
@@ -142,17 +143,17 @@ __global__ void __launch_bounds__(DUAL ? 128 : 256, 1) decode_gemm_kernel(const 
   };
 
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the next product may start its own prologue
-  if (s_lo < s_hi) issue(s_lo);
-  if (s_lo + 1 < s_hi) issue(s_lo + 1);
+  if (my_steps > 0) issue(0);
+  if (my_steps > 1) issue(1);
   // everything below reads or writes what the previous kernel of the stream produced or still reads
   asm volatile("griddepcontrol.wait;" ::: "memory");
-  for (int s = s_lo; s < s_hi; ++s) {
-    if (s + 1 < s_hi) asm volatile("cp.async.wait_group 1;" ::: "memory");
+  for (int i = 0; i < my_steps; ++i) {
+    if (i + 1 < my_steps) asm volatile("cp.async.wait_group 1;" ::: "memory");
     else asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncwarp();
-    compute(s);
+    compute(i);
     __syncwarp();
-    if (s + 2 < s_hi) issue(s + 2);
+    if (i + 2 < my_steps) issue(i + 2);
   }
 
   // ---- the WK accumulators of each row group are added in warp order (staging buffers are free now)
