@@ -46,22 +46,40 @@ def random_factors(cfg, device, gen):
     return f
 
 
-def time_calls(fn, reps, warmup):
+def time_calls(fn, batch, reps, warmup, use_graph=True):
+    """Milliseconds per call of `fn`, one sample per timed batch of `batch` consecutive calls.
+
+    A single few-token forward lasts tens of microseconds, less than the host needs to issue it, so
+    the batch is recorded once into a CUDA graph and the replays are timed (device events around each
+    replay); with use_graph=False, or if the capture fails, the batch is issued call by call."""
     for _ in range(warmup):
         fn()
+    torch.cuda.synchronize()
+    run = lambda: [fn() for _ in range(batch)]
+    mode = "stream"
+    if use_graph:
+        try:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                run()
+            run, mode = graph.replay, "cuda_graph"
+        except Exception as exc:  # capture not possible: time the plain launches
+            torch.cuda.synchronize()
+            mode = f"stream (graph capture failed: {type(exc).__name__})"
+    run()
     torch.cuda.synchronize()
     ts = []
     for _ in range(reps):
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record()
-        fn()
+        run()
         b.record()
         b.synchronize()
-        ts.append(a.elapsed_time(b))
-    return ts
+        ts.append(a.elapsed_time(b) / batch)
+    return ts, mode
 
 
-def run_point(ctx, cfg, tokens, copies, reps, svd, device="cuda"):
+def run_point(ctx, cfg, tokens, copies, reps, svd, device="cuda", use_graph=True):
     hbm, tf, src = peaks()
     shape = make_shape(cfg.d, cfg.m, cfg.act, cfg.torch_dtype)
     es = 2 if cfg.dtype == "bf16" else 4
@@ -105,8 +123,10 @@ def run_point(ctx, cfg, tokens, copies, reps, svd, device="cuda"):
                 ctx.forward(bl[state["i"] % copies], X, Y)
                 state["i"] += 1
 
-            ts = time_calls(call, reps, max(3, copies))
+            # every batch walks all weight copies (more than L2 holds) the same number of times
+            ts, mode = time_calls(call, copies * max(1, 16 // copies), reps, max(3, copies), use_graph)
             ctx.poll()
+            res["launch_mode"] = mode
             ms = statistics.median(ts)
             flops = 2.0 * params * T
             bytes_ = es * (params + cfg.m + cfg.d) + 2 * T * cfg.d * es
@@ -130,6 +150,7 @@ def main():
     ap.add_argument("--svd", action="store_true", help="true SVD factors instead of random ones")
     ap.add_argument("--sweep5", action="store_true", help="config 5: all heavy fractions x ranks")
     ap.add_argument("--out", default=None)
+    ap.add_argument("--no-graph", action="store_true", help="issue the timed calls one by one instead of replaying a CUDA graph")
     args = ap.parse_args()
     build.build()
     ctx = Context(0)
@@ -143,7 +164,7 @@ def main():
         es = 2 if cfg.dtype == "bf16" else 4
         split_bytes = es * (cfg.n_in + 1) * (cfg.d * cfg.k + cfg.r * (cfg.d + cfg.m - cfg.k))
         copies = args.copies or max(2, min(24, -(-2 * 126 * (1 << 20) // split_bytes)))
-        for res in run_point(ctx, cfg, tokens, copies, args.reps, args.svd):
+        for res in run_point(ctx, cfg, tokens, copies, args.reps, args.svd, use_graph=not args.no_graph):
             line = json.dumps(res)
             print(line, flush=True)
             lines.append(line)
