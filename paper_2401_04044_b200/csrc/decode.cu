@@ -18,16 +18,12 @@
 // output element, after the reduction.
 #include <cstring>
 
+#include "decode_common.cuh"
 #include "epilogue.cuh"
 #include "internal.h"
 
 namespace ffsp {
 namespace dec {
-
-constexpr int KSTEP = 256;          // k elements per warp step: 512 contiguous bytes of one weight row per load
-constexpr int ROW_PITCH = 576;      // bytes between staged rows: 512 + 64 keeps the fragment reads conflict free
-constexpr int TILE_BYTES = 16 * ROW_PITCH;
-constexpr int STAGES = 2;
 
 struct Params {
   const __nv_bfloat16* X0; const __nv_bfloat16* X1; long long ldx;   // [T, K]; X1 for the gated pair
@@ -39,23 +35,6 @@ struct Params {
   float* partial;   // [splits][row groups][WR][16 TILES][8 NT] fp32
   int* tickets;     // [row groups], zero before and after the launch
 };
-
-__device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gsrc, bool valid) {
-  const int bytes = valid ? 16 : 0;   // 0: nothing is read, the 16 bytes are zero filled
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_dst), "l"(gsrc), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ uint4 lds128(uint32_t addr) {
-  uint4 v;
-  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
-  return v;
-}
-__device__ __forceinline__ void mma_bf16(float* c, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                         uint32_t b1) {
-  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
-               "{%0, %1, %2, %3};"
-               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
 
 // NT token tiles of 8.  DUAL: two tiles of the same 16 rows, (X0, W0) and (X1, W1); output
 // row n = silu(acc0[n]) * acc1[n].  WARPS warps per CTA (8 plain, 4 gated: shared memory).
@@ -332,24 +311,32 @@ static ffsplit_status decode_forward_impl(ffsplit_ctx* ctx, const BlobHeader& h,
   const double xy = 2.0 * T * d * 2;   // X read once, Y written once: charged to the first and last product
   ffsplit_status s;
   Epilogue e;
+  // T <= 32: the products are collected and run by one persistent kernel; above that, one launch each
+  const bool one_kernel = decode_layer_applies(T);
+  DecodeLayerPlan plan;
+  auto emit = [&](const void* X0, const void* X1, long long ldx, const void* W0, const void* W1, long long ldw, int T_,
+                  int N, int K, const Epilogue& epi, float* partial, double algo_bytes) -> ffsplit_status {
+    if (one_kernel) return decode_layer_add(ctx, &plan, X0, X1, ldx, W0, W1, ldw, N, K, epi, algo_bytes);
+    return decode_gemm(ctx, X0, X1, ldx, W0, W1, ldw, T_, N, K, epi, partial, algo_bytes, st, tickets, scratch_bytes);
+  };
   auto clear = [&]() { std::memset(&e, 0, sizeof(e)); e.act = h.act; };
   // ---- stage 1
   if (!gated) {
     clear();
     e.C0 = AP; e.ld0 = kp_rp; e.C1 = Q; e.ld1 = r_pad;
     e.n_split = k_pad; e.n_act = k_pad; e.n_bias = k_pad; e.bias = b1h;
-    if ((s = decode_gemm(ctx, X, nullptr, d, blob + h.off[SEC_U1T], nullptr, d, T, kp_rp, d, e, part,
-                         2.0 * d * (h.k + h.r) + 4.0 * h.k + xy / 2, st, tickets, scratch_bytes)) != FFSPLIT_OK) return s;
+    if ((s = emit(X, nullptr, d, blob + h.off[SEC_U1T], nullptr, d, T, kp_rp, d, e, part,
+                         2.0 * d * (h.k + h.r) + 4.0 * h.k + xy / 2)) != FFSPLIT_OK) return s;
   } else {
     clear();
     e.C0 = AP; e.ld0 = kp_rp; e.n_split = k_pad;
-    if ((s = decode_gemm(ctx, X, X, d, blob + h.off[SEC_U1T], blob + h.off[SEC_U1UT], d, T, k_pad, d, e, part,
-                         4.0 * d * h.k + xy / 2, st, tickets, scratch_bytes)) != FFSPLIT_OK) return s;
+    if ((s = emit(X, X, d, blob + h.off[SEC_U1T], blob + h.off[SEC_U1UT], d, T, k_pad, d, e, part,
+                         4.0 * d * h.k + xy / 2)) != FFSPLIT_OK) return s;
     if (light) {
       clear();
       e.C0 = Q; e.ld0 = 2 * r_pad; e.n_split = 2 * r_pad;
-      if ((s = decode_gemm(ctx, X, nullptr, d, blob + h.off[SEC_A1T], nullptr, d, T, 2 * r_pad, d, e, part,
-                           4.0 * d * h.r, st, tickets, scratch_bytes)) != FFSPLIT_OK) return s;
+      if ((s = emit(X, nullptr, d, blob + h.off[SEC_A1T], nullptr, d, T, 2 * r_pad, d, e, part,
+                           4.0 * d * h.r)) != FFSPLIT_OK) return s;
     }
   }
   // ---- stage 2
@@ -358,19 +345,25 @@ static ffsplit_status decode_forward_impl(ffsplit_ctx* ctx, const BlobHeader& h,
     e.C0 = HL; e.ld0 = ml_pad; e.n_split = ml_pad;
     if (!gated) { e.n_act = ml_pad; e.n_bias = ml_pad; e.bias = b1l; }
     const long long ldq = static_cast<long long>(h.n_in) * r_pad;
-    if ((s = decode_gemm(ctx, Q, gated ? Q + static_cast<size_t>(r_pad) * 2 : nullptr, ldq, blob + h.off[SEC_B1T],
+    if ((s = emit(Q, gated ? Q + static_cast<size_t>(r_pad) * 2 : nullptr, ldq, blob + h.off[SEC_B1T],
                          gated ? blob + h.off[SEC_B1UT] : nullptr, r_pad, T, ml_pad, r_pad, e, part,
-                         2.0 * h.n_in * h.r * h.ml + (gated ? 0.0 : 4.0 * h.ml), st, tickets, scratch_bytes)) != FFSPLIT_OK) return s;
+                         2.0 * h.n_in * h.r * h.ml + (gated ? 0.0 : 4.0 * h.ml))) != FFSPLIT_OK) return s;
     clear();
     e.C0 = AP + static_cast<size_t>(k_pad) * 2; e.ld0 = kp_rp; e.n_split = r_pad;
-    if ((s = decode_gemm(ctx, HL, nullptr, ml_pad, blob + h.off[SEC_A2T], nullptr, ml_pad, T, r_pad, ml_pad, e, part,
-                         2.0 * h.r * h.ml, st, tickets, scratch_bytes)) != FFSPLIT_OK) return s;
+    if ((s = emit(HL, nullptr, ml_pad, blob + h.off[SEC_A2T], nullptr, ml_pad, T, r_pad, ml_pad, e, part,
+                         2.0 * h.r * h.ml)) != FFSPLIT_OK) return s;
   }
   // ---- stage 3
   clear();
   e.C0 = Y; e.ld0 = d; e.n_split = d; e.n_bias = d; e.bias = b2;
-  return decode_gemm(ctx, AP, nullptr, kp_rp, blob + h.off[SEC_V1B2T], nullptr, kp_rp, T, d, light ? kp_rp : k_pad, e,
-                     part, 2.0 * d * (h.k + (light ? h.r : 0)) + 4.0 * d + xy / 2, st, tickets, scratch_bytes);
+  if ((s = emit(AP, nullptr, kp_rp, blob + h.off[SEC_V1B2T], nullptr, kp_rp, T, d, light ? kp_rp : k_pad, e,
+                     part, 2.0 * d * (h.k + (light ? h.r : 0)) + 4.0 * d + xy / 2)) != FFSPLIT_OK) return s;
+  if (!one_kernel) return FFSPLIT_OK;
+  if (static_cast<long long>(decode_layer_scratch_bytes(ctx->num_sms, T)) > scratch_bytes)
+    return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL, "few-token forward: scratch smaller than two partials per SM");
+  // control block: the caller's (status and barrier words, then the tickets), else the workspace's
+  int* ctrl = tickets ? tickets : ctx->status();
+  return decode_layer_launch(ctx, &plan, T, part, ctrl, st);
 }
 
 // Scratch from the caller's workspace, ticket counters from its control block.

@@ -1,0 +1,35 @@
+// Pieces shared by the few-token (decode) kernels: the staging geometry of a weight tile and the
+// three instructions they are built from.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+namespace ffsp {
+namespace dec {
+
+constexpr int KSTEP = 256;          // k elements per step: 512 contiguous bytes of one weight row per warp-wide copy
+constexpr int ROW_PITCH = 576;      // bytes between staged rows: 512 + 64 keeps the fragment reads conflict free
+constexpr int TILE_BYTES = 16 * ROW_PITCH;   // 16 weight rows of one step
+constexpr int STAGES = 2;
+
+__device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* gsrc, bool valid) {
+  const int bytes = valid ? 16 : 0;   // 0: nothing is read, the 16 bytes are zero filled
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(smem_dst), "l"(gsrc), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+  return v;
+}
+__device__ __forceinline__ void mma_bf16(float* c, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1) {
+  asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+               "{%0, %1, %2, %3};"
+               : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+               : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+}  // namespace dec
+}  // namespace ffsp

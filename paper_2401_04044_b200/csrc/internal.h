@@ -162,7 +162,8 @@ struct ffsplit_ctx {
   bool attr_fused_set = false;
   int* status() const { return reinterpret_cast<int*>(ws); }
   int* tickets() const { return reinterpret_cast<int*>(ws + ffsp::kStatusBytes); }
-  int decode_ctas_per_sm_target = 6;   // CTAs per SM the few-token kernels aim for when splitting K (FFSPLIT_DECODE_CTAS overrides)
+  int decode_ctas_per_sm_target = 6;   // T > 32: CTAs per SM the per-product kernel aims for when splitting K (FFSPLIT_DECODE_CTAS overrides)
+  int decode_one_launch = 0;   // T <= 32: 1 = all products in one cooperative launch (FFSPLIT_DECODE_LAYER=1), 0 = one launch per product
   int use_fused = -1;  // -1: not decided yet (environment FFSPLIT_NO_FUSED=1 turns the fused kernel off)
 };
 
@@ -175,6 +176,31 @@ inline int round_up(int v, int q) { return (v + q - 1) / q * q; }
 inline long long round_up_ll(long long v, long long q) { return (v + q - 1) / q * q; }
 inline size_t elem_size(int dtype) { return dtype == FFSPLIT_BF16 ? 2 : 4; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// ----------------------------------------------------------------------------
+// Few-token forward (T <= 32): the products of one layer, run by one persistent kernel
+// (decode_layer.cu).  C[t, n] = epi(sum_k X[t, k] W[n, k]); W1 != nullptr: gated pair.
+// ----------------------------------------------------------------------------
+struct DecodeProduct {
+  const void* X0; const void* X1; long long ldx;   // [T, K] bf16; X1 for the gated pair
+  const void* W0; const void* W1; long long ldw;   // [N, K] bf16
+  int N, K;
+  int tiles, steps;   // row tiles (128 rows, gated 64) and k steps of 256
+  Epilogue epi;
+};
+constexpr int kMaxDecodeProducts = 5;
+struct DecodeLayerPlan {
+  DecodeProduct prod[kMaxDecodeProducts];
+  int n = 0;
+  double algo_bytes = 0.0;
+};
+bool decode_layer_applies(long long T);
+size_t decode_layer_scratch_bytes(int num_sms, long long T);
+ffsplit_status decode_layer_add(ffsplit_ctx* ctx, DecodeLayerPlan* plan, const void* X0, const void* X1, long long ldx,
+                                const void* W0, const void* W1, long long ldw, int N, int K, const Epilogue& epi,
+                                double algo_bytes);
+ffsplit_status decode_layer_launch(ffsplit_ctx* ctx, const DecodeLayerPlan* plan, int T, float* partial, int* ctrl,
+                                   cudaStream_t st);
 
 // Profiling brackets: no-ops unless ffsplit_profile_begin() is active.
 enum ProfClass : int { PROF_GEMM_TC = 0, PROF_GEMM_SIMT = 1, PROF_DECODE = 2 };
