@@ -7,19 +7,23 @@
 //
 //  * One CTA per SM stays resident for the whole layer.  A product is cut into units of
 //    128 weight rows x 256 k (64 KB of W); the units, in row-tile-major order, are dealt to the CTAs in
-//    equal contiguous shares (a tile's K range may straddle two or more CTAs), and a CTA walks its share
-//    with a two-stage cp.async pipeline that does not drain at tile boundaries.
-//  * A tile finished inside one CTA goes through the epilogue straight from the accumulator registers.
-//    A tile shared by several CTAs: each writes an fp32 partial (at most two per CTA and product: the
-//    tile its share starts in and the tile it ends in), takes an atomic ticket, and the last to arrive
-//    adds the partials in CTA order -- the result does not depend on who arrives when.
-//  * Each warp-wide copy moves 512 contiguous bytes of one weight row; the token rows of the same k
-//    range are staged beside the weights, once per CTA.  Fragments for the warp-level MMA (m16n8k16,
-//    weights as the 16-row operand, tokens as the 8-wide one) are read from shared memory with
-//    128-bit loads; since a contraction does not care in which order k is visited, a thread's 16
-//    bytes feed two MMAs as they are, and the token operand is read with the same pattern.
+//    equal contiguous shares (a tile's K range may straddle two or more CTAs).
+//  * The warps of a CTA walk its share side by side -- each owns 16 NT rows of every tile, NT = token
+//    tiles of 8 -- but never wait for one another: each has its own two-stage cp.async ring, so a late
+//    DRAM reply holds up one warp, not the SM, and the ring does not drain at tile boundaries.
+//  * Each warp-wide copy moves 512 contiguous bytes of one weight row.  The token rows of the same k
+//    range travel in the same copy group into the warp's own stage (they come from L2 and add half
+//    the weight bytes at most); loading them at the point of use instead costs a quarter of the
+//    bandwidth, and sharing one copy per CTA ties the warps together.  Fragments for the warp-level
+//    MMA (m16n8k16, weights as the 16-row operand, tokens as the 8-wide one) are read from shared
+//    memory with 128-bit loads; since a contraction does not care in which order k is visited, a
+//    thread's 16 bytes feed two MMAs as they are, and the token operand is read with the same pattern.
+//  * Rows finished inside one CTA go through the epilogue straight from the accumulator registers.
+//    Rows shared by several CTAs: each warp writes an fp32 partial (at most two per CTA and product:
+//    the tile its share starts in and the tile it ends in), takes an atomic ticket, and the last to
+//    arrive adds the partials in CTA order -- the result does not depend on who arrives when.
 //  * Products are separated by a grid-wide barrier (cooperative launch: all CTAs are resident), before
-//    which each CTA has already issued the first weight copies of the next product.
+//    which each warp has already issued the first weight copies of the next product.
 //  * The code is kept small (one call site per building block, short unrolls): the weights stream
 //    through L2 and push the kernel's instructions out of it between launches, so every launch
 //    fetches its code from DRAM again and straight-line code is paid for in fetch latency.
@@ -38,11 +42,9 @@ namespace dsk {
 using namespace dec;
 
 constexpr int WARPS = 8, THREADS = WARPS * 32;
-constexpr int W_STAGE = WARPS * TILE_BYTES;     // eight 16-row tiles: 128 rows, or 64 rows of a gated pair
-constexpr int W_BYTES = STAGES * W_STAGE;
+constexpr int SMEM_BYTES = 3 * 8 * TILE_BYTES;   // the same for every shape below
 constexpr int kBarCount = 16, kBarGen = 17;     // words of the control block used by the grid barrier
 constexpr int kTicketWord0 = static_cast<int>(kStatusBytes / 4);   // tickets follow the status block
-constexpr int kSlotTable = 256;                 // partial slots looked up per pass when a tile's partials are added
 constexpr long long kWaitLimit = 2000000000ll;  // clock cycles (about a second) before a barrier wait gives up
 
 using Product = DecodeProduct;
@@ -52,11 +54,26 @@ struct Params {
   int nprod;
   int T;
   float* partial;   // [2 * gridDim.x] slots of 128 * 8 NT floats
-  int* ctrl;        // control block: status words, barrier words, then one ticket per row tile (zero between launches)
+  int* ctrl;        // control block: status words, barrier words, then eight tickets per row tile (zero between launches)
 };
 
-template <int NT>
-constexpr int smem_bytes() { return W_BYTES + STAGES * 2 * (8 * NT) * ROW_PITCH; }
+// A CTA tile is 128 weight rows (64 rows of each matrix for a gated pair); warp w owns 16 of them.
+// Up to 8 tokens (NT = 1 token tile) a warp's stage holds its weight rows and a private copy of the
+// token rows, two stages deep.  With more tokens the copies would not fit: the token rows are then
+// loaded where they are used (through L1), and the ring is three stages of weights.
+template <int NT, bool DUAL>
+struct Shape {
+  static constexpr bool PRIV = NT == 1;              // token rows staged with the weights
+  static constexpr int NST = PRIV ? 2 : 3;           // stages of a warp's ring
+  static constexpr int TILES = DUAL ? 2 : 1;
+  static constexpr int AW = DUAL ? 4 : 8;            // working warps
+  static constexpr int TR = AW * 16;                 // rows of a CTA tile
+  static constexpr int TP = 8 * NT;                  // token rows, padded
+  static constexpr int W_BYTES = TILES * TILE_BYTES;
+  static constexpr int X_BYTES = PRIV ? TILES * TP * ROW_PITCH : 0;   // a gated pair may have two inputs
+  static constexpr int STAGE = W_BYTES + X_BYTES;
+  static_assert(AW * NST * STAGE == SMEM_BYTES, "shared memory plan");
+};
 
 // Shares of the `ge` CTAs that have one: CTA c owns units [c U / ge, (c + 1) U / ge).  U * (ge + 1) fits
 // in 32 bits (checked when the product is planned).
@@ -66,20 +83,18 @@ __device__ __forceinline__ int cta_of(unsigned u, unsigned U, unsigned ge) {
   return static_cast<int>(((u + 1) * ge - 1) / U);
 }
 
-// ---- copies of one unit ---------------------------------------------------------------------------
-// weights: warp w stages rows [16 w, 16 w + 16) of the tile (gated: warps 0..3, both matrices)
-template <bool DUAL>
-__device__ __forceinline__ void issue_w(const Product& pr, int u, int buf, uint32_t smem0, int warp, int lane) {
-  constexpr int AW = DUAL ? 4 : 8;
-  if (warp >= AW) return;
+// weights of one unit: the warp's rows (gated: of both matrices), 512 bytes each, one row per warp-wide copy
+template <int NT, bool DUAL>
+__device__ __forceinline__ void issue_w(const Product& pr, int u, uint32_t stage_smem, int warp, int lane) {
+  using S = Shape<NT, DUAL>;
   const int tile = u / pr.steps, step = u - tile * pr.steps;
-  const int row0 = tile * (AW * 16) + warp * 16;
+  const int row0 = tile * S::TR + warp * 16;
   const int k = step * KSTEP + lane * 8;
   const bool kin = k < pr.K;   // K is a multiple of 8
 #pragma unroll
-  for (int ti = 0; ti < (DUAL ? 2 : 1); ++ti) {
+  for (int ti = 0; ti < S::TILES; ++ti) {
     const __nv_bfloat16* W = static_cast<const __nv_bfloat16*>(ti ? pr.W1 : pr.W0) + k;
-    const uint32_t dst = smem0 + buf * W_STAGE + (DUAL ? 2 * warp + ti : warp) * TILE_BYTES + lane * 16;
+    const uint32_t dst = stage_smem + ti * TILE_BYTES + lane * 16;
 #pragma unroll 4
     for (int r = 0; r < 16; ++r) {
       const int n = row0 + r;
@@ -88,50 +103,58 @@ __device__ __forceinline__ void issue_w(const Product& pr, int u, int buf, uint3
     }
   }
 }
-// tokens: T rows of 512 bytes (twice that for a gated pair with two inputs), dealt to the eight warps;
-// rows T .. 8 NT - 1 of a slab are never written and only feed accumulator columns that nobody reads
-template <int NT>
-__device__ __forceinline__ void issue_x(const Product& pr, int T, int u, int buf, uint32_t xs0, int warp, int lane) {
-  constexpr int TP = 8 * NT;
+// the warp's own copy of the token rows of the unit's k range; rows T .. 8 NT - 1 of a slab are never
+// written and only feed accumulator columns that nobody reads
+template <int NT, bool DUAL>
+__device__ __forceinline__ void issue_x(const Product& pr, int T, int u, uint32_t stage_smem, int lane) {
+  using S = Shape<NT, DUAL>;
   const int step = u % pr.steps;
-  const int slabs = (pr.W1 != nullptr && pr.X1 != pr.X0) ? 2 : 1;
   const int k = step * KSTEP + lane * 8;
   const bool ok = k < pr.K;
-  for (int q = warp; q < slabs * T; q += WARPS) {
-    const int xi = q >= T ? 1 : 0, t = q - xi * T;
-    const __nv_bfloat16* X = static_cast<const __nv_bfloat16*>(xi ? pr.X1 : pr.X0);
-    cp_async16(xs0 + buf * (2 * TP * ROW_PITCH) + (xi * TP + t) * ROW_PITCH + lane * 16,
-               X + (ok ? static_cast<long long>(t) * pr.ldx + k : 0), ok);
+  const int slabs = (DUAL && pr.X1 != pr.X0) ? 2 : 1;
+  for (int xi = 0; xi < slabs; ++xi) {
+    const __nv_bfloat16* X = static_cast<const __nv_bfloat16*>(xi ? pr.X1 : pr.X0) + (ok ? k : 0);
+    const uint32_t dst = stage_smem + S::W_BYTES + xi * (S::TP * ROW_PITCH) + lane * 16;
+    for (int t = 0; t < T; ++t) cp_async16(dst + t * ROW_PITCH, ok ? X + static_cast<long long>(t) * pr.ldx : X, ok);
   }
 }
 
+// One unit: the warp's 16 rows x 256 k against the token rows.
 template <int NT, bool DUAL>
-__device__ __forceinline__ void compute(float (&acc)[DUAL ? 2 : 1][NT][4], bool two_slabs, int buf, uint32_t smem0,
-                                        uint32_t xs0, int warp, int lane) {
-  constexpr int AW = DUAL ? 4 : 8, TILES = DUAL ? 2 : 1, TP = 8 * NT;
-  if (warp >= AW) return;
+__device__ __forceinline__ void compute(float (&acc)[DUAL ? 2 : 1][NT][4], const Product& pr, int T, int step,
+                                        uint32_t stage_smem, int lane) {
+  using S = Shape<NT, DUAL>;
   const int g = lane >> 2, c = lane & 3;
-  const uint32_t src0 = smem0 + buf * W_STAGE + (DUAL ? 2 * warp : warp) * TILE_BYTES + g * ROW_PITCH + c * 16;
-  const uint32_t xsrc = xs0 + buf * (2 * TP * ROW_PITCH) + g * ROW_PITCH + c * 16;
-  const uint32_t x1off = two_slabs ? TP * ROW_PITCH : 0;
+  const bool two = DUAL && pr.X1 != pr.X0;
+  const uint32_t wsrc = stage_smem + g * ROW_PITCH + c * 16;
+  const uint32_t xsrc = stage_smem + S::W_BYTES + g * ROW_PITCH + c * 16;
 #pragma unroll 2
   for (int it = 0; it < 8; ++it) {
-    // rows g and g + 8 of the tile, the same 16 bytes of k: used as they are for two MMAs
-    uint4 lo[TILES], hi[TILES];
+    const int k = step * KSTEP + (it * 4 + c) * 8;
 #pragma unroll
-    for (int ti = 0; ti < TILES; ++ti) {
-      lo[ti] = lds128(src0 + ti * TILE_BYTES + it * 64);
-      hi[ti] = lds128(src0 + ti * TILE_BYTES + 8 * ROW_PITCH + it * 64);
-    }
+    for (int ti = 0; ti < S::TILES; ++ti) {
+      uint4 xb[NT];
+      if (S::PRIV) {
+        const uint32_t xs = xsrc + ((ti && two) ? S::TP * ROW_PITCH : 0) + it * 64;
 #pragma unroll
-    for (int j = 0; j < NT; ++j) {
-      const uint4 xb = lds128(xsrc + 8 * j * ROW_PITCH + it * 64);
-      mma_bf16(acc[0][j], lo[0].x, hi[0].x, lo[0].y, hi[0].y, xb.x, xb.y);
-      mma_bf16(acc[0][j], lo[0].z, hi[0].z, lo[0].w, hi[0].w, xb.z, xb.w);
-      if (DUAL) {
-        const uint4 xu = two_slabs ? lds128(xsrc + x1off + 8 * j * ROW_PITCH + it * 64) : xb;
-        mma_bf16(acc[TILES - 1][j], lo[TILES - 1].x, hi[TILES - 1].x, lo[TILES - 1].y, hi[TILES - 1].y, xu.x, xu.y);
-        mma_bf16(acc[TILES - 1][j], lo[TILES - 1].z, hi[TILES - 1].z, lo[TILES - 1].w, hi[TILES - 1].w, xu.z, xu.w);
+        for (int j = 0; j < NT; ++j) xb[j] = lds128(xs + 8 * j * ROW_PITCH);
+      } else {
+        const __nv_bfloat16* X = static_cast<const __nv_bfloat16*>((ti && two) ? pr.X1 : pr.X0) + k;
+#pragma unroll
+        for (int j = 0; j < NT; ++j) {
+          const int t = 8 * j + g;
+          xb[j] = (k < pr.K && t < T) ? __ldg(reinterpret_cast<const uint4*>(X + static_cast<long long>(t) * pr.ldx))
+                                      : make_uint4(0u, 0u, 0u, 0u);
+        }
+      }
+      // rows g and g + 8 of the tile, the same 16 bytes of k: used as they are for two MMAs (the order
+      // in which a contraction visits k is free as long as both operands agree on it)
+      const uint32_t ws = wsrc + ti * TILE_BYTES + it * 64;
+      const uint4 lo = lds128(ws), hi = lds128(ws + 8 * ROW_PITCH);
+#pragma unroll
+      for (int j = 0; j < NT; ++j) {
+        mma_bf16(acc[ti][j], lo.x, hi.x, lo.y, hi.y, xb[j].x, xb[j].y);
+        mma_bf16(acc[ti][j], lo.z, hi.z, lo.w, hi.w, xb[j].z, xb[j].w);
       }
     }
   }
@@ -181,25 +204,29 @@ __device__ __noinline__ bool grid_barrier(int* ctrl, int* s_flag) {
 }
 
 // ---- one product -------------------------------------------------------------------------------
+// The working warps of a CTA walk the CTA's share side by side but do not wait for one another: each
+// has its own ring of stages, its own accumulators, and finishes its rows of a tile by itself (ticket
+// per tile and warp).
 // `first`: the product opens the kernel (its inputs come from the launch before: wait for that one);
 // otherwise its inputs come from the product before (grid barrier).  Either wait sits behind the
-// first two weight copies.  Returns false if the barrier gave up.
+// first weight copies.  Returns false if the barrier gave up.
 template <int NT, bool DUAL>
 __device__ __forceinline__ bool run_product(const Product& pr, const Params& p, bool first, uint32_t smem0,
-                                            uint32_t xs0, int* s_flag, int* s_slot) {
-  constexpr int AW = DUAL ? 4 : 8, TR = AW * 16, TILES = DUAL ? 2 : 1, TP = 8 * NT;
-  constexpr int SLOT = 128 * TP;   // floats of one partial: [TILES][TR][TP]
-  constexpr int EPT = TR * TP / (4 * THREADS) > 0 ? TR * TP / (4 * THREADS) : 1;   // float4 sums per thread when partials are added
+                                            int* s_flag) {
+  using S = Shape<NT, DUAL>;
+  constexpr int TILES = S::TILES, TR = S::TR, TP = S::TP, NST = S::NST;
+  constexpr int SLOT = 128 * TP;              // floats of one CTA partial: [TILES][TR][TP]
+  constexpr int ROWV = 16 * TP / 4;           // float4 values of the warp's rows (one matrix)
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = lane >> 2, c = lane & 3;
   const unsigned U = static_cast<unsigned>(pr.tiles) * pr.steps;
   const unsigned ge = U < gridDim.x ? U : gridDim.x;   // CTAs with a share
   const int cta = blockIdx.x;
-  const bool mine = cta < static_cast<int>(ge);
+  const bool mine = cta < static_cast<int>(ge) && warp < S::AW;
   const int u0 = mine ? share_lo(cta, U, ge) : 0, u1 = mine ? share_lo(cta + 1, U, ge) : 0;
   const int n = u1 - u0;
-  const bool two_slabs = DUAL && pr.X1 != pr.X0;
   const GeluCoef gc = gelu_coef(pr.epi.act);
+  const uint32_t my_smem = smem0 + warp * (NST * S::STAGE);
 
   float acc[TILES][NT][4];
 #pragma unroll
@@ -212,108 +239,99 @@ __device__ __forceinline__ bool run_product(const Product& pr, const Params& p, 
   const int first_tile = u0 / pr.steps;
   int tile = first_tile, step = u0 - first_tile * pr.steps;
   int seg_lo = step;
-  // q = -2, -1: the weights of units 0 and 1 go out ahead of the wait; from q = 0 on the pipeline runs
-  for (int q = -2; q < n || q <= 0; ++q) {
+  // q < 0: the weights of the first units go out ahead of the wait; from q = 0 on the pipeline runs.
+  // Copy groups: with private token rows the first group holds W(0), W(1), X(0), the second X(1), then
+  // one group per unit; without, one group per unit from the start.
+  for (int q = -NST; q < n || q <= 0; ++q) {
     if (q == 0) {
       if (first) asm volatile("griddepcontrol.wait;" ::: "memory");
       else if (!grid_barrier(p.ctrl, s_flag)) return false;
-      if (n > 0) { issue_x<NT>(pr, p.T, u0, 0, xs0, warp, lane); asm volatile("cp.async.commit_group;" ::: "memory"); }
-      if (n > 1) { issue_x<NT>(pr, p.T, u0 + 1, 1, xs0, warp, lane); asm volatile("cp.async.commit_group;" ::: "memory"); }
       if (n == 0) break;
-    }
-    if (q >= 0) {
-      if (q + 1 < n) asm volatile("cp.async.wait_group 1;" ::: "memory");
-      else asm volatile("cp.async.wait_group 0;" ::: "memory");
-      __syncthreads();   // unit q of every warp has landed: the token rows are shared
-      compute<NT, DUAL>(acc, two_slabs, q & 1, smem0, xs0, warp, lane);
-      __syncthreads();   // its stage is free again
-    }
-    if (q + 2 < n) {
-      issue_w<DUAL>(pr, u0 + q + 2, q & 1, smem0, warp, lane);
-      if (q >= 0) {
-        issue_x<NT>(pr, p.T, u0 + q + 2, q & 1, xs0, warp, lane);
+      if (S::PRIV) {
+        issue_x<NT, DUAL>(pr, p.T, u0, my_smem, lane);
         asm volatile("cp.async.commit_group;" ::: "memory");
+        if (n > 1) {
+          issue_x<NT, DUAL>(pr, p.T, u0 + 1, my_smem + S::STAGE, lane);
+          asm volatile("cp.async.commit_group;" ::: "memory");
+        }
       }
+    }
+    const uint32_t stage_smem = my_smem + ((q + NST) % NST) * S::STAGE;
+    if (q >= 0) {
+      const int ahead = n - 1 - q;   // units issued behind this one, NST - 1 at most
+      if (NST >= 3 && ahead >= 2) asm volatile("cp.async.wait_group 2;" ::: "memory");
+      else if (ahead >= 1) asm volatile("cp.async.wait_group 1;" ::: "memory");
+      else asm volatile("cp.async.wait_group 0;" ::: "memory");
+      __syncwarp();
+      compute<NT, DUAL>(acc, pr, p.T, step, stage_smem, lane);
+      __syncwarp();
+    }
+    if (q + NST < n) {
+      issue_w<NT, DUAL>(pr, u0 + q + NST, stage_smem, warp, lane);
+      if (S::PRIV && q >= 0) issue_x<NT, DUAL>(pr, p.T, u0 + q + NST, stage_smem, lane);
+      if (!S::PRIV || q >= 0) asm volatile("cp.async.commit_group;" ::: "memory");
     }
     if (q < 0) continue;
     if (step == pr.steps - 1 || q == n - 1) {
-      // ---- end of this CTA's part of the tile
+      // ---- end of this warp's part of the tile
+      const int wrow = warp * 16;   // the warp's first row inside the tile
       if (seg_lo == 0 && step == pr.steps - 1) {
-        if (warp < AW) {
-          const int n0 = tile * TR + warp * 16 + g;
 #pragma unroll
-          for (int j = 0; j < NT; ++j)
+        for (int j = 0; j < NT; ++j)
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-              const int nn = n0 + (e >= 2 ? 8 : 0), t = 8 * j + 2 * c + (e & 1);
-              const float v = DUAL ? silu_fast(acc[0][j][e]) * acc[TILES - 1][j][e] : acc[0][j][e];
-              if (nn < pr.N && t < p.T) store_out<DUAL>(pr.epi, gc, nn, t, v);
-            }
-        }
+          for (int e = 0; e < 4; ++e) {
+            const int nn = tile * TR + wrow + g + (e >= 2 ? 8 : 0), t = 8 * j + 2 * c + (e & 1);
+            const float v = DUAL ? silu_fast(acc[0][j][e]) * acc[TILES - 1][j][e] : acc[0][j][e];
+            if (nn < pr.N && t < p.T) store_out<DUAL>(pr.epi, gc, nn, t, v);
+          }
       } else {
         float* dst = p.partial + static_cast<long long>(2 * cta + (tile == first_tile ? 0 : 1)) * SLOT;
-        if (warp < AW) {
 #pragma unroll
-          for (int i = 0; i < TILES; ++i)
+        for (int i = 0; i < TILES; ++i)
 #pragma unroll
-            for (int j = 0; j < NT; ++j) {
-              float* d0 = dst + (i * TR + warp * 16 + g) * TP + 8 * j + 2 * c;
-              *reinterpret_cast<float2*>(d0) = make_float2(acc[i][j][0], acc[i][j][1]);
-              *reinterpret_cast<float2*>(d0 + 8 * TP) = make_float2(acc[i][j][2], acc[i][j][3]);
-            }
-        }
+          for (int j = 0; j < NT; ++j) {
+            float* d0 = dst + (i * TR + wrow + g) * TP + 8 * j + 2 * c;
+            *reinterpret_cast<float2*>(d0) = make_float2(acc[i][j][0], acc[i][j][1]);
+            *reinterpret_cast<float2*>(d0 + 8 * TP) = make_float2(acc[i][j][2], acc[i][j][3]);
+          }
         const unsigned t_lo = static_cast<unsigned>(tile) * pr.steps;
         const int c_first = cta_of(t_lo, U, ge), c_last = cta_of(t_lo + pr.steps - 1, U, ge);
         __threadfence();
-        __syncthreads();
-        if (threadIdx.x == 0) {
-          int* ticket = p.ctrl + kTicketWord0 + tile;
-          const int arrived = atomicAdd(ticket, 1);
-          const int last = arrived == c_last - c_first;
-          if (last) *ticket = 0;   // nobody else comes for this tile; the next product starts behind a barrier
-          *s_flag = last;
+        __syncwarp();
+        int last = 0;
+        if (lane == 0) {
+          int* ticket = p.ctrl + kTicketWord0 + tile * WARPS + warp;
+          last = atomicAdd(ticket, 1) == c_last - c_first;
+          if (last) *ticket = 0;   // nobody else comes for these rows; the next product starts behind a barrier
           __threadfence();
         }
-        __syncthreads();
-        if (*s_flag) {
-          // The partials of the tile, added in CTA order.  Which of its two slots a CTA used is worked
-          // out once per CTA; then every thread sums four neighbouring values, with many loads in flight.
+        last = __shfl_sync(0xffffffffu, last, 0);
+        if (last) {
+          // The partials of these rows, added in CTA order.  Which of its two slots a CTA used is worked
+          // out by one lane per CTA and handed round; each lane sums four neighbouring values at a time.
           const int ncon = c_last - c_first + 1;
-          float4 sum0[EPT], sum1[EPT];
-#pragma unroll
-          for (int e = 0; e < EPT; ++e) sum0[e] = sum1[e] = make_float4(0.f, 0.f, 0.f, 0.f);
-          for (int i0 = 0; i0 < ncon; i0 += kSlotTable) {
-            const int nc = ncon - i0 < kSlotTable ? ncon - i0 : kSlotTable;
-            __syncthreads();
-            for (int i = threadIdx.x; i < nc; i += THREADS) {
-              const int cc = c_first + i0 + i;
-              s_slot[i] = 2 * cc + (share_lo(cc, U, ge) / pr.steps == tile ? 0 : 1);
-            }
-            __syncthreads();
-#pragma unroll
-            for (int e = 0; e < EPT; ++e) {
-              const int idx = 4 * (threadIdx.x + e * THREADS);
-              if (idx >= TR * TP) break;
+          const float* base = p.partial + wrow * TP;
+          for (int v4 = lane; v4 < ROWV; v4 += 32) {
+            float4 s0 = make_float4(0.f, 0.f, 0.f, 0.f), s1 = s0;
+            for (int i0 = 0; i0 < ncon; i0 += 32) {
+              const int nc = ncon - i0 < 32 ? ncon - i0 : 32;
+              const int cc = c_first + i0 + (lane < nc ? lane : 0);
+              const int my_slot = 2 * cc + (share_lo(cc, U, ge) / pr.steps == tile ? 0 : 1);
 #pragma unroll 8
               for (int i = 0; i < nc; ++i) {
-                const float* src = p.partial + static_cast<long long>(s_slot[i]) * SLOT + idx;
-                const float4 a = __ldcg(reinterpret_cast<const float4*>(src));
-                sum0[e].x += a.x; sum0[e].y += a.y; sum0[e].z += a.z; sum0[e].w += a.w;
+                const float* src = base + static_cast<long long>(__shfl_sync(0xffffffffu, my_slot, i)) * SLOT;
+                const float4 a = __ldcg(reinterpret_cast<const float4*>(src) + v4);
+                s0.x += a.x; s0.y += a.y; s0.z += a.z; s0.w += a.w;
                 if (DUAL) {
-                  const float4 b = __ldcg(reinterpret_cast<const float4*>(src + TR * TP));
-                  sum1[e].x += b.x; sum1[e].y += b.y; sum1[e].z += b.z; sum1[e].w += b.w;
+                  const float4 b = __ldcg(reinterpret_cast<const float4*>(src + TR * TP) + v4);
+                  s1.x += b.x; s1.y += b.y; s1.z += b.z; s1.w += b.w;
                 }
               }
             }
-          }
-#pragma unroll
-          for (int e = 0; e < EPT; ++e) {
-            const int idx = 4 * (threadIdx.x + e * THREADS);
-            if (idx >= TR * TP) break;
-            const int r = idx / TP, t = idx - r * TP;
-            const int nn = tile * TR + r;
-            const float a[4] = {sum0[e].x, sum0[e].y, sum0[e].z, sum0[e].w};
-            const float b[4] = {sum1[e].x, sum1[e].y, sum1[e].z, sum1[e].w};
+            const int r = (4 * v4) / TP, t = 4 * v4 - r * TP;
+            const int nn = tile * TR + wrow + r;
+            const float a[4] = {s0.x, s0.y, s0.z, s0.w};
+            const float b[4] = {s1.x, s1.y, s1.z, s1.w};
 #pragma unroll
             for (int x = 0; x < 4; ++x)
               if (nn < pr.N && t + x < p.T) store_out<DUAL>(pr.epi, gc, nn, t + x, DUAL ? silu_fast(a[x]) * b[x] : a[x]);
@@ -338,15 +356,13 @@ template <int NT, bool GATED>
 __global__ void __launch_bounds__(THREADS, 1) decode_layer_kernel(const __grid_constant__ Params p) {
   extern __shared__ __align__(16) unsigned char smem[];
   __shared__ int s_flag;
-  __shared__ int s_slot[kSlotTable];
   const uint32_t smem0 = static_cast<uint32_t>(__cvta_generic_to_shared(smem));
-  const uint32_t xs0 = smem0 + W_BYTES;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // a dependent launch may start its own first copies
   for (int pi = 0; pi < p.nprod; ++pi) {
     const Product& pr = p.prod[pi];
     bool ok;
-    if (GATED && pr.W1) ok = run_product<NT, true>(pr, p, pi == 0, smem0, xs0, &s_flag, s_slot);
-    else ok = run_product<NT, false>(pr, p, pi == 0, smem0, xs0, &s_flag, s_slot);
+    if (GATED && pr.W1) ok = run_product<NT, true>(pr, p, pi == 0, smem0, &s_flag);
+    else ok = run_product<NT, false>(pr, p, pi == 0, smem0, &s_flag);
     if (!ok) {
       asm volatile("cp.async.wait_all;" ::: "memory");
       return;
@@ -359,14 +375,14 @@ template <int NT, bool GATED>
 cudaError_t launch_nt(const Params& p, int grid, bool cooperative, cudaStream_t st) {
   static bool attr_done = false;
   if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(decode_layer_kernel<NT, GATED>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_bytes<NT>());
+    cudaError_t e = cudaFuncSetAttribute(decode_layer_kernel<NT, GATED>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
     attr_done = true;
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid);
   cfg.blockDim = dim3(THREADS);
-  cfg.dynamicSmemBytes = smem_bytes<NT>();
+  cfg.dynamicSmemBytes = SMEM_BYTES;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   if (cooperative) {
@@ -413,7 +429,7 @@ ffsplit_status decode_layer_add(ffsplit_ctx* ctx, DecodeLayerPlan* plan, const v
   pr.tiles = (N + tr - 1) / tr;
   pr.steps = (K + dec::KSTEP - 1) / dec::KSTEP;
   pr.epi = epi;
-  if (pr.tiles > kMaxTicketTiles) return fail(ctx, FFSPLIT_ERR_SHAPE, "few-token forward: more row tiles than ticket counters");
+  if (static_cast<long long>(pr.tiles) * 8 > kMaxTicketTiles) return fail(ctx, FFSPLIT_ERR_SHAPE, "few-token forward: more row tiles than ticket counters");
   if (static_cast<double>(pr.tiles) * pr.steps * (ctx->num_sms + 1) >= 2147483648.0)
     return fail(ctx, FFSPLIT_ERR_SHAPE, "few-token forward: product too large for the unit arithmetic");
   plan->prod[plan->n++] = pr;
