@@ -352,10 +352,6 @@ ffsplit_status ffsplit_create(ffsplit_ctx** out, int device) {
   c->cc_major = major;
   c->cc_minor = minor;
   c->num_sms = sms;
-  if (const char* env = std::getenv("FFSPLIT_DECODE_CTAS")) {
-    const int v = std::atoi(env);
-    if (v >= 1 && v <= 64) c->decode_ctas_per_sm_target = v;
-  }
   if (const char* env = std::getenv("FFSPLIT_DECODE_LAYER")) c->decode_one_launch = env[0] == '0' ? 0 : 1;
   *out = c;
   return FFSPLIT_OK;

@@ -1,4 +1,4 @@
-// Few-token (decode) split forward, T <= 32 tokens: every product of Eq. 2 in one persistent kernel.
+// Few-token (decode) split forward, T <= 64 tokens: every product of Eq. 2 in one persistent kernel.
 //
 // With a handful of tokens each stage of Eq. 2 is a skinny product
 //     C[t, n] = epi( sum_k X[t, k] * W[n, k] )        W: [N, K] K-major weights from the packed blob
@@ -401,18 +401,19 @@ cudaError_t launch_any(int nt, bool gated, const Params& p, int grid, bool coope
 #define FFS_DL(NT_) (gated ? launch_nt<NT_, true>(p, grid, cooperative, st) : launch_nt<NT_, false>(p, grid, cooperative, st))
   if (nt == 1) return FFS_DL(1);
   if (nt == 2) return FFS_DL(2);
-  return FFS_DL(4);
+  if (nt == 4) return FFS_DL(4);
+  return FFS_DL(8);
 #undef FFS_DL
 }
 
 }  // namespace dsk
 
 // ---- host side ---------------------------------------------------------------------------------
-bool decode_layer_applies(long long T) { return T >= 1 && T <= 32; }
+bool decode_layer_applies(long long T) { return T >= 1 && T <= 64; }
 
 // fp32 partials: two slots per CTA
 size_t decode_layer_scratch_bytes(int num_sms, long long T) {
-  const int nt = T <= 8 ? 1 : T <= 16 ? 2 : 4;
+  const int nt = T <= 8 ? 1 : T <= 16 ? 2 : T <= 32 ? 4 : 8;
   return static_cast<size_t>(2) * num_sms * 128 * 8 * nt * 4;
 }
 
@@ -441,7 +442,7 @@ ffsplit_status decode_layer_add(ffsplit_ctx* ctx, DecodeLayerPlan* plan, const v
 ffsplit_status decode_layer_launch(ffsplit_ctx* ctx, const DecodeLayerPlan* plan, int T, float* partial, int* ctrl,
                                    cudaStream_t st) {
   if (plan->n == 0) return FFSPLIT_OK;
-  const int nt = T <= 8 ? 1 : T <= 16 ? 2 : 4;
+  const int nt = T <= 8 ? 1 : T <= 16 ? 2 : T <= 32 ? 4 : 8;
   bool gated = false;
   for (int i = 0; i < plan->n; ++i) gated = gated || plan->prod[i].W1 != nullptr;
   // cooperative launch: supported, and one CTA per SM fits

@@ -162,8 +162,7 @@ struct ffsplit_ctx {
   bool attr_fused_set = false;
   int* status() const { return reinterpret_cast<int*>(ws); }
   int* tickets() const { return reinterpret_cast<int*>(ws + ffsp::kStatusBytes); }
-  int decode_ctas_per_sm_target = 6;   // T > 32: CTAs per SM the per-product kernel aims for when splitting K (FFSPLIT_DECODE_CTAS overrides)
-  int decode_one_launch = 0;   // T <= 32: 1 = all products in one cooperative launch (FFSPLIT_DECODE_LAYER=1), 0 = one launch per product
+  int decode_one_launch = 0;   // few-token forward: 1 = all products in one cooperative launch (FFSPLIT_DECODE_LAYER=1), 0 = one launch per product
   int use_fused = -1;  // -1: not decided yet (environment FFSPLIT_NO_FUSED=1 turns the fused kernel off)
 };
 
@@ -178,7 +177,7 @@ inline size_t elem_size(int dtype) { return dtype == FFSPLIT_BF16 ? 2 : 4; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // ----------------------------------------------------------------------------
-// Few-token forward (T <= 32): the products of one layer, run by one persistent kernel
+// Few-token forward (T <= 64): the products of one layer, run by one persistent kernel
 // (decode_layer.cu).  C[t, n] = epi(sum_k X[t, k] W[n, k]); W1 != nullptr: gated pair.
 // ----------------------------------------------------------------------------
 struct DecodeProduct {
