@@ -35,6 +35,7 @@
 #include "decode_common.cuh"
 #include "epilogue.cuh"
 #include "internal.h"
+#include "ptx.cuh"
 
 namespace ffsp {
 namespace dsk {
@@ -43,6 +44,9 @@ using namespace dec;
 
 constexpr int WARPS = 8, THREADS = WARPS * 32;
 constexpr int SMEM_BYTES = 3 * 8 * TILE_BYTES;   // the same for every shape below
+constexpr int RING_BYTES = 2 * 8 * TILE_BYTES;   // weight rings of the warps; the rest holds token rows
+constexpr int XCAP_BYTES = SMEM_BYTES - RING_BYTES;   // shared token slabs (more than 8 tokens)
+constexpr int kMaxSlots = 8;                     // slabs in the shared ring, at most
 constexpr int kBarCount = 16, kBarGen = 17;     // words of the control block used by the grid barrier
 constexpr int kTicketWord0 = static_cast<int>(kStatusBytes / 4);   // tickets follow the status block
 constexpr long long kWaitLimit = 2000000000ll;  // clock cycles (about a second) before a barrier wait gives up
@@ -57,14 +61,18 @@ struct Params {
   int* ctrl;        // control block: status words, barrier words, then eight tickets per row tile (zero between launches)
 };
 
-// A CTA tile is 128 weight rows (64 rows of each matrix for a gated pair); warp w owns 16 of them.
-// Up to 8 tokens (NT = 1 token tile) a warp's stage holds its weight rows and a private copy of the
-// token rows, two stages deep.  With more tokens the copies would not fit: the token rows are then
-// loaded where they are used (through L1), and the ring is three stages of weights.
+// A CTA tile is 128 weight rows (64 rows of each matrix for a gated pair); warp w owns 16 of them and
+// has a two-stage ring for them.  The token rows of a unit's k range (a slab) are staged too:
+//  * up to 8 tokens (NT = 1 token tile) every warp copies them for itself, in the same copy group as its
+//    weights: no warp ever waits for another;
+//  * with more tokens private copies neither fit nor pay (they would outweigh the weights), so the CTA
+//    keeps one ring of slabs.  All warps load a share of each slab, a few units ahead, and meet only
+//    through two mbarriers per slot: `full` (the slab has landed: every thread's copies, tracked by
+//    cp.async.mbarrier.arrive) and `empty` (every warp is done reading it).
 template <int NT, bool DUAL>
 struct Shape {
-  static constexpr bool PRIV = NT == 1;              // token rows staged with the weights
-  static constexpr int NST = PRIV ? 2 : 3;           // stages of a warp's ring
+  static constexpr bool PRIV = NT == 1;              // token rows staged per warp
+  static constexpr int NST = 2;                      // stages of a warp's ring
   static constexpr int TILES = DUAL ? 2 : 1;
   static constexpr int AW = DUAL ? 4 : 8;            // working warps
   static constexpr int TR = AW * 16;                 // rows of a CTA tile
@@ -72,7 +80,8 @@ struct Shape {
   static constexpr int W_BYTES = TILES * TILE_BYTES;
   static constexpr int X_BYTES = PRIV ? TILES * TP * ROW_PITCH : 0;   // a gated pair may have two inputs
   static constexpr int STAGE = W_BYTES + X_BYTES;
-  static_assert(AW * NST * STAGE == SMEM_BYTES, "shared memory plan");
+  static_assert(AW * NST * STAGE == (PRIV ? SMEM_BYTES : RING_BYTES), "shared memory plan");
+  static_assert(PRIV || TILES * TP * ROW_PITCH <= XCAP_BYTES, "one slab must fit");
 };
 
 // Shares of the `ge` CTAs that have one: CTA c owns units [c U / ge, (c + 1) U / ge).  U * (ge + 1) fits
@@ -119,34 +128,23 @@ __device__ __forceinline__ void issue_x(const Product& pr, int T, int u, uint32_
   }
 }
 
-// One unit: the warp's 16 rows x 256 k against the token rows.
+// One unit: the warp's 16 rows x 256 k against the token rows at xsmem (a second input, if there
+// is one, follows 8 NT rows later).
 template <int NT, bool DUAL>
-__device__ __forceinline__ void compute(float (&acc)[DUAL ? 2 : 1][NT][4], const Product& pr, int T, int step,
-                                        uint32_t stage_smem, int lane) {
+__device__ __forceinline__ void compute(float (&acc)[DUAL ? 2 : 1][NT][4], bool two, uint32_t stage_smem,
+                                        uint32_t xsmem, int lane) {
   using S = Shape<NT, DUAL>;
   const int g = lane >> 2, c = lane & 3;
-  const bool two = DUAL && pr.X1 != pr.X0;
   const uint32_t wsrc = stage_smem + g * ROW_PITCH + c * 16;
-  const uint32_t xsrc = stage_smem + S::W_BYTES + g * ROW_PITCH + c * 16;
+  const uint32_t xsrc = xsmem + g * ROW_PITCH + c * 16;
 #pragma unroll 2
   for (int it = 0; it < 8; ++it) {
-    const int k = step * KSTEP + (it * 4 + c) * 8;
 #pragma unroll
     for (int ti = 0; ti < S::TILES; ++ti) {
       uint4 xb[NT];
-      if (S::PRIV) {
-        const uint32_t xs = xsrc + ((ti && two) ? S::TP * ROW_PITCH : 0) + it * 64;
+      const uint32_t xs = xsrc + ((ti && two) ? S::TP * ROW_PITCH : 0) + it * 64;
 #pragma unroll
-        for (int j = 0; j < NT; ++j) xb[j] = lds128(xs + 8 * j * ROW_PITCH);
-      } else {
-        const __nv_bfloat16* X = static_cast<const __nv_bfloat16*>((ti && two) ? pr.X1 : pr.X0) + k;
-#pragma unroll
-        for (int j = 0; j < NT; ++j) {
-          const int t = 8 * j + g;
-          xb[j] = (k < pr.K && t < T) ? __ldg(reinterpret_cast<const uint4*>(X + static_cast<long long>(t) * pr.ldx))
-                                      : make_uint4(0u, 0u, 0u, 0u);
-        }
-      }
+      for (int j = 0; j < NT; ++j) xb[j] = lds128(xs + 8 * j * ROW_PITCH);
       // rows g and g + 8 of the tile, the same 16 bytes of k: used as they are for two MMAs (the order
       // in which a contraction visits k is free as long as both operands agree on it)
       const uint32_t ws = wsrc + ti * TILE_BYTES + it * 64;
@@ -158,6 +156,21 @@ __device__ __forceinline__ void compute(float (&acc)[DUAL ? 2 : 1][NT][4], const
       }
     }
   }
+}
+
+// This warp's share of a shared slab: token rows warp, warp + 8, ... of each input; then every lane
+// tells the slot's `full` barrier to count it in once its copies have landed.
+__device__ __forceinline__ void issue_x_shared(const Product& pr, int T, int TP, int slabs, int u, uint32_t slab_smem,
+                                               uint64_t* full, int warp, int lane) {
+  const int step = u % pr.steps;
+  const int k = step * KSTEP + lane * 8;
+  const bool ok = k < pr.K;
+  for (int xi = 0; xi < slabs; ++xi) {
+    const __nv_bfloat16* X = static_cast<const __nv_bfloat16*>(xi ? pr.X1 : pr.X0) + (ok ? k : 0);
+    const uint32_t dst = slab_smem + xi * (TP * ROW_PITCH) + lane * 16;
+    for (int t = warp; t < T; t += WARPS) cp_async16(dst + t * ROW_PITCH, ok ? X + static_cast<long long>(t) * pr.ldx : X, ok);
+  }
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(ptx::smem_u32(full)) : "memory");
 }
 
 // bias, activation and the [C0 | C1] column split for one output value (gated values arrive finished)
@@ -204,15 +217,14 @@ __device__ __noinline__ bool grid_barrier(int* ctrl, int* s_flag) {
 }
 
 // ---- one product -------------------------------------------------------------------------------
-// The working warps of a CTA walk the CTA's share side by side but do not wait for one another: each
-// has its own ring of stages, its own accumulators, and finishes its rows of a tile by itself (ticket
-// per tile and warp).
+// The working warps of a CTA walk the CTA's share side by side: each has its own ring of weight
+// stages, its own accumulators, and finishes its rows of a tile by itself (ticket per tile and warp).
 // `first`: the product opens the kernel (its inputs come from the launch before: wait for that one);
 // otherwise its inputs come from the product before (grid barrier).  Either wait sits behind the
-// first weight copies.  Returns false if the barrier gave up.
+// first weight copies.  Returns false if a wait gave up.
 template <int NT, bool DUAL>
 __device__ __forceinline__ bool run_product(const Product& pr, const Params& p, bool first, uint32_t smem0,
-                                            int* s_flag) {
+                                            int* s_flag, uint64_t* full, uint64_t* empty, volatile int* s_abort) {
   using S = Shape<NT, DUAL>;
   constexpr int TILES = S::TILES, TR = S::TR, TP = S::TP, NST = S::NST;
   constexpr int SLOT = 128 * TP;              // floats of one CTA partial: [TILES][TR][TP]
@@ -222,11 +234,19 @@ __device__ __forceinline__ bool run_product(const Product& pr, const Params& p, 
   const unsigned U = static_cast<unsigned>(pr.tiles) * pr.steps;
   const unsigned ge = U < gridDim.x ? U : gridDim.x;   // CTAs with a share
   const int cta = blockIdx.x;
-  const bool mine = cta < static_cast<int>(ge) && warp < S::AW;
-  const int u0 = mine ? share_lo(cta, U, ge) : 0, u1 = mine ? share_lo(cta + 1, U, ge) : 0;
-  const int n = u1 - u0;
+  const bool has = cta < static_cast<int>(ge);
+  const bool worker = warp < S::AW;            // the other warps only help with shared slabs
+  const int u0 = has ? share_lo(cta, U, ge) : 0, u1 = has ? share_lo(cta + 1, U, ge) : 0;
+  const int n = (S::PRIV && !worker) ? 0 : u1 - u0;
+  const bool two = DUAL && pr.X1 != pr.X0;
   const GeluCoef gc = gelu_coef(pr.epi.act);
   const uint32_t my_smem = smem0 + warp * (NST * S::STAGE);
+  // shared slabs: as many slots as fit, filled LOOK units ahead of their use
+  const int slabs = two ? 2 : 1;
+  const int slab_bytes = slabs * TP * ROW_PITCH;
+  const int R = XCAP_BYTES / slab_bytes < kMaxSlots ? XCAP_BYTES / slab_bytes : kMaxSlots;
+  const int LOOK = R - 1;
+  const uint32_t xring = smem0 + RING_BYTES;
 
   float acc[TILES][NT][4];
 #pragma unroll
@@ -240,8 +260,8 @@ __device__ __forceinline__ bool run_product(const Product& pr, const Params& p, 
   int tile = first_tile, step = u0 - first_tile * pr.steps;
   int seg_lo = step;
   // q < 0: the weights of the first units go out ahead of the wait; from q = 0 on the pipeline runs.
-  // Copy groups: with private token rows the first group holds W(0), W(1), X(0), the second X(1), then
-  // one group per unit; without, one group per unit from the start.
+  // Copy groups of a worker, private token rows: W(0), W(1), X(0) | X(1) | then one per unit.
+  // Shared slabs: one group per unit from the start (a warp's slab copies ride in its next group).
   for (int q = -NST; q < n || q <= 0; ++q) {
     if (q == 0) {
       if (first) asm volatile("griddepcontrol.wait;" ::: "memory");
@@ -254,24 +274,44 @@ __device__ __forceinline__ bool run_product(const Product& pr, const Params& p, 
           issue_x<NT, DUAL>(pr, p.T, u0 + 1, my_smem + S::STAGE, lane);
           asm volatile("cp.async.commit_group;" ::: "memory");
         }
+      } else {
+        for (int j = 0; j < LOOK && j < n; ++j)
+          issue_x_shared(pr, p.T, TP, slabs, u0 + j, xring + j * slab_bytes, full + j, warp, lane);
       }
     }
     const uint32_t stage_smem = my_smem + ((q + NST) % NST) * S::STAGE;
     if (q >= 0) {
-      const int ahead = n - 1 - q;   // units issued behind this one, NST - 1 at most
-      if (NST >= 3 && ahead >= 2) asm volatile("cp.async.wait_group 2;" ::: "memory");
-      else if (ahead >= 1) asm volatile("cp.async.wait_group 1;" ::: "memory");
-      else asm volatile("cp.async.wait_group 0;" ::: "memory");
+      uint32_t xsmem = stage_smem + S::W_BYTES;
+      if (!S::PRIV) {
+        // the slab LOOK units ahead goes into the slot that unit q - 1 used: wait until every warp has read it
+        const int j = q + LOOK;
+        if (j < n) {
+          const int slot = j % R, use = j / R;
+          if (use > 0 && !ptx::mbar_wait(empty + slot, (use - 1) & 1, s_abort)) return false;
+          issue_x_shared(pr, p.T, TP, slabs, u0 + j, xring + slot * slab_bytes, full + slot, warp, lane);
+        }
+        xsmem = xring + (q % R) * slab_bytes;
+      }
+      if (worker) {
+        if (n - 1 - q >= 1) asm volatile("cp.async.wait_group 1;" ::: "memory");
+        else asm volatile("cp.async.wait_group 0;" ::: "memory");
+      }
+      if (!S::PRIV && !ptx::mbar_wait(full + q % R, (q / R) & 1, s_abort)) return false;
       __syncwarp();
-      compute<NT, DUAL>(acc, pr, p.T, step, stage_smem, lane);
+      if (worker) compute<NT, DUAL>(acc, two, stage_smem, xsmem, lane);
       __syncwarp();
+      if (!S::PRIV && lane == 0) ptx::mbar_arrive(empty + q % R);
     }
-    if (q + NST < n) {
+    if (worker && q + NST < n) {
       issue_w<NT, DUAL>(pr, u0 + q + NST, stage_smem, warp, lane);
       if (S::PRIV && q >= 0) issue_x<NT, DUAL>(pr, p.T, u0 + q + NST, stage_smem, lane);
       if (!S::PRIV || q >= 0) asm volatile("cp.async.commit_group;" ::: "memory");
     }
     if (q < 0) continue;
+    if (!worker) {
+      if (++step == pr.steps) { step = 0; ++tile; }
+      continue;
+    }
     if (step == pr.steps - 1 || q == n - 1) {
       // ---- end of this warp's part of the tile
       const int wrow = warp * 16;   // the warp's first row inside the tile
@@ -356,14 +396,27 @@ template <int NT, bool GATED>
 __global__ void __launch_bounds__(THREADS, 1) decode_layer_kernel(const __grid_constant__ Params p) {
   extern __shared__ __align__(16) unsigned char smem[];
   __shared__ int s_flag;
+  __shared__ int s_abort;
+  __shared__ __align__(8) uint64_t s_full[kMaxSlots], s_empty[kMaxSlots];
   const uint32_t smem0 = static_cast<uint32_t>(__cvta_generic_to_shared(smem));
+  if (threadIdx.x == 0) s_abort = 0;
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // a dependent launch may start its own first copies
   for (int pi = 0; pi < p.nprod; ++pi) {
     const Product& pr = p.prod[pi];
+    if (NT > 1) {
+      // slab barriers start every product in phase 0: `full` counts every thread, `empty` every warp
+      if (threadIdx.x == 0) {
+        for (int i = 0; i < kMaxSlots; ++i) { ptx::mbar_init(s_full + i, THREADS); ptx::mbar_init(s_empty + i, WARPS); }
+        ptx::mbar_fence_init();
+      }
+      __syncthreads();
+    }
     bool ok;
-    if (GATED && pr.W1) ok = run_product<NT, true>(pr, p, pi == 0, smem0, &s_flag);
-    else ok = run_product<NT, false>(pr, p, pi == 0, smem0, &s_flag);
+    if (GATED && pr.W1) ok = run_product<NT, true>(pr, p, pi == 0, smem0, &s_flag, s_full, s_empty, &s_abort);
+    else ok = run_product<NT, false>(pr, p, pi == 0, smem0, &s_flag, s_full, s_empty, &s_abort);
     if (!ok) {
+      // a wait ran out: say so, let the copies in flight land, leave
+      if ((threadIdx.x & 31) == 0) record_status(p.ctrl, FFSPLIT_ERR_TIMEOUT, static_cast<int>(blockIdx.x), KID_DECODE);
       asm volatile("cp.async.wait_all;" ::: "memory");
       return;
     }
