@@ -92,39 +92,43 @@ __device__ __forceinline__ int cta_of(unsigned u, unsigned U, unsigned ge) {
   return static_cast<int>(((u + 1) * ge - 1) / U);
 }
 
-// weights of one unit: the warp's rows (gated: of both matrices), 512 bytes each, one row per warp-wide copy
+// weights of one unit: the warp's 16 rows (gated: of both matrices), 512 bytes each, one row per warp-wide copy
 template <int NT, bool DUAL>
-__device__ __forceinline__ void issue_w(const Product& pr, int u, uint32_t stage_smem, int warp, int lane) {
+__device__ __forceinline__ void issue_w(const Product& pr, int tile, int step, uint32_t stage_smem, int warp, int lane) {
   using S = Shape<NT, DUAL>;
-  const int tile = u / pr.steps, step = u - tile * pr.steps;
   const int row0 = tile * S::TR + warp * 16;
   const int k = step * KSTEP + lane * 8;
-  const bool kin = k < pr.K;   // K is a multiple of 8
+  const bool inside = row0 + 16 <= pr.N && (step + 1) * KSTEP <= pr.K;   // the same for the whole warp
 #pragma unroll
   for (int ti = 0; ti < S::TILES; ++ti) {
-    const __nv_bfloat16* W = static_cast<const __nv_bfloat16*>(ti ? pr.W1 : pr.W0) + k;
-    const uint32_t dst = stage_smem + ti * TILE_BYTES + lane * 16;
+    const __nv_bfloat16* W = static_cast<const __nv_bfloat16*>(ti ? pr.W1 : pr.W0);
+    const __nv_bfloat16* src = W + static_cast<long long>(row0) * pr.ldw + k;
+    uint32_t dst = stage_smem + ti * TILE_BYTES + lane * 16;
+    if (inside) {
+#pragma unroll 8
+      for (int r = 0; r < 16; ++r, src += pr.ldw, dst += ROW_PITCH) cp_async16_full(dst, src);
+    } else {
+      const bool kin = k < pr.K;   // K is a multiple of 8
 #pragma unroll 4
-    for (int r = 0; r < 16; ++r) {
-      const int n = row0 + r;
-      const bool ok = kin && n < pr.N;
-      cp_async16(dst + r * ROW_PITCH, ok ? W + static_cast<long long>(n) * pr.ldw : W - k, ok);
+      for (int r = 0; r < 16; ++r, src += pr.ldw, dst += ROW_PITCH) {
+        const bool ok = kin && row0 + r < pr.N;
+        cp_async16(dst, ok ? src : W, ok);
+      }
     }
   }
 }
 // the warp's own copy of the token rows of the unit's k range; rows T .. 8 NT - 1 of a slab are never
 // written and only feed accumulator columns that nobody reads
 template <int NT, bool DUAL>
-__device__ __forceinline__ void issue_x(const Product& pr, int T, int u, uint32_t stage_smem, int lane) {
+__device__ __forceinline__ void issue_x(const Product& pr, int T, int step, uint32_t stage_smem, int lane) {
   using S = Shape<NT, DUAL>;
-  const int step = u % pr.steps;
   const int k = step * KSTEP + lane * 8;
   const bool ok = k < pr.K;
   const int slabs = (DUAL && pr.X1 != pr.X0) ? 2 : 1;
   for (int xi = 0; xi < slabs; ++xi) {
     const __nv_bfloat16* X = static_cast<const __nv_bfloat16*>(xi ? pr.X1 : pr.X0) + (ok ? k : 0);
-    const uint32_t dst = stage_smem + S::W_BYTES + xi * (S::TP * ROW_PITCH) + lane * 16;
-    for (int t = 0; t < T; ++t) cp_async16(dst + t * ROW_PITCH, ok ? X + static_cast<long long>(t) * pr.ldx : X, ok);
+    uint32_t dst = stage_smem + S::W_BYTES + xi * (S::TP * ROW_PITCH) + lane * 16;
+    for (int t = 0; t < T; ++t, dst += ROW_PITCH, X += (ok ? pr.ldx : 0)) cp_async16(dst, X, ok);
   }
 }
 
@@ -160,9 +164,8 @@ __device__ __forceinline__ void compute(float (&acc)[DUAL ? 2 : 1][NT][4], bool 
 
 // This warp's share of a shared slab: token rows warp, warp + 8, ... of each input; then every lane
 // tells the slot's `full` barrier to count it in once its copies have landed.
-__device__ __forceinline__ void issue_x_shared(const Product& pr, int T, int TP, int slabs, int u, uint32_t slab_smem,
+__device__ __forceinline__ void issue_x_shared(const Product& pr, int T, int TP, int slabs, int step, uint32_t slab_smem,
                                                uint64_t* full, int warp, int lane) {
-  const int step = u % pr.steps;
   const int k = step * KSTEP + lane * 8;
   const bool ok = k < pr.K;
   for (int xi = 0; xi < slabs; ++xi) {
@@ -259,6 +262,8 @@ __device__ __forceinline__ bool run_product(const Product& pr, const Params& p, 
   const int first_tile = u0 / pr.steps;
   int tile = first_tile, step = u0 - first_tile * pr.steps;
   int seg_lo = step;
+  int tile_a = tile, step_a = step;   // the next unit whose weights go out
+  int step_x = step;                  // the k step of the next shared slab
   // q < 0: the weights of the first units go out ahead of the wait; from q = 0 on the pipeline runs.
   // Copy groups of a worker, private token rows: W(0), W(1), X(0) | X(1) | then one per unit.
   // Shared slabs: one group per unit from the start (a warp's slab copies ride in its next group).
@@ -268,15 +273,17 @@ __device__ __forceinline__ bool run_product(const Product& pr, const Params& p, 
       else if (!grid_barrier(p.ctrl, s_flag)) return false;
       if (n == 0) break;
       if (S::PRIV) {
-        issue_x<NT, DUAL>(pr, p.T, u0, my_smem, lane);
+        issue_x<NT, DUAL>(pr, p.T, step, my_smem, lane);
         asm volatile("cp.async.commit_group;" ::: "memory");
         if (n > 1) {
-          issue_x<NT, DUAL>(pr, p.T, u0 + 1, my_smem + S::STAGE, lane);
+          issue_x<NT, DUAL>(pr, p.T, step + 1 == pr.steps ? 0 : step + 1, my_smem + S::STAGE, lane);
           asm volatile("cp.async.commit_group;" ::: "memory");
         }
       } else {
-        for (int j = 0; j < LOOK && j < n; ++j)
-          issue_x_shared(pr, p.T, TP, slabs, u0 + j, xring + j * slab_bytes, full + j, warp, lane);
+        for (int j = 0; j < LOOK && j < n; ++j) {
+          issue_x_shared(pr, p.T, TP, slabs, step_x, xring + j * slab_bytes, full + j, warp, lane);
+          if (++step_x == pr.steps) step_x = 0;
+        }
       }
     }
     const uint32_t stage_smem = my_smem + ((q + NST) % NST) * S::STAGE;
@@ -288,7 +295,8 @@ __device__ __forceinline__ bool run_product(const Product& pr, const Params& p, 
         if (j < n) {
           const int slot = j % R, use = j / R;
           if (use > 0 && !ptx::mbar_wait(empty + slot, (use - 1) & 1, s_abort)) return false;
-          issue_x_shared(pr, p.T, TP, slabs, u0 + j, xring + slot * slab_bytes, full + slot, warp, lane);
+          issue_x_shared(pr, p.T, TP, slabs, step_x, xring + slot * slab_bytes, full + slot, warp, lane);
+          if (++step_x == pr.steps) step_x = 0;
         }
         xsmem = xring + (q % R) * slab_bytes;
       }
@@ -303,8 +311,9 @@ __device__ __forceinline__ bool run_product(const Product& pr, const Params& p, 
       if (!S::PRIV && lane == 0) ptx::mbar_arrive(empty + q % R);
     }
     if (worker && q + NST < n) {
-      issue_w<NT, DUAL>(pr, u0 + q + NST, stage_smem, warp, lane);
-      if (S::PRIV && q >= 0) issue_x<NT, DUAL>(pr, p.T, u0 + q + NST, stage_smem, lane);
+      issue_w<NT, DUAL>(pr, tile_a, step_a, stage_smem, warp, lane);
+      if (S::PRIV && q >= 0) issue_x<NT, DUAL>(pr, p.T, step_a, stage_smem, lane);
+      if (++step_a == pr.steps) { step_a = 0; ++tile_a; }
       if (!S::PRIV || q >= 0) asm volatile("cp.async.commit_group;" ::: "memory");
     }
     if (q < 0) continue;

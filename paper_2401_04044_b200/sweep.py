@@ -79,7 +79,7 @@ def time_calls(fn, batch, reps, warmup, use_graph=True):
     return ts, mode
 
 
-def run_point(ctx, cfg, tokens, copies, reps, svd, device="cuda", use_graph=True):
+def run_point(ctx, cfg, tokens, copies, reps, svd, device="cuda", use_graph=True, which=("split", "dense")):
     hbm, tf, src = peaks()
     shape = make_shape(cfg.d, cfg.m, cfg.act, cfg.torch_dtype)
     es = 2 if cfg.dtype == "bf16" else 4
@@ -117,6 +117,8 @@ def run_point(ctx, cfg, tokens, copies, reps, svd, device="cuda", use_graph=True
                "tokens": T, "layers": cfg.layers, "weight_copies_cycled": copies, "peaks": src}
         for name, bl, params, lbytes in (("split", blobs, (n_in + 1) * (cfg.d * cfg.k + cfg.r * (cfg.d + cfg.m - cfg.k)), logical),
                                         ("dense", blobs_d, (n_in + 1) * cfg.d * cfg.m, logical_d)):
+            if name not in which:
+                continue
             state = {"i": 0}
 
             def call():
@@ -135,7 +137,8 @@ def run_point(ctx, cfg, tokens, copies, reps, svd, device="cuda", use_graph=True
                          "tokens_per_s_per_stack": T / (ms * 1e-3 * cfg.layers), "roofline_ms": roof_ms,
                          "roofline_frac": roof_ms / ms, "bound": "tensor" if flops / (tf * 1e12) > bytes_ / (hbm * 1e9) else "hbm",
                          "tflops": flops / (ms * 1e-3) / 1e12, "gbs": bytes_ / (ms * 1e-3) / 1e9, "model_bytes_per_layer": lbytes}
-        res["split_vs_dense_speedup"] = res["dense"]["ms_per_layer"] / res["split"]["ms_per_layer"]
+        if "split" in res and "dense" in res:
+            res["split_vs_dense_speedup"] = res["dense"]["ms_per_layer"] / res["split"]["ms_per_layer"]
         res["size_ratio"] = logical / logical_d
         out.append(res)
     return out
@@ -150,6 +153,8 @@ def main():
     ap.add_argument("--svd", action="store_true", help="true SVD factors instead of random ones")
     ap.add_argument("--sweep5", action="store_true", help="config 5: all heavy fractions x ranks")
     ap.add_argument("--out", default=None)
+    ap.add_argument("--which", nargs="*", default=["split", "dense"], choices=["split", "dense"],
+                    help="time the split layer, its dense counterpart, or both")
     ap.add_argument("--no-graph", action="store_true", help="issue the timed calls one by one instead of replaying a CUDA graph")
     args = ap.parse_args()
     build.build()
@@ -164,7 +169,7 @@ def main():
         es = 2 if cfg.dtype == "bf16" else 4
         split_bytes = es * (cfg.n_in + 1) * (cfg.d * cfg.k + cfg.r * (cfg.d + cfg.m - cfg.k))
         copies = args.copies or max(2, min(24, -(-2 * 126 * (1 << 20) // split_bytes)))
-        for res in run_point(ctx, cfg, tokens, copies, args.reps, args.svd, use_graph=not args.no_graph):
+        for res in run_point(ctx, cfg, tokens, copies, args.reps, args.svd, use_graph=not args.no_graph, which=tuple(args.which)):
             line = json.dumps(res)
             print(line, flush=True)
             lines.append(line)
