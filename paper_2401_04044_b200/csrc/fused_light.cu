@@ -153,6 +153,14 @@ fused_light_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
+  // Launched with programmatic stream serialisation: everything above (barriers, tensor maps, tensor
+  // memory) overlapped the tail of the kernel before; nothing below may start until that kernel is
+  // complete and its writes are visible.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  // Only now may the kernel after this one begin its set-up: it will block in its tensor-memory allocation
+  // until this CTA frees its columns, which is safe because this CTA already holds its own (a dependent
+  // that got the columns first would wait for this kernel, and this kernel for the columns).
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   if (warp == 0) {
     if (ptx::elect_one()) {
@@ -508,10 +516,20 @@ ffsplit_status launch_fused_light(ffsplit_ctx* ctx, const void* Q, long long ldq
   }
   dim3 grid(p.splits, static_cast<unsigned>(tiles_m));
   const int ph = prof_open(ctx, PROF_GEMM_TC, algo_flops, st);
-  fl::fused_light_kernel<<<grid, fl::NUM_THREADS, smem_bytes, st>>>(tQ, tB1, tA2, p);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(fl::NUM_THREADS);
+  cfg.dynamicSmemBytes = smem_bytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const cudaError_t le = cudaLaunchKernelEx(&cfg, fl::fused_light_kernel, tQ, tB1, tA2, p);
   prof_close(ctx, ph, st);
   ctx->launches++;
-  return check_cuda(ctx, cudaGetLastError(), "fused_light_kernel launch");
+  return check_cuda(ctx, le, "fused_light_kernel launch");
 }
 
 }  // namespace ffsp

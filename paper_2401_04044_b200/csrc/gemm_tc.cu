@@ -171,6 +171,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   __syncthreads();
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_holder;
+  // Launched with programmatic stream serialisation: everything above (barriers, tensor maps, tensor
+  // memory) overlapped the tail of the kernel before; nothing below may start until that kernel is
+  // complete and its writes are visible.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  // Only now may the kernel after this one begin its set-up: it will block in its tensor-memory allocation
+  // until this CTA frees its columns, which is safe because this CTA already holds its own (a dependent
+  // that got the columns first would wait for this kernel, and this kernel for the columns).
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   const int nkb = (p.K + BLOCK_K - 1) / BLOCK_K;
   const int total_kb = p.dual ? 2 * nkb : nkb;
@@ -409,10 +417,20 @@ ffsplit_status launch_gemm_tc(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_t 
   const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n;
   const int grid = static_cast<int>(tiles < ctx->num_sms ? tiles : ctx->num_sms);
   const int ph = prof_open(ctx, PROF_GEMM_TC, g.algo_flops, st);
-  tc::gemm_tc_kernel<<<grid, tc::NUM_THREADS, smem_bytes, st>>>(tA0, tB0, tA1, tB1, p);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(grid);
+  cfg.blockDim = dim3(tc::NUM_THREADS);
+  cfg.dynamicSmemBytes = smem_bytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  const cudaError_t le = cudaLaunchKernelEx(&cfg, tc::gemm_tc_kernel, tA0, tB0, tA1, tB1, p);
   prof_close(ctx, ph, st);
   ctx->launches++;
-  return check_cuda(ctx, cudaGetLastError(), "gemm_tc_kernel launch");
+  return check_cuda(ctx, le, "gemm_tc_kernel launch");
 }
 
 }  // namespace ffsp
