@@ -82,8 +82,15 @@ __device__ __forceinline__ void epilogue_chunk_store(const Params& p, const Gelu
     a.z = pack_bf16x2(v[4], v[5]);   a.w = pack_bf16x2(v[6], v[7]);
     b.x = pack_bf16x2(v[8], v[9]);   b.y = pack_bf16x2(v[10], v[11]);
     b.z = pack_bf16x2(v[12], v[13]); b.w = pack_bf16x2(v[14], v[15]);
-    reinterpret_cast<uint4*>(base)[0] = a;
-    reinterpret_cast<uint4*>(base)[1] = b;
+    if ((reinterpret_cast<uintptr_t>(base) & 31u) == 0) {
+      // one whole 32-byte sector per lane and instruction: half as many write requests as two 16-byte stores
+      asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(base), "r"(a.x), "r"(a.y), "r"(a.z),
+                   "r"(a.w), "r"(b.x), "r"(b.y), "r"(b.z), "r"(b.w)
+                   : "memory");
+    } else {
+      reinterpret_cast<uint4*>(base)[0] = a;
+      reinterpret_cast<uint4*>(base)[1] = b;
+    }
   } else {
 #pragma unroll
     for (int i = 0; i < 16; ++i)
@@ -269,21 +276,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       ptx::tc_fence_after();
       const long long row = static_cast<long long>(m_blk) * BLOCK_M + q * 32 + lane;
       const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * ACC_STRIDE;
-      for (int c = half * 16; c < p.block_n; c += 4 * EPI_WARPS) {
-        const int n0 = n_blk * p.block_n + c;
-        if (n0 >= p.N) break;
-        float v[16];
-        ptx::tmem_ld16(t_row + c, v);
-        if (p.dual) {
-          float u[16];
-          ptx::tmem_ld16(t_row + GATE_OFFSET + c, u);
-          ptx::tmem_ld_wait();
-#pragma unroll
-          for (int i = 0; i < 16; ++i)
-            v[i] = (p.epi.col_partial ? silu_precise_f(v[i]) : silu_fast(v[i])) * u[i];
-        } else {
-          ptx::tmem_ld_wait();
-        }
+      // one 16-column chunk: v holds the accumulators of this lane's row
+      auto finish_chunk = [&](float* v, int n0) {
         if (p.epi.col_partial == nullptr) {
           epilogue_chunk_store(p, gc, row, n0, v);
         } else {
@@ -300,6 +294,43 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           const int n = n0 + (lane >> 1);
           if ((lane & 1) == 0 && n < p.N)
             e.col_partial[(static_cast<long long>(m_blk) * 4 + q) * p.N + n] = tot;
+        }
+      };
+      const int nbase = n_blk * p.block_n;
+      constexpr int CSTEP = 4 * EPI_WARPS;
+      if (!p.dual) {
+        // Two register buffers: the tensor-memory load of the next chunk is in flight while this one goes
+        // through bias, activation and stores (a load's registers may be read only after the next wait).
+        float va[16], vb[16];
+        int c = half * 16;
+        bool more = c < p.block_n && nbase + c < p.N;
+        if (more) ptx::tmem_ld16(t_row + c, va);
+        while (more) {
+          ptx::tmem_ld_wait();
+          bool next = c + CSTEP < p.block_n && nbase + c + CSTEP < p.N;
+          if (next) ptx::tmem_ld16(t_row + c + CSTEP, vb);
+          finish_chunk(va, nbase + c);
+          if (!next) break;
+          c += CSTEP;
+          ptx::tmem_ld_wait();
+          next = c + CSTEP < p.block_n && nbase + c + CSTEP < p.N;
+          if (next) ptx::tmem_ld16(t_row + c + CSTEP, va);
+          finish_chunk(vb, nbase + c);
+          more = next;
+          c += CSTEP;
+        }
+      } else {
+        for (int c = half * 16; c < p.block_n; c += CSTEP) {
+          const int n0 = nbase + c;
+          if (n0 >= p.N) break;
+          float v[16], u[16];
+          ptx::tmem_ld16(t_row + c, v);
+          ptx::tmem_ld16(t_row + GATE_OFFSET + c, u);
+          ptx::tmem_ld_wait();
+#pragma unroll
+          for (int i = 0; i < 16; ++i)
+            v[i] = (p.epi.col_partial ? silu_precise_f(v[i]) : silu_fast(v[i])) * u[i];
+          finish_chunk(v, n0);
         }
       }
       ptx::tc_fence_before();
