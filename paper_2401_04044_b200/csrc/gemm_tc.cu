@@ -286,7 +286,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
 #pragma unroll
           for (int i = 0; i < 16; ++i) {
             float x = v[i];
-            if (!p.dual) x = act_gelu(x, e.act);   // scores decide indices: full-precision activation
+            if (!p.dual) x = act_gelu_score(x, e.act);   // scores decide indices: fp32-accurate activation, not the one-MUFU form
             x = e.score_abs ? fabsf(x) : x * x;
             v[i] = (row < p.M) ? x : 0.0f;
           }
