@@ -13,6 +13,8 @@
 
 #include "ffsplit.h"
 
+#include <utility>
+
 namespace ffsp {
 
 // ----------------------------------------------------------------------------
@@ -200,6 +202,32 @@ ffsplit_status decode_layer_add(ffsplit_ctx* ctx, DecodeLayerPlan* plan, const v
                                 double algo_bytes);
 ffsplit_status decode_layer_launch(ffsplit_ctx* ctx, const DecodeLayerPlan* plan, int T, float* partial, int* ctrl,
                                    cudaStream_t st);
+
+// Launch with programmatic stream serialisation: the kernel may be scheduled while the kernel before it in
+// the stream is still running.  Every kernel launched this way executes `griddepcontrol.wait` before its
+// first global-memory access (pdl_wait() below), so only its launch latency overlaps.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+#ifdef __CUDACC__
+// Wait for the kernel before this one (complete, writes visible), then let the one after start launching.
+__device__ __forceinline__ void pdl_wait() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+#endif
 
 // Profiling brackets: no-ops unless ffsplit_profile_begin() is active.
 enum ProfClass : int { PROF_GEMM_TC = 0, PROF_GEMM_SIMT = 1, PROF_DECODE = 2 };

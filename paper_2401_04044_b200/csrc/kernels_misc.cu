@@ -28,6 +28,7 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
   __shared__ unsigned wsum_gt[32], wsum_eq[32];
   const int tid = threadIdx.x;
   const int lane = tid & 31, warp = tid >> 5;
+  pdl_wait();
 
   if (tid == 0) {
     s_prefix = 0u;
@@ -138,9 +139,9 @@ __global__ void __launch_bounds__(kSelThreads) select_kernel(const float* __rest
 
 ffsplit_status launch_select(ffsplit_ctx* ctx, const float* scores, int m, int k, int* heavy, int* light,
                              cudaStream_t st) {
-  select_kernel<<<1, kSelThreads, 0, st>>>(scores, m, k, heavy, light, ctx->status());
+  const cudaError_t le = launch_pdl(select_kernel, dim3(1), dim3(kSelThreads), 0, st, scores, m, k, heavy, light, ctx->status());
   ctx->launches++;
-  return check_cuda(ctx, cudaGetLastError(), "select_kernel launch");
+  return check_cuda(ctx, le, "select_kernel launch");
 }
 
 // ============================================================================
@@ -152,6 +153,7 @@ __global__ void __launch_bounds__(256) score_finalize_kernel(const float* __rest
                                                              const float* __restrict__ w, float* __restrict__ energy,
                                                              float* __restrict__ scores, int mode, int accumulate) {
   __shared__ float part[8][32];
+  pdl_wait();
   const int cx = threadIdx.x & 31, gy = threadIdx.x >> 5;
   const int j = blockIdx.x * 32 + cx;
   float s = 0.f;
@@ -175,9 +177,9 @@ __global__ void __launch_bounds__(256) score_finalize_kernel(const float* __rest
 
 ffsplit_status launch_score_finalize(ffsplit_ctx* ctx, const float* partial, int groups, int m, const float* w,
                                      float* energy, float* scores, int mode, int accumulate, cudaStream_t st) {
-  score_finalize_kernel<<<(m + 31) / 32, 256, 0, st>>>(partial, groups, m, w, energy, scores, mode, accumulate);
+  const cudaError_t le = launch_pdl(score_finalize_kernel, dim3((m + 31) / 32), dim3(256), 0, st, partial, groups, m, w, energy, scores, mode, accumulate);
   ctx->launches++;
-  return check_cuda(ctx, cudaGetLastError(), "score_finalize_kernel launch");
+  return check_cuda(ctx, le, "score_finalize_kernel launch");
 }
 
 // ============================================================================
@@ -308,6 +310,7 @@ __device__ __forceinline__ void pack_bias_chunk(const PrepJob& q, int blk, int* 
 template <typename T>
 __global__ void __launch_bounds__(256) prep_kernel(const PrepBatch batch, int* status) {
   __shared__ T tile[32][33];
+  pdl_wait();
   int i = 0;
   while (i + 1 < batch.n && static_cast<int>(blockIdx.x) >= batch.job[i + 1].block_begin) ++i;
   const PrepJob& q = batch.job[i];
@@ -335,11 +338,12 @@ ffsplit_status prep_flush(ffsplit_ctx* ctx, int dtype, cudaStream_t st) {
   ctx->prep_active = false;
   if (ctx->prep.n == 0) return FFSPLIT_OK;
   const int blocks = ctx->prep_blocks;
-  if (dtype == FFSPLIT_BF16) prep_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(ctx->prep, ctx->status());
-  else prep_kernel<float><<<blocks, 256, 0, st>>>(ctx->prep, ctx->status());
+  const cudaError_t le = dtype == FFSPLIT_BF16
+                             ? launch_pdl(prep_kernel<__nv_bfloat16>, dim3(blocks), dim3(256), 0, st, ctx->prep, ctx->status())
+                             : launch_pdl(prep_kernel<float>, dim3(blocks), dim3(256), 0, st, ctx->prep, ctx->status());
   ctx->prep.n = 0;
   ctx->launches++;
-  return check_cuda(ctx, cudaGetLastError(), "prep_kernel launch");
+  return check_cuda(ctx, le, "prep_kernel launch");
 }
 
 // Records a job; outside a prep_begin/prep_flush bracket the job is launched on its own.
