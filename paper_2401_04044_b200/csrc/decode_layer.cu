@@ -412,7 +412,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_layer_kernel(const __grid_c
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // a dependent launch may start its own first copies
   for (int pi = 0; pi < p.nprod; ++pi) {
     const Product& pr = p.prod[pi];
-    if (NT > 1) {
+    if (!Shape<NT, false>::PRIV) {
       // slab barriers start every product in phase 0: `full` counts every thread, `empty` every warp
       if (threadIdx.x == 0) {
         for (int i = 0; i < kMaxSlots; ++i) { ptx::mbar_init(s_full + i, THREADS); ptx::mbar_init(s_empty + i, WARPS); }
