@@ -8,16 +8,16 @@
 //  * One CTA per SM stays resident for the whole layer.  A product is cut into units of
 //    128 weight rows x 256 k (64 KB of W); the units, in row-tile-major order, are dealt to the CTAs in
 //    equal contiguous shares (a tile's K range may straddle two or more CTAs).
-//  * The warps of a CTA walk its share side by side -- each owns 16 NT rows of every tile, NT = token
-//    tiles of 8 -- but never wait for one another: each has its own two-stage cp.async ring, so a late
-//    DRAM reply holds up one warp, not the SM, and the ring does not drain at tile boundaries.
-//  * Each warp-wide copy moves 512 contiguous bytes of one weight row.  The token rows of the same k
-//    range travel in the same copy group into the warp's own stage (they come from L2 and add half
-//    the weight bytes at most); loading them at the point of use instead costs a quarter of the
-//    bandwidth, and sharing one copy per CTA ties the warps together.  Fragments for the warp-level
-//    MMA (m16n8k16, weights as the 16-row operand, tokens as the 8-wide one) are read from shared
-//    memory with 128-bit loads; since a contraction does not care in which order k is visited, a
-//    thread's 16 bytes feed two MMAs as they are, and the token operand is read with the same pattern.
+//  * The warps of a CTA walk its share side by side -- each owns 16 rows of every tile -- and never wait
+//    for one another's weights: each has its own two-stage cp.async ring, so a late DRAM reply holds up
+//    one warp, not the SM, and the ring does not drain at tile boundaries.
+//  * Each warp-wide copy moves 512 contiguous bytes of one weight row.  The token rows of a unit's k
+//    range are staged once per CTA, a few units ahead, in a ring of slabs guarded by mbarriers (loading
+//    them at the point of use costs a quarter of the bandwidth: they queue behind the weight stream).
+//    Fragments for the warp-level MMA (m16n8k16, weights as the 16-row operand, tokens as the 8-wide
+//    one) are read from shared memory with 128-bit loads; since a contraction does not care in which
+//    order k is visited, a thread's 16 bytes feed two MMAs as they are, and the token operand is read
+//    with the same pattern.
 //  * Rows finished inside one CTA go through the epilogue straight from the accumulator registers.
 //    Rows shared by several CTAs: each warp writes an fp32 partial (at most two per CTA and product:
 //    the tile its share starts in and the tile it ends in), takes an atomic ticket, and the last to
@@ -62,26 +62,23 @@ struct Params {
 };
 
 // A CTA tile is 128 weight rows (64 rows of each matrix for a gated pair); warp w owns 16 of them and
-// has a two-stage ring for them.  The token rows of a unit's k range (a slab) are staged too:
-//  * up to 8 tokens (NT = 1 token tile) every warp copies them for itself, in the same copy group as its
-//    weights: no warp ever waits for another;
-//  * with more tokens private copies neither fit nor pay (they would outweigh the weights), so the CTA
-//    keeps one ring of slabs.  All warps load a share of each slab, a few units ahead, and meet only
-//    through two mbarriers per slot: `full` (the slab has landed: every thread's copies, tracked by
-//    cp.async.mbarrier.arrive) and `empty` (every warp is done reading it).
+// has a two-stage ring for them.  The token rows of a unit's k range (a slab) are staged once per CTA, in
+// a ring of slabs beside the weight rings: all warps load a share of each slab, a few units ahead of its
+// use, and meet only through two mbarriers per slot -- `full` (the slab has landed: every thread's copies,
+// tracked by cp.async.mbarrier.arrive) and `empty` (every warp is done reading it).  No warp waits for
+// another's weights.  (Measured alternatives, OPT-13B dense layer, 1 / 8 tokens: every warp copying the
+// token rows for itself 87 / 103 us; this ring 88 / 87 us.)
 template <int NT, bool DUAL>
 struct Shape {
-  static constexpr bool PRIV = NT == 1;              // token rows staged per warp
-  static constexpr int NST = 2;                      // stages of a warp's ring
+  static constexpr int NST = 2;                      // stages of a warp's weight ring
   static constexpr int TILES = DUAL ? 2 : 1;
   static constexpr int AW = DUAL ? 4 : 8;            // working warps
   static constexpr int TR = AW * 16;                 // rows of a CTA tile
   static constexpr int TP = 8 * NT;                  // token rows, padded
   static constexpr int W_BYTES = TILES * TILE_BYTES;
-  static constexpr int X_BYTES = PRIV ? TILES * TP * ROW_PITCH : 0;   // a gated pair may have two inputs
-  static constexpr int STAGE = W_BYTES + X_BYTES;
-  static_assert(AW * NST * STAGE == (PRIV ? SMEM_BYTES : RING_BYTES), "shared memory plan");
-  static_assert(PRIV || TILES * TP * ROW_PITCH <= XCAP_BYTES, "one slab must fit");
+  static constexpr int STAGE = W_BYTES;
+  static_assert(AW * NST * STAGE == RING_BYTES, "shared memory plan");
+  static_assert(TILES * TP * ROW_PITCH <= XCAP_BYTES, "one slab must fit");
 };
 
 // Shares of the `ge` CTAs that have one: CTA c owns units [c U / ge, (c + 1) U / ge).  U * (ge + 1) fits
@@ -117,21 +114,6 @@ __device__ __forceinline__ void issue_w(const Product& pr, int tile, int step, u
     }
   }
 }
-// the warp's own copy of the token rows of the unit's k range; rows T .. 8 NT - 1 of a slab are never
-// written and only feed accumulator columns that nobody reads
-template <int NT, bool DUAL>
-__device__ __forceinline__ void issue_x(const Product& pr, int T, int step, uint32_t stage_smem, int lane) {
-  using S = Shape<NT, DUAL>;
-  const int k = step * KSTEP + lane * 8;
-  const bool ok = k < pr.K;
-  const int slabs = (DUAL && pr.X1 != pr.X0) ? 2 : 1;
-  for (int xi = 0; xi < slabs; ++xi) {
-    const __nv_bfloat16* X = static_cast<const __nv_bfloat16*>(xi ? pr.X1 : pr.X0) + (ok ? k : 0);
-    uint32_t dst = stage_smem + S::W_BYTES + xi * (S::TP * ROW_PITCH) + lane * 16;
-    for (int t = 0; t < T; ++t, dst += ROW_PITCH, X += (ok ? pr.ldx : 0)) cp_async16(dst, X, ok);
-  }
-}
-
 // One unit: the warp's 16 rows x 256 k against the token rows at xsmem (a second input, if there
 // is one, follows 8 NT rows later).
 template <int NT, bool DUAL>
@@ -164,7 +146,7 @@ __device__ __forceinline__ void compute(float (&acc)[DUAL ? 2 : 1][NT][4], bool 
 
 // This warp's share of a shared slab: token rows warp, warp + 8, ... of each input; then every lane
 // tells the slot's `full` barrier to count it in once its copies have landed.
-__device__ __forceinline__ void issue_x_shared(const Product& pr, int T, int TP, int slabs, int step, uint32_t slab_smem,
+__device__ __forceinline__ void issue_slab(const Product& pr, int T, int TP, int slabs, int step, uint32_t slab_smem,
                                                uint64_t* full, int warp, int lane) {
   const int k = step * KSTEP + lane * 8;
   const bool ok = k < pr.K;
@@ -240,7 +222,7 @@ __device__ __forceinline__ bool run_product(const Product& pr, const Params& p, 
   const bool has = cta < static_cast<int>(ge);
   const bool worker = warp < S::AW;            // the other warps only help with shared slabs
   const int u0 = has ? share_lo(cta, U, ge) : 0, u1 = has ? share_lo(cta + 1, U, ge) : 0;
-  const int n = (S::PRIV && !worker) ? 0 : u1 - u0;
+  const int n = u1 - u0;
   const bool two = DUAL && pr.X1 != pr.X0;
   const GeluCoef gc = gelu_coef(pr.epi.act);
   const uint32_t my_smem = smem0 + warp * (NST * S::STAGE);
@@ -265,56 +247,42 @@ __device__ __forceinline__ bool run_product(const Product& pr, const Params& p, 
   int tile_a = tile, step_a = step;   // the next unit whose weights go out
   int step_x = step;                  // the k step of the next shared slab
   // q < 0: the weights of the first units go out ahead of the wait; from q = 0 on the pipeline runs.
-  // Copy groups of a worker, private token rows: W(0), W(1), X(0) | X(1) | then one per unit.
-  // Shared slabs: one group per unit from the start (a warp's slab copies ride in its next group).
+  // A worker commits one copy group per unit (its slab copies ride in whichever group comes next).
   for (int q = -NST; q < n || q <= 0; ++q) {
     if (q == 0) {
       if (first) asm volatile("griddepcontrol.wait;" ::: "memory");
       else if (!grid_barrier(p.ctrl, s_flag)) return false;
       if (n == 0) break;
-      if (S::PRIV) {
-        issue_x<NT, DUAL>(pr, p.T, step, my_smem, lane);
-        asm volatile("cp.async.commit_group;" ::: "memory");
-        if (n > 1) {
-          issue_x<NT, DUAL>(pr, p.T, step + 1 == pr.steps ? 0 : step + 1, my_smem + S::STAGE, lane);
-          asm volatile("cp.async.commit_group;" ::: "memory");
-        }
-      } else {
-        for (int j = 0; j < LOOK && j < n; ++j) {
-          issue_x_shared(pr, p.T, TP, slabs, step_x, xring + j * slab_bytes, full + j, warp, lane);
-          if (++step_x == pr.steps) step_x = 0;
-        }
+      for (int j = 0; j < LOOK && j < n; ++j) {
+        issue_slab(pr, p.T, TP, slabs, step_x, xring + j * slab_bytes, full + j, warp, lane);
+        if (++step_x == pr.steps) step_x = 0;
       }
     }
     const uint32_t stage_smem = my_smem + ((q + NST) % NST) * S::STAGE;
     if (q >= 0) {
-      uint32_t xsmem = stage_smem + S::W_BYTES;
-      if (!S::PRIV) {
-        // the slab LOOK units ahead goes into the slot that unit q - 1 used: wait until every warp has read it
-        const int j = q + LOOK;
-        if (j < n) {
-          const int slot = j % R, use = j / R;
-          if (use > 0 && !ptx::mbar_wait(empty + slot, (use - 1) & 1, s_abort)) return false;
-          issue_x_shared(pr, p.T, TP, slabs, step_x, xring + slot * slab_bytes, full + slot, warp, lane);
-          if (++step_x == pr.steps) step_x = 0;
-        }
-        xsmem = xring + (q % R) * slab_bytes;
+      // the slab LOOK units ahead goes into the slot that unit q - 1 used: wait until every warp has read it
+      const int j = q + LOOK;
+      if (j < n) {
+        const int slot = j % R, use = j / R;
+        if (use > 0 && !ptx::mbar_wait(empty + slot, (use - 1) & 1, s_abort)) return false;
+        issue_slab(pr, p.T, TP, slabs, step_x, xring + slot * slab_bytes, full + slot, warp, lane);
+        if (++step_x == pr.steps) step_x = 0;
       }
+      const uint32_t xsmem = xring + (q % R) * slab_bytes;
       if (worker) {
         if (n - 1 - q >= 1) asm volatile("cp.async.wait_group 1;" ::: "memory");
         else asm volatile("cp.async.wait_group 0;" ::: "memory");
       }
-      if (!S::PRIV && !ptx::mbar_wait(full + q % R, (q / R) & 1, s_abort)) return false;
+      if (!ptx::mbar_wait(full + q % R, (q / R) & 1, s_abort)) return false;
       __syncwarp();
       if (worker) compute<NT, DUAL>(acc, two, stage_smem, xsmem, lane);
       __syncwarp();
-      if (!S::PRIV && lane == 0) ptx::mbar_arrive(empty + q % R);
+      if (lane == 0) ptx::mbar_arrive(empty + q % R);
     }
     if (worker && q + NST < n) {
       issue_w<NT, DUAL>(pr, tile_a, step_a, stage_smem, warp, lane);
-      if (S::PRIV && q >= 0) issue_x<NT, DUAL>(pr, p.T, step_a, stage_smem, lane);
       if (++step_a == pr.steps) { step_a = 0; ++tile_a; }
-      if (!S::PRIV || q >= 0) asm volatile("cp.async.commit_group;" ::: "memory");
+      asm volatile("cp.async.commit_group;" ::: "memory");
     }
     if (q < 0) continue;
     if (!worker) {
@@ -412,7 +380,7 @@ __global__ void __launch_bounds__(THREADS, 1) decode_layer_kernel(const __grid_c
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // a dependent launch may start its own first copies
   for (int pi = 0; pi < p.nprod; ++pi) {
     const Product& pr = p.prod[pi];
-    if (!Shape<NT, false>::PRIV) {
+    {
       // slab barriers start every product in phase 0: `full` counts every thread, `empty` every warp
       if (threadIdx.x == 0) {
         for (int i = 0; i < kMaxSlots; ++i) { ptx::mbar_init(s_full + i, THREADS); ptx::mbar_init(s_empty + i, WARPS); }
