@@ -160,6 +160,31 @@ class StackWorkload:
             assert torch.equal(e["heavy"], e["heavy_setup"]), "selection changed between set-up and the timed steps"
 
 
+# DRAM traffic of the tensor-core kernels (gemm_tc_kernel and fused_light_kernel: the launches the roofline
+# object covers), average per launch over one step, from an ncu capture of
+#   python bench.py --only step --steps 1 --warmup 1 --no-graph --no-cpu-baseline
+# (dram__bytes_read.sum + dram__bytes_write.sum, last 48 launches; profiles/gemm_tc_and_fused_light__cfg2_traffic.md).
+# Valid only for the kernel sources it was taken with: any change to them turns the field back to null.
+TC_TRAFFIC_BYTES_PER_LAUNCH = 6350752
+TC_TRAFFIC_SOURCES_SHA256 = "09c6ec0f62197e4928950c96eab968ffda12c9b30464a22905be4d81ce475ca6"
+TC_SOURCES = ("gemm_tc.cu", "fused_light.cu", "ptx.cuh", "epilogue.cuh", "internal.h")
+
+
+def tc_sources_sha256():
+    import hashlib
+    h = hashlib.sha256()
+    for name in TC_SOURCES:
+        with open(os.path.join(ROOT, "paper_2401_04044_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def measured_traffic():
+    if TC_TRAFFIC_BYTES_PER_LAUNCH is None or tc_sources_sha256() != TC_TRAFFIC_SOURCES_SHA256:
+        return None
+    return TC_TRAFFIC_BYTES_PER_LAUNCH
+
+
 def time_region(fn, steps, warmup, flush, dist_barrier):
     """W untimed + K timed calls of fn, each timed with CUDA events on the current
     stream, L2 flushed (untimed) before every call.  Returns per-step milliseconds."""
@@ -294,7 +319,7 @@ def run_ours(args):
                 "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": round(achieved / peaks["bf16_tflops"], 4),
                 "peak_source": f"{peaks['source']} (burst bf16; kernels of 5-40 us timed one by one)",
                 "launches_per_step": n_l // 3, "avg_launch_us": round(1e3 * ms_l / max(n_l, 1), 2),
-                "traffic": None}
+                "traffic": measured_traffic()}
     ctx.profile_begin()
     for _ in range(3):
         flush()

@@ -16,6 +16,7 @@ import argparse
 import json
 import os
 import statistics
+import time
 import sys
 
 import torch
@@ -46,7 +47,7 @@ def random_factors(cfg, device, gen):
     return f
 
 
-def time_calls(fn, batch, reps, warmup, use_graph=True):
+def time_calls(fn, batch, reps, warmup, use_graph=True, settle=0.0):
     """Milliseconds per call of `fn`, one sample per timed batch of `batch` consecutive calls.
 
     A single few-token forward lasts tens of microseconds, less than the host needs to issue it, so
@@ -68,6 +69,11 @@ def time_calls(fn, batch, reps, warmup, use_graph=True):
             mode = f"stream (graph capture failed: {type(exc).__name__})"
     run()
     torch.cuda.synchronize()
+    if settle > 0:
+        # a long tensor-bound case leaves the SM clock power-capped for a while: let it recover, then warm up
+        time.sleep(settle)
+        run()
+        torch.cuda.synchronize()
     ts = []
     for _ in range(reps):
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -79,7 +85,7 @@ def time_calls(fn, batch, reps, warmup, use_graph=True):
     return ts, mode
 
 
-def run_point(ctx, cfg, tokens, copies, reps, svd, device="cuda", use_graph=True, which=("split", "dense")):
+def run_point(ctx, cfg, tokens, copies, reps, svd, device="cuda", use_graph=True, which=("split", "dense"), settle=0.0):
     hbm, tf, src, tf_sus = peaks()
     shape = make_shape(cfg.d, cfg.m, cfg.act, cfg.torch_dtype)
     es = 2 if cfg.dtype == "bf16" else 4
@@ -126,7 +132,7 @@ def run_point(ctx, cfg, tokens, copies, reps, svd, device="cuda", use_graph=True
                 state["i"] += 1
 
             # every batch walks all weight copies (more than L2 holds) the same number of times
-            ts, mode = time_calls(call, copies * max(1, 16 // copies), reps, max(3, copies), use_graph)
+            ts, mode = time_calls(call, copies * max(1, 16 // copies), reps, max(3, copies), use_graph, settle)
             ctx.poll()
             res["launch_mode"] = mode
             ms = statistics.median(ts)
@@ -157,6 +163,8 @@ def main():
     ap.add_argument("--out", default=None)
     ap.add_argument("--which", nargs="*", default=["split", "dense"], choices=["split", "dense"],
                     help="time the split layer, its dense counterpart, or both")
+    ap.add_argument("--settle", type=float, default=1.0,
+                    help="seconds of idle time before each timed case (the clocks recover from the case before)")
     ap.add_argument("--no-graph", action="store_true", help="issue the timed calls one by one instead of replaying a CUDA graph")
     args = ap.parse_args()
     build.build()
@@ -171,7 +179,7 @@ def main():
         es = 2 if cfg.dtype == "bf16" else 4
         split_bytes = es * (cfg.n_in + 1) * (cfg.d * cfg.k + cfg.r * (cfg.d + cfg.m - cfg.k))
         copies = args.copies or max(2, min(24, -(-2 * 126 * (1 << 20) // split_bytes)))
-        for res in run_point(ctx, cfg, tokens, copies, args.reps, args.svd, use_graph=not args.no_graph, which=tuple(args.which)):
+        for res in run_point(ctx, cfg, tokens, copies, args.reps, args.svd, use_graph=not args.no_graph, which=tuple(args.which), settle=args.settle):
             line = json.dumps(res)
             print(line, flush=True)
             lines.append(line)
