@@ -277,6 +277,36 @@ def test_decode_forward_matches_oracle(ctx, act, d, m, k, r, T):
         assert_close(G.forward(blobd, X), dense_ref, "bf16", "decode dense forward")
 
 
+@pytest.mark.parametrize("act,d,m,k,r", [("gelu_erf", 1024, 4096, 205, 256), ("swiglu", 512, 1400, 70, 128)])
+@pytest.mark.parametrize("T", [1, 8, 24, 64])
+def test_decode_single_launch_mode(ctx, monkeypatch, act, d, m, k, r, T):
+    """The few-token forward as one cooperative launch per layer (products separated by a grid-wide
+    barrier, FFSPLIT_DECODE_LAYER=1) gives the same bits as the default one-launch-per-product mode:
+    the work split and the order of every sum are the same."""
+    from paper_2401_04044_b200 import Context
+    cfg = custom_config(d, m, k, r, act=act, dtype="bf16")
+    L = make_layer(cfg, 9)
+    G = GpuLayer(ctx, L)
+    G.reserve(T, 0, k, r)
+    fac = oracle_factors(L, L.planted.numpy(), r)
+    blob, _ = G.pack(L.planted, fac)
+    X = L.tokens(T)
+    Y = G.forward(blob, X)
+    monkeypatch.setenv("FFSPLIT_DECODE_LAYER", "1")
+    ctx2 = Context(0)
+    try:
+        ctx2.ensure_workspace(ctx2.workspace_size(G.shape, T, 0, k, r))
+        Xd = X.cuda()
+        Y2 = torch.empty_like(Xd)
+        for _ in range(2):   # the barrier and ticket words must be back in their rest state after a call
+            ctx2.forward(blob, Xd, Y2)
+            ctx2.poll()
+    finally:
+        ctx2.close()
+    assert_close(Y2, oracle_split(L, L.planted.numpy(), fac, X), "bf16", "single-launch decode forward")
+    assert torch.equal(Y2.cpu(), Y.cpu()), "single-launch mode differs from the per-product mode"
+
+
 @pytest.mark.parametrize("dt,act", [("f32", "gelu_erf"), ("bf16", "gelu_erf"), ("bf16", "swiglu"), ("f32", "swiglu")])
 def test_degenerate_splits(ctx, dt, act):
     """k = m is the dense FFN; k = 0 is plain low-rank; r = 0 keeps FFN_1 only;
