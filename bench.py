@@ -94,7 +94,7 @@ class ClockSampler:
 class StackWorkload:
     """Device-resident synthetic stack plus everything one step touches."""
 
-    def __init__(self, cfg, ctx, layers, T, device):
+    def __init__(self, cfg, ctx, layers, T, device, cal_lanes=1):
         import torch
         from ffsplit_synth import make_layer
         from paper_2401_04044_b200 import make_shape
@@ -104,6 +104,15 @@ class StackWorkload:
         ws = max(ctx.workspace_size(self.shape, T, cfg.t_cal, cfg.k, cfg.r),
                  ctx.workspace_size(self.shape, T, 0, cfg.m, 0))
         ctx.ensure_workspace(ws)
+        # The calibrations of different layers do not depend on one another, and most of their kernels
+        # (top-k in one CTA, the small preparation jobs) leave the GPU nearly idle: they are issued round
+        # robin on `cal_lanes` streams, each with a library context (workspace, tickets) of its own.
+        from paper_2401_04044_b200 import Context
+        self.lanes = [(ctx, None)]   # lane 0: the calling stream (forward chain; everything when alone)
+        for _ in range(cal_lanes if cal_lanes > 1 else 0):
+            c = Context(ctx.device if hasattr(ctx, "device") else 0)
+            c.ensure_workspace(c.workspace_size(self.shape, T, cfg.t_cal, cfg.k, cfg.r))
+            self.lanes.append((c, torch.cuda.Stream(device=device)))
         self.layers = []
         padded, self.logical_bytes = ctx.pack_size(self.shape, cfg.k, cfg.r)
         padded_dense, self.logical_bytes_dense = ctx.pack_size(self.shape, cfg.m, 0)
@@ -132,16 +141,47 @@ class StackWorkload:
             ctx.pack(self.shape, L.W1, L.b1, L.W2, L.b2, all_idx, cfg.m, None, e["blob_dense"], W1u=L.W1u)
         ctx.poll()
 
-    def calibrate_layer(self, e, pack=True):
-        L, cfg, ctx = e["L"], self.cfg, self.ctx
+    def calibrate_layer(self, e, pack=True, ctx=None):
+        L, cfg, ctx = e["L"], self.cfg, ctx or self.ctx
         ctx.score(self.shape, L.W1, L.b1, L.W2, e["Xcal"], e["energy"], e["scores"], W1u=L.W1u)
         ctx.select(e["scores"], cfg.k, e["heavy"], e["light"])
         if pack:
             ctx.pack(self.shape, L.W1, L.b1, L.W2, L.b2, e["heavy"], cfg.k, e["factors"], e["blob"], W1u=L.W1u)
 
-    def calibrate(self):
-        for e in self.layers:
-            self.calibrate_layer(e)
+    def calibrate(self, events=None):
+        """Score, select and pack every layer.  With several lanes the layers go round robin over the
+        lanes' streams; `events`, if given, receives one event per layer, recorded behind its pack."""
+        import torch
+        if len(self.lanes) == 1:
+            for e in self.layers:
+                self.calibrate_layer(e)
+            return
+        main = torch.cuda.current_stream()
+        fork = torch.cuda.Event()
+        fork.record(main)
+        side = self.lanes[1:]
+        for _, s in side:
+            s.wait_event(fork)
+        for i, e in enumerate(self.layers):
+            c, s = side[i % len(side)]
+            with torch.cuda.stream(s):
+                self.calibrate_layer(e, ctx=c)
+                if events is not None:
+                    ev = torch.cuda.Event()
+                    ev.record(s)
+                    events.append(ev)
+        if events is None:
+            for _, s in side:
+                join = torch.cuda.Event()
+                join.record(s)
+                main.wait_event(join)
+
+    def launch_count(self):
+        return sum(c.launch_count() for c, _ in self.lanes)
+
+    def poll(self):
+        for c, _ in self.lanes:
+            c.poll()
 
     def forward(self, x=None, dense=False):
         x = self.X if x is None else x
@@ -151,7 +191,26 @@ class StackWorkload:
         return x
 
     def step(self):
-        self.calibrate()
+        """One pass of the whole path.  With several lanes, layer l's forward (on the calling stream) waits
+        only for layer l's pack, so the forward chain runs under the calibrations of the later layers."""
+        import torch
+        if len(self.lanes) == 1:
+            self.calibrate()
+            return self.forward()
+        events = []
+        self.calibrate(events)
+        main = torch.cuda.current_stream()
+        x = self.X
+        for e, ev in zip(self.layers, events):
+            main.wait_event(ev)
+            self.ctx.forward(e["blob"], x, e["Y"])
+            x = e["Y"]
+        return x
+
+    def step_serial(self):
+        """The same work on one stream and one context: what the per-kernel profile is taken on."""
+        for e in self.layers:
+            self.calibrate_layer(e)
         return self.forward()
 
     def check_selection_stable(self):
@@ -260,7 +319,7 @@ def run_ours(args):
     T = cfg.t_fwd[0]
     ctx = Context(local_rank)
     n_layers = args.layers or cfg.layers
-    wl = StackWorkload(cfg, ctx, n_layers, T, device)
+    wl = StackWorkload(cfg, ctx, n_layers, T, device, cal_lanes=1 if args.only else args.cal_lanes)
     flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=device)
 
     def flush():
@@ -281,11 +340,11 @@ def run_ours(args):
     # The step is launch-bound on the host (about a hundred launches of 5-50 us): capture it once in a
     # CUDA graph and time replays.  --no-graph times the plain stream launches instead.
     wl.step()
-    ctx.poll()
-    n0 = ctx.launch_count()
+    wl.poll()
+    n0 = wl.launch_count()
     wl.step()
-    launches_per_step = ctx.launch_count() - n0
-    ctx.poll()
+    launches_per_step = wl.launch_count() - n0
+    wl.poll()
     step_fn, launch_mode = wl.step, "stream"
     if not args.no_graph:
         try:
@@ -297,7 +356,7 @@ def run_ours(args):
             launch_mode = f"stream (graph capture failed: {type(exc).__name__})"
             torch.cuda.synchronize()
     step_ms = time_region(step_fn, args.steps, args.warmup, flush, barrier)
-    ctx.poll()
+    wl.poll()
     wl.check_selection_stable()
     total_ms = max_over_ranks(sum(step_ms), world, device)
     value = world * T * args.steps / (total_ms * 1e-3)
@@ -312,7 +371,7 @@ def run_ours(args):
     ctx.profile_begin()
     for _ in range(3):
         flush()
-        wl.step()
+        wl.step_serial()
     n_l, ms_l, flops_l = ctx.profile_end(0)
     achieved = flops_l / (ms_l * 1e-3) / 1e12 if ms_l > 0 else 0.0
     roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel", "achieved": round(achieved, 2),
@@ -367,7 +426,7 @@ def run_ours(args):
                                    "4096 calibration tokens/layer, prefill 32x128=4096 tokens; step = score+select+pack "
                                    "per layer, then the 12-layer split forward",
                        "l2": "256 MiB buffer rewritten before every timed step (L2 flush)",
-                       "launch": launch_mode,
+                       "launch": launch_mode, "calibration_streams": max(1, len(wl.lanes) - 1),
                        "tokens_per_step": T, "layers": cfg.layers},
             "roofline": roofline,
             "e2e": e2e,
@@ -497,6 +556,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of a CUDA-graph replay")
+    ap.add_argument("--cal-lanes", type=int, default=3,
+                    help="streams (each with its own library context) the per-layer calibrations are spread over")
     ap.add_argument("--only", default=None, choices=["step", "forward", "dense", "calibrate"],
                     help="run one phase alone and print its times (for profiler captures)")
     ap.add_argument("--layers", type=int, default=0, help="with --only: number of layers of the stack to build")
