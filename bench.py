@@ -148,12 +148,15 @@ class StackWorkload:
         if pack:
             ctx.pack(self.shape, L.W1, L.b1, L.W2, L.b2, e["heavy"], cfg.k, e["factors"], e["blob"], W1u=L.W1u)
 
-    def calibrate(self, events=None):
+    def calibrate(self, events=None, before=None):
         """Score, select and pack every layer.  With several lanes the layers go round robin over the
-        lanes' streams; `events`, if given, receives one event per layer, recorded behind its pack."""
+        lanes' streams; `events`, if given, receives one event per layer, recorded behind its pack;
+        `before(i)`, if given, is issued on the layer's stream ahead of its calibration (input copies)."""
         import torch
         if len(self.lanes) == 1:
-            for e in self.layers:
+            for i, e in enumerate(self.layers):
+                if before is not None:
+                    before(i)
                 self.calibrate_layer(e)
             return
         main = torch.cuda.current_stream()
@@ -165,6 +168,8 @@ class StackWorkload:
         for i, e in enumerate(self.layers):
             c, s = side[i % len(side)]
             with torch.cuda.stream(s):
+                if before is not None:
+                    before(i)
                 self.calibrate_layer(e, ctx=c)
                 if events is not None:
                     ev = torch.cuda.Event()
@@ -190,17 +195,17 @@ class StackWorkload:
             x = e["Y"]
         return x
 
-    def step(self):
+    def step(self, x=None, before=None):
         """One pass of the whole path.  With several lanes, layer l's forward (on the calling stream) waits
         only for layer l's pack, so the forward chain runs under the calibrations of the later layers."""
         import torch
         if len(self.lanes) == 1:
-            self.calibrate()
-            return self.forward()
+            self.calibrate(before=before)
+            return self.forward(x)
         events = []
-        self.calibrate(events)
+        self.calibrate(events, before)
         main = torch.cuda.current_stream()
-        x = self.X
+        x = self.X if x is None else x
         for e, ev in zip(self.layers, events):
             main.wait_event(ev)
             self.ctx.forward(e["blob"], x, e["Y"])
@@ -393,14 +398,26 @@ def run_ours(args):
     x_dev = torch.empty_like(wl.X)
 
     def e2e_step():
-        for e, xh in zip(wl.layers, Xcal_host):
-            e["Xcal"].copy_(xh, non_blocking=True)
-            wl.calibrate_layer(e)
+        # every layer's calibration tokens are copied on the stream that calibrates that layer, so the
+        # copy engine works under the kernels of the other streams
         x_dev.copy_(X_host, non_blocking=True)
-        y = wl.forward(x_dev)
+        y = wl.step(x_dev, before=lambda i: wl.layers[i]["Xcal"].copy_(Xcal_host[i], non_blocking=True))
         Y_host.copy_(y, non_blocking=True)
 
-    e2e_ms = time_region(e2e_step, k_ph, w_ph, flush, barrier)
+    e2e_fn = e2e_step
+    if not args.no_graph:
+        # the copies are graph nodes like the kernels (pinned host buffers at fixed addresses)
+        try:
+            e2e_step()
+            torch.cuda.synchronize()
+            e2e_graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(e2e_graph):
+                e2e_step()
+            e2e_fn = e2e_graph.replay
+        except Exception:
+            torch.cuda.synchronize()
+            e2e_fn = e2e_step
+    e2e_ms = time_region(e2e_fn, k_ph, w_ph, flush, barrier)
     e2e_total = max_over_ranks(sum(e2e_ms), world, device)
     es = 2
     h2d = cfg.layers * cfg.t_cal * cfg.d * es + T * cfg.d * es
