@@ -230,7 +230,7 @@ __device__ __forceinline__ bool run_product(const Product& pr, const Params& p, 
   const int slabs = two ? 2 : 1;
   const int slab_bytes = slabs * TP * ROW_PITCH;
   const int R = XCAP_BYTES / slab_bytes < kMaxSlots ? XCAP_BYTES / slab_bytes : kMaxSlots;
-  const int LOOK = R - 1;
+  const int LOOK = R > 1 ? R / 2 : 0;   // slabs in flight ahead of their use; the other slots let the warps drift apart
   const uint32_t xring = smem0 + RING_BYTES;
 
   float acc[TILES][NT][4];
