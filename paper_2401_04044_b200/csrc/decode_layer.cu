@@ -135,11 +135,12 @@ __device__ __forceinline__ void compute(float (&acc)[DUAL ? 2 : 1][NT][4], bool 
       // in which a contraction visits k is free as long as both operands agree on it)
       const uint32_t ws = wsrc + ti * TILE_BYTES + it * 64;
       const uint4 lo = lds128(ws), hi = lds128(ws + 8 * ROW_PITCH);
+      // all token tiles with the first half of k, then all with the second: two MMAs into the same
+      // accumulator are NT instructions apart instead of back to back
 #pragma unroll
-      for (int j = 0; j < NT; ++j) {
-        mma_bf16(acc[ti][j], lo.x, hi.x, lo.y, hi.y, xb[j].x, xb[j].y);
-        mma_bf16(acc[ti][j], lo.z, hi.z, lo.w, hi.w, xb[j].z, xb[j].w);
-      }
+      for (int j = 0; j < NT; ++j) mma_bf16(acc[ti][j], lo.x, hi.x, lo.y, hi.y, xb[j].x, xb[j].y);
+#pragma unroll
+      for (int j = 0; j < NT; ++j) mma_bf16(acc[ti][j], lo.z, hi.z, lo.w, hi.w, xb[j].z, xb[j].w);
     }
   }
 }
