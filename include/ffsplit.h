@@ -174,6 +174,19 @@ ffsplit_status ffsplit_blob_section(ffsplit_ctx* ctx, const void* blob, int32_t 
 ffsplit_status ffsplit_forward(ffsplit_ctx* ctx, const void* blob, const void* X, int64_t T,
                                void* Y, void* stream);
 
+/* Dense (unsplit) FFN straight from the row-major weights: Y = act(X W1 + b1) W2 + b2, the first
+ * equation of Section 2 (SwiGLU: Y = (SiLU(X W1) * (X W1u)) W2).  It is the split forward with every
+ * neuron heavy (h2 = all, no light part: Eq. 2 with FFN_2 empty), run by the same kernels: on every call
+ * the weights are first brought into the packed form inside the workspace, so the result is bit for bit
+ * that of ffsplit_pack with heavy_idx = 0 .. m-1, k = m followed by ffsplit_forward.  Meant as the
+ * comparator of the split forward; for repeated use pack once with k = m and call ffsplit_forward.
+ *   shape, wt   as for ffsplit_pack (dev pointers, row-major, 16-byte aligned, not retained)
+ *   X, Y        dev [T, d], 16-byte aligned
+ * Workspace needed: ffsplit_workspace_size(shape, T, 0, m, 0), rounded up to 256, plus the padded size
+ * ffsplit_pack_size(shape, m, 0) reports; FFSPLIT_ERR_BUFFER_TOO_SMALL otherwise, nothing launched. */
+ffsplit_status ffsplit_forward_dense(ffsplit_ctx* ctx, const ffsplit_shape* shape, const ffsplit_weights* wt,
+                                     const void* X, int64_t T, void* Y, void* stream);
+
 /* Same computation with HOST buffers: X_host [T, d] is copied to the device,
  * the forward runs, Y is copied back to Y_host [T, d]; all three on `stream`
  * (pinned host memory makes the copies asynchronous).  The workspace must have

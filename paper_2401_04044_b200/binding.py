@@ -33,6 +33,7 @@ EXPORTS = [
     "ffsplit_select", "ffsplit_pack_size", "ffsplit_pack", "ffsplit_blob_open", "ffsplit_blob_section",
     "ffsplit_forward", "ffsplit_forward_host", "ffsplit_poll", "ffsplit_launch_count", "ffsplit_last_error",
     "ffsplit_version", "ffsplit_profile_begin", "ffsplit_profile_end", "ffsplit_forward_noalloc",
+    "ffsplit_forward_dense",
 ]
 
 
@@ -205,6 +206,12 @@ class Context:
     def forward(self, blob, X, Y, stream=None):
         self._check(self.lib.ffsplit_forward(self.h, _ptr(blob), _ptr(X), X.shape[0], _ptr(Y), _stream_ptr(stream)),
                     "ffsplit_forward")
+
+    def forward_dense(self, shape: Shape, W1, b1, W2, b2, X, Y, W1u=None, stream=None):
+        """ffsplit_forward_dense: the unsplit FFN from the row-major weights (packed into the workspace per call)."""
+        w = Weights(_ptr(W1), _ptr(W1u), _ptr(b1), _ptr(W2), _ptr(b2))
+        self._check(self.lib.ffsplit_forward_dense(self.h, C.byref(shape), C.byref(w), _ptr(X), X.shape[0], _ptr(Y),
+                                                   _stream_ptr(stream)), "ffsplit_forward_dense")
 
     def forward_noalloc(self, blob, X, Y, stream=None):
         """ffsplit_forward_noalloc: up to 8 tokens, bf16, scratch built into the library (no workspace needed)."""

@@ -479,6 +479,10 @@ ffsplit_status ffsplit_pack_size(const ffsplit_shape* shape, int32_t k, int32_t 
   return FFSPLIT_OK;
 }
 
+static ffsplit_status pack_into(ffsplit_ctx* ctx, const ffsplit_shape* shape, const ffsplit_weights* wt,
+                                const int32_t* heavy_idx, int32_t k, const ffsplit_factors* f, const SplitDims& D,
+                                const BlobHeader& h, void* blob, cudaStream_t st);
+
 ffsplit_status ffsplit_pack(ffsplit_ctx* ctx, const ffsplit_shape* shape, const ffsplit_weights* wt,
                             const int32_t* heavy_idx, int32_t k, const ffsplit_factors* f, void* blob,
                             size_t blob_bytes, void* stream) {
@@ -500,18 +504,37 @@ ffsplit_status ffsplit_pack(ffsplit_ctx* ctx, const ffsplit_shape* shape, const 
   BlobHeader h;
   layout_blob(*shape, D, &h);
   if (blob_bytes < h.total_bytes) return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL, "blob buffer too small (ffsplit_pack_size)");
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  return pack_into(ctx, shape, wt, heavy_idx, k, f, D, h, blob, static_cast<cudaStream_t>(stream));
+}
+
+// Fills a blob whose layout `h` has been worked out.  heavy_idx == nullptr with k == m stands for the
+// identity 0 .. m-1 (the dense FFN): the heavy slices are then the whole matrices.
+static ffsplit_status pack_into(ffsplit_ctx* ctx, const ffsplit_shape* shape, const ffsplit_weights* wt,
+                                const int32_t* heavy_idx, int32_t k, const ffsplit_factors* f, const SplitDims& D,
+                                const BlobHeader& h, void* blob, cudaStream_t st) {
+  ffsplit_status s;
+  const int r = f ? f->r : 0;
+  const bool gated = shape->act == FFSPLIT_SWIGLU;
   char* b = static_cast<char*>(blob);
   const int d = shape->d, m = shape->m, dt = shape->dtype;
   const size_t es = elem_size(dt);
   // heavy slices: U1^T = (U[:, h2])^T, V1 = V[h2, :] -- plain copies of the inputs; all of the
   // gathers, transposes and bias conversions of the layer run as one batched launch
   prep_begin(ctx);
-  if ((s = launch_gather_cols_t(ctx, dt, wt->W1, m, d, heavy_idx, k, m, b + h.off[SEC_U1T], d, D.k_pad, st)) != FFSPLIT_OK)
-    return s;
-  if (gated &&
-      (s = launch_gather_cols_t(ctx, dt, wt->W1u, m, d, heavy_idx, k, m, b + h.off[SEC_U1UT], d, D.k_pad, st)) != FFSPLIT_OK)
-    return s;
+  if (heavy_idx || k == 0) {
+    if ((s = launch_gather_cols_t(ctx, dt, wt->W1, m, d, heavy_idx, k, m, b + h.off[SEC_U1T], d, D.k_pad, st)) != FFSPLIT_OK)
+      return s;
+    if (gated &&
+        (s = launch_gather_cols_t(ctx, dt, wt->W1u, m, d, heavy_idx, k, m, b + h.off[SEC_U1UT], d, D.k_pad, st)) != FFSPLIT_OK)
+      return s;
+  } else {
+    // all columns, in order: U1^T is the transpose of the whole matrix
+    if ((s = launch_transpose(ctx, dt, wt->W1, m, d, m, b + h.off[SEC_U1T], d, d, D.k_pad, nullptr, d, st)) != FFSPLIT_OK)
+      return s;
+    if (gated &&
+        (s = launch_transpose(ctx, dt, wt->W1u, m, d, m, b + h.off[SEC_U1UT], d, d, D.k_pad, nullptr, d, st)) != FFSPLIT_OK)
+      return s;
+  }
   if ((s = launch_transpose(ctx, dt, wt->W2, d, k, d, b + h.off[SEC_V1B2T], D.kp_rp, D.k_pad, d, heavy_idx, m, st)) !=
       FFSPLIT_OK)
     return s;
@@ -590,6 +613,33 @@ ffsplit_status ffsplit_forward(ffsplit_ctx* ctx, const void* blob, const void* X
   const BlobHeader* h = find_blob(ctx, blob, &s);
   if (!h) return s;
   return run_forward(ctx, *h, static_cast<const char*>(blob), X, T, Y, static_cast<cudaStream_t>(stream));
+}
+
+ffsplit_status ffsplit_forward_dense(ffsplit_ctx* ctx, const ffsplit_shape* shape, const ffsplit_weights* wt,
+                                     const void* X, int64_t T, void* Y, void* stream) {
+  ffsplit_status s = check_ctx(ctx, true);
+  if (s != FFSPLIT_OK) return s;
+  if ((s = check_shape(ctx, shape)) != FFSPLIT_OK) return s;
+  if (!wt || !wt->W1 || !wt->W2 || !X || !Y) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "NULL tensor");
+  if (T < 1) return fail(ctx, FFSPLIT_ERR_SHAPE, "T must be >= 1");
+  const bool gated = shape->act == FFSPLIT_SWIGLU;
+  if (gated && (!wt->W1u || wt->b1)) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "SwiGLU needs W1u and no b1");
+  if (!aligned16(X) || !aligned16(Y) || !aligned16(wt->W1) || !aligned16(wt->W2) || (gated && !aligned16(wt->W1u)))
+    return fail(ctx, FFSPLIT_ERR_ALIGN, "tensors must be 16-byte aligned");
+  // the dense FFN is the split with every neuron heavy: its packed form goes behind the forward buffers
+  const SplitDims D = make_dims(*shape, shape->m, 0);
+  BlobHeader h;
+  layout_blob(*shape, D, &h);
+  const FwdLayout L = fwd_layout(D, shape->d, shape->dtype, shape->act, T);
+  const size_t blob_off = align_up(kCtrlBytes + L.end);
+  if (blob_off + h.total_bytes > ctx->ws_bytes)
+    return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL,
+                "workspace too small for ffsplit_forward_dense: ffsplit_workspace_size(T, 0, k = m, r = 0) + "
+                "256 + the padded size of ffsplit_pack_size(k = m, r = 0)");
+  char* blob = ctx->ws + blob_off;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if ((s = pack_into(ctx, shape, wt, nullptr, shape->m, nullptr, D, h, blob, st)) != FFSPLIT_OK) return s;
+  return run_forward(ctx, h, blob, X, T, Y, st);
 }
 
 ffsplit_status ffsplit_forward_host(ffsplit_ctx* ctx, const void* blob, const void* X_host, int64_t T, void* Y_host,

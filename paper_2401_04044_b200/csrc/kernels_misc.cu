@@ -338,6 +338,14 @@ __device__ __forceinline__ void pack_bias_chunk(const PrepJob& q, int blk, int* 
   float* b2o = static_cast<float*>(q.out3);
   const int m = q.rows, k = q.cols, d = q.rows_pad, k_pad = q.cols_pad, ml_pad = q.idx_limit;
   const int j = blk * 256 + threadIdx.x;
+  if (heavy == nullptr && k == m && k > 0) {
+    // every neuron heavy, in order (k = m): b1[h2] is b1 itself and there is no light bias
+    if (j < k) b1h[j] = b1 ? to_float<T>(b1[j]) : 0.f;
+    if (j >= k && j < k_pad) b1h[j] = 0.f;
+    if (j < ml_pad) b1l[j] = 0.f;
+    if (j < d) b2o[j] = b2 ? to_float<T>(b2[j]) : 0.f;
+    return;
+  }
   if (j < k) {
     const int h = heavy[j];
     if (h < 0 || h >= m || (j > 0 && heavy[j - 1] >= h)) record_status(status, FFSPLIT_ERR_BAD_INDEX, j, KID_PACK);

@@ -277,6 +277,41 @@ def test_decode_forward_matches_oracle(ctx, act, d, m, k, r, T):
         assert_close(G.forward(blobd, X), dense_ref, "bf16", "decode dense forward")
 
 
+@pytest.mark.parametrize("dt,act,d,m,T", [("bf16", "gelu_erf", 256, 1000, 300), ("bf16", "swiglu", 192, 520, 5),
+                                         ("f32", "gelu_erf", 64, 192, 70), ("bf16", "gelu_tanh", 128, 384, 40)])
+def test_forward_dense_entry_point(ctx, dt, act, d, m, T):
+    """ffsplit_forward_dense (the dense FFN from the row-major weights) against the oracle's dense FFN, and bit
+    for bit against pack(heavy = 0 .. m-1, k = m) followed by ffsplit_forward: k = m is the dense FFN."""
+    cfg = custom_config(d, m, 16, 16, act=act, dtype=dt)
+    L = make_layer(cfg, 5)
+    G = GpuLayer(ctx, L)
+    G.reserve(T, 0, m, 0)
+    padded, _ = ctx.pack_size(G.shape, m, 0)
+    ctx.ensure_workspace(ctx.workspace_size(G.shape, T, 0, m, 0) + 256 + padded)
+    X = L.tokens(T)
+    Xd = X.cuda()
+    Y = torch.empty_like(Xd)
+    W1, b1, W2, b2, W1u = G.W1, G.b1, G.W2, G.b2, G.W1u
+    ctx.forward_dense(G.shape, W1, b1, W2, b2, Xd, Y, W1u=W1u)
+    ctx.poll()
+    dense_ref = orc.dense_ffn(f64(X), f64(L.W1), f64(L.b1), f64(L.W2), f64(L.b2), act, f64(L.W1u))
+    assert_close(Y, dense_ref, dt, "ffsplit_forward_dense")
+    blob, _ = G.pack(torch.arange(m), None)
+    assert torch.equal(G.forward(blob, X).cpu(), Y.cpu()), "forward_dense differs from pack(k = m) + forward"
+    # a workspace without room for the packed form is refused before anything is launched
+    ctx2_ws = ctx.workspace_size(G.shape, T, 0, m, 0)
+    from paper_2401_04044_b200 import Context
+    from paper_2401_04044_b200.binding import FFSplitError
+    c2 = Context(0)
+    try:
+        c2.ensure_workspace(ctx2_ws)
+        with pytest.raises(FFSplitError) as e:
+            c2.forward_dense(G.shape, W1, b1, W2, b2, Xd, Y, W1u=W1u)
+        assert e.value.code == 5
+    finally:
+        c2.close()
+
+
 @pytest.mark.parametrize("act,d,m,k,r", [("gelu_erf", 1024, 4096, 205, 256), ("swiglu", 512, 1400, 70, 128)])
 @pytest.mark.parametrize("T", [1, 8, 24, 64])
 def test_decode_single_launch_mode(ctx, monkeypatch, act, d, m, k, r, T):
