@@ -127,6 +127,20 @@ ffsplit_status ffsplit_score(ffsplit_ctx* ctx, const ffsplit_shape* shape, const
                              const void* X, int64_t T, int32_t mode, int32_t accumulate,
                              float* energy, float* scores, void* stream);
 
+/* Eq. 3 from a stored activation matrix: the same energy, scores and modes as ffsplit_score, for a
+ * caller that already holds H = sigma(X U) [T, m] in device memory (kept from a forward pass, say), so
+ * that scoring is one streaming read of H instead of a product: e_j (+)= sum_t H[t,j]^2 (SUM_NORM:
+ * sum_t |H[t,j]|), then s_j as in ffsplit_score.  For SwiGLU, H is SiLU(X Wg) * (X Wu).
+ *   H          dev [T, m] row-major, shape->dtype, 16-byte aligned
+ *   W2         dev [m, d]; may be NULL when scores is NULL or mode is ACT_ONLY
+ *   energy, scores, accumulate, mode: as for ffsplit_score
+ * Workspace: what ffsplit_workspace_size(shape, 0, T, 0, 0) reports is enough.  Partial sums are added
+ * in a fixed order: results are bitwise reproducible.  Rounding differs from ffsplit_score, which
+ * squares the un-rounded fp32 activations: here H has already been rounded to its storage type. */
+ffsplit_status ffsplit_score_activations(ffsplit_ctx* ctx, const ffsplit_shape* shape, const void* H, int64_t T,
+                                         const void* W2, int32_t mode, int32_t accumulate, float* energy,
+                                         float* scores, void* stream);
+
 /* Deterministic top-k (Section 4.1: the neurons with the highest output norm
  * are the heavy hitters).  Equal scores go to the lower index.
  *   scores     dev float[m], finite (a NaN/Inf sets FFSPLIT_ERR_NONFINITE in the status block)

@@ -33,7 +33,7 @@ EXPORTS = [
     "ffsplit_select", "ffsplit_pack_size", "ffsplit_pack", "ffsplit_blob_open", "ffsplit_blob_section",
     "ffsplit_forward", "ffsplit_forward_host", "ffsplit_poll", "ffsplit_launch_count", "ffsplit_last_error",
     "ffsplit_version", "ffsplit_profile_begin", "ffsplit_profile_end", "ffsplit_forward_noalloc",
-    "ffsplit_forward_dense",
+    "ffsplit_forward_dense", "ffsplit_score_activations",
 ]
 
 
@@ -172,6 +172,13 @@ class Context:
         self._check(self.lib.ffsplit_score(self.h, C.byref(shape), C.byref(w), _ptr(X), X.shape[0], int(mode),
                                            int(bool(accumulate)), _ptr(energy), _ptr(scores), _stream_ptr(stream)),
                     "ffsplit_score")
+
+    def score_activations(self, shape: Shape, H, W2, energy, scores=None, mode=SCORE_EQ3, accumulate=False,
+                          stream=None):
+        """ffsplit_score_activations: Eq. 3 from a stored activation matrix H [T, m]."""
+        self._check(self.lib.ffsplit_score_activations(self.h, C.byref(shape), _ptr(H), H.shape[0], _ptr(W2), mode,
+                                                       1 if accumulate else 0, _ptr(energy), _ptr(scores),
+                                                       _stream_ptr(stream)), "ffsplit_score_activations")
 
     def select(self, scores, k: int, heavy_idx, light_idx=None, stream=None):
         self._check(self.lib.ffsplit_select(self.h, _ptr(scores), scores.numel(), k, _ptr(heavy_idx), _ptr(light_idx),

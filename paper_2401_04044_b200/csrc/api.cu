@@ -457,6 +457,33 @@ ffsplit_status ffsplit_score(ffsplit_ctx* ctx, const ffsplit_shape* shape, const
   return launch_score_finalize(ctx, partial, L.groups, m, w, energy, scores, mode, accumulate, st);
 }
 
+ffsplit_status ffsplit_score_activations(ffsplit_ctx* ctx, const ffsplit_shape* shape, const void* H, int64_t T,
+                                         const void* W2, int32_t mode, int32_t accumulate, float* energy,
+                                         float* scores, void* stream) {
+  ffsplit_status s = check_ctx(ctx, true);
+  if (s != FFSPLIT_OK) return s;
+  if ((s = check_shape(ctx, shape)) != FFSPLIT_OK) return s;
+  if (!H || !energy) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "NULL tensor");
+  if (T < 1) return fail(ctx, FFSPLIT_ERR_SHAPE, "T must be >= 1");
+  if (mode < 0 || mode > 2) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "unknown score mode");
+  const bool need_w = scores && mode != FFSPLIT_SCORE_ACT_ONLY;
+  if (need_w && !W2) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "W2 is NULL");
+  if (!aligned16(H) || (W2 && !aligned16(W2))) return fail(ctx, FFSPLIT_ERR_ALIGN, "tensors must be 16-byte aligned");
+  const int d = shape->d, m = shape->m, dt = shape->dtype;
+  const int groups = column_energy_groups(T);
+  const size_t w_off = 0, part_off = align_up((size_t)m * 4);
+  const size_t end = part_off + align_up((size_t)groups * m * 4);
+  if (kCtrlBytes + end > ctx->ws_bytes)
+    return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL, "workspace too small for this score call");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  char* base = ctx->ws + kCtrlBytes;
+  float* w = reinterpret_cast<float*>(base + w_off);
+  float* partial = reinterpret_cast<float*>(base + part_off);
+  if (need_w && (s = launch_row_energy(ctx, dt, W2, m, d, w, st)) != FFSPLIT_OK) return s;
+  if ((s = launch_column_energy(ctx, dt, H, m, T, m, partial, mode == FFSPLIT_SCORE_SUM_NORM, st)) != FFSPLIT_OK) return s;
+  return launch_score_finalize(ctx, partial, groups, m, w, energy, scores, mode, accumulate, st);
+}
+
 ffsplit_status ffsplit_select(ffsplit_ctx* ctx, const float* scores, int32_t m, int32_t k, int32_t* heavy_idx,
                               int32_t* light_idx, void* stream) {
   ffsplit_status s = check_ctx(ctx, true);

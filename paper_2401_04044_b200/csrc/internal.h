@@ -230,7 +230,7 @@ __device__ __forceinline__ void pdl_wait() {
 #endif
 
 // Profiling brackets: no-ops unless ffsplit_profile_begin() is active.
-enum ProfClass : int { PROF_GEMM_TC = 0, PROF_GEMM_SIMT = 1, PROF_DECODE = 2 };
+enum ProfClass : int { PROF_GEMM_TC = 0, PROF_GEMM_SIMT = 1, PROF_DECODE = 2, PROF_ENERGY = 3 };
 int prof_open(ffsplit_ctx* ctx, int cls, double work, cudaStream_t st);
 void prof_close(ffsplit_ctx* ctx, int handle, cudaStream_t st);
 
@@ -252,6 +252,9 @@ ffsplit_status launch_gather_cols_t(ffsplit_ctx* ctx, int dtype, const void* in,
 ffsplit_status launch_pack_bias(ffsplit_ctx* ctx, int dtype, const void* b1, const void* b2, const int* heavy, int m,
                                 int k, int d, float* b1h, int k_pad, float* b1l, int ml_pad, float* b2o,
                                 cudaStream_t st);
+int column_energy_groups(long long rows);
+ffsplit_status launch_column_energy(ffsplit_ctx* ctx, int dtype, const void* H, long long ldh, long long rows, int m,
+                                    float* partial, int use_abs, cudaStream_t st);
 ffsplit_status launch_score_finalize(ffsplit_ctx* ctx, const float* partial, int groups, int m, const float* w,
                                      float* energy, float* scores, int mode, int accumulate, cudaStream_t st);
 bool fused_light_applies(int dtype, int act, int r_pad, int ml_pad);

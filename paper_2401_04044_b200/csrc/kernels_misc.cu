@@ -183,6 +183,81 @@ ffsplit_status launch_score_finalize(ffsplit_ctx* ctx, const float* partial, int
 }
 
 // ============================================================================
+// Column energy of a stored activation matrix (Eq. 3, the factor ||sigma(X U_{:,j})||^2 when the
+// activations H [T, m] already exist in memory): partial[g, j] = sum over the rows of group g of
+// H[t, j]^2 (or |H[t, j]|).  Pure streaming: every warp-wide load takes 512 contiguous bytes of one
+// row; a thread keeps its 16 bytes' worth of columns in registers over the group's rows, the eight
+// warps of the CTA are added through shared memory in warp order.  score_finalize_kernel then adds
+// the groups.
+// ============================================================================
+constexpr int kEnergyRows = 256;   // rows of H per group
+
+template <typename T>
+__global__ void __launch_bounds__(256) column_energy_kernel(const T* __restrict__ H, long long ldh, long long rows,
+                                                            int m, float* __restrict__ partial, int use_abs) {
+  constexpr int VEC = 16 / sizeof(T);
+  __shared__ float red[8][32 * VEC];
+  pdl_wait();
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  const int c0 = blockIdx.x * (32 * VEC) + tx * VEC;
+  const long long r0 = static_cast<long long>(blockIdx.y) * kEnergyRows;
+  const long long r1 = r0 + kEnergyRows < rows ? r0 + kEnergyRows : rows;
+  float acc[VEC];
+#pragma unroll
+  for (int i = 0; i < VEC; ++i) acc[i] = 0.f;
+  const bool vec = c0 + VEC <= m && (ldh % VEC) == 0 && (reinterpret_cast<uintptr_t>(H) & 15u) == 0;
+  if (vec) {
+#pragma unroll 4
+    for (long long r = r0 + ty; r < r1; r += 8) {
+      const uint4 raw = __ldcs(reinterpret_cast<const uint4*>(H + r * ldh + c0));   // read once: streaming load
+      const T* e = reinterpret_cast<const T*>(&raw);
+#pragma unroll
+      for (int i = 0; i < VEC; ++i) {
+        const float x = to_float<T>(e[i]);
+        acc[i] = use_abs ? acc[i] + fabsf(x) : fmaf(x, x, acc[i]);
+      }
+    }
+  } else {
+    for (long long r = r0 + ty; r < r1; r += 8)
+      for (int i = 0; i < VEC; ++i)
+        if (c0 + i < m) {
+          const float x = to_float<T>(H[r * ldh + c0 + i]);
+          acc[i] = use_abs ? acc[i] + fabsf(x) : fmaf(x, x, acc[i]);
+        }
+  }
+#pragma unroll
+  for (int i = 0; i < VEC; ++i) red[ty][tx * VEC + i] = acc[i];
+  __syncthreads();
+  for (int c = threadIdx.x; c < 32 * VEC; c += 256) {
+    float s = 0.f;
+#pragma unroll
+    for (int w = 0; w < 8; ++w) s += red[w][c];   // fixed order
+    const int col = blockIdx.x * (32 * VEC) + c;
+    if (col < m) partial[static_cast<long long>(blockIdx.y) * m + col] = s;
+  }
+}
+
+int column_energy_groups(long long rows) { return static_cast<int>((rows + kEnergyRows - 1) / kEnergyRows); }
+
+ffsplit_status launch_column_energy(ffsplit_ctx* ctx, int dtype, const void* H, long long ldh, long long rows, int m,
+                                    float* partial, int use_abs, cudaStream_t st) {
+  const int groups = column_energy_groups(rows);
+  if (groups > 65535) return fail(ctx, FFSPLIT_ERR_SHAPE, "more than 65535*256 activation rows in one call");
+  const int ph = prof_open(ctx, PROF_ENERGY, static_cast<double>(rows) * m * elem_size(dtype), st);
+  cudaError_t le;
+  if (dtype == FFSPLIT_BF16) {
+    le = launch_pdl(column_energy_kernel<__nv_bfloat16>, dim3((m + 255) / 256, groups), dim3(256), 0, st,
+                    static_cast<const __nv_bfloat16*>(H), ldh, rows, m, partial, use_abs);
+  } else {
+    le = launch_pdl(column_energy_kernel<float>, dim3((m + 127) / 128, groups), dim3(256), 0, st,
+                    static_cast<const float*>(H), ldh, rows, m, partial, use_abs);
+  }
+  prof_close(ctx, ph, st);
+  ctx->launches++;
+  return check_cuda(ctx, le, "column_energy_kernel launch");
+}
+
+// ============================================================================
 // Small data-movement and reduction jobs of scoring and packing, batched: the
 // jobs recorded between prep_begin() and prep_flush() run as ONE launch whose
 // blocks are dealt out to the jobs (each job is far too small to fill the GPU,

@@ -98,6 +98,45 @@ def test_score_matches_oracle(ctx, dt, act, d, m, T, mode):
     assert torch.equal(scores, scores3) and torch.equal(energy, energy3)
 
 
+@pytest.mark.parametrize("dt,act,d,m,T", [("bf16", "gelu_erf", 96, 1000, 700), ("bf16", "swiglu", 64, 520, 300),
+                                         ("f32", "gelu_erf", 48, 200, 530), ("bf16", "gelu_tanh", 64, 2051, 257)])
+@pytest.mark.parametrize("mode", [0, 1, 2])
+def test_score_activations_matches_oracle(ctx, dt, act, d, m, T, mode):
+    """Eq. 3 from a stored activation matrix: the oracle's activations are rounded to the storage type once,
+    and both sides reduce those same stored values (fp32 sums on the GPU, fp64 in the check)."""
+    cfg = custom_config(d, m, max(1, m // 20), 16, act=act, dtype=dt)
+    L = make_layer(cfg, 2)
+    G = GpuLayer(ctx, L)
+    G.reserve(0, T, 0, 0)
+    X = L.tokens(T)
+    H = torch.from_numpy(orc.neuron_activations(f64(X), f64(L.W1), f64(L.b1), act, f64(L.W1u))).to(cfg.torch_dtype)
+    Hs = f64(H)                                   # the stored values
+    W2 = f64(L.W2)
+    w_ref = np.sum(W2 * W2, axis=1)
+    e_ref = np.sum(np.abs(Hs), axis=0) if mode == 2 else np.sum(Hs * Hs, axis=0)
+    s_ref = [e_ref * w_ref, e_ref, e_ref * np.sqrt(w_ref)][mode]
+    Hd = H.cuda()
+    energy = torch.empty(m, dtype=torch.float32, device="cuda")
+    scores = torch.empty(m, dtype=torch.float32, device="cuda")
+    ctx.score_activations(G.shape, Hd, G.W2, energy, scores, mode=mode)
+    ctx.poll()
+    assert np.allclose(f64(energy), e_ref, rtol=1e-5, atol=1e-6 * e_ref.max())
+    assert np.allclose(f64(scores), s_ref, rtol=2e-5, atol=1e-6 * s_ref.max())
+    # two batches accumulate to the same totals; a repeated call is bitwise identical
+    e2 = torch.empty_like(energy)
+    s2 = torch.empty_like(scores)
+    cut = (T // 2 // 8) * 8
+    ctx.score_activations(G.shape, Hd[:cut].clone(), G.W2, e2, None, mode=mode)
+    ctx.score_activations(G.shape, Hd[cut:].clone(), G.W2, e2, s2, mode=mode, accumulate=True)
+    ctx.poll()
+    assert np.allclose(f64(s2), s_ref, rtol=2e-5, atol=1e-6 * s_ref.max())
+    e3 = torch.empty_like(energy)
+    s3 = torch.empty_like(scores)
+    ctx.score_activations(G.shape, Hd, G.W2, e3, s3, mode=mode)
+    ctx.poll()
+    assert torch.equal(e3, energy) and torch.equal(s3, scores)
+
+
 @pytest.mark.parametrize("dt,act", [("f32", "gelu_erf"), ("bf16", "gelu_erf"), ("bf16", "swiglu")])
 def test_planted_heavy_hitters_recovered_end_to_end(ctx, dt, act):
     cfg = custom_config(128, 640, 32, 16, act=act, dtype=dt)
