@@ -152,6 +152,46 @@ def run_point(ctx, cfg, tokens, copies, reps, svd, device="cuda", use_graph=True
     return out
 
 
+def run_scoring(ctx, cfg, reps, device="cuda", t_cal=None):
+    """Scoring pass of one layer, both forms: from the calibration tokens (product + fused column energy)
+    and from a stored activation matrix (one streaming read of H).  Events around each call, median."""
+    hbm, tf, src, _ = peaks()
+    shape = make_shape(cfg.d, cfg.m, cfg.act, cfg.torch_dtype)
+    T = t_cal or cfg.t_cal
+    es = 2 if cfg.dtype == "bf16" else 4
+    ctx.ensure_workspace(ctx.workspace_size(shape, 0, T, 0, 0))
+    L = make_layer(cfg, 0, device=device)
+    X = L.tokens(T)
+    H = torch.randn(T, cfg.m, device=device, dtype=torch.float32).mul_(0.5).to(cfg.torch_dtype)
+    energy = torch.empty(cfg.m, dtype=torch.float32, device=device)
+    scores = torch.empty(cfg.m, dtype=torch.float32, device=device)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+    out = {"config": cfg.name, "d": cfg.d, "m": cfg.m, "T_cal": T, "dtype": cfg.dtype, "peaks": src}
+    forms = (("fused", lambda: ctx.score(shape, L.W1, L.b1, L.W2, X, energy, scores, W1u=L.W1u)),
+             ("stored", lambda: ctx.score_activations(shape, H, L.W2, energy, scores)))
+    for name, fn in forms:
+        ts = []
+        for i in range(reps + 3):
+            flush.add_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            b.synchronize()
+            if i >= 3:
+                ts.append(a.elapsed_time(b))
+        ctx.poll()
+        ms = statistics.median(ts)
+        flops = 2.0 * cfg.n_in * T * cfg.d * cfg.m if name == "fused" else 0.0
+        bytes_ = (es * (T * cfg.d + (cfg.n_in + 1) * cfg.d * cfg.m) if name == "fused"
+                  else es * (T * cfg.m + cfg.m * cfg.d))
+        roof_ms = max(flops / (tf * 1e12), bytes_ / (hbm * 1e9)) * 1e3
+        out[name] = {"ms": ms, "roofline_ms": roof_ms, "roofline_frac": roof_ms / ms,
+                     "bound": "tensor" if flops / (tf * 1e12) > bytes_ / (hbm * 1e9) else "hbm",
+                     "tflops": flops / (ms * 1e-3) / 1e12, "gbs": bytes_ / (ms * 1e-3) / 1e9}
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--config", type=int, required=True)
@@ -163,6 +203,8 @@ def main():
     ap.add_argument("--out", default=None)
     ap.add_argument("--which", nargs="*", default=["split", "dense"], choices=["split", "dense"],
                     help="time the split layer, its dense counterpart, or both")
+    ap.add_argument("--scoring", action="store_true", help="time the scoring pass (both forms) instead of the forward")
+    ap.add_argument("--t-cal", type=int, default=0, help="with --scoring: calibration tokens (default: the config's)")
     ap.add_argument("--settle", type=float, default=1.0,
                     help="seconds of idle time before each timed case (the clocks recover from the case before)")
     ap.add_argument("--no-graph", action="store_true", help="issue the timed calls one by one instead of replaying a CUDA graph")
@@ -173,6 +215,9 @@ def main():
     points = [base]
     if args.config == 5 and args.sweep5:
         points = [cfg5_point(h, r) for h in CFG5_HEAVY_PERCENT for r in CFG5_RANKS]
+    if args.scoring:
+        print(json.dumps(run_scoring(ctx, base, args.reps, t_cal=args.t_cal or None)), flush=True)
+        return
     tokens = args.tokens or list(base.t_fwd)
     lines = []
     for cfg in points:
