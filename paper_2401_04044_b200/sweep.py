@@ -203,6 +203,9 @@ def main():
     ap.add_argument("--out", default=None)
     ap.add_argument("--which", nargs="*", default=["split", "dense"], choices=["split", "dense"],
                     help="time the split layer, its dense counterpart, or both")
+    ap.add_argument("--paper-point", action="store_true",
+                    help="the paper's own hyper-parameters at BERT-base shape (Section 5.1.1): top 25 %% of the neurons "
+                         "heavy (k = 768), light rank = 10 %% of full rank (r = 77); --config is ignored")
     ap.add_argument("--scoring", action="store_true", help="time the scoring pass (both forms) instead of the forward")
     ap.add_argument("--t-cal", type=int, default=0, help="with --scoring: calibration tokens (default: the config's)")
     ap.add_argument("--settle", type=float, default=1.0,
@@ -212,6 +215,11 @@ def main():
     build.build()
     ctx = Context(0)
     base = CONFIGS[args.config]
+    if args.paper_point:
+        from ffsplit_synth import custom_config
+        import dataclasses
+        base = dataclasses.replace(custom_config(768, 3072, 768, 77, act="gelu_erf", dtype="bf16", t_cal=4096),
+                                   name="bert_base_paper_point_k768_r77", layers=12, t_fwd=(4096,))
     points = [base]
     if args.config == 5 and args.sweep5:
         points = [cfg5_point(h, r) for h in CFG5_HEAVY_PERCENT for r in CFG5_RANKS]
