@@ -42,6 +42,9 @@ struct Params {
   int stages;        // depth of the shared-memory ring (as many as fit, at most 8)
   int tiles_m, tiles_n;
   int dual;
+  int shared_a;      // gated pair with one left operand (A0 == A1): A is staged once per k block, the two
+                     // weight tiles sit one behind the other and ONE MMA of width 2 block_n fills both accumulators
+  int gate_off;      // tensor-memory column of the second accumulator of a gated tile: 128, or block_n when shared_a
   Epilogue epi;
   int* status;
 };
@@ -136,7 +139,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   const int STAGES = p.stages;
-  const int B_STAGE_BYTES = p.block_n * BLOCK_K * 2;
+  const int B_TILE_BYTES = p.block_n * BLOCK_K * 2;
+  const int B_STAGE_BYTES = p.shared_a ? 2 * B_TILE_BYTES : B_TILE_BYTES;
   uint8_t* smem_a = smem;
   uint8_t* smem_b = smem + STAGES * A_STAGE_BYTES;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES));
@@ -188,7 +192,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   const int nkb = (p.K + BLOCK_K - 1) / BLOCK_K;
-  const int total_kb = p.dual ? 2 * nkb : nkb;
+  const int total_kb = (p.dual && !p.shared_a) ? 2 * nkb : nkb;
   const int num_tiles = p.tiles_m * p.tiles_n;
   const uint32_t stage_tx = A_STAGE_BYTES + B_STAGE_BYTES;
 
@@ -208,6 +212,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           const int kk = (second ? kb - nkb : kb) * BLOCK_K;
           ptx::tma_load_2d(second ? &tmA1 : &tmA0, smem_a + s * A_STAGE_BYTES, &full[s], kk, m_blk * BLOCK_M);
           ptx::tma_load_2d(second ? &tmB1 : &tmB0, smem_b + s * B_STAGE_BYTES, &full[s], kk, n_blk * p.block_n);
+          if (p.shared_a)   // the second weight tile right behind the first: rows block_n .. 2 block_n - 1 of one operand
+            ptx::tma_load_2d(&tmB1, smem_b + s * B_STAGE_BYTES + B_TILE_BYTES, &full[s], kk, n_blk * p.block_n);
         }
       }
       if (!ok) {
@@ -224,7 +230,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   } else if (warp == 1) {
     if (ptx::elect_one()) {
       // ------------------------------------------------------------ MMA issuer
-      const uint32_t idesc = ptx::umma_idesc_bf16(BLOCK_M, p.block_n);
+      const uint32_t idesc = ptx::umma_idesc_bf16(BLOCK_M, p.shared_a ? 2 * p.block_n : p.block_n);
       uint32_t it = 0, tl = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tl) {
@@ -238,7 +244,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           ptx::tc_fence_after();
           const bool second = p.dual && kb >= nkb;
           const int kbl = second ? kb - nkb : kb;
-          const uint32_t d_tmem = tmem_base + acc * ACC_STRIDE + (second ? GATE_OFFSET : 0);
+          const uint32_t d_tmem = tmem_base + acc * ACC_STRIDE + (second ? p.gate_off : 0);
           const uint64_t a_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_a + s * A_STAGE_BYTES));
           const uint64_t b_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_b + s * B_STAGE_BYTES));
 #pragma unroll
@@ -325,7 +331,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           if (n0 >= p.N) break;
           float v[16], u[16];
           ptx::tmem_ld16(t_row + c, v);
-          ptx::tmem_ld16(t_row + GATE_OFFSET + c, u);
+          ptx::tmem_ld16(t_row + p.gate_off + c, u);
           ptx::tmem_ld_wait();
 #pragma unroll
           for (int i = 0; i < 16; ++i)
@@ -419,9 +425,11 @@ ffsplit_status launch_gemm_tc(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_t 
   p.N = g.N;
   p.K = g.K;
   p.dual = dual ? 1 : 0;
+  p.shared_a = (dual && g.A0 == g.A1 && g.lda0 == g.lda1) ? 1 : 0;
   p.tiles_m = static_cast<int>((g.M + tc::BLOCK_M - 1) / tc::BLOCK_M);
   p.block_n = choose_block_n(g.N, p.tiles_m, ctx->num_sms, dual);
   p.tiles_n = (g.N + p.block_n - 1) / p.block_n;
+  p.gate_off = p.shared_a ? p.block_n : tc::GATE_OFFSET;
   p.epi = g.epi;
   p.status = ctx->status();
   CUtensorMap tA0, tB0, tA1, tB1;
@@ -441,7 +449,7 @@ ffsplit_status launch_gemm_tc(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_t 
     if (e != cudaSuccess) return check_cuda(ctx, e, "cudaFuncSetAttribute(gemm_tc_kernel)");
     ctx->attr_tc_set = true;
   }
-  const int stage_bytes = tc::A_STAGE_BYTES + p.block_n * tc::BLOCK_K * 2;
+  const int stage_bytes = tc::A_STAGE_BYTES + (p.shared_a ? 2 : 1) * p.block_n * tc::BLOCK_K * 2;
   p.stages = (tc::MAX_SMEM - tc::BAR_BYTES - 1024) / stage_bytes;
   if (p.stages > tc::MAX_STAGES) p.stages = tc::MAX_STAGES;
   const int smem_bytes = p.stages * stage_bytes + tc::BAR_BYTES + 1024;
