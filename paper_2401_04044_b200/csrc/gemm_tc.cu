@@ -44,6 +44,9 @@ struct Params {
   int dual;
   int shared_a;      // gated pair with one left operand (A0 == A1): A is staged once per k block, the two
                      // weight tiles sit one behind the other and ONE MMA of width 2 block_n fills both accumulators
+  int two_m;         // 256 x block_n tiles: two 128-row blocks of A against one weight tile (half the weight
+                     // traffic per FLOP); the two accumulator buffers hold the halves, so the epilogue of a tile
+                     // does not overlap the MMAs of the next one
   int gate_off;      // tensor-memory column of the second accumulator of a gated tile: 128, or block_n when shared_a
   Epilogue epi;
   int* status;
@@ -141,9 +144,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   const int STAGES = p.stages;
   const int B_TILE_BYTES = p.block_n * BLOCK_K * 2;
   const int B_STAGE_BYTES = p.shared_a ? 2 * B_TILE_BYTES : B_TILE_BYTES;
+  const int MT = p.two_m ? 2 : 1;                 // 128-row blocks of A per tile
+  const int A_STAGE = MT * A_STAGE_BYTES;
   uint8_t* smem_a = smem;
-  uint8_t* smem_b = smem + STAGES * A_STAGE_BYTES;
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * (A_STAGE_BYTES + B_STAGE_BYTES));
+  uint8_t* smem_b = smem + STAGES * A_STAGE;
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * (A_STAGE + B_STAGE_BYTES));
   uint64_t* full = bars;                      // [MAX_STAGES] TMA -> MMA
   uint64_t* empty = bars + MAX_STAGES;        // [MAX_STAGES] MMA -> TMA
   uint64_t* tfull = bars + 2 * MAX_STAGES;    // [2] MMA -> epilogue
@@ -194,7 +199,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   const int nkb = (p.K + BLOCK_K - 1) / BLOCK_K;
   const int total_kb = (p.dual && !p.shared_a) ? 2 * nkb : nkb;
   const int num_tiles = p.tiles_m * p.tiles_n;
-  const uint32_t stage_tx = A_STAGE_BYTES + B_STAGE_BYTES;
+  const uint32_t stage_tx = A_STAGE + B_STAGE_BYTES;
 
   if (warp == 0) {
     if (ptx::elect_one()) {
@@ -210,7 +215,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           ptx::mbar_expect_tx(&full[s], stage_tx);
           const bool second = p.dual && kb >= nkb;
           const int kk = (second ? kb - nkb : kb) * BLOCK_K;
-          ptx::tma_load_2d(second ? &tmA1 : &tmA0, smem_a + s * A_STAGE_BYTES, &full[s], kk, m_blk * BLOCK_M);
+          for (int mt = 0; mt < MT; ++mt)
+            ptx::tma_load_2d(second ? &tmA1 : &tmA0, smem_a + s * A_STAGE + mt * A_STAGE_BYTES, &full[s], kk,
+                             (m_blk * MT + mt) * BLOCK_M);
           ptx::tma_load_2d(second ? &tmB1 : &tmB0, smem_b + s * B_STAGE_BYTES, &full[s], kk, n_blk * p.block_n);
           if (p.shared_a)   // the second weight tile right behind the first: rows block_n .. 2 block_n - 1 of one operand
             ptx::tma_load_2d(&tmB1, smem_b + s * B_STAGE_BYTES + B_TILE_BYTES, &full[s], kk, n_blk * p.block_n);
@@ -234,8 +241,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       uint32_t it = 0, tl = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tl) {
-        const uint32_t acc = tl & 1, aph = (tl >> 1) & 1;
+        // one buffer per tile, alternating -- or, with 256-row tiles, both buffers for the two halves
+        const uint32_t acc = p.two_m ? 0 : (tl & 1), aph = p.two_m ? (tl & 1) : ((tl >> 1) & 1);
         if (!ptx::mbar_wait(&tempty[acc], aph ^ 1, abort_flag)) { ok = false; break; }
+        if (p.two_m && !ptx::mbar_wait(&tempty[1], aph ^ 1, abort_flag)) { ok = false; break; }
         ptx::tc_fence_after();
         for (int kb = 0; kb < total_kb; ++kb, ++it) {
           const int s = it % STAGES;
@@ -245,16 +254,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           const bool second = p.dual && kb >= nkb;
           const int kbl = second ? kb - nkb : kb;
           const uint32_t d_tmem = tmem_base + acc * ACC_STRIDE + (second ? p.gate_off : 0);
-          const uint64_t a_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_a + s * A_STAGE_BYTES));
+          const uint64_t a_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_a + s * A_STAGE));
           const uint64_t b_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_b + s * B_STAGE_BYTES));
 #pragma unroll
           for (int k = 0; k < BLOCK_K / 16; ++k) {
             // 16 elements (32 bytes) further along K inside the swizzled row: +2 in the address field
             ptx::umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kbl | k) != 0 ? 1u : 0u);
           }
+          if (p.two_m) {
+            // the second 128 rows of A against the same weights, into the other accumulator buffer
+            const uint64_t a2_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_a + s * A_STAGE + A_STAGE_BYTES));
+#pragma unroll
+            for (int k = 0; k < BLOCK_K / 16; ++k)
+              ptx::umma_bf16(d_tmem + ACC_STRIDE, a2_desc + 2 * k, b_desc + 2 * k, idesc, (kbl | k) != 0 ? 1u : 0u);
+          }
           ptx::umma_commit(&empty[s]);
         }
-        if (ok) ptx::umma_commit(&tfull[acc]);
+        if (ok) {
+          ptx::umma_commit(&tfull[acc]);
+          if (p.two_m) ptx::umma_commit(&tfull[1]);
+        }
       }
       if (!ok) {
         // wait (bounded) until the MMAs issued so far have retired before TMEM is freed
@@ -269,16 +288,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     const int q = warp & 3;             // TMEM lane quarter this warp may read
     const int half = (warp - 2) >> 2;   // which of every EPI_WARPS / 4 consecutive 16-column chunks this warp takes
     const GeluCoef gc = gelu_coef(p.epi.act);
-    uint32_t tl = 0;
-    for (int tile = blockIdx.x; tile < num_tiles; tile += gridDim.x, ++tl) {
-      const int m_blk = tile / p.tiles_n, n_blk = tile % p.tiles_n;
-      const uint32_t acc = tl & 1, aph = (tl >> 1) & 1;
+    // The epilogue walks 128-row blocks: one per tile, or the two halves of a 256-row tile one after the
+    // other -- either way block number vt uses accumulator buffer vt & 1 in phase (vt >> 1) & 1.
+    uint32_t vt = 0;
+    bool live = true;
+    for (int tile = blockIdx.x; tile < num_tiles && live; tile += gridDim.x)
+    for (int mt = 0; mt < MT; ++mt, ++vt) {
+      const int m_blk = (tile / p.tiles_n) * MT + mt, n_blk = tile % p.tiles_n;
+      const uint32_t acc = vt & 1, aph = (vt >> 1) & 1;
       if (warp == 2 && p.epi.n_bias > 0) {
         // this tile's slice of the bias vector, on its way to L1 while the MMAs run
         const int nb = n_blk * p.block_n + lane * 32;
         if (lane * 32 < p.block_n && nb < p.epi.n_bias) asm volatile("prefetch.global.L1 [%0];" ::"l"(p.epi.bias + nb));
       }
-      if (!ptx::mbar_wait(&tfull[acc], aph, abort_flag)) break;
+      if (!ptx::mbar_wait(&tfull[acc], aph, abort_flag)) { live = false; break; }
       ptx::tc_fence_after();
       const long long row = static_cast<long long>(m_blk) * BLOCK_M + q * 32 + lane;
       const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * ACC_STRIDE;
@@ -428,6 +451,25 @@ ffsplit_status launch_gemm_tc(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_t 
   p.shared_a = (dual && g.A0 == g.A1 && g.lda0 == g.lda1) ? 1 : 0;
   p.tiles_m = static_cast<int>((g.M + tc::BLOCK_M - 1) / tc::BLOCK_M);
   p.block_n = choose_block_n(g.N, p.tiles_m, ctx->num_sms, dual);
+  p.two_m = 0;
+  if (ctx->gemm_two_m && !dual && g.epi.col_partial == nullptr && g.K >= 1024 && g.M > tc::BLOCK_M) {
+    // 256-row tiles halve the weight bytes staged per FLOP (the kernels are bound by the shared-memory
+    // fill rate, not by the tensor pipe) but expose each tile's epilogue and make the tiles coarser:
+    // taken when the K loop is long and the waves stay about as full as with 128-row tiles.
+    const long long tm2 = (g.M + 2 * tc::BLOCK_M - 1) / (2 * tc::BLOCK_M);
+    const int bn2 = choose_block_n(g.N, tm2, ctx->num_sms, false);
+    const auto wave_fill = [&](long long tiles) {
+      const long long waves = (tiles + ctx->num_sms - 1) / ctx->num_sms;
+      return static_cast<double>(tiles) / static_cast<double>(waves * ctx->num_sms);
+    };
+    const long long t1 = static_cast<long long>(p.tiles_m) * ((g.N + p.block_n - 1) / p.block_n);
+    const long long t2 = tm2 * ((g.N + bn2 - 1) / bn2);
+    if (bn2 >= 128 && wave_fill(t2) >= 0.9 * wave_fill(t1)) {
+      p.two_m = 1;
+      p.tiles_m = static_cast<int>(tm2);
+      p.block_n = bn2;
+    }
+  }
   p.tiles_n = (g.N + p.block_n - 1) / p.block_n;
   p.gate_off = p.shared_a ? p.block_n : tc::GATE_OFFSET;
   p.epi = g.epi;
@@ -449,7 +491,7 @@ ffsplit_status launch_gemm_tc(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_t 
     if (e != cudaSuccess) return check_cuda(ctx, e, "cudaFuncSetAttribute(gemm_tc_kernel)");
     ctx->attr_tc_set = true;
   }
-  const int stage_bytes = tc::A_STAGE_BYTES + (p.shared_a ? 2 : 1) * p.block_n * tc::BLOCK_K * 2;
+  const int stage_bytes = (p.two_m ? 2 : 1) * tc::A_STAGE_BYTES + (p.shared_a ? 2 : 1) * p.block_n * tc::BLOCK_K * 2;
   p.stages = (tc::MAX_SMEM - tc::BAR_BYTES - 1024) / stage_bytes;
   if (p.stages > tc::MAX_STAGES) p.stages = tc::MAX_STAGES;
   const int smem_bytes = p.stages * stage_bytes + tc::BAR_BYTES + 1024;
