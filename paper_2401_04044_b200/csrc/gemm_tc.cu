@@ -321,7 +321,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           }
           const float tot = warp_column_sums16(v, lane);
           const int n = n0 + (lane >> 1);
-          if ((lane & 1) == 0 && n < p.N)
+          // (the second half of a 256-row tile may lie wholly behind the last row: it has no partial)
+          if ((lane & 1) == 0 && n < p.N && static_cast<long long>(m_blk) * BLOCK_M < p.M)
             e.col_partial[(static_cast<long long>(m_blk) * 4 + q) * p.N + n] = tot;
         }
       };
@@ -452,19 +453,19 @@ ffsplit_status launch_gemm_tc(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_t 
   p.tiles_m = static_cast<int>((g.M + tc::BLOCK_M - 1) / tc::BLOCK_M);
   p.block_n = choose_block_n(g.N, p.tiles_m, ctx->num_sms, dual);
   p.two_m = 0;
-  if (ctx->gemm_two_m && !dual && g.epi.col_partial == nullptr && g.K >= 1024 && g.M > tc::BLOCK_M) {
+  if (ctx->gemm_two_m && (!dual || p.shared_a) && g.K >= 1024 && g.M > tc::BLOCK_M) {
     // 256-row tiles halve the weight bytes staged per FLOP (the kernels are bound by the shared-memory
     // fill rate, not by the tensor pipe) but expose each tile's epilogue and make the tiles coarser:
     // taken when the K loop is long and the waves stay about as full as with 128-row tiles.
     const long long tm2 = (g.M + 2 * tc::BLOCK_M - 1) / (2 * tc::BLOCK_M);
-    const int bn2 = choose_block_n(g.N, tm2, ctx->num_sms, false);
+    const int bn2 = choose_block_n(g.N, tm2, ctx->num_sms, dual);
     const auto wave_fill = [&](long long tiles) {
       const long long waves = (tiles + ctx->num_sms - 1) / ctx->num_sms;
       return static_cast<double>(tiles) / static_cast<double>(waves * ctx->num_sms);
     };
     const long long t1 = static_cast<long long>(p.tiles_m) * ((g.N + p.block_n - 1) / p.block_n);
     const long long t2 = tm2 * ((g.N + bn2 - 1) / bn2);
-    if (bn2 >= 128 && wave_fill(t2) >= 0.9 * wave_fill(t1)) {
+    if (bn2 >= (dual ? 64 : 128) && wave_fill(t2) >= 0.9 * wave_fill(t1)) {
       p.two_m = 1;
       p.tiles_m = static_cast<int>(tm2);
       p.block_n = bn2;
