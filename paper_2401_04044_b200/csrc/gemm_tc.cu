@@ -453,7 +453,7 @@ ffsplit_status launch_gemm_tc(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_t 
   p.tiles_m = static_cast<int>((g.M + tc::BLOCK_M - 1) / tc::BLOCK_M);
   p.block_n = choose_block_n(g.N, p.tiles_m, ctx->num_sms, dual);
   p.two_m = 0;
-  if (ctx->gemm_two_m && (!dual || p.shared_a) && g.K >= 1024 && g.M > tc::BLOCK_M) {
+  if (ctx->gemm_two_m && (!dual || p.shared_a) && g.K >= 2048 && g.M > tc::BLOCK_M) {
     // 256-row tiles halve the weight bytes staged per FLOP (the kernels are bound by the shared-memory
     // fill rate, not by the tensor pipe) but expose each tile's epilogue and make the tiles coarser:
     // taken when the K loop is long and the waves stay about as full as with 128-row tiles.
