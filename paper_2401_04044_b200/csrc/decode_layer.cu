@@ -404,11 +404,15 @@ __global__ void __launch_bounds__(THREADS, 1) decode_layer_kernel(const __grid_c
 
 template <int NT, bool GATED>
 cudaError_t launch_nt(const Params& p, int grid, bool cooperative, cudaStream_t st) {
-  static bool attr_done = false;
-  if (!attr_done) {
-    cudaError_t e = cudaFuncSetAttribute(decode_layer_kernel<NT, GATED>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+  // the shared-memory allowance is a per-device property of the function: set once on every device used
+  static bool attr_done[64] = {false};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64 || !attr_done[dev]) {
+    e = cudaFuncSetAttribute(decode_layer_kernel<NT, GATED>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
     if (e != cudaSuccess) return e;
-    attr_done = true;
+    if (dev >= 0 && dev < 64) attr_done[dev] = true;
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(grid);
