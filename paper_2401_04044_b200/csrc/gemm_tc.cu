@@ -312,12 +312,25 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         } else {
           const Epilogue& e = p.epi;
           if (n0 < e.n_bias) add_bias16(e, n0, v);
+          // scores decide indices: fp32-accurate activation, not the one-MUFU form
+          if (!p.dual && e.act == FFSPLIT_GELU_ERF && !e.score_abs) {
+            // the common case, without per-element selects
 #pragma unroll
-          for (int i = 0; i < 16; ++i) {
-            float x = v[i];
-            if (!p.dual) x = act_gelu_score(x, e.act);   // scores decide indices: fp32-accurate activation, not the one-MUFU form
-            x = e.score_abs ? fabsf(x) : x * x;
-            v[i] = (row < p.M) ? x : 0.0f;
+            for (int i = 0; i < 16; ++i) {
+              const float x = gelu_erf_score_f(v[i]);
+              v[i] = x * x;
+            }
+          } else {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) {
+              float x = v[i];
+              if (!p.dual) x = act_gelu_score(x, e.act);
+              v[i] = e.score_abs ? fabsf(x) : x * x;
+            }
+          }
+          if (row >= p.M) {
+#pragma unroll
+            for (int i = 0; i < 16; ++i) v[i] = 0.0f;
           }
           const float tot = warp_column_sums16(v, lane);
           const int n = n0 + (lane >> 1);
