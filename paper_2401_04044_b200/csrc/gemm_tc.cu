@@ -478,7 +478,7 @@ ffsplit_status launch_gemm_tc(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_t 
     };
     const long long t1 = static_cast<long long>(p.tiles_m) * ((g.N + p.block_n - 1) / p.block_n);
     const long long t2 = tm2 * ((g.N + bn2 - 1) / bn2);
-    if (bn2 >= (dual ? 64 : 128) && wave_fill(t2) >= 0.9 * wave_fill(t1)) {
+    if (ctx->gemm_two_m == 2 || (bn2 >= (dual ? 64 : 128) && wave_fill(t2) >= 0.9 * wave_fill(t1))) {
       p.two_m = 1;
       p.tiles_m = static_cast<int>(tm2);
       p.block_n = bn2;

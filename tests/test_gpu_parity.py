@@ -316,6 +316,46 @@ def test_decode_forward_matches_oracle(ctx, act, d, m, k, r, T):
         assert_close(G.forward(blobd, X), dense_ref, "bf16", "decode dense forward")
 
 
+@pytest.mark.parametrize("act", ["gelu_erf", "swiglu"])
+@pytest.mark.parametrize("T", [300, 520])
+def test_long_contraction_tiles(monkeypatch, act, T):
+    """d = 2048 with FFSPLIT_GEMM_TWO_M=2 puts the scoring product and stage 1 on the 256-row tiles (two row
+    blocks per weight tile; at full size the library picks them by itself) and, for SwiGLU, on the
+    one-MMA-per-pair form; T = 300 leaves the second half of the last tile wholly behind the last token row,
+    T = 520 ends inside a first half."""
+    from paper_2401_04044_b200 import Context
+    d, m, k, r = 2048, 640, 96, 64
+    cfg = custom_config(d, m, k, r, act=act, dtype="bf16")
+    L = make_layer(cfg, 3)
+    monkeypatch.setenv("FFSPLIT_GEMM_TWO_M", "2")
+    ctx = Context(0)
+    try:
+        _long_contraction_body(ctx, L, cfg, act, T, d, m, k, r)
+    finally:
+        ctx.close()
+
+
+def _long_contraction_body(ctx, L, cfg, act, T, d, m, k, r):
+    G = GpuLayer(ctx, L)
+    G.reserve(T, T, k, r)
+    G.reserve(T, 0, m, 0)
+    X = L.tokens(T)
+    energy, scores = G.score(X)
+    e_ref, _, s_ref = orc.neuron_scores(f64(X), f64(L.W1), f64(L.b1), f64(L.W2), act, orc.SCORE_EQ3, f64(L.W1u))
+    rt = SCORE_RTOL["bf16"]
+    assert np.allclose(f64(energy), e_ref, rtol=rt, atol=rt * e_ref.max() * 1e-3)
+    assert np.allclose(f64(scores), s_ref, rtol=rt, atol=rt * s_ref.max() * 1e-3)
+    heavy, _ = G.select(scores, k)
+    heavy_ref, _ = orc.select_heavy(s_ref, k)
+    assert np.array_equal(heavy.cpu().numpy(), heavy_ref)
+    fac = oracle_factors(L, heavy_ref, r)
+    blob, _ = G.pack(torch.from_numpy(heavy_ref), fac)
+    assert_close(G.forward(blob, X), oracle_split(L, heavy_ref, fac, X), "bf16", "split forward, long K")
+    blobd, _ = G.pack(torch.arange(m), None)
+    dense_ref = orc.dense_ffn(f64(X), f64(L.W1), f64(L.b1), f64(L.W2), f64(L.b2), act, f64(L.W1u))
+    assert_close(G.forward(blobd, X), dense_ref, "bf16", "dense forward, long K")
+
+
 @pytest.mark.parametrize("dt,act,d,m,T", [("bf16", "gelu_erf", 256, 1000, 300), ("bf16", "swiglu", 192, 520, 5),
                                          ("f32", "gelu_erf", 64, 192, 70), ("bf16", "gelu_tanh", 128, 384, 40)])
 def test_forward_dense_entry_point(ctx, dt, act, d, m, T):
