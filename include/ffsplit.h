@@ -13,15 +13,17 @@
  *   - All tensors are row-major and dense.  "dev" pointers are CUDA device
  *     memory owned by the caller; the library never allocates, frees or keeps
  *     a tensor pointer past the call (the workspace is kept until replaced;
- *     a packed blob's address is remembered as a cache key only).
+ *     a packed blob's address is remembered as the key under which its header
+ *     is registered, see ffsplit_blob_open()).
  *   - Storage dtype (ffsplit_dtype) applies to X, Y, weights, biases and
  *     factors alike: FFSPLIT_BF16 computes with bf16 tensor-core products and
  *     fp32 accumulation; FFSPLIT_F32 computes in plain fp32 (no TF32).
  *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls
  *     enqueue work and return; argument errors are returned synchronously and
  *     launch nothing.  Conditions only the device can see (non-finite score,
- *     unsorted index list, a wait that ran out) are recorded in a status word
- *     inside the workspace and returned by ffsplit_poll().
+ *     unsorted index list, a blob whose bytes changed after registration, a
+ *     wait that ran out) are recorded in a status word inside the workspace
+ *     and returned by ffsplit_poll().
  *   - Device pointers must be 16-byte aligned (FFSPLIT_ERR_ALIGN otherwise).
  *     For FFSPLIT_BF16, d must be a multiple of 8 (rows of X start 16-byte aligned).
  *   - Same inputs give bitwise the same outputs on every call.
@@ -114,7 +116,7 @@ ffsplit_status ffsplit_workspace_size(const ffsplit_shape* shape, int64_t T_fwd,
 ffsplit_status ffsplit_set_workspace(ffsplit_ctx* ctx, void* dev_ptr, size_t bytes);
 
 /* Heavy-hitter scoring over one batch of calibration tokens (Eq. 3; Section
- * 4.2, "go over a small training set").
+ * 4.2: the calibration pass over a small token set).
  *   X       dev [T, d] calibration tokens, T >= 1
  *   energy  dev float[m], caller-owned accumulator: e_j = sum_t H[t,j]^2 with
  *           H = sigma(X W1 + b1) (sum_t |H[t,j]| for SCORE_SUM_NORM).
@@ -122,10 +124,34 @@ ffsplit_status ffsplit_set_workspace(ffsplit_ctx* ctx, void* dev_ptr, size_t byt
  *   scores  dev float[m] or NULL.  When given: s_j = e_j * w_j (EQ3),
  *           e_j (ACT_ONLY) or e_j * sqrt(w_j) (SUM_NORM), w_j = sum_c W2[j,c]^2,
  *           formed from the accumulated energy after this batch.
- * The T x m activation matrix is never written to memory.  Uses the workspace. */
+ * The T x m activation matrix is never written to memory.  Uses the workspace.
+ * With accumulate = 1, the transposed weights a previous batch left in the workspace
+ * are reused when the weight pointers and the shape are the same and no other call
+ * has used the workspace in between: do not change the weights during an accumulation. */
 ffsplit_status ffsplit_score(ffsplit_ctx* ctx, const ffsplit_shape* shape, const ffsplit_weights* weights,
                              const void* X, int64_t T, int32_t mode, int32_t accumulate,
                              float* energy, float* scores, void* stream);
+
+/* ffsplit_score() with the calibration tokens in HOST memory (Eq. 3; Section 4.2): X_host [T, d] is
+ * copied to the device in chunks that pass through the workspace (pinned host memory makes the copies
+ * asynchronous), each chunk is scored and added to `energy`; `scores` is formed after the last one.
+ * Weights, energy and scores are device memory as for ffsplit_score().  The workspace must hold the
+ * scoring buffers plus at least 128 staged tokens (ffsplit_workspace_size(shape, 0, T_cal, 0, 0) plus
+ * T_cal * d * sizeof(dtype) stages all of a T_cal-token batch at once); FFSPLIT_ERR_BUFFER_TOO_SMALL
+ * otherwise.  Copies and kernels are all enqueued on `stream`. */
+ffsplit_status ffsplit_score_host(ffsplit_ctx* ctx, const ffsplit_shape* shape, const ffsplit_weights* weights,
+                                  const void* X_host, int64_t T, int32_t mode, int32_t accumulate,
+                                  float* energy, float* scores, void* stream);
+
+/* Scores from an energy vector that is already complete (Eq. 3: s_j = e_j * ||V_j||^2, or the other
+ * modes of ffsplit_score): for calibration runs whose energy was accumulated elsewhere -- over several
+ * calls with scores = NULL, or summed over the ranks of a token-sharded calibration (Section 4.2; every
+ * rank then forms bitwise the same scores from the same summed energy).
+ *   W2      dev [m, d]; may be NULL for SCORE_ACT_ONLY
+ *   energy  dev float[m], read (and left unchanged); scores dev float[m], written
+ * Workspace: 65536 + 4 m bytes. */
+ffsplit_status ffsplit_score_finalize(ffsplit_ctx* ctx, const ffsplit_shape* shape, const void* W2, int32_t mode,
+                                      float* energy, float* scores, void* stream);
 
 /* Eq. 3 from a stored activation matrix: the same energy, scores and modes as ffsplit_score, for a
  * caller that already holds H = sigma(X U) [T, m] in device memory (kept from a forward pass, say), so
@@ -169,10 +195,22 @@ ffsplit_status ffsplit_pack(ffsplit_ctx* ctx, const ffsplit_shape* shape, const 
                             const int32_t* heavy_idx, int32_t k, const ffsplit_factors* factors,
                             void* blob, size_t blob_bytes, void* stream);
 
-/* Register a blob that reached device memory by other means than ffsplit_pack()
- * on this context (a copy, a reload).  Reads and validates its header
- * (synchronous 256-byte copy).  FFSPLIT_ERR_BAD_BLOB if it is not a blob. */
-ffsplit_status ffsplit_blob_open(ffsplit_ctx* ctx, const void* blob, size_t blob_bytes);
+/* Register a blob that reached device memory by other means than ffsplit_pack() on this context (a
+ * copy, a reload, a pack on another context).  The forward calls accept only blobs that were packed or
+ * opened on the context they are called on (FFSPLIT_ERR_BAD_BLOB otherwise; nothing is opened
+ * implicitly).  The 256-byte header is copied to the host on `stream`, which is then synchronised, and
+ * validated against blob_bytes, the size of the caller's buffer: FFSPLIT_ERR_BAD_BLOB if it is not a
+ * blob or claims more than blob_bytes.  The bytes of the blob must be complete in `stream`'s order
+ * (pass the stream that produced them, or synchronise first).
+ * A registration is keyed by the blob's address and describes the bytes that were there at the time:
+ * after overwriting a registered buffer with another blob, or before reusing its address for something
+ * else, call ffsplit_blob_open() again or ffsplit_blob_close().  As a safeguard the first kernel of
+ * every forward compares the header in device memory with the registered one and reports a mismatch
+ * as FFSPLIT_ERR_BAD_BLOB through ffsplit_poll(); the output of such a call is undefined. */
+ffsplit_status ffsplit_blob_open(ffsplit_ctx* ctx, const void* blob, size_t blob_bytes, void* stream);
+
+/* Forget a blob (packed or opened on this context).  FFSPLIT_ERR_BAD_BLOB if it is not known. */
+ffsplit_status ffsplit_blob_close(ffsplit_ctx* ctx, const void* blob);
 
 /* Where one matrix of the blob lives, for inspection and tests.
  * which: 0 heavy U1^T [k_pad, d] (1: SwiGLU up), 2 A1^T [r_pad, d] (3: up),
@@ -208,6 +246,20 @@ ffsplit_status ffsplit_forward_dense(ffsplit_ctx* ctx, const ffsplit_shape* shap
 ffsplit_status ffsplit_forward_host(ffsplit_ctx* ctx, const void* blob, const void* X_host, int64_t T,
                                     void* Y_host, void* stream);
 
+/* A stack of split layers (Eq. 2 applied layer after layer, the per-stack figure of the throughput
+ * reports): layer l reads what layer l-1 wrote, Y = FFN_{n-1}( ... FFN_0(X)).  Nothing sits between the
+ * layers (no residual, no normalisation).  All blobs must be known to the context and share d and dtype.
+ *   blobs   host array of n_layers dev pointers
+ *   X, Y    dev [T, d] (ffsplit_forward_stack) or host [T, d] (ffsplit_forward_stack_host: copied in
+ *           and out on `stream`, like ffsplit_forward_host)
+ * Workspace: ffsplit_stack_workspace_size() (the largest per-layer need plus two [T, d] buffers). */
+ffsplit_status ffsplit_stack_workspace_size(ffsplit_ctx* ctx, const void* const* blobs, int32_t n_layers, int64_t T,
+                                            size_t* bytes);
+ffsplit_status ffsplit_forward_stack(ffsplit_ctx* ctx, const void* const* blobs, int32_t n_layers, const void* X,
+                                     int64_t T, void* Y, void* stream);
+ffsplit_status ffsplit_forward_stack_host(ffsplit_ctx* ctx, const void* const* blobs, int32_t n_layers,
+                                          const void* X_host, int64_t T, void* Y_host, void* stream);
+
 /* The split forward of ffsplit_forward() for callers that cannot allocate device memory.
  * (The paper has no counterpart to this entry point; it exists for deployment.)
  *
@@ -228,13 +280,24 @@ ffsplit_status ffsplit_forward_host(ffsplit_ctx* ctx, const void* blob, const vo
  * make that first call outside any stream capture.
  * All calls on a device share the one array and it keeps the previous call's contents: the call
  * clears the counters it needs at zero itself, but two calls that overlap on the GPU (different
- * streams, no ordering between them) race on it.  Results equal those of ffsplit_forward(). */
+ * streams, no ordering between them) race on it.  Results equal those of ffsplit_forward().
+ * Like ffsplit_forward() it accepts only blobs packed or opened on `ctx`.  A device-side condition of
+ * this call (a wait that ran out, a changed blob) is kept in the array's own status words until
+ * ffsplit_poll() on any context of that device reports it; ffsplit_poll() needs no workspace for that. */
 ffsplit_status ffsplit_forward_noalloc(ffsplit_ctx* ctx, const void* blob, const void* X, int64_t T,
                                        void* Y, void* stream);
 
-/* Synchronise `stream`, then return and clear the device status word
- * (FFSPLIT_OK if no kernel recorded a condition). */
+/* Synchronise `stream`, then return and clear the first device-side condition found in the workspace's
+ * status word or in that of the built-in scratch of ffsplit_forward_noalloc() on the context's device
+ * (FFSPLIT_OK if no kernel recorded one).  Works on a context without a workspace. */
 ffsplit_status ffsplit_poll(ffsplit_ctx* ctx, void* stream);
+
+/* Self-test of the bounded waits (every wait inside the library's kernels gives up after a limit
+ * instead of spinning forever): launches a one-CTA kernel whose wait on a barrier that nothing signals
+ * is limited to `limit_cycles` SM clocks (1 .. 1e8).  The wait runs out, the kernel returns normally,
+ * and the next ffsplit_poll() reports FFSPLIT_ERR_TIMEOUT; the context stays usable.  (The paper has no
+ * counterpart; this is a diagnostic.)  Needs a workspace (for the status word). */
+ffsplit_status ffsplit_debug_wait_timeout(ffsplit_ctx* ctx, int64_t limit_cycles, void* stream);
 
 /* Per-launch device timing of the library's main kernels, for roofline reports.
  * Between ffsplit_profile_begin() and ffsplit_profile_end() every launch of a

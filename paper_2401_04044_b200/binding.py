@@ -33,7 +33,9 @@ EXPORTS = [
     "ffsplit_select", "ffsplit_pack_size", "ffsplit_pack", "ffsplit_blob_open", "ffsplit_blob_section",
     "ffsplit_forward", "ffsplit_forward_host", "ffsplit_poll", "ffsplit_launch_count", "ffsplit_last_error",
     "ffsplit_version", "ffsplit_profile_begin", "ffsplit_profile_end", "ffsplit_forward_noalloc",
-    "ffsplit_forward_dense", "ffsplit_score_activations",
+    "ffsplit_forward_dense", "ffsplit_score_activations", "ffsplit_score_host", "ffsplit_score_finalize",
+    "ffsplit_blob_close", "ffsplit_stack_workspace_size", "ffsplit_forward_stack", "ffsplit_forward_stack_host",
+    "ffsplit_debug_wait_timeout",
 ]
 
 
@@ -79,7 +81,16 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.ffsplit_select.argtypes = [vp, vp, i32, i32, vp, vp, vp]
     lib.ffsplit_pack_size.argtypes = [P(Shape), i32, i32, P(sz), P(sz)]
     lib.ffsplit_pack.argtypes = [vp, P(Shape), P(Weights), vp, i32, P(Factors), vp, sz, vp]
-    lib.ffsplit_blob_open.argtypes = [vp, vp, sz]
+    lib.ffsplit_blob_open.argtypes = [vp, vp, sz, vp]
+    lib.ffsplit_blob_close.argtypes = [vp, vp]
+    lib.ffsplit_score_host.argtypes = [vp, P(Shape), P(Weights), vp, i64, i32, i32, vp, vp, vp]
+    lib.ffsplit_score_finalize.argtypes = [vp, P(Shape), vp, i32, vp, vp, vp]
+    lib.ffsplit_score_activations.argtypes = [vp, P(Shape), vp, i64, vp, i32, i32, vp, vp, vp]
+    lib.ffsplit_forward_dense.argtypes = [vp, P(Shape), P(Weights), vp, i64, vp, vp]
+    lib.ffsplit_stack_workspace_size.argtypes = [vp, P(vp), i32, i64, P(sz)]
+    lib.ffsplit_forward_stack.argtypes = [vp, P(vp), i32, vp, i64, vp, vp]
+    lib.ffsplit_forward_stack_host.argtypes = [vp, P(vp), i32, vp, i64, vp, vp]
+    lib.ffsplit_debug_wait_timeout.argtypes = [vp, i64, vp]
     lib.ffsplit_blob_section.argtypes = [vp, vp, i32, P(sz), P(i64), P(i64), P(i64)]
     lib.ffsplit_forward.argtypes = [vp, vp, vp, i64, vp, vp]
     lib.ffsplit_forward_host.argtypes = [vp, vp, vp, i64, vp, vp]
@@ -200,9 +211,49 @@ class Context:
         self._check(self.lib.ffsplit_pack(self.h, C.byref(shape), C.byref(w), _ptr(heavy_idx), k, fp, _ptr(blob),
                                           blob.numel() * blob.element_size(), _stream_ptr(stream)), "ffsplit_pack")
 
-    def blob_open(self, blob):
-        self._check(self.lib.ffsplit_blob_open(self.h, _ptr(blob), blob.numel() * blob.element_size()),
-                    "ffsplit_blob_open")
+    def blob_open(self, blob, stream=None):
+        self._check(self.lib.ffsplit_blob_open(self.h, _ptr(blob), blob.numel() * blob.element_size(),
+                                               _stream_ptr(stream)), "ffsplit_blob_open")
+
+    def blob_close(self, blob):
+        self._check(self.lib.ffsplit_blob_close(self.h, _ptr(blob)), "ffsplit_blob_close")
+
+    def score_host(self, shape: Shape, W1, b1, W2, X_host, energy, scores=None, mode=SCORE_EQ3, accumulate=False,
+                   W1u=None, stream=None):
+        """ffsplit_score_host: calibration tokens in (pinned) host memory, staged through the workspace in chunks."""
+        w = Weights(_ptr(W1), _ptr(W1u), _ptr(b1), _ptr(W2), None)
+        self._check(self.lib.ffsplit_score_host(self.h, C.byref(shape), C.byref(w), _ptr(X_host), X_host.shape[0],
+                                                int(mode), int(bool(accumulate)), _ptr(energy), _ptr(scores),
+                                                _stream_ptr(stream)), "ffsplit_score_host")
+
+    def score_finalize(self, shape: Shape, W2, energy, scores, mode=SCORE_EQ3, stream=None):
+        """ffsplit_score_finalize: scores from a complete energy vector (after a sharded or multi-call accumulation)."""
+        self._check(self.lib.ffsplit_score_finalize(self.h, C.byref(shape), _ptr(W2), int(mode), _ptr(energy),
+                                                    _ptr(scores), _stream_ptr(stream)), "ffsplit_score_finalize")
+
+    @staticmethod
+    def _blob_array(blobs):
+        arr = (C.c_void_p * len(blobs))(*[b.data_ptr() for b in blobs])
+        return arr
+
+    def stack_workspace_size(self, blobs, T: int) -> int:
+        n = C.c_size_t()
+        self._check(self.lib.ffsplit_stack_workspace_size(self.h, self._blob_array(blobs), len(blobs), T, C.byref(n)),
+                    "ffsplit_stack_workspace_size")
+        return n.value
+
+    def forward_stack(self, blobs, X, Y, stream=None):
+        self._check(self.lib.ffsplit_forward_stack(self.h, self._blob_array(blobs), len(blobs), _ptr(X), X.shape[0],
+                                                   _ptr(Y), _stream_ptr(stream)), "ffsplit_forward_stack")
+
+    def forward_stack_host(self, blobs, X_host, Y_host, stream=None):
+        self._check(self.lib.ffsplit_forward_stack_host(self.h, self._blob_array(blobs), len(blobs), _ptr(X_host),
+                                                        X_host.shape[0], _ptr(Y_host), _stream_ptr(stream)),
+                    "ffsplit_forward_stack_host")
+
+    def debug_wait_timeout(self, limit_cycles: int, stream=None):
+        self._check(self.lib.ffsplit_debug_wait_timeout(self.h, int(limit_cycles), _stream_ptr(stream)),
+                    "ffsplit_debug_wait_timeout")
 
     def blob_section(self, blob, which: int):
         off, r, c, ld = C.c_size_t(), C.c_int64(), C.c_int64(), C.c_int64()

@@ -38,8 +38,9 @@ void prof_close(ffsplit_ctx* ctx, int handle, cudaStream_t st) {
 
 ffsplit_status launch_decode_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* blob, const void* X,
                                      long long T, void* Y, char* AP, char* Q, char* HL, char* scratch,
-                                     cudaStream_t st);
+                                     cudaStream_t st, unsigned long long guard_hash);
 bool decode_path_applies(const ffsplit_ctx* ctx, const BlobHeader& h, long long T);
+char* noalloc_control_block(int device);   // nullptr until ffsplit_forward_noalloc has run on that device
 size_t decode_scratch_bytes(int dtype, long long T);
 
 namespace {
@@ -180,21 +181,26 @@ ffsplit_status check_ctx(ffsplit_ctx* ctx, bool need_ws) {
   return FFSPLIT_OK;
 }
 
-const BlobHeader* find_blob(ffsplit_ctx* ctx, const void* blob, ffsplit_status* st) {
+// A blob is known to a context once ffsplit_pack() wrote it or ffsplit_blob_open() registered it there;
+// nothing is opened implicitly (a header read inside a forward would be a synchronous copy that is not
+// ordered after whatever produced the blob).
+const ffsplit_ctx::BlobEntry* find_blob(ffsplit_ctx* ctx, const void* blob, ffsplit_status* st) {
   auto it = ctx->blobs.find(blob);
   if (it != ctx->blobs.end()) return &it->second;
-  *st = ffsplit_blob_open(ctx, blob, 0);
-  if (*st != FFSPLIT_OK) return nullptr;
-  return &ctx->blobs.find(blob)->second;
+  *st = fail(ctx, FFSPLIT_ERR_BAD_BLOB,
+             "blob not known to this context: pack it here or register it with ffsplit_blob_open()");
+  return nullptr;
 }
 
 // The three-stage split forward (Eq. 2) as a sequence of GEMMs with fused epilogues.
+// guard_hash != 0: the first kernel checks that the header in device memory still is the one registered.
 ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* blob, const void* X, long long T,
-                           void* Y, cudaStream_t st) {
+                           void* Y, cudaStream_t st, unsigned long long guard_hash) {
   const SplitDims D = dims_of(h);
   const size_t es = elem_size(h.dtype);
   const int d = h.d;
   char* base = ctx->ws + kCtrlBytes;
+  ctx->score_prep.valid = false;   // the forward buffers share the workspace with the scoring buffers
   const FwdLayout L = fwd_layout(D, d, h.dtype, h.act, T);
   const bool few = decode_path_applies(ctx, h, T);
   if (kCtrlBytes + (few ? L.end : L.xs) > ctx->ws_bytes)
@@ -202,7 +208,8 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
   char* AP = base + L.ap;
   char* Q = base + L.q;
   char* HL = base + L.hl;
-  if (few) return launch_decode_forward(ctx, h, blob, X, T, Y, AP, Q, HL, base + L.dscratch, st);
+  if (few) return launch_decode_forward(ctx, h, blob, X, T, Y, AP, Q, HL, base + L.dscratch, st, guard_hash);
+  const unsigned long long* guard = guard_hash ? reinterpret_cast<const unsigned long long*>(blob) : nullptr;
   const float* b1h = reinterpret_cast<const float*>(blob + h.off[SEC_B1H]);
   const float* b1l = reinterpret_cast<const float*>(blob + h.off[SEC_B1L]);
   const float* b2 = reinterpret_cast<const float*>(blob + h.off[SEC_B2]);
@@ -222,6 +229,7 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
     g.epi.C1 = Q; g.epi.ld1 = D.r_pad;
     g.epi.n_split = D.k_pad; g.epi.n_act = D.k_pad; g.epi.n_bias = D.k_pad;
     g.epi.bias = b1h; g.epi.act = h.act;
+    g.epi.guard = guard; g.epi.guard_hash = guard_hash;
     if ((s = launch_gemm(ctx, h.dtype, g, st)) != FFSPLIT_OK) return s;
   } else {
     std::memset(&g, 0, sizeof(g));
@@ -231,6 +239,7 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
     g.algo_flops = 4.0 * T * d * D.k;
     g.epi.C0 = AP; g.epi.ld0 = D.kp_rp;
     g.epi.n_split = D.k_pad; g.epi.n_act = D.k_pad; g.epi.act = h.act;
+    g.epi.guard = guard; g.epi.guard_hash = guard_hash;
     if ((s = launch_gemm(ctx, h.dtype, g, st)) != FFSPLIT_OK) return s;
     if (light) {
       std::memset(&g, 0, sizeof(g));
@@ -287,8 +296,71 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
   return launch_gemm(ctx, h.dtype, g, st);
 }
 
+
+// ---- a stack of layers, layer l reading layer l-1's output ------------------------------------
+// The intermediate outputs alternate between two buffers placed behind the largest per-layer forward layout.
+struct StackLayout { size_t ping, pong, end; };
+ffsplit_status stack_layout(ffsplit_ctx* ctx, const void* const* blobs, int n_layers, long long T, StackLayout* out) {
+  size_t body = 0;
+  int d = -1, dtype = -1;
+  for (int l = 0; l < n_layers; ++l) {
+    ffsplit_status s = FFSPLIT_OK;
+    const ffsplit_ctx::BlobEntry* ent = find_blob(ctx, blobs[l], &s);
+    if (!ent) return s;
+    const BlobHeader& h = ent->h;
+    if (l == 0) { d = h.d; dtype = h.dtype; }
+    else if (h.d != d || h.dtype != dtype)
+      return fail(ctx, FFSPLIT_ERR_SHAPE, "the layers of a stack must share the hidden width and the dtype");
+    const size_t e = fwd_layout(dims_of(h), h.d, h.dtype, h.act, T).end;
+    if (e > body) body = e;
+  }
+  const size_t act = align_up(static_cast<size_t>(T) * d * elem_size(dtype));
+  out->ping = body;
+  out->pong = body + act;
+  out->end = body + 2 * act;
+  return FFSPLIT_OK;
+}
+
 }  // namespace
 }  // namespace ffsp
+
+static ffsplit_status forward_stack_impl(ffsplit_ctx* ctx, const void* const* blobs, int n_layers, const void* X,
+                                         long long T, void* Y, cudaStream_t st, bool host) {
+  ffsplit_status s = check_ctx(ctx, true);
+  if (s != FFSPLIT_OK) return s;
+  if (!blobs || n_layers < 1 || !X || !Y) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "NULL tensor or empty stack");
+  if (T < 1) return fail(ctx, FFSPLIT_ERR_SHAPE, "T must be >= 1");
+  if (!host && (!aligned16(X) || !aligned16(Y))) return fail(ctx, FFSPLIT_ERR_ALIGN, "X and Y must be 16-byte aligned");
+  StackLayout SL;
+  if ((s = stack_layout(ctx, blobs, n_layers, T, &SL)) != FFSPLIT_OK) return s;
+  if (kCtrlBytes + SL.end > ctx->ws_bytes)
+    return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL, "workspace too small for this stack (ffsplit_stack_workspace_size)");
+  char* base = ctx->ws + kCtrlBytes;
+  char* buf[2] = {base + SL.ping, base + SL.pong};
+  const BlobHeader& h0 = ctx->blobs.find(blobs[0])->second.h;
+  const size_t bytes = static_cast<size_t>(T) * h0.d * elem_size(h0.dtype);
+  const void* in = X;
+  int which = 0;
+  if (host) {
+    cudaError_t e = cudaMemcpyAsync(buf[0], X, bytes, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return check_cuda(ctx, e, "cudaMemcpyAsync(X)");
+    in = buf[0];
+    which = 1;
+  }
+  for (int l = 0; l < n_layers; ++l) {
+    const ffsplit_ctx::BlobEntry& ent = ctx->blobs.find(blobs[l])->second;
+    const bool last = l == n_layers - 1;
+    void* out = (last && !host) ? Y : static_cast<void*>(buf[which]);
+    if ((s = run_forward(ctx, ent.h, static_cast<const char*>(blobs[l]), in, T, out, st, ent.hash)) != FFSPLIT_OK) return s;
+    in = out;
+    which ^= 1;
+  }
+  if (host) {
+    cudaError_t e = cudaMemcpyAsync(Y, in, bytes, cudaMemcpyDeviceToHost, st);
+    return check_cuda(ctx, e, "cudaMemcpyAsync(Y)");
+  }
+  return FFSPLIT_OK;
+}
 
 // =====================================================================================
 extern "C" {
@@ -395,27 +467,37 @@ ffsplit_status ffsplit_set_workspace(ffsplit_ctx* ctx, void* dev_ptr, size_t byt
   ctx->ws = static_cast<char*>(dev_ptr);
   ctx->ws_bytes = bytes;
   ctx->tmaps.clear();
+  ctx->score_prep.valid = false;
   return FFSPLIT_OK;
 }
 
 ffsplit_status ffsplit_poll(ffsplit_ctx* ctx, void* stream) {
-  ffsplit_status s = check_ctx(ctx, true);
+  ffsplit_status s = check_ctx(ctx, false);
   if (s != FFSPLIT_OK) return s;
   cudaError_t e = cudaStreamSynchronize(static_cast<cudaStream_t>(stream));
   if (e != cudaSuccess) return check_cuda(ctx, e, "cudaStreamSynchronize");
-  int words[4] = {0, 0, 0, 0};
-  e = cudaMemcpy(words, ctx->ws, sizeof(words), cudaMemcpyDeviceToHost);
-  if (e != cudaSuccess) return check_cuda(ctx, e, "cudaMemcpy(status block)");
-  if (words[0] == 0) return FFSPLIT_OK;
-  e = cudaMemset(ctx->ws, 0, kCtrlBytes);
-  if (e != cudaSuccess) return check_cuda(ctx, e, "cudaMemset(control block)");
-  ctx->err = "device status " + std::to_string(words[0]) + " (detail " + std::to_string(words[1]) + ", kernel " +
-             std::to_string(words[2]) + ")";
-  return static_cast<ffsplit_status>(words[0]);
+  // Two places can hold a device-side condition: the control block of the workspace (if one is set) and
+  // the control block inside the built-in scratch of ffsplit_forward_noalloc (if that has run on this device).
+  char* blocks[2] = {ctx->ws, noalloc_control_block(ctx->device)};
+  const char* where[2] = {"workspace", "built-in scratch"};
+  for (int b = 0; b < 2; ++b) {
+    if (!blocks[b]) continue;
+    int words[4] = {0, 0, 0, 0};
+    e = cudaMemcpy(words, blocks[b], sizeof(words), cudaMemcpyDeviceToHost);
+    if (e != cudaSuccess) return check_cuda(ctx, e, "cudaMemcpy(status block)");
+    if (words[0] == 0) continue;
+    e = cudaMemset(blocks[b], 0, kCtrlBytes);
+    if (e != cudaSuccess) return check_cuda(ctx, e, "cudaMemset(control block)");
+    ctx->err = "device status " + std::to_string(words[0]) + " (detail " + std::to_string(words[1]) + ", kernel " +
+               std::to_string(words[2]) + ", " + where[b] + ")";
+    return static_cast<ffsplit_status>(words[0]);
+  }
+  return FFSPLIT_OK;
 }
 
-ffsplit_status ffsplit_score(ffsplit_ctx* ctx, const ffsplit_shape* shape, const ffsplit_weights* wt, const void* X,
-                             int64_t T, int32_t mode, int32_t accumulate, float* energy, float* scores, void* stream) {
+// Arguments of a scoring call, checked.
+static ffsplit_status check_score_args(ffsplit_ctx* ctx, const ffsplit_shape* shape, const ffsplit_weights* wt,
+                                       const void* X, int64_t T, int32_t mode, const float* energy) {
   ffsplit_status s = check_ctx(ctx, true);
   if (s != FFSPLIT_OK) return s;
   if ((s = check_shape(ctx, shape)) != FFSPLIT_OK) return s;
@@ -424,27 +506,48 @@ ffsplit_status ffsplit_score(ffsplit_ctx* ctx, const ffsplit_shape* shape, const
   if (mode < 0 || mode > 2) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "unknown score mode");
   const bool gated = shape->act == FFSPLIT_SWIGLU;
   if (gated && (!wt->W1u || wt->b1)) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "SwiGLU needs W1u and no b1");
-  if (!aligned16(wt->W1) || !aligned16(wt->W2) || !aligned16(X) || (gated && !aligned16(wt->W1u)))
+  if (!aligned16(wt->W1) || !aligned16(wt->W2) || (gated && !aligned16(wt->W1u)))
     return fail(ctx, FFSPLIT_ERR_ALIGN, "tensors must be 16-byte aligned");
-  const ScoreLayout L = score_layout(*shape, T);
-  if (kCtrlBytes + L.end > ctx->ws_bytes)
-    return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL, "workspace too small for this score call");
-  cudaStream_t st = static_cast<cudaStream_t>(stream);
-  char* base = ctx->ws + kCtrlBytes;
+  return FFSPLIT_OK;
+}
+
+// U^T (K-major for the contraction over d), the fp32 bias and ||V_j||^2 into the scoring region of the
+// workspace, as one batched launch -- unless that region still holds them from an earlier batch of the same
+// accumulation.
+static ffsplit_status score_prepare(ffsplit_ctx* ctx, const ffsplit_shape* shape, const ffsplit_weights* wt,
+                                    const ScoreLayout& L, bool need_w, bool may_reuse, cudaStream_t st) {
+  const bool gated = shape->act == FFSPLIT_SWIGLU;
   const int d = shape->d, m = shape->m, dt = shape->dtype;
-  // U^T (K-major for the contraction over d), fp32 bias, ||V_j||^2: one batched launch
+  ffsplit_ctx::ScorePrep& c = ctx->score_prep;
+  const bool same = c.valid && c.W1 == wt->W1 && c.W1u == wt->W1u && c.b1 == wt->b1 && c.W2 == wt->W2 && c.d == d &&
+                    c.m == m && c.act == shape->act && c.dtype == dt;
+  if (may_reuse && same && (c.has_w || !need_w)) return FFSPLIT_OK;
+  char* base = ctx->ws + kCtrlBytes;
+  ffsplit_status s;
+  c.valid = false;
   prep_begin(ctx);
   if ((s = launch_transpose(ctx, dt, wt->W1, m, d, m, base + L.w1t, d, d, m, nullptr, d, st)) != FFSPLIT_OK) return s;
   if (gated && (s = launch_transpose(ctx, dt, wt->W1u, m, d, m, base + L.w1ut, d, d, m, nullptr, d, st)) != FFSPLIT_OK)
     return s;
+  if (!gated && (s = launch_to_f32(ctx, dt, wt->b1, m, reinterpret_cast<float*>(base + L.b1f), st)) != FFSPLIT_OK) return s;
+  if (need_w && (s = launch_row_energy(ctx, dt, wt->W2, m, d, reinterpret_cast<float*>(base + L.w), st)) != FFSPLIT_OK)
+    return s;
+  if ((s = prep_flush(ctx, dt, st)) != FFSPLIT_OK) return s;
+  c.valid = true; c.has_w = need_w;
+  c.W1 = wt->W1; c.W1u = wt->W1u; c.b1 = wt->b1; c.W2 = wt->W2; c.d = d; c.m = m; c.act = shape->act; c.dtype = dt;
+  return FFSPLIT_OK;
+}
+
+// One batch of calibration tokens (device memory) through the product with the column-energy epilogue.
+static ffsplit_status score_batch(ffsplit_ctx* ctx, const ffsplit_shape* shape, const ScoreLayout& L, const void* X,
+                                  int64_t T, int32_t mode, int32_t accumulate, float* energy, float* scores,
+                                  cudaStream_t st) {
+  const bool gated = shape->act == FFSPLIT_SWIGLU;
+  const int d = shape->d, m = shape->m, dt = shape->dtype;
+  char* base = ctx->ws + kCtrlBytes;
   float* b1f = reinterpret_cast<float*>(base + L.b1f);
   float* w = reinterpret_cast<float*>(base + L.w);
   float* partial = reinterpret_cast<float*>(base + L.partial);
-  if (!gated && (s = launch_to_f32(ctx, dt, wt->b1, m, b1f, st)) != FFSPLIT_OK) return s;
-  if (scores && mode != FFSPLIT_SCORE_ACT_ONLY &&
-      (s = launch_row_energy(ctx, dt, wt->W2, m, d, w, st)) != FFSPLIT_OK)
-    return s;
-  if ((s = prep_flush(ctx, dt, st)) != FFSPLIT_OK) return s;
   GemmArgs g;
   std::memset(&g, 0, sizeof(g));
   g.A0 = X; g.lda0 = d; g.B0 = base + L.w1t; g.ldb0 = d;
@@ -454,8 +557,87 @@ ffsplit_status ffsplit_score(ffsplit_ctx* ctx, const ffsplit_shape* shape, const
   g.epi.col_partial = partial;
   g.epi.n_bias = gated ? 0 : m; g.epi.bias = b1f; g.epi.n_act = m; g.epi.n_split = m;
   g.epi.act = shape->act; g.epi.score_abs = mode == FFSPLIT_SCORE_SUM_NORM;
+  ffsplit_status s;
   if ((s = launch_gemm(ctx, dt, g, st)) != FFSPLIT_OK) return s;
-  return launch_score_finalize(ctx, partial, L.groups, m, w, energy, scores, mode, accumulate, st);
+  // row groups this batch produced (a last, shorter chunk fills fewer than the layout has room for)
+  const int groups = dt == FFSPLIT_BF16 ? 4 * static_cast<int>((T + 127) / 128) : static_cast<int>((T + 63) / 64);
+  return launch_score_finalize(ctx, partial, groups, m, w, energy, scores, mode, accumulate, st);
+}
+
+ffsplit_status ffsplit_score(ffsplit_ctx* ctx, const ffsplit_shape* shape, const ffsplit_weights* wt, const void* X,
+                             int64_t T, int32_t mode, int32_t accumulate, float* energy, float* scores, void* stream) {
+  ffsplit_status s = check_score_args(ctx, shape, wt, X, T, mode, energy);
+  if (s != FFSPLIT_OK) return s;
+  if (!aligned16(X)) return fail(ctx, FFSPLIT_ERR_ALIGN, "tensors must be 16-byte aligned");
+  const ScoreLayout L = score_layout(*shape, T);
+  if (kCtrlBytes + L.end > ctx->ws_bytes)
+    return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL, "workspace too small for this score call");
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const bool need_w = scores && mode != FFSPLIT_SCORE_ACT_ONLY;
+  if ((s = score_prepare(ctx, shape, wt, L, need_w, accumulate != 0, st)) != FFSPLIT_OK) return s;
+  return score_batch(ctx, shape, L, X, T, mode, accumulate, energy, scores, st);
+}
+
+ffsplit_status ffsplit_score_host(ffsplit_ctx* ctx, const ffsplit_shape* shape, const ffsplit_weights* wt,
+                                  const void* X_host, int64_t T, int32_t mode, int32_t accumulate, float* energy,
+                                  float* scores, void* stream) {
+  ffsplit_status s = check_score_args(ctx, shape, wt, X_host, T, mode, energy);
+  if (s != FFSPLIT_OK) return s;
+  // The tokens pass through the workspace in chunks: behind the scoring buffers of a chunk of Tc tokens sits
+  // the chunk itself.  Tc is the largest multiple of 128 (at most T) for which both fit.
+  const size_t es = elem_size(shape->dtype);
+  const size_t row = static_cast<size_t>(shape->d) * es;
+  const size_t room = ctx->ws_bytes - kCtrlBytes;
+  int64_t Tc = T;
+  auto fits = [&](int64_t t) { return score_layout(*shape, t).end + align_up(static_cast<size_t>(t) * row) <= room; };
+  if (!fits(Tc)) {
+    int64_t lo = 0, hi = (T + 127) / 128;   // in units of 128 tokens: fits(128 lo) holds, fits(128 hi) does not
+    if (!fits(128)) return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL, "workspace too small to stage 128 calibration tokens");
+    lo = 1;
+    while (hi - lo > 1) {
+      const int64_t mid = (lo + hi) / 2;
+      if (fits(128 * mid)) lo = mid; else hi = mid;
+    }
+    Tc = 128 * lo;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const ScoreLayout L = score_layout(*shape, Tc);
+  char* stage = ctx->ws + kCtrlBytes + L.end;
+  const bool need_w = scores && mode != FFSPLIT_SCORE_ACT_ONLY;
+  if ((s = score_prepare(ctx, shape, wt, L, need_w, accumulate != 0, st)) != FFSPLIT_OK) return s;
+  const char* src = static_cast<const char*>(X_host);
+  for (int64_t t0 = 0; t0 < T; t0 += Tc) {
+    const int64_t tn = T - t0 < Tc ? T - t0 : Tc;
+    cudaError_t e = cudaMemcpyAsync(stage, src + static_cast<size_t>(t0) * row, static_cast<size_t>(tn) * row,
+                                    cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return check_cuda(ctx, e, "cudaMemcpyAsync(calibration tokens)");
+    const bool last = t0 + tn >= T;
+    if ((s = score_batch(ctx, shape, L, stage, tn, mode, (accumulate || t0 > 0) ? 1 : 0, energy, last ? scores : nullptr,
+                         st)) != FFSPLIT_OK)
+      return s;
+  }
+  return FFSPLIT_OK;
+}
+
+ffsplit_status ffsplit_score_finalize(ffsplit_ctx* ctx, const ffsplit_shape* shape, const void* W2, int32_t mode,
+                                      float* energy, float* scores, void* stream) {
+  ffsplit_status s = check_ctx(ctx, true);
+  if (s != FFSPLIT_OK) return s;
+  if ((s = check_shape(ctx, shape)) != FFSPLIT_OK) return s;
+  if (!energy || !scores) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "NULL tensor");
+  if (mode < 0 || mode > 2) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "unknown score mode");
+  const bool need_w = mode != FFSPLIT_SCORE_ACT_ONLY;
+  if (need_w && !W2) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "W2 is NULL");
+  if (W2 && !aligned16(W2)) return fail(ctx, FFSPLIT_ERR_ALIGN, "tensors must be 16-byte aligned");
+  const int m = shape->m;
+  if (kCtrlBytes + align_up(static_cast<size_t>(m) * 4) > ctx->ws_bytes)
+    return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL, "workspace too small (needs 65536 + 4 m bytes)");
+  ctx->score_prep.valid = false;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  float* w = reinterpret_cast<float*>(ctx->ws + kCtrlBytes);
+  if (need_w && (s = launch_row_energy(ctx, shape->dtype, W2, m, shape->d, w, st)) != FFSPLIT_OK) return s;
+  // no partials to add (groups = 0): the energy passes through unchanged and the scores are formed from it
+  return launch_score_finalize(ctx, w, 0, m, w, energy, scores, mode, 1, st);
 }
 
 ffsplit_status ffsplit_score_activations(ffsplit_ctx* ctx, const ffsplit_shape* shape, const void* H, int64_t T,
@@ -471,6 +653,7 @@ ffsplit_status ffsplit_score_activations(ffsplit_ctx* ctx, const ffsplit_shape* 
   if (need_w && !W2) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "W2 is NULL");
   if (!aligned16(H) || (W2 && !aligned16(W2))) return fail(ctx, FFSPLIT_ERR_ALIGN, "tensors must be 16-byte aligned");
   const int d = shape->d, m = shape->m, dt = shape->dtype;
+  ctx->score_prep.valid = false;
   const int groups = column_energy_groups(T);
   const size_t w_off = 0, part_off = align_up((size_t)m * 4);
   const size_t end = part_off + align_up((size_t)groups * m * 4);
@@ -584,22 +767,41 @@ static ffsplit_status pack_into(ffsplit_ctx* ctx, const ffsplit_shape* shape, co
                             reinterpret_cast<float*>(b + h.off[SEC_B2]), st)) != FFSPLIT_OK)
     return s;
   if ((s = prep_flush(ctx, dt, st)) != FFSPLIT_OK) return s;
-  ctx->blobs[blob] = h;   // the copy below reads this entry, which outlives the call
-  cudaError_t e = cudaMemcpyAsync(blob, &ctx->blobs[blob], sizeof(h), cudaMemcpyHostToDevice, st);
+  ffsplit_ctx::BlobEntry& ent = ctx->blobs[blob];   // replaces whatever was registered at this address
+  ent.h = h;
+  ent.bytes = h.total_bytes;
+  ent.hash = header_hash_host(&h);
+  // the copy below reads this entry, which outlives the call
+  cudaError_t e = cudaMemcpyAsync(blob, &ent.h, sizeof(h), cudaMemcpyHostToDevice, st);
   if (e != cudaSuccess) return check_cuda(ctx, e, "cudaMemcpyAsync(blob header)");
   return FFSPLIT_OK;
 }
 
-ffsplit_status ffsplit_blob_open(ffsplit_ctx* ctx, const void* blob, size_t blob_bytes) {
+ffsplit_status ffsplit_blob_open(ffsplit_ctx* ctx, const void* blob, size_t blob_bytes, void* stream) {
   ffsplit_status s = check_ctx(ctx, false);
   if (s != FFSPLIT_OK) return s;
   if (!blob) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "blob is NULL");
   if (reinterpret_cast<uintptr_t>(blob) % kAlign != 0) return fail(ctx, FFSPLIT_ERR_ALIGN, "blob must be 256-byte aligned");
+  if (blob_bytes < sizeof(BlobHeader)) return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL, "blob_bytes is smaller than a header");
+  ctx->blobs.erase(blob);   // whatever was registered at this address is stale from here on
   BlobHeader h;
-  cudaError_t e = cudaMemcpy(&h, blob, sizeof(h), cudaMemcpyDeviceToHost);
-  if (e != cudaSuccess) return check_cuda(ctx, e, "cudaMemcpy(blob header)");
-  if (!header_valid(h, blob_bytes)) return fail(ctx, FFSPLIT_ERR_BAD_BLOB, "not a packed layer (bad header)");
-  ctx->blobs[blob] = h;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  cudaError_t e = cudaMemcpyAsync(&h, blob, sizeof(h), cudaMemcpyDeviceToHost, st);
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return check_cuda(ctx, e, "cudaMemcpyAsync(blob header)");
+  if (!header_valid(h, blob_bytes)) return fail(ctx, FFSPLIT_ERR_BAD_BLOB, "not a packed layer (bad header, or larger than blob_bytes)");
+  ffsplit_ctx::BlobEntry& ent = ctx->blobs[blob];
+  ent.h = h;
+  ent.bytes = blob_bytes;
+  ent.hash = header_hash_host(&h);
+  return FFSPLIT_OK;
+}
+
+ffsplit_status ffsplit_blob_close(ffsplit_ctx* ctx, const void* blob) {
+  ffsplit_status s = check_ctx(ctx, false);
+  if (s != FFSPLIT_OK) return s;
+  if (ctx->blobs.erase(blob) == 0) return fail(ctx, FFSPLIT_ERR_BAD_BLOB, "blob not known to this context");
+  ctx->tmaps.clear();   // tensor maps are keyed by address too
   return FFSPLIT_OK;
 }
 
@@ -608,8 +810,9 @@ ffsplit_status ffsplit_blob_section(ffsplit_ctx* ctx, const void* blob, int32_t 
   ffsplit_status s = check_ctx(ctx, false);
   if (s != FFSPLIT_OK) return s;
   if (which < 0 || which >= kNumSections) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "unknown section");
-  const BlobHeader* h = find_blob(ctx, blob, &s);
-  if (!h) return s;
+  const ffsplit_ctx::BlobEntry* ent = find_blob(ctx, blob, &s);
+  if (!ent) return s;
+  const BlobHeader* h = &ent->h;
   const SplitDims D = dims_of(*h);
   int64_t R = 0, C = 0, LD = 0;
   switch (which) {
@@ -638,9 +841,9 @@ ffsplit_status ffsplit_forward(ffsplit_ctx* ctx, const void* blob, const void* X
   if (!blob || !X || !Y) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "NULL tensor");
   if (T < 1) return fail(ctx, FFSPLIT_ERR_SHAPE, "T must be >= 1");
   if (!aligned16(X) || !aligned16(Y)) return fail(ctx, FFSPLIT_ERR_ALIGN, "X and Y must be 16-byte aligned");
-  const BlobHeader* h = find_blob(ctx, blob, &s);
-  if (!h) return s;
-  return run_forward(ctx, *h, static_cast<const char*>(blob), X, T, Y, static_cast<cudaStream_t>(stream));
+  const ffsplit_ctx::BlobEntry* ent = find_blob(ctx, blob, &s);
+  if (!ent) return s;
+  return run_forward(ctx, ent->h, static_cast<const char*>(blob), X, T, Y, static_cast<cudaStream_t>(stream), ent->hash);
 }
 
 ffsplit_status ffsplit_forward_dense(ffsplit_ctx* ctx, const ffsplit_shape* shape, const ffsplit_weights* wt,
@@ -667,7 +870,7 @@ ffsplit_status ffsplit_forward_dense(ffsplit_ctx* ctx, const ffsplit_shape* shap
   char* blob = ctx->ws + blob_off;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if ((s = pack_into(ctx, shape, wt, nullptr, shape->m, nullptr, D, h, blob, st)) != FFSPLIT_OK) return s;
-  return run_forward(ctx, h, blob, X, T, Y, st);
+  return run_forward(ctx, h, blob, X, T, Y, st, 0);
 }
 
 ffsplit_status ffsplit_forward_host(ffsplit_ctx* ctx, const void* blob, const void* X_host, int64_t T, void* Y_host,
@@ -676,8 +879,9 @@ ffsplit_status ffsplit_forward_host(ffsplit_ctx* ctx, const void* blob, const vo
   if (s != FFSPLIT_OK) return s;
   if (!blob || !X_host || !Y_host) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "NULL tensor");
   if (T < 1) return fail(ctx, FFSPLIT_ERR_SHAPE, "T must be >= 1");
-  const BlobHeader* h = find_blob(ctx, blob, &s);
-  if (!h) return s;
+  const ffsplit_ctx::BlobEntry* ent = find_blob(ctx, blob, &s);
+  if (!ent) return s;
+  const BlobHeader* h = &ent->h;
   const SplitDims D = dims_of(*h);
   const size_t es = elem_size(h->dtype);
   const FwdLayout L = fwd_layout(D, h->d, h->dtype, h->act, T);
@@ -688,9 +892,38 @@ ffsplit_status ffsplit_forward_host(ffsplit_ctx* ctx, const void* blob, const vo
   const size_t bytes = (size_t)T * h->d * es;
   cudaError_t e = cudaMemcpyAsync(base + L.xs, X_host, bytes, cudaMemcpyHostToDevice, st);
   if (e != cudaSuccess) return check_cuda(ctx, e, "cudaMemcpyAsync(X)");
-  if ((s = run_forward(ctx, *h, static_cast<const char*>(blob), base + L.xs, T, base + L.ys, st)) != FFSPLIT_OK) return s;
+  if ((s = run_forward(ctx, *h, static_cast<const char*>(blob), base + L.xs, T, base + L.ys, st, ent->hash)) != FFSPLIT_OK) return s;
   e = cudaMemcpyAsync(Y_host, base + L.ys, bytes, cudaMemcpyDeviceToHost, st);
   return check_cuda(ctx, e, "cudaMemcpyAsync(Y)");
+}
+
+ffsplit_status ffsplit_forward_stack(ffsplit_ctx* ctx, const void* const* blobs, int32_t n_layers, const void* X,
+                                     int64_t T, void* Y, void* stream) {
+  return forward_stack_impl(ctx, blobs, n_layers, X, T, Y, static_cast<cudaStream_t>(stream), false);
+}
+
+ffsplit_status ffsplit_forward_stack_host(ffsplit_ctx* ctx, const void* const* blobs, int32_t n_layers,
+                                          const void* X_host, int64_t T, void* Y_host, void* stream) {
+  return forward_stack_impl(ctx, blobs, n_layers, X_host, T, Y_host, static_cast<cudaStream_t>(stream), true);
+}
+
+ffsplit_status ffsplit_stack_workspace_size(ffsplit_ctx* ctx, const void* const* blobs, int32_t n_layers, int64_t T,
+                                            size_t* bytes) {
+  ffsplit_status s = check_ctx(ctx, false);
+  if (s != FFSPLIT_OK) return s;
+  if (!blobs || n_layers < 1 || !bytes || T < 1) return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "bad argument");
+  StackLayout SL;
+  if ((s = stack_layout(ctx, blobs, n_layers, T, &SL)) != FFSPLIT_OK) return s;
+  *bytes = kCtrlBytes + SL.end;
+  return FFSPLIT_OK;
+}
+
+ffsplit_status ffsplit_debug_wait_timeout(ffsplit_ctx* ctx, int64_t limit_cycles, void* stream) {
+  ffsplit_status s = check_ctx(ctx, true);
+  if (s != FFSPLIT_OK) return s;
+  if (limit_cycles < 1 || limit_cycles > 100000000)
+    return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "limit_cycles must be in [1, 1e8] (well under a tenth of a second)");
+  return launch_wait_timeout_probe(ctx, limit_cycles, static_cast<cudaStream_t>(stream));
 }
 
 }  // extern "C"

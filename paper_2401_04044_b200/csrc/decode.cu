@@ -8,6 +8,7 @@
 // decode_layer.cu.  It also holds the entry point that runs the same path out of a built-in scratch
 // array, for callers that cannot allocate.
 #include <cstring>
+#include <mutex>
 
 #include "epilogue.cuh"
 #include "internal.h"
@@ -29,7 +30,8 @@ size_t decode_scratch_bytes(int dtype, long long T) {
 
 static ffsplit_status decode_forward_impl(ffsplit_ctx* ctx, const BlobHeader& h, const char* blob, const void* X,
                                           long long T64, void* Y, char* AP, char* Q, char* HL, char* scratch,
-                                          cudaStream_t st, int* tickets, long long scratch_bytes) {
+                                          cudaStream_t st, int* tickets, long long scratch_bytes,
+                                          unsigned long long guard_hash) {
   const int T = static_cast<int>(T64);
   const int d = h.d, k_pad = h.k_pad, r_pad = h.r_pad, ml_pad = h.ml_pad, kp_rp = h.k_pad + h.r_pad;
   const bool gated = h.act == FFSPLIT_SWIGLU;
@@ -47,7 +49,16 @@ static ffsplit_status decode_forward_impl(ffsplit_ctx* ctx, const BlobHeader& h,
                   int N, int K, const Epilogue& epi, float*, double algo_bytes) -> ffsplit_status {
     return decode_layer_add(ctx, &plan, X0, X1, ldx, W0, W1, ldw, N, K, epi, algo_bytes);
   };
-  auto clear = [&]() { std::memset(&e, 0, sizeof(e)); e.act = h.act; };
+  bool guard_pending = guard_hash != 0;   // the first product checks the blob header
+  auto clear = [&]() {
+    std::memset(&e, 0, sizeof(e));
+    e.act = h.act;
+    if (guard_pending) {
+      e.guard = reinterpret_cast<const unsigned long long*>(blob);
+      e.guard_hash = guard_hash;
+      guard_pending = false;
+    }
+  };
   // ---- stage 1
   if (!gated) {
     clear();
@@ -96,8 +107,8 @@ static ffsplit_status decode_forward_impl(ffsplit_ctx* ctx, const BlobHeader& h,
 // Scratch from the caller's workspace, ticket counters from its control block.
 ffsplit_status launch_decode_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* blob, const void* X,
                                      long long T, void* Y, char* AP, char* Q, char* HL, char* scratch,
-                                     cudaStream_t st) {
-  return decode_forward_impl(ctx, h, blob, X, T, Y, AP, Q, HL, scratch, st, nullptr, kDecodeScratchBytes);
+                                     cudaStream_t st, unsigned long long guard_hash) {
+  return decode_forward_impl(ctx, h, blob, X, T, Y, AP, Q, HL, scratch, st, nullptr, kDecodeScratchBytes, guard_hash);
 }
 
 }  // namespace ffsp
@@ -118,10 +129,21 @@ constexpr size_t kNoAllocBytes = kNoAllocTicketBytes + kNoAllocPartialBytes + kN
 // device address and must never be handed to a kernel as a pointer.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocBytes];
 
+// Device address of the array on each device, resolved on first use.  Contexts are independent and may be
+// driven from different host threads: the table is read and written under a lock.
 constexpr int kMaxDevices = 64;
+std::mutex g_noalloc_mutex;
 char* g_noalloc_ptr[kMaxDevices] = {nullptr};
 
 }  // namespace
+
+namespace ffsp {
+char* noalloc_control_block(int device) {
+  if (device < 0 || device >= kMaxDevices) return nullptr;
+  std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+  return g_noalloc_ptr[device];
+}
+}  // namespace ffsp
 
 extern "C" ffsplit_status ffsplit_forward_noalloc(ffsplit_ctx* ctx, const void* blob, const void* X, int64_t T,
                                                   void* Y, void* stream) {
@@ -138,12 +160,10 @@ extern "C" ffsplit_status ffsplit_forward_noalloc(ffsplit_ctx* ctx, const void* 
   if (T < 1 || T > kNoAllocMaxTokens)
     return fail(ctx, FFSPLIT_ERR_SHAPE, "ffsplit_forward_noalloc handles 1..8 tokens per call");
   auto it = ctx->blobs.find(blob);
-  if (it == ctx->blobs.end()) {
-    const ffsplit_status s = ffsplit_blob_open(ctx, blob, 0);
-    if (s != FFSPLIT_OK) return s;
-    it = ctx->blobs.find(blob);
-  }
-  const BlobHeader& h = it->second;
+  if (it == ctx->blobs.end())
+    return fail(ctx, FFSPLIT_ERR_BAD_BLOB,
+                "blob not known to this context: pack it here or register it with ffsplit_blob_open()");
+  const BlobHeader& h = it->second.h;
   if (h.dtype != FFSPLIT_BF16) return fail(ctx, FFSPLIT_ERR_DTYPE, "ffsplit_forward_noalloc handles bf16 layers only");
   // intermediates of one call: [A_H | P], Q, light activations, each 256-byte aligned
   auto up = [](size_t v) { return (v + 255) / 256 * 256; };
@@ -154,21 +174,30 @@ extern "C" ffsplit_status ffsplit_forward_noalloc(ffsplit_ctx* ctx, const void* 
     return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL,
                 "layer too wide for the built-in scratch of ffsplit_forward_noalloc (2 MiB of intermediates)");
   // one-time set-up per device: the device address of the built-in scratch
-  if (!g_noalloc_ptr[dev]) {
-    void* ptr = nullptr;
-    ce = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
-    if (ce != cudaSuccess || !ptr) return check_cuda(ctx, ce != cudaSuccess ? ce : cudaErrorInvalidSymbol, "cudaGetSymbolAddress(scratch)");
-    g_noalloc_ptr[dev] = static_cast<char*>(ptr);
+  char* base = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_ptr[dev]) {
+      void* ptr = nullptr;
+      ce = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
+      if (ce != cudaSuccess || !ptr) return check_cuda(ctx, ce != cudaSuccess ? ce : cudaErrorInvalidSymbol, "cudaGetSymbolAddress(scratch)");
+      ce = cudaMemset(ptr, 0, kNoAllocTicketBytes);   // first use on this device: status words, barrier words and tickets start at zero
+      if (ce != cudaSuccess) return check_cuda(ctx, ce, "cudaMemset(built-in control block)");
+      g_noalloc_ptr[dev] = static_cast<char*>(ptr);
+    }
+    base = g_noalloc_ptr[dev];
   }
-  char* base = g_noalloc_ptr[dev];
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  // the ticket counters must read zero when the kernels start; the rest is overwritten before it is read
-  ce = cudaMemsetAsync(base, 0, kNoAllocTicketBytes, st);
+  // The barrier and ticket words must read zero when the kernels start (a call that gave up may have left
+  // them mid-way); the status words in front of them stay as they are until ffsplit_poll() has reported them.
+  constexpr size_t kStatusWordsBytes = 64;   // words 0..15; the barrier words start at word 16
+  ce = cudaMemsetAsync(base + kStatusWordsBytes, 0, kNoAllocTicketBytes - kStatusWordsBytes, st);
   if (ce != cudaSuccess) return check_cuda(ctx, ce, "cudaMemsetAsync(tickets)");
   char* part = base + kNoAllocTicketBytes;
   char* AP = part + kNoAllocPartialBytes;
   char* Q = AP + ap_b;
   char* HL = Q + q_b;
   return decode_forward_impl(ctx, h, static_cast<const char*>(blob), X, T, Y, AP, Q, HL, part, st,
-                             reinterpret_cast<int*>(base), static_cast<long long>(kNoAllocPartialBytes));
+                             reinterpret_cast<int*>(base), static_cast<long long>(kNoAllocPartialBytes),
+                             it->second.hash);
 }

@@ -253,6 +253,7 @@ __device__ __forceinline__ bool run_product(const Product& pr, const Params& p, 
     if (q == 0) {
       if (first) asm volatile("griddepcontrol.wait;" ::: "memory");
       else if (!grid_barrier(p.ctrl, s_flag)) return false;
+      if (cta == 0 && warp == 0) check_blob_guard(pr.epi, p.ctrl, KID_DECODE);
       if (n == 0) break;
       for (int j = 0; j < LOOK && j < n; ++j) {
         issue_slab(pr, p.T, TP, slabs, step_x, xring + j * slab_bytes, full + j, warp, lane);

@@ -20,6 +20,7 @@ struct Params {
   long long M;
   int N, K;
   Epilogue epi;
+  int* status;
 };
 
 __device__ __forceinline__ void load_slice(const float* __restrict__ src, long long ld, long long row0,
@@ -53,6 +54,7 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(const Params p) {
 
   const int tid = threadIdx.x;
   const int tx = tid & 15, ty = tid >> 4;
+  if (blockIdx.x == 0 && blockIdx.y == 0 && tid < 32) check_blob_guard(p.epi, p.status, KID_GEMM_SIMT);
   const long long row0 = static_cast<long long>(blockIdx.y) * TM;
   const int col0 = blockIdx.x * TN;
 
@@ -140,6 +142,7 @@ ffsplit_status launch_gemm_simt(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_
   p.lda0 = g.lda0; p.ldb0 = g.ldb0; p.lda1 = g.lda1; p.ldb1 = g.ldb1;
   p.M = g.M; p.N = g.N; p.K = g.K;
   p.epi = g.epi;
+  p.status = ctx->status();
   const long long tiles_m = (g.M + simt::TM - 1) / simt::TM;
   if (tiles_m > 65535) return fail(ctx, FFSPLIT_ERR_SHAPE, "fp32 path: more than 65535*64 rows in one call");
   dim3 grid((g.N + simt::TN - 1) / simt::TN, static_cast<unsigned>(tiles_m));

@@ -292,6 +292,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     // other -- either way block number vt uses accumulator buffer vt & 1 in phase (vt >> 1) & 1.
     uint32_t vt = 0;
     bool live = true;
+    if (blockIdx.x == 0 && warp == 2) check_blob_guard(p.epi, p.status, KID_GEMM_TC);
     for (int tile = blockIdx.x; tile < num_tiles && live; tile += gridDim.x)
     for (int mt = 0; mt < MT; ++mt, ++vt) {
       const int m_blk = (tile / p.tiles_n) * MT + mt, n_blk = tile % p.tiles_n;

@@ -30,7 +30,7 @@ constexpr size_t kCtrlBytes = 65536;
 constexpr long long kMaxTicketTiles = (kCtrlBytes - kStatusBytes) / 4;
 
 enum KernelId : int {
-  KID_SELECT = 1, KID_PACK = 2, KID_GEMM_TC = 3, KID_GEMM_SIMT = 4, KID_SCORE = 5, KID_DECODE = 6, KID_FUSED = 7
+  KID_SELECT = 1, KID_PACK = 2, KID_GEMM_TC = 3, KID_GEMM_SIMT = 4, KID_SCORE = 5, KID_DECODE = 6, KID_FUSED = 7, KID_PROBE = 8, KID_QUANT = 9
 };
 
 __device__ __forceinline__ void record_status(int* status, int code, int detail, int kid) {
@@ -65,7 +65,35 @@ struct Epilogue {
   int n_bias;
   int act;        // ffsplit_act
   int score_abs;  // 1: accumulate |v| instead of v^2
+  // Blob guard (first kernel of a forward only, else nullptr): the 256-byte header at `guard` must still
+  // hash to `guard_hash`, the value taken when the blob was packed or opened on this context; a blob whose
+  // bytes were replaced behind the library's back is reported as FFSPLIT_ERR_BAD_BLOB through the status block.
+  const unsigned long long* guard;
+  unsigned long long guard_hash;
 };
+
+// Hash of a 256-byte blob header (32 words of 8 bytes), the same on host and device.
+__host__ __device__ __forceinline__ unsigned long long header_word_mix(unsigned long long w, int i) {
+  unsigned long long v = (w + static_cast<unsigned long long>(i) + 1ull) * 0x9E3779B97F4A7C15ull;
+  return v ^ (v >> 29);
+}
+inline unsigned long long header_hash_host(const void* hdr256) {
+  const unsigned long long* w = static_cast<const unsigned long long*>(hdr256);
+  unsigned long long h = 0;
+  for (int i = 0; i < 32; ++i) h ^= header_word_mix(w[i], i);
+  return h;
+}
+#ifdef __CUDACC__
+// Called by one whole warp.
+__device__ __forceinline__ void check_blob_guard(const Epilogue& e, int* status, int kid) {
+  if (e.guard == nullptr) return;
+  const int lane = threadIdx.x & 31;
+  unsigned long long h = header_word_mix(e.guard[lane], lane);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) h ^= __shfl_xor_sync(0xffffffffu, h, o);
+  if (lane == 0 && h != e.guard_hash) record_status(status, FFSPLIT_ERR_BAD_BLOB, 0, kid);
+}
+#endif
 
 struct GemmArgs {
   const void* A0;   // [M, K], leading dimension lda0
@@ -151,7 +179,8 @@ struct ffsplit_ctx {
   size_t ws_bytes = 0;
   long long launches = 0;
   std::string err;
-  std::unordered_map<const void*, ffsp::BlobHeader> blobs;
+  struct BlobEntry { ffsp::BlobHeader h; size_t bytes; unsigned long long hash; };
+  std::unordered_map<const void*, BlobEntry> blobs;   // blobs packed or opened on this context, by address
   std::unordered_map<ffsp::TmapKey, CUtensorMap, ffsp::TmapKeyHash> tmaps;
   void* encode_fn = nullptr;  // cuTensorMapEncodeTiled
   struct ProfRec { int cls; cudaEvent_t a, b; double work; };
@@ -167,6 +196,14 @@ struct ffsplit_ctx {
   int gemm_two_m = 1;          // tensor-core GEMM: 256-row tiles where they pay (FFSPLIT_GEMM_TWO_M=0: never, 2: wherever allowed)
   int decode_one_launch = 0;   // few-token forward: 1 = all products in one cooperative launch (FFSPLIT_DECODE_LAYER=1), 0 = one launch per product
   int use_fused = -1;  // -1: not decided yet (environment FFSPLIT_NO_FUSED=1 turns the fused kernel off)
+  // What the scoring region of the workspace holds from the last ffsplit_score() call: U^T, the fp32 bias
+  // and ||V_j||^2 of these weights.  A later batch of the same accumulation (accumulate = 1, same pointers
+  // and shape) reuses them; any other call that writes the workspace clears `valid`.
+  struct ScorePrep {
+    bool valid = false, has_w = false;
+    const void *W1 = nullptr, *W1u = nullptr, *b1 = nullptr, *W2 = nullptr;
+    int d = 0, m = 0, act = 0, dtype = 0;
+  } score_prep;
 };
 
 namespace ffsp {
@@ -264,6 +301,7 @@ ffsplit_status launch_fused_light(ffsplit_ctx* ctx, const void* Q, long long ldq
                                   const void* A2T, const float* b1l, int r_pad, int ml_pad, int act, void* P,
                                   long long ldp, char* scratch, int* tickets, double algo_flops,
                                   cudaStream_t st);
+ffsplit_status launch_wait_timeout_probe(ffsplit_ctx* ctx, long long limit_cycles, cudaStream_t st);
 ffsplit_status launch_to_f32(ffsplit_ctx* ctx, int dtype, const void* in, int n, float* out, cudaStream_t st);
 
 }  // namespace ffsp

@@ -2,8 +2,47 @@
 // transpose kernels of the pack step.
 #include "epilogue.cuh"
 #include "internal.h"
+#include "ptx.cuh"
 
 namespace ffsp {
+
+// ============================================================================
+// Self-test of the bounded wait every kernel of the library is built on: one CTA of two warps.  Warp 0
+// waits, through the same routine the tensor-core and few-token kernels use, on an mbarrier that nothing
+// will ever signal, with a limit of `limit_cycles`; the wait runs out, raises the CTA's abort flag and
+// returns; warp 1, waiting on a second unsignalled barrier, sees the flag and leaves too (the way the
+// other roles of a kernel leave when one of them gives up).  The kernel then records FFSPLIT_ERR_TIMEOUT
+// in the status block and exits normally: no trap, no fault, and the context stays usable.
+// ============================================================================
+__global__ void __launch_bounds__(64) wait_timeout_probe_kernel(long long limit_cycles, int* status) {
+  __shared__ __align__(8) uint64_t bars[2];
+  __shared__ int abort_flag;
+  __shared__ int gave_up[2];
+  if (threadIdx.x == 0) {
+    ptx::mbar_init(&bars[0], 1);
+    ptx::mbar_init(&bars[1], 1);
+    ptx::mbar_fence_init();
+    abort_flag = 0;
+    gave_up[0] = gave_up[1] = 0;
+  }
+  __syncthreads();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (lane == 0) {
+    // warp 0: the short limit; warp 1: the library's normal limit (about a second), cut short by the flag
+    const bool ok = warp == 0 ? ptx::mbar_wait_limit(&bars[0], 0, &abort_flag, limit_cycles)
+                              : ptx::mbar_wait(&bars[1], 0, &abort_flag);
+    gave_up[warp] = ok ? 0 : 1;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0 && abort_flag)
+    record_status(status, FFSPLIT_ERR_TIMEOUT, gave_up[0] + 2 * gave_up[1], KID_PROBE);
+}
+
+ffsplit_status launch_wait_timeout_probe(ffsplit_ctx* ctx, long long limit_cycles, cudaStream_t st) {
+  wait_timeout_probe_kernel<<<1, 64, 0, st>>>(limit_cycles, ctx->status());
+  ctx->launches++;
+  return check_cuda(ctx, cudaGetLastError(), "wait_timeout_probe_kernel launch");
+}
 
 // ============================================================================
 // Top-k selection (Section 4.1: the neurons with the highest score are the heavy

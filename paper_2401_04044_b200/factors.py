@@ -10,8 +10,9 @@ import torch
 
 def truncated_factors(W: torch.Tensor, r: int, out_dtype: torch.dtype):
     """W [p, q] -> A [p, r], B [r, q] with A @ B the best rank-r approximation,
-    singular values split evenly between the factors."""
-    Wf = W.to(torch.float64 if W.device.type == "cpu" else torch.float32)
+    singular values split evenly between the factors.  The decomposition is taken in
+    float64 on whichever device holds W; only the factors are rounded to out_dtype."""
+    Wf = W.to(torch.float64)
     U, S, Vh = torch.linalg.svd(Wf, full_matrices=False)
     root = S[:r].sqrt()
     A = (U[:, :r] * root[None, :]).to(out_dtype).contiguous()

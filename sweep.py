@@ -1,7 +1,7 @@
 """Throughput sweep over the synthetic configurations: split vs dense forward per
 FFN layer (prefill and few-token sizes), scoring, and model size.
 
-    python -m paper_2401_04044_b200.sweep --config 5 --tokens 1 32 4096 --out gpurun_out/sweep_cfg5.jsonl
+    python sweep.py --config 5 --tokens 1 32 4096 --out sweep_cfg5.jsonl
 
 One JSON line per point: tokens/s per layer and per stack, achieved fraction of
 the roofline (the slower of FLOPs at the bf16 tensor peak and bytes at the HBM
@@ -21,7 +21,7 @@ import sys
 
 import torch
 
-ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 

@@ -455,6 +455,44 @@ def test_degenerate_splits(ctx, dt, act):
     assert orc.rel_frobenius(f64(Yf), dense_ref) < loose
 
 
+def test_split_output_invariant_under_neuron_permutation_bf16(ctx):
+    """Eq. 1: the FFN is a sum over neurons, so relabelling the neurons (columns of W1, entries of b1, rows
+    of W2, and the heavy set with them) must not change a SPLIT layer's output beyond summation order: the
+    heavy slices are gathered in a different order and the light factors are those of the permuted slices."""
+    cfg = custom_config(128, 640, 40, 32, act="gelu_erf", dtype="bf16")
+    L = make_layer(cfg, 5)
+    G = GpuLayer(ctx, L)
+    T = 200
+    G.reserve(T, 0, cfg.k, cfg.r)
+    X = L.tokens(T)
+    heavy = L.planted
+    fac = oracle_factors(L, heavy.numpy(), cfg.r)
+    blob, _ = G.pack(heavy, fac)
+    Y = G.forward(blob, X)
+    perm = torch.randperm(cfg.m, generator=torch.Generator().manual_seed(2))     # new position p holds old neuron perm[p]
+    inv = torch.empty_like(perm)
+    inv[perm] = torch.arange(cfg.m)
+    L2 = make_layer(cfg, 5)
+    L2.W1, L2.b1, L2.W2 = L.W1[:, perm].contiguous(), L.b1[perm].contiguous(), L.W2[perm, :].contiguous()
+    heavy2 = torch.sort(inv[heavy]).values
+    # the light neurons of the permuted layer, ascending, and the same factors with their neuron axis reordered to match
+    mask = torch.ones(cfg.m, dtype=torch.bool)
+    mask[heavy] = False
+    light_old = torch.nonzero(mask).flatten()                 # ascending old indices: the order fac's neuron axis uses
+    mask2 = torch.ones(cfg.m, dtype=torch.bool)
+    mask2[heavy2] = False
+    light_new = torch.nonzero(mask2).flatten()
+    pos = {int(o): i for i, o in enumerate(light_old)}
+    reorder = torch.tensor([pos[int(perm[p])] for p in light_new])
+    fac2 = {"A1": fac["A1"], "B1": fac["B1"][:, reorder].contiguous(), "A2": fac["A2"][reorder, :].contiguous(),
+            "B2": fac["B2"]}
+    G2 = GpuLayer(ctx, L2)
+    blob2, _ = G2.pack(heavy2, fac2)
+    Y2 = G2.forward(blob2, X)
+    assert_close(Y2, oracle_split(L2, heavy2.numpy(), fac2, X), "bf16", "permuted split layer vs oracle")
+    assert orc.rel_frobenius(f64(Y2), f64(Y)) < 4e-3       # two bf16 roundings of the same values, summed in another order
+
+
 def test_output_invariant_under_neuron_permutation(ctx):
     cfg = custom_config(64, 256, 16, 0, dtype="f32")
     L = make_layer(cfg, 5)
@@ -531,3 +569,148 @@ def test_bf16_configs_one_layer_end_to_end(ctx, cid, layer, T):
     blobd, _ = G.pack(torch.arange(cfg.m), None)
     dense_ref = orc.dense_ffn(f64(X), f64(L.W1), f64(L.b1), f64(L.W2), f64(L.b2), cfg.act)
     assert_close(G.forward(blobd, X), dense_ref, "bf16", f"config {cid} dense")
+
+
+# ------------------------------------------------------------------ registry, stacks, host buffers, bounded waits
+def test_blob_registry_and_changed_bytes(ctx):
+    """A forward accepts only blobs packed or opened on its context; a registration describes the bytes that were
+    there when it was made.  Overwriting a registered buffer with a blob of another (k, r) and re-opening it gives
+    the new layer's output; forgetting to re-open is caught by the header check inside the first kernel
+    (FFSPLIT_ERR_BAD_BLOB at the next poll) -- nothing faults either way."""
+    from paper_2401_04044_b200 import Context, FFSplitError
+    cfg_a = custom_config(128, 512, 26, 32, dtype="bf16")
+    cfg_b = custom_config(128, 512, 60, 16, dtype="bf16")
+    La, Lb = make_layer(cfg_a, 1), make_layer(cfg_b, 2)
+    Ga, Gb = GpuLayer(ctx, La), GpuLayer(ctx, Lb)
+    for T in (40, 300):
+        Ga.reserve(T, 0, cfg_a.k, cfg_a.r)
+        Gb.reserve(T, 0, cfg_b.k, cfg_b.r)
+    fa = oracle_factors(La, La.planted.numpy(), cfg_a.r)
+    fb = oracle_factors(Lb, Lb.planted.numpy(), cfg_b.r)
+    blob_a, _ = Ga.pack(La.planted, fa)
+    blob_b, _ = Gb.pack(Lb.planted, fb)
+    n = max(blob_a.numel(), blob_b.numel())
+    buf = torch.zeros(n, dtype=torch.uint8, device="cuda")
+    for T in (40, 300):                                     # few-token kernel and tensor-core kernel
+        X = La.tokens(T)
+        Xd = X.cuda()
+        Y = torch.empty_like(Xd)
+        ctx.blob_close(buf) if T == 300 else None
+        with pytest.raises(FFSplitError) as e:             # never registered here
+            ctx.forward(buf, Xd, Y)
+        assert e.value.code == 7
+        buf[:blob_a.numel()].copy_(blob_a)
+        ctx.blob_open(buf)
+        ctx.forward(buf, Xd, Y)
+        ctx.poll()
+        assert torch.equal(Y, Ga.forward(blob_a, X))
+        buf[:blob_b.numel()].copy_(blob_b)                  # another layer now lives at this address
+        ctx.forward(buf, Xd, Y)                             # stale registration: reported, not trusted
+        with pytest.raises(FFSplitError) as e:
+            ctx.poll()
+        assert e.value.code == 7
+        ctx.blob_open(buf)                                  # re-registered: the new layer's output
+        ctx.forward(buf, Xd, Y)
+        ctx.poll()
+        assert_close(Y, oracle_split(Lb, Lb.planted.numpy(), fb, X), "bf16", "re-opened blob")
+    # a header that claims more bytes than the buffer has is refused
+    small = buf[:1024]
+    with pytest.raises(FFSplitError) as e:
+        ctx.blob_open(small)
+    assert e.value.code == 7
+    ctx.blob_close(buf)
+    with pytest.raises(FFSplitError) as e:
+        ctx.blob_close(buf)
+    assert e.value.code == 7
+
+
+def test_bounded_wait_runs_out_and_reports_timeout(ctx):
+    """A wait that nothing will ever satisfy gives up after its limit, the kernel returns, and the condition
+    comes back through ffsplit_poll(); the context keeps working afterwards."""
+    from paper_2401_04044_b200 import FFSplitError
+    ctx.poll()
+    ctx.debug_wait_timeout(200000)          # 2e5 SM clocks: about a tenth of a millisecond
+    with pytest.raises(FFSplitError) as e:
+        ctx.poll()
+    assert e.value.code == 10 and "detail 3" in str(e.value)   # both waiting warps gave up
+    ctx.poll()                               # cleared
+    s = random_scores(1000, seed=1).cuda()
+    heavy = torch.zeros(10, dtype=torch.int32, device="cuda")
+    ctx.select(s, 10, heavy, None)
+    ctx.poll()
+    assert np.array_equal(heavy.cpu().numpy(), orc.select_heavy(s.cpu().numpy(), 10)[0])
+
+
+@pytest.mark.parametrize("dt,act,d,m,T", [("bf16", "gelu_erf", 128, 520, 1000), ("bf16", "swiglu", 64, 256, 300),
+                                         ("f32", "gelu_erf", 64, 200, 333)])
+def test_score_from_host_buffers_and_finalize(ctx, dt, act, d, m, T):
+    """ffsplit_score_host stages the calibration tokens through the workspace in chunks (here the workspace
+    leaves room for 256 tokens at a time, so several chunks and a ragged last one) and must give the scores of
+    one device-resident call up to summation order; ffsplit_score_finalize forms the same scores from an energy
+    vector accumulated with scores = NULL."""
+    cfg = custom_config(d, m, max(1, m // 20), 16, act=act, dtype=dt)
+    L = make_layer(cfg, 4)
+    G = GpuLayer(ctx, L)
+    X = L.tokens(T)
+    es = 2 if dt == "bf16" else 4
+    ws_one = ctx.workspace_size(G.shape, 0, T, 0, 0)
+    G.reserve(0, T, 0, 0)
+    energy, scores = G.score(X)
+    _, _, s_ref = orc.neuron_scores(f64(X), f64(L.W1), f64(L.b1), f64(L.W2), act, orc.SCORE_EQ3, f64(L.W1u))
+    rt = SCORE_RTOL[dt]
+    from paper_2401_04044_b200 import Context
+    c2 = Context(0)
+    try:
+        c2.set_workspace(torch.empty(c2.workspace_size(G.shape, 0, 256, 0, 0) + 256 * d * es + 4096, dtype=torch.uint8,
+                                     device="cuda"))
+        Xh = X.pin_memory()
+        e2 = torch.empty_like(energy)
+        s2 = torch.empty_like(scores)
+        c2.score_host(G.shape, G.W1, G.b1, G.W2, Xh, e2, s2, W1u=G.W1u)
+        c2.poll()
+        assert np.allclose(f64(s2), s_ref, rtol=rt, atol=rt * s_ref.max() * 1e-3)
+        assert np.allclose(f64(e2), f64(energy), rtol=1e-5)
+        # energy only, then the scores from it
+        e3 = torch.empty_like(energy)
+        s3 = torch.empty_like(scores)
+        c2.score_host(G.shape, G.W1, G.b1, G.W2, Xh, e3, None, W1u=G.W1u)
+        c2.score_finalize(G.shape, G.W2, e3, s3)
+        c2.poll()
+        assert torch.equal(e3, e2) and torch.equal(s3, s2)
+    finally:
+        c2.close()
+    assert ws_one > 0
+
+
+@pytest.mark.parametrize("T", [5, 300])
+def test_forward_stack_device_and_host(ctx, T):
+    """Three layers with different splits, layer l reading layer l-1's output: the stack call equals the layers
+    called one by one (bit for bit), from device and from host buffers; each layer is compared with the oracle on
+    the exact input it consumed."""
+    d = 128
+    cfgs = [custom_config(d, 512, 26, 32, dtype="bf16"), custom_config(d, 384, 40, 16, dtype="bf16"),
+            custom_config(d, 640, 10, 48, act="gelu_tanh", dtype="bf16")]
+    layers, blobs, facs = [], [], []
+    for i, cfg in enumerate(cfgs):
+        L = make_layer(cfg, 20 + i)
+        G = GpuLayer(ctx, L)
+        G.reserve(T, 0, cfg.k, cfg.r)
+        fac = oracle_factors(L, L.planted.numpy(), cfg.r)
+        blob, _ = G.pack(L.planted, fac)
+        layers.append((L, G)); blobs.append(blob); facs.append(fac)
+    ctx.ensure_workspace(ctx.stack_workspace_size(blobs, T))
+    X = layers[0][0].tokens(T)
+    x = X
+    for (L, G), blob, fac in zip(layers, blobs, facs):
+        y = G.forward(blob, x)
+        assert_close(y, oracle_split(L, L.planted.numpy(), fac, x), "bf16", "stack layer")
+        x = y.cpu()
+    Xd = X.cuda()
+    Y = torch.empty_like(Xd)
+    ctx.forward_stack(blobs, Xd, Y)
+    ctx.poll()
+    assert torch.equal(Y.cpu(), x)
+    Xh, Yh = X.pin_memory(), torch.empty_like(X).pin_memory()
+    ctx.forward_stack_host(blobs, Xh, Yh)
+    ctx.poll()
+    assert torch.equal(Yh, x)
