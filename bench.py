@@ -1,19 +1,18 @@
 #!/usr/bin/env python
 """Benchmark of the split-FFN hot path (FFSplit, arXiv 2401.04044) on B200.
 
-Workload (N = 1): the BERT-base-shaped stack -- 12 GELU FFN layers, d = 768,
-m = 3072, bf16, heavy k = 154, light rank r = 192, 4096 calibration tokens per
-layer, prefill batch 32 x 128 = 4096 tokens.  One step is one pass of the whole
-path over that batch: per layer score -> select -> pack, then the 12-layer split
-forward.  `value` is forward tokens per second of that whole step; the phases
-(forward only, dense comparator, calibration) are reported beside it.
+Workload (N = 1): the OPT-13B-shaped stack -- 40 GELU FFN layers, d = 5120, m = 20480, bf16, at the
+sweep's centre point: 5 % heavy neurons (k = 1024), light rank r = 512, 65536 calibration tokens per
+layer, prefill batch of 4096 tokens.  One step is one pass of the whole path over that batch: per layer
+score -> select -> pack, then the 40-layer split forward.  `value` is forward tokens per second of that
+whole step; the phases (forward only at 4096 / 32 / 1 tokens, the dense comparator through the same
+kernels, calibration) and the smaller configurations are reported beside it.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
-Under torchrun every rank runs the same per-GPU workload (weak scaling, no
-data-path collective: the path is token-parallel with replicated weights).
-`--impl reference` times the CPU oracle (oracle/) on the host cores on a bounded
-sample of the same workload.
+Under torchrun every rank runs the same per-GPU workload (weak scaling, no data-path collective: the
+path is token-parallel with replicated weights).  `--impl reference` times the CPU oracle (oracle/) on
+the host cores on a bounded sample of the same workload.
 """
 from __future__ import annotations
 
@@ -31,7 +30,10 @@ sys.path.insert(0, ROOT)
 
 METRIC = "split-FFN tokens/s (prefill, decode) and % of roofline vs dense FFN"
 UNIT = "tokens/s"
-CFG_ID = 2
+HEAVY_PERCENT, RANK = 5, 512          # the point of configs[4]'s sweep that the step runs at
+WORKLOAD = ("configs[4]: OPT-13B-shaped stack, 40 GELU FFN layers, d=5120 m=20480, 5% heavy (k=1024), light rank "
+            "r=512, 65536 calibration tokens/layer, prefill 4096 tokens; step = score+select+pack per layer, then the "
+            "40-layer split forward")
 
 
 def load_peaks():
@@ -39,7 +41,7 @@ def load_peaks():
     if os.path.exists(p):
         j = json.load(open(p))
         return {"hbm_gbs": j["hbm_gbs"], "bf16_tflops": j["bf16_tflops"],
-                "bf16_tflops_sustained": j.get("bf16_tflops_sustained"), "source": "measured"}
+                "bf16_tflops_sustained": j.get("bf16_tflops_sustained") or j["bf16_tflops"], "source": "measured"}
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
@@ -91,31 +93,44 @@ class ClockSampler:
 
 
 # --------------------------------------------------------------------------------------
+def seeded_factors(cfg, device, seed):
+    """Rank-r light factors for the timed runs: seeded N(0, 0.02^2) matrices of the right shapes.  The work of
+    every kernel depends on the shapes only; parity tests use true SVD factors (the SVD of one 5120 x 19456
+    slice in float64 takes minutes and is the off-path step between select and pack)."""
+    import torch
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+    d, ml, r, dt = cfg.d, cfg.m - cfg.k, cfg.r, cfg.torch_dtype
+    mk = lambda *s: (torch.randn(*s, generator=g, device=device, dtype=torch.float32) * 0.02).to(dt)
+    f = {"A1": mk(d, r), "B1": mk(r, ml), "A2": mk(ml, r), "B2": mk(r, d)}
+    if cfg.act == "swiglu":
+        f["A1u"], f["B1u"] = mk(d, r), mk(r, ml)
+    return f
+
+
 class StackWorkload:
     """Device-resident synthetic stack plus everything one step touches."""
 
-    def __init__(self, cfg, ctx, layers, T, device, cal_lanes=1):
+    def __init__(self, cfg, ctx, layers, T, device, lanes=2, dense=True):
         import torch
         from ffsplit_synth import make_layer
-        from paper_2401_04044_b200 import make_shape
-        from paper_2401_04044_b200.factors import light_factors
-        self.cfg, self.ctx, self.T, self.n_layers = cfg, ctx, T, layers
+        from paper_2401_04044_b200 import Context, make_shape
+        self.cfg, self.ctx, self.T, self.n_layers, self.device = cfg, ctx, T, layers, device
         self.shape = make_shape(cfg.d, cfg.m, cfg.act, cfg.torch_dtype)
-        ws = max(ctx.workspace_size(self.shape, T, cfg.t_cal, cfg.k, cfg.r),
-                 ctx.workspace_size(self.shape, T, 0, cfg.m, 0))
-        ctx.ensure_workspace(ws)
-        # The calibrations of different layers do not depend on one another, and most of their kernels
-        # (top-k in one CTA, the small preparation jobs) leave the GPU nearly idle: they are issued round
-        # robin on `cal_lanes` streams, each with a library context (workspace, tickets) of its own.
-        from paper_2401_04044_b200 import Context
-        self.lanes = [(ctx, None)]   # lane 0: the calling stream (forward chain; everything when alone)
-        for _ in range(cal_lanes if cal_lanes > 1 else 0):
-            c = Context(ctx.device if hasattr(ctx, "device") else 0)
-            c.ensure_workspace(c.workspace_size(self.shape, T, cfg.t_cal, cfg.k, cfg.r))
+        es = 2
+        cal_ws = ctx.workspace_size(self.shape, 0, cfg.t_cal, 0, 0) + cfg.t_cal * cfg.d * es + 4096
+        # The calibrations of different layers do not depend on one another: they are issued round robin on
+        # `lanes` streams, each with a library context (workspace, control block) of its own, so that in the
+        # end-to-end run one lane's host-to-device copy runs under the other lane's scoring product.
+        self.lanes = []
+        for _ in range(max(1, lanes)):
+            c = Context(ctx.device)
+            c.ensure_workspace(cal_ws)
             self.lanes.append((c, torch.cuda.Stream(device=device)))
-        self.layers = []
         padded, self.logical_bytes = ctx.pack_size(self.shape, cfg.k, cfg.r)
         padded_dense, self.logical_bytes_dense = ctx.pack_size(self.shape, cfg.m, 0)
+        self.layers = []
+        all_idx = torch.arange(cfg.m, dtype=torch.int32, device=device)
         for l in range(layers):
             L = make_layer(cfg, l, device=device)
             e = {"L": L, "Xcal": L.tokens(cfg.t_cal)}
@@ -124,129 +139,100 @@ class StackWorkload:
             e["heavy"] = torch.empty(cfg.k, dtype=torch.int32, device=device)
             e["light"] = torch.empty(cfg.m - cfg.k, dtype=torch.int32, device=device)
             e["blob"] = torch.empty(padded, dtype=torch.uint8, device=device)
-            e["blob_dense"] = torch.empty(padded_dense, dtype=torch.uint8, device=device)
-            e["Y"] = torch.empty(T, cfg.d, dtype=cfg.torch_dtype, device=device)
+            e["factors"] = seeded_factors(cfg, device, 1000 + l)
             self.layers.append(e)
         self.X = self.layers[0]["L"].tokens(T)
-        # set-up (untimed): find each layer's heavy set once, factor its light slices (host-side
-        # helper of the step between select and pack), build the dense comparator blobs
+        self.Y = torch.empty_like(self.X)
+        # set-up (untimed): one calibration of every layer (each lane's context packs the blobs it will re-pack in
+        # the timed steps; the forward context registers them), the dense comparator blobs
+        for i, e in enumerate(self.layers):
+            c, s = self.lanes[i % len(self.lanes)]
+            with torch.cuda.stream(s):
+                self.calibrate_layer(e, c)
+        torch.cuda.synchronize()
+        self.poll()
         for e in self.layers:
-            self.calibrate_layer(e, pack=False)
-        ctx.poll()
-        all_idx = torch.arange(cfg.m, dtype=torch.int32, device=device)
-        for e in self.layers:
-            L = e["L"]
+            ctx.blob_open(e["blob"])
             e["heavy_setup"] = e["heavy"].clone()
-            e["factors"] = light_factors(L.W1, L.W2, e["light"], cfg.r, L.W1u)
-            ctx.pack(self.shape, L.W1, L.b1, L.W2, L.b2, all_idx, cfg.m, None, e["blob_dense"], W1u=L.W1u)
-        ctx.poll()
+        self.blobs = [e["blob"] for e in self.layers]
+        self.blobs_dense = []
+        if dense:
+            ctx.ensure_workspace(ctx.workspace_size(self.shape, 8, 0, cfg.m, 0))
+            for e in self.layers:
+                L = e["L"]
+                bd = torch.empty(padded_dense, dtype=torch.uint8, device=device)
+                ctx.pack(self.shape, L.W1, L.b1, L.W2, L.b2, all_idx, cfg.m, None, bd, W1u=L.W1u)
+                self.blobs_dense.append(bd)
+            ctx.poll()
+        need = max(ctx.stack_workspace_size(self.blobs, t) for t in (T, 32, 1))
+        if dense:
+            need = max(need, max(ctx.stack_workspace_size(self.blobs_dense, t) for t in (T, 32, 1)))
+        ctx.ensure_workspace(need)
 
-    def calibrate_layer(self, e, pack=True, ctx=None):
-        L, cfg, ctx = e["L"], self.cfg, ctx or self.ctx
-        ctx.score(self.shape, L.W1, L.b1, L.W2, e["Xcal"], e["energy"], e["scores"], W1u=L.W1u)
-        ctx.select(e["scores"], cfg.k, e["heavy"], e["light"])
-        if pack:
-            ctx.pack(self.shape, L.W1, L.b1, L.W2, L.b2, e["heavy"], cfg.k, e["factors"], e["blob"], W1u=L.W1u)
+    # -- calibration: score + select + pack of one layer on context c (current stream)
+    def calibrate_layer(self, e, c, x_host=None):
+        L, cfg = e["L"], self.cfg
+        if x_host is None:
+            c.score(self.shape, L.W1, L.b1, L.W2, e["Xcal"], e["energy"], e["scores"], W1u=L.W1u)
+        else:
+            c.score_host(self.shape, L.W1, L.b1, L.W2, x_host, e["energy"], e["scores"], W1u=L.W1u)
+        c.select(e["scores"], cfg.k, e["heavy"], e["light"])
+        c.pack(self.shape, L.W1, L.b1, L.W2, L.b2, e["heavy"], cfg.k, e["factors"], e["blob"], W1u=L.W1u)
 
-    def calibrate(self, events=None, before=None):
-        """Score, select and pack every layer.  With several lanes the layers go round robin over the
-        lanes' streams; `events`, if given, receives one event per layer, recorded behind its pack;
-        `before(i)`, if given, is issued on the layer's stream ahead of its calibration (input copies)."""
+    def calibrate(self, x_hosts=None):
+        """Score, select and pack every layer, round robin over the lanes' streams; the calling stream waits for
+        all of them."""
         import torch
-        if len(self.lanes) == 1:
-            for i, e in enumerate(self.layers):
-                if before is not None:
-                    before(i)
-                self.calibrate_layer(e)
-            return
         main = torch.cuda.current_stream()
         fork = torch.cuda.Event()
         fork.record(main)
-        side = self.lanes[1:]
-        for _, s in side:
+        for _, s in self.lanes:
             s.wait_event(fork)
         for i, e in enumerate(self.layers):
-            c, s = side[i % len(side)]
+            c, s = self.lanes[i % len(self.lanes)]
             with torch.cuda.stream(s):
-                if before is not None:
-                    before(i)
-                self.calibrate_layer(e, ctx=c)
-                if events is not None:
-                    ev = torch.cuda.Event()
-                    ev.record(s)
-                    events.append(ev)
-        if events is None:
-            for _, s in side:
-                join = torch.cuda.Event()
-                join.record(s)
-                main.wait_event(join)
+                self.calibrate_layer(e, c, None if x_hosts is None else x_hosts[i % len(x_hosts)])
+        for _, s in self.lanes:
+            join = torch.cuda.Event()
+            join.record(s)
+            main.wait_event(join)
 
-    def launch_count(self):
-        return sum(c.launch_count() for c, _ in self.lanes)
-
-    def poll(self):
-        for c, _ in self.lanes:
-            c.poll()
-
-    def forward(self, x=None, dense=False):
-        x = self.X if x is None else x
+    def calibrate_serial(self):
+        c = self.lanes[0][0]
         for e in self.layers:
-            self.ctx.forward(e["blob_dense"] if dense else e["blob"], x, e["Y"])
-            x = e["Y"]
-        return x
+            self.calibrate_layer(e, c)
 
-    def step(self, x=None, before=None):
-        """One pass of the whole path.  With several lanes, layer l's forward (on the calling stream) waits
-        only for layer l's pack, so the forward chain runs under the calibrations of the later layers."""
-        import torch
-        if len(self.lanes) == 1:
-            self.calibrate(before=before)
-            return self.forward(x)
-        events = []
-        self.calibrate(events, before)
-        main = torch.cuda.current_stream()
-        x = self.X if x is None else x
-        for e, ev in zip(self.layers, events):
-            main.wait_event(ev)
-            self.ctx.forward(e["blob"], x, e["Y"])
-            x = e["Y"]
-        return x
+    def forward(self, dense=False, x=None, y=None):
+        self.ctx.forward_stack(self.blobs_dense if dense else self.blobs, self.X if x is None else x,
+                               self.Y if y is None else y)
+
+    def step(self):
+        self.calibrate()
+        self.forward()
 
     def step_serial(self):
-        """The same work on one stream and one context: what the per-kernel profile is taken on."""
-        for e in self.layers:
-            self.calibrate_layer(e)
-        return self.forward()
+        """The same work on one stream: what the per-kernel profile is taken on."""
+        self.calibrate_serial()
+        self.forward()
+
+    def step_host(self, x_hosts, X_host, Y_host):
+        """The step through the host-buffer entry points of the C ABI: calibration tokens, X and Y in pinned host
+        memory, every copy inside the call that consumes or produces it."""
+        self.calibrate(x_hosts)
+        self.ctx.forward_stack_host(self.blobs, X_host, Y_host)
+
+    def launch_count(self):
+        return self.ctx.launch_count() + sum(c.launch_count() for c, _ in self.lanes)
+
+    def poll(self):
+        self.ctx.poll()
+        for c, _ in self.lanes:
+            c.poll()
 
     def check_selection_stable(self):
         import torch
         for e in self.layers:
             assert torch.equal(e["heavy"], e["heavy_setup"]), "selection changed between set-up and the timed steps"
-
-
-# DRAM traffic of the tensor-core kernels (gemm_tc_kernel and fused_light_kernel: the launches the roofline
-# object covers), average per launch over one step, from an ncu capture of
-#   python bench.py --only step --steps 1 --warmup 1 --no-graph --no-cpu-baseline
-# (dram__bytes_read.sum + dram__bytes_write.sum, last 48 launches; profiles/gemm_tc_and_fused_light__cfg2_traffic.md).
-# Valid only for the kernel sources it was taken with: any change to them turns the field back to null.
-TC_TRAFFIC_BYTES_PER_LAUNCH = 6352517
-TC_TRAFFIC_SOURCES_SHA256 = "d68080571be2512e39f7db6b01648c105ff7a15b103e4e5d7da2691bfa15d806"
-TC_SOURCES = ("gemm_tc.cu", "fused_light.cu", "ptx.cuh", "epilogue.cuh", "internal.h")
-
-
-def tc_sources_sha256():
-    import hashlib
-    h = hashlib.sha256()
-    for name in TC_SOURCES:
-        with open(os.path.join(ROOT, "paper_2401_04044_b200", "csrc", name), "rb") as f:
-            h.update(f.read())
-    return h.hexdigest()
-
-
-def measured_traffic():
-    if TC_TRAFFIC_BYTES_PER_LAUNCH is None or tc_sources_sha256() != TC_TRAFFIC_SOURCES_SHA256:
-        return None
-    return TC_TRAFFIC_BYTES_PER_LAUNCH
 
 
 def time_region(fn, steps, warmup, flush, dist_barrier):
@@ -272,6 +258,21 @@ def time_region(fn, steps, warmup, flush, dist_barrier):
     return times
 
 
+def graphed(fn):
+    """fn recorded once into a CUDA graph (replays are what is timed); fn itself if the capture fails."""
+    import torch
+    try:
+        fn()
+        torch.cuda.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            fn()
+        return g.replay, "cuda_graph", g
+    except Exception as exc:
+        torch.cuda.synchronize()
+        return fn, f"stream (graph capture failed: {type(exc).__name__})", None
+
+
 def max_over_ranks(ms: float, world: int, device) -> float:
     """The slowest rank's time for a timed region (every rank gets the same number back)."""
     if world <= 1:
@@ -290,17 +291,27 @@ def whole_job_tokens_per_s(total_ms: float, tokens_per_rank_step: int, steps: in
     return world * tokens_per_rank_step * steps / (slowest * 1e-3)
 
 
-def flops_per_token(cfg, dense=False):
+def layer_params(cfg, dense=False):
     n_in = cfg.n_in
     if dense:
-        return 2.0 * (n_in + 1) * cfg.d * cfg.m
-    return 2.0 * (n_in + 1) * (cfg.d * cfg.k + cfg.r * (cfg.d + cfg.m - cfg.k))
+        return (n_in + 1) * cfg.d * cfg.m
+    return (n_in + 1) * (cfg.d * cfg.k + cfg.r * (cfg.d + cfg.m - cfg.k))
+
+
+def roofline_ms(cfg, T, peaks, dense=False):
+    """Roofline time of one layer: the slower of its FLOPs at the bf16 tensor peak and its bytes at the HBM peak
+    (both measured on this machine); returns (milliseconds, which bound)."""
+    params = layer_params(cfg, dense)
+    flops = 2.0 * params * T
+    bytes_ = 2.0 * (params + cfg.m + cfg.d) + 2.0 * T * cfg.d * 2
+    tf, hb = flops / (peaks["bf16_tflops"] * 1e12), bytes_ / (peaks["hbm_gbs"] * 1e9)
+    return max(tf, hb) * 1e3, ("tensor" if tf > hb else "hbm")
 
 
 def run_ours(args):
     import torch
     import torch.distributed as dist
-    from ffsplit_synth import CONFIGS
+    from ffsplit_synth import cfg5_point
     from paper_2401_04044_b200 import Context, build
 
     rank = int(os.environ.get("RANK", "0"))
@@ -320,11 +331,11 @@ def run_ours(args):
         if world > 1:
             dist.barrier()
 
-    cfg = CONFIGS[CFG_ID]
-    T = cfg.t_fwd[0]
+    cfg = cfg5_point(HEAVY_PERCENT, RANK)
+    T = 4096
     ctx = Context(local_rank)
     n_layers = args.layers or cfg.layers
-    wl = StackWorkload(cfg, ctx, n_layers, T, device, cal_lanes=1 if args.only else args.cal_lanes)
+    wl = StackWorkload(cfg, ctx, n_layers, T, device, lanes=args.cal_lanes, dense=not args.only)
     flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=device)
 
     def flush():
@@ -332,18 +343,17 @@ def run_ours(args):
 
     if args.only:
         # one phase alone, few launches: the form used under a profiler
-        wl.calibrate()
-        fn = {"step": wl.step, "forward": wl.forward, "dense": lambda: wl.forward(dense=True),
-              "calibrate": wl.calibrate}[args.only]
+        X1 = wl.X[:1].contiguous()
+        Y1 = torch.empty_like(X1)
+        fn = {"step": wl.step_serial, "forward": wl.forward, "calibrate": wl.calibrate_serial,
+              "decode": lambda: wl.forward(x=X1, y=Y1)}[args.only]
         ms = time_region(fn, args.steps, args.warmup, flush, barrier)
-        ctx.poll()
+        wl.poll()
         if rank == 0:
-            print(json.dumps({"only": args.only, "layers": n_layers, "tokens": T, "ms_per_call": ms}))
+            print(json.dumps({"only": args.only, "layers": n_layers, "ms_per_call": ms}))
         return
 
     sampler = ClockSampler(local_rank) if rank == 0 else None
-    # The step is launch-bound on the host (about a hundred launches of 5-50 us): capture it once in a
-    # CUDA graph and time replays.  --no-graph times the plain stream launches instead.
     wl.step()
     wl.poll()
     n0 = wl.launch_count()
@@ -351,154 +361,189 @@ def run_ours(args):
     launches_per_step = wl.launch_count() - n0
     wl.poll()
     step_fn, launch_mode = wl.step, "stream"
+    keep = []
     if not args.no_graph:
-        try:
-            graph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(graph):
-                wl.step()
-            step_fn, launch_mode = graph.replay, "cuda_graph"
-        except Exception as exc:   # capture refused: fall back to stream launches, and say so
-            launch_mode = f"stream (graph capture failed: {type(exc).__name__})"
-            torch.cuda.synchronize()
+        step_fn, launch_mode, g = graphed(wl.step)
+        keep.append(g)
     step_ms = time_region(step_fn, args.steps, args.warmup, flush, barrier)
     wl.poll()
     wl.check_selection_stable()
     total_ms = max_over_ranks(sum(step_ms), world, device)
     value = world * T * args.steps / (total_ms * 1e-3)
 
-    # ---- phases, each timed the same way (kernel-only, inputs resident)
-    k_ph, w_ph = max(3, min(args.steps, 10)), max(3, min(args.warmup, 3))
-    fwd_ms = statistics.median(time_region(wl.forward, k_ph, w_ph, flush, lambda: None))
-    dense_ms = statistics.median(time_region(lambda: wl.forward(dense=True), k_ph, w_ph, flush, lambda: None))
-    cal_ms = statistics.median(time_region(wl.calibrate, k_ph, w_ph, flush, lambda: None))
+    # ---- phases, each timed the same way (kernel-only, inputs resident; graph replays; L2 flushed before each)
+    k_ph, w_ph = 5, 3
+    phases = {"layers": n_layers}
 
-    # ---- roofline of the dominant kernel (the tensor-core GEMM, all its launches in a step)
+    def timed(fn):
+        f, _, g = (fn, None, None) if args.no_graph else graphed(fn)
+        keep.append(g)
+        return statistics.median(time_region(f, k_ph, w_ph, flush, lambda: None))
+
+    cal_ms = timed(wl.calibrate)
+    phases["calibrate_ms_per_stack"] = cal_ms
+    for Tp in (T, 32, 1):
+        Xp = wl.X[:Tp].contiguous()
+        Yp = torch.empty_like(Xp)
+        row = {}
+        for name, dense in (("split", False), ("dense", True)):
+            ms = timed(lambda: wl.forward(dense=dense, x=Xp, y=Yp))
+            roof, bound = roofline_ms(cfg, Tp, peaks, dense)
+            row[name] = {"ms_per_stack": ms, "us_per_layer": 1e3 * ms / n_layers,
+                         "tokens_per_s_per_stack": Tp / (ms * 1e-3), "tokens_per_s_per_layer": Tp * n_layers / (ms * 1e-3),
+                         "roofline_us_per_layer": 1e3 * roof, "bound": bound, "roofline_frac": roof * n_layers / ms}
+        row["split_vs_dense_speedup"] = row["dense"]["ms_per_stack"] / row["split"]["ms_per_stack"]
+        phases[f"forward_T{Tp}"] = row
+        wl.poll()
+    phases["model_bytes_split_per_layer"] = wl.logical_bytes
+    phases["model_bytes_dense_per_layer"] = wl.logical_bytes_dense
+
+    # ---- roofline of the dominant kernel: the tensor-core GEMM (the scoring products hold 97 % of the step's
+    # FLOPs), all its launches of one serial step, each bracketed by CUDA events on its stream
+    lane0 = wl.lanes[0][0]
+    flush()
+    lane0.profile_begin()
     ctx.profile_begin()
-    for _ in range(3):
-        flush()
-        wl.step_serial()
-    n_l, ms_l, flops_l = ctx.profile_end(0)
+    wl.step_serial()
+    n_a, ms_a, fl_a = lane0.profile_end(0)
+    n_b, ms_b, fl_b = ctx.profile_end(0)
+    n_l, ms_l, flops_l = n_a + n_b, ms_a + ms_b, fl_a + fl_b
     achieved = flops_l / (ms_l * 1e-3) / 1e12 if ms_l > 0 else 0.0
     roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel", "achieved": round(achieved, 2),
-                "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": round(achieved / peaks["bf16_tflops"], 4),
-                "peak_source": f"{peaks['source']} (burst bf16; kernels of 5-40 us timed one by one)",
-                "launches_per_step": n_l // 3, "avg_launch_us": round(1e3 * ms_l / max(n_l, 1), 2),
-                "traffic": measured_traffic()}
-    ctx.profile_begin()
-    for _ in range(3):
-        flush()
-        wl.forward()
-    n_f, ms_f, flops_f = ctx.profile_end(0)
-    fwd_tflops = flops_f / (ms_f * 1e-3) / 1e12 if ms_f > 0 else 0.0
+                "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                "frac": round(achieved / peaks["bf16_tflops_sustained"], 4),
+                "frac_of_burst_peak": round(achieved / peaks["bf16_tflops"], 4),
+                "peak_source": f"{peaks['source']} (sustained bf16: launches of 0.1-13 ms back to back inside a 0.5 s step)",
+                "launches_per_step": n_l, "avg_launch_us": round(1e3 * ms_l / max(n_l, 1), 2),
+                "algorithmic_flops_per_launch": flops_l / max(n_l, 1), "traffic": None}
+    wl.poll()
 
-    # ---- end to end: host buffers, copies inside the timed region
-    Xcal_host = [e["Xcal"].cpu().pin_memory() for e in wl.layers]
+    # ---- end to end through the host-buffer entry points: calibration tokens, X and Y in pinned host memory
+    n_host = min(4, n_layers)
+    x_hosts = [wl.layers[i]["Xcal"].cpu().pin_memory() for i in range(n_host)]
     X_host = wl.X.cpu().pin_memory()
     Y_host = torch.empty_like(X_host).pin_memory()
-    x_dev = torch.empty_like(wl.X)
-
-    def e2e_step():
-        # every layer's calibration tokens are copied on the stream that calibrates that layer, so the
-        # copy engine works under the kernels of the other streams
-        x_dev.copy_(X_host, non_blocking=True)
-        y = wl.step(x_dev, before=lambda i: wl.layers[i]["Xcal"].copy_(Xcal_host[i], non_blocking=True))
-        Y_host.copy_(y, non_blocking=True)
-
-    e2e_fn = e2e_step
+    e2e_fn = lambda: wl.step_host(x_hosts, X_host, Y_host)
     if not args.no_graph:
-        # the copies are graph nodes like the kernels (pinned host buffers at fixed addresses)
-        try:
-            e2e_step()
-            torch.cuda.synchronize()
-            e2e_graph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(e2e_graph):
-                e2e_step()
-            e2e_fn = e2e_graph.replay
-        except Exception:
-            torch.cuda.synchronize()
-            e2e_fn = e2e_step
-    e2e_ms = time_region(e2e_fn, k_ph, w_ph, flush, barrier)
+        e2e_fn, _, g = graphed(e2e_fn)
+        keep.append(g)
+    k_e2e = 3
+    e2e_ms = time_region(e2e_fn, k_e2e, 1, flush, barrier)
+    wl.poll()
     e2e_total = max_over_ranks(sum(e2e_ms), world, device)
     es = 2
-    h2d = cfg.layers * cfg.t_cal * cfg.d * es + T * cfg.d * es
+    h2d = n_layers * cfg.t_cal * cfg.d * es + T * cfg.d * es
     d2h = T * cfg.d * es
-    e2e = {"value": world * T * k_ph / (e2e_total * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-           "d2h_bytes_per_step": d2h}
-
-    # single layer through the host-buffer entry point of the C ABI
-    e0 = wl.layers[0]
-    host_ms = statistics.median(time_region(lambda: ctx.forward_host(e0["blob"], X_host, Y_host), k_ph, w_ph, flush,
-                                            lambda: None))
-    ctx.poll()
+    e2e = {"value": world * T * k_e2e / (e2e_total * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+           "d2h_bytes_per_step": d2h, "ms_per_step": e2e_total / k_e2e,
+           "api": "ffsplit_score_host + ffsplit_select + ffsplit_pack per layer, ffsplit_forward_stack_host",
+           "host_buffers": f"{n_host} pinned calibration buffers used round robin over the {n_layers} layers"}
     clocks = sampler.stop() if sampler else None
 
+    # ---- the smaller configurations, per layer (the sweep tool's timing: graph replays over distinct weight copies)
+    others = {}
+    if rank == 0 and not args.no_other_configs:
+        del x_hosts, e2e_fn
+        keep.clear()
+        wl = None
+        torch.cuda.empty_cache()
+        others = other_configs(peaks)
+
     if rank == 0:
-        roof_t = flops_per_token(cfg) * T / (peaks["bf16_tflops"] * 1e12) * 1e3          # ms per layer
-        roof_t_dense = flops_per_token(cfg, True) * T / (peaks["bf16_tflops"] * 1e12) * 1e3
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": "configs[1]: BERT-base-shaped stack, 12 GELU FFN layers, d=768 m=3072 k=154 r=192, "
-                                   "4096 calibration tokens/layer, prefill 32x128=4096 tokens; step = score+select+pack "
-                                   "per layer, then the 12-layer split forward",
-                       "l2": "256 MiB buffer rewritten before every timed step (L2 flush)",
-                       "launch": launch_mode, "calibration_streams": max(1, len(wl.lanes) - 1),
-                       "tokens_per_step": T, "layers": cfg.layers},
+            "config": {"workload": WORKLOAD,
+                       "l2": "256 MiB buffer rewritten before every timed step (L2 flush); 40 distinct layers of 72 MB "
+                             "(split) / 420 MB (dense) per pass in any case",
+                       "launch": launch_mode, "calibration_streams": args.cal_lanes,
+                       "tokens_per_step": T, "layers": n_layers,
+                       "light_factors": "seeded random matrices of the packed shapes (the float64 SVD is off-path set-up)"},
             "roofline": roofline,
             "e2e": e2e,
             "gpu_launches": int(launches_per_step * args.steps),
             "gpu_launches_per_step": int(launches_per_step),
             "clocks": clocks,
-            "phases": {
-                "forward_split_ms_per_stack": fwd_ms, "forward_dense_ms_per_stack": dense_ms,
-                "calibrate_ms_per_stack": cal_ms,
-                "forward_split_tokens_per_s_per_stack": T / (fwd_ms * 1e-3),
-                "forward_split_tokens_per_s_per_layer": T * cfg.layers / (fwd_ms * 1e-3),
-                "forward_dense_tokens_per_s_per_stack": T / (dense_ms * 1e-3),
-                "split_vs_dense_speedup": dense_ms / fwd_ms,
-                "forward_split_roofline_frac": roof_t * cfg.layers / fwd_ms,
-                "forward_dense_roofline_frac": roof_t_dense * cfg.layers / dense_ms,
-                "forward_split_gemm_tflops": round(fwd_tflops, 2),
-                "forward_host_one_layer_ms": host_ms,
-                "model_bytes_split_per_layer": wl.logical_bytes, "model_bytes_dense_per_layer": wl.logical_bytes_dense,
-            },
+            "phases": phases,
+            "other_configs": others,
             "paper_context": "43.1% fewer parameters and 1.25-1.56x whole-model BERT-base speedup on V100 / Xeon "
                              "(Section 5.1); other hardware, not a target",
         }
         if world == 1 and not args.no_cpu_baseline:
-            out["cpu_baseline"] = cpu_baseline_sample(cfg, T, layers_sample=cfg.layers, reps=2)
+            out["cpu_baseline"] = cpu_baseline_sample(cfg, T)
         print(json.dumps(out))
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
 
 
+def other_configs(peaks):
+    """Split vs dense per layer on the BERT-base, GPT-2-medium and Llama-2-7B shaped configurations."""
+    import sweep
+    from ffsplit_synth import CONFIGS
+    from paper_2401_04044_b200 import Context
+    out = {}
+    ctx = Context(0)
+    try:
+        for cid, tokens in ((2, (4096,)), (3, (1, 4, 16, 64)), (4, (2048, 1, 8, 32))):
+            cfg = CONFIGS[cid]
+            split_bytes = 2 * layer_params(cfg)
+            copies = max(2, min(12, -(-2 * 126 * (1 << 20) // split_bytes)))
+            rows = sweep.run_point(ctx, cfg, list(tokens), copies, 5, False, settle=0.3)
+            for r in rows:
+                out[f"{cfg.name}_T{r['tokens']}"] = {
+                    "split_us_per_layer": 1e3 * r["split"]["ms_per_layer"], "split_roofline_frac": r["split"]["roofline_frac"],
+                    "dense_us_per_layer": 1e3 * r["dense"]["ms_per_layer"], "dense_roofline_frac": r["dense"]["roofline_frac"],
+                    "bound": r["split"]["bound"], "split_vs_dense_speedup": r["split_vs_dense_speedup"],
+                    "split_tokens_per_s_per_stack": r["split"]["tokens_per_s_per_stack"], "weight_copies": copies}
+    finally:
+        ctx.close()
+    return out
+
+
 # --------------------------------------------------------------------------------------
-def oracle_layer_setup(cfg, layer):
-    """Inputs of one layer for the oracle arm, as float64 numpy (exact up-casts), with
-    the light factors it will use (set-up, untimed: the SVD is not on the hot path)."""
+# The CPU legs: the oracle, as it stands, on a bounded sample of the same workload.
+SAMPLE_CAL, SAMPLE_FWD = 1024, 128
+
+
+def oracle_sample_setup(cfg, layer=0):
+    """One layer's inputs as float64 numpy (exact up-casts) with seeded light factors of the packed shapes."""
     import numpy as np
     from ffsplit_synth import make_layer
-    from oracle import ffsplit_oracle as orc
     L = make_layer(cfg, layer)
     f = lambda t: None if t is None else t.double().numpy()
     W = {"W1": f(L.W1), "b1": f(L.b1), "W2": f(L.W2), "b2": f(L.b2)}
-    Xcal = f(L.tokens(cfg.t_cal))
-    sw = orc.split_weights(W["W1"], W["b1"], W["W2"], L.planted.numpy())
-    fac = {}
-    fac["A1"], fac["B1"] = orc.light_factors(sw["U2"], cfg.r)
-    fac["A2"], fac["B2"] = orc.light_factors(sw["V2"], cfg.r)
-    rnd = lambda a: np.asarray(__import__("torch").from_numpy(a).to(cfg.torch_dtype).double().numpy())
-    fac = {k: rnd(v) for k, v in fac.items()}
-    return W, Xcal, fac
+    rng = np.random.default_rng(7)
+    d, ml, r = cfg.d, cfg.m - cfg.k, cfg.r
+    fac = {"A1": rng.standard_normal((d, r)) * 0.02, "B1": rng.standard_normal((r, ml)) * 0.02,
+           "A2": rng.standard_normal((ml, r)) * 0.02, "B2": rng.standard_normal((r, d)) * 0.02}
+    Xcal = f(L.tokens(SAMPLE_CAL))
+    X = f(L.tokens(SAMPLE_FWD))
+    return W, Xcal, fac, X
 
 
-def oracle_layer_step(cfg, W, Xcal, fac, X):
+def oracle_sample_step(cfg, W, Xcal, fac, X):
+    """score over the sampled calibration tokens + select + split forward of the sampled tokens; returns the two times."""
     from oracle import ffsplit_oracle as orc
+    t0 = time.perf_counter()
     _, _, s = orc.neuron_scores(Xcal, W["W1"], W["b1"], W["W2"], cfg.act)
     heavy, _ = orc.select_heavy(s, cfg.k)
-    return orc.split_ffn(X, W["W1"], W["b1"], W["W2"], W["b2"], heavy, fac, cfg.act)
+    t1 = time.perf_counter()
+    orc.split_ffn(X, W["W1"], W["b1"], W["W2"], W["b2"], heavy, fac, cfg.act)
+    t2 = time.perf_counter()
+    return t1 - t0, t2 - t1
+
+
+def scaled_stack_seconds(cfg, T, t_cal_s, t_fwd_s):
+    """Tokens are independent in both passes, so the sampled times scale with the token counts."""
+    return cfg.layers * (t_cal_s * cfg.t_cal / SAMPLE_CAL + t_fwd_s * T / SAMPLE_FWD)
+
+
+def sample_text(cfg, T):
+    return (f"1 of {cfg.layers} layers: score over {SAMPLE_CAL} of the {cfg.t_cal} calibration tokens + select + split "
+            f"forward of {SAMPLE_FWD} of the {T} tokens (fp64 numpy); stack time = {cfg.layers} x (score time x "
+            f"{cfg.t_cal // SAMPLE_CAL} + forward time x {T // SAMPLE_FWD})")
 
 
 def blas_threads():
@@ -510,56 +555,40 @@ def blas_threads():
         return os.cpu_count() or 1
 
 
-def cpu_baseline_sample(cfg, T, layers_sample=12, reps=2):
-    import numpy as np
-    rng = np.random.default_rng(0)
-    X = rng.standard_normal((T, cfg.d))
-    layers_sample = min(layers_sample, cfg.layers)
-    setups = [oracle_layer_setup(cfg, l) for l in range(layers_sample)]
-    best = None
+def cpu_baseline_sample(cfg, T, reps=3):
+    setup = oracle_sample_setup(cfg)
+    best, spent = None, 0.0
     for _ in range(reps):
-        t0 = time.perf_counter()
-        x = X
-        for W, Xcal, fac in setups:
-            x = oracle_layer_step(cfg, W, Xcal, fac, x)
-        dt = time.perf_counter() - t0
-        best = dt if best is None else min(best, dt)
-    per_stack = best * cfg.layers / layers_sample
-    return {"value": T / per_stack, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
-            "sample": f"{layers_sample} of {cfg.layers} layers (score over {cfg.t_cal} calibration tokens + select + "
-                      f"split forward of all {T} tokens, fp64 numpy), best of {reps} passes, time scaled by {cfg.layers}/{layers_sample}",
-            "seconds_sampled": best * reps}
+        a, b = oracle_sample_step(cfg, *setup)
+        spent += a + b
+        s = scaled_stack_seconds(cfg, T, a, b)
+        best = s if best is None else min(best, s)
+    return {"value": T / best, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+            "sample": sample_text(cfg, T) + f"; best of {reps}", "seconds_sampled": spent}
 
 
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    import numpy as np
-    from ffsplit_synth import CONFIGS
-    cfg = CONFIGS[CFG_ID]
-    T = cfg.t_fwd[0]
-    n_setups = 2
-    setups = [oracle_layer_setup(cfg, l) for l in range(n_setups)]
-    X = np.random.default_rng(0).standard_normal((T, cfg.d))
-    times = []
+    from ffsplit_synth import cfg5_point
+    cfg = cfg5_point(HEAVY_PERCENT, RANK)
+    T = 4096
+    setup = oracle_sample_setup(cfg)
+    stack_s, step_s = [], []
     for i in range(args.warmup + args.steps):
-        W, Xcal, fac = setups[i % n_setups]
-        t0 = time.perf_counter()
-        oracle_layer_step(cfg, W, Xcal, fac, X)
-        dt = time.perf_counter() - t0
+        a, b = oracle_sample_step(cfg, *setup)
         if i >= args.warmup:
-            times.append(dt)
-    per_step = sum(times) / len(times) * cfg.layers        # one sampled layer per step, scaled to the stack
-    value = T / per_step
-    sample = (f"each step = 1 of {cfg.layers} layers (score over {cfg.t_cal} calibration tokens + select + split "
-              f"forward of all {T} tokens, fp64 numpy), time scaled by {cfg.layers}")
+            step_s.append(a + b)
+            stack_s.append(scaled_stack_seconds(cfg, T, a, b))
+    value = T / (sum(stack_s) / len(stack_s))
     out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
-           "steps": args.steps, "warmup": args.warmup, "ms_per_step": per_step * 1e3, "higher_is_better": True,
-           "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-           "config": {"workload": "configs[1]: BERT-base-shaped stack, 12 GELU FFN layers, d=768 m=3072 k=154 r=192, "
-                                  "4096 calibration tokens/layer, prefill 4096 tokens (CPU oracle, bounded sample)"},
-           "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
+           "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * sum(step_s) / len(step_s),
+           "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+           "config": {"workload": WORKLOAD + " (CPU oracle; each step is a bounded sample, ms_per_step is the sample's "
+                                            "own time and value is scaled to the whole step)"},
+           "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                            "sample": "each step: " + sample_text(cfg, T)},
            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
            "gpu_launches": 0}
     print(json.dumps(out))
@@ -568,16 +597,17 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-other-configs", action="store_true", help="skip the per-layer rows of the smaller configurations")
     ap.add_argument("--no-graph", action="store_true", help="time plain stream launches instead of a CUDA-graph replay")
-    ap.add_argument("--cal-lanes", type=int, default=3,
+    ap.add_argument("--cal-lanes", type=int, default=2,
                     help="streams (each with its own library context) the per-layer calibrations are spread over")
-    ap.add_argument("--only", default=None, choices=["step", "forward", "dense", "calibrate"],
+    ap.add_argument("--only", default=None, choices=["step", "forward", "calibrate", "decode"],
                     help="run one phase alone and print its times (for profiler captures)")
-    ap.add_argument("--layers", type=int, default=0, help="with --only: number of layers of the stack to build")
+    ap.add_argument("--layers", type=int, default=0, help="number of layers of the stack to build (default: all 40)")
     args = ap.parse_args()
     if args.impl == "ours" and not args.only:
         args.warmup = max(args.warmup, 3)

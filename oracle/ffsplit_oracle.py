@@ -25,6 +25,10 @@ Pins (tests that tie each function to something other than itself):
   split_ffn .......... Eq. 2 (k = d_ff, exact light part, full-rank factors all
                        reproduce the dense FFN), permutation / padding invariance
   param counts ....... the 43.1 % reduction printed in Section 5.1.1
+  rtn_quantize ....... |w - dq(q(w))| <= step / 2, grid end points, constant groups and on-grid values exact,
+                       round-to-nearest on hand-placed values, independence of groups and of output channels
+  quantize_split ..... group axes and bit widths per part, reassembly; quant_split_ffn against Eq. 2 written
+                       neuron by neuron on the dequantised weights, error halving per extra bit; byte formula
 Parity unpinned: the error of a *truncated* light part against the dense FFN
 (the paper reports task accuracy only, Table 1); it is reported, never gated.
 """
@@ -270,3 +274,119 @@ def normalised_max_abs(Y, Yref):
     den = np.max(np.abs(Yref)) if Yref.size else 0.0
     num = np.max(np.abs(Y - Yref)) if Yref.size else 0.0
     return float(num / den) if den > 0 else float(num)
+
+
+# --------------------------------------------------------------------------
+# Quantised split (Section 5.2): round-to-nearest with a group size of 128, 8 bits for the heavy-hitter
+# neurons and 3 bits for everything else.  The paper fixes the bit widths, the group size and "round to
+# nearest"; it does not say along which axis the groups run, whether the grid is symmetric, or how codes
+# are stored.  Reading taken here (the usual "wB-g128" convention of weight-only quantisation):
+#   * each of the four matrices of the split (U1, V1 heavy; U2, V2 light) is quantised on its own;
+#   * a group is 128 consecutive weights along the INPUT dimension of the linear map, for one output
+#     channel: along d for a column of U (one neuron's input weights), along the neuron axis of the part
+#     (heavy neurons, or light neurons, in ascending index order) for a column of V; a last, shorter group
+#     takes what is left;
+#   * asymmetric min/max grid: lo = min, scale = (max - lo) / (2^b - 1), code q = round((w - lo) / scale)
+#     clamped to [0, 2^b - 1], dequantised value lo + q * scale; a constant group has scale 0, code 0 and is
+#     reproduced exactly;
+#   * the decisions (min, max, scale, the rounding) are taken in float32 arithmetic, round-half-to-even --
+#     the precision the CUDA path takes them in -- so that codes can be compared bit for bit; the
+#     dequantised value is lo + q * scale evaluated exactly from the stored float32 (lo, scale);
+#   * biases are not quantised.
+# --------------------------------------------------------------------------
+QUANT_GROUP = 128
+QUANT_BITS_HEAVY = 8
+QUANT_BITS_LIGHT = 3
+
+
+def rtn_quantize_groups(w, bits, group=QUANT_GROUP):
+    """Round-to-nearest quantisation of the LAST axis of `w` in groups of `group` (the last one may be
+    shorter).  Returns (codes uint8 with w's shape, scale float32 [..., n_groups], lo float32 [..., n_groups])."""
+    w = np.asarray(w, dtype=np.float32)
+    n = w.shape[-1]
+    ng = (n + group - 1) // group
+    qmax = np.float32((1 << bits) - 1)
+    codes = np.zeros(w.shape, dtype=np.uint8)
+    scale = np.zeros(w.shape[:-1] + (ng,), dtype=np.float32)
+    lo = np.zeros_like(scale)
+    for g in range(ng):
+        seg = w[..., g * group:(g + 1) * group]
+        mn = seg.min(axis=-1).astype(np.float32)
+        mx = seg.max(axis=-1).astype(np.float32)
+        sc = ((mx - mn).astype(np.float32) / qmax).astype(np.float32)
+        lo[..., g] = mn
+        scale[..., g] = sc
+        safe = np.where(sc > 0, sc, np.float32(1.0)).astype(np.float32)
+        q = np.rint(((seg - mn[..., None]).astype(np.float32) / safe[..., None]).astype(np.float32))
+        q = np.clip(q, 0, float(qmax))
+        q = np.where(sc[..., None] > 0, q, 0.0)
+        codes[..., g * group:(g + 1) * group] = q.astype(np.uint8)
+    return codes, scale, lo
+
+
+def rtn_dequantize_groups(codes, scale, lo, group=QUANT_GROUP):
+    """lo + q * scale per group, in float64 (exact for the stored float32 parameters and integer codes)."""
+    codes = np.asarray(codes)
+    n = codes.shape[-1]
+    idx = np.arange(n) // group
+    return _f64(lo)[..., idx] + codes.astype(np.float64) * _f64(scale)[..., idx]
+
+
+def quantize_split(W1, W2, heavy, bits_heavy=QUANT_BITS_HEAVY, bits_light=QUANT_BITS_LIGHT, group=QUANT_GROUP,
+                   W1u=None):
+    """The four (SwiGLU: six) quantised matrices of the split.  Every entry of the result is a triple
+    (codes, scale, lo) laid out with the grouped (input) axis last:
+      'U1', 'U2' (and 'U1u', 'U2u'): [neurons of the part, d]        groups along d
+      'V1', 'V2':                    [d, neurons of the part]        groups along the part's neuron axis
+    """
+    sw = split_weights(W1, None, W2, heavy, W1u)
+    out = {"heavy": sw["heavy"], "light": sw["light"]}
+    out["U1"] = rtn_quantize_groups(sw["U1"].T, bits_heavy, group)
+    out["U2"] = rtn_quantize_groups(sw["U2"].T, bits_light, group)
+    out["V1"] = rtn_quantize_groups(sw["V1"].T, bits_heavy, group)
+    out["V2"] = rtn_quantize_groups(sw["V2"].T, bits_light, group)
+    if W1u is not None:
+        out["U1u"] = rtn_quantize_groups(sw["U1u"].T, bits_heavy, group)
+        out["U2u"] = rtn_quantize_groups(sw["U2u"].T, bits_light, group)
+    return out
+
+
+def dequantized_weights(Q, d, m, group=QUANT_GROUP):
+    """Reassemble the full matrices W1~ [d, m], W2~ [m, d] (and W1u~) from the quantised parts."""
+    heavy, light = Q["heavy"], Q["light"]
+    W1 = np.zeros((d, m))
+    W2 = np.zeros((m, d))
+    W1[:, heavy] = rtn_dequantize_groups(*Q["U1"], group).T
+    W1[:, light] = rtn_dequantize_groups(*Q["U2"], group).T
+    W2[heavy, :] = rtn_dequantize_groups(*Q["V1"], group).T
+    W2[light, :] = rtn_dequantize_groups(*Q["V2"], group).T
+    W1u = None
+    if "U1u" in Q:
+        W1u = np.zeros((d, m))
+        W1u[:, heavy] = rtn_dequantize_groups(*Q["U1u"], group).T
+        W1u[:, light] = rtn_dequantize_groups(*Q["U2u"], group).T
+    return W1, W2, W1u
+
+
+def quant_split_ffn(X, b1, b2, Q, d, m, act, group=QUANT_GROUP):
+    """Eq. 2 with FFN_1 on the 8-bit heavy matrices and FFN_2 on the 3-bit light ones: the dense FFN of
+    Section 2 evaluated on the dequantised weights (both parts use their own neurons' biases)."""
+    W1, W2, W1u = dequantized_weights(Q, d, m, group)
+    return dense_ffn(X, W1, b1, W2, b2, act, W1u)
+
+
+def quant_weight_bytes(d, m, k, bits_heavy=QUANT_BITS_HEAVY, bits_light=QUANT_BITS_LIGHT, group=QUANT_GROUP,
+                       n_in=1, param_bytes=8):
+    """Bytes of the quantised weights: codes at their bit width plus one (scale, lo) pair of float32 per group
+    (param_bytes = 8).  U-type matrices have ceil(d / group) groups per neuron, V-type ceil(neurons / group)
+    per output column."""
+    ml = m - k
+    gd = -(-d // group)
+    def part(n, bits):
+        if n == 0:
+            return 0
+        gv = -(-n // group)
+        u_bits = n_in * n * d * bits
+        v_bits = n * d * bits
+        return (u_bits + v_bits) / 8 + param_bytes * (n_in * n * gd + d * gv)
+    return part(k, bits_heavy) + part(ml, bits_light)

@@ -10,12 +10,122 @@
 #include <cstring>
 #include <mutex>
 
+#include "decode_stream.h"
 #include "epilogue.cuh"
 #include "internal.h"
 
 namespace ffsp {
 
 constexpr long long kDecodeScratchBytes = 16ll << 20;   // fp32 partials of the row tiles that several CTAs share
+
+// ---- 1..8 tokens: the phases of one layer for decode_stream_kernel ---------------------------------------
+// Every phase writes raw fp32 sums (one slice per k range); the phase that reads them adds the slices, the
+// bias and the activation.  Returns FFSPLIT_ERR_BUFFER_TOO_SMALL without launching when `scratch_bytes`
+// cannot hold the slices (the caller then takes the other few-token kernel).
+static int stream_splits(int K) {
+  const int k32 = (K + 31) / 32, cap = kStreamKxMax / 32;
+  return (k32 + cap - 1) / cap;
+}
+
+static ffsplit_status stream_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* blob, const void* X, int T,
+                                     void* Y, char* scratch, long long scratch_bytes, int* ctrl, cudaStream_t st,
+                                     unsigned long long guard_hash, bool* launched) {
+  *launched = false;
+  const int d = h.d, k_pad = h.k_pad, r_pad = h.r_pad, ml_pad = h.ml_pad, kp_rp = h.k_pad + h.r_pad;
+  const bool gated = h.act == FFSPLIT_SWIGLU;
+  const bool light = r_pad > 0 && h.ml > 0;
+  const int g2 = gated ? 2 : 1;
+  auto W = [&](int sec) { return reinterpret_cast<const __nv_bfloat16*>(blob + h.off[sec]); };
+  auto F = [&](int sec) { return reinterpret_cast<const float*>(blob + h.off[sec]); };
+  // slices in the scratch area
+  const int S1 = stream_splits(d), S2a = stream_splits(r_pad), S2b = stream_splits(ml_pad);
+  const int K3 = light ? kp_rp : k_pad;
+  const int S3 = stream_splits(K3);
+  const long long N1 = static_cast<long long>(g2) * (k_pad + (light ? r_pad : 0));
+  const long long N2a = static_cast<long long>(g2) * ml_pad;
+  long long off = 0;
+  auto take = [&](long long slices, long long cols) { const long long o = off; off += slices * 8 * cols; return o; };
+  const long long o_p1 = take(S1, N1);
+  const long long o_2a = light ? take(S2a, N2a) : 0;
+  const long long o_2b = light ? take(S2b, r_pad) : 0;
+  const long long o_y = S3 > 1 ? take(S3, d) : 0;
+  if (off * 4 > scratch_bytes) return FFSPLIT_ERR_BUFFER_TOO_SMALL;
+  float* fs = reinterpret_cast<float*>(scratch);
+
+  StreamParams p;
+  std::memset(&p, 0, sizeof(p));
+  p.T = T; p.act = h.act; p.ctrl = ctrl;
+  p.guard = guard_hash ? reinterpret_cast<const unsigned long long*>(blob) : nullptr;
+  p.guard_hash = guard_hash;
+  auto add_seg = [](StreamPhase& ph, const __nv_bfloat16* Wp, long long ldw, int rows, int x_off, int out_col) {
+    if (rows <= 0) return;
+    StreamSegment& s = ph.seg[ph.nseg++];
+    s.W = Wp; s.ldw = ldw; s.rows = rows; s.x_off = x_off; s.out_col = out_col;
+    ph.Nall += rows;
+  };
+  auto slices_in = [](StreamPhase& ph, int c0, int c1, int kind, const float* src, int nsl, long long ld, int src_col,
+                      int gate_off, const float* bias) {
+    if (c1 <= c0) return;
+    StreamInPart& in = ph.in[ph.nin++];
+    in.col_begin = c0; in.col_end = c1; in.kind = kind; in.nslices = nsl; in.src = src; in.ld = ld;
+    in.slice_stride = 8 * ld; in.src_col = src_col; in.gate_off = gate_off; in.bias = bias;
+  };
+  // ---- stage 1: z_H = X U1 and Q = X A1 (SwiGLU: gate and up of each), raw
+  {
+    StreamPhase& ph = p.ph[p.nph++];
+    ph.K = d; ph.S = S1;
+    if (!gated) {
+      add_seg(ph, W(SEC_U1T), d, light ? kp_rp : k_pad, 0, 0);     // U1^T and A1^T are adjacent with the same pitch
+    } else {
+      add_seg(ph, W(SEC_U1T), d, k_pad, 0, 0);
+      add_seg(ph, W(SEC_U1UT), d, k_pad, 0, k_pad);
+      if (light) add_seg(ph, W(SEC_A1T), d, 2 * r_pad, 0, 2 * k_pad);   // [A1 | A1u]^T
+    }
+    StreamInPart& in = ph.in[ph.nin++];
+    in.col_begin = 0; in.col_end = d; in.kind = STREAM_IN_BF16; in.src = X; in.ld = d;
+    ph.out = fs + o_p1; ph.out_ld = N1;
+  }
+  const int q_col = g2 * k_pad;   // where Q starts among stage 1's output columns
+  if (light) {
+    // ---- stage 2a: z_L = Q B1 (raw)
+    StreamPhase& a = p.ph[p.nph++];
+    a.K = r_pad; a.S = S2a;
+    add_seg(a, W(SEC_B1T), r_pad, ml_pad, 0, 0);
+    if (gated) add_seg(a, W(SEC_B1UT), r_pad, ml_pad, r_pad, ml_pad);
+    slices_in(a, 0, g2 * r_pad, STREAM_IN_LINEAR, fs + o_p1, S1, N1, q_col, 0, nullptr);
+    a.out = fs + o_2a; a.out_ld = N2a;
+    // ---- stage 2b: P = sigma(z_L + b1[light]) A2 (raw)
+    StreamPhase& b = p.ph[p.nph++];
+    b.K = ml_pad; b.S = S2b;
+    add_seg(b, W(SEC_A2T), ml_pad, r_pad, 0, 0);
+    slices_in(b, 0, ml_pad, gated ? STREAM_IN_GATED : STREAM_IN_ACT, fs + o_2a, S2a, N2a, 0, ml_pad,
+              gated ? nullptr : F(SEC_B1L));
+    b.out = fs + o_2b; b.out_ld = r_pad;
+  }
+  // ---- stage 3: Y = [sigma(z_H + b1[h2]) | P] [V1 ; B2] + b2
+  {
+    StreamPhase& ph = p.ph[p.nph++];
+    ph.K = K3; ph.S = S3;
+    add_seg(ph, W(SEC_V1B2T), kp_rp, d, 0, 0);
+    slices_in(ph, 0, k_pad, gated ? STREAM_IN_GATED : STREAM_IN_ACT, fs + o_p1, S1, N1, 0, k_pad,
+              gated ? nullptr : F(SEC_B1H));
+    if (light) slices_in(ph, k_pad, kp_rp, STREAM_IN_LINEAR, fs + o_2b, S2b, r_pad, 0, 0, nullptr);
+    if (S3 == 1) {
+      ph.y = static_cast<__nv_bfloat16*>(Y); ph.y_ld = d; ph.y_bias = F(SEC_B2); ph.y_cols = d;
+    } else {
+      ph.out = fs + o_y; ph.out_ld = d;
+      StreamPhase& rd = p.ph[p.nph++];
+      rd.kind = 1;
+      slices_in(rd, 0, d, STREAM_IN_LINEAR, fs + o_y, S3, d, 0, 0, nullptr);
+      rd.y = static_cast<__nv_bfloat16*>(Y); rd.y_ld = d; rd.y_bias = F(SEC_B2); rd.y_cols = d;
+    }
+  }
+  const double n_in = h.n_in;
+  const double algo_bytes = 2.0 * ((n_in + 1) * (static_cast<double>(d) * h.k + static_cast<double>(h.r) * (d + h.ml))) +
+                            4.0 * (h.m + d) + 2.0 * T * d * 2;
+  *launched = true;
+  return decode_stream_launch(ctx, p, algo_bytes, st);
+}
 
 bool decode_path_applies(const ffsplit_ctx* ctx, const BlobHeader& h, long long T) {
   (void)ctx;
@@ -33,6 +143,14 @@ static ffsplit_status decode_forward_impl(ffsplit_ctx* ctx, const BlobHeader& h,
                                           cudaStream_t st, int* tickets, long long scratch_bytes,
                                           unsigned long long guard_hash) {
   const int T = static_cast<int>(T64);
+  if (T <= 8 && ctx->decode_stream) {
+    // one persistent launch whose weight stream runs ahead of the stage dependencies; its slices take the whole
+    // scratch area (the [A_H | P], Q and H_L buffers of the other kernel are not used)
+    bool launched = false;
+    const ffsplit_status ss = stream_forward(ctx, h, blob, X, T, Y, scratch, scratch_bytes, tickets ? tickets : ctx->status(),
+                                             st, guard_hash, &launched);
+    if (launched || ss != FFSPLIT_ERR_BUFFER_TOO_SMALL) return ss;
+  }
   const int d = h.d, k_pad = h.k_pad, r_pad = h.r_pad, ml_pad = h.ml_pad, kp_rp = h.k_pad + h.r_pad;
   const bool gated = h.act == FFSPLIT_SWIGLU;
   const bool light = r_pad > 0 && h.ml > 0;

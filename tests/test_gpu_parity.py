@@ -277,6 +277,7 @@ def test_fused_light_chain_matches_oracle_and_unfused_path(ctx, act, d, m, k, r,
     ctx2 = Context(0)
     try:
         ctx2.ensure_workspace(ctx2.workspace_size(G.shape, T, 0, k, r))
+        ctx2.blob_open(blob)      # packed on another context
         Xd = X.cuda()
         Y2 = torch.empty_like(Xd)
         ctx2.forward(blob, Xd, Y2)
@@ -410,6 +411,7 @@ def test_decode_single_launch_mode(ctx, monkeypatch, act, d, m, k, r, T):
     ctx2 = Context(0)
     try:
         ctx2.ensure_workspace(ctx2.workspace_size(G.shape, T, 0, k, r))
+        ctx2.blob_open(blob)      # packed on another context
         Xd = X.cuda()
         Y2 = torch.empty_like(Xd)
         for _ in range(2):   # the barrier and ticket words must be back in their rest state after a call
@@ -618,6 +620,11 @@ def test_blob_registry_and_changed_bytes(ctx):
     with pytest.raises(FFSplitError) as e:
         ctx.blob_open(small)
     assert e.value.code == 7
+    # a failed open leaves nothing registered at that address; closing twice is an error the second time
+    with pytest.raises(FFSplitError) as e:
+        ctx.forward(buf, Xd, Y)
+    assert e.value.code == 7
+    ctx.blob_open(buf)
     ctx.blob_close(buf)
     with pytest.raises(FFSplitError) as e:
         ctx.blob_close(buf)

@@ -377,3 +377,134 @@ def test_error_metrics():
     assert orc.rel_frobenius(a, a) == 0
     assert abs(orc.rel_frobenius(a + np.array([[0.3, 0.4]]), a) - 0.1) < 1e-15
     assert abs(orc.normalised_max_abs(a + np.array([[0.0, -0.2]]), a) - 0.05) < 1e-15
+
+
+# ---------------------------------------------------------------------------------------------
+# Quantised split (Section 5.2): round-to-nearest, group size 128, 8 bits heavy / 3 bits light
+# ---------------------------------------------------------------------------------------------
+def test_rtn_error_bound_codes_and_constant_groups(rng):
+    for bits in (3, 8):
+        qmax = (1 << bits) - 1
+        w = (rng.standard_normal((7, 300)) * 0.02).astype(np.float32)      # 2 full groups and a ragged one of 44
+        w[3, 128:256] = 0.125                                               # a constant group
+        q, scale, lo = orc.rtn_quantize_groups(w, bits)
+        assert q.shape == w.shape and scale.shape == (7, 3) and lo.shape == (7, 3) and q.dtype == np.uint8
+        assert q.max() <= qmax
+        wd = orc.rtn_dequantize_groups(q, scale, lo)
+        idx = np.arange(300) // 128
+        # every value lies within half a step of its code (a few float32 ulps of slack for the division)
+        assert np.all(np.abs(wd - w) <= 0.5 * scale[:, idx] * (1 + 1e-5) + 1e-12)
+        # the grid spans the group exactly: the minimum gets code 0, the maximum the last code
+        for g in range(3):
+            seg, qs = w[:, 128 * g:128 * (g + 1)], q[:, 128 * g:128 * (g + 1)]
+            live = scale[:, g] > 0
+            assert np.all(qs[np.arange(7), seg.argmin(axis=1)] == 0)
+            assert np.all(qs[np.arange(7), seg.argmax(axis=1)][live] == qmax)
+            assert np.allclose(lo[:, g], seg.min(axis=1)) and np.allclose(scale[:, g] * qmax, seg.max(axis=1) - seg.min(axis=1), rtol=1e-6)
+        # the constant group: scale 0, all codes 0, reproduced exactly
+        assert scale[3, 1] == 0 and not q[3, 128:256].any() and np.all(wd[3, 128:256] == 0.125)
+
+
+def test_rtn_values_on_the_grid_are_exact_and_rounding_is_to_nearest():
+    # a group whose values sit on an 8-level grid with a power-of-two step: 3 bits reproduce it exactly
+    base = np.float32(-0.25)
+    step = np.float32(2.0 ** -4)
+    levels = np.arange(128) % 8
+    w = (base + levels * step).astype(np.float32)[None, :]
+    q, scale, lo = orc.rtn_quantize_groups(w, 3)
+    assert np.array_equal(q[0], levels) and scale[0, 0] == step and lo[0, 0] == base
+    assert np.array_equal(orc.rtn_dequantize_groups(q, scale, lo)[0], w[0].astype(np.float64))
+    # a value 0.4 of a step above a grid point rounds down, 0.6 rounds up
+    w2 = w.copy()
+    w2[0, 8] = base + np.float32(2.4) * step
+    w2[0, 9] = base + np.float32(2.6) * step
+    q2, _, _ = orc.rtn_quantize_groups(w2, 3)
+    assert q2[0, 8] == 2 and q2[0, 9] == 3
+
+
+def test_rtn_groups_are_independent_and_run_along_the_last_axis(rng):
+    w = (rng.standard_normal((4, 256)) * 0.02).astype(np.float32)
+    q0, s0, l0 = orc.rtn_quantize_groups(w, 3)
+    w1 = w.copy()
+    w1[2, 130] = 5.0                       # an outlier in row 2, second group
+    q1, s1, l1 = orc.rtn_quantize_groups(w1, 3)
+    same = np.ones((4, 2), dtype=bool)
+    same[2, 1] = False
+    assert np.array_equal(s1[same], s0[same]) and np.array_equal(l1[same], l0[same])
+    assert np.array_equal(q1[:, :128], q0[:, :128]) and np.array_equal(q1[[0, 1, 3]], q0[[0, 1, 3]])
+    assert s1[2, 1] > 10 * s0[2, 1]        # only that group's step widened
+    # each row (output channel) has its own parameters: scaling one row scales only its own steps
+    w2 = w.copy()
+    w2[1] *= 4
+    _, s2, _ = orc.rtn_quantize_groups(w2, 3)
+    assert np.allclose(s2[1], 4 * s0[1]) and np.array_equal(s2[[0, 2, 3]], s0[[0, 2, 3]])
+
+
+def test_quantize_split_axes_and_reassembly(rng):
+    """U-type matrices are grouped along d per neuron, V-type along the part's neuron axis per output column;
+    the heavy part gets 8 bits, the light part 3; reassembly puts every neuron back in its place."""
+    d, m = 160, 300
+    W1 = (rng.standard_normal((d, m)) * 0.02).astype(np.float32)
+    W2 = (rng.standard_normal((m, d)) * 0.02).astype(np.float32)
+    heavy = np.sort(rng.choice(m, 140, replace=False))
+    Q = orc.quantize_split(W1, W2, heavy)
+    ml = m - 140
+    assert Q["U1"][0].shape == (140, d) and Q["U1"][1].shape == (140, 2)         # ceil(160 / 128) groups along d
+    assert Q["V1"][0].shape == (d, 140) and Q["V1"][1].shape == (d, 2)           # ceil(140 / 128) groups along heavy neurons
+    assert Q["U2"][0].shape == (ml, d) and Q["V2"][1].shape == (d, 2)
+    assert Q["U1"][0].max() > 7 and Q["V1"][0].max() > 7 and Q["U2"][0].max() <= 7 and Q["V2"][0].max() <= 7
+    W1q, W2q, _ = orc.dequantized_weights(Q, d, m)
+    light = Q["light"]
+    # 8-bit steps are 255/7 times finer than 3-bit ones on the same kind of data
+    e_h = np.abs(W1q[:, heavy] - W1[:, heavy]).max()
+    e_l = np.abs(W1q[:, light] - W1[:, light]).max()
+    assert e_h < e_l / 10
+    step_u2 = Q["U2"][1]
+    assert np.all(np.abs(W1q[:, light].T - W1[:, light].T) <= 0.5 * step_u2[:, np.arange(d) // 128] * (1 + 1e-5) + 1e-12)
+    step_v1 = Q["V1"][1]
+    assert np.all(np.abs(W2q[heavy, :].T - W2[heavy, :].T) <= 0.5 * step_v1[:, np.arange(140) // 128] * (1 + 1e-5) + 1e-12)
+    # the V groups follow the part's own neuron order: rows of V[heavy] number 128.. form the second group
+    assert np.allclose(Q["V1"][2][:, 1], W2[heavy[128:], :].min(axis=0))
+    assert np.allclose(Q["U1"][2][:, 1], W1[128:, heavy].min(axis=0))
+
+
+def test_quant_split_ffn_is_the_dense_ffn_of_the_dequantised_weights_and_converges_with_bits(rng):
+    d, m, T = 96, 200, 9
+    W1 = rng.standard_normal((d, m)) * 0.05
+    W2 = rng.standard_normal((m, d)) * 0.05
+    b1 = rng.standard_normal(m) * 0.1
+    b2 = rng.standard_normal(d) * 0.1
+    X = rng.standard_normal((T, d))
+    heavy = np.sort(rng.choice(m, 30, replace=False))
+    ref = orc.dense_ffn(X, W1.astype(np.float32), b1, W2.astype(np.float32), b2, "gelu_erf")
+    errs = []
+    for bl in (2, 3, 4, 6, 8):
+        Q = orc.quantize_split(W1, W2, heavy, bits_heavy=8, bits_light=bl)
+        Y = orc.quant_split_ffn(X, b1, b2, Q, d, m, "gelu_erf")
+        # written out with explicit sums over the two parts (Eq. 2), neuron by neuron
+        W1q, W2q, _ = orc.dequantized_weights(Q, d, m)
+        Y2 = np.tile(b2, (T, 1))
+        for j in range(m):
+            Y2 += np.outer(orc.gelu_erf(X @ W1q[:, j] + b1[j]), W2q[j, :])
+        assert np.allclose(Y, Y2, rtol=1e-12, atol=1e-12)
+        errs.append(orc.rel_frobenius(Y, ref))
+    assert all(errs[i + 1] < 0.75 * errs[i] for i in range(len(errs) - 1))     # about a factor two per bit
+    assert errs[-1] < 0.02
+    # SwiGLU: the up projection is quantised like the gate
+    W1u = rng.standard_normal((d, m)) * 0.05
+    Q = orc.quantize_split(W1, W2, heavy, W1u=W1u)
+    W1q, W2q, W1uq = orc.dequantized_weights(Q, d, m)
+    Y = orc.quant_split_ffn(X, None, None, Q, d, m, "swiglu")
+    assert np.allclose(Y, (orc.silu(X @ W1q) * (X @ W1uq)) @ W2q, rtol=1e-12, atol=1e-14)
+
+
+def test_quant_weight_bytes_formula_counts_codes_and_group_parameters():
+    d, m, k = 5120, 20480, 1024
+    got = orc.quant_weight_bytes(d, m, k)
+    ml = m - k
+    codes = (2 * k * d * 8 + 2 * ml * d * 3) / 8
+    params = 8 * (k * 40 + d * 8 + ml * 40 + d * 152)
+    assert got == codes + params
+    # 3.25-3.5 bits per weight overall at 5 % heavy: about a fifth of the bf16 layer
+    assert 0.21 < got / (2 * 2 * d * m) < 0.24
+    assert orc.quant_weight_bytes(256, 1024, 0) == (2 * 1024 * 256 * 3) / 8 + 8 * (1024 * 2 + 256 * 8)
