@@ -426,7 +426,7 @@ ffsplit_status ffsplit_create(ffsplit_ctx** out, int device) {
   c->num_sms = sms;
   if (const char* env = std::getenv("FFSPLIT_GEMM_TWO_M")) c->gemm_two_m = env[0] == '0' ? 0 : env[0] == '2' ? 2 : 1;
   if (const char* env = std::getenv("FFSPLIT_DECODE_LAYER")) c->decode_one_launch = env[0] == '0' ? 0 : 1;
-  if (const char* env = std::getenv("FFSPLIT_DECODE_STREAM")) c->decode_stream = env[0] == '0' ? 0 : 1;
+  if (const char* env = std::getenv("FFSPLIT_DECODE_STREAM")) c->decode_stream = env[0] == '0' ? 0 : env[0] == '2' ? 2 : 1;
   *out = c;
   return FFSPLIT_OK;
 }

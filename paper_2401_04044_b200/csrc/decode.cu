@@ -22,9 +22,28 @@ constexpr long long kDecodeScratchBytes = 16ll << 20;   // fp32 partials of the 
 // Every phase writes raw fp32 sums (one slice per k range); the phase that reads them adds the slices, the
 // bias and the activation.  Returns FFSPLIT_ERR_BUFFER_TOO_SMALL without launching when `scratch_bytes`
 // cannot hold the slices (the caller then takes the other few-token kernel).
-static int stream_splits(int K) {
-  const int k32 = (K + 31) / 32, cap = kStreamKxMax / 32;
-  return (k32 + cap - 1) / cap;
+// k ranges for a contraction of length K over `rows` output rows: at least as many as the activation operand's
+// capacity demands.  One k range lets the phase finish its outputs itself (bias, activation, bf16), so more are
+// taken only when the row shares would come out badly uneven over the CTAs of a phase that is big enough for
+// that to matter.
+static int stream_splits(int K, long long rows, int kx_max, int ncta) {
+  const int k32 = (K + 31) / 32, cap = kx_max / 32;
+  const int s_min = k32 <= cap ? 1 : (k32 + cap - 1) / cap;
+  auto waste = [&](int s) {
+    const long long U = rows * s;
+    return static_cast<double>((U + ncta - 1) / ncta) * ncta / static_cast<double>(U > 0 ? U : 1);
+  };
+  const double bytes_per_cta = 2.0 * static_cast<double>(rows) * K / ncta;
+  if (bytes_per_cta < 49152.0 || waste(s_min) <= 1.08) return s_min;
+  int best = s_min;
+  double best_waste = waste(s_min);
+  for (int s = s_min + 1; s < s_min + 4 && s <= k32; ++s) {
+    if ((k32 + s - 1) / s > cap) continue;
+    const double w = waste(s);
+    if (w < best_waste - 1e-9) { best_waste = w; best = s; }
+    if (w <= 1.03) break;
+  }
+  return best;
 }
 
 static ffsplit_status stream_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* blob, const void* X, int T,
@@ -37,45 +56,66 @@ static ffsplit_status stream_forward(ffsplit_ctx* ctx, const BlobHeader& h, cons
   const int g2 = gated ? 2 : 1;
   auto W = [&](int sec) { return reinterpret_cast<const __nv_bfloat16*>(blob + h.off[sec]); };
   auto F = [&](int sec) { return reinterpret_cast<const float*>(blob + h.off[sec]); };
-  // slices in the scratch area
-  const int S1 = stream_splits(d), S2a = stream_splits(r_pad), S2b = stream_splits(ml_pad);
-  const int K3 = light ? kp_rp : k_pad;
-  const int S3 = stream_splits(K3);
+  const int x_rows = stream_x_rows(T), kx = stream_kx_max(x_rows), G = ctx->num_sms;
   const long long N1 = static_cast<long long>(g2) * (k_pad + (light ? r_pad : 0));
   const long long N2a = static_cast<long long>(g2) * ml_pad;
+  const int K3 = light ? kp_rp : k_pad;
+  const int S1 = stream_splits(d, N1, kx, G), S2a = stream_splits(r_pad, N2a, kx, G);
+  const int S2b = stream_splits(ml_pad, r_pad, kx, G);
+  // the layer output is written by the stage-3 phase itself when its contraction fits one k range
+  const int S3 = (K3 + 31) / 32 <= kx / 32 ? 1 : stream_splits(K3, d, kx, G);
+  // A phase with one k range whose outputs are not gated pairs finishes them itself (bf16); the others leave
+  // raw fp32 slices for their readers.
+  const bool fin1 = S1 == 1 && !gated, fin2a = S2a == 1 && !gated, fin2b = S2b == 1;
+  // the unit arithmetic of the kernel is 32-bit
+  for (long long u : {S1 * N1, S2a * N2a, static_cast<long long>(S2b) * r_pad, static_cast<long long>(S3) * d})
+    if (u * (G + 1) >= 2147483648ll) return FFSPLIT_ERR_BUFFER_TOO_SMALL;
+  // slices and finished vectors in the scratch area (256-byte aligned pieces)
   long long off = 0;
-  auto take = [&](long long slices, long long cols) { const long long o = off; off += slices * 8 * cols; return o; };
-  const long long o_p1 = take(S1, N1);
-  const long long o_2a = light ? take(S2a, N2a) : 0;
-  const long long o_2b = light ? take(S2b, r_pad) : 0;
-  const long long o_y = S3 > 1 ? take(S3, d) : 0;
-  if (off * 4 > scratch_bytes) return FFSPLIT_ERR_BUFFER_TOO_SMALL;
-  float* fs = reinterpret_cast<float*>(scratch);
+  auto take = [&](long long bytes) { const long long o = off; off += (bytes + 255) / 256 * 256; return o; };
+  const long long o_p1 = take(fin1 ? 8 * N1 * 2 : S1 * 8 * N1 * 4);
+  const long long o_2a = light ? take(fin2a ? 8 * N2a * 2 : S2a * 8 * N2a * 4) : 0;
+  const long long o_2b = light ? take(fin2b ? 8ll * r_pad * 2 : static_cast<long long>(S2b) * 8 * r_pad * 4) : 0;
+  const long long o_y = S3 > 1 ? take(static_cast<long long>(S3) * 8 * d * 4) : 0;
+  if (off > scratch_bytes) return FFSPLIT_ERR_BUFFER_TOO_SMALL;
+  auto FS = [&](long long o) { return reinterpret_cast<float*>(scratch + o); };
+  auto BS = [&](long long o) { return reinterpret_cast<__nv_bfloat16*>(scratch + o); };
 
   StreamParams p;
   std::memset(&p, 0, sizeof(p));
   p.T = T; p.act = h.act; p.ctrl = ctrl;
+  p.x_rows = x_rows; p.x_pitch = 2 * kx + 64;
   p.guard = guard_hash ? reinterpret_cast<const unsigned long long*>(blob) : nullptr;
   p.guard_hash = guard_hash;
-  auto add_seg = [](StreamPhase& ph, const __nv_bfloat16* Wp, long long ldw, int rows, int x_off, int out_col) {
+  auto add_seg = [](StreamPhase& ph, const __nv_bfloat16* Wp, long long ldw, int rows, int x_off, int out_col,
+                    int fin_kind = STREAM_IN_LINEAR, const float* fin_bias = nullptr) {
     if (rows <= 0) return;
     StreamSegment& s = ph.seg[ph.nseg++];
     s.W = Wp; s.ldw = ldw; s.rows = rows; s.x_off = x_off; s.out_col = out_col;
+    s.fin_kind = fin_kind; s.fin_bias = fin_bias;
     ph.Nall += rows;
   };
-  auto slices_in = [](StreamPhase& ph, int c0, int c1, int kind, const float* src, int nsl, long long ld, int src_col,
-                      int gate_off, const float* bias) {
+  // columns [c0, c1) of a phase's activation matrix from what an earlier phase left: finished bf16 values
+  // (`fin`) or `nsl` raw slices to be added, biased and activated as `kind` says
+  auto feed = [](StreamPhase& ph, int c0, int c1, bool fin, int kind, const void* src, int nsl, long long ld,
+                 int src_col, int gate_off, const float* bias) {
     if (c1 <= c0) return;
     StreamInPart& in = ph.in[ph.nin++];
-    in.col_begin = c0; in.col_end = c1; in.kind = kind; in.nslices = nsl; in.src = src; in.ld = ld;
-    in.slice_stride = 8 * ld; in.src_col = src_col; in.gate_off = gate_off; in.bias = bias;
+    in.col_begin = c0; in.col_end = c1; in.kind = fin ? STREAM_IN_BF16 : kind; in.nslices = fin ? 1 : nsl;
+    in.src = src; in.ld = ld; in.slice_stride = 8 * ld; in.src_col = src_col; in.gate_off = gate_off;
+    in.bias = fin ? nullptr : bias;
   };
-  // ---- stage 1: z_H = X U1 and Q = X A1 (SwiGLU: gate and up of each), raw
+  auto set_out = [&](StreamPhase& ph, bool fin, long long o, long long ld) {
+    if (fin) ph.outb = BS(o); else ph.out = FS(o);
+    ph.out_ld = ld;
+  };
+  // ---- stage 1: z_H = X U1 (+ b1[h2], sigma when finished here) and Q = X A1 (SwiGLU: gate and up of each)
   {
     StreamPhase& ph = p.ph[p.nph++];
     ph.K = d; ph.S = S1;
     if (!gated) {
-      add_seg(ph, W(SEC_U1T), d, light ? kp_rp : k_pad, 0, 0);     // U1^T and A1^T are adjacent with the same pitch
+      add_seg(ph, W(SEC_U1T), d, k_pad, 0, 0, STREAM_IN_ACT, F(SEC_B1H));
+      if (light) add_seg(ph, W(SEC_A1T), d, r_pad, 0, k_pad);
     } else {
       add_seg(ph, W(SEC_U1T), d, k_pad, 0, 0);
       add_seg(ph, W(SEC_U1UT), d, k_pad, 0, k_pad);
@@ -83,40 +123,40 @@ static ffsplit_status stream_forward(ffsplit_ctx* ctx, const BlobHeader& h, cons
     }
     StreamInPart& in = ph.in[ph.nin++];
     in.col_begin = 0; in.col_end = d; in.kind = STREAM_IN_BF16; in.src = X; in.ld = d;
-    ph.out = fs + o_p1; ph.out_ld = N1;
+    set_out(ph, fin1, o_p1, N1);
   }
   const int q_col = g2 * k_pad;   // where Q starts among stage 1's output columns
+  const void* p1 = scratch + o_p1;
   if (light) {
-    // ---- stage 2a: z_L = Q B1 (raw)
+    // ---- stage 2a: z_L = Q B1 (+ b1[light], sigma when finished here)
     StreamPhase& a = p.ph[p.nph++];
     a.K = r_pad; a.S = S2a;
-    add_seg(a, W(SEC_B1T), r_pad, ml_pad, 0, 0);
+    add_seg(a, W(SEC_B1T), r_pad, ml_pad, 0, 0, STREAM_IN_ACT, gated ? nullptr : F(SEC_B1L));
     if (gated) add_seg(a, W(SEC_B1UT), r_pad, ml_pad, r_pad, ml_pad);
-    slices_in(a, 0, g2 * r_pad, STREAM_IN_LINEAR, fs + o_p1, S1, N1, q_col, 0, nullptr);
-    a.out = fs + o_2a; a.out_ld = N2a;
-    // ---- stage 2b: P = sigma(z_L + b1[light]) A2 (raw)
+    feed(a, 0, g2 * r_pad, fin1, STREAM_IN_LINEAR, p1, S1, N1, q_col, 0, nullptr);
+    set_out(a, fin2a, o_2a, N2a);
+    // ---- stage 2b: P = sigma(z_L + b1[light]) A2
     StreamPhase& b = p.ph[p.nph++];
     b.K = ml_pad; b.S = S2b;
     add_seg(b, W(SEC_A2T), ml_pad, r_pad, 0, 0);
-    slices_in(b, 0, ml_pad, gated ? STREAM_IN_GATED : STREAM_IN_ACT, fs + o_2a, S2a, N2a, 0, ml_pad,
-              gated ? nullptr : F(SEC_B1L));
-    b.out = fs + o_2b; b.out_ld = r_pad;
+    feed(b, 0, ml_pad, fin2a, gated ? STREAM_IN_GATED : STREAM_IN_ACT, scratch + o_2a, S2a, N2a, 0, ml_pad,
+         gated ? nullptr : F(SEC_B1L));
+    set_out(b, fin2b, o_2b, r_pad);
   }
   // ---- stage 3: Y = [sigma(z_H + b1[h2]) | P] [V1 ; B2] + b2
   {
     StreamPhase& ph = p.ph[p.nph++];
     ph.K = K3; ph.S = S3;
     add_seg(ph, W(SEC_V1B2T), kp_rp, d, 0, 0);
-    slices_in(ph, 0, k_pad, gated ? STREAM_IN_GATED : STREAM_IN_ACT, fs + o_p1, S1, N1, 0, k_pad,
-              gated ? nullptr : F(SEC_B1H));
-    if (light) slices_in(ph, k_pad, kp_rp, STREAM_IN_LINEAR, fs + o_2b, S2b, r_pad, 0, 0, nullptr);
+    feed(ph, 0, k_pad, fin1, gated ? STREAM_IN_GATED : STREAM_IN_ACT, p1, S1, N1, 0, k_pad, gated ? nullptr : F(SEC_B1H));
+    if (light) feed(ph, k_pad, kp_rp, fin2b, STREAM_IN_LINEAR, scratch + o_2b, S2b, r_pad, 0, 0, nullptr);
     if (S3 == 1) {
       ph.y = static_cast<__nv_bfloat16*>(Y); ph.y_ld = d; ph.y_bias = F(SEC_B2); ph.y_cols = d;
     } else {
-      ph.out = fs + o_y; ph.out_ld = d;
+      ph.out = FS(o_y); ph.out_ld = d;
       StreamPhase& rd = p.ph[p.nph++];
       rd.kind = 1;
-      slices_in(rd, 0, d, STREAM_IN_LINEAR, fs + o_y, S3, d, 0, 0, nullptr);
+      feed(rd, 0, d, false, STREAM_IN_LINEAR, scratch + o_y, S3, d, 0, 0, nullptr);
       rd.y = static_cast<__nv_bfloat16*>(Y); rd.y_ld = d; rd.y_bias = F(SEC_B2); rd.y_cols = d;
     }
   }
@@ -143,7 +183,15 @@ static ffsplit_status decode_forward_impl(ffsplit_ctx* ctx, const BlobHeader& h,
                                           cudaStream_t st, int* tickets, long long scratch_bytes,
                                           unsigned long long guard_hash) {
   const int T = static_cast<int>(T64);
-  if (T <= 8 && ctx->decode_stream) {
+  // Which of the two few-token kernels: the single-launch streaming kernel wins where a layer's weights are
+  // many megabytes and the activation operand of a pass fits four token rows (measured, 1 token: OPT-13B-shaped
+  // split layer 38 vs 42 us, Llama-2-7B-shaped 45 vs 51 us, their dense layers 86 vs 85 and 55 vs 61 us; at
+  // 5 to 8 tokens the per-product kernel is ahead, 43 vs 64 us, and so it is on layers of a few megabytes, whose
+  // time is all hand-over: GPT-2-medium-shaped split layer 17 vs 20 us).  FFSPLIT_DECODE_STREAM=2 forces the
+  // streaming kernel for every T <= 8, 0 turns it off.
+  const double layer_bytes = 2.0 * (h.n_in + 1) * (static_cast<double>(h.d) * h.k + static_cast<double>(h.r) * (h.d + h.ml));
+  const bool stream = ctx->decode_stream == 2 || (ctx->decode_stream == 1 && T <= 4 && layer_bytes >= 16e6);
+  if (T <= 8 && stream) {
     // one persistent launch whose weight stream runs ahead of the stage dependencies; its slices take the whole
     // scratch area (the [A_H | P], Q and H_L buffers of the other kernel are not used)
     bool launched = false;

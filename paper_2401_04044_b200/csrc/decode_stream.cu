@@ -6,11 +6,13 @@
 // chain, stage 3) of a few megabytes each.  What bounds such a layer is not bandwidth but the hand-over
 // between dependent products.  This kernel is built around two facts:
 //
-//  * The weights do not depend on the activations.  One warp per CTA (the producer) walks the CTA's share of
-//    ALL phases of the layer and copies it into a ring of shared-memory stages with bulk asynchronous copies
-//    (cp.async.bulk, one 512-byte row segment per lane and instruction, completion counted on an mbarrier).
-//    It never waits for a grid barrier: while the consumers wait for the previous phase to finish everywhere,
-//    the next phase's weights are already landing, and HBM stays busy as long as the ring has a free stage.
+//  * The weights do not depend on the activations.  Producer warps walk the CTA's share of ALL phases of the
+//    layer and copy it into a ring of shared-memory stages with asynchronous copies (cp.async, 16 bytes per
+//    lane: one warp-wide instruction moves 512 contiguous bytes of one weight row; completion is counted on
+//    the stage's mbarrier).  They never wait for a grid barrier: while the consumers wait for the previous
+//    phase to finish everywhere, the next phase's weights are already landing, and HBM stays busy as long as
+//    the ring has a free stage.  (Bulk copies, cp.async.bulk, of one 512-byte row segment each measured
+//    1.9 TB/s on this path: about 77 clocks per copy whatever its size.)
 //  * Eq. 1: output rows (neurons, or output columns of V) are independent.  Every phase's rows -- times a
 //    small number S of k ranges when K is long -- are dealt to the CTAs in equal contiguous shares with
 //    single-row granularity, so the load balance does not depend on tile shapes.  Inside a CTA the eight
@@ -40,13 +42,12 @@ using namespace dec;
 
 constexpr int CWARPS = 8;                                // consumer warps
 constexpr int CTHREADS = 32 * CWARPS;
-constexpr int THREADS = CTHREADS + 32;                   // + the producer warp
-constexpr int BLOCK_ROWS = 32;                           // weight rows per stage: one bulk copy per lane
-constexpr int KC = 256;                                  // k elements per stage: 512 contiguous bytes per row
-constexpr int STAGE_BYTES = BLOCK_ROWS * ROW_PITCH;      // 18432
+constexpr int PWARPS = 4;                                // producer warps: stage i is filled by warp i mod 4
+constexpr int THREADS = CTHREADS + 32 * PWARPS;
+constexpr int BLOCK_ROWS = 32;                           // weight rows per stage, at most
+constexpr int STAGE_BYTES = kStreamStageBytes;           // 18432
 constexpr int NSTAGE = 9;
-constexpr int X_PITCH = kStreamKxMax * 2 + 64;           // bytes between token rows of the activation operand
-constexpr int X_BYTES = 8 * X_PITCH;
+constexpr int X_BYTES = kStreamXBytes;                   // activation operand of a pass: x_rows token rows, x_pitch apart
 constexpr int RED_TOK = 36;                              // floats between token rows of a warp's partial block
 constexpr int RED_WARP = 8 * RED_TOK;
 constexpr int RED_BYTES = 2 * CWARPS * RED_WARP * 4;     // two buffers, used alternately
@@ -54,174 +55,226 @@ constexpr int OFF_X = NSTAGE * STAGE_BYTES;
 constexpr int OFF_RED = OFF_X + X_BYTES;
 constexpr int OFF_BAR = OFF_RED + RED_BYTES;
 constexpr int SMEM_BYTES = OFF_BAR + 256;
-static_assert(X_PITCH % 128 == 64 && ROW_PITCH % 128 == 64, "conflict-free 128-bit fragment reads");
 static_assert(SMEM_BYTES <= 232448, "shared memory plan");
-constexpr int kBarCount = 16, kBarGen = 17;              // words of the control block used by the grid barrier
+constexpr int kBarTicket = 18;                           // words 18-19 of the control block: the grid barrier's 64-bit ticket counter
 constexpr long long kWaitLimit = 2000000000ll;           // SM clocks (about a second)
 
 __device__ __forceinline__ void cbar() { asm volatile("bar.sync 1, %0;" ::"n"(CTHREADS) : "memory"); }
 
-// ---- the walk over a CTA's share of one phase, taken identically by the producer and the consumers -----
+// ---- the walk over a CTA's share of one phase, taken identically by the producers and the consumers -----
+// (32-bit arithmetic: the host checks S * Nall * (grid + 1) < 2^31 when it plans a phase)
 struct Pass {
   int seg, s;          // segment, k range
   int row0, rows;      // rows [row0, row0 + rows) of the segment
   int kbeg, klen;      // k range in elements
 };
-struct Share { long long lo, hi; };   // units [lo, hi) of the phase: unit = s * Nall + row
+struct Share { unsigned lo, hi; };   // units [lo, hi) of the phase: unit = s * Nall + row
 
-__device__ __forceinline__ Share share_of(const StreamPhase& ph, int cta, int ncta) {
-  const long long U = static_cast<long long>(ph.S) * ph.Nall;
+__device__ __forceinline__ Share share_of(const StreamPhase& ph, unsigned cta, unsigned ncta) {
+  const unsigned U = static_cast<unsigned>(ph.S) * ph.Nall;
   Share sh;
   sh.lo = U * cta / ncta;
   sh.hi = U * (cta + 1) / ncta;
   return sh;
 }
 // the pass that starts at unit u (u < hi)
-__device__ __forceinline__ Pass pass_at(const StreamPhase& ph, long long u, long long hi) {
+__device__ __forceinline__ Pass pass_at(const StreamPhase& ph, unsigned u, unsigned hi) {
   Pass p;
-  p.s = static_cast<int>(u / ph.Nall);
-  const int row = static_cast<int>(u - static_cast<long long>(p.s) * ph.Nall);
+  const unsigned nall = ph.Nall;
+  p.s = static_cast<int>(u / nall);
+  const int row = static_cast<int>(u - p.s * nall);
   int j = 0, start = 0;
   while (j + 1 < ph.nseg && row >= start + ph.seg[j].rows) { start += ph.seg[j].rows; ++j; }
   p.seg = j;
   p.row0 = row - start;
-  long long end = static_cast<long long>(p.s) * ph.Nall + start + ph.seg[j].rows;   // end of the segment in this k range
+  unsigned end = p.s * nall + start + ph.seg[j].rows;   // end of the segment in this k range
   if (end > hi) end = hi;
   p.rows = static_cast<int>(end - u);
-  const int k32 = (ph.K + 31) / 32;
-  p.kbeg = 32 * static_cast<int>(static_cast<long long>(p.s) * k32 / ph.S);
-  const int kend = p.s + 1 == ph.S ? ph.K : 32 * static_cast<int>(static_cast<long long>(p.s + 1) * k32 / ph.S);
+  const unsigned k32 = (ph.K + 31) / 32;
+  p.kbeg = 32 * static_cast<int>(p.s * k32 / ph.S);
+  const int kend = p.s + 1 == ph.S ? ph.K : 32 * static_cast<int>((p.s + 1) * k32 / ph.S);
   p.klen = kend - p.kbeg;
   return p;
 }
 // rows of a pass are cut into blocks of at most 32 rows of nearly equal size
 __device__ __forceinline__ int blocks_of(int rows) { return (rows + BLOCK_ROWS - 1) / BLOCK_ROWS; }
-__device__ __forceinline__ int block_lo(int rows, int nb, int b) { return static_cast<int>(static_cast<long long>(rows) * b / nb); }
+__device__ __forceinline__ int block_lo(int rows, int nb, int b) { return rows * b / nb; }
 
-// ---- producer ---------------------------------------------------------------------------------------
-__device__ void producer(const StreamParams& p, uint32_t ring, uint64_t* full, uint64_t* empty, volatile int* s_abort) {
+// ---- producers -------------------------------------------------------------------------------------
+// 16 bytes per lane of each of `nr` rows (src_step bytes apart; a lane outside the k range copies nothing and its
+// 16 bytes are zero filled)
+__device__ __forceinline__ void issue_rows(uint32_t dst, int dst_pitch, const char* src, long long src_step, int nr,
+                                           bool valid) {
+  int r = 0;
+#pragma unroll 1
+  for (; r + 4 <= nr; r += 4) {
+    cp_async16(dst, src, valid);
+    cp_async16(dst + dst_pitch, src + src_step, valid);
+    cp_async16(dst + 2 * dst_pitch, src + 2 * src_step, valid);
+    cp_async16(dst + 3 * dst_pitch, src + 3 * src_step, valid);
+    dst += 4 * dst_pitch;
+    src += 4 * src_step;
+  }
+  for (; r < nr; ++r, dst += dst_pitch, src += src_step) cp_async16(dst, src, valid);
+}
+
+__device__ void producer(const StreamParams& p, uint32_t ring, uint64_t* full, uint64_t* empty, volatile int* s_abort,
+                         int pw) {
   const int lane = threadIdx.x & 31;
+  if (pw == 0 && blockIdx.x == 0) {
+    Epilogue e;
+    e.guard = p.guard;
+    e.guard_hash = p.guard_hash;
+    check_blob_guard(e, p.ctrl, KID_DECODE);
+  }
   uint32_t it = 0;
   bool ok = true;
   for (int pi = 0; pi < p.nph && ok; ++pi) {
     const StreamPhase& ph = p.ph[pi];
     if (ph.kind != 0) continue;
     const Share sh = share_of(ph, blockIdx.x, gridDim.x);
-    for (long long u = sh.lo; u < sh.hi && ok;) {
+    for (unsigned u = sh.lo; u < sh.hi && ok;) {
       const Pass ps = pass_at(ph, u, sh.hi);
       const StreamSegment& sg = ph.seg[ps.seg];
       const int nb = blocks_of(ps.rows);
-      const int nch = (ps.klen + KC - 1) / KC;
+      const long long pitch = sg.ldw * 2;
       for (int b = 0; b < nb && ok; ++b) {
         const int r_lo = block_lo(ps.rows, nb, b), r_hi = block_lo(ps.rows, nb, b + 1);
-        const char* src = reinterpret_cast<const char*>(sg.W) +
-                          (static_cast<long long>(ps.row0 + r_lo + lane) * sg.ldw + ps.kbeg) * 2;
+        const int sub = stream_stage_sub(r_hi - r_lo);
+        const int chunk = 512 * sub, row_pitch = chunk + 64;
+        const int nch = (2 * ps.klen + chunk - 1) / chunk;
+        const char* base = reinterpret_cast<const char*>(sg.W) +
+                           (static_cast<long long>(ps.row0 + r_lo) * sg.ldw + ps.kbeg) * 2 + lane * 16;
         for (int ch = 0; ch < nch; ++ch, ++it) {
+          if (static_cast<int>(it % PWARPS) != pw) continue;
           const int slot = it % NSTAGE;
           // every lane waits; lane 0's verdict is taken by all, so that the warp stays together
           const bool got = ptx::mbar_wait_limit(&empty[slot], ((it / NSTAGE) & 1) ^ 1, s_abort, kWaitLimit);
           if (__shfl_sync(0xffffffffu, got ? 1 : 0, 0) == 0) { ok = false; break; }
-          const int bytes = 2 * (ps.klen - ch * KC < KC ? ps.klen - ch * KC : KC);
-          if (lane == 0) ptx::mbar_expect_tx(&full[slot], static_cast<uint32_t>((r_hi - r_lo) * bytes));
-          __syncwarp();
-          if (lane < r_hi - r_lo) {
-            asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
-                             ring + slot * STAGE_BYTES + lane * ROW_PITCH),
-                         "l"(src + ch * (KC * 2)), "r"(bytes), "r"(ptx::smem_u32(&full[slot]))
-                         : "memory");
+          const int bytes = 2 * ps.klen - ch * chunk < chunk ? 2 * ps.klen - ch * chunk : chunk;   // multiple of 16
+          const char* src0 = base + static_cast<long long>(ch) * chunk;
+          const uint32_t dst0 = ring + slot * STAGE_BYTES + lane * 16;
+          for (int j = 0; j < sub && j * 512 < bytes; ++j) {
+            // one 512-byte piece of every row of the block: a warp-wide copy per row, four rows per turn
+            const bool valid = j * 512 + lane * 16 < bytes;
+            issue_rows(dst0 + j * 512, row_pitch, valid ? src0 + j * 512 : reinterpret_cast<const char*>(sg.W),
+                       valid ? pitch : 0, r_hi - r_lo, valid);
           }
+          asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(ptx::smem_u32(&full[slot])) : "memory");
         }
       }
       u += ps.rows;
     }
   }
-  if (!ok) {
-    // give the copies already issued a bounded chance to land before the CTA exits
-    const uint32_t first = it > NSTAGE ? it - NSTAGE : 0;
-    for (uint32_t j = first; j < it; ++j) {
-      const long long t0 = clock64();
-      while (!ptx::mbar_try_wait(&full[j % NSTAGE], (j / NSTAGE) & 1) && clock64() - t0 < kWaitLimit / 8) {}
-    }
-  }
+  // on every way out: this thread's copies have landed before the CTA may exit
+  asm volatile("cp.async.wait_all;" ::: "memory");
 }
 
 // ---- consumers ----------------------------------------------------------------------------------------
-// One value of a phase's activation matrix from its source: the layer input as it is, or the raw sums of an
-// earlier phase with their slices added in order, bias, activation.
+// Four columns of a phase's activation matrix from raw sums of an earlier phase: the slices added in order.
+// The loads of up to four slices are in flight together.
 __device__ __forceinline__ float4 load_sum4(const StreamInPart& in, int t, long long col) {
   const float* base = static_cast<const float*>(in.src) + static_cast<long long>(t) * in.ld + col;
   float4 a = __ldcg(reinterpret_cast<const float4*>(base));
-  for (int s = 1; s < in.nslices; ++s) {
-    const float4 b = __ldcg(reinterpret_cast<const float4*>(base + s * in.slice_stride));
-    a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+  for (int s0 = 1; s0 < in.nslices; s0 += 4) {
+    float4 b[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      b[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (s0 + j < in.nslices) b[j] = __ldcg(reinterpret_cast<const float4*>(base + (s0 + j) * in.slice_stride));
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      if (s0 + j < in.nslices) { a.x += b[j].x; a.y += b[j].y; a.z += b[j].z; a.w += b[j].w; }
   }
   return a;
 }
 
-// Activation operand of a pass: columns [c0, c0 + klen) of the phase's activation matrix for tokens 0..7
-// (rows beyond T are zero), bf16, token rows X_PITCH bytes apart.  Four columns per thread and step.
-__device__ void build_x(const StreamPhase& ph, int T, int act, int c0, int klen, unsigned char* xbuf) {
+// Activation operand of a pass: columns [c0, c0 + klen) of the phase's activation matrix for tokens
+// 0 .. x_rows - 1 (rows beyond T are zero), bf16, token rows X_PITCH bytes apart.  Four columns per thread and
+// element.  Values that an earlier phase finished (or the layer input) are copied asynchronously as they are;
+// raw sums are added, biased, activated and rounded here, eight elements' loads in flight per thread.
+__device__ void build_x(const StreamPhase& ph, int T, int act, int c0, int klen, unsigned char* xbuf, uint32_t xs0,
+                        int x_rows, int X_PITCH) {
   const GeluCoef gc = gelu_coef(act);
   const int tid = threadIdx.x;
   const int groups = (klen + 3) >> 2;          // klen is a multiple of 8
-  for (int e = tid; e < 8 * groups; e += CTHREADS) {
-    const int t = e / groups, q = e - t * groups;
-    const int col = c0 + 4 * q;
-    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (t < T) {
+  constexpr int B = 8;
+  const int total = x_rows * groups;
+  for (int e0 = tid; e0 < total; e0 += B * CTHREADS) {
+    float4 v[B], u[B];
+    int kind[B];
+#pragma unroll
+    for (int j = 0; j < B; ++j) {
+      const int e = e0 + j * CTHREADS;
+      v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+      u[j] = v[j];
+      kind[j] = -1;                              // nothing to do, or a zero row
+      if (e >= total) continue;
+      const int t = e / groups, q = e - t * groups;
+      kind[j] = -2;                              // zero row
+      if (t >= T) continue;
+      const int col = c0 + 4 * q;
       const StreamInPart& in = (ph.nin > 1 && col >= ph.in[1].col_begin) ? ph.in[1] : ph.in[0];
       const long long sc = in.src_col + (col - in.col_begin);
+      kind[j] = in.kind;
       if (in.kind == STREAM_IN_BF16) {
-        const uint2 raw = __ldg(reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(in.src) +
-                                                               static_cast<long long>(t) * in.ld + sc));
-        *reinterpret_cast<uint2*>(xbuf + t * X_PITCH + 8 * q) = raw;
-        continue;
-      }
-      v = load_sum4(in, t, sc);
-      if (in.kind == STREAM_IN_GATED) {
-        const float4 u = load_sum4(in, t, sc + in.gate_off);
-        v.x = silu_fast(v.x) * u.x; v.y = silu_fast(v.y) * u.y; v.z = silu_fast(v.z) * u.z; v.w = silu_fast(v.w) * u.w;
+        const __nv_bfloat16* src = static_cast<const __nv_bfloat16*>(in.src) + static_cast<long long>(t) * in.ld + sc;
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(xs0 + t * X_PITCH + 8 * q), "l"(src) : "memory");
       } else {
-        if (in.bias) {
-          const float4 b = __ldg(reinterpret_cast<const float4*>(in.bias + (col - in.col_begin)));
-          v.x += b.x; v.y += b.y; v.z += b.z; v.w += b.w;
-        }
-        if (in.kind == STREAM_IN_ACT) {
-          v.x = gelu_fast(v.x, gc); v.y = gelu_fast(v.y, gc); v.z = gelu_fast(v.z, gc); v.w = gelu_fast(v.w, gc);
-        }
+        v[j] = load_sum4(in, t, sc);
+        if (in.kind == STREAM_IN_GATED) u[j] = load_sum4(in, t, sc + in.gate_off);
+        else if (in.bias) u[j] = __ldg(reinterpret_cast<const float4*>(in.bias + (col - in.col_begin)));
       }
     }
-    uint2 o;
-    o.x = pack_bf16x2(v.x, v.y);
-    o.y = pack_bf16x2(v.z, v.w);
-    *reinterpret_cast<uint2*>(xbuf + t * X_PITCH + 8 * q) = o;
+#pragma unroll
+    for (int j = 0; j < B; ++j) {
+      if (kind[j] == -1 || kind[j] == STREAM_IN_BF16) continue;
+      const int e = e0 + j * CTHREADS;
+      const int t = e / groups, q = e - t * groups;
+      float4 a = v[j];
+      if (kind[j] == STREAM_IN_GATED) {
+        a.x = silu_fast(a.x) * u[j].x; a.y = silu_fast(a.y) * u[j].y;
+        a.z = silu_fast(a.z) * u[j].z; a.w = silu_fast(a.w) * u[j].w;
+      } else if (kind[j] >= 0) {
+        a.x += u[j].x; a.y += u[j].y; a.z += u[j].z; a.w += u[j].w;     // bias (zero when there is none)
+        if (kind[j] == STREAM_IN_ACT) {
+          a.x = gelu_fast(a.x, gc); a.y = gelu_fast(a.y, gc); a.z = gelu_fast(a.z, gc); a.w = gelu_fast(a.w, gc);
+        }
+      }
+      uint2 o;
+      o.x = pack_bf16x2(a.x, a.y);
+      o.y = pack_bf16x2(a.z, a.w);
+      *reinterpret_cast<uint2*>(xbuf + t * X_PITCH + 8 * q) = o;
+    }
   }
+  asm volatile("cp.async.wait_all;" ::: "memory");
 }
 
-// All CTAs are resident (cooperative launch).  Called by the consumer threads; count in, the last one opens
-// the next generation.  Always arrives; gives up waiting after the limit or when the CTA has already given up.
+// All CTAs are resident (cooperative launch).  Called by the consumer threads.  One 64-bit counter that only
+// ever grows: an arrival takes a ticket v, and the barrier it belongs to is complete when the counter reaches
+// the next multiple of the grid size above v (every barrier receives exactly one arrival per CTA, so the
+// counter stays aligned from launch to launch; a run that gave up leaves it misaligned, and ffsplit_poll()
+// clears the control block when it reports that).  The arrival is a release at GPU scope, ordered after the
+// whole CTA's writes by the CTA barrier before it, and the wait ends with an acquire: no separate fences, one
+// atomic round trip on the critical path.  Always arrives; gives up waiting after the limit or when the CTA has
+// already given up.
 __device__ void grid_barrier(int* ctrl, volatile int* s_abort) {
-  __threadfence();
   cbar();
   if (threadIdx.x == 0) {
-    unsigned* count = reinterpret_cast<unsigned*>(ctrl + kBarCount);
-    unsigned* genp = reinterpret_cast<unsigned*>(ctrl + kBarGen);
-    unsigned gen;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(gen) : "l"(genp) : "memory");
-    __threadfence();
-    if (atomicAdd(count, 1u) == gridDim.x - 1) {
-      atomicExch(count, 0u);
-      __threadfence();
-      asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(genp), "r"(gen + 1) : "memory");
-    } else {
+    unsigned long long* ctr = reinterpret_cast<unsigned long long*>(ctrl + kBarTicket);
+    unsigned long long v;
+    asm volatile("atom.add.acq_rel.gpu.global.u64 %0, [%1], 1;" : "=l"(v) : "l"(ctr) : "memory");
+    const unsigned long long target = (v / gridDim.x + 1ull) * gridDim.x;
+    if (v + 1ull != target) {
       const long long t0 = clock64();
-      unsigned now = gen;
-      while (now == gen && !*s_abort) {
-        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(now) : "l"(genp) : "memory");
-        if (now == gen && clock64() - t0 > kWaitLimit) *s_abort = 1;
+      while (!*s_abort) {
+        unsigned long long now;
+        asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(now) : "l"(ctr) : "memory");
+        if (now >= target) break;
+        if (clock64() - t0 > kWaitLimit) *s_abort = 1;
       }
     }
-    __threadfence();
   }
   cbar();
 }
@@ -231,28 +284,32 @@ __device__ void consumers(const StreamParams& p, unsigned char* smem, uint32_t r
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, c = lane & 3;
   unsigned char* xbuf = smem + OFF_X;
-  const uint32_t xs = ring + OFF_X;
+  const int X_PITCH = p.x_pitch;
+  const bool my_token = g < p.x_rows;      // token rows beyond the operand's are zero
+  const uint32_t xs = ring + OFF_X + (my_token ? g * X_PITCH : 0);
   float* red = reinterpret_cast<float*>(smem + OFF_RED);
   const int kb = warp * 64 + c * 16;     // this lane's 16 bytes inside a 512-byte row segment
+  const GeluCoef gc = gelu_coef(p.act);
   uint32_t it = 0;
   unsigned flushes = 0;
-  if (blockIdx.x == 0 && warp == 0) {
-    Epilogue e;
-    e.guard = p.guard;
-    e.guard_hash = p.guard_hash;
-    check_blob_guard(e, p.ctrl, KID_DECODE);
-  }
   for (int pi = 0; pi < p.nph; ++pi) {
     const StreamPhase& ph = p.ph[pi];
+    // this CTA's share and its first pass: arithmetic only, done before the wait for the phase before
+    Share sh;
+    sh.lo = sh.hi = 0;
+    Pass ps;
+    if (ph.kind == 0) {
+      sh = share_of(ph, blockIdx.x, gridDim.x);
+      if (sh.lo < sh.hi) ps = pass_at(ph, sh.lo, sh.hi);
+    }
     if (pi > 0) grid_barrier(p.ctrl, s_abort);
     if (ph.kind != 0) {
       // ---- closing reduction: y[t, n] = sum of the slices + bias, for a share of the columns
       const StreamInPart& in = ph.in[0];
       const int q4 = ph.y_cols >> 2;
-      const long long total = static_cast<long long>(p.T) * q4;
-      for (long long e = static_cast<long long>(blockIdx.x) * CTHREADS + tid; e < total;
-           e += static_cast<long long>(gridDim.x) * CTHREADS) {
-        const int t = static_cast<int>(e / q4), n = 4 * static_cast<int>(e - static_cast<long long>(t) * q4);
+      const int total = p.T * q4;
+      for (int e = blockIdx.x * CTHREADS + tid; e < total; e += gridDim.x * CTHREADS) {
+        const int t = e / q4, n = 4 * (e - t * q4);
         float4 v = load_sum4(in, t, n);
         if (ph.y_bias) {
           const float4 b = __ldg(reinterpret_cast<const float4*>(ph.y_bias + n));
@@ -265,51 +322,76 @@ __device__ void consumers(const StreamParams& p, unsigned char* smem, uint32_t r
       }
       continue;
     }
-    const Share sh = share_of(ph, blockIdx.x, gridDim.x);
     int x_c0 = -1, x_len = -1;
-    for (long long u = sh.lo; u < sh.hi;) {
-      const Pass ps = pass_at(ph, u, sh.hi);
+    for (unsigned u = sh.lo; u < sh.hi;) {
       const StreamSegment& sg = ph.seg[ps.seg];
       // ---- the activation operand of this pass, unless the pass before left exactly it in place
       const int c0 = sg.x_off + ps.kbeg;
       if (c0 != x_c0 || ps.klen != x_len) {
         if (x_c0 >= 0) cbar();               // everyone is done with the operand of the pass before
-        build_x(ph, p.T, p.act, c0, ps.klen, xbuf);
+        build_x(ph, p.T, p.act, c0, ps.klen, xbuf, ring + OFF_X, p.x_rows, X_PITCH);
         cbar();
         x_c0 = c0; x_len = ps.klen;
       }
       const int nb = blocks_of(ps.rows);
-      const int nch = (ps.klen + KC - 1) / KC;
       for (int b = 0; b < nb; ++b) {
         const int r_lo = block_lo(ps.rows, nb, b), r_hi = block_lo(ps.rows, nb, b + 1);
-        float acc[2][4];
+        const int sub = stream_stage_sub(r_hi - r_lo);
+        const int chunk = 512 * sub, row_pitch = chunk + 64;
+        const int nch = (2 * ps.klen + chunk - 1) / chunk;
+        // Four accumulator sets per group of 16 rows, used in turn: a chain of MMAs into one accumulator runs at
+        // the instruction's latency (about a hundred clocks each), and a stage of few rows and long chunks is a
+        // chain of up to sixteen.
+        float acc[2][4][4];
 #pragma unroll
         for (int i = 0; i < 2; ++i)
 #pragma unroll
-          for (int e = 0; e < 4; ++e) acc[i][e] = 0.f;
+          for (int a = 0; a < 4; ++a)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) acc[i][a][e] = 0.f;
         const bool second = r_hi - r_lo > 16;   // the block has rows in its second group of 16
+        // what the flush of this block will add to this thread's output value: on its way while the weights stream
+        float fbias = 0.f;
+        {
+          const int t = tid >> 5, r = tid & 31;
+          if (r < r_hi - r_lo && t < p.T && !ph.out) {
+            const int nl = ps.row0 + r_lo + r;
+            if (ph.outb) { if (sg.fin_bias) fbias = __ldg(sg.fin_bias + nl); }
+            else if (ph.y_bias) fbias = __ldg(ph.y_bias + sg.out_col + nl);
+          }
+        }
         for (int ch = 0; ch < nch; ++ch, ++it) {
           const int slot = it % NSTAGE;
-          const int bytes = 2 * (ps.klen - ch * KC < KC ? ps.klen - ch * KC : KC);
+          const int bytes = 2 * ps.klen - ch * chunk < chunk ? 2 * ps.klen - ch * chunk : chunk;
           ptx::mbar_wait_limit(&full[slot], (it / NSTAGE) & 1, s_abort, kWaitLimit);
-          if (warp * 64 < bytes) {               // the same for the whole warp (the MMAs need all 32 lanes)
-            const uint32_t ws = ring + slot * STAGE_BYTES + g * ROW_PITCH + kb;
-            uint4 xb = lds128(xs + g * X_PITCH + ch * (KC * 2) + kb);
-            uint4 lo = lds128(ws), hi = lds128(ws + 8 * ROW_PITCH);
-            const bool tail = kb >= bytes;       // a row segment ends inside this warp's 64 bytes: nothing was copied
-            if (tail) {                          // here, and what the buffers hold must not reach the sums
-              xb = make_uint4(0u, 0u, 0u, 0u);
-              lo = xb; hi = xb;
+          // rows beyond the block's last one were not copied: read row 0 instead (their sums are never stored)
+          const int nr = r_hi - r_lo;
+          const uint32_t st0 = ring + slot * STAGE_BYTES + kb;
+          const uint32_t ws0 = st0 + (g < nr ? g : 0) * row_pitch, ws1 = st0 + (g + 8 < nr ? g + 8 : 0) * row_pitch;
+          const uint32_t ws2 = st0 + (g + 16 < nr ? g + 16 : 0) * row_pitch, ws3 = st0 + (g + 24 < nr ? g + 24 : 0) * row_pitch;
+          const uint32_t xs0 = xs + ch * chunk + kb;
+#pragma unroll 2
+          for (int j = 0; j < sub; ++j) {
+            if (j * 512 + warp * 64 >= bytes) break;     // the same for the whole warp (the MMAs need all 32 lanes)
+            uint4 xb = lds128(xs0 + j * 512);
+            uint4 lo = lds128(ws0 + j * 512), hi = lds128(ws1 + j * 512);
+            const bool tail = j * 512 + kb >= bytes;     // a row segment ends inside this warp's 64 bytes: nothing was
+            if (tail || !my_token) xb = make_uint4(0u, 0u, 0u, 0u);   // copied here, and what the buffers hold must not
+            if (tail) {                                               // reach the sums
+              lo = make_uint4(0u, 0u, 0u, 0u);
+              hi = lo;
             }
             // the same 16 bytes of k from rows g and g + 8 and from token g feed two MMAs as they are: the order
             // in which a contraction visits k is free as long as both operands agree on it
-            mma_bf16(acc[0], lo.x, hi.x, lo.y, hi.y, xb.x, xb.y);
-            mma_bf16(acc[0], lo.z, hi.z, lo.w, hi.w, xb.z, xb.w);
+            float* a0 = acc[0][(2 * j) & 3];
+            float* a1 = acc[0][(2 * j + 1) & 3];
+            mma_bf16(a0, lo.x, hi.x, lo.y, hi.y, xb.x, xb.y);
+            mma_bf16(a1, lo.z, hi.z, lo.w, hi.w, xb.z, xb.w);
             if (second) {
-              uint4 lo2 = lds128(ws + 16 * ROW_PITCH), hi2 = lds128(ws + 24 * ROW_PITCH);
-              if (tail) { lo2 = xb; hi2 = xb; }
-              mma_bf16(acc[1], lo2.x, hi2.x, lo2.y, hi2.y, xb.x, xb.y);
-              mma_bf16(acc[1], lo2.z, hi2.z, lo2.w, hi2.w, xb.z, xb.w);
+              uint4 lo2 = lds128(ws2 + j * 512), hi2 = lds128(ws3 + j * 512);
+              if (tail) { lo2 = lo; hi2 = lo; }
+              mma_bf16(acc[1][(2 * j) & 3], lo2.x, hi2.x, lo2.y, hi2.y, xb.x, xb.y);
+              mma_bf16(acc[1][(2 * j + 1) & 3], lo2.z, hi2.z, lo2.w, hi2.w, xb.z, xb.w);
             }
           }
           __syncwarp();
@@ -320,10 +402,13 @@ __device__ void consumers(const StreamParams& p, unsigned char* smem, uint32_t r
         ++flushes;
 #pragma unroll
         for (int i = 0; i < 2; ++i) {
-          rb[(2 * c) * RED_TOK + 16 * i + g] = acc[i][0];
-          rb[(2 * c + 1) * RED_TOK + 16 * i + g] = acc[i][1];
-          rb[(2 * c) * RED_TOK + 16 * i + g + 8] = acc[i][2];
-          rb[(2 * c + 1) * RED_TOK + 16 * i + g + 8] = acc[i][3];
+          float v4[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) v4[e] = (acc[i][0][e] + acc[i][1][e]) + (acc[i][2][e] + acc[i][3][e]);
+          rb[(2 * c) * RED_TOK + 16 * i + g] = v4[0];
+          rb[(2 * c + 1) * RED_TOK + 16 * i + g] = v4[1];
+          rb[(2 * c) * RED_TOK + 16 * i + g + 8] = v4[2];
+          rb[(2 * c + 1) * RED_TOK + 16 * i + g + 8] = v4[3];
         }
         cbar();
         {
@@ -333,17 +418,22 @@ __device__ void consumers(const StreamParams& p, unsigned char* smem, uint32_t r
 #pragma unroll
           for (int w = 0; w < CWARPS; ++w) v += src[w * RED_WARP];
           if (r < r_hi - r_lo && t < p.T) {
-            const int n = sg.out_col + ps.row0 + r_lo + r;
+            const int nl = ps.row0 + r_lo + r;             // row inside the segment
+            const int n = sg.out_col + nl;
             if (ph.out) {
               ph.out[(static_cast<long long>(ps.s) * 8 + t) * ph.out_ld + n] = v;
+            } else if (ph.outb) {
+              v += fbias;
+              if (sg.fin_kind == STREAM_IN_ACT) v = gelu_fast(v, gc);
+              ph.outb[static_cast<long long>(t) * ph.out_ld + n] = __float2bfloat16_rn(v);
             } else {
-              if (ph.y_bias) v += __ldg(ph.y_bias + n);
-              ph.y[static_cast<long long>(t) * ph.y_ld + n] = __float2bfloat16_rn(v);
+              ph.y[static_cast<long long>(t) * ph.y_ld + n] = __float2bfloat16_rn(v + fbias);
             }
           }
         }
       }
       u += ps.rows;
+      if (u < sh.hi) ps = pass_at(ph, u, sh.hi);
     }
   }
 }
@@ -356,14 +446,14 @@ __global__ void __launch_bounds__(THREADS, 1) decode_stream_kernel(const __grid_
   const uint32_t ring = static_cast<uint32_t>(__cvta_generic_to_shared(smem));
   if (threadIdx.x == 0) {
     for (int i = 0; i < NSTAGE; ++i) {
-      ptx::mbar_init(&full[i], 1);
+      ptx::mbar_init(&full[i], 32);          // every lane of the warp that fills the stage
       ptx::mbar_init(&empty[i], CWARPS);
     }
     *s_abort = 0;
     ptx::mbar_fence_init();
   }
   __syncthreads();
-  if (threadIdx.x >= CTHREADS) producer(p, ring, full, empty, s_abort);
+  if (threadIdx.x >= CTHREADS) producer(p, ring, full, empty, s_abort, (threadIdx.x - CTHREADS) >> 5);
   else consumers(p, smem, ring, full, empty, s_abort);
   __syncthreads();
   if (threadIdx.x == 0 && *s_abort) record_status(p.ctrl, FFSPLIT_ERR_TIMEOUT, static_cast<int>(blockIdx.x), KID_DECODE);

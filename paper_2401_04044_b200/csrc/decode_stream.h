@@ -12,8 +12,12 @@ struct ffsplit_ctx;
 
 namespace ffsp {
 
-constexpr int kStreamKxMax = 2560;     // longest k range of one pass (elements): the activation operand of a pass
-                                       // lives in shared memory, 8 token rows of this many bf16 values
+// The activation operand of a pass lives in shared memory: x_rows token rows (1, 2, 4 or 8: the token count
+// rounded up) of x_pitch bytes, kStreamXBytes in all.  The fewer tokens, the longer the k range a pass may cover
+// (20672 elements for one token, 2560 for eight), and the fewer slices a long contraction has to be cut into.
+constexpr int kStreamXBytes = 41472;
+inline int stream_x_rows(int T) { return T <= 1 ? 1 : T <= 2 ? 2 : T <= 4 ? 4 : 8; }
+inline int stream_kx_max(int x_rows) { return (kStreamXBytes / x_rows - 64) / 128 * 64; }   // elements; pitch = 2 kx + 64
 constexpr int kStreamMaxPhases = 6;
 constexpr int kStreamMaxSegments = 4;
 
@@ -46,7 +50,18 @@ struct StreamSegment {
   int rows;
   int x_off;
   int out_col;
+  int fin_kind;             // when the phase writes finished values: STREAM_IN_LINEAR (sum + bias) or STREAM_IN_ACT
+  const float* fin_bias;    // indexed by the row inside the segment, or nullptr
 };
+
+// Geometry of one ring stage: a block of `rows` weight rows (at most 32) times a k chunk of 256 * sub elements;
+// the fewer rows a block has, the longer its chunks, so that a stage carries about the same bytes either way
+// (a stage of 7 rows x 512 bytes would leave most of the ring, and of the memory pipeline, empty).
+constexpr int kStreamStageBytes = 32 * 576;
+__host__ __device__ inline int stream_stage_sub(int rows) {
+  const int s = (kStreamStageBytes / rows - 64) / 512;
+  return s < 1 ? 1 : (s > 8 ? 8 : s);
+}
 
 struct StreamPhase {
   int kind;                 // 0: product; 1: closing reduction (y = sum of in[0]'s slices + y_bias)
@@ -57,6 +72,7 @@ struct StreamPhase {
   StreamSegment seg[kStreamMaxSegments];
   StreamInPart in[2];
   float* out;               // raw sums, float [S][8][out_ld]; nullptr for the phase that writes the layer output
+  __nv_bfloat16* outb;      // S == 1 only: finished values (bias, activation, rounded), bf16 [8][out_ld], instead of `out`
   long long out_ld;
   __nv_bfloat16* y;         // layer output [T, y_ld] (+ y_bias), written when out == nullptr
   long long y_ld;
@@ -68,6 +84,7 @@ struct StreamParams {
   StreamPhase ph[kStreamMaxPhases];
   int nph;
   int T;                    // 1..8
+  int x_rows, x_pitch;      // geometry of the activation operand in shared memory
   int act;                  // ffsplit_act of the layer
   int* ctrl;                // control block: status words, grid-barrier words
   const unsigned long long* guard;   // blob header to verify (or nullptr) and its registered hash

@@ -721,3 +721,60 @@ def test_forward_stack_device_and_host(ctx, T):
     ctx.forward_stack_host(blobs, Xh, Yh)
     ctx.poll()
     assert torch.equal(Yh, x)
+
+
+def test_token_sharded_scoring_flow_on_one_rank(ctx):
+    """The sharded-calibration flow bound to the library (batches with scores = NULL, the all-reduce -- a no-op
+    on one rank --, ffsplit_score_finalize) gives the scores of one ffsplit_score call up to summation order,
+    and the oracle's heavy set."""
+    from paper_2401_04044_b200 import sharded
+    cfg = custom_config(128, 640, 32, 16, act="gelu_erf", dtype="bf16")
+    L = make_layer(cfg, 1)
+    G = GpuLayer(ctx, L)
+    T = 1000
+    G.reserve(0, T, 0, 0)
+    X = L.tokens(T)
+    _, scores_one = G.score(X)
+    energy = torch.empty(cfg.m, dtype=torch.float32, device="cuda")
+    scores = torch.empty(cfg.m, dtype=torch.float32, device="cuda")
+    lo, hi = sharded.shard_bounds(T, 1, 0)
+    n = sharded.ctx_score_token_sharded(ctx, G.shape, G.W1, G.b1, G.W2, X[lo:hi].cuda(), energy, scores, batch=384)
+    ctx.poll()
+    assert n == T
+    _, _, s_ref = orc.neuron_scores(f64(X), f64(L.W1), f64(L.b1), f64(L.W2), cfg.act)
+    rt = SCORE_RTOL["bf16"]
+    assert np.allclose(f64(scores), s_ref, rtol=rt, atol=rt * s_ref.max() * 1e-3)
+    assert np.allclose(f64(scores), f64(scores_one), rtol=1e-5)
+    heavy, _ = G.select(scores, cfg.k)
+    assert np.array_equal(heavy.cpu().numpy(), orc.select_heavy(s_ref, cfg.k)[0])
+
+
+@pytest.mark.parametrize("act,d,m,k,r", DECODE_CASES + [("gelu_erf", 1024, 4096, 4096, 0), ("swiglu", 256, 1200, 0, 64),
+                                                         ("gelu_erf", 4096, 2304, 64, 32)])
+@pytest.mark.parametrize("T", [1, 2, 3, 4, 5, 8])
+def test_decode_streaming_kernel_matches_oracle(monkeypatch, act, d, m, k, r, T):
+    """The single-launch streaming kernel (one persistent kernel per layer, weights streamed ahead of the stage
+    dependencies), forced for every shape with FFSPLIT_DECODE_STREAM=2 -- by itself the library takes it only for
+    layers of many megabytes at up to four tokens.  Covers: finished (bf16) and raw (fp32 slices) hand-over between
+    the phases, several k ranges per contraction (d = 4096 at 5 or 8 tokens; the dense layer's stage 3 with its
+    closing reduction), gated pairs, a layer without heavy neurons (k = 0) and the dense layer (k = m)."""
+    from paper_2401_04044_b200 import Context
+    cfg = custom_config(d, m, k, r, act=act, dtype="bf16")
+    L = make_layer(cfg, 8)
+    monkeypatch.setenv("FFSPLIT_DECODE_STREAM", "2")
+    c = Context(0)
+    try:
+        G = GpuLayer(c, L)
+        G.reserve(T, 0, k, r)
+        fac = oracle_factors(L, L.planted.numpy(), r) if r > 0 else None
+        blob, _ = G.pack(L.planted, fac)
+        X = L.tokens(T)
+        Y = G.forward(blob, X)
+        fac_o = fac
+        if fac is None:
+            fac_o = {n: torch.zeros((d, 0) if n.startswith("A1") else (0, m - k) if n.startswith("B1") else
+                                    (m - k, 0) if n == "A2" else (0, d)) for n in ("A1", "B1", "A2", "B2")}
+        assert_close(Y, oracle_split(L, L.planted.numpy(), fac_o, X), "bf16", "streaming decode forward")
+        assert torch.equal(G.forward(blob, X), Y), "streaming decode forward is not bitwise reproducible"
+    finally:
+        c.close()
