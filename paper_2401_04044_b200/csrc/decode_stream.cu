@@ -29,95 +29,16 @@
 // flight are given a bounded time to land, and FFSPLIT_ERR_TIMEOUT is recorded in the status block.
 #include <cstring>
 
-#include "decode_common.cuh"
 #include "decode_stream.h"
 #include "epilogue.cuh"
-#include "internal.h"
-#include "ptx.cuh"
+#include "stream_common.cuh"
 
 namespace ffsp {
 namespace dst {
 
-using namespace dec;
-
-constexpr int CWARPS = 8;                                // consumer warps
-constexpr int CTHREADS = 32 * CWARPS;
-constexpr int PWARPS = 4;                                // producer warps: stage i is filled by warp i mod 4
-constexpr int THREADS = CTHREADS + 32 * PWARPS;
-constexpr int BLOCK_ROWS = 32;                           // weight rows per stage, at most
-constexpr int STAGE_BYTES = kStreamStageBytes;           // 18432
-constexpr int NSTAGE = 9;
-constexpr int X_BYTES = kStreamXBytes;                   // activation operand of a pass: x_rows token rows, x_pitch apart
-constexpr int RED_TOK = 36;                              // floats between token rows of a warp's partial block
-constexpr int RED_WARP = 8 * RED_TOK;
-constexpr int RED_BYTES = 2 * CWARPS * RED_WARP * 4;     // two buffers, used alternately
-constexpr int OFF_X = NSTAGE * STAGE_BYTES;
-constexpr int OFF_RED = OFF_X + X_BYTES;
-constexpr int OFF_BAR = OFF_RED + RED_BYTES;
-constexpr int SMEM_BYTES = OFF_BAR + 256;
-static_assert(SMEM_BYTES <= 232448, "shared memory plan");
-constexpr int kBarTicket = 18;                           // words 18-19 of the control block: the grid barrier's 64-bit ticket counter
-constexpr long long kWaitLimit = 2000000000ll;           // SM clocks (about a second)
-
-__device__ __forceinline__ void cbar() { asm volatile("bar.sync 1, %0;" ::"n"(CTHREADS) : "memory"); }
-
-// ---- the walk over a CTA's share of one phase, taken identically by the producers and the consumers -----
-// (32-bit arithmetic: the host checks S * Nall * (grid + 1) < 2^31 when it plans a phase)
-struct Pass {
-  int seg, s;          // segment, k range
-  int row0, rows;      // rows [row0, row0 + rows) of the segment
-  int kbeg, klen;      // k range in elements
-};
-struct Share { unsigned lo, hi; };   // units [lo, hi) of the phase: unit = s * Nall + row
-
-__device__ __forceinline__ Share share_of(const StreamPhase& ph, unsigned cta, unsigned ncta) {
-  const unsigned U = static_cast<unsigned>(ph.S) * ph.Nall;
-  Share sh;
-  sh.lo = U * cta / ncta;
-  sh.hi = U * (cta + 1) / ncta;
-  return sh;
-}
-// the pass that starts at unit u (u < hi)
-__device__ __forceinline__ Pass pass_at(const StreamPhase& ph, unsigned u, unsigned hi) {
-  Pass p;
-  const unsigned nall = ph.Nall;
-  p.s = static_cast<int>(u / nall);
-  const int row = static_cast<int>(u - p.s * nall);
-  int j = 0, start = 0;
-  while (j + 1 < ph.nseg && row >= start + ph.seg[j].rows) { start += ph.seg[j].rows; ++j; }
-  p.seg = j;
-  p.row0 = row - start;
-  unsigned end = p.s * nall + start + ph.seg[j].rows;   // end of the segment in this k range
-  if (end > hi) end = hi;
-  p.rows = static_cast<int>(end - u);
-  const unsigned k32 = (ph.K + 31) / 32;
-  p.kbeg = 32 * static_cast<int>(p.s * k32 / ph.S);
-  const int kend = p.s + 1 == ph.S ? ph.K : 32 * static_cast<int>((p.s + 1) * k32 / ph.S);
-  p.klen = kend - p.kbeg;
-  return p;
-}
-// rows of a pass are cut into blocks of at most 32 rows of nearly equal size
-__device__ __forceinline__ int blocks_of(int rows) { return (rows + BLOCK_ROWS - 1) / BLOCK_ROWS; }
-__device__ __forceinline__ int block_lo(int rows, int nb, int b) { return rows * b / nb; }
+static_assert(STAGE_BYTES == kStreamStageBytes && X_BYTES == kStreamXBytes, "the host's plan and the kernel agree");
 
 // ---- producers -------------------------------------------------------------------------------------
-// 16 bytes per lane of each of `nr` rows (src_step bytes apart; a lane outside the k range copies nothing and its
-// 16 bytes are zero filled)
-__device__ __forceinline__ void issue_rows(uint32_t dst, int dst_pitch, const char* src, long long src_step, int nr,
-                                           bool valid) {
-  int r = 0;
-#pragma unroll 1
-  for (; r + 4 <= nr; r += 4) {
-    cp_async16(dst, src, valid);
-    cp_async16(dst + dst_pitch, src + src_step, valid);
-    cp_async16(dst + 2 * dst_pitch, src + 2 * src_step, valid);
-    cp_async16(dst + 3 * dst_pitch, src + 3 * src_step, valid);
-    dst += 4 * dst_pitch;
-    src += 4 * src_step;
-  }
-  for (; r < nr; ++r, dst += dst_pitch, src += src_step) cp_async16(dst, src, valid);
-}
-
 __device__ void producer(const StreamParams& p, uint32_t ring, uint64_t* full, uint64_t* empty, volatile int* s_abort,
                          int pw) {
   const int lane = threadIdx.x & 31;
@@ -249,34 +170,6 @@ __device__ void build_x(const StreamPhase& ph, int T, int act, int c0, int klen,
     }
   }
   asm volatile("cp.async.wait_all;" ::: "memory");
-}
-
-// All CTAs are resident (cooperative launch).  Called by the consumer threads.  One 64-bit counter that only
-// ever grows: an arrival takes a ticket v, and the barrier it belongs to is complete when the counter reaches
-// the next multiple of the grid size above v (every barrier receives exactly one arrival per CTA, so the
-// counter stays aligned from launch to launch; a run that gave up leaves it misaligned, and ffsplit_poll()
-// clears the control block when it reports that).  The arrival is a release at GPU scope, ordered after the
-// whole CTA's writes by the CTA barrier before it, and the wait ends with an acquire: no separate fences, one
-// atomic round trip on the critical path.  Always arrives; gives up waiting after the limit or when the CTA has
-// already given up.
-__device__ void grid_barrier(int* ctrl, volatile int* s_abort) {
-  cbar();
-  if (threadIdx.x == 0) {
-    unsigned long long* ctr = reinterpret_cast<unsigned long long*>(ctrl + kBarTicket);
-    unsigned long long v;
-    asm volatile("atom.add.acq_rel.gpu.global.u64 %0, [%1], 1;" : "=l"(v) : "l"(ctr) : "memory");
-    const unsigned long long target = (v / gridDim.x + 1ull) * gridDim.x;
-    if (v + 1ull != target) {
-      const long long t0 = clock64();
-      while (!*s_abort) {
-        unsigned long long now;
-        asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(now) : "l"(ctr) : "memory");
-        if (now >= target) break;
-        if (clock64() - t0 > kWaitLimit) *s_abort = 1;
-      }
-    }
-  }
-  cbar();
 }
 
 __device__ void consumers(const StreamParams& p, unsigned char* smem, uint32_t ring, uint64_t* full, uint64_t* empty,

@@ -64,6 +64,7 @@ __host__ __device__ inline int stream_stage_sub(int rows) {
 }
 
 struct StreamPhase {
+  static constexpr unsigned kQuantum = 32;   // k ranges start on multiples of 32 elements
   int kind;                 // 0: product; 1: closing reduction (y = sum of in[0]'s slices + y_bias)
   int nseg, nin;
   int K;                    // contraction length of every segment (multiple of 8)
