@@ -287,6 +287,45 @@ ffsplit_status ffsplit_forward_stack_host(ffsplit_ctx* ctx, const void* const* b
 ffsplit_status ffsplit_forward_noalloc(ffsplit_ctx* ctx, const void* blob, const void* X, int64_t T,
                                        void* Y, void* stream);
 
+/* ---- Quantised split (Section 5.2, Table 3: round-to-nearest, group size 128, 8 bits for the heavy-hitter
+ * neurons, 3 bits for everything else) ------------------------------------------------------------------
+ * The second way the paper compresses the light part: instead of rank-r factors, U2 and V2 are kept whole at
+ * 3 bits and U1, V1 at 8 bits.  Reading taken where the paper is silent: each of the four matrices is quantised
+ * on its own, per output channel, in groups of 128 consecutive weights along its input dimension (along d for a
+ * neuron's column of U; along the part's neurons, in ascending index order, for a column of V; a last group may
+ * be shorter); asymmetric min/max grid, weight = lo + code * scale with lo = min, scale = (max - min) / (2^b - 1),
+ * code = round-half-even((w - lo) / scale), all decided in float32; scale and lo are stored as float32; biases
+ * are not quantised.  bf16 layers only (GELU or SwiGLU). */
+
+/* Size of the quantised packed layer.  logical_bytes = the codes at their bit width + 8 bytes per group
+ * + 4 (m + d) bytes of float32 biases. */
+ffsplit_status ffsplit_quant_pack_size(const ffsplit_shape* shape, int32_t k, size_t* padded_bytes, size_t* logical_bytes);
+
+/* Workspace ffsplit_quant_forward() needs for a layer of this shape and split (any token count). */
+ffsplit_status ffsplit_quant_workspace_size(const ffsplit_shape* shape, int32_t k, size_t* bytes);
+
+/* Quantise and pack a layer.  heavy_idx dev int32[k] and light_idx dev int32[m-k] are the two ascending
+ * lists ffsplit_select() writes (heavy_idx is validated like in ffsplit_pack(); light_idx must be its
+ * complement).  blob dev, 256-byte aligned, >= padded_bytes.  Needs a workspace (status word only). */
+ffsplit_status ffsplit_quant_pack(ffsplit_ctx* ctx, const ffsplit_shape* shape, const ffsplit_weights* weights,
+                                  const int32_t* heavy_idx, int32_t k, const int32_t* light_idx, void* blob,
+                                  size_t blob_bytes, void* stream);
+
+/* Register a quantised blob that was not packed on this context (see ffsplit_blob_open()). */
+ffsplit_status ffsplit_quant_blob_open(ffsplit_ctx* ctx, const void* blob, size_t blob_bytes, void* stream);
+
+/* Expand one matrix of a quantised blob, for inspection and tests.
+ * which: 0 U1 [k, d]   1 U2 [m-k, d]   2 / 3 the SwiGLU up projections likewise   4 V1 [d, k]   5 V2 [d, m-k]
+ * (rows = output channels, columns = the grouped input axis).
+ *   codes dev uint8 [rows, cols]; scale, lo dev float [rows, ceil(cols / 128)] */
+ffsplit_status ffsplit_quant_unpack(ffsplit_ctx* ctx, const void* blob, int32_t which, uint8_t* codes, float* scale,
+                                    float* lo, void* stream);
+
+/* Eq. 2 on the quantised weights: Y = sigma(X U1~ + b1[h2]) V1~ + sigma(X U2~ + b1[light]) V2~ + b2, with
+ * w~ = lo + code * scale applied inside the weight-streaming kernel (the few-token path: the tokens are taken
+ * eight at a time, one launch each; meant for decode, T <= 8).  X, Y dev bf16 [T, d].  Uses the workspace. */
+ffsplit_status ffsplit_quant_forward(ffsplit_ctx* ctx, const void* blob, const void* X, int64_t T, void* Y, void* stream);
+
 /* Synchronise `stream`, then return and clear the first device-side condition found in the workspace's
  * status word or in that of the built-in scratch of ffsplit_forward_noalloc() on the context's device
  * (FFSPLIT_OK if no kernel recorded one).  Works on a context without a workspace. */

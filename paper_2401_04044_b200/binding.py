@@ -35,7 +35,8 @@ EXPORTS = [
     "ffsplit_version", "ffsplit_profile_begin", "ffsplit_profile_end", "ffsplit_forward_noalloc",
     "ffsplit_forward_dense", "ffsplit_score_activations", "ffsplit_score_host", "ffsplit_score_finalize",
     "ffsplit_blob_close", "ffsplit_stack_workspace_size", "ffsplit_forward_stack", "ffsplit_forward_stack_host",
-    "ffsplit_debug_wait_timeout",
+    "ffsplit_debug_wait_timeout", "ffsplit_quant_pack_size", "ffsplit_quant_workspace_size", "ffsplit_quant_pack",
+    "ffsplit_quant_blob_open", "ffsplit_quant_unpack", "ffsplit_quant_forward",
 ]
 
 
@@ -91,6 +92,12 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.ffsplit_forward_stack.argtypes = [vp, P(vp), i32, vp, i64, vp, vp]
     lib.ffsplit_forward_stack_host.argtypes = [vp, P(vp), i32, vp, i64, vp, vp]
     lib.ffsplit_debug_wait_timeout.argtypes = [vp, i64, vp]
+    lib.ffsplit_quant_pack_size.argtypes = [P(Shape), i32, P(sz), P(sz)]
+    lib.ffsplit_quant_workspace_size.argtypes = [P(Shape), i32, P(sz)]
+    lib.ffsplit_quant_pack.argtypes = [vp, P(Shape), P(Weights), vp, i32, vp, vp, sz, vp]
+    lib.ffsplit_quant_blob_open.argtypes = [vp, vp, sz, vp]
+    lib.ffsplit_quant_unpack.argtypes = [vp, vp, i32, vp, vp, vp, vp]
+    lib.ffsplit_quant_forward.argtypes = [vp, vp, vp, i64, vp, vp]
     lib.ffsplit_blob_section.argtypes = [vp, vp, i32, P(sz), P(i64), P(i64), P(i64)]
     lib.ffsplit_forward.argtypes = [vp, vp, vp, i64, vp, vp]
     lib.ffsplit_forward_host.argtypes = [vp, vp, vp, i64, vp, vp]
@@ -250,6 +257,42 @@ class Context:
         self._check(self.lib.ffsplit_forward_stack_host(self.h, self._blob_array(blobs), len(blobs), _ptr(X_host),
                                                         X_host.shape[0], _ptr(Y_host), _stream_ptr(stream)),
                     "ffsplit_forward_stack_host")
+
+    # ------------------------------------------------------------------ quantised split (Section 5.2)
+    def quant_pack_size(self, shape: Shape, k: int):
+        a, b = C.c_size_t(), C.c_size_t()
+        self._check(self.lib.ffsplit_quant_pack_size(C.byref(shape), k, C.byref(a), C.byref(b)), "ffsplit_quant_pack_size")
+        return a.value, b.value
+
+    def quant_workspace_size(self, shape: Shape, k: int) -> int:
+        n = C.c_size_t()
+        self._check(self.lib.ffsplit_quant_workspace_size(C.byref(shape), k, C.byref(n)), "ffsplit_quant_workspace_size")
+        return n.value
+
+    def quant_pack(self, shape: Shape, W1, b1, W2, b2, heavy_idx, k: int, light_idx, blob, W1u=None, stream=None):
+        w = Weights(_ptr(W1), _ptr(W1u), _ptr(b1), _ptr(W2), _ptr(b2))
+        self._check(self.lib.ffsplit_quant_pack(self.h, C.byref(shape), C.byref(w), _ptr(heavy_idx), k, _ptr(light_idx),
+                                                _ptr(blob), blob.numel() * blob.element_size(), _stream_ptr(stream)),
+                    "ffsplit_quant_pack")
+
+    def quant_blob_open(self, blob, stream=None):
+        self._check(self.lib.ffsplit_quant_blob_open(self.h, _ptr(blob), blob.numel() * blob.element_size(),
+                                                     _stream_ptr(stream)), "ffsplit_quant_blob_open")
+
+    def quant_unpack(self, blob, which: int, rows: int, cols: int, stream=None):
+        """-> (codes uint8 [rows, cols], scale float32 [rows, ceil(cols / 128)], lo likewise) of one packed matrix."""
+        dev = blob.device
+        codes = torch.zeros(rows, cols, dtype=torch.uint8, device=dev)
+        ng = (cols + 127) // 128
+        scale = torch.zeros(rows, ng, dtype=torch.float32, device=dev)
+        lo = torch.zeros(rows, ng, dtype=torch.float32, device=dev)
+        self._check(self.lib.ffsplit_quant_unpack(self.h, _ptr(blob), which, _ptr(codes), _ptr(scale), _ptr(lo),
+                                                  _stream_ptr(stream)), "ffsplit_quant_unpack")
+        return codes, scale, lo
+
+    def quant_forward(self, blob, X, Y, stream=None):
+        self._check(self.lib.ffsplit_quant_forward(self.h, _ptr(blob), _ptr(X), X.shape[0], _ptr(Y), _stream_ptr(stream)),
+                    "ffsplit_quant_forward")
 
     def debug_wait_timeout(self, limit_cycles: int, stream=None):
         self._check(self.lib.ffsplit_debug_wait_timeout(self.h, int(limit_cycles), _stream_ptr(stream)),

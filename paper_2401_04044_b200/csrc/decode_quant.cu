@@ -137,11 +137,10 @@ __device__ void producer(const QParams& p, uint32_t ring, uint64_t* full, uint64
           const int bytes = gcnt * gb;                                             // a multiple of 16
           const char* src0 = base + static_cast<long long>(ch) * gch * gb;
           const uint32_t dst0 = ring + slot * STAGE_BYTES + lane * 16;
-          for (int j = 0; j * 512 < bytes; ++j) {
-            const bool valid = j * 512 + lane * 16 < bytes;
-            issue_rows(dst0 + j * 512, row_pitch, valid ? src0 + j * 512 : reinterpret_cast<const char*>(sg.W),
-                       valid ? sg.row_bytes : 0, r_hi - r_lo, valid);
-          }
+          // a lane past the end of the row's groups copies nothing at all: the rows of a stage lie closer together
+          // than the next multiple of 512 bytes, and a zero fill there would land in the next row
+          for (int j = 0; j * 512 < bytes; ++j)
+            if (j * 512 + lane * 16 < bytes) issue_rows(dst0 + j * 512, row_pitch, src0 + j * 512, sg.row_bytes, r_hi - r_lo, true);
           asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(ptx::smem_u32(&full[slot])) : "memory");
         }
       }

@@ -181,6 +181,8 @@ struct ffsplit_ctx {
   std::string err;
   struct BlobEntry { ffsp::BlobHeader h; size_t bytes; unsigned long long hash; };
   std::unordered_map<const void*, BlobEntry> blobs;   // blobs packed or opened on this context, by address
+  struct QuantEntry { unsigned char header[256]; size_t bytes; unsigned long long hash; };
+  std::unordered_map<const void*, QuantEntry> qblobs; // quantised blobs (Section 5.2), likewise
   std::unordered_map<ffsp::TmapKey, CUtensorMap, ffsp::TmapKeyHash> tmaps;
   void* encode_fn = nullptr;  // cuTensorMapEncodeTiled
   struct ProfRec { int cls; cudaEvent_t a, b; double work; };

@@ -101,7 +101,7 @@ __device__ __forceinline__ void issue_rows(uint32_t dst, int dst_pitch, const ch
 // whole CTA's writes by the CTA barrier before it, and the wait ends with an acquire: no separate fences, one
 // atomic round trip on the critical path.  Always arrives; gives up waiting after the limit or when the CTA has
 // already given up.
-__device__ void grid_barrier(int* ctrl, volatile int* s_abort) {
+__device__ __forceinline__ void grid_barrier(int* ctrl, volatile int* s_abort) {
   cbar();
   if (threadIdx.x == 0) {
     unsigned long long* ctr = reinterpret_cast<unsigned long long*>(ctrl + kBarTicket);
