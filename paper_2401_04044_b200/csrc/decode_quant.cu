@@ -150,23 +150,6 @@ __device__ void producer(const QParams& p, uint32_t ring, uint64_t* full, uint64
 }
 
 // ---- consumers ----------------------------------------------------------------------------------------
-__device__ __forceinline__ float4 load_sum4(const StreamInPart& in, int t, long long col) {
-  const float* base = static_cast<const float*>(in.src) + static_cast<long long>(t) * in.ld + col;
-  float4 a = __ldcg(reinterpret_cast<const float4*>(base));
-  for (int s0 = 1; s0 < in.nslices; s0 += 4) {
-    float4 b[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      b[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (s0 + j < in.nslices) b[j] = __ldcg(reinterpret_cast<const float4*>(base + (s0 + j) * in.slice_stride));
-    }
-#pragma unroll
-    for (int j = 0; j < 4; ++j)
-      if (s0 + j < in.nslices) { a.x += b[j].x; a.y += b[j].y; a.z += b[j].z; a.w += b[j].w; }
-  }
-  return a;
-}
-
 // Byte offset, inside a token row of the activation operand, of the 8 bytes that hold columns e .. e+3 (e a
 // multiple of 4) of group `grp`: a group is four runs of 64 bytes (one per lane c of the MMA fragment), and the
 // four 16-byte chunks of a run are stored rotated by the run's number so that the lanes' 128-bit loads of chunk j
@@ -184,14 +167,17 @@ __device__ __forceinline__ uint32_t pack_f16x2(float lo, float hi) {
 // Activation operand of a pass: columns [c0, c0 + 128 glen) of the phase's activation matrix for tokens
 // 0 .. x_rows - 1 as fp16 (zero beyond the last token and beyond the part's last real column), then the sum of
 // every token's values per group, from the rounded values, in a fixed order.
-__device__ void build_x(const QPhase& ph, int T, int act, int c0, int glen, unsigned char* xbuf, float* xsum, int x_rows,
-                        int X_PITCH) {
-  const GeluCoef gc = gelu_coef(act);
+// A thread takes eight elements of four columns per turn.  The loads of a turn are all issued before the first
+// is used and the loop body has no branch that depends on the element (an element with nothing to load reads a
+// valid address and is masked afterwards): with branches between them the loads went out one latency at a time
+// (23 us for one 19456-column operand).
+template <int KIND>
+__device__ __forceinline__ void build_x_kind(const StreamInPart& in, int T, const GeluCoef& gc, int c0, int glen,
+                                             unsigned char* xbuf, int x_rows, int X_PITCH) {
   const int tid = threadIdx.x;
   const int groups = glen * 32;                // 4-column elements per token row
   constexpr int B = 8;
   const int total = x_rows * groups;
-  const StreamInPart& in = ph.in[0];
   for (int e0 = tid; e0 < total; e0 += B * CTHREADS) {
     float4 v[B], u[B];
     uint2 raw[B];
@@ -199,23 +185,44 @@ __device__ void build_x(const QPhase& ph, int T, int act, int c0, int glen, unsi
 #pragma unroll
     for (int j = 0; j < B; ++j) {
       const int e = e0 + j * CTHREADS;
-      v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-      u[j] = v[j];
-      raw[j] = make_uint2(0u, 0u);
-      live[j] = false;
-      if (e >= total) continue;
-      const int t = e / groups, q = e - t * groups;
+      const int ee = e < total ? e : tid;      // a valid element to read in any case
+      const int t = ee / groups, q = ee - t * groups;
       const int col = c0 + 4 * q;
-      if (t >= T || col >= in.col_end) continue;
-      live[j] = true;
-      const long long sc = in.src_col + (col - in.col_begin);
-      if (in.kind == STREAM_IN_BF16) {
+      live[j] = e < total && t < T && col < in.col_end;
+      const int tt = live[j] ? t : 0;
+      const long long sc = in.src_col + (live[j] ? col - in.col_begin : 0);
+      if (KIND == STREAM_IN_BF16) {
         raw[j] = __ldg(reinterpret_cast<const uint2*>(static_cast<const __nv_bfloat16*>(in.src) +
-                                                      static_cast<long long>(t) * in.ld + sc));
+                                                      static_cast<long long>(tt) * in.ld + sc));
       } else {
-        v[j] = load_sum4(in, t, sc);
-        if (in.kind == STREAM_IN_GATED) u[j] = load_sum4(in, t, sc + in.gate_off);
-        else if (in.bias) u[j] = __ldg(reinterpret_cast<const float4*>(in.bias + (col - in.col_begin)));
+        const float* base = static_cast<const float*>(in.src) + static_cast<long long>(tt) * in.ld + sc;
+        v[j] = __ldcg(reinterpret_cast<const float4*>(base));
+        if (KIND == STREAM_IN_GATED) u[j] = __ldcg(reinterpret_cast<const float4*>(base + in.gate_off));
+        else u[j] = in.bias ? __ldg(reinterpret_cast<const float4*>(in.bias + (live[j] ? col - in.col_begin : 0)))
+                            : make_float4(0.f, 0.f, 0.f, 0.f);
+      }
+    }
+    if (KIND != STREAM_IN_BF16) {
+      // further k ranges of the phase before: slice by slice, the eight elements' loads together
+      for (int s = 1; s < in.nslices; ++s) {
+        float4 b[B], bu[B];
+#pragma unroll
+        for (int j = 0; j < B; ++j) {
+          const int e = e0 + j * CTHREADS;
+          const int ee = e < total ? e : tid;
+          const int t = ee / groups, q = ee - t * groups;
+          const int col = c0 + 4 * q;
+          const int tt = live[j] ? t : 0;
+          const long long sc = in.src_col + (live[j] ? col - in.col_begin : 0);
+          const float* base = static_cast<const float*>(in.src) + s * in.slice_stride + static_cast<long long>(tt) * in.ld + sc;
+          b[j] = __ldcg(reinterpret_cast<const float4*>(base));
+          if (KIND == STREAM_IN_GATED) bu[j] = __ldcg(reinterpret_cast<const float4*>(base + in.gate_off));
+        }
+#pragma unroll
+        for (int j = 0; j < B; ++j) {
+          v[j].x += b[j].x; v[j].y += b[j].y; v[j].z += b[j].z; v[j].w += b[j].w;
+          if (KIND == STREAM_IN_GATED) { u[j].x += bu[j].x; u[j].y += bu[j].y; u[j].z += bu[j].z; u[j].w += bu[j].w; }
+        }
       }
     }
 #pragma unroll
@@ -223,18 +230,18 @@ __device__ void build_x(const QPhase& ph, int T, int act, int c0, int glen, unsi
       const int e = e0 + j * CTHREADS;
       if (e >= total) continue;
       const int t = e / groups, q = e - t * groups;
-      float4 a = v[j];
+      float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
       if (live[j]) {
-        if (in.kind == STREAM_IN_BF16) {
+        if (KIND == STREAM_IN_BF16) {
           const __nv_bfloat162 p0 = *reinterpret_cast<const __nv_bfloat162*>(&raw[j].x);
           const __nv_bfloat162 p1 = *reinterpret_cast<const __nv_bfloat162*>(&raw[j].y);
           a = make_float4(__low2float(p0), __high2float(p0), __low2float(p1), __high2float(p1));
-        } else if (in.kind == STREAM_IN_GATED) {
-          a.x = silu_fast(a.x) * u[j].x; a.y = silu_fast(a.y) * u[j].y;
-          a.z = silu_fast(a.z) * u[j].z; a.w = silu_fast(a.w) * u[j].w;
+        } else if (KIND == STREAM_IN_GATED) {
+          a.x = silu_fast(v[j].x) * u[j].x; a.y = silu_fast(v[j].y) * u[j].y;
+          a.z = silu_fast(v[j].z) * u[j].z; a.w = silu_fast(v[j].w) * u[j].w;
         } else {
-          a.x += u[j].x; a.y += u[j].y; a.z += u[j].z; a.w += u[j].w;
-          if (in.kind == STREAM_IN_ACT) {
+          a.x = v[j].x + u[j].x; a.y = v[j].y + u[j].y; a.z = v[j].z + u[j].z; a.w = v[j].w + u[j].w;
+          if (KIND == STREAM_IN_ACT) {
             a.x = gelu_fast(a.x, gc); a.y = gelu_fast(a.y, gc); a.z = gelu_fast(a.z, gc); a.w = gelu_fast(a.w, gc);
           }
         }
@@ -251,9 +258,20 @@ __device__ void build_x(const QPhase& ph, int T, int act, int c0, int glen, unsi
       *reinterpret_cast<uint2*>(xbuf + t * X_PITCH + x_offset(q >> 5, 4 * (q & 31))) = o;
     }
   }
+}
+
+__device__ void build_x(const QPhase& ph, int T, int act, int c0, int glen, unsigned char* xbuf, float* xsum, int x_rows,
+                        int X_PITCH) {
+  const GeluCoef gc = gelu_coef(act);
+  const StreamInPart& in = ph.in[0];
+  if (in.kind == STREAM_IN_BF16) build_x_kind<STREAM_IN_BF16>(in, T, gc, c0, glen, xbuf, x_rows, X_PITCH);
+  else if (in.kind == STREAM_IN_GATED) build_x_kind<STREAM_IN_GATED>(in, T, gc, c0, glen, xbuf, x_rows, X_PITCH);
+  else if (in.kind == STREAM_IN_ACT) build_x_kind<STREAM_IN_ACT>(in, T, gc, c0, glen, xbuf, x_rows, X_PITCH);
+  else build_x_kind<STREAM_IN_LINEAR>(in, T, gc, c0, glen, xbuf, x_rows, X_PITCH);
   cbar();
   // sums per (group, token): one warp per pair, lane l adds the 4 values in bytes [8l, 8l+8) of the group, then
   // a fixed shuffle tree
+  const int tid = threadIdx.x;
   const int warp = tid >> 5, lane = tid & 31;
   for (int task = warp; task < glen * x_rows; task += CWARPS) {
     const int grp = task / x_rows, t = task - grp * x_rows;
@@ -300,37 +318,64 @@ __device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
   return r;
 }
 
-// One group (128 k) of the 16 rows (ra, rb = rows g and g + 8 of the granule) against the tokens: acc8 receives
-// sum_k (1024 + q_k) x_k for (row ra, tokens 2c, 2c+1) and (row rb, tokens 2c, 2c+1).
-template <int BITS>
-__device__ __forceinline__ void group_mma(float (&acc8)[4], uint32_t ga, uint32_t gb_, int c, const uint32_t (&xr)[16]) {
+// One group (128 k) of up to 32 rows against the tokens.  ga, gb: the group's bytes in rows g and g + 8; gc, gd:
+// in rows g + 16 and g + 24 (SECOND).  acc[i] receives sum_k (1024 + q_k) x_k for (row g + 16 i, tokens 2c, 2c+1)
+// and (row g + 8 + 16 i, tokens 2c, 2c+1).  The eight MMAs of a 16-row block alternate between two accumulators
+// (and the two blocks are interleaved): a chain of MMAs into one accumulator runs at the instruction's latency.
+template <int BITS, bool SECOND>
+__device__ __forceinline__ void group_mma(float (&acc)[2][4], uint32_t ga, uint32_t gb_, uint32_t gc_, uint32_t gd_, int c,
+                                          const uint32_t (&xr)[16]) {
+  float a0[2][4], a1[2][4];
 #pragma unroll
-  for (int e = 0; e < 4; ++e) acc8[e] = 0.f;
+  for (int i = 0; i < 2; ++i)
+#pragma unroll
+    for (int e = 0; e < 4; ++e) { a0[i][e] = 0.f; a1[i][e] = 0.f; }
   if (BITS == 3) {
-    uint32_t wa[3], wb[3];
+    uint32_t wa[3], wb[3], wc[3], wd[3];
 #pragma unroll
-    for (int i = 0; i < 3; ++i) { wa[i] = lds32(ga + 12 * c + 4 * i); wb[i] = lds32(gb_ + 12 * c + 4 * i); }
-#define FFS_Q3(I) mma_f16(acc8, pair3<2 * I>(wa), pair3<2 * I>(wb), pair3<2 * I + 1>(wa), pair3<2 * I + 1>(wb), xr[2 * I], xr[2 * I + 1]);
+    for (int i = 0; i < 3; ++i) {
+      wa[i] = lds32(ga + 12 * c + 4 * i); wb[i] = lds32(gb_ + 12 * c + 4 * i);
+      if (SECOND) { wc[i] = lds32(gc_ + 12 * c + 4 * i); wd[i] = lds32(gd_ + 12 * c + 4 * i); }
+    }
+#define FFS_Q3(I)                                                                                                              \
+    mma_f16(a0[(I) & 1], pair3<2 * (I)>(wa), pair3<2 * (I)>(wb), pair3<2 * (I) + 1>(wa), pair3<2 * (I) + 1>(wb), xr[2 * (I)],  \
+            xr[2 * (I) + 1]);                                                                                                  \
+    if (SECOND)                                                                                                                \
+      mma_f16(a1[(I) & 1], pair3<2 * (I)>(wc), pair3<2 * (I)>(wd), pair3<2 * (I) + 1>(wc), pair3<2 * (I) + 1>(wd), xr[2 * (I)], \
+              xr[2 * (I) + 1]);
     FFS_Q3(0) FFS_Q3(1) FFS_Q3(2) FFS_Q3(3) FFS_Q3(4) FFS_Q3(5) FFS_Q3(6) FFS_Q3(7)
 #undef FFS_Q3
   } else {
-    uint32_t wa[8], wb[8];
+    uint32_t wa[8], wb[8], wc[8], wd[8];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const uint2 a = lds64(ga + 32 * c + 8 * i), b = lds64(gb_ + 32 * c + 8 * i);
       wa[2 * i] = a.x; wa[2 * i + 1] = a.y; wb[2 * i] = b.x; wb[2 * i + 1] = b.y;
+      if (SECOND) {
+        const uint2 cc = lds64(gc_ + 32 * c + 8 * i), dd = lds64(gd_ + 32 * c + 8 * i);
+        wc[2 * i] = cc.x; wc[2 * i + 1] = cc.y; wd[2 * i] = dd.x; wd[2 * i + 1] = dd.y;
+      }
     }
 #pragma unroll
-    for (int i = 0; i < 8; ++i)
-      mma_f16(acc8, prmt(wa[i], 0x64646464u, 0x4140u), prmt(wb[i], 0x64646464u, 0x4140u), prmt(wa[i], 0x64646464u, 0x4342u),
+    for (int i = 0; i < 8; ++i) {
+      mma_f16(a0[i & 1], prmt(wa[i], 0x64646464u, 0x4140u), prmt(wb[i], 0x64646464u, 0x4140u), prmt(wa[i], 0x64646464u, 0x4342u),
               prmt(wb[i], 0x64646464u, 0x4342u), xr[2 * i], xr[2 * i + 1]);
+      if (SECOND)
+        mma_f16(a1[i & 1], prmt(wc[i], 0x64646464u, 0x4140u), prmt(wd[i], 0x64646464u, 0x4140u), prmt(wc[i], 0x64646464u, 0x4342u),
+                prmt(wd[i], 0x64646464u, 0x4342u), xr[2 * i], xr[2 * i + 1]);
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    acc[0][e] = a0[0][e] + a0[1][e];
+    acc[1][e] = SECOND ? a1[0][e] + a1[1][e] : 0.f;
   }
 }
 
-template <int BITS>
-__device__ __forceinline__ void consume_stage(float (&tot)[2][4], uint32_t stage, int row_pitch, int nr, bool second,
-                                              int gcnt, int g_first, uint32_t xs, bool my_token, const float* xsum,
-                                              int warp, int g, int c) {
+template <int BITS, bool SECOND>
+__device__ __forceinline__ void consume_stage(float (&tot)[2][4], uint32_t stage, int row_pitch, int nr, int gcnt,
+                                              int g_first, uint32_t xs, bool my_token, const float* xsum, int warp, int g,
+                                              int c) {
   constexpr int GB = BITS == 8 ? qnt::kGroupBytes8 : qnt::kGroupBytes3;
   constexpr int PAR = BITS == 8 ? 128 : 48;
   const uint32_t r0 = stage + (g < nr ? g : 0) * row_pitch, r1 = stage + (g + 8 < nr ? g + 8 : 0) * row_pitch;
@@ -351,22 +396,21 @@ __device__ __forceinline__ void consume_stage(float (&tot)[2][4], uint32_t stage
       for (int j = 0; j < 16; ++j) xr[j] = 0u;
     }
     const float2 sx = *reinterpret_cast<const float2*>(xsum + grp * 8 + 2 * c);    // tokens 2c, 2c + 1
-    float acc8[4];
+    const uint2 pa = lds64(r0 + gi * GB + PAR), pb = lds64(r1 + gi * GB + PAR);
+    float acc[2][4];
+    group_mma<BITS, SECOND>(acc, r0 + gi * GB, r1 + gi * GB, r2 + gi * GB, r3 + gi * GB, c, xr);
     {
-      group_mma<BITS>(acc8, r0 + gi * GB, r1 + gi * GB, c, xr);
-      const uint2 pa = lds64(r0 + gi * GB + PAR), pb = lds64(r1 + gi * GB + PAR);
       const float sa = __uint_as_float(pa.x), la = __uint_as_float(pa.y) - 1024.f * sa;
       const float sb = __uint_as_float(pb.x), lb = __uint_as_float(pb.y) - 1024.f * sb;
-      tot[0][0] += fmaf(sa, acc8[0], la * sx.x); tot[0][1] += fmaf(sa, acc8[1], la * sx.y);
-      tot[0][2] += fmaf(sb, acc8[2], lb * sx.x); tot[0][3] += fmaf(sb, acc8[3], lb * sx.y);
+      tot[0][0] += fmaf(sa, acc[0][0], la * sx.x); tot[0][1] += fmaf(sa, acc[0][1], la * sx.y);
+      tot[0][2] += fmaf(sb, acc[0][2], lb * sx.x); tot[0][3] += fmaf(sb, acc[0][3], lb * sx.y);
     }
-    if (second) {
-      group_mma<BITS>(acc8, r2 + gi * GB, r3 + gi * GB, c, xr);
-      const uint2 pa = lds64(r2 + gi * GB + PAR), pb = lds64(r3 + gi * GB + PAR);
-      const float sa = __uint_as_float(pa.x), la = __uint_as_float(pa.y) - 1024.f * sa;
-      const float sb = __uint_as_float(pb.x), lb = __uint_as_float(pb.y) - 1024.f * sb;
-      tot[1][0] += fmaf(sa, acc8[0], la * sx.x); tot[1][1] += fmaf(sa, acc8[1], la * sx.y);
-      tot[1][2] += fmaf(sb, acc8[2], lb * sx.x); tot[1][3] += fmaf(sb, acc8[3], lb * sx.y);
+    if (SECOND) {
+      const uint2 pc = lds64(r2 + gi * GB + PAR), pd = lds64(r3 + gi * GB + PAR);
+      const float sa = __uint_as_float(pc.x), la = __uint_as_float(pc.y) - 1024.f * sa;
+      const float sb = __uint_as_float(pd.x), lb = __uint_as_float(pd.y) - 1024.f * sb;
+      tot[1][0] += fmaf(sa, acc[1][0], la * sx.x); tot[1][1] += fmaf(sa, acc[1][1], la * sx.y);
+      tot[1][2] += fmaf(sb, acc[1][2], lb * sx.x); tot[1][3] += fmaf(sb, acc[1][3], lb * sx.y);
     }
   }
 }
@@ -443,8 +487,14 @@ __device__ void consumers(const QParams& p, unsigned char* smem, uint32_t ring, 
           const int gcnt = ps.glen - ch * gch < gch ? ps.glen - ch * gch : gch;
           ptx::mbar_wait_limit(&full[slot], (it / NSTAGE) & 1, s_abort, kWaitLimit);
           const uint32_t stage = ring + slot * STAGE_BYTES;
-          if (sg.bits == 8) consume_stage<8>(tot, stage, row_pitch, r_hi - r_lo, second, gcnt, ch * gch, xs, my_token, xsum, warp, g, c);
-          else consume_stage<3>(tot, stage, row_pitch, r_hi - r_lo, second, gcnt, ch * gch, xs, my_token, xsum, warp, g, c);
+          const int nr = r_hi - r_lo;
+          if (sg.bits == 8) {
+            if (second) consume_stage<8, true>(tot, stage, row_pitch, nr, gcnt, ch * gch, xs, my_token, xsum, warp, g, c);
+            else consume_stage<8, false>(tot, stage, row_pitch, nr, gcnt, ch * gch, xs, my_token, xsum, warp, g, c);
+          } else {
+            if (second) consume_stage<3, true>(tot, stage, row_pitch, nr, gcnt, ch * gch, xs, my_token, xsum, warp, g, c);
+            else consume_stage<3, false>(tot, stage, row_pitch, nr, gcnt, ch * gch, xs, my_token, xsum, warp, g, c);
+          }
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(&empty[slot]);
         }

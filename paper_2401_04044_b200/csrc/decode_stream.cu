@@ -92,82 +92,107 @@ __device__ void producer(const StreamParams& p, uint32_t ring, uint64_t* full, u
 }
 
 // ---- consumers ----------------------------------------------------------------------------------------
-// Four columns of a phase's activation matrix from raw sums of an earlier phase: the slices added in order.
-// The loads of up to four slices are in flight together.
-__device__ __forceinline__ float4 load_sum4(const StreamInPart& in, int t, long long col) {
-  const float* base = static_cast<const float*>(in.src) + static_cast<long long>(t) * in.ld + col;
-  float4 a = __ldcg(reinterpret_cast<const float4*>(base));
-  for (int s0 = 1; s0 < in.nslices; s0 += 4) {
-    float4 b[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      b[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (s0 + j < in.nslices) b[j] = __ldcg(reinterpret_cast<const float4*>(base + (s0 + j) * in.slice_stride));
-    }
-#pragma unroll
-    for (int j = 0; j < 4; ++j)
-      if (s0 + j < in.nslices) { a.x += b[j].x; a.y += b[j].y; a.z += b[j].z; a.w += b[j].w; }
-  }
-  return a;
-}
-
 // Activation operand of a pass: columns [c0, c0 + klen) of the phase's activation matrix for tokens
 // 0 .. x_rows - 1 (rows beyond T are zero), bf16, token rows X_PITCH bytes apart.  Four columns per thread and
 // element.  Values that an earlier phase finished (or the layer input) are copied asynchronously as they are;
-// raw sums are added, biased, activated and rounded here, eight elements' loads in flight per thread.
-__device__ void build_x(const StreamPhase& ph, int T, int act, int c0, int klen, unsigned char* xbuf, uint32_t xs0,
-                        int x_rows, int X_PITCH) {
-  const GeluCoef gc = gelu_coef(act);
+// raw sums are added slice by slice, biased, activated and rounded here.  A thread takes eight elements per turn:
+// the loads of a turn are all issued before the first is used, and the loop body has no branch that depends on
+// the element (an element with nothing to load reads a valid address and is masked afterwards) -- with branches
+// between them the loads went out one latency at a time.
+// One part of the operand: columns [a0, a1) of the activation matrix, all of one kind.
+template <int KIND>
+__device__ __forceinline__ void build_part(const StreamInPart& in, int T, const GeluCoef& gc, int c0, int a0, int a1,
+                                           unsigned char* xbuf, uint32_t xs0, int x_rows, int X_PITCH) {
   const int tid = threadIdx.x;
-  const int groups = (klen + 3) >> 2;          // klen is a multiple of 8
-  constexpr int B = 8;
+  const int groups = (a1 - a0) >> 2;           // part boundaries and k ranges are multiples of 8 columns
   const int total = x_rows * groups;
+  const int qoff = (a0 - c0) >> 2;             // where the part starts inside the operand, in 4-column elements
+  if (KIND == STREAM_IN_BF16) {
+    for (int e = tid; e < total; e += CTHREADS) {
+      const int t = e / groups, q = e - t * groups;
+      if (t < T) {
+        const __nv_bfloat16* src = static_cast<const __nv_bfloat16*>(in.src) + static_cast<long long>(t) * in.ld +
+                                   in.src_col + (a0 - in.col_begin) + 4 * q;
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(xs0 + t * X_PITCH + 8 * (qoff + q)), "l"(src) : "memory");
+      } else {
+        *reinterpret_cast<uint2*>(xbuf + t * X_PITCH + 8 * (qoff + q)) = make_uint2(0u, 0u);
+      }
+    }
+    return;
+  }
+  constexpr int B = 8;
   for (int e0 = tid; e0 < total; e0 += B * CTHREADS) {
     float4 v[B], u[B];
-    int kind[B];
+    bool live[B];
 #pragma unroll
     for (int j = 0; j < B; ++j) {
       const int e = e0 + j * CTHREADS;
-      v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-      u[j] = v[j];
-      kind[j] = -1;                              // nothing to do, or a zero row
-      if (e >= total) continue;
-      const int t = e / groups, q = e - t * groups;
-      kind[j] = -2;                              // zero row
-      if (t >= T) continue;
-      const int col = c0 + 4 * q;
-      const StreamInPart& in = (ph.nin > 1 && col >= ph.in[1].col_begin) ? ph.in[1] : ph.in[0];
-      const long long sc = in.src_col + (col - in.col_begin);
-      kind[j] = in.kind;
-      if (in.kind == STREAM_IN_BF16) {
-        const __nv_bfloat16* src = static_cast<const __nv_bfloat16*>(in.src) + static_cast<long long>(t) * in.ld + sc;
-        asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(xs0 + t * X_PITCH + 8 * q), "l"(src) : "memory");
-      } else {
-        v[j] = load_sum4(in, t, sc);
-        if (in.kind == STREAM_IN_GATED) u[j] = load_sum4(in, t, sc + in.gate_off);
-        else if (in.bias) u[j] = __ldg(reinterpret_cast<const float4*>(in.bias + (col - in.col_begin)));
+      const int ee = e < total ? e : tid % total;   // a valid element to read in any case
+      const int t = ee / groups, q = ee - t * groups;
+      live[j] = e < total && t < T;
+      const long long at = static_cast<long long>(live[j] ? t : 0) * in.ld + in.src_col + (a0 - in.col_begin) + 4 * q;
+      const float* base = static_cast<const float*>(in.src) + at;
+      v[j] = __ldcg(reinterpret_cast<const float4*>(base));
+      if (KIND == STREAM_IN_GATED) u[j] = __ldcg(reinterpret_cast<const float4*>(base + in.gate_off));
+      else u[j] = in.bias ? __ldg(reinterpret_cast<const float4*>(in.bias + (a0 - in.col_begin) + 4 * q))
+                          : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    // further k ranges of the phase before: slice by slice, the eight elements' loads together
+    for (int s = 1; s < in.nslices; ++s) {
+      float4 b[B], bu[B];
+#pragma unroll
+      for (int j = 0; j < B; ++j) {
+        const int e = e0 + j * CTHREADS;
+        const int ee = e < total ? e : tid % total;
+        const int t = ee / groups, q = ee - t * groups;
+        const long long at = static_cast<long long>(live[j] ? t : 0) * in.ld + in.src_col + (a0 - in.col_begin) + 4 * q;
+        const float* base = static_cast<const float*>(in.src) + s * in.slice_stride + at;
+        b[j] = __ldcg(reinterpret_cast<const float4*>(base));
+        if (KIND == STREAM_IN_GATED) bu[j] = __ldcg(reinterpret_cast<const float4*>(base + in.gate_off));
+      }
+#pragma unroll
+      for (int j = 0; j < B; ++j) {
+        v[j].x += b[j].x; v[j].y += b[j].y; v[j].z += b[j].z; v[j].w += b[j].w;
+        if (KIND == STREAM_IN_GATED) { u[j].x += bu[j].x; u[j].y += bu[j].y; u[j].z += bu[j].z; u[j].w += bu[j].w; }
       }
     }
 #pragma unroll
     for (int j = 0; j < B; ++j) {
-      if (kind[j] == -1 || kind[j] == STREAM_IN_BF16) continue;
       const int e = e0 + j * CTHREADS;
+      if (e >= total) continue;
       const int t = e / groups, q = e - t * groups;
-      float4 a = v[j];
-      if (kind[j] == STREAM_IN_GATED) {
-        a.x = silu_fast(a.x) * u[j].x; a.y = silu_fast(a.y) * u[j].y;
-        a.z = silu_fast(a.z) * u[j].z; a.w = silu_fast(a.w) * u[j].w;
-      } else if (kind[j] >= 0) {
-        a.x += u[j].x; a.y += u[j].y; a.z += u[j].z; a.w += u[j].w;     // bias (zero when there is none)
-        if (kind[j] == STREAM_IN_ACT) {
-          a.x = gelu_fast(a.x, gc); a.y = gelu_fast(a.y, gc); a.z = gelu_fast(a.z, gc); a.w = gelu_fast(a.w, gc);
+      float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (live[j]) {
+        if (KIND == STREAM_IN_GATED) {
+          a.x = silu_fast(v[j].x) * u[j].x; a.y = silu_fast(v[j].y) * u[j].y;
+          a.z = silu_fast(v[j].z) * u[j].z; a.w = silu_fast(v[j].w) * u[j].w;
+        } else {
+          a.x = v[j].x + u[j].x; a.y = v[j].y + u[j].y; a.z = v[j].z + u[j].z; a.w = v[j].w + u[j].w;
+          if (KIND == STREAM_IN_ACT) {
+            a.x = gelu_fast(a.x, gc); a.y = gelu_fast(a.y, gc); a.z = gelu_fast(a.z, gc); a.w = gelu_fast(a.w, gc);
+          }
         }
       }
       uint2 o;
       o.x = pack_bf16x2(a.x, a.y);
       o.y = pack_bf16x2(a.z, a.w);
-      *reinterpret_cast<uint2*>(xbuf + t * X_PITCH + 8 * q) = o;
+      *reinterpret_cast<uint2*>(xbuf + t * X_PITCH + 8 * (qoff + q)) = o;
     }
+  }
+}
+
+__device__ void build_x(const StreamPhase& ph, int T, int act, int c0, int klen, unsigned char* xbuf, uint32_t xs0,
+                        int x_rows, int X_PITCH) {
+  const GeluCoef gc = gelu_coef(act);
+  for (int pi = 0; pi < ph.nin; ++pi) {
+    const StreamInPart& in = ph.in[pi];
+    const int a0 = in.col_begin > c0 ? in.col_begin : c0;
+    const int a1 = in.col_end < c0 + klen ? in.col_end : c0 + klen;
+    if (a1 <= a0) continue;
+    if (in.kind == STREAM_IN_BF16) build_part<STREAM_IN_BF16>(in, T, gc, c0, a0, a1, xbuf, xs0, x_rows, X_PITCH);
+    else if (in.kind == STREAM_IN_GATED) build_part<STREAM_IN_GATED>(in, T, gc, c0, a0, a1, xbuf, xs0, x_rows, X_PITCH);
+    else if (in.kind == STREAM_IN_ACT) build_part<STREAM_IN_ACT>(in, T, gc, c0, a0, a1, xbuf, xs0, x_rows, X_PITCH);
+    else build_part<STREAM_IN_LINEAR>(in, T, gc, c0, a0, a1, xbuf, xs0, x_rows, X_PITCH);
   }
   asm volatile("cp.async.wait_all;" ::: "memory");
 }

@@ -4,6 +4,7 @@
 #pragma once
 
 #include "decode_common.cuh"
+#include "decode_stream.h"
 #include "internal.h"
 #include "ptx.cuh"
 
@@ -119,6 +120,25 @@ __device__ __forceinline__ void grid_barrier(int* ctrl, volatile int* s_abort) {
     }
   }
   cbar();
+}
+
+// Four columns of a phase's activation matrix from raw sums of an earlier phase: the slices added in order.
+// The loads of up to four slices are in flight together.
+__device__ __forceinline__ float4 load_sum4(const StreamInPart& in, int t, long long col) {
+  const float* base = static_cast<const float*>(in.src) + static_cast<long long>(t) * in.ld + col;
+  float4 a = __ldcg(reinterpret_cast<const float4*>(base));
+  for (int s0 = 1; s0 < in.nslices; s0 += 4) {
+    float4 b[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      b[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+      if (s0 + j < in.nslices) b[j] = __ldcg(reinterpret_cast<const float4*>(base + (s0 + j) * in.slice_stride));
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      if (s0 + j < in.nslices) { a.x += b[j].x; a.y += b[j].y; a.z += b[j].z; a.w += b[j].w; }
+  }
+  return a;
 }
 
 }  // namespace dst

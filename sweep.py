@@ -152,6 +152,52 @@ def run_point(ctx, cfg, tokens, copies, reps, svd, device="cuda", use_graph=True
     return out
 
 
+def run_quant(ctx, cfg, tokens, copies, reps, device="cuda", use_graph=True, settle=0.0):
+    """The quantised split (Section 5.2: 8-bit heavy / 3-bit light, group 128) at few tokens: time per layer and
+    fraction of the HBM roofline of the QUANTISED bytes, beside the bf16 dense layer's bytes."""
+    hbm, tf, src, _ = peaks()
+    shape = make_shape(cfg.d, cfg.m, cfg.act, cfg.torch_dtype)
+    ctx.ensure_workspace(ctx.quant_workspace_size(shape, cfg.k))
+    padded, logical = ctx.quant_pack_size(shape, cfg.k)
+    _, logical_dense = ctx.pack_size(shape, cfg.m, 0)
+    blobs = []
+    for c in range(copies):
+        L = make_layer(cfg, c, device=device)
+        heavy = L.planted.to(torch.int32)
+        mask = torch.ones(cfg.m, dtype=torch.bool, device=device)
+        mask[heavy.long()] = False
+        light = torch.nonzero(mask).flatten().to(torch.int32)
+        b = torch.empty(padded, dtype=torch.uint8, device=device)
+        ctx.quant_pack(shape, L.W1, L.b1, L.W2, L.b2, heavy, cfg.k, light, b, W1u=L.W1u)
+        ctx.poll()
+        blobs.append(b)
+        del L
+    out = []
+    gen = torch.Generator(device=device)
+    gen.manual_seed(4321)
+    for T in tokens:
+        X = (torch.randn(T, cfg.d, generator=gen, device=device, dtype=torch.float32)).to(cfg.torch_dtype)
+        Y = torch.empty_like(X)
+        state = {"i": 0}
+
+        def call():
+            ctx.quant_forward(blobs[state["i"] % copies], X, Y)
+            state["i"] += 1
+
+        ts, mode = time_calls(call, copies * max(1, 16 // copies), reps, max(3, copies), use_graph, settle)
+        ctx.poll()
+        ms = statistics.median(ts)
+        bytes_ = logical + 2 * T * cfg.d * 2
+        out.append({"config": cfg.name, "d": cfg.d, "m": cfg.m, "k": cfg.k, "act": cfg.act, "tokens": T, "launch_mode": mode,
+                    "weight_copies_cycled": copies, "peaks": src,
+                    "quant": {"ms_per_layer": ms, "ms_best": min(ts), "tokens_per_s_per_layer": T / (ms * 1e-3),
+                              "tokens_per_s_per_stack": T / (ms * 1e-3 * cfg.layers), "model_bytes_per_layer": logical,
+                              "roofline_ms": bytes_ / (hbm * 1e9) * 1e3, "roofline_frac": bytes_ / (hbm * 1e9) * 1e3 / ms,
+                              "gbs": bytes_ / (ms * 1e-3) / 1e9, "bits_per_weight": 8.0 * (logical - 4 * (cfg.m + cfg.d)) / ((cfg.n_in + 1) * cfg.d * cfg.m)},
+                    "size_ratio_vs_bf16_dense": logical / logical_dense})
+    return out
+
+
 def run_scoring(ctx, cfg, reps, device="cuda", t_cal=None):
     """Scoring pass of one layer, both forms: from the calibration tokens (product + fused column energy)
     and from a stored activation matrix (one streaming read of H).  Events around each call, median."""
@@ -207,6 +253,7 @@ def main():
                     help="the paper's own hyper-parameters at BERT-base shape (Section 5.1.1): top 25 %% of the neurons "
                          "heavy (k = 768), light rank = 10 %% of full rank (r = 77); --config is ignored")
     ap.add_argument("--scoring", action="store_true", help="time the scoring pass (both forms) instead of the forward")
+    ap.add_argument("--quant", action="store_true", help="time the quantised split (Section 5.2) at the given few-token counts")
     ap.add_argument("--t-cal", type=int, default=0, help="with --scoring: calibration tokens (default: the config's)")
     ap.add_argument("--settle", type=float, default=1.0,
                     help="seconds of idle time before each timed case (the clocks recover from the case before)")
@@ -228,6 +275,13 @@ def main():
         return
     tokens = args.tokens or list(base.t_fwd)
     lines = []
+    if args.quant:
+        qbytes = 0.45 * (base.n_in + 1) * base.d * base.m          # about 3.5 bits per weight
+        copies = args.copies or max(2, min(24, int(-(-2 * 126 * (1 << 20) // qbytes))))
+        for res in run_quant(ctx, base, [t for t in tokens if t <= 8] or [1], copies, args.reps, use_graph=not args.no_graph,
+                             settle=args.settle):
+            print(json.dumps(res), flush=True)
+        return
     for cfg in points:
         es = 2 if cfg.dtype == "bf16" else 4
         split_bytes = es * (cfg.n_in + 1) * (cfg.d * cfg.k + cfg.r * (cfg.d + cfg.m - cfg.k))
