@@ -167,7 +167,20 @@ class StackWorkload:
         need = max(ctx.stack_workspace_size(self.blobs, t) for t in (T, 32, 1))
         if dense:
             need = max(need, max(ctx.stack_workspace_size(self.blobs_dense, t) for t in (T, 32, 1)))
+            need = max(need, ctx.quant_workspace_size(self.shape, cfg.k))
         ctx.ensure_workspace(need)
+        # the quantised split of the same layers (Section 5.2: 8-bit heavy, 3-bit light, group 128), for the few-token phase
+        self.blobs_quant = []
+        if dense:
+            qpadded, self.logical_bytes_quant = ctx.quant_pack_size(self.shape, cfg.k)
+            for e in self.layers:
+                L = e["L"]
+                bq = torch.empty(qpadded, dtype=torch.uint8, device=device)
+                ctx.quant_pack(self.shape, L.W1, L.b1, L.W2, L.b2, e["heavy"], cfg.k, e["light"], bq, W1u=L.W1u)
+                self.blobs_quant.append(bq)
+            ctx.poll()
+            self.q_ping = torch.empty(8, cfg.d, dtype=cfg.torch_dtype, device=device)
+            self.q_pong = torch.empty(8, cfg.d, dtype=cfg.torch_dtype, device=device)
 
     # -- calibration: score + select + pack of one layer on context c (current stream)
     def calibrate_layer(self, e, c, x_host=None):
@@ -205,6 +218,16 @@ class StackWorkload:
     def forward(self, dense=False, x=None, y=None):
         self.ctx.forward_stack(self.blobs_dense if dense else self.blobs, self.X if x is None else x,
                                self.Y if y is None else y)
+
+    def forward_quant(self, x, y):
+        """The quantised stack at a few tokens: layer l reads what layer l - 1 wrote."""
+        t = x.shape[0]
+        bufs = (self.q_ping[:t], self.q_pong[:t])
+        src = x
+        for i, b in enumerate(self.blobs_quant):
+            dst = y if i == len(self.blobs_quant) - 1 else bufs[i & 1]
+            self.ctx.quant_forward(b, src, dst)
+            src = dst
 
     def step(self):
         self.calibrate()
@@ -393,6 +416,14 @@ def run_ours(args):
                          "tokens_per_s_per_stack": Tp / (ms * 1e-3), "tokens_per_s_per_layer": Tp * n_layers / (ms * 1e-3),
                          "roofline_us_per_layer": 1e3 * roof, "bound": bound, "roofline_frac": roof * n_layers / ms}
         row["split_vs_dense_speedup"] = row["dense"]["ms_per_stack"] / row["split"]["ms_per_stack"]
+        if Tp == 1:
+            ms = timed(lambda: wl.forward_quant(Xp, Yp))
+            qb = wl.logical_bytes_quant + 2.0 * Tp * cfg.d * 2
+            roof = qb / (peaks["hbm_gbs"] * 1e9) * 1e3
+            row["quantised_8bit_heavy_3bit_light_g128"] = {
+                "ms_per_stack": ms, "us_per_layer": 1e3 * ms / n_layers, "tokens_per_s_per_stack": Tp / (ms * 1e-3),
+                "model_bytes_per_layer": wl.logical_bytes_quant, "roofline_us_per_layer": 1e3 * roof, "bound": "hbm",
+                "roofline_frac": roof * n_layers / ms}
         phases[f"forward_T{Tp}"] = row
         wl.poll()
     phases["model_bytes_split_per_layer"] = wl.logical_bytes
