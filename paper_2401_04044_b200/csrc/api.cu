@@ -425,6 +425,7 @@ ffsplit_status ffsplit_create(ffsplit_ctx** out, int device) {
   c->cc_minor = minor;
   c->num_sms = sms;
   if (const char* env = std::getenv("FFSPLIT_GEMM_TWO_M")) c->gemm_two_m = env[0] == '0' ? 0 : env[0] == '2' ? 2 : 1;
+  if (const char* env = std::getenv("FFSPLIT_GEMM_PANEL")) c->gemm_panel = std::atoi(env);
   if (const char* env = std::getenv("FFSPLIT_DECODE_LAYER")) c->decode_one_launch = env[0] == '0' ? 0 : 1;
   if (const char* env = std::getenv("FFSPLIT_DECODE_STREAM")) c->decode_stream = env[0] == '0' ? 0 : env[0] == '2' ? 2 : 1;
   *out = c;
