@@ -144,6 +144,10 @@ FwdLayout fwd_layout(const SplitDims& D, int d, int dtype, int act, long long T)
     const size_t fs = fused_light_scratch_bytes(T, D.r_pad);
     if (fs > hl) hl = fs;
   }
+  if (fused_layer_applies(dtype, act, d, D.k, D.k_pad, D.r_pad, D.ml_pad, T, 1 << 20)) {   // whatever the SM count
+    const size_t fs = fused_layer_scratch_bytes(T, D.r_pad);
+    if (fs > hl) hl = fs;
+  }
   L.hl = off; off = align_up(off + hl);
   L.xs = off; off = align_up(off + (size_t)T * d * es);
   L.ys = off; off = align_up(off + (size_t)T * d * es);
@@ -217,6 +221,10 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
   const bool light = D.r_pad > 0 && D.ml > 0;
   ffsplit_status s;
   GemmArgs g;
+
+  // ---- small hidden widths: the whole layer in one launch, a cluster of four CTAs per 128-token tile
+  if (light && ctx->use_layer_kernel && fused_layer_applies(h.dtype, h.act, d, D.k, D.k_pad, D.r_pad, D.ml_pad, T, ctx->num_sms))
+    return launch_fused_layer(ctx, h, blob, X, T, HL, Y, guard_hash, st);
 
   // ---- stage 1: [A_H | Q] = X [U1 | A1], activation on the heavy columns only
   if (!gated) {
@@ -426,6 +434,7 @@ ffsplit_status ffsplit_create(ffsplit_ctx** out, int device) {
   c->num_sms = sms;
   if (const char* env = std::getenv("FFSPLIT_GEMM_TWO_M")) c->gemm_two_m = env[0] == '0' ? 0 : env[0] == '2' ? 2 : 1;
   if (const char* env = std::getenv("FFSPLIT_GEMM_PANEL")) c->gemm_panel = std::atoi(env);
+  if (const char* env = std::getenv("FFSPLIT_LAYER_KERNEL")) c->use_layer_kernel = env[0] == '0' ? 0 : 1;
   if (const char* env = std::getenv("FFSPLIT_DECODE_LAYER")) c->decode_one_launch = env[0] == '0' ? 0 : 1;
   if (const char* env = std::getenv("FFSPLIT_DECODE_STREAM")) c->decode_stream = env[0] == '0' ? 0 : env[0] == '2' ? 2 : 1;
   *out = c;

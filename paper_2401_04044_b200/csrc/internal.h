@@ -193,6 +193,7 @@ struct ffsplit_ctx {
   bool prep_active = false;
   bool attr_tc_set = false;
   bool attr_fused_set = false;
+  bool attr_layer_set = false;
   int* status() const { return reinterpret_cast<int*>(ws); }
   int* tickets() const { return reinterpret_cast<int*>(ws + ffsp::kStatusBytes); }
   int gemm_two_m = 1;          // tensor-core GEMM: 256-row tiles where they pay (FFSPLIT_GEMM_TWO_M=0: never, 2: wherever allowed)
@@ -200,6 +201,7 @@ struct ffsplit_ctx {
   int decode_one_launch = 0;   // few-token forward: 1 = all products in one cooperative launch (FFSPLIT_DECODE_LAYER=1), 0 = one launch per product
   int decode_stream = 1;       // few tokens: 1 = the single-launch streaming kernel where it is the faster one, 2 = for every T <= 8, 0 = never (FFSPLIT_DECODE_STREAM)
   int use_fused = -1;  // -1: not decided yet (environment FFSPLIT_NO_FUSED=1 turns the fused kernel off)
+  int use_layer_kernel = 1;    // small hidden widths at prefill: the whole split layer in one cluster launch (FFSPLIT_LAYER_KERNEL=0: off)
   // What the scoring region of the workspace holds from the last ffsplit_score() call: U^T, the fp32 bias
   // and ||V_j||^2 of these weights.  A later batch of the same accumulation (accumulate = 1, same pointers
   // and shape) reuses them; any other call that writes the workspace clears `valid`.
@@ -305,6 +307,10 @@ ffsplit_status launch_fused_light(ffsplit_ctx* ctx, const void* Q, long long ldq
                                   const void* A2T, const float* b1l, int r_pad, int ml_pad, int act, void* P,
                                   long long ldp, char* scratch, int* tickets, double algo_flops,
                                   cudaStream_t st);
+bool fused_layer_applies(int dtype, int act, int d, int k, int k_pad, int r_pad, int ml_pad, long long T, int num_sms);
+size_t fused_layer_scratch_bytes(long long T, int r_pad);
+ffsplit_status launch_fused_layer(ffsplit_ctx* ctx, const BlobHeader& h, const char* blob, const void* X, long long T,
+                                  char* scratch, void* Y, unsigned long long guard_hash, cudaStream_t st);
 ffsplit_status launch_wait_timeout_probe(ffsplit_ctx* ctx, long long limit_cycles, cudaStream_t st);
 ffsplit_status launch_to_f32(ffsplit_ctx* ctx, int dtype, const void* in, int n, float* out, cudaStream_t st);
 

@@ -257,10 +257,31 @@ FUSED_CASES = [
 ]
 
 
+def forward_on_fresh_context(G, blob, X, T, k, r):
+    """The same blob through a context created under the current environment switches."""
+    from paper_2401_04044_b200 import Context
+    c = Context(0)
+    try:
+        c.ensure_workspace(c.workspace_size(G.shape, T, 0, k, r))
+        c.blob_open(blob)      # packed on another context
+        Xd = X.cuda()
+        Y = torch.empty_like(Xd)
+        c.forward(blob, Xd, Y)
+        c.poll()
+        Y2 = torch.empty_like(Xd)
+        c.forward(blob, Xd, Y2)
+        c.poll()
+        assert torch.equal(Y, Y2), "forward is not bitwise reproducible"
+    finally:
+        c.close()
+    return Y
+
+
 @pytest.mark.parametrize("d,m,k,r,T", FUSED_CASES)
 @pytest.mark.parametrize("act", ["gelu_erf", "gelu_tanh"])
 def test_fused_light_chain_matches_oracle_and_unfused_path(ctx, act, d, m, k, r, T, monkeypatch):
-    from paper_2401_04044_b200 import Context
+    """Three launches per layer (stage 1, fused light chain, stage 3) against the oracle and against the
+    four-GEMM path; the one-launch layer kernel, which would take these shapes, is switched off."""
     cfg = custom_config(d, m, k, r, act=act, dtype="bf16")
     L = make_layer(cfg, 7)
     G = GpuLayer(ctx, L)
@@ -268,23 +289,48 @@ def test_fused_light_chain_matches_oracle_and_unfused_path(ctx, act, d, m, k, r,
     fac = oracle_factors(L, L.planted.numpy(), r)
     blob, _ = G.pack(L.planted, fac)
     X = L.tokens(T)
-    Y = G.forward(blob, X)
     Yref = oracle_split(L, L.planted.numpy(), fac, X)
+    monkeypatch.setenv("FFSPLIT_LAYER_KERNEL", "0")
+    Y = forward_on_fresh_context(G, blob, X, T, k, r)
     assert_close(Y, Yref, "bf16", "fused light chain")
-    assert torch.equal(G.forward(blob, X), Y), "fused forward is not bitwise reproducible"
-    # the same blob through the unfused GEMM chain (second context, fused kernel switched off)
     monkeypatch.setenv("FFSPLIT_NO_FUSED", "1")
-    ctx2 = Context(0)
-    try:
-        ctx2.ensure_workspace(ctx2.workspace_size(G.shape, T, 0, k, r))
-        ctx2.blob_open(blob)      # packed on another context
-        Xd = X.cuda()
-        Y2 = torch.empty_like(Xd)
-        ctx2.forward(blob, Xd, Y2)
-        ctx2.poll()
-    finally:
-        ctx2.close()
+    Y2 = forward_on_fresh_context(G, blob, X, T, k, r)
     assert_close(Y2, Yref, "bf16", "unfused light chain")
+    assert orc.rel_frobenius(f64(Y2), f64(Y)) < 1e-2
+
+
+# one-launch layer (bf16 GELU, d <= 1024, k_pad and r_pad <= 256): a cluster of four CTAs per 128-token tile
+LAYER_CASES = [
+    # d, m, k, r, T
+    (768, 3072, 154, 192, 4096),   # BERT-base shape: one full wave of clusters
+    (768, 3072, 154, 192, 333),    # ragged last tile
+    (1024, 4096, 205, 256, 200),   # GPT-2-medium shape: widest accumulators, two-slot rings
+    (64, 130, 2, 48, 77),          # 16 output columns per CTA; one chunk only: three ranks have no light neurons
+    (128, 2000, 30, 80, 65),       # r_pad = 80: partial k-block of Q and P; smallest token count of the path
+    (256, 1024, 250, 16, 700),     # k_pad = 256 (widest heavy part), smallest rank
+    (512, 700, 1, 64, 129),        # one heavy neuron
+]
+
+
+@pytest.mark.parametrize("d,m,k,r,T", LAYER_CASES)
+@pytest.mark.parametrize("act", ["gelu_erf", "gelu_tanh"])
+def test_one_launch_layer_matches_oracle_and_staged_path(ctx, act, d, m, k, r, T, monkeypatch):
+    cfg = custom_config(d, m, k, r, act=act, dtype="bf16")
+    L = make_layer(cfg, 11)
+    G = GpuLayer(ctx, L)
+    G.reserve(T, 0, k, r)
+    fac = oracle_factors(L, L.planted.numpy(), r)
+    blob, _ = G.pack(L.planted, fac)
+    X = L.tokens(T)
+    n0 = ctx.launch_count()
+    Y = G.forward(blob, X)
+    assert ctx.launch_count() - n0 == 1, "the whole layer is one launch"
+    rows = slice(None) if T <= 1024 else slice(5, None, 8)
+    Yref = oracle_split(L, L.planted.numpy(), fac, X[rows])
+    assert_close(Y[rows], Yref, "bf16", "one-launch layer")
+    assert torch.equal(G.forward(blob, X), Y), "forward is not bitwise reproducible"
+    monkeypatch.setenv("FFSPLIT_LAYER_KERNEL", "0")
+    Y2 = forward_on_fresh_context(G, blob, X, T, k, r)
     assert orc.rel_frobenius(f64(Y2), f64(Y)) < 1e-2
 
 
