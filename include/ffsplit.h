@@ -287,6 +287,31 @@ ffsplit_status ffsplit_forward_stack_host(ffsplit_ctx* ctx, const void* const* b
 ffsplit_status ffsplit_forward_noalloc(ffsplit_ctx* ctx, const void* blob, const void* X, int64_t T,
                                        void* Y, void* stream);
 
+/* ---- On-device factors of the light slices (Section 5.1.1: the low-rank decomposition is applied to U2
+ * and V2 only; Section 5.1.1 fixes the rank, not the algorithm) --------------------------------------------
+ * The step between ffsplit_select() and ffsplit_pack() without leaving the GPU.  For W = U2 = W1[:, light]
+ * (d x (m-k)), for the SwiGLU up slice likewise, and for W = V2^T with V2 = W2[light, :], an orthonormal basis
+ * Q [d, r] of the dominant left singular subspace is found by `iters` rounds of block power iteration
+ * (Y = W W^T Q on the tensor cores in bf16 with fp32 accumulation, Q = orth(Y) by Cholesky QR in fp32) from
+ * the starting basis the caller supplies, and the factors of the projection Q Q^T W are returned:
+ *     U2 ~ A1 B1,  A1 = Q, B1 = Q^T U2            V2 ~ A2 B2,  A2 = V2 Q, B2 = Q^T
+ * As span(Q) converges to the leading singular subspace, A B converges to the truncated SVD's product, the
+ * best rank-r approximation (Eckart-Young); the factors themselves differ from U_r S_r^(1/2), S_r^(1/2) V_r^T
+ * by an invertible r x r mixing, which the forward does not see.  With a random starting basis, 6 rounds bring
+ * the Frobenius error within about 1 % of the optimum on the layers the tests use (tests/test_gpu_factor.py).
+ *   light_idx  dev int32[m-k], ascending (ffsplit_select's output); an index outside [0, m) reads as a zero neuron
+ *   start      dev bf16 [n][r, d], n = 2 (GELU: bases for U2, V2) or 3 (SwiGLU: gate, V2, up); full row rank
+ *              (draw it from a normal distribution: the library draws no random numbers)
+ *   A1 [d, r], B1 [r, m-k], A2 [m-k, r], B2 [r, d] (and A1u, B1u for SwiGLU, else NULL): dev bf16, written;
+ *              the layouts ffsplit_factors takes
+ * bf16 layers, 1 <= r <= min(d, m-k, 2048), 0 <= iters <= 64.  Uses the workspace (ffsplit_factor_workspace_size).
+ * A Gram matrix that is not positive definite (a rank-deficient start or slice) is reported as
+ * FFSPLIT_ERR_NONFINITE through ffsplit_poll(); the factors are then finite but meaningless. */
+ffsplit_status ffsplit_factor_workspace_size(const ffsplit_shape* shape, int32_t k, int32_t r, size_t* bytes);
+ffsplit_status ffsplit_factor_light(ffsplit_ctx* ctx, const ffsplit_shape* shape, const ffsplit_weights* weights,
+                                    const int32_t* light_idx, int32_t k, int32_t r, int32_t iters, const void* start,
+                                    void* A1, void* B1, void* A2, void* B2, void* A1u, void* B1u, void* stream);
+
 /* ---- Quantised split (Section 5.2, Table 3: round-to-nearest, group size 128, 8 bits for the heavy-hitter
  * neurons, 3 bits for everything else) ------------------------------------------------------------------
  * The second way the paper compresses the light part: instead of rank-r factors, U2 and V2 are kept whole at

@@ -37,6 +37,7 @@ EXPORTS = [
     "ffsplit_blob_close", "ffsplit_stack_workspace_size", "ffsplit_forward_stack", "ffsplit_forward_stack_host",
     "ffsplit_debug_wait_timeout", "ffsplit_quant_pack_size", "ffsplit_quant_workspace_size", "ffsplit_quant_pack",
     "ffsplit_quant_blob_open", "ffsplit_quant_unpack", "ffsplit_quant_forward",
+    "ffsplit_factor_workspace_size", "ffsplit_factor_light",
 ]
 
 
@@ -98,6 +99,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.ffsplit_quant_blob_open.argtypes = [vp, vp, sz, vp]
     lib.ffsplit_quant_unpack.argtypes = [vp, vp, i32, vp, vp, vp, vp]
     lib.ffsplit_quant_forward.argtypes = [vp, vp, vp, i64, vp, vp]
+    lib.ffsplit_factor_workspace_size.argtypes = [vp, i32, i32, P(sz)]
+    lib.ffsplit_factor_light.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.ffsplit_blob_section.argtypes = [vp, vp, i32, P(sz), P(i64), P(i64), P(i64)]
     lib.ffsplit_forward.argtypes = [vp, vp, vp, i64, vp, vp]
     lib.ffsplit_forward_host.argtypes = [vp, vp, vp, i64, vp, vp]
@@ -257,6 +260,30 @@ class Context:
         self._check(self.lib.ffsplit_forward_stack_host(self.h, self._blob_array(blobs), len(blobs), _ptr(X_host),
                                                         X_host.shape[0], _ptr(Y_host), _stream_ptr(stream)),
                     "ffsplit_forward_stack_host")
+
+    # ------------------------------------------------------------------ on-device light factors (Section 5.1.1)
+    def factor_workspace_size(self, shape: Shape, k: int, r: int) -> int:
+        n = C.c_size_t()
+        self._check(self.lib.ffsplit_factor_workspace_size(C.byref(shape), k, r, C.byref(n)), "ffsplit_factor_workspace_size")
+        return n.value
+
+    def factor_light(self, shape: Shape, W1, W2, light_idx, k: int, r: int, iters: int, start, W1u=None, stream=None) -> dict:
+        """ffsplit_factor_light: rank-r factors of the light slices as a dict ready for pack().  `start` is the
+        [n, r, d] starting basis (n = 2, or 3 with W1u) in the layer's dtype."""
+        d, m = shape.d, shape.m
+        ml = m - k
+        dev, dt = W1.device, W1.dtype
+        f = {"A1": torch.empty(d, r, dtype=dt, device=dev), "B1": torch.empty(r, ml, dtype=dt, device=dev),
+             "A2": torch.empty(ml, r, dtype=dt, device=dev), "B2": torch.empty(r, d, dtype=dt, device=dev)}
+        if W1u is not None:
+            f["A1u"] = torch.empty(d, r, dtype=dt, device=dev)
+            f["B1u"] = torch.empty(r, ml, dtype=dt, device=dev)
+        w = Weights(_ptr(W1), _ptr(W1u), None, _ptr(W2), None)
+        self._check(self.lib.ffsplit_factor_light(self.h, C.byref(shape), C.byref(w), _ptr(light_idx), k, r, iters,
+                                                  _ptr(start), _ptr(f["A1"]), _ptr(f["B1"]), _ptr(f["A2"]), _ptr(f["B2"]),
+                                                  _ptr(f.get("A1u")), _ptr(f.get("B1u")), _stream_ptr(stream)),
+                    "ffsplit_factor_light")
+        return f
 
     # ------------------------------------------------------------------ quantised split (Section 5.2)
     def quant_pack_size(self, shape: Shape, k: int):

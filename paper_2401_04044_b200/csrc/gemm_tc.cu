@@ -82,6 +82,20 @@ __device__ __forceinline__ void epilogue_chunk_store(const Params& p, const Gelu
     for (int i = 0; i < 16; ++i) v[i] = gelu_fast(v[i], gc);
   }
   if (row >= p.M) return;
+  if (e.c0_f32) {
+    // fp32 output (n_split >= N): 64 bytes per lane, in 16-byte pieces where the address allows
+    float* base = reinterpret_cast<float*>(e.C0) + row * e.ld0 + n0;
+    if (n0 + 16 <= p.N && (reinterpret_cast<uintptr_t>(base) & 15u) == 0) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+        reinterpret_cast<float4*>(base)[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+    } else {
+#pragma unroll
+      for (int i = 0; i < 16; ++i)
+        if (n0 + i < p.N) base[i] = v[i];
+    }
+    return;
+  }
   const bool first = n0 < e.n_split;
   __nv_bfloat16* base = first ? reinterpret_cast<__nv_bfloat16*>(e.C0) + row * e.ld0 + n0
                               : reinterpret_cast<__nv_bfloat16*>(e.C1) + row * e.ld1 + (n0 - e.n_split);

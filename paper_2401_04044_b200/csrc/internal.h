@@ -30,7 +30,7 @@ constexpr size_t kCtrlBytes = 65536;
 constexpr long long kMaxTicketTiles = (kCtrlBytes - kStatusBytes) / 4;
 
 enum KernelId : int {
-  KID_SELECT = 1, KID_PACK = 2, KID_GEMM_TC = 3, KID_GEMM_SIMT = 4, KID_SCORE = 5, KID_DECODE = 6, KID_FUSED = 7, KID_PROBE = 8, KID_QUANT = 9
+  KID_SELECT = 1, KID_PACK = 2, KID_GEMM_TC = 3, KID_GEMM_SIMT = 4, KID_SCORE = 5, KID_DECODE = 6, KID_FUSED = 7, KID_PROBE = 8, KID_QUANT = 9, KID_FACTOR = 10
 };
 
 __device__ __forceinline__ void record_status(int* status, int code, int detail, int kid) {
@@ -65,6 +65,7 @@ struct Epilogue {
   int n_bias;
   int act;        // ffsplit_act
   int score_abs;  // 1: accumulate |v| instead of v^2
+  int c0_f32;     // tensor-core kernel only: C0 is float (the Gram matrices of the on-device factorisation)
   // Blob guard (first kernel of a forward only, else nullptr): the 256-byte header at `guard` must still
   // hash to `guard_hash`, the value taken when the blob was packed or opened on this context; a blob whose
   // bytes were replaced behind the library's back is reported as FFSPLIT_ERR_BAD_BLOB through the status block.

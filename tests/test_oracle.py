@@ -225,6 +225,46 @@ def test_light_factors_known_spectrum(rng):
     assert np.allclose(A @ B, (Q1[:, :3] * s[:3]) @ Q2[:, :3].T, atol=1e-12)
 
 
+def test_orthogonal_iteration_factors_against_eckart_young(rng):
+    """The iteration the on-device factorisation follows, pinned to what the mathematics fixes: a projection can
+    never beat the truncated SVD, it equals it when the spectrum has a gap and the iteration has converged, it is
+    exact for a matrix of rank <= r, and on a flat (Gaussian) spectrum six rounds come within 1 % of the optimum."""
+    d, n, r = 24, 70, 6
+    # gapped spectrum: known singular vectors
+    P, _ = np.linalg.qr(rng.normal(size=(d, d)))
+    V, _ = np.linalg.qr(rng.normal(size=(n, d)))
+    sv = np.concatenate([np.linspace(10, 6, r), np.linspace(1.0, 0.1, d - r)])
+    W = (P * sv) @ V.T
+    start = rng.normal(size=(d, r))
+    opt = np.sqrt(np.sum(sv[r:] ** 2))
+    prev = np.inf
+    for iters in (0, 1, 2, 6, 12):
+        A, B = orc.orthogonal_iteration_factors(W, r, iters, start)
+        assert A.shape == (d, r) and B.shape == (r, n)
+        err = np.linalg.norm(W - A @ B)
+        assert err >= opt * (1 - 1e-12) and err <= prev * (1 + 1e-12)      # never below Eckart-Young, monotone here
+        prev = err
+        if iters > 0:
+            assert np.allclose(A.T @ A, np.eye(r), atol=1e-12)            # orthonormal basis
+            assert np.allclose(A @ B, A @ (A.T @ W), atol=1e-12)          # the projection Q Q^T W
+    assert abs(prev - opt) < 1e-6 * opt
+    A, B = orc.orthogonal_iteration_factors(W, r, 12, start)
+    assert np.allclose(A @ B, (P[:, :r] * sv[:r]) @ V[:, :r].T, atol=1e-6)  # the truncated SVD's product itself
+    # rank(W) <= r: one round reproduces W
+    W0 = rng.normal(size=(d, 4)) @ rng.normal(size=(4, n))
+    A, B = orc.orthogonal_iteration_factors(W0, r, 1, start)
+    assert np.allclose(A @ B, W0, atol=1e-10)
+    # flat spectrum (the synthetic layers' light slices are Gaussian): within 1 % of the optimum after 6 rounds
+    G = rng.normal(size=(64, 400))
+    s2 = np.linalg.svd(G, compute_uv=False) ** 2
+    for rr in (8, 16):
+        A, B = orc.orthogonal_iteration_factors(G, rr, 6, rng.normal(size=(64, rr)))
+        err, best = np.linalg.norm(G - A @ B), np.sqrt(np.sum(s2[rr:]))
+        assert best <= err <= 1.01 * best
+    with pytest.raises(ValueError):
+        orc.orthogonal_iteration_factors(W, r, 1, rng.normal(size=(d, r + 1)))
+
+
 # ---------------------------------------------------------------- split FFN
 def _full_rank_factors(sw, act):
     f = {}
