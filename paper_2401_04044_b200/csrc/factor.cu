@@ -25,15 +25,20 @@
 namespace ffsp {
 namespace fac {
 
-// In-place Cholesky factorisation of the leading r x r block of G (row-major, pitch ld), lower triangle.
-// One CTA; right-looking, one column per step.  A pivot that is not a positive finite number is reported
-// (FFSPLIT_ERR_NONFINITE, detail = column) and replaced by 1 so that the kernel finishes with finite numbers.
+// In-place Cholesky factorisation of the leading r x r block of G (row-major, pitch ld), lower triangle,
+// right-looking in block columns of NB: one CTA factors the block column (panel_kernel), then a grid of CTAs
+// applies it to the trailing matrix, one 32 x 32 tile of the lower triangle each (update_kernel).  A pivot
+// that is not a positive finite number is reported (FFSPLIT_ERR_NONFINITE, detail = column) and replaced by 1
+// so that the factorisation finishes with finite numbers.
+constexpr int NB = 32;
 constexpr int CHOL_THREADS = 1024;
-__global__ void __launch_bounds__(CHOL_THREADS) cholesky_kernel(float* G, int r, int ld, int* status) {
+__global__ void __launch_bounds__(CHOL_THREADS) chol_panel_kernel(float* G, int r, int ld, int j0, int* status) {
   __shared__ float col[2048];
   __shared__ float pivot;
   pdl_wait();
-  for (int j = 0; j < r; ++j) {
+  const int j1 = j0 + NB < r ? j0 + NB : r;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int j = j0; j < j1; ++j) {
     if (threadIdx.x == 0) {
       float p = G[static_cast<size_t>(j) * ld + j];
       if (!(p > 0.f) || !isfinite(p)) {
@@ -51,15 +56,38 @@ __global__ void __launch_bounds__(CHOL_THREADS) cholesky_kernel(float* G, int r,
       col[i] = v;
     }
     __syncthreads();
-    // trailing update of the lower triangle: G[i, l] -= L[i, j] L[l, j] for j < l <= i
-    // (one warp per row, lanes along the row: coalesced and free of index divisions)
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // the rest of this block column: G[i, l] -= L[i, j] L[l, j] for j < l < j1, l <= i (one warp per row)
     for (int i = j + 1 + warp; i < r; i += CHOL_THREADS / 32) {
-      const float li = col[i];
-      float* row = G + static_cast<size_t>(i) * ld;
-      for (int l = j + 1 + lane; l <= i; l += 32) row[l] -= li * col[l];
+      const int l = j + 1 + lane;
+      if (l < j1 && l <= i) G[static_cast<size_t>(i) * ld + l] -= col[i] * col[l];
     }
     __syncthreads();
+  }
+}
+
+// Trailing update with a finished block column P = L[:, j0 .. j0 + NB): G[i, l] -= sum_k P[i, k] P[l, k] for
+// j0 + NB <= l <= i.  CTA t owns tile (a, b), b <= a, of the trailing lower triangle (t = a (a + 1) / 2 + b).
+__global__ void __launch_bounds__(CHOL_THREADS) chol_update_kernel(float* G, int r, int ld, int j0) {
+  __shared__ float Pi[NB][NB + 1];
+  __shared__ float Pl[NB][NB + 1];
+  pdl_wait();
+  const int t = blockIdx.x;
+  int a = static_cast<int>((sqrtf(8.0f * t + 1.0f) - 1.0f) * 0.5f);
+  while (a * (a + 1) / 2 > t) --a;
+  while ((a + 1) * (a + 2) / 2 <= t) ++a;
+  const int b = t - a * (a + 1) / 2;
+  const int n0 = j0 + NB;
+  const int ty = threadIdx.x >> 5, tx = threadIdx.x & 31;
+  const int ri = n0 + NB * a + ty, rl = n0 + NB * b + ty;
+  Pi[ty][tx] = ri < r ? G[static_cast<size_t>(ri) * ld + j0 + tx] : 0.f;
+  Pl[ty][tx] = rl < r ? G[static_cast<size_t>(rl) * ld + j0 + tx] : 0.f;
+  __syncthreads();
+  const int i = n0 + NB * a + ty, l = n0 + NB * b + tx;
+  if (i < r && l <= i) {
+    float s = 0.f;
+#pragma unroll
+    for (int k = 0; k < NB; ++k) s = fmaf(Pi[ty][k], Pl[tx][k], s);
+    G[static_cast<size_t>(i) * ld + l] -= s;
   }
 }
 
@@ -190,9 +218,17 @@ ffsplit_status iterate(ffsplit_ctx* ctx, const FactorLayout& L, char* base, int 
     if ((s = thin_gemm(ctx, cur, d, Wd, d, r, L.np, d, Zt, L.np, false, st)) != FFSPLIT_OK) return s;
     if ((s = thin_gemm(ctx, Zt, L.np, Wn, L.np, r, d, L.np, Yt, d, false, st)) != FFSPLIT_OK) return s;
     if ((s = thin_gemm(ctx, Yt, d, Yt, d, r, r, d, G, L.rp, true, st)) != FFSPLIT_OK) return s;
-    cudaError_t e = launch_pdl(fac::cholesky_kernel, dim3(1), dim3(fac::CHOL_THREADS), 0, st, G, r, L.rp, ctx->status());
-    ctx->launches++;
-    if (e != cudaSuccess) return check_cuda(ctx, e, "cholesky_kernel launch");
+    cudaError_t e = cudaSuccess;
+    for (int j0 = 0; j0 < r && e == cudaSuccess; j0 += fac::NB) {
+      e = launch_pdl(fac::chol_panel_kernel, dim3(1), dim3(fac::CHOL_THREADS), 0, st, G, r, L.rp, j0, ctx->status());
+      ctx->launches++;
+      const int tb = (r - j0 - fac::NB + fac::NB - 1) / fac::NB;   // tile rows of the trailing matrix
+      if (e == cudaSuccess && tb > 0) {
+        e = launch_pdl(fac::chol_update_kernel, dim3(tb * (tb + 1) / 2), dim3(fac::CHOL_THREADS), 0, st, G, r, L.rp, j0);
+        ctx->launches++;
+      }
+    }
+    if (e != cudaSuccess) return check_cuda(ctx, e, "Cholesky kernel launch");
     e = launch_pdl(fac::trsm_kernel, dim3((d + fac::TRSM_THREADS - 1) / fac::TRSM_THREADS), dim3(fac::TRSM_THREADS), 0,
                    st, static_cast<const float*>(G), L.rp, reinterpret_cast<const __nv_bfloat16*>(Yt), r, d, Qf,
                    reinterpret_cast<__nv_bfloat16*>(Qt));

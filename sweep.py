@@ -198,6 +198,43 @@ def run_quant(ctx, cfg, tokens, copies, reps, device="cuda", use_graph=True, set
     return out
 
 
+def run_factor(ctx, cfg, iters, reps, device="cuda"):
+    """On-device factors of one layer's light slices (Section 5.1.1): time per call, tensor-core rate of the block
+    power iteration's products, and the Frobenius residual of U2 ~ A1 B1; the call without a round (gathers, one product, transposes) beside it."""
+    hbm, tf, src, _ = peaks()
+    shape = make_shape(cfg.d, cfg.m, cfg.act, cfg.torch_dtype)
+    ctx.ensure_workspace(ctx.factor_workspace_size(shape, cfg.k, cfg.r))
+    L = make_layer(cfg, 0, device=device)
+    mask = torch.ones(cfg.m, dtype=torch.bool, device=device)
+    mask[L.planted.long()] = False
+    light = torch.nonzero(mask).flatten().to(torch.int32)
+    n_mat = cfg.n_in + 1
+    gen = torch.Generator(device=device)
+    gen.manual_seed(99)
+    start = torch.randn(n_mat, cfg.r, cfg.d, generator=gen, device=device, dtype=torch.float32).to(cfg.torch_dtype)
+    ml = cfg.m - cfg.k
+    U2 = L.W1[:, light.long()].float()
+    out = {"config": cfg.name, "d": cfg.d, "m": cfg.m, "k": cfg.k, "r": cfg.r, "iters": iters, "peaks": src}
+    for label, it in (("start_basis_only", 0), ("iterated", iters)):
+        ts = []
+        for i in range(reps + 1):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fac = ctx.factor_light(shape, L.W1, L.W2, light, cfg.k, cfg.r, it, start, W1u=L.W1u)
+            b.record()
+            b.synchronize()
+            if i >= 1:
+                ts.append(a.elapsed_time(b))
+        ctx.poll()
+        ms = statistics.median(ts)
+        resid = torch.linalg.matrix_norm(U2 - fac["A1"].float() @ fac["B1"].float()).item()
+        flops = n_mat * (it * 4.0 + 2.0) * cfg.r * cfg.d * ml
+        out[label] = {"ms": ms, "product_tflops": flops / (ms * 1e-3) / 1e12}
+        if it > 0:      # (without a round the start basis is not orthonormal and A1 B1 is no projection)
+            out[label]["rel_residual_U2"] = resid / torch.linalg.matrix_norm(U2).item()
+    return out
+
+
 def run_scoring(ctx, cfg, reps, device="cuda", t_cal=None):
     """Scoring pass of one layer, both forms: from the calibration tokens (product + fused column energy)
     and from a stored activation matrix (one streaming read of H).  Events around each call, median."""
@@ -254,6 +291,8 @@ def main():
                          "heavy (k = 768), light rank = 10 %% of full rank (r = 77); --config is ignored")
     ap.add_argument("--scoring", action="store_true", help="time the scoring pass (both forms) instead of the forward")
     ap.add_argument("--quant", action="store_true", help="time the quantised split (Section 5.2) at the given few-token counts")
+    ap.add_argument("--factor", type=int, default=-1, metavar="ITERS",
+                    help="time the on-device factorisation of the light slices with this many rounds of block power iteration")
     ap.add_argument("--t-cal", type=int, default=0, help="with --scoring: calibration tokens (default: the config's)")
     ap.add_argument("--settle", type=float, default=1.0,
                     help="seconds of idle time before each timed case (the clocks recover from the case before)")
@@ -272,6 +311,9 @@ def main():
         points = [cfg5_point(h, r) for h in CFG5_HEAVY_PERCENT for r in CFG5_RANKS]
     if args.scoring:
         print(json.dumps(run_scoring(ctx, base, args.reps, t_cal=args.t_cal or None)), flush=True)
+        return
+    if args.factor >= 0:
+        print(json.dumps(run_factor(ctx, base, args.factor, min(args.reps, 5))), flush=True)
         return
     tokens = args.tokens or list(base.t_fwd)
     lines = []
