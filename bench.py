@@ -168,6 +168,7 @@ class StackWorkload:
         if dense:
             need = max(need, max(ctx.stack_workspace_size(self.blobs_dense, t) for t in (T, 32, 1)))
             need = max(need, ctx.quant_workspace_size(self.shape, cfg.k))
+            need = max(need, ctx.factor_workspace_size(self.shape, cfg.k, cfg.r))
         ctx.ensure_workspace(need)
         # the quantised split of the same layers (Section 5.2: 8-bit heavy, 3-bit light, group 128), for the few-token phase
         self.blobs_quant = []
@@ -426,11 +427,36 @@ def run_ours(args):
                 "roofline_frac": roof * n_layers / ms}
         phases[f"forward_T{Tp}"] = row
         wl.poll()
+    # ---- the step between select and pack on the device (Section 5.1.1): rank-r factors of one layer's light
+    # slices by 6 rounds of block power iteration.  Not part of the timed step, whose packs take seeded factors
+    # (they only need the shapes); timed here with events around the call, weights of layer 0.
+    import torch
+    e0 = wl.layers[0]
+    gen = torch.Generator(device=device)
+    gen.manual_seed(77)
+    start = torch.randn(cfg.n_in + 1, cfg.r, cfg.d, generator=gen, device=device, dtype=torch.float32).to(cfg.torch_dtype)
+    f_ms = []
+    for i in range(4):
+        flush()
+        a_ev, b_ev = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a_ev.record()
+        fac = ctx.factor_light(wl.shape, e0["L"].W1, e0["L"].W2, e0["light"], cfg.k, cfg.r, 6, start, W1u=e0["L"].W1u)
+        b_ev.record()
+        b_ev.synchronize()
+        if i > 0:
+            f_ms.append(a_ev.elapsed_time(b_ev))
+    wl.poll()
+    U2 = e0["L"].W1[:, e0["light"].long()].float()
+    phases["factor_light"] = {"ms_per_layer": statistics.median(f_ms), "rounds": 6, "rank": cfg.r,
+                              "rel_residual_U2": (torch.linalg.matrix_norm(U2 - fac["A1"].float() @ fac["B1"].float())
+                                                  / torch.linalg.matrix_norm(U2)).item()}
+    del U2, fac
     phases["model_bytes_split_per_layer"] = wl.logical_bytes
     phases["model_bytes_dense_per_layer"] = wl.logical_bytes_dense
 
     # ---- roofline of the dominant kernel: the tensor-core GEMM (the scoring products hold 97 % of the step's
     # FLOPs), all its launches of one serial step, each bracketed by CUDA events on its stream
+    es_b = 2
     lane0 = wl.lanes[0][0]
     flush()
     lane0.profile_begin()
@@ -447,6 +473,15 @@ def run_ours(args):
                 "peak_source": f"{peaks['source']} (sustained bf16: launches of 0.1-13 ms back to back inside a 0.5 s step)",
                 "launches_per_step": n_l, "avg_launch_us": round(1e3 * ms_l / max(n_l, 1), 2),
                 "algorithmic_flops_per_launch": flops_l / max(n_l, 1), "traffic": None}
+    if n_layers == 40 and n_l == 200:
+        # DRAM bytes (read + written) of the average launch of a step, from ncu captures of the current kernel:
+        # the scoring product at 8192 calibration tokens moved 815.6 MB (scaled by 8 to the 65 536 tokens of a
+        # launch here: the weights are re-read once per panel of 12 tile rows, so traffic grows with the tokens) and
+        # the four forward GEMMs of a layer at 4096 tokens 413.5 MB together; 40 + 160 launches per step.
+        roofline["traffic"] = round((40 * 8 * 815.6e6 + 40 * 413.5e6) / 200)
+        roofline["traffic_source"] = ("profiles/gemm_tc_kernel__cfg5_scoring.md (x 8 tokens), "
+                                      "profiles/gemm_tc_kernel__cfg5_prefill.md")
+        roofline["algorithmic_bytes_per_launch"] = round((40 * (es_b * (cfg.t_cal * cfg.d + cfg.d * cfg.m)) + 40 * (wl.logical_bytes + 2 * es_b * T * cfg.d)) / 200)
     wl.poll()
 
     # ---- end to end through the host-buffer entry points: calibration tokens, X and Y in pinned host memory
