@@ -40,6 +40,29 @@ __device__ __forceinline__ float gelu_fast(float x, const GeluCoef& c) {
   const float hx = 0.5f * x;
   return fmaf(hx, tanh_approx(u), hx);
 }
+// The same for two values at once with the packed fp32 instructions of sm_100 (fma / mul on register pairs):
+// every component goes through exactly the operations of gelu_fast, so the results are bit-identical, at
+// 10 instead of 16 instructions per pair.
+__device__ __forceinline__ float2 gelu_fast2(float2 x, const GeluCoef& c) {
+  float2 x2 = __fmul2_rn(x, x);
+  x2.x = fminf(x2.x, 36.0f);
+  x2.y = fminf(x2.y, 36.0f);
+  float2 t = __ffma2_rn(make_float2(c.c2, c.c2), x2, make_float2(c.c1, c.c1));
+  t = __ffma2_rn(t, x2, make_float2(c.c0, c.c0));
+  const float2 u = __fmul2_rn(x, t);
+  const float2 hx = __fmul2_rn(make_float2(0.5f, 0.5f), x);
+  const float2 th = make_float2(tanh_approx(u.x), tanh_approx(u.y));
+  return __ffma2_rn(hx, th, hx);
+}
+// 16 values in place.
+__device__ __forceinline__ void gelu_fast16(float* v, const GeluCoef& c) {
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const float2 r = gelu_fast2(make_float2(v[2 * i], v[2 * i + 1]), c);
+    v[2 * i] = r.x;
+    v[2 * i + 1] = r.y;
+  }
+}
 // SiLU with one MUFU: x * sigmoid(x) = 0.5 x (1 + tanh(x / 2)).
 __device__ __forceinline__ float silu_fast(float x) {
   const float hx = 0.5f * x;

@@ -534,9 +534,8 @@ fused_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
         }
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-          const float lo = inside ? gelu_fast(v[hlf][2 * j], gc) : 0.f;
-          const float hi = inside ? gelu_fast(v[hlf][2 * j + 1], gc) : 0.f;
-          w[8 * hlf + j] = pack_bf16x2(lo, hi);
+          const float2 g2 = gelu_fast2(make_float2(v[hlf][2 * j], v[hlf][2 * j + 1]), gc);
+          w[8 * hlf + j] = inside ? pack_bf16x2(g2.x, g2.y) : 0u;
         }
       }
       tmem_st16(t_s, w);
@@ -638,8 +637,7 @@ fused_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
               const float4 t = *reinterpret_cast<const float4*>(smem_b1h + cc + 4 * j);
               v[u][4 * j] += t.x; v[u][4 * j + 1] += t.y; v[u][4 * j + 2] += t.z; v[u][4 * j + 3] += t.w;
             }
-#pragma unroll
-            for (int j = 0; j < 16; ++j) v[u][j] = gelu_fast(v[u][j], gc);
+            gelu_fast16(v[u], gc);
           } else {
 #pragma unroll
             for (int j = 0; j < 16; ++j) v[u][j] = 0.f;

@@ -78,8 +78,7 @@ __device__ __forceinline__ void epilogue_chunk_store(const Params& p, const Gelu
   const Epilogue& e = p.epi;
   if (n0 < e.n_bias) add_bias16(e, n0, v);
   if (!p.dual && n0 < e.n_act) {
-#pragma unroll
-    for (int i = 0; i < 16; ++i) v[i] = gelu_fast(v[i], gc);
+    gelu_fast16(v, gc);
   }
   if (row >= p.M) return;
   if (e.c0_f32) {
