@@ -312,6 +312,36 @@ ffsplit_status ffsplit_factor_light(ffsplit_ctx* ctx, const ffsplit_shape* shape
                                     const int32_t* light_idx, int32_t k, int32_t r, int32_t iters, const void* start,
                                     void* A1, void* B1, void* A2, void* B2, void* A1u, void* B1u, void* stream);
 
+/* ---- The transformer block around the FFN (Section 5.1.2, Table 2: the paper times whole BERT-base models) --
+ * One post-LayerNorm encoder layer, so that the split FFN can be timed in its context:
+ *     A  = MultiHeadAttention(X)          Q, K, V = X Wq, X Wk, X Wv (+ biases), heads of width 64,
+ *                                         softmax(Q K^T / 8) V per head and sequence, heads concatenated, times Wo (+ bo)
+ *     X1 = LayerNorm(X + A)               over the d features, with gain and bias
+ *     Y  = LayerNorm(X1 + FFN(X1))        FFN = the packed layer `ffn_blob`, split or dense (Eq. 2)
+ * Scope: bf16, d = heads * 64 <= 1024, sequences of `seq` <= 128 tokens attended whole (no padding mask),
+ * T = batch * seq tokens stored sequence after sequence.  The projection weights are given K-major (row j of
+ * Wqkv_t holds the d input weights of output feature j; features 0..d-1 are Q, d..2d-1 K, 2d..3d-1 V, head h
+ * owning columns 64 h .. 64 h + 63 of each), the way every right operand of this library is stored. */
+typedef struct {
+  int32_t batch, seq, heads;
+  const void* Wqkv_t;      /* dev bf16 [3 d, d]  */
+  const float* bqkv;       /* dev float [3 d]    */
+  const void* Wo_t;        /* dev bf16 [d, d]    */
+  const float* bo;         /* dev float [d]      */
+  const float* ln1_gamma;  /* dev float [d]      */
+  const float* ln1_beta;
+  const float* ln2_gamma;
+  const float* ln2_beta;
+  float ln_eps;            /* added to the variance (BERT: 1e-12) */
+  const void* ffn_blob;    /* packed FFN of width d, packed or opened on the context */
+} ffsplit_encoder_layer;
+
+/* Workspace ffsplit_encoder_forward() needs for this layer (the FFN's own forward buffers included). */
+ffsplit_status ffsplit_encoder_workspace_size(ffsplit_ctx* ctx, const ffsplit_encoder_layer* layer, size_t* bytes);
+/* X, Y dev bf16 [batch * seq, d], 16-byte aligned; X and Y may not overlap.  Uses the workspace. */
+ffsplit_status ffsplit_encoder_forward(ffsplit_ctx* ctx, const ffsplit_encoder_layer* layer, const void* X, void* Y,
+                                       void* stream);
+
 /* ---- Quantised split (Section 5.2, Table 3: round-to-nearest, group size 128, 8 bits for the heavy-hitter
  * neurons, 3 bits for everything else) ------------------------------------------------------------------
  * The second way the paper compresses the light part: instead of rank-r factors, U2 and V2 are kept whole at

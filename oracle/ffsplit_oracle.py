@@ -31,6 +31,10 @@ Pins (tests that tie each function to something other than itself):
                        round-to-nearest on hand-placed values, independence of groups and of output channels
   quantize_split ..... group axes and bit widths per part, reassembly; quant_split_ffn against Eq. 2 written
                        neuron by neuron on the dequantised weights, error halving per extra bit; byte formula
+  layer_norm, multi_head_attention, encoder_layer ... attention written token by token with explicit loops,
+                       uniform attention when Q = 0 (output = mean of V), constant V passes through, sequences and
+                       heads independent, permutation equivariance inside a sequence; LayerNorm moments, shift
+                       invariance; the block with zero attention and zero FFN weights is LN2(LN1(X)) in closed form
 Parity unpinned: the error of a *truncated* light part against the dense FFN
 (the paper reports task accuracy only, Table 1); it is reported, never gated.
 """
@@ -408,3 +412,50 @@ def quant_weight_bytes(d, m, k, bits_heavy=QUANT_BITS_HEAVY, bits_light=QUANT_BI
         v_bits = n * d * bits
         return (u_bits + v_bits) / 8 + param_bytes * (n_in * n * gd + d * gv)
     return part(k, bits_heavy) + part(ml, bits_light)
+
+
+# ---------------------------------------------------------------------------------------------------
+# The transformer block around the FFN (Section 5.1.2 / Table 2 time whole BERT-base models).  The paper gives no
+# formulas for it; these are the standard post-LayerNorm encoder definitions (Vaswani et al. 2017, Devlin et al.
+# 2019): scaled dot-product attention over whole sequences without a padding mask, heads of equal width.
+# ---------------------------------------------------------------------------------------------------
+def layer_norm(x, gamma, beta, eps):
+    """Per row: (x - mean) / sqrt(var + eps) * gamma + beta, var the biased variance over the features."""
+    x = _f64(x)
+    mu = x.mean(axis=-1, keepdims=True)
+    var = ((x - mu) ** 2).mean(axis=-1, keepdims=True)
+    return (x - mu) / np.sqrt(var + eps) * _f64(gamma) + _f64(beta)
+
+
+def multi_head_attention(X, Wqkv, bqkv, Wo, bo, batch, seq, heads):
+    """X [batch * seq, d], sequence after sequence; Wqkv [d, 3 d] = [Wq | Wk | Wv], head h owning columns
+    h dh .. (h + 1) dh - 1 of each; per sequence and head softmax(Q K^T / sqrt(dh)) V, heads concatenated, times Wo."""
+    X, Wqkv, bqkv, Wo, bo = _f64(X), _f64(Wqkv), _f64(bqkv), _f64(Wo), _f64(bo)
+    T, d = X.shape
+    if T != batch * seq or d % heads:
+        raise ValueError("shape mismatch")
+    dh = d // heads
+    qkv = X @ Wqkv + bqkv
+    out = np.empty((T, d))
+    for b in range(batch):
+        rows = slice(b * seq, (b + 1) * seq)
+        for h in range(heads):
+            q = qkv[rows, h * dh:(h + 1) * dh]
+            k = qkv[rows, d + h * dh:d + (h + 1) * dh]
+            v = qkv[rows, 2 * d + h * dh:2 * d + (h + 1) * dh]
+            s = q @ k.T / math.sqrt(dh)
+            s = s - s.max(axis=1, keepdims=True)
+            p = np.exp(s)
+            p = p / p.sum(axis=1, keepdims=True)
+            out[rows, h * dh:(h + 1) * dh] = p @ v
+    return out @ Wo + bo
+
+
+def encoder_layer(X, attn, ln1, ln2, eps, batch, seq, heads, ffn):
+    """Y = LN2(X1 + ffn(X1)), X1 = LN1(X + MHA(X)); attn = (Wqkv, bqkv, Wo, bo), ln = (gamma, beta), ffn a function
+    of the token matrix (dense_ffn or split_ffn with its weights bound)."""
+    X = _f64(X)
+    A = multi_head_attention(X, *attn, batch, seq, heads)
+    X1 = layer_norm(X + A, ln1[0], ln1[1], eps)
+    return layer_norm(X1 + _f64(ffn(X1)), ln2[0], ln2[1], eps)
+

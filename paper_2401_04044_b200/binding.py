@@ -37,8 +37,14 @@ EXPORTS = [
     "ffsplit_blob_close", "ffsplit_stack_workspace_size", "ffsplit_forward_stack", "ffsplit_forward_stack_host",
     "ffsplit_debug_wait_timeout", "ffsplit_quant_pack_size", "ffsplit_quant_workspace_size", "ffsplit_quant_pack",
     "ffsplit_quant_blob_open", "ffsplit_quant_unpack", "ffsplit_quant_forward",
-    "ffsplit_factor_workspace_size", "ffsplit_factor_light",
+    "ffsplit_factor_workspace_size", "ffsplit_factor_light", "ffsplit_encoder_workspace_size", "ffsplit_encoder_forward",
 ]
+
+
+class EncoderLayer(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("seq", C.c_int32), ("heads", C.c_int32), ("Wqkv_t", C.c_void_p), ("bqkv", C.c_void_p),
+                ("Wo_t", C.c_void_p), ("bo", C.c_void_p), ("ln1_gamma", C.c_void_p), ("ln1_beta", C.c_void_p),
+                ("ln2_gamma", C.c_void_p), ("ln2_beta", C.c_void_p), ("ln_eps", C.c_float), ("ffn_blob", C.c_void_p)]
 
 
 class Shape(C.Structure):
@@ -99,6 +105,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.ffsplit_quant_blob_open.argtypes = [vp, vp, sz, vp]
     lib.ffsplit_quant_unpack.argtypes = [vp, vp, i32, vp, vp, vp, vp]
     lib.ffsplit_quant_forward.argtypes = [vp, vp, vp, i64, vp, vp]
+    lib.ffsplit_encoder_workspace_size.argtypes = [vp, vp, P(sz)]
+    lib.ffsplit_encoder_forward.argtypes = [vp, vp, vp, vp, vp]
     lib.ffsplit_factor_workspace_size.argtypes = [vp, i32, i32, P(sz)]
     lib.ffsplit_factor_light.argtypes = [vp, vp, vp, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     lib.ffsplit_blob_section.argtypes = [vp, vp, i32, P(sz), P(i64), P(i64), P(i64)]
@@ -260,6 +268,22 @@ class Context:
         self._check(self.lib.ffsplit_forward_stack_host(self.h, self._blob_array(blobs), len(blobs), _ptr(X_host),
                                                         X_host.shape[0], _ptr(Y_host), _stream_ptr(stream)),
                     "ffsplit_forward_stack_host")
+
+    # ------------------------------------------------------------------ the transformer block around the FFN
+    def encoder_desc(self, batch: int, seq: int, heads: int, Wqkv_t, bqkv, Wo_t, bo, ln1, ln2, eps: float, ffn_blob):
+        """ffsplit_encoder_layer from device tensors; ln1, ln2 = (gamma, beta).  The tensors must stay alive."""
+        return EncoderLayer(batch, seq, heads, Wqkv_t.data_ptr(), bqkv.data_ptr(), Wo_t.data_ptr(), bo.data_ptr(),
+                            ln1[0].data_ptr(), ln1[1].data_ptr(), ln2[0].data_ptr(), ln2[1].data_ptr(), eps,
+                            ffn_blob.data_ptr())
+
+    def encoder_workspace_size(self, layer: "EncoderLayer") -> int:
+        n = C.c_size_t()
+        self._check(self.lib.ffsplit_encoder_workspace_size(self.h, C.byref(layer), C.byref(n)), "ffsplit_encoder_workspace_size")
+        return n.value
+
+    def encoder_forward(self, layer: "EncoderLayer", X, Y, stream=None):
+        self._check(self.lib.ffsplit_encoder_forward(self.h, C.byref(layer), _ptr(X), _ptr(Y), _stream_ptr(stream)),
+                    "ffsplit_encoder_forward")
 
     # ------------------------------------------------------------------ on-device light factors (Section 5.1.1)
     def factor_workspace_size(self, shape: Shape, k: int, r: int) -> int:

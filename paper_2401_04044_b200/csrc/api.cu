@@ -370,6 +370,24 @@ static ffsplit_status forward_stack_impl(ffsplit_ctx* ctx, const void* const* bl
   return FFSPLIT_OK;
 }
 
+namespace ffsp {
+// One packed FFN layer inside another entry point (the encoder block): same checks and path as ffsplit_forward.
+ffsplit_status run_ffn_forward(ffsplit_ctx* ctx, const void* blob, const void* X, long long T, void* Y, cudaStream_t st) {
+  ffsplit_status s = FFSPLIT_OK;
+  const ffsplit_ctx::BlobEntry* ent = find_blob(ctx, blob, &s);
+  if (!ent) return s;
+  return run_forward(ctx, ent->h, static_cast<const char*>(blob), X, T, Y, st, ent->hash);
+}
+// Bytes of the workspace (behind the control block) that forward of this blob at T tokens uses.
+size_t ffn_forward_workspace_end(ffsplit_ctx* ctx, const void* blob, long long T, ffsplit_status* status, int* d, int* dtype) {
+  const ffsplit_ctx::BlobEntry* ent = find_blob(ctx, blob, status);
+  if (!ent) return 0;
+  if (d) *d = ent->h.d;
+  if (dtype) *dtype = ent->h.dtype;
+  return fwd_layout(dims_of(ent->h), ent->h.d, ent->h.dtype, ent->h.act, T).end;
+}
+}  // namespace ffsp
+
 // =====================================================================================
 extern "C" {
 

@@ -30,7 +30,7 @@ constexpr size_t kCtrlBytes = 65536;
 constexpr long long kMaxTicketTiles = (kCtrlBytes - kStatusBytes) / 4;
 
 enum KernelId : int {
-  KID_SELECT = 1, KID_PACK = 2, KID_GEMM_TC = 3, KID_GEMM_SIMT = 4, KID_SCORE = 5, KID_DECODE = 6, KID_FUSED = 7, KID_PROBE = 8, KID_QUANT = 9, KID_FACTOR = 10
+  KID_SELECT = 1, KID_PACK = 2, KID_GEMM_TC = 3, KID_GEMM_SIMT = 4, KID_SCORE = 5, KID_DECODE = 6, KID_FUSED = 7, KID_PROBE = 8, KID_QUANT = 9, KID_FACTOR = 10, KID_ENCODER = 11
 };
 
 __device__ __forceinline__ void record_status(int* status, int code, int detail, int kid) {
@@ -195,6 +195,7 @@ struct ffsplit_ctx {
   bool attr_tc_set = false;
   bool attr_fused_set = false;
   bool attr_layer_set = false;
+  bool attr_att_set = false;
   int* status() const { return reinterpret_cast<int*>(ws); }
   int* tickets() const { return reinterpret_cast<int*>(ws + ffsp::kStatusBytes); }
   int gemm_two_m = 1;          // tensor-core GEMM: 256-row tiles where they pay (FFSPLIT_GEMM_TWO_M=0: never, 2: wherever allowed)
@@ -312,6 +313,9 @@ bool fused_layer_applies(int dtype, int act, int d, int k, int k_pad, int r_pad,
 size_t fused_layer_scratch_bytes(long long T, int r_pad);
 ffsplit_status launch_fused_layer(ffsplit_ctx* ctx, const BlobHeader& h, const char* blob, const void* X, long long T,
                                   char* scratch, void* Y, unsigned long long guard_hash, cudaStream_t st);
+// forward of one packed FFN layer (split or dense) inside another entry point; defined in api.cu
+ffsplit_status run_ffn_forward(ffsplit_ctx* ctx, const void* blob, const void* X, long long T, void* Y, cudaStream_t st);
+size_t ffn_forward_workspace_end(ffsplit_ctx* ctx, const void* blob, long long T, ffsplit_status* status, int* d, int* dtype);
 ffsplit_status launch_wait_timeout_probe(ffsplit_ctx* ctx, long long limit_cycles, cudaStream_t st);
 ffsplit_status launch_to_f32(ffsplit_ctx* ctx, int dtype, const void* in, int n, float* out, cudaStream_t st);
 

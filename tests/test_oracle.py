@@ -548,3 +548,81 @@ def test_quant_weight_bytes_formula_counts_codes_and_group_parameters():
     # 3.25-3.5 bits per weight overall at 5 % heavy: about a fifth of the bf16 layer
     assert 0.21 < got / (2 * 2 * d * m) < 0.24
     assert orc.quant_weight_bytes(256, 1024, 0) == (2 * 1024 * 256 * 3) / 8 + 8 * (1024 * 2 + 256 * 8)
+
+
+# ---------------------------------------------------------------- the block around the FFN
+def test_layer_norm_moments_and_invariances(rng):
+    x = rng.normal(size=(7, 24)) * 3 + 1.5
+    y = orc.layer_norm(x, np.ones(24), np.zeros(24), 0.0)
+    assert np.allclose(y.mean(axis=1), 0, atol=1e-12) and np.allclose((y ** 2).mean(axis=1), 1, atol=1e-12)
+    assert np.allclose(orc.layer_norm(x + 5.0, np.ones(24), np.zeros(24), 0.0), y, atol=1e-12)      # shift
+    assert np.allclose(orc.layer_norm(2.0 * x, np.ones(24), np.zeros(24), 0.0), y, atol=1e-12)      # scale (eps = 0)
+    g, b = rng.normal(size=24), rng.normal(size=24)
+    assert np.allclose(orc.layer_norm(x, g, b, 0.0), y * g + b, atol=1e-12)
+    # eps enters under the root: a row of variance v is divided by sqrt(v + eps)
+    v = ((x - x.mean(axis=1, keepdims=True)) ** 2).mean(axis=1)
+    assert np.allclose(orc.layer_norm(x, np.ones(24), np.zeros(24), 0.3), y * np.sqrt(v / (v + 0.3))[:, None], atol=1e-12)
+
+
+def test_multi_head_attention_against_token_loops_and_closed_forms(rng):
+    batch, seq, heads, dh = 2, 5, 3, 4
+    d = heads * dh
+    X = rng.normal(size=(batch * seq, d))
+    Wqkv, bqkv = rng.normal(size=(d, 3 * d)) * 0.4, rng.normal(size=3 * d) * 0.1
+    Wo, bo = rng.normal(size=(d, d)) * 0.4, rng.normal(size=d) * 0.1
+    out = orc.multi_head_attention(X, Wqkv, bqkv, Wo, bo, batch, seq, heads)
+    # the definition, one query token and one head at a time
+    ref = np.zeros((batch * seq, d))
+    for b in range(batch):
+        for i in range(seq):
+            t = b * seq + i
+            for h in range(heads):
+                q = X[t] @ Wqkv[:, h * dh:(h + 1) * dh] + bqkv[h * dh:(h + 1) * dh]
+                w = np.zeros(seq)
+                vs = []
+                for j in range(seq):
+                    u = b * seq + j
+                    k = X[u] @ Wqkv[:, d + h * dh:d + (h + 1) * dh] + bqkv[d + h * dh:d + (h + 1) * dh]
+                    vs.append(X[u] @ Wqkv[:, 2 * d + h * dh:2 * d + (h + 1) * dh] + bqkv[2 * d + h * dh:2 * d + (h + 1) * dh])
+                    w[j] = math.exp(float(q @ k) / math.sqrt(dh))
+                ref[t, h * dh:(h + 1) * dh] = sum(wj * vj for wj, vj in zip(w, vs)) / w.sum()
+    assert np.allclose(out, ref @ Wo + bo, atol=1e-12)
+    # Q = 0: uniform attention, every token gets the mean of its sequence's V
+    W0, b0 = Wqkv.copy(), bqkv.copy()
+    W0[:, :d] = 0
+    b0[:d] = 0
+    V = X @ W0[:, 2 * d:] + b0[2 * d:]
+    mean_v = np.repeat(V.reshape(batch, seq, d).mean(axis=1), seq, axis=0)
+    assert np.allclose(orc.multi_head_attention(X, W0, b0, Wo, bo, batch, seq, heads), mean_v @ Wo + bo, atol=1e-12)
+    # V constant (Wv = 0): the softmax weights sum to one, so the output is bv Wo + bo whatever Q and K are
+    W1 = Wqkv.copy()
+    W1[:, 2 * d:] = 0
+    assert np.allclose(orc.multi_head_attention(X, W1, bqkv, Wo, bo, batch, seq, heads),
+                       np.tile(bqkv[2 * d:] @ Wo + bo, (batch * seq, 1)), atol=1e-12)
+    # sequences do not see one another; tokens of a sequence are exchangeable
+    X2 = X.copy()
+    X2[seq:] = rng.normal(size=(seq, d))
+    assert np.allclose(orc.multi_head_attention(X2, Wqkv, bqkv, Wo, bo, batch, seq, heads)[:seq], out[:seq], atol=1e-12)
+    perm = rng.permutation(seq)
+    Xp = X.copy()
+    Xp[:seq] = X[:seq][perm]
+    assert np.allclose(orc.multi_head_attention(Xp, Wqkv, bqkv, Wo, bo, batch, seq, heads)[:seq], out[:seq][perm], atol=1e-12)
+
+
+def test_encoder_layer_composition(rng):
+    batch, seq, heads, d, m = 2, 4, 2, 8, 20
+    X = rng.normal(size=(batch * seq, d))
+    attn = (rng.normal(size=(d, 3 * d)) * 0.3, rng.normal(size=3 * d) * 0.1, rng.normal(size=(d, d)) * 0.3, rng.normal(size=d) * 0.1)
+    ln1, ln2 = (rng.normal(size=d), rng.normal(size=d)), (rng.normal(size=d), rng.normal(size=d))
+    W1, b1, W2, b2 = rng.normal(size=(d, m)), rng.normal(size=m), rng.normal(size=(m, d)), rng.normal(size=d)
+    ffn = lambda Z: orc.dense_ffn(Z, W1, b1, W2, b2, orc.ACT_GELU_ERF)
+    Y = orc.encoder_layer(X, attn, ln1, ln2, 1e-5, batch, seq, heads, ffn)
+    A = orc.multi_head_attention(X, *attn, batch, seq, heads)
+    X1 = orc.layer_norm(X + A, *ln1, 1e-5)
+    assert np.allclose(Y, orc.layer_norm(X1 + ffn(X1), *ln2, 1e-5), atol=1e-12)
+    # no attention, no FFN: two LayerNorms of X in closed form (the second one of an already normalised row)
+    zero_attn = (np.zeros((d, 3 * d)), np.zeros(3 * d), np.zeros((d, d)), np.zeros(d))
+    one = (np.ones(d), np.zeros(d))
+    Y0 = orc.encoder_layer(X, zero_attn, one, one, 0.0, batch, seq, heads, lambda Z: np.zeros_like(Z))
+    xc = X - X.mean(axis=1, keepdims=True)
+    assert np.allclose(Y0, xc / np.sqrt((xc ** 2).mean(axis=1, keepdims=True)), atol=1e-12)
