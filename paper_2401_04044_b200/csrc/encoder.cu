@@ -27,7 +27,7 @@ constexpr int SEQ_TILE = 128;     // query rows = key rows per CTA
 constexpr int DH = 64;            // head width
 constexpr int ATT_THREADS = 160;  // warps 0-3: one query row per thread; warp 4: TMA and MMA issue
 constexpr int TILE_BYTES = SEQ_TILE * DH * 2;   // 16 KB: a Q, K or V tile, or the transposed V
-constexpr int TMEM_COLS = 256;    // S / P at columns 0..127, O at 128..191
+constexpr int TMEM_COLS = 128;    // S at columns 0..127; P (bf16, two per column) compacted in place into 0..63; O at 64..127
 constexpr int ATT_SMEM = 4 * TILE_BYTES + 1024 + 256;
 
 struct AttParams {
@@ -134,9 +134,9 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttParams p) {
         const uint64_t v_desc = ptx::umma_desc_k128(ptx::smem_u32(sVt));
 #pragma unroll
         for (int jj = 0; jj < SEQ_TILE / 16; ++jj) {
-          // 16 keys per step: P sits as packed bf16 in the first half of each 32-column group of S
+          // 16 keys per step: P sits as packed bf16 in columns 0..63, 8 columns per step
           const uint64_t b_desc = v_desc + static_cast<uint64_t>(((jj >> 2) * (TILE_BYTES / 2)) >> 4) + 2 * (jj & 3);
-          umma_bf16_ts(tmem_base + 128, tmem_base + 32 * (jj >> 1) + 8 * (jj & 1), b_desc, idesc, jj != 0 ? 1u : 0u);
+          umma_bf16_ts(tmem_base + 64, tmem_base + 8 * jj, b_desc, idesc, jj != 0 ? 1u : 0u);
         }
         ptx::umma_commit(o_full);
       }
@@ -179,7 +179,8 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttParams p) {
           for (int i = 0; i < 16; ++i)
             if (c + 16 * u + i < p.seq) mx = fmaxf(mx, v[u][i]);
       }
-      // pass 2: exponentials, their sum, P as bf16 back into the columns it came from
+      // pass 2: exponentials, their sum, P as bf16 compacted into columns 0..63 (the 32 columns of group c become
+      // the 16 columns from c / 2: always columns this thread has already consumed)
       float sum = 0.f;
       const float off = mx * p.scale_log2e;
 #pragma unroll
@@ -201,7 +202,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttParams p) {
             w[8 * u + i] = pk;
             sum += __uint_as_float(pk << 16) + __uint_as_float(pk & 0xffff0000u);
           }
-        tmem_st16(t_row + c, w);
+        tmem_st16(t_row + (c >> 1), w);
       }
       tmem_st_wait();
       inv_sum = 1.0f / sum;
@@ -216,8 +217,8 @@ attention_kernel(const __grid_constant__ CUtensorMap tmQKV, const AttParams p) {
 #pragma unroll
       for (int c = 0; c < DH; c += 32) {
         float v[2][16];
-        ptx::tmem_ld16(t_row + 128 + c, v[0]);
-        ptx::tmem_ld16(t_row + 128 + c + 16, v[1]);
+        ptx::tmem_ld16(t_row + 64 + c, v[0]);
+        ptx::tmem_ld16(t_row + 64 + c + 16, v[1]);
         ptx::tmem_ld_wait();
         if (row < p.seq) {
 #pragma unroll
@@ -296,11 +297,14 @@ __global__ void __launch_bounds__(256) add_layernorm_kernel(const __nv_bfloat16*
       uint4 o;
       uint32_t* ow = reinterpret_cast<uint32_t*>(&o);
 #pragma unroll
-      for (int e = 0; e < 8; e += 2) {
-        const float a = (v[i][e] - mean) * rstd * __ldg(gamma + 8 * j + e) + __ldg(beta + 8 * j + e);
-        const float b = (v[i][e + 1] - mean) * rstd * __ldg(gamma + 8 * j + e + 1) + __ldg(beta + 8 * j + e + 1);
-        ow[e / 2] = pack_bf16x2(a, b);
-      }
+      float gm[8], bt[8];
+      *reinterpret_cast<float4*>(gm) = __ldg(reinterpret_cast<const float4*>(gamma + 8 * j));
+      *reinterpret_cast<float4*>(gm + 4) = __ldg(reinterpret_cast<const float4*>(gamma + 8 * j) + 1);
+      *reinterpret_cast<float4*>(bt) = __ldg(reinterpret_cast<const float4*>(beta + 8 * j));
+      *reinterpret_cast<float4*>(bt + 4) = __ldg(reinterpret_cast<const float4*>(beta + 8 * j) + 1);
+#pragma unroll
+      for (int e = 0; e < 8; e += 2)
+        ow[e / 2] = pack_bf16x2(fmaf((v[i][e] - mean) * rstd, gm[e], bt[e]), fmaf((v[i][e + 1] - mean) * rstd, gm[e + 1], bt[e + 1]));
       *reinterpret_cast<uint4*>(y + row * d + 8 * j) = o;
     }
   }
@@ -334,7 +338,9 @@ ffsplit_status check_encoder(ffsplit_ctx* ctx, const ffsplit_encoder_layer* e) {
   if (!e->Wqkv_t || !e->bqkv || !e->Wo_t || !e->bo || !e->ln1_gamma || !e->ln1_beta || !e->ln2_gamma || !e->ln2_beta ||
       !e->ffn_blob)
     return fail(ctx, FFSPLIT_ERR_INVALID_ARG, "NULL tensor in the layer description");
-  if (!aligned16(e->Wqkv_t) || !aligned16(e->Wo_t)) return fail(ctx, FFSPLIT_ERR_ALIGN, "weights must be 16-byte aligned");
+  if (!aligned16(e->Wqkv_t) || !aligned16(e->Wo_t) || !aligned16(e->bqkv) || !aligned16(e->bo) || !aligned16(e->ln1_gamma) ||
+      !aligned16(e->ln1_beta) || !aligned16(e->ln2_gamma) || !aligned16(e->ln2_beta))
+    return fail(ctx, FFSPLIT_ERR_ALIGN, "weights, biases and LayerNorm parameters must be 16-byte aligned");
   return FFSPLIT_OK;
 }
 

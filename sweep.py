@@ -235,6 +235,66 @@ def run_factor(ctx, cfg, iters, reps, device="cuda"):
     return out
 
 
+def run_encoder(ctx, cfg, batch, seq, layers, reps, device="cuda", use_graph=True, settle=0.0):
+    """Whole transformer layers (attention, LayerNorms, FFN) of width cfg.d, `layers` distinct ones back to back as in
+    a BERT-base encoder (Table 2's shape: batch 32, sequence 128): time per layer with the split FFN and with the
+    dense FFN packed from the same weights, and the parts that are not the FFN."""
+    hbm, tf, src, _ = peaks()
+    d, heads = cfg.d, cfg.d // 64
+    shape = make_shape(d, cfg.m, cfg.act, cfg.torch_dtype)
+    T = batch * seq
+    ctx.ensure_workspace(max(ctx.workspace_size(shape, T, 0, cfg.k, cfg.r), ctx.workspace_size(shape, T, 0, cfg.m, 0)))
+    padded, _ = ctx.pack_size(shape, cfg.k, cfg.r)
+    padded_d, _ = ctx.pack_size(shape, cfg.m, 0)
+    gen = torch.Generator(device=device)
+    gen.manual_seed(2024)
+    rn = lambda *sz, std=1.0: torch.randn(*sz, generator=gen, device=device, dtype=torch.float32) * std
+    all_idx = torch.arange(cfg.m, dtype=torch.int32, device=device)
+    descs = {"split": [], "dense": []}
+    keep = []
+    for l in range(layers):
+        L = make_layer(cfg, l, device=device)
+        b = torch.empty(padded, dtype=torch.uint8, device=device)
+        ctx.pack(shape, L.W1, L.b1, L.W2, L.b2, L.planted.to(torch.int32), cfg.k, random_factors(cfg, device, gen), b)
+        bd = torch.empty(padded_d, dtype=torch.uint8, device=device)
+        ctx.pack(shape, L.W1, L.b1, L.W2, L.b2, all_idx, cfg.m, None, bd)
+        ctx.poll()
+        w = (rn(3 * d, d, std=0.05).to(cfg.torch_dtype), rn(3 * d, std=0.02), rn(d, d, std=0.05).to(cfg.torch_dtype), rn(d, std=0.02),
+             (1 + rn(d, std=0.1), rn(d, std=0.05)), (1 + rn(d, std=0.1), rn(d, std=0.05)))
+        keep.append((w, b, bd))
+        descs["split"].append(ctx.encoder_desc(batch, seq, heads, *w, 1e-12, b))
+        descs["dense"].append(ctx.encoder_desc(batch, seq, heads, *w, 1e-12, bd))
+        del L
+    ctx.ensure_workspace(max(ctx.encoder_workspace_size(descs["split"][0]), ctx.encoder_workspace_size(descs["dense"][0])))
+    X = rn(T, d).to(cfg.torch_dtype)
+    bufs = [X, torch.empty_like(X), torch.empty_like(X)]
+    out = {"config": cfg.name, "d": d, "m": cfg.m, "k": cfg.k, "r": cfg.r, "heads": heads, "batch": batch, "seq": seq,
+           "layers": layers, "peaks": src}
+    for name in ("split", "dense"):
+        def stack():
+            src_i = 0
+            for l in range(layers):          # layer l reads layer l - 1's output
+                dst_i = 1 + (l & 1)
+                ctx.encoder_forward(descs[name][l], bufs[src_i], bufs[dst_i])
+                src_i = dst_i
+        ts, mode = time_calls(stack, 1, reps, 3, use_graph, settle)
+        ctx.poll()
+        ms = statistics.median(ts)
+        out[name] = {"ms_per_stack": ms, "us_per_layer": 1e3 * ms / layers, "launch_mode": mode,
+                     "sequences_per_s": batch / (ms * 1e-3)}
+    # the FFN alone, same blobs, for the share of the layer it holds
+    for name, idx in (("split", 1), ("dense", 2)):
+        def ffn_only():
+            for l in range(layers):
+                ctx.forward(keep[l][idx], bufs[1], bufs[2])
+        ts, _ = time_calls(ffn_only, 1, reps, 3, use_graph, settle)
+        ctx.poll()
+        out[name]["ffn_us_per_layer"] = 1e3 * statistics.median(ts) / layers
+    out["split_vs_dense_speedup_whole_layer"] = out["dense"]["ms_per_stack"] / out["split"]["ms_per_stack"]
+    out["split_vs_dense_speedup_ffn_only"] = out["dense"]["ffn_us_per_layer"] / out["split"]["ffn_us_per_layer"]
+    return out
+
+
 def run_scoring(ctx, cfg, reps, device="cuda", t_cal=None):
     """Scoring pass of one layer, both forms: from the calibration tokens (product + fused column energy)
     and from a stored activation matrix (one streaming read of H).  Events around each call, median."""
@@ -291,6 +351,9 @@ def main():
                          "heavy (k = 768), light rank = 10 %% of full rank (r = 77); --config is ignored")
     ap.add_argument("--scoring", action="store_true", help="time the scoring pass (both forms) instead of the forward")
     ap.add_argument("--quant", action="store_true", help="time the quantised split (Section 5.2) at the given few-token counts")
+    ap.add_argument("--encoder", action="store_true",
+                    help="time whole transformer layers (attention + LayerNorms + FFN) of the config's width at batch 32 x "
+                         "sequence 128, the config's layer count back to back, split FFN against dense FFN")
     ap.add_argument("--factor", type=int, default=-1, metavar="ITERS",
                     help="time the on-device factorisation of the light slices with this many rounds of block power iteration")
     ap.add_argument("--t-cal", type=int, default=0, help="with --scoring: calibration tokens (default: the config's)")
@@ -311,6 +374,9 @@ def main():
         points = [cfg5_point(h, r) for h in CFG5_HEAVY_PERCENT for r in CFG5_RANKS]
     if args.scoring:
         print(json.dumps(run_scoring(ctx, base, args.reps, t_cal=args.t_cal or None)), flush=True)
+        return
+    if args.encoder:
+        print(json.dumps(run_encoder(ctx, base, 32, 128, base.layers, args.reps, use_graph=not args.no_graph, settle=args.settle)), flush=True)
         return
     if args.factor >= 0:
         print(json.dumps(run_factor(ctx, base, args.factor, min(args.reps, 5))), flush=True)
