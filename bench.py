@@ -563,6 +563,15 @@ def other_configs(peaks):
                     "dense_us_per_layer": 1e3 * r["dense"]["ms_per_layer"], "dense_roofline_frac": r["dense"]["roofline_frac"],
                     "bound": r["split"]["bound"], "split_vs_dense_speedup": r["split_vs_dense_speedup"],
                     "split_tokens_per_s_per_stack": r["split"]["tokens_per_s_per_stack"], "weight_copies": copies}
+        # whole transformer layers at Table 2's shape (batch 32 x sequence 128, 12 BERT-base layers back to back):
+        # attention + LayerNorms + FFN through ffsplit_encoder_forward, split FFN against dense FFN
+        enc = sweep.run_encoder(ctx, CONFIGS[2], 32, 128, CONFIGS[2].layers, 5, settle=0.3)
+        out["bert_base_whole_layer_b32_s128"] = {
+            "split_us_per_layer": enc["split"]["us_per_layer"], "dense_us_per_layer": enc["dense"]["us_per_layer"],
+            "split_ffn_only_us": enc["split"]["ffn_us_per_layer"], "dense_ffn_only_us": enc["dense"]["ffn_us_per_layer"],
+            "split_vs_dense_speedup_whole_layer": enc["split_vs_dense_speedup_whole_layer"],
+            "split_vs_dense_speedup_ffn_only": enc["split_vs_dense_speedup_ffn_only"],
+            "split_sequences_per_s_per_stack": enc["split"]["sequences_per_s"]}
     finally:
         ctx.close()
     return out
