@@ -224,7 +224,7 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
 
   // ---- small hidden widths: the whole layer in one launch, a cluster of four CTAs per 128-token tile
   if (light && ctx->use_layer_kernel && fused_layer_applies(h.dtype, h.act, d, D.k, D.k_pad, D.r_pad, D.ml_pad, T, ctx->num_sms))
-    return launch_fused_layer(ctx, h, blob, X, T, HL, Y, guard_hash, st);
+    return launch_fused_layer(ctx, h, blob, X, T, HL, AP, D.kp_rp, Y, guard_hash, st);
 
   // ---- stage 1: [A_H | Q] = X [U1 | A1], activation on the heavy columns only
   if (!gated) {

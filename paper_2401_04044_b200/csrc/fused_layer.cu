@@ -60,9 +60,14 @@ struct Params {
   int kbx, kbq, kbh;                // k-blocks of X (d / 64), of Q / P (ceil r_pad / 64), of A_H (ceil k_pad / 64)
   int n_chunks;
   int nq;                           // output columns per CTA, d / CL
+  int hsplit;                       // wide heavy part (k_pad > 256): each rank computes k_pad / CL columns of A_H and
+                                    // stores them to global memory; the last product streams A_H back by TMA
+  int kq;                           // heavy columns this CTA computes: k_pad, or k_pad / CL when hsplit
+  __nv_bfloat16* H; long long ldh;  // hsplit: A_H [T, ldh] in global memory
   int b1_slots, a2_slots, a2_slot_bytes;
   int ring_a_slots, ring_a_bytes;   // phase A ring: X k-block + A1^T k-block; starts right behind the Q region
-  int ring_c_slots, ring_c_bytes;   // ring of phases C and D; starts behind the A_H region
+  int ring_c_slots, ring_c_bytes;   // ring of phases C and D
+  int ring_c_off;                   // its byte offset: behind the A_H region (behind the Q region when hsplit)
   int bias_off;                     // byte offset of the bias ring
   const float* b1h;
   const float* b1l;
@@ -172,7 +177,7 @@ __global__ void __launch_bounds__(NUM_THREADS, 1)
 fused_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constant__ CUtensorMap tmA1,
                    const __grid_constant__ CUtensorMap tmU1, const __grid_constant__ CUtensorMap tmB1,
                    const __grid_constant__ CUtensorMap tmA2, const __grid_constant__ CUtensorMap tmW3,
-                   const Params p) {
+                   const __grid_constant__ CUtensorMap tmH, const Params p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* smem_z = smem;                                   // Q, later P: kbq k-blocks
@@ -180,7 +185,7 @@ fused_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
   uint8_t* ring_a = smem_h1;                                // phase A ring (A_H is not there yet)
   uint8_t* smem_b1 = smem_h1;                               // phase B rings, over the same bytes
   uint8_t* smem_a2 = smem_b1 + p.b1_slots * B1KB_BYTES;
-  uint8_t* ring_c = smem_h1 + p.kbh * KB_BYTES;             // ring of phases C and D
+  uint8_t* ring_c = smem + p.ring_c_off;                    // ring of phases C and D
   float* smem_bias = reinterpret_cast<float*>(smem + p.bias_off);
   float* smem_b1h = smem_bias + BIAS_SLOTS * CHUNK;          // [256] b1 of the heavy neurons
   float* smem_b2 = smem_b1h + 256;                           // [256] b2 of this rank's output columns
@@ -204,7 +209,8 @@ fused_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
   uint64_t* yacc = opfull + 1;                   // [1] phase D MMAs complete
   uint64_t* xbar1 = yacc + 1;                    // [1] all ranks stored their partial (remote arrivals)
   uint64_t* xbar2 = xbar1 + 1;                   // [1] all ranks stored their quarter of P (remote arrivals)
-  uint64_t* drain = xbar2 + 1;                   // [1]
+  uint64_t* xbar3 = xbar2 + 1;                   // [1] hsplit: all ranks stored their columns of A_H (remote arrivals)
+  uint64_t* drain = xbar3 + 1;                   // [1]
   uint32_t* tmem_holder = reinterpret_cast<uint32_t*>(drain + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_holder + 1);
 
@@ -234,6 +240,7 @@ fused_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     ptx::mbar_init(yacc, 1);
     ptx::mbar_init(xbar1, CL * EPI_WARPS);
     ptx::mbar_init(xbar2, CL * EPI_WARPS);
+    ptx::mbar_init(xbar3, CL * EPI_WARPS);
     ptx::mbar_init(drain, 1);
     *abort_flag = 0;
     ptx::mbar_fence_init();
@@ -243,6 +250,7 @@ fused_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     ptx::prefetch_tmap(&tmB1);
     ptx::prefetch_tmap(&tmA2);
     ptx::prefetch_tmap(&tmW3);
+    ptx::prefetch_tmap(&tmH);
   }
   if (warp == 1) {
     ptx::tmem_alloc(tmem_holder, TMEM_COLS);
@@ -294,23 +302,34 @@ fused_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
       // phases C and D share one ring, which lies over the rings of phase B: wait for that phase's MMAs
       if (ok) ok = ptx::mbar_wait(pfull, 0, abort_flag);
       Cursor cc;
-      const uint32_t c_tx = KB_BYTES + p.k_pad * KB * 2;
+      const uint32_t c_tx = KB_BYTES + p.kq * KB * 2;
       for (int kb = 0; kb < p.kbx && ok; ++kb, cc.next(p.ring_c_slots)) {
         const int slot = cc.slot;
         if (!ptx::mbar_wait(&cempty[slot], cc.phase ^ 1u, abort_flag)) { ok = false; break; }
         ptx::mbar_expect_tx(&cfull[slot], c_tx);
         uint8_t* dst = ring_c + slot * p.ring_c_bytes;
         ptx::tma_load_2d(&tmX, dst, &cfull[slot], kb * KB, m_blk * BLOCK_M);
-        ptx::tma_load_2d(&tmU1, dst + KB_BYTES, &cfull[slot], kb * KB, 0);
+        ptx::tma_load_2d(&tmU1, dst + KB_BYTES, &cfull[slot], kb * KB, p.hsplit ? rank * p.kq : 0);
       }
-      // phase D: k-blocks of [B2 ; V1]^T for this rank's output columns, in the operand's order [P | A_H]
+      // phase D: k-blocks of [B2 ; V1]^T for this rank's output columns, in the operand's order [P | A_H]; with a
+      // wide heavy part the matching k-block of A_H comes with them, from the global buffer all ranks wrote
+      const uint32_t w_off = p.hsplit ? KB_BYTES : 0;
       const uint32_t d_tx = p.nq * KB * 2;
+      bool h_ready = false;
       for (int b = 0; b < kb3 && ok; ++b, cc.next(p.ring_c_slots)) {
         const int slot = cc.slot;
         if (!ptx::mbar_wait(&cempty[slot], cc.phase ^ 1u, abort_flag)) { ok = false; break; }
-        ptx::mbar_expect_tx(&cfull[slot], d_tx);
+        const bool hblk = p.hsplit && b >= p.kbq;
+        if (hblk && !h_ready) {
+          if (!mbar_wait_cluster(xbar3, 0, abort_flag)) { ok = false; break; }
+          asm volatile("fence.proxy.async;" ::: "memory");   // the peers' generic-proxy stores before this thread's TMA reads
+          h_ready = true;
+        }
+        ptx::mbar_expect_tx(&cfull[slot], d_tx + (hblk ? KB_BYTES : 0));
         const int x = b < p.kbq ? p.k_pad + b * KB : (b - p.kbq) * KB;
-        ptx::tma_load_2d(&tmW3, ring_c + slot * p.ring_c_bytes, &cfull[slot], x, rank * p.nq);
+        uint8_t* dst = ring_c + slot * p.ring_c_bytes;
+        if (hblk) ptx::tma_load_2d(&tmH, dst, &cfull[slot], x, m_blk * BLOCK_M);
+        ptx::tma_load_2d(&tmW3, dst + w_off, &cfull[slot], x, rank * p.nq);
       }
       if (!ok) {
         // bounded chance for the copies in flight to land before the CTA goes away
@@ -412,7 +431,7 @@ fused_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
       // phase C: A_H accumulator at TMEM_S0 (the S buffers' last reader was issued above)
       Cursor cc;
       if (ok) {
-        const uint32_t idesc = ptx::umma_idesc_bf16(BLOCK_M, p.k_pad);
+        const uint32_t idesc = ptx::umma_idesc_bf16(BLOCK_M, p.kq);
         for (int kb = 0; kb < p.kbx && ok; ++kb, cc.next(p.ring_c_slots)) {
           const int slot = cc.slot;
           if (!ptx::mbar_wait(&cfull[slot], cc.phase, abort_flag)) { ok = false; break; }
@@ -435,8 +454,10 @@ fused_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
           const int slot = cc.slot;
           if (!ptx::mbar_wait(&cfull[slot], cc.phase, abort_flag)) { ok = false; break; }
           ptx::tc_fence_after();
-          const uint64_t a_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_z + b * KB_BYTES));
-          const uint64_t b_desc = ptx::umma_desc_k128(ptx::smem_u32(ring_c + slot * p.ring_c_bytes));
+          uint8_t* slot_p = ring_c + slot * p.ring_c_bytes;
+          const bool hblk = p.hsplit && b >= p.kbq;     // A_H block streamed into the slot, in front of the weights
+          const uint64_t a_desc = ptx::umma_desc_k128(ptx::smem_u32(hblk ? slot_p : smem_z + b * KB_BYTES));
+          const uint64_t b_desc = ptx::umma_desc_k128(ptx::smem_u32(slot_p + (p.hsplit ? KB_BYTES : 0)));
 #pragma unroll
           for (int k = 0; k < KB / 16; ++k)   // the operand's columns past r_pad and past k_pad are zero
             ptx::umma_bf16(tmem_base + TMEM_S0, a_desc + 2 * k, b_desc + 2 * k, idesc, (b | k) != 0 ? 1u : 0u);
@@ -479,7 +500,7 @@ fused_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
       *reinterpret_cast<uint4*>(blk + swz_piece(row_in_tile, j + 1)) = b;
     };
     // b1[heavy] and this rank's slice of b2 into shared memory, long before they are needed
-    if (te < p.k_pad) smem_b1h[te] = __ldg(p.b1h + te);
+    if (te < p.kq) smem_b1h[te] = __ldg(p.b1h + (p.hsplit ? rank * p.kq : 0) + te);
     if (te < p.nq) smem_b2[te] = __ldg(p.b2 + rank * p.nq + te);
     asm volatile("bar.sync 1, %0;" ::"n"(EPI_THREADS) : "memory");
     bool ok = ptx::mbar_wait(qacc, 0, abort_flag);
@@ -621,17 +642,18 @@ fused_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
     if (ok) ok = ptx::mbar_wait(hacc, 0, abort_flag);
     if (ok) {
       ptx::tc_fence_after();
-      for (int c = cg * 16; c < p.kbh * KB; c += 128) {
+      const int hcols = p.hsplit ? p.kq : p.kbh * KB;      // columns to walk: this rank's slice, or the padded operand
+      for (int c = cg * 16; c < hcols; c += 128) {
         float v[2][16];
 #pragma unroll
         for (int u = 0; u < 2; ++u)
-          if (c + 64 * u < p.k_pad) ptx::tmem_ld16(t_lane + TMEM_S0 + c + 64 * u, v[u]);
+          if (c + 64 * u < p.kq) ptx::tmem_ld16(t_lane + TMEM_S0 + c + 64 * u, v[u]);
         ptx::tmem_ld_wait();
 #pragma unroll
         for (int u = 0; u < 2; ++u) {
           const int cc = c + 64 * u;
-          if (cc >= p.kbh * KB) continue;
-          if (cc < p.k_pad) {
+          if (cc >= hcols) continue;
+          if (cc < p.kq) {
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
               const float4 t = *reinterpret_cast<const float4*>(smem_b1h + cc + 4 * j);
@@ -642,8 +664,25 @@ fused_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
 #pragma unroll
             for (int j = 0; j < 16; ++j) v[u][j] = 0.f;
           }
-          put16(smem_h1, cc, v[u]);
+          if (!p.hsplit) {
+            put16(smem_h1, cc, v[u]);
+          } else if (row0 + row_in_tile < p.T) {
+            uint4 a, bb;
+            a.x = pack_bf16x2(v[u][0], v[u][1]);    a.y = pack_bf16x2(v[u][2], v[u][3]);
+            a.z = pack_bf16x2(v[u][4], v[u][5]);    a.w = pack_bf16x2(v[u][6], v[u][7]);
+            bb.x = pack_bf16x2(v[u][8], v[u][9]);   bb.y = pack_bf16x2(v[u][10], v[u][11]);
+            bb.z = pack_bf16x2(v[u][12], v[u][13]); bb.w = pack_bf16x2(v[u][14], v[u][15]);
+            uint4* dst = reinterpret_cast<uint4*>(p.H + (row0 + row_in_tile) * p.ldh + rank * p.kq + cc);
+            dst[0] = a;
+            dst[1] = bb;
+          }
         }
+      }
+      if (p.hsplit) {
+        __threadfence();
+        __syncwarp();
+        if (lane == 0)
+          for (int c = 0; c < CL; ++c) mbar_arrive_remote(xbar3, c);
       }
       ok = mbar_wait_cluster(xbar2, 0, abort_flag);
     }
@@ -727,14 +766,19 @@ fused_layer_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_constan
 
 namespace {
 struct LayerPlan {
-  int b1_slots, a2_slots, ring_a_slots, ring_a_bytes, ring_c_slots, ring_c_bytes, bias_off, smem_bytes;
+  int b1_slots, a2_slots, ring_a_slots, ring_a_bytes, ring_c_slots, ring_c_bytes, ring_c_off, bias_off, smem_bytes;
   bool ok;
 };
+// hsplit: the heavy part is wider than one accumulator; each rank computes k_pad / CL of its columns and the
+// operand of the last product is streamed from global memory instead of being held in shared memory.
+bool layer_hsplit(int k_pad) { return k_pad > 256; }
 LayerPlan plan_layer(int d, int k_pad, int r_pad) {
   LayerPlan L{};
+  const bool hsplit = layer_hsplit(k_pad);
+  const int kq = hsplit ? k_pad / ly::CL : k_pad;
   const int kbq = (r_pad + ly::KB - 1) / ly::KB, kbh = (k_pad + ly::KB - 1) / ly::KB;
   const int nq = d / ly::CL;
-  const int z_bytes = kbq * ly::KB_BYTES, h_bytes = kbh * ly::KB_BYTES;
+  const int z_bytes = kbq * ly::KB_BYTES, h_bytes = hsplit ? 0 : kbh * ly::KB_BYTES;
   const int tail = ly::BIAS_BYTES + ly::BAR_BYTES;
   const int avail = ly::MAX_SMEM - 1024 - z_bytes - tail;   // behind the Q region, before the bias ring
   // phase A ring
@@ -742,9 +786,11 @@ LayerPlan plan_layer(int d, int k_pad, int r_pad) {
   L.ring_a_slots = avail / L.ring_a_bytes;
   if (L.ring_a_slots > ly::MAX_RING) L.ring_a_slots = ly::MAX_RING;
   // ring of phases C and D, behind the A_H region
-  int cb = ly::KB_BYTES + k_pad * ly::KB * 2;
-  if (nq * ly::KB * 2 > cb) cb = nq * ly::KB * 2;
+  int cb = ly::KB_BYTES + kq * ly::KB * 2;
+  const int db = (hsplit ? ly::KB_BYTES : 0) + nq * ly::KB * 2;
+  if (db > cb) cb = db;
   L.ring_c_bytes = (cb + 1023) / 1024 * 1024;
+  L.ring_c_off = z_bytes + h_bytes;
   L.ring_c_slots = (avail - h_bytes) / L.ring_c_bytes;
   if (L.ring_c_slots > ly::MAX_RING) L.ring_c_slots = ly::MAX_RING;
   // rings of phase B, balanced in units of chunks
@@ -771,7 +817,8 @@ LayerPlan plan_layer(int d, int k_pad, int r_pad) {
 // 125 us against 82 us at 16 384 tokens, where the clusters take four turns).
 bool fused_layer_applies(int dtype, int act, int d, int k, int k_pad, int r_pad, int ml_pad, long long T, int num_sms) {
   if (dtype != FFSPLIT_BF16 || act == FFSPLIT_SWIGLU) return false;
-  if (k < 1 || k_pad > 256 || r_pad < 16 || r_pad > 256 || ml_pad < 1) return false;
+  if (k < 1 || r_pad < 16 || r_pad > 256 || ml_pad < 1) return false;
+  if (k_pad > 256 && (k_pad % (16 * ly::CL) != 0 || k_pad > 256 * ly::CL)) return false;   // wide heavy part: equal column slices
   if (d % 64 != 0 || d / ly::CL > 256 || d / ly::CL < 16) return false;
   if (T <= 64 || (T + ly::BLOCK_M - 1) / ly::BLOCK_M * ly::CL > num_sms) return false;
   return plan_layer(d, k_pad, r_pad).ok;
@@ -784,7 +831,8 @@ size_t fused_layer_scratch_bytes(long long T, int r_pad) {
 }
 
 ffsplit_status launch_fused_layer(ffsplit_ctx* ctx, const BlobHeader& h, const char* blob, const void* X, long long T,
-                                  char* scratch, void* Y, unsigned long long guard_hash, cudaStream_t st) {
+                                  char* scratch, void* H, long long ldh, void* Y, unsigned long long guard_hash,
+                                  cudaStream_t st) {
   const int d = h.d, k_pad = h.k_pad, r_pad = h.r_pad, ml_pad = h.ml_pad, kp_rp = h.k_pad + h.r_pad;
   const LayerPlan L = plan_layer(d, k_pad, r_pad);
   if (!L.ok) return fail(ctx, FFSPLIT_ERR_SHAPE, "one-launch layer: shared memory too small");
@@ -798,7 +846,10 @@ ffsplit_status launch_fused_layer(ffsplit_ctx* ctx, const BlobHeader& h, const c
   p.nq = d / ly::CL;
   p.b1_slots = L.b1_slots; p.a2_slots = L.a2_slots; p.a2_slot_bytes = r_pad * ly::KB * 2;
   p.ring_a_slots = L.ring_a_slots; p.ring_a_bytes = L.ring_a_bytes;
-  p.ring_c_slots = L.ring_c_slots; p.ring_c_bytes = L.ring_c_bytes;
+  p.ring_c_slots = L.ring_c_slots; p.ring_c_bytes = L.ring_c_bytes; p.ring_c_off = L.ring_c_off;
+  p.hsplit = layer_hsplit(k_pad) ? 1 : 0;
+  p.kq = p.hsplit ? k_pad / ly::CL : k_pad;
+  p.H = static_cast<__nv_bfloat16*>(H); p.ldh = ldh;
   p.bias_off = L.bias_off;
   p.b1h = reinterpret_cast<const float*>(blob + h.off[SEC_B1H]);
   p.b1l = reinterpret_cast<const float*>(blob + h.off[SEC_B1L]);
@@ -812,14 +863,16 @@ ffsplit_status launch_fused_layer(ffsplit_ctx* ctx, const BlobHeader& h, const c
   p.guard = guard_hash ? reinterpret_cast<const unsigned long long*>(blob) : nullptr;
   p.guard_hash = guard_hash;
   const char* u1t = blob + h.off[SEC_U1T];
-  CUtensorMap tX, tA1, tU1, tB1, tA2, tW3;
+  CUtensorMap tX, tA1, tU1, tB1, tA2, tW3, tH;
   ffsplit_status s;
   if ((s = get_tmap_bf16(ctx, X, T, d, d, ly::BLOCK_M, &tX)) != FFSPLIT_OK) return s;
   if ((s = get_tmap_bf16(ctx, u1t + static_cast<size_t>(k_pad) * d * 2, r_pad, d, d, r_pad, &tA1)) != FFSPLIT_OK) return s;
-  if ((s = get_tmap_bf16(ctx, u1t, k_pad, d, d, k_pad, &tU1)) != FFSPLIT_OK) return s;
+  if ((s = get_tmap_bf16(ctx, u1t, k_pad, d, d, p.kq, &tU1)) != FFSPLIT_OK) return s;
   if ((s = get_tmap_bf16(ctx, blob + h.off[SEC_B1T], ml_pad, r_pad, r_pad, ly::CHUNK, &tB1)) != FFSPLIT_OK) return s;
   if ((s = get_tmap_bf16(ctx, blob + h.off[SEC_A2T], r_pad, ml_pad, ml_pad, r_pad, &tA2)) != FFSPLIT_OK) return s;
   if ((s = get_tmap_bf16(ctx, blob + h.off[SEC_V1B2T], d, kp_rp, kp_rp, p.nq, &tW3)) != FFSPLIT_OK) return s;
+  // (without hsplit the kernel never uses this map; it is given a valid one all the same)
+  if ((s = get_tmap_bf16(ctx, H, T, k_pad, ldh, ly::BLOCK_M, &tH)) != FFSPLIT_OK) return s;
   if (!ctx->attr_layer_set) {
     cudaError_t e = cudaFuncSetAttribute(ly::fused_layer_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          ly::MAX_SMEM);
@@ -842,7 +895,7 @@ ffsplit_status launch_fused_layer(ffsplit_ctx* ctx, const BlobHeader& h, const c
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  const cudaError_t le = cudaLaunchKernelEx(&cfg, ly::fused_layer_kernel, tX, tA1, tU1, tB1, tA2, tW3, p);
+  const cudaError_t le = cudaLaunchKernelEx(&cfg, ly::fused_layer_kernel, tX, tA1, tU1, tB1, tA2, tW3, tH, p);
   prof_close(ctx, ph, st);
   ctx->launches++;
   return check_cuda(ctx, le, "fused_layer_kernel launch");

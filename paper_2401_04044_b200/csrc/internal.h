@@ -312,7 +312,8 @@ ffsplit_status launch_fused_light(ffsplit_ctx* ctx, const void* Q, long long ldq
 bool fused_layer_applies(int dtype, int act, int d, int k, int k_pad, int r_pad, int ml_pad, long long T, int num_sms);
 size_t fused_layer_scratch_bytes(long long T, int r_pad);
 ffsplit_status launch_fused_layer(ffsplit_ctx* ctx, const BlobHeader& h, const char* blob, const void* X, long long T,
-                                  char* scratch, void* Y, unsigned long long guard_hash, cudaStream_t st);
+                                  char* scratch, void* H, long long ldh, void* Y, unsigned long long guard_hash,
+                                  cudaStream_t st);
 // forward of one packed FFN layer (split or dense) inside another entry point; defined in api.cu
 ffsplit_status run_ffn_forward(ffsplit_ctx* ctx, const void* blob, const void* X, long long T, void* Y, cudaStream_t st);
 size_t ffn_forward_workspace_end(ffsplit_ctx* ctx, const void* blob, long long T, ffsplit_status* status, int* d, int* dtype);

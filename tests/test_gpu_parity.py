@@ -309,6 +309,10 @@ LAYER_CASES = [
     (128, 2000, 30, 80, 65),       # r_pad = 80: partial k-block of Q and P; smallest token count of the path
     (256, 1024, 250, 16, 700),     # k_pad = 256 (widest heavy part), smallest rank
     (512, 700, 1, 64, 129),        # one heavy neuron
+    (768, 3072, 768, 77, 4096),    # the paper's own point at BERT-base shape (25 % heavy, rank 77): heavy part wider than
+                                   # one accumulator, computed in column slices by the four ranks and streamed back
+    (256, 1024, 500, 32, 300),     # k_pad = 512: slices of 128
+    (512, 2048, 320, 64, 200),     # k_pad = 320: slices of 80
 ]
 
 
