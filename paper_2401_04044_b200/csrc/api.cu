@@ -130,7 +130,7 @@ bool header_valid(const BlobHeader& h, size_t blob_bytes) {
   return blob_bytes == 0 || blob_bytes >= h.total_bytes;
 }
 
-struct FwdLayout { size_t ap, q, hl, xs, ys, dscratch, end; };
+struct FwdLayout { size_t ap, q, hl, skp, skp_bytes, xs, ys, dscratch, end; };
 // The T x mL buffer of the unfused light chain doubles as the fp32 partial buffer of
 // the fused kernel (only one of the two paths runs in a call).
 FwdLayout fwd_layout(const SplitDims& D, int d, int dtype, int act, long long T) {
@@ -149,6 +149,9 @@ FwdLayout fwd_layout(const SplitDims& D, int d, int dtype, int act, long long T)
     if (fs > hl) hl = fs;
   }
   L.hl = off; off = align_up(off + hl);
+  // fp32 partials of the light chain's second product when it is cut along K (up to four of [T, r_pad])
+  L.skp_bytes = (dtype == FFSPLIT_BF16 && D.r_pad > 0 && T > 64) ? static_cast<size_t>(4) * T * D.r_pad * 4 : 0;
+  L.skp = off; off = align_up(off + L.skp_bytes);
   L.xs = off; off = align_up(off + (size_t)T * d * es);
   L.ys = off; off = align_up(off + (size_t)T * d * es);
   L.dscratch = off; off = align_up(off + decode_scratch_bytes(dtype, T));   // few-token path: split-K partials
@@ -291,6 +294,7 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
     g.algo_flops = 2.0 * T * D.r * D.ml;
     g.epi.C0 = AP + (size_t)D.k_pad * es; g.epi.ld0 = D.kp_rp;
     g.epi.n_split = g.N; g.epi.act = h.act;
+    g.splitk = L.skp_bytes ? base + L.skp : nullptr; g.splitk_bytes = L.skp_bytes;
     if ((s = launch_gemm(ctx, h.dtype, g, st)) != FFSPLIT_OK) return s;
   }
   // ---- stage 3: Y = [A_H | P] [V1 ; B2] + b2 (heavy and light parts in one accumulator)
@@ -452,6 +456,7 @@ ffsplit_status ffsplit_create(ffsplit_ctx** out, int device) {
   c->num_sms = sms;
   if (const char* env = std::getenv("FFSPLIT_GEMM_TWO_M")) c->gemm_two_m = env[0] == '0' ? 0 : env[0] == '2' ? 2 : 1;
   if (const char* env = std::getenv("FFSPLIT_GEMM_PANEL")) c->gemm_panel = std::atoi(env);
+  if (const char* env = std::getenv("FFSPLIT_GEMM_SPLIT_K")) c->gemm_split_k = env[0] == '0' ? 0 : 1;
   if (const char* env = std::getenv("FFSPLIT_LAYER_KERNEL")) c->use_layer_kernel = env[0] == '0' ? 0 : 1;
   if (const char* env = std::getenv("FFSPLIT_DECODE_LAYER")) c->decode_one_launch = env[0] == '0' ? 0 : 1;
   if (const char* env = std::getenv("FFSPLIT_DECODE_STREAM")) c->decode_stream = env[0] == '0' ? 0 : env[0] == '2' ? 2 : 1;

@@ -52,6 +52,10 @@ struct Params {
                      // tiles in flight at any time form a block about as high as wide: their operands then fit L2
                      // (row-major order re-read the whole weight matrix from DRAM once per wave: 3.96 GB for 0.29 GB
                      // of operands on the OPT-13B-shaped scoring product)
+  int split_k;       // > 1: the K loop is cut into this many ranges, each a tile of its own (tiles_m x tiles_n x split_k
+                     // work units) writing an fp32 partial [split][M][N]; a small kernel adds them (thin outputs with a
+                     // long contraction: fewer tiles than SMs otherwise)
+  int kb_split;      // k-blocks per range
   Epilogue epi;
   int* status;
 };
@@ -74,7 +78,7 @@ __device__ __forceinline__ void add_bias16(const Epilogue& e, int n0, float* v) 
 }
 
 __device__ __forceinline__ void epilogue_chunk_store(const Params& p, const GeluCoef& gc, long long row, int n0,
-                                                     float* v) {
+                                                     float* v, int ks) {
   const Epilogue& e = p.epi;
   if (n0 < e.n_bias) add_bias16(e, n0, v);
   if (!p.dual && n0 < e.n_act) {
@@ -83,7 +87,7 @@ __device__ __forceinline__ void epilogue_chunk_store(const Params& p, const Gelu
   if (row >= p.M) return;
   if (e.c0_f32) {
     // fp32 output (n_split >= N): 64 bytes per lane, in 16-byte pieces where the address allows
-    float* base = reinterpret_cast<float*>(e.C0) + row * e.ld0 + n0;
+    float* base = reinterpret_cast<float*>(e.C0) + (row + static_cast<long long>(ks) * p.M) * e.ld0 + n0;   // ks-th partial
     if (n0 + 16 <= p.N && (reinterpret_cast<uintptr_t>(base) & 15u) == 0) {
 #pragma unroll
       for (int i = 0; i < 4; ++i)
@@ -226,8 +230,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   const int nkb = (p.K + BLOCK_K - 1) / BLOCK_K;
-  const int total_kb = (p.dual && !p.shared_a) ? 2 * nkb : nkb;
-  const int num_tiles = p.tiles_m * p.tiles_n;
+  const int tiles_mn = p.tiles_m * p.tiles_n;
+  const int num_tiles = tiles_mn * p.split_k;
+  // k-blocks of a work unit of K range ks (the last range may be shorter)
+  const int kb_last = nkb - (p.split_k - 1) * p.kb_split;
+  const int kb_mul = (p.dual && !p.shared_a) ? 2 : 1;
+#define UNIT_KB(ks) (kb_mul * ((ks) == p.split_k - 1 ? kb_last : p.kb_split))
   const uint32_t stage_tx = A_STAGE + B_STAGE_BYTES;
 
   if (warp == 0) {
@@ -237,14 +245,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       bool ok = true;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
         int m_blk, n_blk;
-        tile_coords(p, tile, &m_blk, &n_blk);
+        const int ks = tile / tiles_mn;
+        tile_coords(p, tile - ks * tiles_mn, &m_blk, &n_blk);
+        const int total_kb = UNIT_KB(ks), nkb_u = p.split_k > 1 ? total_kb : nkb;
         for (int kb = 0; kb < total_kb; ++kb, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1;
           if (!ptx::mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; break; }
           ptx::mbar_expect_tx(&full[s], stage_tx);
-          const bool second = p.dual && kb >= nkb;
-          const int kk = (second ? kb - nkb : kb) * BLOCK_K;
+          const bool second = p.dual && kb >= nkb_u;
+          const int kk = (ks * p.kb_split + (second ? kb - nkb_u : kb)) * BLOCK_K;
           for (int mt = 0; mt < MT; ++mt)
             ptx::tma_load_2d(second ? &tmA1 : &tmA0, smem_a + s * A_STAGE + mt * A_STAGE_BYTES, &full[s], kk,
                              (m_blk * MT + mt) * BLOCK_M);
@@ -276,12 +286,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         if (!ptx::mbar_wait(&tempty[acc], aph ^ 1, abort_flag)) { ok = false; break; }
         if (p.two_m && !ptx::mbar_wait(&tempty[1], aph ^ 1, abort_flag)) { ok = false; break; }
         ptx::tc_fence_after();
+        const int total_kb = UNIT_KB(tile / tiles_mn);
         for (int kb = 0; kb < total_kb; ++kb, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1;
           if (!ptx::mbar_wait(&full[s], ph, abort_flag)) { ok = false; break; }
           ptx::tc_fence_after();
-          const bool second = p.dual && kb >= nkb;
+          const bool second = p.dual && kb >= nkb;   // (a gated product is never cut along K)
           const int kbl = second ? kb - nkb : kb;
           const uint32_t d_tmem = tmem_base + acc * ACC_STRIDE + (second ? p.gate_off : 0);
           const uint64_t a_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_a + s * A_STAGE));
@@ -326,7 +337,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     for (int tile = blockIdx.x; tile < num_tiles && live; tile += gridDim.x)
     for (int mt = 0; mt < MT; ++mt, ++vt) {
       int m_tile, n_blk;
-      tile_coords(p, tile, &m_tile, &n_blk);
+      const int ks = tile / tiles_mn;
+      tile_coords(p, tile - ks * tiles_mn, &m_tile, &n_blk);
       const int m_blk = m_tile * MT + mt;
       const uint32_t acc = vt & 1, aph = (vt >> 1) & 1;
       if (warp == 2 && p.epi.n_bias > 0) {
@@ -341,7 +353,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       // one 16-column chunk: v holds the accumulators of this lane's row
       auto finish_chunk = [&](float* v, int n0) {
         if (p.epi.col_partial == nullptr) {
-          epilogue_chunk_store(p, gc, row, n0, v);
+          epilogue_chunk_store(p, gc, row, n0, v, ks);
         } else {
           const Epilogue& e = p.epi;
           if (n0 < e.n_bias) add_bias16(e, n0, v);
@@ -423,6 +435,28 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     ptx::tmem_dealloc(tmem_base, TMEM_COLS);
   }
 }
+
+// C [M, N] (bf16, pitch ldc) = sum over the `split` fp32 partials [split][M][N], in order.  N % 4 == 0.
+__global__ void __launch_bounds__(256) splitk_reduce_kernel(const float* partial, int split, long long M, int N,
+                                                            __nv_bfloat16* C, long long ldc) {
+  pdl_wait();
+  const long long q = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x;     // float4 index
+  const int n4 = N >> 2;
+  if (q >= M * n4) return;
+  const long long row = q / n4;
+  const int c = static_cast<int>(q - row * n4) * 4;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (int s = 0; s < split; ++s) {
+    const float4 v = __ldcg(reinterpret_cast<const float4*>(partial + (static_cast<long long>(s) * M + row) * N + c));
+    acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+  }
+  uint2 o;
+  o.x = pack_bf16x2(acc.x, acc.y);
+  o.y = pack_bf16x2(acc.z, acc.w);
+  *reinterpret_cast<uint2*>(C + row * ldc + c) = o;
+}
+
+#undef UNIT_KB
 
 }  // namespace tc
 
@@ -518,6 +552,34 @@ ffsplit_status launch_gemm_tc(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_t 
     }
   }
   p.tiles_n = (g.N + p.block_n - 1) / p.block_n;
+  // Thin output, long contraction: with 256-wide tiles of 128 rows there are fewer than half as many tiles as SMs;
+  // cut K so that the work units cover the SMs.  (Measured on the OPT-13B-shaped light chain, 4096 x 512 x 19456:
+  // 128 tiles of 128 x 128 ran the tensor pipe at 47 %.)
+  p.split_k = 1;
+  p.kb_split = (g.K + tc::BLOCK_K - 1) / tc::BLOCK_K;
+  const bool plain = !dual && !g.epi.col_partial && !g.epi.c0_f32 && g.epi.n_bias == 0 && g.epi.n_act == 0 &&
+                     g.epi.n_split >= g.N && g.N % 4 == 0 && (reinterpret_cast<uintptr_t>(g.epi.C0) & 7u) == 0 && g.epi.ld0 % 4 == 0;
+  if (ctx->gemm_split_k && g.splitk && plain && g.K >= 4096) {
+    const int bn = g.N >= 256 ? 256 : round_up(g.N, 16);
+    const int nkb = p.kb_split;
+    // 128-row tiles (256-row tiles with K cut in four were measured too: 284 us per OPT-13B-shaped split layer against
+    // 272 us with 128-row tiles and K cut in two, 283 us without the cut: twice the partials, an exposed epilogue)
+    for (int mt = 1; mt >= 1 && p.split_k == 1; --mt) {
+      const long long tm = (g.M + mt * tc::BLOCK_M - 1) / (mt * tc::BLOCK_M);
+      const long long tiles1 = tm * ((g.N + bn - 1) / bn);
+      int split = static_cast<int>(ctx->num_sms / tiles1);
+      if (split > 4) split = 4;
+      while (split > 1 && (nkb / split < 16 * mt || static_cast<size_t>(split) * g.M * g.N * 4 > g.splitk_bytes)) --split;
+      if (split > 1) {
+        p.two_m = mt == 2 ? 1 : 0;
+        p.tiles_m = static_cast<int>(tm);
+        p.block_n = bn;
+        p.tiles_n = (g.N + bn - 1) / bn;
+        p.split_k = split;
+        p.kb_split = (nkb + split - 1) / split;
+      }
+    }
+  }
   {
     // panel height: the tiles of one wave (one per SM) form a block of panel_m x (SMs / panel_m) tiles; the
     // operand bytes that block touches are smallest when its two sides carry about the same bytes
@@ -533,6 +595,11 @@ ffsplit_status launch_gemm_tc(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_t 
   }
   p.gate_off = p.shared_a ? p.block_n : tc::GATE_OFFSET;
   p.epi = g.epi;
+  if (p.split_k > 1) {
+    p.epi.C0 = g.splitk;      // fp32 partials [split][M][N]
+    p.epi.ld0 = g.N;
+    p.epi.c0_f32 = 1;
+  }
   p.status = ctx->status();
   CUtensorMap tA0, tB0, tA1, tB1;
   ffsplit_status s;
@@ -555,7 +622,7 @@ ffsplit_status launch_gemm_tc(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_t 
   p.stages = (tc::MAX_SMEM - tc::BAR_BYTES - 1024) / stage_bytes;
   if (p.stages > tc::MAX_STAGES) p.stages = tc::MAX_STAGES;
   const int smem_bytes = p.stages * stage_bytes + tc::BAR_BYTES + 1024;
-  const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n;
+  const long long tiles = static_cast<long long>(p.tiles_m) * p.tiles_n * p.split_k;
   const int grid = static_cast<int>(tiles < ctx->num_sms ? tiles : ctx->num_sms);
   const int ph = prof_open(ctx, PROF_GEMM_TC, g.algo_flops, st);
   cudaLaunchConfig_t cfg = {};
@@ -569,9 +636,18 @@ ffsplit_status launch_gemm_tc(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_t 
   cfg.attrs = attr;
   cfg.numAttrs = 1;
   const cudaError_t le = cudaLaunchKernelEx(&cfg, tc::gemm_tc_kernel, tA0, tB0, tA1, tB1, p);
+  ctx->launches++;
+  if (le != cudaSuccess || p.split_k == 1) {
+    prof_close(ctx, ph, st);
+    return check_cuda(ctx, le, "gemm_tc_kernel launch");
+  }
+  const long long quads = g.M * (g.N / 4);
+  const cudaError_t re = launch_pdl(tc::splitk_reduce_kernel, dim3(static_cast<unsigned>((quads + 255) / 256)), dim3(256), 0, st,
+                                    static_cast<const float*>(g.splitk), p.split_k, g.M, g.N,
+                                    static_cast<__nv_bfloat16*>(g.epi.C0), g.epi.ld0);
   prof_close(ctx, ph, st);
   ctx->launches++;
-  return check_cuda(ctx, le, "gemm_tc_kernel launch");
+  return check_cuda(ctx, re, "splitk_reduce_kernel launch");
 }
 
 }  // namespace ffsp

@@ -106,6 +106,8 @@ struct GemmArgs {
   int N;
   int K;
   double algo_flops;  // unpadded FLOPs of this product, for profiling reports
+  void* splitk;       // optional scratch for fp32 partials: lets a thin product with a long contraction (bf16, no bias,
+  size_t splitk_bytes; // no activation, one output) be cut along K over the SMs; nullptr = never
   Epilogue epi;
 };
 
@@ -199,6 +201,7 @@ struct ffsplit_ctx {
   int* status() const { return reinterpret_cast<int*>(ws); }
   int* tickets() const { return reinterpret_cast<int*>(ws + ffsp::kStatusBytes); }
   int gemm_two_m = 1;          // tensor-core GEMM: 256-row tiles where they pay (FFSPLIT_GEMM_TWO_M=0: never, 2: wherever allowed)
+  int gemm_split_k = 1;        // tensor-core GEMM: cut thin products with a long contraction along K (FFSPLIT_GEMM_SPLIT_K=0: never)
   int gemm_panel = 0;          // tensor-core GEMM: tile rows per panel of the tile walk (0: chosen per launch; FFSPLIT_GEMM_PANEL)
   int decode_one_launch = 0;   // few-token forward: 1 = all products in one cooperative launch (FFSPLIT_DECODE_LAYER=1), 0 = one launch per product
   int decode_stream = 1;       // few tokens: 1 = the single-launch streaming kernel where it is the faster one, 2 = for every T <= 8, 0 = never (FFSPLIT_DECODE_STREAM)

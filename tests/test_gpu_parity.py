@@ -407,6 +407,32 @@ def _long_contraction_body(ctx, L, cfg, act, T, d, m, k, r):
     assert_close(G.forward(blobd, X), dense_ref, "bf16", "dense forward, long K")
 
 
+@pytest.mark.parametrize("act,d,m,k,r,T", [("gelu_erf", 256, 9000, 40, 128, 300),     # 3 tiles of 128 x 128: K cut in four
+                                          ("swiglu", 320, 6100, 60, 256, 500),       # gated chain, K = 6048 cut in four, ragged ranges
+                                          ("gelu_tanh", 192, 4300, 20, 48, 2000)])   # 16 tiles: K cut in four of 17 / 16 k-blocks
+def test_light_chain_second_product_cut_along_k(ctx, monkeypatch, act, d, m, k, r, T):
+    """P = H_L A2 has a thin output (r columns) and a long contraction (m - k): the GEMM cuts K into ranges that run as
+    work units of their own with fp32 partials and a fixed-order sum.  Against the oracle, and against the same GEMM
+    with the cut switched off."""
+    cfg = custom_config(d, m, k, r, act=act, dtype="bf16")
+    L = make_layer(cfg, 4)
+    G = GpuLayer(ctx, L)
+    G.reserve(T, 0, k, r)
+    fac = oracle_factors(L, L.planted.numpy(), r)
+    blob, _ = G.pack(L.planted, fac)
+    X = L.tokens(T)
+    Yref = oracle_split(L, L.planted.numpy(), fac, X)
+    monkeypatch.setenv("FFSPLIT_NO_FUSED", "1")          # the four-GEMM chain
+    monkeypatch.setenv("FFSPLIT_LAYER_KERNEL", "0")
+    n0 = ctx.launch_count()
+    Y = forward_on_fresh_context(G, blob, X, T, k, r)
+    assert_close(Y, Yref, "bf16", "light chain cut along K")
+    monkeypatch.setenv("FFSPLIT_GEMM_SPLIT_K", "0")
+    Y2 = forward_on_fresh_context(G, blob, X, T, k, r)
+    assert_close(Y2, Yref, "bf16", "light chain, whole K")
+    assert orc.rel_frobenius(f64(Y2), f64(Y)) < 5e-3
+
+
 @pytest.mark.parametrize("dt,act,d,m,T", [("bf16", "gelu_erf", 256, 1000, 300), ("bf16", "swiglu", 192, 520, 5),
                                          ("f32", "gelu_erf", 64, 192, 70), ("bf16", "gelu_tanh", 128, 384, 40)])
 def test_forward_dense_entry_point(ctx, dt, act, d, m, T):
