@@ -84,6 +84,31 @@ __device__ __forceinline__ float gelu_erf_score_f(float z) {
   const float erf_abs = fmaf(-poly * t, __expf(-x * x), 1.0f);
   return 0.5f * z * (1.0f + copysignf(erf_abs, z));
 }
+// The square of the same GELU for two values at once, on the packed fp32 instructions: with
+// q = (a1 t + ... + a5 t^5) exp(-x^2) / 2 (the coefficients carry the 1/2), Phi(z) = 1 - q for z >= 0 and q for z < 0,
+// so GELU(z) = z Phi(z) without forming erf.  Ten instructions per value instead of nineteen; the same rational
+// approximation, reciprocal and exponential, hence the same accuracy (about 1e-6 absolute).
+__device__ __forceinline__ float2 gelu_erf_score_sq2(float2 z) {
+  const float2 x = __fmul2_rn(make_float2(fabsf(z.x), fabsf(z.y)), make_float2(0.70710678118654752f, 0.70710678118654752f));
+  const float2 den = __ffma2_rn(make_float2(0.3275911f, 0.3275911f), x, make_float2(1.0f, 1.0f));
+  float2 t;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t.x) : "f"(den.x));
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t.y) : "f"(den.y));
+  float2 poly = __ffma2_rn(make_float2(0.5f * 1.061405429f, 0.5f * 1.061405429f), t, make_float2(0.5f * -1.453152027f, 0.5f * -1.453152027f));
+  poly = __ffma2_rn(poly, t, make_float2(0.5f * 1.421413741f, 0.5f * 1.421413741f));
+  poly = __ffma2_rn(poly, t, make_float2(0.5f * -0.284496736f, 0.5f * -0.284496736f));
+  poly = __ffma2_rn(poly, t, make_float2(0.5f * 0.254829592f, 0.5f * 0.254829592f));
+  const float2 pt = __fmul2_rn(poly, t);
+  const float2 ex = __fmul2_rn(__fmul2_rn(x, x), make_float2(-1.4426950408889634f, -1.4426950408889634f));
+  float2 e;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e.x) : "f"(ex.x));
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e.y) : "f"(ex.y));
+  const float2 q = __fmul2_rn(pt, e);
+  const float2 om = __ffma2_rn(q, make_float2(-1.0f, -1.0f), make_float2(1.0f, 1.0f));
+  const float2 phi = make_float2(z.x >= 0.f ? om.x : q.x, z.y >= 0.f ? om.y : q.y);
+  const float2 g = __fmul2_rn(z, phi);
+  return __fmul2_rn(g, g);
+}
 __device__ __forceinline__ float act_gelu_score(float z, int act) {
   return act == FFSPLIT_GELU_TANH ? gelu_tanh_f(z) : gelu_erf_score_f(z);
 }

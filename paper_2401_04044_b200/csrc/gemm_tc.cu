@@ -361,9 +361,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           if (!p.dual && e.act == FFSPLIT_GELU_ERF && !e.score_abs) {
             // the common case, without per-element selects
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-              const float x = gelu_erf_score_f(v[i]);
-              v[i] = x * x;
+            for (int i = 0; i < 8; ++i) {
+              const float2 sq = gelu_erf_score_sq2(make_float2(v[2 * i], v[2 * i + 1]));
+              v[2 * i] = sq.x;
+              v[2 * i + 1] = sq.y;
             }
           } else {
 #pragma unroll
