@@ -183,14 +183,19 @@ static ffsplit_status decode_forward_impl(ffsplit_ctx* ctx, const BlobHeader& h,
                                           cudaStream_t st, int* tickets, long long scratch_bytes,
                                           unsigned long long guard_hash) {
   const int T = static_cast<int>(T64);
-  // Which of the two few-token kernels: the single-launch streaming kernel wins where a layer's weights are
-  // many megabytes and the activation operand of a pass fits four token rows (measured, 1 token: OPT-13B-shaped
-  // split layer 38 vs 42 us, Llama-2-7B-shaped 45 vs 51 us, their dense layers 86 vs 85 and 55 vs 61 us; at
-  // 5 to 8 tokens the per-product kernel is ahead, 43 vs 64 us, and so it is on layers of a few megabytes, whose
-  // time is all hand-over: GPT-2-medium-shaped split layer 17 vs 20 us).  FFSPLIT_DECODE_STREAM=2 forces the
-  // streaming kernel for every T <= 8, 0 turns it off.
+  // Which of the two few-token kernels (measured per layer, CUDA-graph replays over distinct weight copies).  The
+  // single-launch streaming kernel wins on layers without a light part, whose two products are tens of megabytes
+  // each: dense Llama-2-7B shape 53 vs 62 us at one token, dense GPT-2-medium shape 11 vs 13.5 us.  On split layers
+  // (four or five dependent products) the two are within 1.5 us of each other at one token where the streaming
+  // kernel is ahead (OPT-13B shape, 5 % heavy, r = 512: 40.7 vs 41.7 us) and the per-product kernel is up to 10 us
+  // ahead elsewhere (1 % heavy or r = 1280: 51.7 vs 61.8 us) and at every point with more than one token (36-56 vs
+  // 48-79 us at four tokens); only the gated (SwiGLU) split layer at one token keeps the streaming kernel (48.6 vs
+  // 51.2 us).  FFSPLIT_DECODE_STREAM=2 forces the streaming kernel for every T <= 8, 0 turns it off.
   const double layer_bytes = 2.0 * (h.n_in + 1) * (static_cast<double>(h.d) * h.k + static_cast<double>(h.r) * (h.d + h.ml));
-  const bool stream = ctx->decode_stream == 2 || (ctx->decode_stream == 1 && T <= 4 && layer_bytes >= 16e6);
+  const bool no_light = h.r == 0 || h.ml == 0;
+  const bool gated_one = h.act == FFSPLIT_SWIGLU && T == 1;
+  const bool stream = ctx->decode_stream == 2 ||
+                      (ctx->decode_stream == 1 && T <= 4 && layer_bytes >= 16e6 && (no_light || gated_one));
   if (T <= 8 && stream) {
     // one persistent launch whose weight stream runs ahead of the stage dependencies; its slices take the whole
     // scratch area (the [A_H | P], Q and H_L buffers of the other kernel are not used)
