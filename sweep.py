@@ -232,6 +232,11 @@ def run_factor(ctx, cfg, iters, reps, device="cuda"):
         out[label] = {"ms": ms, "product_tflops": flops / (ms * 1e-3) / 1e12}
         if it > 0:      # (without a round the start basis is not orthonormal and A1 B1 is no projection)
             out[label]["rel_residual_U2"] = resid / torch.linalg.matrix_norm(U2).item()
+            if cfg.d <= 1024:
+                # the optimum (Eckart-Young) from the singular values of the slice, in float64 on the device
+                sv = torch.linalg.svdvals(U2.double())
+                best = sv[cfg.r:].square().sum().sqrt().item()
+                out[label]["residual_over_truncated_svd"] = resid / best
     return out
 
 
