@@ -210,7 +210,7 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
   ctx->score_prep.valid = false;   // the forward buffers share the workspace with the scoring buffers
   const FwdLayout L = fwd_layout(D, d, h.dtype, h.act, T);
   const bool few = decode_path_applies(ctx, h, T);
-  if (kCtrlBytes + (few ? L.end : L.xs) > ctx->ws_bytes)
+  if (kCtrlBytes + (T <= 64 ? L.end : L.xs) > ctx->ws_bytes)
     return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL, "workspace too small for this forward (ffsplit_workspace_size)");
   char* AP = base + L.ap;
   char* Q = base + L.q;
@@ -224,6 +224,10 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
   const bool light = D.r_pad > 0 && D.ml > 0;
   ffsplit_status s;
   GemmArgs g;
+  // 13..64 tokens of a bf16 layer: the stage GEMMs below with the operands exchanged (weights as accumulator rows)
+  const bool few_tc = h.dtype == FFSPLIT_BF16 && T <= 64;
+  void* few_ptr = few_tc ? base + L.dscratch : nullptr;
+  const size_t few_bytes = few_tc ? decode_scratch_bytes(h.dtype, T) : 0;
 
   // ---- small hidden widths: the whole layer in one launch, a cluster of four CTAs per 128-token tile
   if (light && ctx->use_layer_kernel && fused_layer_applies(h.dtype, h.act, d, D.k, D.k_pad, D.r_pad, D.ml_pad, T, ctx->num_sms))
@@ -232,6 +236,7 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
   // ---- stage 1: [A_H | Q] = X [U1 | A1], activation on the heavy columns only
   if (!gated) {
     std::memset(&g, 0, sizeof(g));
+    g.few = few_ptr; g.few_bytes = few_bytes;
     g.A0 = X; g.lda0 = d;
     g.B0 = blob + h.off[SEC_U1T]; g.ldb0 = d;
     g.M = T; g.N = D.kp_rp; g.K = d;
@@ -244,6 +249,7 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
     if ((s = launch_gemm(ctx, h.dtype, g, st)) != FFSPLIT_OK) return s;
   } else {
     std::memset(&g, 0, sizeof(g));
+    g.few = few_ptr; g.few_bytes = few_bytes;
     g.A0 = X; g.lda0 = d; g.B0 = blob + h.off[SEC_U1T]; g.ldb0 = d;
     g.A1 = X; g.lda1 = d; g.B1 = blob + h.off[SEC_U1UT]; g.ldb1 = d;
     g.M = T; g.N = D.k_pad; g.K = d;
@@ -254,6 +260,7 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
     if ((s = launch_gemm(ctx, h.dtype, g, st)) != FFSPLIT_OK) return s;
     if (light) {
       std::memset(&g, 0, sizeof(g));
+    g.few = few_ptr; g.few_bytes = few_bytes;
       g.A0 = X; g.lda0 = d; g.B0 = blob + h.off[SEC_A1T]; g.ldb0 = d;  // [A1 | A1u]^T
       g.M = T; g.N = 2 * D.r_pad; g.K = d;
       g.algo_flops = 4.0 * T * d * D.r;
@@ -267,13 +274,14 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
     ctx->use_fused = (env && env[0] == '1') ? 0 : 1;
   }
   const long long tiles_m = (T + 127) / 128;
-  if (light && ctx->use_fused && fused_light_applies(h.dtype, h.act, D.r_pad, D.ml_pad) && tiles_m <= kMaxTicketTiles) {
+  if (light && ctx->use_fused && !few_tc && fused_light_applies(h.dtype, h.act, D.r_pad, D.ml_pad) && tiles_m <= kMaxTicketTiles) {
     if ((s = launch_fused_light(ctx, Q, D.r_pad, T, blob + h.off[SEC_B1T], blob + h.off[SEC_A2T], b1l, D.r_pad,
                                 D.ml_pad, h.act, AP + (size_t)D.k_pad * es, D.kp_rp, HL, ctx->tickets(),
                                 4.0 * T * D.r * D.ml, st)) != FFSPLIT_OK)
       return s;
   } else if (light) {
     std::memset(&g, 0, sizeof(g));
+    g.few = few_ptr; g.few_bytes = few_bytes;
     g.A0 = Q; g.lda0 = (long long)D.n_in * D.r_pad;
     g.B0 = blob + h.off[SEC_B1T]; g.ldb0 = D.r_pad;
     if (gated) {
@@ -288,6 +296,7 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
     if ((s = launch_gemm(ctx, h.dtype, g, st)) != FFSPLIT_OK) return s;
 
     std::memset(&g, 0, sizeof(g));
+    g.few = few_ptr; g.few_bytes = few_bytes;
     g.A0 = HL; g.lda0 = D.ml_pad;
     g.B0 = blob + h.off[SEC_A2T]; g.ldb0 = D.ml_pad;
     g.M = T; g.N = D.r_pad; g.K = D.ml_pad;
@@ -299,6 +308,7 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
   }
   // ---- stage 3: Y = [A_H | P] [V1 ; B2] + b2 (heavy and light parts in one accumulator)
   std::memset(&g, 0, sizeof(g));
+    g.few = few_ptr; g.few_bytes = few_bytes;
   g.A0 = AP; g.lda0 = D.kp_rp;
   g.B0 = blob + h.off[SEC_V1B2T]; g.ldb0 = D.kp_rp;
   g.M = T; g.N = d; g.K = light ? D.kp_rp : D.k_pad;
@@ -457,6 +467,7 @@ ffsplit_status ffsplit_create(ffsplit_ctx** out, int device) {
   if (const char* env = std::getenv("FFSPLIT_GEMM_TWO_M")) c->gemm_two_m = env[0] == '0' ? 0 : env[0] == '2' ? 2 : 1;
   if (const char* env = std::getenv("FFSPLIT_GEMM_PANEL")) c->gemm_panel = std::atoi(env);
   if (const char* env = std::getenv("FFSPLIT_GEMM_SPLIT_K")) c->gemm_split_k = env[0] == '0' ? 0 : 1;
+  if (const char* env = std::getenv("FFSPLIT_FEW_TENSOR_MIN")) c->few_tensor_min = std::atoi(env);
   if (const char* env = std::getenv("FFSPLIT_LAYER_KERNEL")) c->use_layer_kernel = env[0] == '0' ? 0 : 1;
   if (const char* env = std::getenv("FFSPLIT_DECODE_LAYER")) c->decode_one_launch = env[0] == '0' ? 0 : 1;
   if (const char* env = std::getenv("FFSPLIT_DECODE_STREAM")) c->decode_stream = env[0] == '0' ? 0 : env[0] == '2' ? 2 : 1;

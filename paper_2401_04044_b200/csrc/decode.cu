@@ -17,6 +17,7 @@
 namespace ffsp {
 
 constexpr long long kDecodeScratchBytes = 16ll << 20;   // fp32 partials of the row tiles that several CTAs share
+constexpr long long kFewScratchBytes = 64ll << 20;      // the region's size: also the fp32 partials of the tensor-core few-token path
 
 // ---- 1..8 tokens: the phases of one layer for decode_stream_kernel ---------------------------------------
 // Every phase writes raw fp32 sums (one slice per k range); the phase that reads them adds the slices, the
@@ -167,15 +168,22 @@ static ffsplit_status stream_forward(ffsplit_ctx* ctx, const BlobHeader& h, cons
   return decode_stream_launch(ctx, p, algo_bytes, st);
 }
 
+// The weight-streaming kernels take bf16 layers at up to few_tensor_min tokens; above that (up to 64) the forward
+// runs its stage GEMMs on the tensor cores with the operands exchanged (GemmArgs::few).
 bool decode_path_applies(const ffsplit_ctx* ctx, const BlobHeader& h, long long T) {
-  (void)ctx;
-  return h.dtype == FFSPLIT_BF16 && T >= 1 && T <= 64;
+  // (measured: on layers of tens of megabytes the tensor path is ahead from 13 tokens on -- OPT-13B-shaped split layer
+  // 46 vs 57 us at 16 tokens, 63 vs 151 us at 64 -- on layers of a few megabytes from about 24 tokens on:
+  // GPT-2-medium-shaped split layer 29 vs 27 us at 16 tokens, 35 vs 67 us at 64)
+  const double layer_bytes = 2.0 * (h.n_in + 1) * (static_cast<double>(h.d) * h.k + static_cast<double>(h.r) * (h.d + h.ml));
+  long long limit = ctx->few_tensor_min < 64 ? ctx->few_tensor_min : 64;
+  if (layer_bytes < 16e6 && limit < 24 && ctx->few_tensor_min >= 0) limit = 24;
+  return h.dtype == FFSPLIT_BF16 && T >= 1 && T <= limit;
 }
 
 // fp32 partials of one product.
 size_t decode_scratch_bytes(int dtype, long long T) {
   if (dtype != FFSPLIT_BF16 || T > 64 || T < 1) return 0;
-  return static_cast<size_t>(kDecodeScratchBytes);
+  return static_cast<size_t>(kFewScratchBytes);
 }
 
 static ffsplit_status decode_forward_impl(ffsplit_ctx* ctx, const BlobHeader& h, const char* blob, const void* X,

@@ -16,6 +16,8 @@
 //
 // Every mbarrier wait is bounded; on expiry the CTA records FFSPLIT_ERR_TIMEOUT in
 // the status block, drains what it has in flight, frees its TMEM and returns.
+#include <cstring>
+
 #include "epilogue.cuh"
 #include "internal.h"
 #include "ptx.cuh"
@@ -457,6 +459,43 @@ __global__ void __launch_bounds__(256) splitk_reduce_kernel(const float* partial
   *reinterpret_cast<uint2*>(C + row * ldc + c) = o;
 }
 
+// Few-token path: Y[t, n] = epi(sum over the `split` partials of acc[n, t]) from the exchanged product's fp32 partials
+// [split][n_out][tp] (and a second set for the gated pair), with the epilogue of internal.h read along n:
+// bias[n], activation for n < n_act (gated: silu(acc0) * acc1), n < n_split to C0[t, n], else to C1[t, n - n_split].
+// Threads run along n, so every token row is written in contiguous runs.
+__global__ void __launch_bounds__(256) few_finish_kernel(const float* p0, const float* p1, int split, int n_out, int T, int tp,
+                                                         Epilogue e) {
+  pdl_wait();
+  const int n = blockIdx.x * 256 + threadIdx.x;
+  const int t0 = blockIdx.y * 4;
+  if (n >= n_out) return;
+  float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+  for (int s = 0; s < split; ++s) {
+    const size_t at = (static_cast<size_t>(s) * n_out + n) * tp + t0;
+    const float4 v = __ldcg(reinterpret_cast<const float4*>(p0 + at));
+    a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+    if (p1) {
+      const float4 u = __ldcg(reinterpret_cast<const float4*>(p1 + at));
+      b.x += u.x; b.y += u.y; b.z += u.z; b.w += u.w;
+    }
+  }
+  float v[4] = {a.x, a.y, a.z, a.w};
+  const float u[4] = {b.x, b.y, b.z, b.w};
+  const float bias = n < e.n_bias ? __ldg(e.bias + n) : 0.f;
+  const GeluCoef gc = gelu_coef(e.act);
+  const bool first = n < e.n_split;
+  __nv_bfloat16* base = first ? reinterpret_cast<__nv_bfloat16*>(e.C0) + n : reinterpret_cast<__nv_bfloat16*>(e.C1) + (n - e.n_split);
+  const long long ld = first ? e.ld0 : e.ld1;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    if (t0 + i >= T) break;
+    float x = v[i] + bias;
+    if (p1) x = silu_fast(x) * u[i];
+    else if (n < e.n_act) x = gelu_fast(x, gc);
+    base[static_cast<long long>(t0 + i) * ld] = __float2bfloat16_rn(x);
+  }
+}
+
 #undef UNIT_KB
 
 }  // namespace tc
@@ -522,7 +561,53 @@ static int choose_block_n(int N, long long tiles_m, int num_sms, bool dual) {
   return best;
 }
 
+ffsplit_status launch_gemm_tc(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_t st);
+
+// C [T, N] = epi(X [T, K] . (W [N, K])^T) for T <= 64 on the tensor cores (see GemmArgs::few).
+static ffsplit_status launch_gemm_few(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_t st) {
+  const int T = static_cast<int>(g.M), tp = round_up(T, 16), n_out = g.N;
+  const bool gated = g.A1 != nullptr;
+  const int nmat = gated ? 2 : 1;
+  const long long tiles = (n_out + tc::BLOCK_M - 1) / tc::BLOCK_M;
+  const int nkb = (g.K + tc::BLOCK_K - 1) / tc::BLOCK_K;
+  // K ranges: fill the last wave of work units, keep at least four k-blocks per unit and the partials inside the scratch
+  int best = 1;
+  double best_eff = -1.0;
+  for (int s = 1; s <= 16; ++s) {
+    if (s > 1 && nkb / s < 4) break;
+    if (nkb - (s - 1) * ((nkb + s - 1) / s) <= 0) continue;   // the last range must not be empty
+    if (static_cast<size_t>(nmat) * s * n_out * tp * 4 > g.few_bytes) break;
+    const long long units = tiles * s;
+    const long long waves = (units + ctx->num_sms - 1) / ctx->num_sms;
+    const double eff = static_cast<double>(units) / static_cast<double>(waves * ctx->num_sms);
+    if (eff > best_eff + 0.02) { best_eff = eff; best = s; }
+  }
+  if (static_cast<size_t>(nmat) * best * n_out * tp * 4 > g.few_bytes)
+    return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL, "workspace too small for the few-token tensor path");
+  float* part[2] = {static_cast<float*>(g.few), static_cast<float*>(g.few) + static_cast<size_t>(best) * n_out * tp};
+  for (int i = 0; i < nmat; ++i) {
+    GemmArgs h;
+    std::memset(&h, 0, sizeof(h));
+    h.A0 = i == 0 ? g.B0 : g.B1; h.lda0 = i == 0 ? g.ldb0 : g.ldb1;     // the weights: rows of the accumulator
+    h.B0 = i == 0 ? g.A0 : g.A1; h.ldb0 = i == 0 ? g.lda0 : g.lda1;     // the tokens: its columns
+    h.M = n_out; h.N = tp; h.K = g.K;
+    h.algo_flops = g.algo_flops / nmat;
+    h.epi.C0 = part[i]; h.epi.ld0 = tp; h.epi.n_split = tp; h.epi.act = FFSPLIT_GELU_ERF;
+    h.epi.guard = i == 0 ? g.epi.guard : nullptr; h.epi.guard_hash = g.epi.guard_hash;
+    h.force_split = best;
+    const ffsplit_status s = launch_gemm_tc(ctx, h, st);
+    if (s != FFSPLIT_OK) return s;
+  }
+  Epilogue e = g.epi;
+  const cudaError_t le = launch_pdl(tc::few_finish_kernel, dim3((n_out + 255) / 256, (T + 3) / 4), dim3(256), 0, st,
+                                    static_cast<const float*>(part[0]), gated ? static_cast<const float*>(part[1]) : nullptr,
+                                    best, n_out, T, tp, e);
+  ctx->launches++;
+  return check_cuda(ctx, le, "few_finish_kernel launch");
+}
+
 ffsplit_status launch_gemm_tc(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_t st) {
+  if (g.few && g.force_split == 0 && g.M <= 64 && !g.epi.col_partial && !g.epi.c0_f32) return launch_gemm_few(ctx, g, st);
   const bool dual = g.A1 != nullptr;
   if (g.M <= 0 || g.N <= 0 || g.K <= 0) return FFSPLIT_OK;
   tc::Params p;
@@ -560,7 +645,15 @@ ffsplit_status launch_gemm_tc(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_t 
   p.kb_split = (g.K + tc::BLOCK_K - 1) / tc::BLOCK_K;
   const bool plain = !dual && !g.epi.col_partial && !g.epi.c0_f32 && g.epi.n_bias == 0 && g.epi.n_act == 0 &&
                      g.epi.n_split >= g.N && g.N % 4 == 0 && (reinterpret_cast<uintptr_t>(g.epi.C0) & 7u) == 0 && g.epi.ld0 % 4 == 0;
-  if (ctx->gemm_split_k && g.splitk && plain && g.K >= 4096) {
+  if (g.force_split >= 1) {
+    // the few-token path: one tile column as wide as the (padded) token count, K cut as asked
+    p.two_m = 0;
+    p.tiles_m = static_cast<int>((g.M + tc::BLOCK_M - 1) / tc::BLOCK_M);
+    p.block_n = g.N;
+    p.tiles_n = 1;
+    p.split_k = g.force_split;
+    p.kb_split = (p.kb_split + g.force_split - 1) / g.force_split;
+  } else if (ctx->gemm_split_k && g.splitk && plain && g.K >= 4096) {
     const int bn = g.N >= 256 ? 256 : round_up(g.N, 16);
     const int nkb = p.kb_split;
     // 128-row tiles (256-row tiles with K cut in four were measured too: 284 us per OPT-13B-shaped split layer against
@@ -596,7 +689,9 @@ ffsplit_status launch_gemm_tc(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_t 
   }
   p.gate_off = p.shared_a ? p.block_n : tc::GATE_OFFSET;
   p.epi = g.epi;
-  if (p.split_k > 1) {
+  if (g.force_split >= 1) {
+    p.epi.c0_f32 = 1;         // the caller's C0 is the fp32 partial buffer [split][M][N] already
+  } else if (p.split_k > 1) {
     p.epi.C0 = g.splitk;      // fp32 partials [split][M][N]
     p.epi.ld0 = g.N;
     p.epi.c0_f32 = 1;
@@ -638,7 +733,7 @@ ffsplit_status launch_gemm_tc(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_t 
   cfg.numAttrs = 1;
   const cudaError_t le = cudaLaunchKernelEx(&cfg, tc::gemm_tc_kernel, tA0, tB0, tA1, tB1, p);
   ctx->launches++;
-  if (le != cudaSuccess || p.split_k == 1) {
+  if (le != cudaSuccess || p.split_k == 1 || g.force_split >= 1) {
     prof_close(ctx, ph, st);
     return check_cuda(ctx, le, "gemm_tc_kernel launch");
   }

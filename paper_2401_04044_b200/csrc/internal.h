@@ -106,6 +106,11 @@ struct GemmArgs {
   int N;
   int K;
   double algo_flops;  // unpadded FLOPs of this product, for profiling reports
+  // Few tokens (M <= 64) on the tensor cores: the product is run with the operands exchanged (weights as the rows of
+  // the accumulator, tokens as its columns), cut along K into enough work units to fill the SMs, and finished by a
+  // small kernel that adds the fp32 partials, applies this epilogue and stores the transpose.  Needs scratch.
+  void* few; size_t few_bytes;
+  int force_split;    // internal: K ranges of the exchanged product (set by the few-token path)
   void* splitk;       // optional scratch for fp32 partials: lets a thin product with a long contraction (bf16, no bias,
   size_t splitk_bytes; // no activation, one output) be cut along K over the SMs; nullptr = never
   Epilogue epi;
@@ -201,6 +206,8 @@ struct ffsplit_ctx {
   int* status() const { return reinterpret_cast<int*>(ws); }
   int* tickets() const { return reinterpret_cast<int*>(ws + ffsp::kStatusBytes); }
   int gemm_two_m = 1;          // tensor-core GEMM: 256-row tiles where they pay (FFSPLIT_GEMM_TWO_M=0: never, 2: wherever allowed)
+  int few_tensor_min = 12;     // few-token forward: token counts above this (up to 64) take the tensor-core path with exchanged
+                               // operands instead of the weight-streaming kernels (FFSPLIT_FEW_TENSOR_MIN; 64 = never)
   int gemm_split_k = 1;        // tensor-core GEMM: cut thin products with a long contraction along K (FFSPLIT_GEMM_SPLIT_K=0: never)
   int gemm_panel = 0;          // tensor-core GEMM: tile rows per panel of the tile walk (0: chosen per launch; FFSPLIT_GEMM_PANEL)
   int decode_one_launch = 0;   // few-token forward: 1 = all products in one cooperative launch (FFSPLIT_DECODE_LAYER=1), 0 = one launch per product

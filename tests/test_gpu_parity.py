@@ -367,6 +367,35 @@ def test_decode_forward_matches_oracle(ctx, act, d, m, k, r, T):
         assert_close(G.forward(blobd, X), dense_ref, "bf16", "decode dense forward")
 
 
+@pytest.mark.parametrize("act,d,m,k,r", DECODE_CASES)
+@pytest.mark.parametrize("T", [13, 16, 33, 64])
+def test_few_token_paths_agree(ctx, monkeypatch, act, d, m, k, r, T):
+    """13 to 64 tokens run on the tensor cores with the operands exchanged (the default; covered against the oracle by
+    the test above); FFSPLIT_FEW_TENSOR_MIN=64 keeps them on the weight-streaming kernel.  Both against the oracle,
+    split and dense, and against each other."""
+    cfg = custom_config(d, m, k, r, act=act, dtype="bf16")
+    L = make_layer(cfg, 8)
+    G = GpuLayer(ctx, L)
+    G.reserve(T, 0, k, r)
+    G.reserve(T, 0, m, 0)
+    fac = oracle_factors(L, L.planted.numpy(), r)
+    blob, _ = G.pack(L.planted, fac)
+    blobd, _ = G.pack(torch.arange(m), None)
+    X = L.tokens(T)
+    ref = oracle_split(L, L.planted.numpy(), fac, X)
+    refd = orc.dense_ffn(f64(X), f64(L.W1), f64(L.b1), f64(L.W2), f64(L.b2), act, f64(L.W1u))
+    n0 = ctx.launch_count()
+    Y = G.forward(blob, X)
+    launches_tensor = ctx.launch_count() - n0
+    assert_close(Y, ref, "bf16", "tensor few-token path, split")
+    assert_close(G.forward(blobd, X), refd, "bf16", "tensor few-token path, dense")
+    monkeypatch.setenv("FFSPLIT_FEW_TENSOR_MIN", "64")
+    Ys = forward_on_fresh_context(G, blob, X, T, k, r)
+    assert_close(Ys, ref, "bf16", "streaming few-token path, split")
+    assert orc.rel_frobenius(f64(Ys), f64(Y)) < 1e-2
+    assert launches_tensor >= 8        # four or five products, each a product launch and a finishing launch
+
+
 @pytest.mark.parametrize("act", ["gelu_erf", "swiglu"])
 @pytest.mark.parametrize("T", [300, 520])
 def test_long_contraction_tiles(monkeypatch, act, T):
