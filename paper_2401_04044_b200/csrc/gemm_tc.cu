@@ -570,9 +570,12 @@ static ffsplit_status launch_gemm_few(ffsplit_ctx* ctx, const GemmArgs& g, cudaS
   const int nmat = gated ? 2 : 1;
   const long long tiles = (n_out + tc::BLOCK_M - 1) / tc::BLOCK_M;
   const int nkb = (g.K + tc::BLOCK_K - 1) / tc::BLOCK_K;
-  // K ranges: fill the last wave of work units, keep at least four k-blocks per unit and the partials inside the scratch
+  // K ranges: more of them fill the last wave of work units better but write and re-read more fp32 partials; take the
+  // count with the least estimated traffic (weight bytes over the wave efficiency plus twice the partial bytes), with at
+  // least four k-blocks per unit and the partials inside the scratch
   int best = 1;
-  double best_eff = -1.0;
+  double best_cost = 1e300;
+  const double weight_bytes = 2.0 * n_out * g.K;
   for (int s = 1; s <= 16; ++s) {
     if (s > 1 && nkb / s < 4) break;
     if (nkb - (s - 1) * ((nkb + s - 1) / s) <= 0) continue;   // the last range must not be empty
@@ -580,7 +583,8 @@ static ffsplit_status launch_gemm_few(ffsplit_ctx* ctx, const GemmArgs& g, cudaS
     const long long units = tiles * s;
     const long long waves = (units + ctx->num_sms - 1) / ctx->num_sms;
     const double eff = static_cast<double>(units) / static_cast<double>(waves * ctx->num_sms);
-    if (eff > best_eff + 0.02) { best_eff = eff; best = s; }
+    const double cost = weight_bytes / eff + 2.0 * s * n_out * tp * 4;
+    if (cost < best_cost) { best_cost = cost; best = s; }
   }
   if (static_cast<size_t>(nmat) * best * n_out * tp * 4 > g.few_bytes)
     return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL, "workspace too small for the few-token tensor path");
