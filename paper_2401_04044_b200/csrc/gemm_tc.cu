@@ -470,13 +470,24 @@ __global__ void __launch_bounds__(256) few_finish_kernel(const float* p0, const 
   const int t0 = blockIdx.y * 4;
   if (n >= n_out) return;
   float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
-  for (int s = 0; s < split; ++s) {
-    const size_t at = (static_cast<size_t>(s) * n_out + n) * tp + t0;
-    const float4 v = __ldcg(reinterpret_cast<const float4*>(p0 + at));
-    a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
-    if (p1) {
-      const float4 u = __ldcg(reinterpret_cast<const float4*>(p1 + at));
-      b.x += u.x; b.y += u.y; b.z += u.z; b.w += u.w;
+  // the partials are added in order, but eight loads are in flight at a time
+  constexpr int FB = 8;
+  const size_t stride = static_cast<size_t>(n_out) * tp, at0 = static_cast<size_t>(n) * tp + t0;
+  for (int s0 = 0; s0 < split; s0 += FB) {
+    float4 v[FB], u[FB];
+#pragma unroll
+    for (int j = 0; j < FB; ++j) {
+      v[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+      u[j] = v[j];
+      if (s0 + j < split) {
+        v[j] = __ldcg(reinterpret_cast<const float4*>(p0 + (s0 + j) * stride + at0));
+        if (p1) u[j] = __ldcg(reinterpret_cast<const float4*>(p1 + (s0 + j) * stride + at0));
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < FB; ++j) {
+      a.x += v[j].x; a.y += v[j].y; a.z += v[j].z; a.w += v[j].w;
+      b.x += u[j].x; b.y += u[j].y; b.z += u[j].z; b.w += u[j].w;
     }
   }
   float v[4] = {a.x, a.y, a.z, a.w};
