@@ -171,8 +171,9 @@ static ffsplit_status stream_forward(ffsplit_ctx* ctx, const BlobHeader& h, cons
 // The weight-streaming kernels take bf16 layers at up to few_tensor_min tokens; above that (up to 64) the forward
 // runs its stage GEMMs on the tensor cores with the operands exchanged (GemmArgs::few).
 bool decode_path_applies(const ffsplit_ctx* ctx, const BlobHeader& h, long long T) {
-  // (measured: on layers of tens of megabytes the tensor path is ahead from 13 tokens on -- OPT-13B-shaped split layer
-  // 46 vs 57 us at 16 tokens, 63 vs 151 us at 64 -- on layers of a few megabytes from about 24 tokens on:
+  // (measured: on layers of tens of megabytes the tensor path is ahead from 9 tokens on -- OPT-13B-shaped split layer
+  // 41 vs 57 us at 9 tokens, 56 vs 151 us at 64; up to 8 tokens the two are level on GELU layers, 41 vs 43 us, and the
+  // streaming kernels are ahead on gated ones, 48 vs 60 us -- on layers of a few megabytes from about 24 tokens on:
   // GPT-2-medium-shaped split layer 29 vs 27 us at 16 tokens, 35 vs 67 us at 64)
   const double layer_bytes = 2.0 * (h.n_in + 1) * (static_cast<double>(h.d) * h.k + static_cast<double>(h.r) * (h.d + h.ml));
   long long limit = ctx->few_tensor_min < 64 ? ctx->few_tensor_min : 64;
