@@ -227,6 +227,7 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
   // 13..64 tokens of a bf16 layer: the stage GEMMs below with the operands exchanged (weights as accumulator rows)
   const bool few_tc = h.dtype == FFSPLIT_BF16 && T <= 64;
   void* few_ptr = few_tc ? base + L.dscratch : nullptr;
+  int n_gemm = 0;       // products launched so far by this call
   const size_t few_bytes = few_tc ? decode_scratch_bytes(h.dtype, T) : 0;
 
   // ---- small hidden widths: the whole layer in one launch, a cluster of four CTAs per 128-token tile
@@ -236,7 +237,7 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
   // ---- stage 1: [A_H | Q] = X [U1 | A1], activation on the heavy columns only
   if (!gated) {
     std::memset(&g, 0, sizeof(g));
-    g.few = few_ptr; g.few_bytes = few_bytes;
+    g.few = few_ptr; g.few_bytes = few_bytes; g.weights_stable = n_gemm++ > 0;
     g.A0 = X; g.lda0 = d;
     g.B0 = blob + h.off[SEC_U1T]; g.ldb0 = d;
     g.M = T; g.N = D.kp_rp; g.K = d;
@@ -249,7 +250,7 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
     if ((s = launch_gemm(ctx, h.dtype, g, st)) != FFSPLIT_OK) return s;
   } else {
     std::memset(&g, 0, sizeof(g));
-    g.few = few_ptr; g.few_bytes = few_bytes;
+    g.few = few_ptr; g.few_bytes = few_bytes; g.weights_stable = n_gemm++ > 0;
     g.A0 = X; g.lda0 = d; g.B0 = blob + h.off[SEC_U1T]; g.ldb0 = d;
     g.A1 = X; g.lda1 = d; g.B1 = blob + h.off[SEC_U1UT]; g.ldb1 = d;
     g.M = T; g.N = D.k_pad; g.K = d;
@@ -260,7 +261,7 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
     if ((s = launch_gemm(ctx, h.dtype, g, st)) != FFSPLIT_OK) return s;
     if (light) {
       std::memset(&g, 0, sizeof(g));
-    g.few = few_ptr; g.few_bytes = few_bytes;
+    g.few = few_ptr; g.few_bytes = few_bytes; g.weights_stable = n_gemm++ > 0;
       g.A0 = X; g.lda0 = d; g.B0 = blob + h.off[SEC_A1T]; g.ldb0 = d;  // [A1 | A1u]^T
       g.M = T; g.N = 2 * D.r_pad; g.K = d;
       g.algo_flops = 4.0 * T * d * D.r;
@@ -281,7 +282,7 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
       return s;
   } else if (light) {
     std::memset(&g, 0, sizeof(g));
-    g.few = few_ptr; g.few_bytes = few_bytes;
+    g.few = few_ptr; g.few_bytes = few_bytes; g.weights_stable = n_gemm++ > 0;
     g.A0 = Q; g.lda0 = (long long)D.n_in * D.r_pad;
     g.B0 = blob + h.off[SEC_B1T]; g.ldb0 = D.r_pad;
     if (gated) {
@@ -296,7 +297,7 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
     if ((s = launch_gemm(ctx, h.dtype, g, st)) != FFSPLIT_OK) return s;
 
     std::memset(&g, 0, sizeof(g));
-    g.few = few_ptr; g.few_bytes = few_bytes;
+    g.few = few_ptr; g.few_bytes = few_bytes; g.weights_stable = n_gemm++ > 0;
     g.A0 = HL; g.lda0 = D.ml_pad;
     g.B0 = blob + h.off[SEC_A2T]; g.ldb0 = D.ml_pad;
     g.M = T; g.N = D.r_pad; g.K = D.ml_pad;
@@ -308,7 +309,7 @@ ffsplit_status run_forward(ffsplit_ctx* ctx, const BlobHeader& h, const char* bl
   }
   // ---- stage 3: Y = [A_H | P] [V1 ; B2] + b2 (heavy and light parts in one accumulator)
   std::memset(&g, 0, sizeof(g));
-    g.few = few_ptr; g.few_bytes = few_bytes;
+    g.few = few_ptr; g.few_bytes = few_bytes; g.weights_stable = n_gemm++ > 0;
   g.A0 = AP; g.lda0 = D.kp_rp;
   g.B0 = blob + h.off[SEC_V1B2T]; g.ldb0 = D.kp_rp;
   g.M = T; g.N = d; g.K = light ? D.kp_rp : D.k_pad;

@@ -58,6 +58,9 @@ struct Params {
                      // work units) writing an fp32 partial [split][M][N]; a small kernel adds them (thin outputs with a
                      // long contraction: fewer tiles than SMs otherwise)
   int kb_split;      // k-blocks per range
+  int early;         // 1: the row operand (A) does not depend on the kernel before this one in the stream (packed weights
+                     // in the few-token path): its first stages are loaded before the programmatic-launch wait, under
+                     // the tail of that kernel; the other operand and every global write come after the wait
   Epilogue epi;
   int* status;
 };
@@ -225,11 +228,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   // Launched with programmatic stream serialisation: everything above (barriers, tensor maps, tensor
   // memory) overlapped the tail of the kernel before; nothing below may start until that kernel is
   // complete and its writes are visible.
-  asm volatile("griddepcontrol.wait;" ::: "memory");
-  // Only now may the kernel after this one begin its set-up: it will block in its tensor-memory allocation
-  // until this CTA frees its columns, which is safe because this CTA already holds its own (a dependent
-  // that got the columns first would wait for this kernel, and this kernel for the columns).
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  if (!p.early) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    // Only now may the kernel after this one begin its set-up: it will block in its tensor-memory allocation
+    // until this CTA frees its columns, which is safe because this CTA already holds its own (a dependent
+    // that got the columns first would wait for this kernel, and this kernel for the columns).
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  }
 
   const int nkb = (p.K + BLOCK_K - 1) / BLOCK_K;
   const int tiles_mn = p.tiles_m * p.tiles_n;
@@ -245,12 +250,34 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       // ------------------------------------------------------------ TMA producer
       uint32_t it = 0;
       bool ok = true;
+      int pre = 0;      // stages of the first unit whose loads were issued ahead of the loop
+      if (p.early) {
+        // weights first: the ring is empty, no slot needs waiting for
+        int m_blk = 0, n_blk = 0, ks = 0;
+        if (static_cast<int>(blockIdx.x) < num_tiles) {
+          ks = blockIdx.x / tiles_mn;
+          tile_coords(p, blockIdx.x - ks * tiles_mn, &m_blk, &n_blk);
+          const int total_kb = UNIT_KB(ks);
+          pre = total_kb < STAGES ? total_kb : STAGES;
+          for (int kb = 0; kb < pre; ++kb) {
+            ptx::mbar_expect_tx(&full[kb], stage_tx);
+            for (int mt = 0; mt < MT; ++mt)
+              ptx::tma_load_2d(&tmA0, smem_a + kb * A_STAGE + mt * A_STAGE_BYTES, &full[kb], (ks * p.kb_split + kb) * BLOCK_K,
+                               (m_blk * MT + mt) * BLOCK_M);
+          }
+        }
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+        for (int kb = 0; kb < pre; ++kb)
+          ptx::tma_load_2d(&tmB0, smem_b + kb * B_STAGE_BYTES, &full[kb], (ks * p.kb_split + kb) * BLOCK_K, n_blk * p.block_n);
+        it = pre;
+      }
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
         int m_blk, n_blk;
         const int ks = tile / tiles_mn;
         tile_coords(p, tile - ks * tiles_mn, &m_blk, &n_blk);
         const int total_kb = UNIT_KB(ks), nkb_u = p.split_k > 1 ? total_kb : nkb;
-        for (int kb = 0; kb < total_kb; ++kb, ++it) {
+        for (int kb = tile == static_cast<int>(blockIdx.x) ? pre : 0; kb < total_kb; ++kb, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1;
           if (!ptx::mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; break; }
@@ -335,6 +362,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     // other -- either way block number vt uses accumulator buffer vt & 1 in phase (vt >> 1) & 1.
     uint32_t vt = 0;
     bool live = true;
+    if (p.early) asm volatile("griddepcontrol.wait;" ::: "memory");   // before this role's first global access
     if (blockIdx.x == 0 && warp == 2) check_blob_guard(p.epi, p.status, KID_GEMM_TC);
     for (int tile = blockIdx.x; tile < num_tiles && live; tile += gridDim.x)
     for (int mt = 0; mt < MT; ++mt, ++vt) {
@@ -610,6 +638,7 @@ static ffsplit_status launch_gemm_few(ffsplit_ctx* ctx, const GemmArgs& g, cudaS
     h.epi.C0 = part[i]; h.epi.ld0 = tp; h.epi.n_split = tp; h.epi.act = FFSPLIT_GELU_ERF;
     h.epi.guard = i == 0 ? g.epi.guard : nullptr; h.epi.guard_hash = g.epi.guard_hash;
     h.force_split = best;
+    h.early_rows = g.weights_stable;  // the weights are this product's row operand
     const ffsplit_status s = launch_gemm_tc(ctx, h, st);
     if (s != FFSPLIT_OK) return s;
   }
@@ -703,6 +732,7 @@ ffsplit_status launch_gemm_tc(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_t 
     p.panel_m = ctx->gemm_panel > 0 ? (ctx->gemm_panel < p.tiles_m ? ctx->gemm_panel : p.tiles_m) : best;
   }
   p.gate_off = p.shared_a ? p.block_n : tc::GATE_OFFSET;
+  p.early = (g.early_rows && !dual) ? 1 : 0;
   p.epi = g.epi;
   if (g.force_split >= 1) {
     p.epi.c0_f32 = 1;         // the caller's C0 is the fp32 partial buffer [split][M][N] already
