@@ -280,7 +280,8 @@ ffsplit_status ffsplit_forward_stack_host(ffsplit_ctx* ctx, const void* const* b
  * make that first call outside any stream capture.
  * All calls on a device share the one array and it keeps the previous call's contents: the call
  * clears the counters it needs at zero itself, but two calls that overlap on the GPU (different
- * streams, no ordering between them) race on it.  Results equal those of ffsplit_forward().
+ * streams, no ordering between them) race on it.  Results equal those of ffsplit_forward() where that call runs the same weight-streaming
+ * kernels (it takes large GELU layers through its tensor-core path instead: equal within rounding there).
  * Like ffsplit_forward() it accepts only blobs packed or opened on `ctx`.  A device-side condition of
  * this call (a wait that ran out, a changed blob) is kept in the array's own status words until
  * ffsplit_poll() on any context of that device reports it; ffsplit_poll() needs no workspace for that. */

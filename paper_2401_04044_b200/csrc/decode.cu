@@ -168,17 +168,27 @@ static ffsplit_status stream_forward(ffsplit_ctx* ctx, const BlobHeader& h, cons
   return decode_stream_launch(ctx, p, algo_bytes, st);
 }
 
-// The weight-streaming kernels take bf16 layers at up to few_tensor_min tokens; above that (up to 64) the forward
-// runs its stage GEMMs on the tensor cores with the operands exchanged (GemmArgs::few).
+// Up to 64 tokens of a bf16 layer: true = the weight-streaming kernels of this file, false = the forward runs its
+// stage GEMMs on the tensor cores with the operands exchanged (GemmArgs::few).
 bool decode_path_applies(const ffsplit_ctx* ctx, const BlobHeader& h, long long T) {
-  // (measured: on layers of tens of megabytes the tensor path is ahead from 9 tokens on -- OPT-13B-shaped split layer
-  // 41 vs 57 us at 9 tokens, 56 vs 151 us at 64; up to 8 tokens the two are level on GELU layers, 41 vs 43 us, and the
-  // streaming kernels are ahead on gated ones, 48 vs 60 us -- on layers of a few megabytes from about 24 tokens on:
-  // GPT-2-medium-shaped split layer 29 vs 27 us at 16 tokens, 35 vs 67 us at 64)
+  // Measured per layer (graph replays over distinct weight copies), tensor path vs streaming kernels:
+  //   layers of tens of megabytes, GELU: ahead at every token count -- OPT-13B shape, 5 % heavy, r = 512: split
+  //     38 vs 42 us at 1 token, 38 vs 44 at 4, 39 vs 57 at 9, 56 vs 151 at 64; dense 83 vs 90 at 1 token, 85 vs 91 at
+  //     16, 102 vs 187 at 64 -- except the dense layer at 2 to 4 tokens (83 vs 80 us);
+  //   gated (SwiGLU) layers: the streaming kernels are ahead up to 8 tokens (Llama-2-7B shape, 1 token: 48 vs 54 us
+  //     split, 54 vs 62 dense), the tensor path from 9 on (61 vs 68 us);
+  //   smaller layers: the streaming kernels up to about 24 tokens on a split layer of a few megabytes (GPT-2-medium
+  //     shape, 16 tokens: 27 vs 29 us; 64 tokens: 67 vs 30 us), up to about 8 on its dense layer of 17 MB (1 token:
+  //     11 vs 15 us; 16 tokens: 19 vs 15.5 us).
+  // FFSPLIT_FEW_TENSOR_MIN = t replaces all of this by "streaming kernels up to t tokens": 64 keeps every count on
+  // them, -1 sends every count to the tensor path.
+  if (h.dtype != FFSPLIT_BF16 || T < 1 || T > 64) return false;
+  if (ctx->few_tensor_min != kFewTensorAuto) return T <= ctx->few_tensor_min;
   const double layer_bytes = 2.0 * (h.n_in + 1) * (static_cast<double>(h.d) * h.k + static_cast<double>(h.r) * (h.d + h.ml));
-  long long limit = ctx->few_tensor_min < 64 ? ctx->few_tensor_min : 64;
-  if (layer_bytes < 16e6 && limit < 24 && ctx->few_tensor_min >= 0) limit = 24;
-  return h.dtype == FFSPLIT_BF16 && T >= 1 && T <= limit;
+  const bool no_light = h.r == 0 || h.ml == 0;
+  if (layer_bytes < 32e6) return T <= (no_light ? 8 : 24);
+  if (h.act == FFSPLIT_SWIGLU) return T <= 8;
+  return no_light && T >= 2 && T <= 4;
 }
 
 // fp32 partials of one product.

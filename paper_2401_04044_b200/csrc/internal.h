@@ -182,6 +182,8 @@ struct TmapKeyHash {
 
 }  // namespace ffsp
 
+constexpr int kFewTensorAuto = -2;
+
 struct ffsplit_ctx {
   int device = 0;
   int num_sms = 0;
@@ -209,8 +211,10 @@ struct ffsplit_ctx {
   int* status() const { return reinterpret_cast<int*>(ws); }
   int* tickets() const { return reinterpret_cast<int*>(ws + ffsp::kStatusBytes); }
   int gemm_two_m = 1;          // tensor-core GEMM: 256-row tiles where they pay (FFSPLIT_GEMM_TWO_M=0: never, 2: wherever allowed)
-  int few_tensor_min = 8;     // few-token forward: token counts above this (up to 64) take the tensor-core path with exchanged
-                               // operands instead of the weight-streaming kernels (FFSPLIT_FEW_TENSOR_MIN; 64 = never)
+  int few_tensor_min = kFewTensorAuto;   // few-token forward (up to 64 tokens): token counts above this take the
+                               // tensor-core path with exchanged operands, the others the weight-streaming kernels
+                               // (FFSPLIT_FEW_TENSOR_MIN; -1 = always the tensor path, 64 = never).  Unset: chosen per
+                               // layer from its size and activation, see decode_path_applies()
   int gemm_split_k = 1;        // tensor-core GEMM: cut thin products with a long contraction along K (FFSPLIT_GEMM_SPLIT_K=0: never)
   int gemm_panel = 0;          // tensor-core GEMM: tile rows per panel of the tile walk (0: chosen per launch; FFSPLIT_GEMM_PANEL)
   int decode_one_launch = 0;   // few-token forward: 1 = all products in one cooperative launch (FFSPLIT_DECODE_LAYER=1), 0 = one launch per product
