@@ -348,6 +348,8 @@ def main():
     ap.add_argument("--reps", type=int, default=20)
     ap.add_argument("--svd", action="store_true", help="true SVD factors instead of random ones")
     ap.add_argument("--sweep5", action="store_true", help="config 5: all heavy fractions x ranks")
+    ap.add_argument("--point5", type=int, nargs=2, default=None, metavar=("HEAVY_PERCENT", "RANK"),
+                    help="config 5: one point of the sweep")
     ap.add_argument("--out", default=None)
     ap.add_argument("--which", nargs="*", default=["split", "dense"], choices=["split", "dense"],
                     help="time the split layer, its dense counterpart, or both")
@@ -377,6 +379,8 @@ def main():
     points = [base]
     if args.config == 5 and args.sweep5:
         points = [cfg5_point(h, r) for h in CFG5_HEAVY_PERCENT for r in CFG5_RANKS]
+    if args.config == 5 and args.point5:
+        points = [cfg5_point(*args.point5)]
     if args.scoring:
         print(json.dumps(run_scoring(ctx, base, args.reps, t_cal=args.t_cal or None)), flush=True)
         return
