@@ -66,6 +66,16 @@ struct Params {
   int* status;
 };
 
+// Position in a ring of n slots: slot index and the parity of the number of completed rounds (no divisions on the
+// producers' and the MMA issuer's paths: they share their schedulers with the epilogue warps).
+struct Cursor {
+  int slot = 0;
+  uint32_t phase = 0;
+  __device__ __forceinline__ void next(int n) {
+    if (++slot == n) { slot = 0; phase ^= 1u; }
+  }
+};
+
 // D[tmem] (+)= A[tmem] * B[smem desc]: A is a 128 x 16 bf16 slab held as 8 TMEM columns.
 __device__ __forceinline__ void umma_bf16_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc, uint32_t idesc,
                                              uint32_t accumulate) {
@@ -169,11 +179,12 @@ fused_light_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       ptx::mbar_expect_tx(qfull, p.kbq * QKB_BYTES);
       for (int kb = 0; kb < p.kbq; ++kb) ptx::tma_load_2d(&tmQ, smem_q + kb * QKB_BYTES, qfull, kb * KB, m_blk * BLOCK_M);
       int g = 0;
+      Cursor cur;
       for (int i = 0; i < my_chunks && ok; ++i) {
         const int chunk = c_begin + i;
-        for (int kb = 0; kb < p.kbq; ++kb, ++g) {
-          const int slot = g % p.b1_slots;
-          if (!ptx::mbar_wait(&b1empty[slot], ((g / p.b1_slots) & 1) ^ 1, abort_flag)) { ok = false; break; }
+        for (int kb = 0; kb < p.kbq; ++kb, ++g, cur.next(p.b1_slots)) {
+          const int slot = cur.slot;
+          if (!ptx::mbar_wait(&b1empty[slot], cur.phase ^ 1u, abort_flag)) { ok = false; break; }
           if (kb == 0) {
             // b1[light] of this chunk; a bias slot is reused 8 chunks later, by when its readers are long done
             const int n0 = chunk * CHUNK;
@@ -202,10 +213,11 @@ fused_light_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       // ------------------------------------------------------------ TMA producer: A2 ring
       bool ok = true;
       int g = 0;
+      Cursor cur;
       for (int i = 0; i < my_chunks && ok; ++i) {
-        for (int kb = 0; kb < CHUNK / KB; ++kb, ++g) {
-          const int slot = g % p.a2_slots;
-          if (!ptx::mbar_wait(&a2empty[slot], ((g / p.a2_slots) & 1) ^ 1, abort_flag)) { ok = false; break; }
+        for (int kb = 0; kb < CHUNK / KB; ++kb, ++g, cur.next(p.a2_slots)) {
+          const int slot = cur.slot;
+          if (!ptx::mbar_wait(&a2empty[slot], cur.phase ^ 1u, abort_flag)) { ok = false; break; }
           ptx::mbar_expect_tx(&a2full[slot], p.a2_slot_bytes);
           ptx::tma_load_2d(&tmA2, smem_a2 + slot * p.a2_slot_bytes, &a2full[slot], (c_begin + i) * CHUNK + kb * KB, 0);
         }
@@ -228,16 +240,21 @@ fused_light_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       bool ok = ptx::mbar_wait(qfull, 0, abort_flag);
       // GEMM-b of chunk j: Pacc += H(j) * A2 tile of chunk j.  H(j) sits in the S buffer j & 1: the
       // 32 fp32 columns [32 c, 32 c + 32) of S became the 16 packed columns [32 c, 32 c + 16).
+      Cursor ca2, cb1;   // gemm_b is called for j = 0, 1, 2, ... in order
+      const uint64_t q_desc0 = ptx::umma_desc_k128(ptx::smem_u32(smem_q));
+      const uint64_t b1_desc0 = ptx::umma_desc_k128(ptx::smem_u32(smem_b1));
+      const uint64_t a2_desc0 = ptx::umma_desc_k128(ptx::smem_u32(smem_a2));
+      const uint32_t a2_step = static_cast<uint32_t>(p.a2_slot_bytes) >> 4;   // descriptor addresses count 16 bytes
       auto gemm_b = [&](int j) -> bool {
         if (!ptx::mbar_wait(&hfull[j & 1], (j >> 1) & 1, abort_flag)) return false;
         ptx::tc_fence_after();
         const uint32_t h_tmem = tmem_base + TMEM_S0 + (j & 1) * CHUNK;
-        for (int kb = 0; kb < CHUNK / KB; ++kb) {
-          const int g = j * (CHUNK / KB) + kb;
-          const int slot = g % p.a2_slots;
-          if (!ptx::mbar_wait(&a2full[slot], (g / p.a2_slots) & 1, abort_flag)) return false;
+#pragma unroll
+        for (int kb = 0; kb < CHUNK / KB; ++kb, ca2.next(p.a2_slots)) {
+          const int slot = ca2.slot;
+          if (!ptx::mbar_wait(&a2full[slot], ca2.phase, abort_flag)) return false;
           ptx::tc_fence_after();
-          const uint64_t b_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_a2 + slot * p.a2_slot_bytes));
+          const uint64_t b_desc = a2_desc0 + static_cast<uint32_t>(slot) * a2_step;
 #pragma unroll
           for (int k = 0; k < KB / 16; ++k) {
             const int jj = kb * (KB / 16) + k;   // 16-element slab of this chunk's K range
@@ -248,16 +265,15 @@ fused_light_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         }
         return true;
       };
-      int g = 0;
       for (int i = 0; i < my_chunks && ok; ++i) {
         // S buffer i & 1 is free: GEMM-b of chunk i - 2 (its last reader) was issued before this point
         const uint32_t d_tmem = tmem_base + TMEM_S0 + (i & 1) * CHUNK;
-        for (int kb = 0; kb < p.kbq; ++kb, ++g) {
-          const int slot = g % p.b1_slots;
-          if (!ptx::mbar_wait(&b1full[slot], (g / p.b1_slots) & 1, abort_flag)) { ok = false; break; }
+        for (int kb = 0; kb < p.kbq; ++kb, cb1.next(p.b1_slots)) {
+          const int slot = cb1.slot;
+          if (!ptx::mbar_wait(&b1full[slot], cb1.phase, abort_flag)) { ok = false; break; }
           ptx::tc_fence_after();
-          const uint64_t a_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_q + kb * QKB_BYTES));
-          const uint64_t b_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_b1 + slot * B1KB_BYTES));
+          const uint64_t a_desc = q_desc0 + static_cast<uint32_t>(kb) * (QKB_BYTES >> 4);
+          const uint64_t b_desc = b1_desc0 + static_cast<uint32_t>(slot) * (B1KB_BYTES >> 4);
 #pragma unroll
           for (int k = 0; k < KB / 16; ++k)
             ptx::umma_bf16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc_a, (kb | k) != 0 ? 1u : 0u);
@@ -293,25 +309,28 @@ fused_light_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       const uint32_t t_s = t_lane + TMEM_S0 + sb * CHUNK + cg * 32;
       const float* bias = smem_bias + (i % BIAS_SLOTS) * CHUNK + cg * 32;
       const int n0 = (c_begin + i) * CHUNK + cg * 32;
+      // both 16-column loads in flight before the one wait; bias and GELU on the packed fp32 instructions (every
+      // component goes through gelu_fast's operations: the same bits)
       uint32_t w[16];
+      float va[16], vb[16];
+      ptx::tmem_ld16(t_s, va);
+      ptx::tmem_ld16(t_s + 16, vb);
+      ptx::tmem_ld_wait();
 #pragma unroll
       for (int hlf = 0; hlf < 2; ++hlf) {
-        float v[16];
-        ptx::tmem_ld16(t_s + 16 * hlf, v);
-        ptx::tmem_ld_wait();
-        const bool inside = n0 + 16 * hlf + 16 <= p.ml_pad;   // ml_pad is a multiple of 16
-        if (inside) {
+        const float* v = hlf ? vb : va;
+        if (n0 + 16 * hlf + 16 <= p.ml_pad) {   // ml_pad is a multiple of 16
 #pragma unroll
           for (int j = 0; j < 4; ++j) {
             const float4 b = *reinterpret_cast<const float4*>(bias + 16 * hlf + 4 * j);
-            v[4 * j] += b.x; v[4 * j + 1] += b.y; v[4 * j + 2] += b.z; v[4 * j + 3] += b.w;
+            const float2 g0 = gelu_fast2(__fadd2_rn(make_float2(v[4 * j], v[4 * j + 1]), make_float2(b.x, b.y)), gc);
+            const float2 g1 = gelu_fast2(__fadd2_rn(make_float2(v[4 * j + 2], v[4 * j + 3]), make_float2(b.z, b.w)), gc);
+            w[8 * hlf + 2 * j] = pack_bf16x2(g0.x, g0.y);
+            w[8 * hlf + 2 * j + 1] = pack_bf16x2(g1.x, g1.y);
           }
-        }
+        } else {
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const float lo = inside ? gelu_fast(v[2 * j], gc) : 0.f;
-          const float hi = inside ? gelu_fast(v[2 * j + 1], gc) : 0.f;
-          w[8 * hlf + j] = pack_bf16x2(lo, hi);
+          for (int j = 0; j < 8; ++j) w[8 * hlf + j] = 0u;
         }
       }
       tmem_st16(t_s, w);   // both 16-column loads of this warp's range have completed
