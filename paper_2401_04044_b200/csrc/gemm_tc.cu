@@ -272,14 +272,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           ptx::tma_load_2d(&tmB0, smem_b + kb * B_STAGE_BYTES, &full[kb], (ks * p.kb_split + kb) * BLOCK_K, n_blk * p.block_n);
         it = pre;
       }
+      // ring position of `it` without divisions (this thread shares its scheduler with epilogue warps)
+      int rs = pre == STAGES ? 0 : pre;
+      uint32_t rph = pre == STAGES ? 1u : 0u;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
         int m_blk, n_blk;
         const int ks = tile / tiles_mn;
         tile_coords(p, tile - ks * tiles_mn, &m_blk, &n_blk);
         const int total_kb = UNIT_KB(ks), nkb_u = p.split_k > 1 ? total_kb : nkb;
         for (int kb = tile == static_cast<int>(blockIdx.x) ? pre : 0; kb < total_kb; ++kb, ++it) {
-          const int s = it % STAGES;
-          const uint32_t ph = (it / STAGES) & 1;
+          const int s = rs;
+          const uint32_t ph = rph;
+          if (++rs == STAGES) { rs = 0; rph ^= 1u; }
           if (!ptx::mbar_wait(&empty[s], ph ^ 1, abort_flag)) { ok = false; break; }
           ptx::mbar_expect_tx(&full[s], stage_tx);
           const bool second = p.dual && kb >= nkb_u;
@@ -307,7 +311,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     if (ptx::elect_one()) {
       // ------------------------------------------------------------ MMA issuer
       const uint32_t idesc = ptx::umma_idesc_bf16(BLOCK_M, p.shared_a ? 2 * p.block_n : p.block_n);
-      uint32_t it = 0, tl = 0;
+      uint32_t tl = 0;
+      int rs = 0;          // ring position, kept without divisions
+      uint32_t rph = 0;
+      const uint64_t a_desc0 = ptx::umma_desc_k128(ptx::smem_u32(smem_a));
+      const uint64_t b_desc0 = ptx::umma_desc_k128(ptx::smem_u32(smem_b));
+      const uint32_t a_step = static_cast<uint32_t>(A_STAGE) >> 4, b_step = static_cast<uint32_t>(B_STAGE_BYTES) >> 4;   // descriptor addresses count 16 bytes
       bool ok = true;
       for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tl) {
         // one buffer per tile, alternating -- or, with 256-row tiles, both buffers for the two halves
@@ -316,16 +325,17 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         if (p.two_m && !ptx::mbar_wait(&tempty[1], aph ^ 1, abort_flag)) { ok = false; break; }
         ptx::tc_fence_after();
         const int total_kb = UNIT_KB(tile / tiles_mn);
-        for (int kb = 0; kb < total_kb; ++kb, ++it) {
-          const int s = it % STAGES;
-          const uint32_t ph = (it / STAGES) & 1;
+        for (int kb = 0; kb < total_kb; ++kb) {
+          const int s = rs;
+          const uint32_t ph = rph;
+          if (++rs == STAGES) { rs = 0; rph ^= 1u; }
           if (!ptx::mbar_wait(&full[s], ph, abort_flag)) { ok = false; break; }
           ptx::tc_fence_after();
           const bool second = p.dual && kb >= nkb;   // (a gated product is never cut along K)
           const int kbl = second ? kb - nkb : kb;
           const uint32_t d_tmem = tmem_base + acc * ACC_STRIDE + (second ? p.gate_off : 0);
-          const uint64_t a_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_a + s * A_STAGE));
-          const uint64_t b_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_b + s * B_STAGE_BYTES));
+          const uint64_t a_desc = a_desc0 + static_cast<uint32_t>(s) * a_step;
+          const uint64_t b_desc = b_desc0 + static_cast<uint32_t>(s) * b_step;
 #pragma unroll
           for (int k = 0; k < BLOCK_K / 16; ++k) {
             // 16 elements (32 bytes) further along K inside the swizzled row: +2 in the address field
@@ -333,7 +343,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           }
           if (p.two_m) {
             // the second 128 rows of A against the same weights, into the other accumulator buffer
-            const uint64_t a2_desc = ptx::umma_desc_k128(ptx::smem_u32(smem_a + s * A_STAGE + A_STAGE_BYTES));
+            const uint64_t a2_desc = a_desc + (static_cast<uint32_t>(A_STAGE_BYTES) >> 4);
 #pragma unroll
             for (int k = 0; k < BLOCK_K / 16; ++k)
               ptx::umma_bf16(d_tmem + ACC_STRIDE, a2_desc + 2 * k, b_desc + 2 * k, idesc, (kbl | k) != 0 ? 1u : 0u);
