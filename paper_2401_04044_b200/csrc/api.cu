@@ -466,6 +466,7 @@ ffsplit_status ffsplit_create(ffsplit_ctx** out, int device) {
   c->cc_minor = minor;
   c->num_sms = sms;
   if (const char* env = std::getenv("FFSPLIT_GEMM_TWO_M")) c->gemm_two_m = env[0] == '0' ? 0 : env[0] == '2' ? 2 : 1;
+  if (const char* env = std::getenv("FFSPLIT_GEMM_ARES")) c->gemm_ares = env[0] == '0' ? 0 : 1;
   if (const char* env = std::getenv("FFSPLIT_GEMM_PANEL")) c->gemm_panel = std::atoi(env);
   if (const char* env = std::getenv("FFSPLIT_GEMM_SPLIT_K")) c->gemm_split_k = env[0] == '0' ? 0 : 1;
   if (const char* env = std::getenv("FFSPLIT_FEW_TENSOR_MIN")) c->few_tensor_min = std::atoi(env);

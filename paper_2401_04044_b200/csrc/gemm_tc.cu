@@ -660,8 +660,12 @@ static ffsplit_status launch_gemm_few(ffsplit_ctx* ctx, const GemmArgs& g, cudaS
   return check_cuda(ctx, le, "few_finish_kernel launch");
 }
 
+bool gemm_ares_applies(const GemmArgs& g);
+ffsplit_status launch_gemm_ares(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_t st);
+
 ffsplit_status launch_gemm_tc(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_t st) {
   if (g.few && g.force_split == 0 && g.M <= 64 && !g.epi.col_partial && !g.epi.c0_f32) return launch_gemm_few(ctx, g, st);
+  if (ctx->gemm_ares && gemm_ares_applies(g)) return launch_gemm_ares(ctx, g, st);
   const bool dual = g.A1 != nullptr;
   if (g.M <= 0 || g.N <= 0 || g.K <= 0) return FFSPLIT_OK;
   tc::Params p;

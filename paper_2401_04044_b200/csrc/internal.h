@@ -30,7 +30,7 @@ constexpr size_t kCtrlBytes = 65536;
 constexpr long long kMaxTicketTiles = (kCtrlBytes - kStatusBytes) / 4;
 
 enum KernelId : int {
-  KID_SELECT = 1, KID_PACK = 2, KID_GEMM_TC = 3, KID_GEMM_SIMT = 4, KID_SCORE = 5, KID_DECODE = 6, KID_FUSED = 7, KID_PROBE = 8, KID_QUANT = 9, KID_FACTOR = 10, KID_ENCODER = 11
+  KID_SELECT = 1, KID_PACK = 2, KID_GEMM_TC = 3, KID_GEMM_SIMT = 4, KID_SCORE = 5, KID_DECODE = 6, KID_FUSED = 7, KID_PROBE = 8, KID_QUANT = 9, KID_FACTOR = 10, KID_ENCODER = 11, KID_GEMM_AR = 12
 };
 
 __device__ __forceinline__ void record_status(int* status, int code, int detail, int kid) {
@@ -206,6 +206,7 @@ struct ffsplit_ctx {
   bool prep_active = false;
   bool attr_tc_set = false;
   bool attr_fused_set = false;
+  bool attr_ares_set = false;
   bool attr_layer_set = false;
   bool attr_att_set = false;
   int* status() const { return reinterpret_cast<int*>(ws); }
@@ -215,6 +216,7 @@ struct ffsplit_ctx {
                                // tensor-core path with exchanged operands, the others the weight-streaming kernels
                                // (FFSPLIT_FEW_TENSOR_MIN; -1 = always the tensor path, 64 = never).  Unset: chosen per
                                // layer from its size and activation, see decode_path_applies()
+  int gemm_ares = 1;           // short contractions (K <= 512) with the row operand resident in tensor memory (FFSPLIT_GEMM_ARES=0: never)
   int gemm_split_k = 1;        // tensor-core GEMM: cut thin products with a long contraction along K (FFSPLIT_GEMM_SPLIT_K=0: never)
   int gemm_panel = 0;          // tensor-core GEMM: tile rows per panel of the tile walk (0: chosen per launch; FFSPLIT_GEMM_PANEL)
   int decode_one_launch = 0;   // few-token forward: 1 = all products in one cooperative launch (FFSPLIT_DECODE_LAYER=1), 0 = one launch per product

@@ -462,6 +462,31 @@ def test_light_chain_second_product_cut_along_k(ctx, monkeypatch, act, d, m, k, 
     assert orc.rel_frobenius(f64(Y2), f64(Y)) < 5e-3
 
 
+@pytest.mark.parametrize("act,d,m,k,r,T", [("gelu_erf", 512, 4200, 48, 320, 700),     # K = 320: five k-blocks, a half-filled ring stage; ragged M and N
+                                          ("gelu_tanh", 384, 2400, 30, 136, 1300),   # K = 144 after padding, three CTAs change their row block
+                                          ("gelu_erf", 512, 6000, 100, 512, 520)])   # the largest K the resident operand takes
+def test_light_chain_first_product_with_resident_rows(ctx, monkeypatch, act, d, m, k, r, T):
+    """H_L = sigma(Q B1 + b) has a short contraction (r): its GEMM keeps the 128 x r block of Q in tensor memory while
+    it walks along the light neurons.  Against the oracle, and bit for bit against the general tensor-core GEMM
+    (the same products and sums in the same order, the same epilogue arithmetic)."""
+    cfg = custom_config(d, m, k, r, act=act, dtype="bf16")
+    L = make_layer(cfg, 6)
+    G = GpuLayer(ctx, L)
+    G.reserve(T, 0, k, r)
+    fac = oracle_factors(L, L.planted.numpy(), r)
+    blob, _ = G.pack(L.planted, fac)
+    X = L.tokens(T)
+    Yref = oracle_split(L, L.planted.numpy(), fac, X)
+    monkeypatch.setenv("FFSPLIT_NO_FUSED", "1")          # the four-GEMM chain
+    monkeypatch.setenv("FFSPLIT_LAYER_KERNEL", "0")
+    Y = forward_on_fresh_context(G, blob, X, T, k, r)
+    assert_close(Y, Yref, "bf16", "light chain, rows of Q resident in tensor memory")
+    monkeypatch.setenv("FFSPLIT_GEMM_ARES", "0")
+    Y2 = forward_on_fresh_context(G, blob, X, T, k, r)
+    assert_close(Y2, Yref, "bf16", "light chain, general GEMM")
+    assert torch.equal(Y, Y2)
+
+
 @pytest.mark.parametrize("dt,act,d,m,T", [("bf16", "gelu_erf", 256, 1000, 300), ("bf16", "swiglu", 192, 520, 5),
                                          ("f32", "gelu_erf", 64, 192, 70), ("bf16", "gelu_tanh", 128, 384, 40)])
 def test_forward_dense_entry_point(ctx, dt, act, d, m, T):
