@@ -171,24 +171,25 @@ static ffsplit_status stream_forward(ffsplit_ctx* ctx, const BlobHeader& h, cons
 // Up to 64 tokens of a bf16 layer: true = the weight-streaming kernels of this file, false = the forward runs its
 // stage GEMMs on the tensor cores with the operands exchanged (GemmArgs::few).
 bool decode_path_applies(const ffsplit_ctx* ctx, const BlobHeader& h, long long T) {
-  // Measured per layer (graph replays over distinct weight copies), tensor path vs streaming kernels:
-  //   layers of tens of megabytes, GELU: ahead at every token count -- OPT-13B shape, 5 % heavy, r = 512: split
-  //     38 vs 42 us at 1 token, 38 vs 44 at 4, 39 vs 57 at 9, 56 vs 151 at 64; dense 83 vs 90 at 1 token, 85 vs 91 at
-  //     16, 102 vs 187 at 64 -- except the dense layer at 2 to 4 tokens (83 vs 80 us);
-  //   gated (SwiGLU) layers: the streaming kernels are ahead up to 8 tokens (Llama-2-7B shape, 1 token: 48 vs 54 us
-  //     split, 54 vs 62 dense), the tensor path from 9 on (61 vs 68 us);
-  //   smaller layers: the streaming kernels up to about 24 tokens on a split layer of a few megabytes (GPT-2-medium
-  //     shape, 16 tokens: 27 vs 29 us; 64 tokens: 67 vs 30 us), up to about 8 on its dense layer of 17 MB (1 token:
-  //     11 vs 15 us; 16 tokens: 19 vs 15.5 us).
+  // Measured per layer (graph replays over distinct weight copies), tensor path vs streaming kernels, split / dense:
+  //   OPT-13B shape (5 % heavy, r = 512; 71 / 419 MB): the tensor path at every token count -- 33 vs 42 us at 1 token,
+  //     34 vs 44 at 4, 35 vs 57 at 16, 46 vs 151 at 64; dense 81 vs 90 at 1 token, 83 vs 91 at 16, 99 vs 187 at 64 --
+  //     except the dense layer at 2 to 4 tokens (83 vs 80 us); the same shape at 1 % heavy, r = 256 (15 MB): 27.5 vs
+  //     34 us at 1 token, 29.5 vs 50 at 16;
+  //   gated (SwiGLU) layers, Llama-2-7B shape: the streaming kernels up to 8 tokens (1 token: 48 vs 54 us split, 53 vs
+  //     62 dense), the tensor path from 9 on (52.5 vs 61 us);
+  //   layers of a few megabytes, and dense ones under 32 MB: the streaming kernels up to 8 tokens (GPT-2-medium shape,
+  //     6 / 17 MB, 1 token: 17.6 vs 20.4 us split, 11 vs 15 dense; BERT-base shape 16.9 vs 19.0 us), the tensor path
+  //     from 9 on (16 tokens: 21.6 vs 26.5 us, 19.9 vs 25.6 us).
   // FFSPLIT_FEW_TENSOR_MIN = t replaces all of this by "streaming kernels up to t tokens": 64 keeps every count on
   // them, -1 sends every count to the tensor path.
   if (h.dtype != FFSPLIT_BF16 || T < 1 || T > 64) return false;
   if (ctx->few_tensor_min != kFewTensorAuto) return T <= ctx->few_tensor_min;
   const double layer_bytes = 2.0 * (h.n_in + 1) * (static_cast<double>(h.d) * h.k + static_cast<double>(h.r) * (h.d + h.ml));
   const bool no_light = h.r == 0 || h.ml == 0;
-  if (layer_bytes < 32e6) return T <= (no_light ? 8 : 24);
   if (h.act == FFSPLIT_SWIGLU) return T <= 8;
-  return no_light && T >= 2 && T <= 4;
+  if (no_light) return layer_bytes < 32e6 ? T <= 8 : (T >= 2 && T <= 4);
+  return layer_bytes < 10e6 && T <= 8;
 }
 
 // fp32 partials of one product.

@@ -61,6 +61,8 @@ struct Params {
   int early;         // 1: the row operand (A) does not depend on the kernel before this one in the stream (packed weights
                      // in the few-token path): its first stages are loaded before the programmatic-launch wait, under
                      // the tail of that kernel; the other operand and every global write come after the wait
+  int trans_tokens;  // > 0: exchanged operands (rows = output columns n, tile columns = tokens), K not cut: the epilogue
+                     // applies bias (per row) and activation and stores the transpose, out[t][n], for t < trans_tokens
   Epilogue epi;
   int* status;
 };
@@ -127,6 +129,26 @@ __device__ __forceinline__ void epilogue_chunk_store(const Params& p, const Gelu
 #pragma unroll
     for (int i = 0; i < 16; ++i)
       if (n0 + i < limit) base[i] = __float2bfloat16_rn(v[i]);
+  }
+}
+
+// Exchanged operands, whole K in one unit: v holds row n (one output column) at tokens t0 .. t0 + 15.  Bias per row,
+// activation, and the transposed store: for one token the lanes of a warp write 32 consecutive outputs.
+__device__ __forceinline__ void epilogue_chunk_transposed(const Params& p, const GeluCoef& gc, long long n, int t0, float* v) {
+  const Epilogue& e = p.epi;
+  if (n >= p.M) return;
+  const float bias = n < e.n_bias ? __ldg(e.bias + n) : 0.f;
+  const bool act = n < e.n_act;
+  const bool first = n < e.n_split;
+  __nv_bfloat16* base = first ? reinterpret_cast<__nv_bfloat16*>(e.C0) + n : reinterpret_cast<__nv_bfloat16*>(e.C1) + (n - e.n_split);
+  const long long ld = first ? e.ld0 : e.ld1;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) {
+    if (t0 + i < p.trans_tokens) {
+      float x = v[i] + bias;
+      if (act) x = gelu_fast(x, gc);
+      base[static_cast<long long>(t0 + i) * ld] = __float2bfloat16_rn(x);
+    }
   }
 }
 
@@ -392,7 +414,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       const uint32_t t_row = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + acc * ACC_STRIDE;
       // one 16-column chunk: v holds the accumulators of this lane's row
       auto finish_chunk = [&](float* v, int n0) {
-        if (p.epi.col_partial == nullptr) {
+        if (p.trans_tokens > 0) {
+          epilogue_chunk_transposed(p, gc, row, n0, v);
+        } else if (p.epi.col_partial == nullptr) {
           epilogue_chunk_store(p, gc, row, n0, v, ks);
         } else {
           const Epilogue& e = p.epi;
@@ -632,11 +656,29 @@ static ffsplit_status launch_gemm_few(ffsplit_ctx* ctx, const GemmArgs& g, cudaS
     const long long units = tiles * s;
     const long long waves = (units + ctx->num_sms - 1) / ctx->num_sms;
     const double eff = static_cast<double>(units) / static_cast<double>(waves * ctx->num_sms);
-    const double cost = weight_bytes / eff + 2.0 * s * n_out * tp * 4;
+    double cost = weight_bytes / eff + 2.0 * s * n_out * tp * 4;
+    // an uncut product finishes its own output (below): no finishing kernel, no launch boundary -- about 3 us, the time
+    // in which 16 MB stream from HBM
+    if (s == 1 && !gated) cost -= 16e6;
     if (cost < best_cost) { best_cost = cost; best = s; }
   }
   if (static_cast<size_t>(nmat) * best * n_out * tp * 4 > g.few_bytes)
     return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL, "workspace too small for the few-token tensor path");
+  if (best == 1 && !gated) {
+    // K in one piece (the light chain's first product: a contraction of r): nothing to add up, so the product's own
+    // epilogue finishes the output and the finishing kernel, with its launch boundary, drops out
+    GemmArgs h;
+    std::memset(&h, 0, sizeof(h));
+    h.A0 = g.B0; h.lda0 = g.ldb0;
+    h.B0 = g.A0; h.ldb0 = g.lda0;
+    h.M = n_out; h.N = tp; h.K = g.K;
+    h.algo_flops = g.algo_flops;
+    h.epi = g.epi;
+    h.force_split = 1;
+    h.trans_tokens = T;
+    h.early_rows = g.weights_stable;
+    return launch_gemm_tc(ctx, h, st);
+  }
   float* part[2] = {static_cast<float*>(g.few), static_cast<float*>(g.few) + static_cast<size_t>(best) * n_out * tp};
   for (int i = 0; i < nmat; ++i) {
     GemmArgs h;
@@ -748,7 +790,10 @@ ffsplit_status launch_gemm_tc(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_t 
   p.gate_off = p.shared_a ? p.block_n : tc::GATE_OFFSET;
   p.early = (g.early_rows && !dual) ? 1 : 0;
   p.epi = g.epi;
-  if (g.force_split >= 1) {
+  p.trans_tokens = 0;
+  if (g.force_split == 1 && g.trans_tokens > 0) {
+    p.trans_tokens = g.trans_tokens;   // the caller's epilogue, applied by the one unit of each row tile
+  } else if (g.force_split >= 1) {
     p.epi.c0_f32 = 1;         // the caller's C0 is the fp32 partial buffer [split][M][N] already
   } else if (p.split_k > 1) {
     p.epi.C0 = g.splitk;      // fp32 partials [split][M][N]

@@ -111,6 +111,8 @@ struct GemmArgs {
   // small kernel that adds the fp32 partials, applies this epilogue and stores the transpose.  Needs scratch.
   void* few; size_t few_bytes;
   int force_split;    // internal: K ranges of the exchanged product (set by the few-token path)
+  int trans_tokens;   // internal: > 0 with force_split == 1: the exchanged product finishes its own output -- bias, activation
+                      // and the transposed bf16 store of this many token rows -- instead of leaving an fp32 partial
   int weights_stable; // the weights (B0 / B1) are not written by the kernel before this launch in the stream (set for every
                       // product of a forward but its first): the few-token path then loads them under that kernel's tail
   int early_rows;     // internal: the row operand A0 may be loaded before the programmatic-launch wait
