@@ -466,7 +466,7 @@ def run_ours(args):
     n_b, ms_b, fl_b = ctx.profile_end(0)
     n_l, ms_l, flops_l = n_a + n_b, ms_a + ms_b, fl_a + fl_b
     achieved = flops_l / (ms_l * 1e-3) / 1e12 if ms_l > 0 else 0.0
-    roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel", "achieved": round(achieved, 2),
+    roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel (160 launches per step; the light chain's first product, 40 launches, is its short-K form gemm_ares_kernel)", "achieved": round(achieved, 2),
                 "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
                 "frac": round(achieved / peaks["bf16_tflops_sustained"], 4),
                 "frac_of_burst_peak": round(achieved / peaks["bf16_tflops"], 4),
@@ -475,11 +475,11 @@ def run_ours(args):
                 "algorithmic_flops_per_launch": flops_l / max(n_l, 1), "traffic": None}
     if n_layers == 40 and n_l == 200:
         # DRAM bytes (read + written) of the average launch of a step, from ncu captures of the current kernel:
-        # the scoring product at 8192 calibration tokens moved 800.8 MB (scaled by 8 to the 65 536 tokens of a
+        # the scoring product at 8192 calibration tokens moved 834.7 MB (scaled by 8 to the 65 536 tokens of a
         # launch here: the weights are re-read once per panel of 12 tile rows, so traffic grows with the tokens) and
         # the four forward GEMMs of a layer at 4096 tokens (the partial-sum kernel of the one cut along K included)
-        # 431.0 MB together; 40 + 160 launches per step.
-        roofline["traffic"] = round((40 * 8 * 800.8e6 + 40 * 431.0e6) / 200)
+        # 419.0 MB together; 40 + 160 launches per step.
+        roofline["traffic"] = round((40 * 8 * 834.7e6 + 40 * 419.0e6) / 200)
         roofline["traffic_source"] = ("profiles/gemm_tc_kernel__cfg5_scoring.md (x 8 tokens), "
                                       "profiles/gemm_tc_kernel__cfg5_prefill.md")
         roofline["algorithmic_bytes_per_launch"] = round((40 * (es_b * (cfg.t_cal * cfg.d + cfg.d * cfg.m)) + 40 * (wl.logical_bytes + 2 * es_b * T * cfg.d)) / 200)
