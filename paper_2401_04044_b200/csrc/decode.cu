@@ -176,9 +176,10 @@ bool decode_path_applies(const ffsplit_ctx* ctx, const BlobHeader& h, long long 
   //     34 vs 44 at 4, 35 vs 57 at 16, 46 vs 151 at 64; dense 81 vs 90 at 1 token, 83 vs 91 at 16, 99 vs 187 at 64 --
   //     except the dense layer at 2 to 4 tokens (83 vs 80 us); the same shape at 1 % heavy, r = 256 (15 MB): 27.5 vs
   //     34 us at 1 token, 29.5 vs 50 at 16;
-  //   gated (SwiGLU) layers, Llama-2-7B shape: the streaming kernels up to 8 tokens (1 token: 48 vs 54 us split, 53 vs
-  //     62 dense), the tensor path from 9 on (52.5 vs 61 us);
-  //   layers of a few megabytes, and dense ones under 32 MB: the streaming kernels up to 8 tokens (GPT-2-medium shape,
+  //   gated (SwiGLU) layers, Llama-2-7B shape: the streaming kernels at one token (48.5 vs 49.4 us split, 53 vs 60.5
+  //     dense), the tensor path above (split 50.4 vs 53.5 us at 4 tokens, 50.5 vs 53 at 8, 51 vs 61 at 9; dense 60 vs
+  //     66 at 4, 60 vs 64.6 at 8);
+  //   split layers under 10 MB and dense ones under 32 MB: the streaming kernels up to 8 tokens (GPT-2-medium shape,
   //     6 / 17 MB, 1 token: 17.6 vs 20.4 us split, 11 vs 15 dense; BERT-base shape 16.9 vs 19.0 us), the tensor path
   //     from 9 on (16 tokens: 21.6 vs 26.5 us, 19.9 vs 25.6 us).
   // FFSPLIT_FEW_TENSOR_MIN = t replaces all of this by "streaming kernels up to t tokens": 64 keeps every count on
@@ -187,9 +188,9 @@ bool decode_path_applies(const ffsplit_ctx* ctx, const BlobHeader& h, long long 
   if (ctx->few_tensor_min != kFewTensorAuto) return T <= ctx->few_tensor_min;
   const double layer_bytes = 2.0 * (h.n_in + 1) * (static_cast<double>(h.d) * h.k + static_cast<double>(h.r) * (h.d + h.ml));
   const bool no_light = h.r == 0 || h.ml == 0;
-  if (h.act == FFSPLIT_SWIGLU) return T <= 8;
-  if (no_light) return layer_bytes < 32e6 ? T <= 8 : (T >= 2 && T <= 4);
-  return layer_bytes < 10e6 && T <= 8;
+  if (no_light ? layer_bytes < 32e6 : layer_bytes < 10e6) return T <= 8;
+  if (h.act == FFSPLIT_SWIGLU) return no_light ? T <= 2 : T == 1;
+  return no_light && T >= 2 && T <= 4;
 }
 
 // fp32 partials of one product.

@@ -138,7 +138,7 @@ __device__ __forceinline__ void epilogue_chunk_transposed(const Params& p, const
   const Epilogue& e = p.epi;
   if (n >= p.M) return;
   const float bias = n < e.n_bias ? __ldg(e.bias + n) : 0.f;
-  const bool act = n < e.n_act;
+  const bool act = !p.dual && n < e.n_act;   // (a gated pair arrives here as SiLU(gate) * up already)
   const bool first = n < e.n_split;
   __nv_bfloat16* base = first ? reinterpret_cast<__nv_bfloat16*>(e.C0) + n : reinterpret_cast<__nv_bfloat16*>(e.C1) + (n - e.n_split);
   const long long ld = first ? e.ld0 : e.ld1;
@@ -649,6 +649,7 @@ static ffsplit_status launch_gemm_few(ffsplit_ctx* ctx, const GemmArgs& g, cudaS
   int best = 1;
   double best_cost = 1e300;
   const double weight_bytes = 2.0 * n_out * g.K;
+  const bool direct_ok = !gated || g.epi.n_bias == 0;   // (the gated epilogue in the kernel adds a bias after the gating)
   for (int s = 1; s <= 16; ++s) {
     if (s > 1 && nkb / s < 4) break;
     if (nkb - (s - 1) * ((nkb + s - 1) / s) <= 0) continue;   // the last range must not be empty
@@ -659,18 +660,23 @@ static ffsplit_status launch_gemm_few(ffsplit_ctx* ctx, const GemmArgs& g, cudaS
     double cost = weight_bytes / eff + 2.0 * s * n_out * tp * 4;
     // an uncut product finishes its own output (below): no finishing kernel, no launch boundary -- about 3 us, the time
     // in which 16 MB stream from HBM
-    if (s == 1 && !gated) cost -= 16e6;
+    if (s == 1 && direct_ok) cost -= 16e6 * nmat;
     if (cost < best_cost) { best_cost = cost; best = s; }
   }
   if (static_cast<size_t>(nmat) * best * n_out * tp * 4 > g.few_bytes)
     return fail(ctx, FFSPLIT_ERR_BUFFER_TOO_SMALL, "workspace too small for the few-token tensor path");
-  if (best == 1 && !gated) {
+  if (best == 1 && direct_ok) {
     // K in one piece (the light chain's first product: a contraction of r): nothing to add up, so the product's own
-    // epilogue finishes the output and the finishing kernel, with its launch boundary, drops out
+    // epilogue finishes the output and the finishing kernel, with its launch boundary, drops out; a gated pair runs
+    // as one launch with two accumulators
     GemmArgs h;
     std::memset(&h, 0, sizeof(h));
     h.A0 = g.B0; h.lda0 = g.ldb0;
     h.B0 = g.A0; h.ldb0 = g.lda0;
+    if (gated) {
+      h.A1 = g.B1; h.lda1 = g.ldb1;
+      h.B1 = g.A1; h.ldb1 = g.lda1;
+    }
     h.M = n_out; h.N = tp; h.K = g.K;
     h.algo_flops = g.algo_flops;
     h.epi = g.epi;

@@ -371,8 +371,8 @@ def test_decode_forward_matches_oracle(ctx, act, d, m, k, r, T):
 @pytest.mark.parametrize("T", [1, 5, 13, 16, 33, 64])
 def test_few_token_paths_agree(ctx, monkeypatch, act, d, m, k, r, T):
     """Up to 64 tokens there are two paths: the weight-streaming kernels and the stage GEMMs on the tensor cores with the
-    operands exchanged (by default: at every count on GELU layers of tens of megabytes, from 9 tokens on gated layers
-    and on layers of a few megabytes).
+    operands exchanged (by default: at every count on GELU layers of tens of megabytes, from 2 tokens on gated ones,
+    from 9 on layers of a few megabytes).
     FFSPLIT_FEW_TENSOR_MIN = -1 / 64 forces either for every token count.  Both against the oracle, split and dense,
     and against each other."""
     cfg = custom_config(d, m, k, r, act=act, dtype="bf16")
