@@ -478,8 +478,8 @@ def run_ours(args):
         # the scoring product at 8192 calibration tokens moved 840.3 MB (scaled by 8 to the 65 536 tokens of a
         # launch here: the weights are re-read once per panel of 12 tile rows, so traffic grows with the tokens) and
         # the four forward GEMMs of a layer at 4096 tokens (the partial-sum kernel of the one cut along K included)
-        # 428.6 MB together; 40 + 160 launches per step.
-        roofline["traffic"] = round((40 * 8 * 840.3e6 + 40 * 428.6e6) / 200)
+        # 424.8 MB together; 40 + 160 launches per step.
+        roofline["traffic"] = round((40 * 8 * 840.3e6 + 40 * 424.8e6) / 200)
         roofline["traffic_source"] = ("profiles/gemm_tc_kernel__cfg5_scoring.md (x 8 tokens), "
                                       "profiles/gemm_tc_kernel__cfg5_prefill.md")
         roofline["algorithmic_bytes_per_launch"] = round((40 * (es_b * (cfg.t_cal * cfg.d + cfg.d * cfg.m)) + 40 * (wl.logical_bytes + 2 * es_b * T * cfg.d)) / 200)

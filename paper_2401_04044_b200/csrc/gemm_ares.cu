@@ -15,15 +15,17 @@
 // eight warps, one per accumulator buffer (even and odd tiles), each warp 32 rows x 64 columns -- the epilogue
 // warps also copy A: each thread reads its own row from global memory and stores it into the quarter's lanes.
 //
-// The output leaves in whole 128-byte lines: a lane holds one row (that is how tensor memory is read), so each
-// warp turns its 32 x 64 block through 4 KB of shared memory of its own (128-byte swizzle, no bank conflicts
-// either way, no barrier beyond the warp's own) and eight lanes write one row's 128 bytes.
+// The output leaves through TMA stores: a lane holds one row (that is how tensor memory is read), so each warp
+// writes its 32 x 64 block into 4 KB of shared memory of its own, in the 128-byte swizzle the output's tensor map
+// expects (no bank conflicts, no barrier beyond the warp's own), and one lane stores the block with one
+// cp.async.bulk.tensor; it waits for that store to have read the buffer only when the warp next writes it, two
+// tiles later.
 //
-// What bounds this product is its output.  Measured on the shape above (single launches): the general GEMM
-// 98.4 us, this kernel 96.8 us, either of them without its stores (a working copy) about 47 us -- and a plain
-// fill of the same 159 MB takes 47 us (3.4 TB/s).  Neither the operand in tensor memory nor the full-line
-// stores changed that sum; in the layer the kernel is 1 to 3 % ahead of the general GEMM on the three rank-512
-// points of the OPT-13B-shaped sweep (interleaved runs), and bit-identical to it.
+// What bounds this product is its output.  Measured on the shape above (single launches): the general GEMM, 32
+// bytes per lane straight from the registers, 98.4 us; the same block turned through the warp's buffer and
+// written as whole 128-byte lines by ordinary stores 95.6 us; through TMA stores 81.4-83.1 us (tensor pipe 51 ->
+// 61 % active); either of the first two without its stores (a working copy) about 47 us -- a plain fill of the
+// same 159 MB takes 47 us (3.4 TB/s).  Bit-identical to the general GEMM.
 // Every wait is bounded (see gemm_tc.cu).
 #include "epilogue.cuh"
 #include "internal.h"
@@ -95,7 +97,7 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r) {
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 __global__ void __launch_bounds__(NUM_THREADS, 1)
-gemm_ares_kernel(const __grid_constant__ CUtensorMap tmB, const Params p) {
+gemm_ares_kernel(const __grid_constant__ CUtensorMap tmB, const __grid_constant__ CUtensorMap tmC, const Params p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* smem_turn = smem + MAX_STAGES * STAGE_BYTES;
@@ -260,7 +262,10 @@ gemm_ares_kernel(const __grid_constant__ CUtensorMap tmB, const Params p) {
         ptx::tc_fence_after();
         const uint32_t t_acc = t_lane + TMEM_ACC0 + acc * BLOCK_N + ch * 64;
         const int n0 = n_blk * BLOCK_N + ch * 64;
-        // ---- this lane's row, 64 columns: bias, activation, bf16, into the warp's turning buffer
+        // ---- this lane's row, 64 columns: bias, activation, bf16, into the warp's turning buffer (once the store of
+        // the warp's tile before has read it: two tiles ago, so this wait does not wait)
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+        __syncwarp();
 #pragma unroll
         for (int pr = 0; pr < 2; ++pr) {
           float va[16], vb[16];
@@ -297,24 +302,21 @@ gemm_ares_kernel(const __grid_constant__ CUtensorMap tmB, const Params p) {
                 make_uint4(pack_bf16x2(v[8], v[9]), pack_bf16x2(v[10], v[11]), pack_bf16x2(v[12], v[13]), pack_bf16x2(v[14], v[15]));
           }
         }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
-        // ---- out: eight lanes per row, four rows per instruction
-        const int pc = lane & 7;
-        const int nn = n0 + pc * 8;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const int r = 4 * i + (lane >> 3);
-          const long long row = m_blk * BLOCK_M + q * 32 + r;
-          const uint4 o = *reinterpret_cast<const uint4*>(turn + r * 128 + ((pc ^ (r & 7)) << 4));
-          if (row < p.M && nn < p.N)     // N is a multiple of 8: a piece is inside or outside
-            *reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(e.C0) + row * e.ld0 + nn) = o;
+        // ---- out: one TMA store of the warp's 32 x 64 block (rows past M and columns past N are clipped)
+        if (lane == 0) {
+          asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];" ::"l"(&tmC),
+                       "r"(ptx::smem_u32(turn)), "r"(n0), "r"(static_cast<int>(m_blk * BLOCK_M + q * 32))
+                       : "memory");
+          asm volatile("cp.async.bulk.commit_group;" ::: "memory");
         }
-        __syncwarp();   // the buffer is read: the next tile of this warp may write it
       }
       if (++n_blk == p.tiles_n) { n_blk = 0; ++m_blk; }
     }
   }
 
+  if (warp >= 2 && lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   ptx::tc_fence_before();
   __syncthreads();
   if (threadIdx.x == 0 && *abort_flag) record_status(p.status, FFSPLIT_ERR_TIMEOUT, blockIdx.x, KID_GEMM_AR);
@@ -347,9 +349,10 @@ ffsplit_status launch_gemm_ares(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_
   p.lda = g.lda0;
   p.epi = g.epi;
   p.status = ctx->status();
-  CUtensorMap tB;
+  CUtensorMap tB, tC;
   ffsplit_status s;
   if ((s = get_tmap_bf16(ctx, g.B0, g.N, g.K, g.ldb0, ar::BLOCK_N, &tB)) != FFSPLIT_OK) return s;
+  if ((s = get_tmap_bf16(ctx, g.epi.C0, g.M, g.N, g.epi.ld0, 32, &tC)) != FFSPLIT_OK) return s;
   if (!ctx->attr_ares_set) {
     cudaError_t e = cudaFuncSetAttribute(ar::gemm_ares_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ar::SMEM_BYTES);
     if (e != cudaSuccess) return check_cuda(ctx, e, "cudaFuncSetAttribute(gemm_ares_kernel)");
@@ -357,7 +360,7 @@ ffsplit_status launch_gemm_ares(ffsplit_ctx* ctx, const GemmArgs& g, cudaStream_
   }
   const int grid = static_cast<int>(p.tiles < ctx->num_sms ? p.tiles : ctx->num_sms);
   const int ph = prof_open(ctx, PROF_GEMM_TC, g.algo_flops, st);
-  const cudaError_t le = launch_pdl(ar::gemm_ares_kernel, dim3(grid), dim3(ar::NUM_THREADS), ar::SMEM_BYTES, st, tB, p);
+  const cudaError_t le = launch_pdl(ar::gemm_ares_kernel, dim3(grid), dim3(ar::NUM_THREADS), ar::SMEM_BYTES, st, tB, tC, p);
   prof_close(ctx, ph, st);
   ctx->launches++;
   return check_cuda(ctx, le, "gemm_ares_kernel launch");
